@@ -1,0 +1,236 @@
+"""Standardised sampling, speculative sampling and the accept/adjust/draw part
+of Algorithm 1, in fp64, one element at a time where order matters.
+
+Test infrastructure (see the package docstring).
+
+What follows the paper, and where it is silent:
+
+* Section 2.2: every sampling method is a draw from an adjusted distribution.
+  Temperature T > 0 gives softmax(logits / T); T = 0 (argmax) zeroes every
+  non-maximal entry and normalises.  Reading for ties: the lowest index keeps
+  all the mass, so the adjusted distribution is always one-hot at T = 0.
+* Section 2.3 / Algorithm 1: a drafted token x_i ~ q_i is rejected iff
+  r_i > p_i(x_i) / q_i(x_i).  The bare `x` printed in the algorithm's test is
+  the drafted token x_i.  The test is evaluated without a division, as
+  r_i * q_i(x_i) > p_i(x_i), which is the same predicate for q_i(x_i) > 0 and
+  never rejects when q_i(x_i) = 0 (a token the draft could not have drawn).
+* n = number of drafted tokens before the first rejection (gamma if none).
+  p' = p_{n+1}; if n < gamma, p' = norm(max(0, p_{n+1} - q_{n+1})).
+  Appendix A.1: the normaliser equals 1 - beta with beta = sum min(p, q).
+  Reading for a vanishing normaliser (unreachable in exact arithmetic after a
+  genuine rejection): draw from p_{n+1} unmodified and report it.
+* How a categorical draw is made is not stated.  Reading: inverse CDF in index
+  order on unnormalised weights w: the smallest k with w_0 + ... + w_k > u * W,
+  W the total; if rounding leaves none, the last k with w_k > 0.
+
+Pins (tests/test_oracle_sampling.py): emitted-token law equals p over 10^6
+seeded trials (Appendix A.1); acceptance frequency equals sum min(p, q)
+(Theorem 3.5); rejected-branch law equals max(0, p - q) / (1 - beta);
+p = q always accepts, disjoint supports never accept (Corollary 3.4); exact
+measures of every outcome on an (r, u) grid for vocabularies <= 8; gamma = 0
+reduces to a textbook inverse-CDF draw from p; T = 0 reduces to greedy.
+"""
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+
+def standardise(logits, temperature):
+    """Section 2.2: logits -> the adjusted distribution that is sampled from.
+
+    T > 0: softmax(logits / T) with the maximum subtracted first.
+    T = 0: one-hot at the maximum (lowest index on ties).
+    """
+    z = np.asarray(logits, dtype=np.float64)
+    if temperature == 0:
+        out = np.zeros_like(z)
+        out[int(np.argmax(z))] = 1.0  # numpy's argmax returns the first maximum
+        return out
+    z = z / float(temperature)
+    z = z - z.max()
+    e = np.exp(z)
+    return e / e.sum()
+
+
+def inverse_cdf(weights, u):
+    """Draw an index from unnormalised `weights` with the uniform `u`.
+
+    Returns (k, margin): k is the smallest index whose running sum exceeds
+    u * W; margin is the distance from u * W to the nearer of the two running
+    sums that bracket it, divided by W (how close the draw was to picking a
+    neighbour instead).
+    """
+    w = np.asarray(weights, dtype=np.float64)
+    running = np.cumsum(w)  # sequential fp64 accumulation in index order
+    total = running[-1]
+    target = u * total
+    k = int(np.searchsorted(running, target, side="right"))  # first running sum > target
+    if k >= w.shape[0]:
+        positive = np.nonzero(w > 0.0)[0]
+        return (int(positive[-1]) if positive.size else w.shape[0] - 1), 0.0
+    prev = running[k - 1] if k > 0 else 0.0
+    margin = min(target - prev, running[k] - target) / total
+    return k, float(margin)
+
+
+def speculative_sampling(p, q, x, r, u):
+    """Section 2.3 for one token: x was drawn from q; returns (accepted, token).
+
+    Keeps x unless r > p(x) / q(x); otherwise draws from norm(max(0, p - q))
+    with the uniform u.
+    """
+    p = np.asarray(p, dtype=np.float64)
+    q = np.asarray(q, dtype=np.float64)
+    if not (r * q[x] > p[x]):
+        return True, int(x)
+    residual = np.maximum(0.0, p - q)
+    if not residual.sum() > 0.0:
+        residual = p
+    k, _ = inverse_cdf(residual, u)
+    return False, k
+
+
+@dataclass
+class VerifyResult:
+    """Outcome of the accept/adjust/draw part of Algorithm 1 for one sequence."""
+
+    n_accepted: int
+    next_token: int
+    accept_margin: float  # min |r_i - p_i(x_i)/q_i(x_i)| over the tests evaluated
+    cdf_margin: float  # see inverse_cdf
+    top2_gap: float  # smallest gap between the two largest target logits, rows used
+    fallback: bool  # the residual vanished and p_{n+1} was used unmodified
+    betas: list = field(default_factory=list)  # sum min(p_i, q_i), tests evaluated
+
+
+def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature):
+    """Algorithm 1 from "determine the number of accepted guesses" to the end.
+
+    target_logits [gamma+1, V]: row i-1 gives p_i (i = 1..gamma+1).
+    draft_logits  [gamma, V]:   row i-1 gives q_i, from which x_i was drawn.
+    draft_tokens  [gamma]:      x_1..x_gamma.
+    uniforms      [gamma+1]:    r_1..r_gamma, then the uniform for t ~ p'.
+    """
+    tl = np.asarray(target_logits, dtype=np.float64)
+    ql = np.asarray(draft_logits, dtype=np.float64)
+    gamma = tl.shape[0] - 1
+    assert ql.shape[0] == gamma and len(draft_tokens) == gamma
+    assert len(uniforms) == gamma + 1
+
+    p = [standardise(tl[i], temperature) for i in range(gamma + 1)]
+    q = [standardise(ql[i], temperature) for i in range(gamma)]
+
+    accept_margin = float("inf")
+    top2_gap = float("inf")
+    betas = []
+    n = gamma
+    for i in range(gamma):
+        x = int(draft_tokens[i])
+        r = float(uniforms[i])
+        betas.append(float(np.minimum(p[i], q[i]).sum()))
+        top2_gap = min(top2_gap, _top2_gap(tl[i]))
+        if q[i][x] > 0.0:
+            accept_margin = min(accept_margin, abs(r - p[i][x] / q[i][x]))
+        if r * q[i][x] > p[i][x]:
+            n = i
+            break
+
+    adjusted = p[n]
+    fallback = False
+    if n < gamma:
+        adjusted = np.maximum(0.0, p[n] - q[n])
+        if not adjusted.sum() > 0.0:
+            adjusted = p[n]
+            fallback = True
+    else:
+        top2_gap = min(top2_gap, _top2_gap(tl[gamma]))
+    t, cdf_margin = inverse_cdf(adjusted, float(uniforms[gamma]))
+    return VerifyResult(n, t, accept_margin, cdf_margin, top2_gap, fallback, betas)
+
+
+def verify_batch(target_logits, draft_logits, draft_tokens, uniforms, temperature):
+    """`verify_step` for every sequence of a batch: [B, ...] inputs -> list."""
+    return [
+        verify_step(target_logits[b], draft_logits[b], draft_tokens[b], uniforms[b], temperature)
+        for b in range(len(target_logits))
+    ]
+
+
+def sample_token(logits, u, temperature):
+    """A plain draw from the standardised distribution: (token, cdf margin).
+
+    This is how the draft model draws x_i ~ q_i and how target-only decoding
+    draws t ~ p.  The weights are left unnormalised, exp((l - max) / T), which
+    the inverse-CDF rule allows.
+    """
+    z = np.asarray(logits, dtype=np.float64)
+    if temperature == 0:
+        return int(np.argmax(z)), float("inf")
+    w = np.exp((z - z.max()) / float(temperature))
+    return inverse_cdf(w, u)
+
+
+def sample_trials(logits, uniforms, temperature):
+    """`sample_token` for many uniforms that share one row of logits -> [N]."""
+    z = np.asarray(logits, dtype=np.float64)
+    us = np.asarray(uniforms, dtype=np.float64)
+    if temperature == 0:
+        return np.full(us.shape[0], int(np.argmax(z)), dtype=np.int64)
+    w = np.exp((z - z.max()) / float(temperature))
+    running = np.cumsum(w)
+    k = np.searchsorted(running, us * running[-1], side="right")
+    positive = np.nonzero(w > 0.0)[0]
+    return np.where(k >= w.shape[0], positive[-1], k).astype(np.int64)
+
+
+def verify_trials(target_logits, draft_logits, draft_tokens, uniforms, temperature):
+    """Many independent trials of `verify_step` that share one set of logits.
+
+    target_logits [gamma+1, V] and draft_logits [gamma, V] are fixed;
+    draft_tokens [N, gamma] and uniforms [N, gamma+1] vary per trial.  Returns
+    (n_accepted [N], next_token [N]).  Same rules as `verify_step`, evaluated
+    for all trials at once (the statistical pins need 10^6 of them); the tests
+    check it against `verify_step` trial by trial on a subset.
+    """
+    tl = np.asarray(target_logits, dtype=np.float64)
+    ql = np.asarray(draft_logits, dtype=np.float64)
+    xs = np.asarray(draft_tokens)
+    us = np.asarray(uniforms, dtype=np.float64)
+    gamma = tl.shape[0] - 1
+    trials = us.shape[0]
+    p = np.stack([standardise(tl[i], temperature) for i in range(gamma + 1)])
+    q = np.stack([standardise(ql[i], temperature) for i in range(gamma)]) if gamma else np.zeros((0, tl.shape[1]))
+
+    n = np.full(trials, gamma, dtype=np.int64)
+    undecided = np.ones(trials, dtype=bool)
+    for i in range(gamma):
+        x = xs[:, i]
+        rejected = us[:, i] * q[i][x] > p[i][x]
+        first = undecided & rejected
+        n[first] = i
+        undecided &= ~rejected
+
+    tokens = np.empty(trials, dtype=np.int64)
+    for row in range(gamma + 1):
+        sel = np.nonzero(n == row)[0]
+        if sel.size == 0:
+            continue
+        adjusted = p[row]
+        if row < gamma:
+            adjusted = np.maximum(0.0, p[row] - q[row])
+            if not adjusted.sum() > 0.0:
+                adjusted = p[row]
+        running = np.cumsum(adjusted)
+        k = np.searchsorted(running, us[sel, gamma] * running[-1], side="right")
+        positive = np.nonzero(adjusted > 0.0)[0]
+        k = np.where(k >= adjusted.shape[0], positive[-1], k)
+        tokens[sel] = k
+    return n, tokens
+
+
+def _top2_gap(row):
+    if row.shape[0] < 2:
+        return float("inf")
+    top = np.partition(row, -2)[-2:]
+    return float(top[1] - top[0])

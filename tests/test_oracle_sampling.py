@@ -1,0 +1,246 @@
+"""Pins for oracle.sampling: what Appendix A.1, Theorem 3.5 and Corollary 3.4 fix."""
+import numpy as np
+import pytest
+from scipy import stats
+
+from oracle import analysis, philox, sampling
+from paper_2211_17192_b200 import workloads
+
+TRIALS = 1_000_000
+VOCAB = 64
+
+
+def _chi_square_p(counts, probs):
+    """Chi-square goodness of fit; bins with expected count < 5 are merged into one."""
+    expected = probs * counts.sum()
+    small = expected < 5
+    if small.any():
+        counts = np.append(counts[~small], counts[small].sum())
+        expected = np.append(expected[~small], expected[small].sum())
+        if expected[-1] == 0:
+            assert counts[-1] == 0
+            counts, expected = counts[:-1], expected[:-1]
+    return stats.chisquare(counts, expected).pvalue
+
+
+def _fixed_pair(noise, seed=11):
+    t, d = workloads.make_sampler_logits(seed, 1, 1, VOCAB, noise)
+    return t[0].astype(np.float64), d[0].astype(np.float64)  # [2, V], [1, V]
+
+
+@pytest.mark.parametrize("noise", [0.5, 1.0, 2.0])
+def test_emitted_token_follows_p_and_acceptance_equals_sum_min(noise):
+    tl, ql = _fixed_pair(noise)
+    p = sampling.standardise(tl[0], 1.0)
+    q = sampling.standardise(ql[0], 1.0)
+    idx = np.arange(TRIALS)
+    x = sampling.sample_trials(ql[0], philox.uniforms_vec(5, idx, 0, philox.PURPOSE_DRAFT), 1.0)
+    r = philox.uniforms_vec(5, idx, 0, philox.PURPOSE_ACCEPT)
+    u = philox.uniforms_vec(5, idx, 0, philox.PURPOSE_FINAL)
+    n, t = sampling.verify_trials(tl, ql, x[:, None], np.stack([r, u], axis=1), 1.0)
+
+    # the draft's own draws follow q
+    assert _chi_square_p(np.bincount(x, minlength=VOCAB), q) > 1e-3
+    # Appendix A.1: the first emitted token (x if accepted, else t) follows p
+    first = np.where(n == 1, x, t)
+    assert _chi_square_p(np.bincount(first, minlength=VOCAB), p) > 1e-3
+    # Theorem 3.5: acceptance frequency = sum min(p, q)
+    beta = analysis.beta(p, q)
+    assert abs((n == 1).mean() - beta) < 4 * np.sqrt(beta * (1 - beta) / TRIALS)
+    # Appendix A.1: after a rejection the token follows max(0, p - q) / (1 - beta)
+    residual = np.maximum(0, p - q)
+    assert residual.sum() == pytest.approx(1 - beta, abs=1e-12)
+    assert _chi_square_p(np.bincount(t[n == 0], minlength=VOCAB), residual / residual.sum()) > 1e-3
+    # when all guesses are accepted the bonus token follows p_{gamma+1}
+    p2 = sampling.standardise(tl[1], 1.0)
+    assert _chi_square_p(np.bincount(t[n == 1], minlength=VOCAB), p2) > 1e-3
+
+
+def test_tokens_per_iteration_match_eq_1():
+    gamma = 4
+    tl1, ql1 = _fixed_pair(1.0, seed=12)
+    tl = np.repeat(tl1[:1], gamma + 1, axis=0)  # the same p at every position
+    ql = np.repeat(ql1[:1], gamma, axis=0)  # the same q at every position
+    alpha = analysis.beta(sampling.standardise(tl[0], 1.0), sampling.standardise(ql[0], 1.0))
+    trials = 400_000
+    idx = np.arange(trials)
+    xs = np.stack([sampling.sample_trials(ql[0], philox.uniforms_vec(9, idx * gamma + i, 0, 0), 1.0)
+                   for i in range(gamma)], axis=1)
+    us = np.stack([philox.uniforms_vec(9, idx * (gamma + 1) + i, 1, 1) for i in range(gamma + 1)], axis=1)
+    n, _ = sampling.verify_trials(tl, ql, xs, us, 1.0)
+    tokens = n + 1
+    assert tokens.min() >= 1 and tokens.max() <= gamma + 1
+    assert abs(tokens.mean() - analysis.expected_tokens(alpha, gamma)) < 4 * tokens.std() / np.sqrt(trials)
+    # the capped geometric law itself
+    law = np.array([alpha**k * (1 - alpha) for k in range(gamma)] + [alpha**gamma])
+    assert _chi_square_p(np.bincount(n, minlength=gamma + 1), law) > 1e-3
+
+
+def test_vectorised_trials_equal_the_scalar_step():
+    gamma = 3
+    t, d = workloads.make_sampler_logits(21, 1, gamma, VOCAB, 1.0)
+    tl, ql = t[0], d[0]
+    trials = 3000
+    idx = np.arange(trials)
+    xs = np.stack([sampling.sample_trials(ql[i], philox.uniforms_vec(3, idx, i, 0), 1.0) for i in range(gamma)], axis=1)
+    us = np.stack([philox.uniforms_vec(3, idx, i, 1) for i in range(gamma + 1)], axis=1)
+    for temperature in (1.0, 0.7, 0.0):
+        n, tok = sampling.verify_trials(tl, ql, xs, us, temperature)
+        for k in range(trials):
+            res = sampling.verify_step(tl, ql, xs[k], us[k], temperature)
+            assert (res.n_accepted, res.next_token) == (n[k], tok[k])
+
+
+def test_identical_distributions_always_accept():
+    t, _ = workloads.make_sampler_logits(31, 4, 3, 50, 1.0)
+    us = workloads.make_uniform_grid(31, (4, 4))
+    xs = np.array([[sampling.sample_token(t[b, i], 0.3 + 0.1 * i, 1.0)[0] for i in range(3)] for b in range(4)])
+    for b in range(4):
+        res = sampling.verify_step(t[b], t[b, :3], xs[b], us[b], 1.0)
+        assert res.n_accepted == 3
+        assert res.next_token == sampling.sample_token(t[b, 3], us[b, 3], 1.0)[0]
+        assert all(beta == pytest.approx(1.0, abs=1e-12) for beta in res.betas)
+
+
+def test_disjoint_supports_never_accept_and_resample_from_p():
+    V = 10
+    big = 800.0  # exp(-800) underflows to exactly 0 in fp64
+    tl = np.full((2, V), -big)
+    ql = np.full((1, V), -big)
+    tl[:, :5] = np.linspace(0, 1, 5)
+    ql[:, 5:] = np.linspace(0, 1, 5)
+    p = sampling.standardise(tl[0], 1.0)
+    for u in (0.01, 0.37, 0.99):
+        res = sampling.verify_step(tl, ql, [7], [1 / 2**24, u], 1.0)  # smallest possible r still rejects
+        assert res.n_accepted == 0 and res.betas == [0.0]
+        assert res.next_token == sampling.inverse_cdf(p, u)[0] and res.next_token < 5
+
+
+def test_uniform_draft_acceptance():
+    V = 32
+    tl, _ = _fixed_pair(1.0, seed=5)
+    p = sampling.standardise(tl[0, :V], 1.0)
+    res = sampling.verify_step(tl[:, :V], np.zeros((1, V)), [3], [0.5, 0.5], 1.0)
+    assert res.betas[0] == pytest.approx(np.minimum(p, 1.0 / V).sum(), abs=1e-14)
+
+
+def test_gamma_zero_is_a_plain_inverse_cdf_draw():
+    w = np.array([1.0, 2.0, 0.0, 1.0])
+    logits = np.log(np.maximum(w, 1e-300))
+    logits[2] = -1e4
+    # boundaries of the CDF at 0.25, 0.75, 0.75, 1: smallest k with running sum > u
+    for u, expect in [(0.1, 0), (0.2499, 0), (0.25, 1), (0.5, 1), (0.7499, 1), (0.75, 3), (0.99, 3)]:
+        assert sampling.inverse_cdf(w, u)[0] == expect
+        res = sampling.verify_step(logits[None, :], np.zeros((0, 4)), [], [u], 1.0)
+        assert (res.n_accepted, res.next_token) == (0, expect)
+    # against numpy's own inverse-CDF categorical draw on the same uniforms
+    rng = np.random.default_rng(0)
+    weights = rng.random(17)
+    us = rng.random(1000)
+    ref = np.searchsorted(np.cumsum(weights) / weights.sum(), us, side="right")
+    got = [sampling.inverse_cdf(weights, u)[0] for u in us]
+    assert np.array_equal(ref, got)
+
+
+def test_inverse_cdf_margin_and_last_positive_fallback():
+    k, margin = sampling.inverse_cdf([1.0, 1.0, 2.0], 0.3)
+    assert k == 1 and margin == pytest.approx(0.05)
+    assert sampling.inverse_cdf([0.5, 0.5, 0.0], 1.0)[0] == 1  # u = 1 is off the grid: last positive weight
+
+
+def test_temperature_zero_is_greedy():
+    gamma = 4
+    t, d = workloads.make_sampler_logits(41, 6, gamma, 100, 1.0)
+    for b in range(6):
+        xs = [int(np.argmax(d[b, i])) for i in range(gamma)]  # the draft's own greedy draws
+        res = sampling.verify_step(t[b], d[b], xs, [0.9] * (gamma + 1), 0.0)
+        greedy = [int(np.argmax(t[b, i])) for i in range(gamma + 1)]
+        n = 0
+        while n < gamma and xs[n] == greedy[n]:
+            n += 1
+        assert (res.n_accepted, res.next_token) == (n, greedy[n])
+    # ties go to the lowest index
+    assert sampling.standardise([1.0, 3.0, 3.0, 0.0], 0.0).tolist() == [0, 1, 0, 0]
+    assert sampling.sample_token([1.0, 3.0, 3.0], 0.5, 0.0)[0] == 1
+
+
+def test_temperature_scales_logits():
+    logits = np.array([0.3, -1.2, 2.0, 0.0])
+    for T in (0.5, 2.0):
+        assert np.allclose(sampling.standardise(logits, T), sampling.standardise(logits / T, 1.0), atol=1e-15)
+    p = sampling.standardise(logits, 1.0)
+    assert p.sum() == pytest.approx(1.0) and np.allclose(p, np.exp(logits) / np.exp(logits).sum())
+
+
+def _threshold(fn, lo=0.0, hi=1.0, iters=60):
+    """Largest v in [lo, hi] with fn(v) true, for fn true on [lo, v] and false above."""
+    if fn(hi):
+        return hi
+    if not fn(lo):
+        return lo
+    for _ in range(iters):
+        mid = 0.5 * (lo + hi)
+        if fn(mid):
+            lo = mid
+        else:
+            hi = mid
+    return lo
+
+
+@pytest.mark.parametrize("V,gamma,seed", [(3, 1, 0), (5, 2, 1), (8, 2, 2), (4, 3, 3)])
+def test_exact_outcome_measures_on_small_vocabularies(V, gamma, seed):
+    """Brute force: drive verify_step over every drafted sequence and locate, by
+    bisection on each uniform, the exact measure of every outcome.  The law of
+    (n, t) must be prod beta-terms times the adjusted distribution, and the law
+    of the first emitted token must be p_1 (Appendix A.1)."""
+    rng = np.random.default_rng(seed)
+    tl = rng.normal(0, 1.5, (gamma + 1, V))
+    ql = rng.normal(0, 1.5, (gamma, V))
+    p = [sampling.standardise(r, 1.0) for r in tl]
+    q = [sampling.standardise(r, 1.0) for r in ql]
+    first_token_law = np.zeros(V)
+    total = 0.0
+    for xs in np.ndindex(*([V] * gamma)):
+        prob_x = np.prod([q[i][xs[i]] for i in range(gamma)])
+        # accept thresholds tau_i: test i passes iff r_i <= tau_i (others forced to pass)
+        taus = []
+        for i in range(gamma):
+            def passes(r, i=i):
+                us = [0.0] * gamma + [0.5]
+                us[i] = r
+                return sampling.verify_step(tl, ql, xs, us, 1.0).n_accepted > i
+            taus.append(_threshold(passes))
+            assert taus[-1] == pytest.approx(min(1.0, p[i][xs[i]] / q[i][xs[i]]), abs=1e-12)
+        for n in range(gamma + 1):
+            prob_n = np.prod(taus[:n]) * ((1 - taus[n]) if n < gamma else 1.0)
+            if prob_n == 0:
+                continue
+            us = [0.0] * n + [1.0] * (gamma - n)
+            # measure of u that yields each token: breakpoints of a step function in u
+            edges = [0.0]
+            for k in range(V - 1):
+                edges.append(_threshold(
+                    lambda u, k=k: sampling.verify_step(tl, ql, xs, us + [u], 1.0).next_token <= k, lo=edges[-1]))
+            edges.append(1.0)
+            law_t = np.diff(edges)
+            expect = p[n] if n == gamma else np.maximum(0, p[n] - q[n]) / np.maximum(0, p[n] - q[n]).sum()
+            assert np.allclose(law_t, expect, atol=1e-10)
+            total += prob_x * prob_n
+            if n >= 1:
+                first_token_law[xs[0]] += prob_x * prob_n
+            else:
+                first_token_law += prob_x * prob_n * law_t
+    assert total == pytest.approx(1.0, abs=1e-10)
+    assert np.allclose(first_token_law, p[0], atol=1e-10)
+
+
+def test_speculative_sampling_single_token_rule():
+    p = np.array([0.5, 0.3, 0.2])
+    q = np.array([0.2, 0.2, 0.6])
+    # q(x) <= p(x): always kept
+    assert sampling.speculative_sampling(p, q, 0, 0.999, 0.5) == (True, 0)
+    # q(x) > p(x): kept iff r <= p/q = 1/3
+    assert sampling.speculative_sampling(p, q, 2, 0.33, 0.5) == (True, 2)
+    # rejected: residual = [0.3, 0.1, 0] / 0.4 -> boundary at 0.75
+    assert sampling.speculative_sampling(p, q, 2, 0.34, 0.74) == (False, 0)
+    assert sampling.speculative_sampling(p, q, 2, 0.34, 0.76) == (False, 1)
