@@ -1,0 +1,169 @@
+"""Parity of the fused speculative-sampling kernel, the plain sampler and the
+device uniforms with the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+from scipy import stats
+
+from gpu_util import MARGIN, compare_verify, dev, to_dev
+from oracle import analysis, philox
+from oracle import sampling as oracle_sampling
+from paper_2211_17192_b200 import binding, workloads
+
+pytestmark = pytest.mark.gpu
+
+
+def _draft_tokens(ql, seed, temperature):
+    """x_i ~ q_i drawn by the oracle with seeded uniforms."""
+    batch, gamma, _ = ql.shape
+    draw = workloads.make_uniform_grid(seed, (batch, max(gamma, 1)))
+    xs = np.zeros((batch, gamma), dtype=np.int32)
+    for b in range(batch):
+        for i in range(gamma):
+            xs[b, i] = oracle_sampling.sample_token(ql[b, i], draw[b, i], temperature)[0]
+    return xs, draw
+
+
+def _run(tl, ql, xs, us, temperature):
+    n, t = binding.spec_verify_sample(to_dev(tl), to_dev(ql) if ql.size else None,
+                                      to_dev(xs) if xs.size else None, to_dev(us), temperature)
+    torch.cuda.synchronize()
+    return n, t
+
+
+@pytest.mark.parametrize("noise", [0.5, 1.0, 2.0])
+def test_standalone_sampler_workload(noise):
+    """Batch 64 x (gamma+1 = 8) x vocab 32000, T = 1: decisions and tokens identical."""
+    batch, gamma, vocab = 64, 7, 32000
+    tl, ql = workloads.make_sampler_logits(100 + int(noise * 10), batch, gamma, vocab, noise)
+    xs, _ = _draft_tokens(ql, 7, 1.0)
+    us = workloads.make_uniform_grid(8, (batch, gamma + 1))
+    n, t = _run(tl, ql, xs, us, 1.0)
+    flagged, total = compare_verify(n, t, tl, ql, xs, us, 1.0)
+    assert flagged <= 2, f"{flagged} of {total} sequences within {MARGIN} of a decision boundary"
+    ns = n.cpu().numpy()
+    assert ns.min() >= 0 and ns.max() <= gamma
+    if noise == 0.5:
+        assert ns.mean() > 2.0  # a close draft is accepted often
+
+
+@pytest.mark.parametrize("batch,gamma,vocab,temperature", [
+    (3, 0, 1000, 1.0),       # gamma = 0: plain draw from p
+    (5, 1, 1, 1.0),          # single-token vocabulary
+    (5, 2, 5, 1.0),
+    (7, 3, 1001, 0.7),       # rows not 16-byte aligned: scalar loads
+    (4, 10, 8192, 1.0),      # exactly one chunk
+    (4, 5, 8193, 1.3),       # one element past a chunk
+    (2, 3, 100003, 1.0),     # several chunks, ragged tail
+    (9, 4, 32000, 0.0),      # greedy
+    (6, 6, 1001, 0.0),
+    (3, 64, 257, 1.0),       # maximum gamma
+])
+def test_shapes_and_edges(batch, gamma, vocab, temperature):
+    tl, ql = workloads.make_sampler_logits(batch * 1000 + gamma, batch, gamma, vocab, 1.0)
+    xs, _ = _draft_tokens(ql, 3, temperature)
+    us = workloads.make_uniform_grid(4, (batch, gamma + 1))
+    n, t = _run(tl, ql, xs, us, temperature)
+    flagged, _ = compare_verify(n, t, tl, ql, xs, us, temperature)
+    assert flagged <= 1
+
+
+def test_identical_and_disjoint_distributions():
+    batch, gamma, vocab = 6, 4, 4096
+    tl, _ = workloads.make_sampler_logits(5, batch, gamma, vocab, 1.0)
+    ql = np.ascontiguousarray(tl[:, :gamma])
+    xs, _ = _draft_tokens(ql, 9, 1.0)
+    us = workloads.make_uniform_grid(10, (batch, gamma + 1))
+    n, t = _run(tl, ql, xs, us, 1.0)
+    assert n.cpu().tolist() == [gamma] * batch  # p = q: everything accepted (Corollary 3.4)
+    compare_verify(n, t, tl, ql, xs, us, 1.0)
+    # disjoint supports: never accepted, t from p restricted to its support
+    tl2, ql2 = tl.copy(), ql.copy()
+    tl2[:, :, vocab // 2:] = -1e4
+    ql2[:, :, : vocab // 2] = -1e4
+    xs2, _ = _draft_tokens(ql2, 9, 1.0)
+    n, t = _run(tl2, ql2, xs2, us, 1.0)
+    assert n.cpu().tolist() == [0] * batch and int(t.max()) < vocab // 2
+    compare_verify(n, t, tl2, ql2, xs2, us, 1.0)
+
+
+def test_out_of_range_draft_token_is_rejected():
+    tl, ql = workloads.make_sampler_logits(6, 2, 3, 500, 0.1)
+    xs = np.array([[1, 500, 2], [-1, 3, 4]], dtype=np.int32)
+    us = np.full((2, 4), 1.0 / 2**24, dtype=np.float32)
+    n, t = _run(tl, ql, xs, us, 1.0)
+    assert n.cpu().tolist() == [1, 0] and 0 <= int(t.min()) and int(t.max()) < 500
+
+
+def test_workspace_is_reusable_and_checked():
+    tl, ql = workloads.make_sampler_logits(7, 4, 2, 3000, 1.0)
+    xs, _ = _draft_tokens(ql, 1, 1.0)
+    us = workloads.make_uniform_grid(2, (4, 3))
+    ws = torch.full((binding.spec_verify_sample_workspace_bytes(4, 2, 3000),), 0xAB, dtype=torch.uint8, device=dev())
+    args = (to_dev(tl), to_dev(ql), to_dev(xs), to_dev(us), 1.0)
+    a = binding.spec_verify_sample(*args, workspace=ws)
+    a = (a[0].clone(), a[1].clone())
+    b = binding.spec_verify_sample(*args, workspace=ws)
+    torch.cuda.synchronize()
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    with pytest.raises(binding.SpecError):
+        binding.spec_verify_sample(*args, workspace=ws[:64])
+
+
+def test_distribution_over_a_million_trials():
+    """Appendix A.1 and Theorem 3.5 on the GPU: vocabulary 64, fixed p and q."""
+    vocab, per_launch, launches = 64, 62500, 16
+    tl, ql = workloads.make_sampler_logits(11, 1, 1, vocab, 1.0)
+    p = oracle_sampling.standardise(tl[0, 0], 1.0)
+    q = oracle_sampling.standardise(ql[0, 0], 1.0)
+    tl_d = to_dev(tl).expand(per_launch, 2, vocab).contiguous()
+    ql_d = to_dev(ql).expand(per_launch, 1, vocab).contiguous()
+    first = np.zeros(vocab)
+    accepted = 0
+    seq = torch.zeros(per_launch, dtype=torch.int32, device=dev())
+    for k in range(launches):
+        pos = torch.arange(k * per_launch, (k + 1) * per_launch, dtype=torch.int32, device=dev())
+        u_draft = binding.spec_uniforms(5, pos, seq, 0)
+        r = binding.spec_uniforms(5, pos, seq, 1)
+        u = binding.spec_uniforms(5, pos, seq, 2)
+        x = binding.spec_sample(ql_d.view(per_launch, vocab), u_draft, 1.0)
+        n, t = binding.spec_verify_sample(tl_d, ql_d, x.view(-1, 1), torch.stack([r, u], dim=1).contiguous(), 1.0)
+        emitted = torch.where(n == 1, x, t)
+        first += np.bincount(emitted.cpu().numpy(), minlength=vocab)
+        accepted += int((n == 1).sum())
+    trials = per_launch * launches
+    expected = p * trials
+    keep = expected >= 5
+    counts = np.append(first[keep], first[~keep].sum())
+    exp = np.append(expected[keep], expected[~keep].sum())
+    if exp[-1] == 0:
+        counts, exp = counts[:-1], exp[:-1]
+    assert stats.chisquare(counts, exp).pvalue > 1e-3
+    beta = analysis.beta(p, q)
+    assert abs(accepted / trials - beta) < 4 * np.sqrt(beta * (1 - beta) / trials)
+
+
+def test_device_uniforms_are_bit_exact():
+    pos = np.array([0, 1, 2, 77, 123456, 2**31 - 1], dtype=np.int32)
+    seqs = np.array([0, 0, 5, 31, 2, 9], dtype=np.int32)
+    for seed in (0, 42, 0xDEADBEEF_12345678):
+        for purpose in (0, 1, 2):
+            got = binding.spec_uniforms(seed, to_dev(pos), to_dev(seqs), purpose).cpu().numpy().astype(np.float64)
+            ref = philox.uniforms_vec(seed, pos, seqs, purpose)
+            assert np.array_equal(got, ref)
+
+
+@pytest.mark.parametrize("rows,vocab,temperature", [(64, 8192, 1.0), (5, 1001, 0.5), (3, 7, 1.0), (16, 32000, 0.0),
+                                                    (2, 100003, 1.0)])
+def test_plain_sampler(rows, vocab, temperature):
+    logits, _ = workloads.make_sampler_logits(rows + vocab, rows, 0, vocab, 1.0)
+    logits = logits[:, 0]
+    us = workloads.make_uniform_grid(12, (rows,))
+    got = binding.spec_sample(to_dev(logits), to_dev(us), temperature).cpu().numpy()
+    flagged = 0
+    for r in range(rows):
+        ref, margin = oracle_sampling.sample_token(logits[r], us[r], temperature)
+        if got[r] != ref:
+            assert margin < MARGIN
+            flagged += 1
+    assert flagged <= 1
