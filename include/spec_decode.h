@@ -72,11 +72,12 @@ const char* spec_last_error(void);
  *   n_accepted    [batch] int32 out, in [0, gamma]
  *   next_token    [batch] int32 out, in [0, vocab)
  *   workspace     scratch of at least spec_verify_sample_workspace_bytes()
- *                 bytes, 256-byte aligned; contents need not be preserved or
- *                 initialised; must not be shared by calls that may overlap
- *                 on the device.
- * One kernel launch (plus a small memset of the workspace) is enqueued on
- * `stream`; the call does not synchronise and allocates nothing.
+ *                 bytes, 256-byte aligned; contents need not be initialised
+ *                 or preserved.  It must not be shared by calls that may
+ *                 overlap on the device.
+ * Two kernel launches are enqueued on `stream` (a streaming statistics pass
+ * over all logits, then one CTA per sequence that decides and draws); the
+ * call does not synchronise and allocates nothing.
  * Errors: SPEC_ERR_BAD_ARG for null pointers, batch < 0, gamma < 0 or > 64,
  * vocab < 1, temperature < 0 or not finite, workspace too small or
  * misaligned; SPEC_ERR_CUDA if the launch fails.  batch == 0 is a no-op.

@@ -1,35 +1,64 @@
-// Fused speculative sampling (Section 2.3 / Algorithm 1, accept-adjust-draw
-// part), plain standardised sampling (Section 2.2) and the method's uniforms.
+// Speculative sampling (Section 2.3 / Algorithm 1, accept-adjust-draw part),
+// plain standardised sampling (Section 2.2) and the method's uniforms.
 //
-// One launch handles a whole batch.  Every logit is read once from HBM by the
-// statistics phase: each CTA reduces one chunk of one row of p_i or q_i to a
-// (max, sum exp) pair.  The CTA that finishes a sequence last (a ticket taken
-// with atomicAdd; nobody waits for anybody) merges the chunk statistics, runs
-// the gamma accept tests, and re-reads only row n+1 of p and q (still in L2)
-// to normalise the residual max(0, p - q) and draw from it by inverse CDF.
+// spec_verify_sample is two kernels on one stream:
+//   1. verify_stats_kernel streams every logit of p_1..p_{gamma+1} and
+//      q_1..q_gamma exactly once from HBM.  A CTA reduces one chunk of one row
+//      to (max, sum exp) with an online rescale, and also picks up the row's
+//      logit at the drafted token.  No CTA talks to another: the kernel is a
+//      pure map-reduce and runs at streaming bandwidth.
+//   2. verify_finish_kernel, one CTA per sequence, merges the chunk statistics,
+//      runs the gamma accept tests, and re-reads only row n+1 of p and q (still
+//      in L2) to normalise the residual max(0, p - q) and draw from it by
+//      inverse CDF.  It is chained with programmatic dependent launch, so its
+//      launch latency and prologue overlap the tail of the first kernel.
+#include <algorithm>
+#include <cfloat>
+
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace spec {
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
-constexpr int kGroupsPerThread = 8;                       // float4 groups held in registers
-constexpr int kChunkGroups = kThreads * kGroupsPerThread;  // 2048 groups = 8192 logits per CTA
+constexpr int kStatThreads = 512;
+constexpr int kStatWarps = kStatThreads / 32;
+constexpr int kUnroll = 4;              // 128-bit loads in flight per thread while streaming
+constexpr int kMinChunkGroups = 1024;   // a CTA streams at least 4096 logits (unless the row is shorter)
+constexpr int kTargetCtas = 148 * 24;   // about six waves of resident CTAs, so that the last wave costs little
+constexpr int kFinishThreads = 512;
+constexpr int kCdfBatch = 8;            // groups fetched per thread before any is consumed (inverse CDF, one CTA)
+constexpr int kClusterCdfBatch = 4;     // the same when a cluster shares the row
+constexpr int kWalkBatch = 4;           // 128-element steps fetched at once by the final walk
+constexpr int kMaxCluster = 4;          // CTAs per sequence in the finishing kernel
+constexpr int kSampleThreads = 512;
 constexpr int kMaxGamma = 64;
 constexpr int kMaxRows = 2 * kMaxGamma + 1;
+constexpr float kLog2e = 1.4426950408889634f;
 
-// A row of fp32 logits addressed in groups of four elements.  Rows whose base
-// is 16-byte aligned use one 128-bit load per group; others fall back to four
-// scalar loads.  Elements past the end of the row read as `pad`.
+// 2^x with one MUFU instruction (2 ulp; results below 2^-126 flush to zero,
+// which is far below anything a sum over the vocabulary can see).
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// A row of fp32 logits addressed in groups of four elements.  VEC: the vocabulary
+// is a multiple of four and every row starts on a 16-byte boundary, so a group
+// is one unconditional 128-bit load.  Otherwise four guarded scalar loads, with
+// elements past the end of the row reading as `pad`.
+template <bool VEC>
 struct Row {
     const float* base;
     int vocab;
-    bool vec;
 
     __device__ __forceinline__ float4 load(int g, float pad) const {
+        if (VEC) return __ldg(reinterpret_cast<const float4*>(base) + g);
         const int j = 4 * g;
-        if (vec && j + 3 < vocab) return __ldg(reinterpret_cast<const float4*>(base) + g);
         float4 v;
         v.x = j + 0 < vocab ? __ldg(base + j + 0) : pad;
         v.y = j + 1 < vocab ? __ldg(base + j + 1) : pad;
@@ -39,363 +68,557 @@ struct Row {
     }
 };
 
-__device__ __forceinline__ Row make_row(const float* base, int vocab) {
-    Row r;
+template <bool VEC>
+__device__ __forceinline__ Row<VEC> make_row(const float* base, int vocab) {
+    Row<VEC> r;
     r.base = base;
     r.vocab = vocab;
-    r.vec = (reinterpret_cast<uintptr_t>(base) & 15u) == 0;
     return r;
 }
 
-// Unnormalised softmax weights exp((l - max) / T) of one row.
+// Weight functors for the inverse-CDF draw.  fetch() only loads, weigh() only
+// computes, so that a caller can put several fetches in flight before it
+// consumes any of them.
+
+// Unnormalised softmax weights exp((l - max) / T) of one row; c2 = log2(e) / T.
+template <bool VEC>
 struct PlainWeights {
-    Row p;
-    float max_p, inv_t;
-    __device__ __forceinline__ float4 operator()(int g) const {
-        const float4 a = p.load(g, -INFINITY);
-        return make_float4(expf((a.x - max_p) * inv_t), expf((a.y - max_p) * inv_t),
-                           expf((a.z - max_p) * inv_t), expf((a.w - max_p) * inv_t));
+    struct Raw { float4 a; };
+    Row<VEC> p;
+    float max_p, c2;
+    __device__ __forceinline__ Raw fetch(int g) const { return Raw{p.load(g, -INFINITY)}; }
+    __device__ __forceinline__ Raw nothing() const {
+        return Raw{make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY)};
     }
+    __device__ __forceinline__ float one(float lp) const { return fast_exp2((lp - max_p) * c2); }
+    __device__ __forceinline__ float4 weigh(const Raw& r) const {
+        return make_float4(one(r.a.x), one(r.a.y), one(r.a.z), one(r.a.w));
+    }
+    __device__ __forceinline__ float4 operator()(int g) const { return weigh(fetch(g)); }
 };
 
 // max(0, p - q) with p, q the normalised softmaxes of two rows (Algorithm 1's
 // adjusted distribution before normalisation).
+template <bool VEC>
 struct ResidualWeights {
-    Row p, q;
-    float max_p, max_q, inv_sum_p, inv_sum_q, inv_t;
+    struct Raw { float4 a, b; };
+    Row<VEC> p, q;
+    float max_p, max_q, inv_sum_p, inv_sum_q, c2;
+    __device__ __forceinline__ Raw fetch(int g) const { return Raw{p.load(g, -INFINITY), q.load(g, -INFINITY)}; }
+    __device__ __forceinline__ Raw nothing() const {
+        const float4 z = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        return Raw{z, z};
+    }
     __device__ __forceinline__ float one(float lp, float lq) const {
-        const float pv = expf((lp - max_p) * inv_t) * inv_sum_p;
-        const float qv = expf((lq - max_q) * inv_t) * inv_sum_q;
+        const float pv = fast_exp2((lp - max_p) * c2) * inv_sum_p;
+        const float qv = fast_exp2((lq - max_q) * c2) * inv_sum_q;
         return fmaxf(0.0f, pv - qv);
     }
-    __device__ __forceinline__ float4 operator()(int g) const {
-        const float4 a = p.load(g, -INFINITY);
-        const float4 b = q.load(g, -INFINITY);
-        return make_float4(one(a.x, b.x), one(a.y, b.y), one(a.z, b.z), one(a.w, b.w));
+    __device__ __forceinline__ float4 weigh(const Raw& r) const {
+        return make_float4(one(r.a.x, r.b.x), one(r.a.y, r.b.y), one(r.a.z, r.b.z), one(r.a.w, r.b.w));
     }
+    __device__ __forceinline__ float4 operator()(int g) const { return weigh(fetch(g)); }
 };
 
+template <int WARPS>
 struct CdfScratch {
-    float warp_total[kWarps];
-    float total;
+    float part[WARPS];              // per-warp totals of the level being scanned
+    float all[kMaxCluster * WARPS];  // the same for every CTA of a cluster
+    float pick_before, pick_total;   // outcome of the cluster-wide scan
+    int pick_part_index, pick_hit;
     int result;
     int last_positive;
 };
 
-// Inverse-CDF draw by one CTA: the smallest index k whose running weight sum
-// exceeds u * (sum of all weights); the last index with positive weight if
-// rounding leaves none.  Each warp owns a contiguous segment of the vocabulary
-// so that running sums follow index order.  Returns the index to all threads
-// and the total through *total_out.
-template <class Weights>
-__device__ int block_inverse_cdf(const Weights& w, int vocab, float u, CdfScratch& s, float* total_out) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int groups = (vocab + 3) >> 2;
-    const int seg = (groups + kWarps - 1) / kWarps;
-    const int g0 = warp * seg;
-    const int g1 = min(groups, g0 + seg);
-
+// Sum of the weights of groups [g0, g1) by one warp, lane-strided so that every
+// load instruction covers 512 contiguous bytes; BATCH fetches are in flight
+// per lane before any is consumed.
+template <int BATCH, class Weights>
+__device__ __forceinline__ float warp_range_sum(const Weights& w, int g0, int g1, int lane) {
     float acc = 0.0f;
-    for (int g = g0 + lane; g < g1; g += 32) {
-        const float4 v = w(g);
-        acc += (v.x + v.y) + (v.z + v.w);
+    for (int base = g0 + lane; base < g1; base += 32 * BATCH) {
+        typename Weights::Raw raw[BATCH];
+#pragma unroll
+        for (int i = 0; i < BATCH; ++i) {
+            const int g = base + 32 * i;
+            raw[i] = g < g1 ? w.fetch(g) : w.nothing();
+        }
+#pragma unroll
+        for (int i = 0; i < BATCH; ++i) {
+            const float4 v = w.weigh(raw[i]);
+            acc += (v.x + v.y) + (v.z + v.w);
+        }
     }
-    acc = warp_sum(acc);
-    if (lane == 0) s.warp_total[warp] = acc;
+    return warp_sum(acc);
+}
+
+// Which of `count` consecutive parts holds `target`: the first part whose
+// running sum exceeds it (the same arithmetic in every thread, so every thread
+// agrees).  Returns -1 if none does; *before gets the running sum in front of
+// the chosen part; *fallback is the last part with positive weight (0 if none),
+// for the case where rounding leaves no part above the target.
+template <class PartAt>
+__device__ __forceinline__ int pick_part(PartAt part_at, int count, float target, float* before, int* fallback) {
+    float run = 0.0f;
+    int hit = -1, last = 0;
+    for (int i = 0; i < count; ++i) {
+        const float v = part_at(i);
+        const float next = run + v;
+        if (hit < 0 && next > target) {
+            hit = i;
+            *before = run;
+        }
+        if (v > 0.0f) last = i;
+        run = next;
+    }
+    *fallback = last;
+    return hit;
+}
+
+// The draw inside one contiguous range of groups [r0, r1) by a whole CTA: `rem`
+// is the target minus the weight in front of the range.  Long ranges are first
+// cut into one sub-range per warp; warp 0 then walks the chosen (sub-)range 128
+// elements at a time with a warp scan.  With want_hit false the answer is the
+// last index of the range with positive weight.  Returns the index (or -1) to
+// all threads.
+template <int WARPS, class Weights>
+__device__ int locate_in_range(const Weights& w, int r0, int r1, float rem, bool want_hit, CdfScratch<WARPS>& s) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
         s.result = -1;
         s.last_positive = -1;
     }
+    if (r1 - r0 > 4 * 32) {  // uniform across the CTA
+        const int sub = (r1 - r0 + WARPS - 1) / WARPS;
+        const int g0 = min(r1, r0 + warp * sub), g1 = min(r1, g0 + sub);
+        const float acc = warp_range_sum<2>(w, g0, g1, lane);
+        __syncthreads();  // previous users of s.part are done
+        if (lane == 0) s.part[warp] = acc;
+        __syncthreads();
+        float before = 0.0f;
+        int fallback = 0;
+        int hit = pick_part([&](int i) { return s.part[i]; }, WARPS, rem, &before, &fallback);
+        if (!want_hit || hit < 0) {
+            want_hit = false;
+            hit = fallback;
+        }
+        rem -= before;
+        r0 = min(r1, r0 + hit * sub);
+        r1 = min(r1, r0 + sub);
+    }
     __syncthreads();
-
-    float total = 0.0f;
-#pragma unroll
-    for (int i = 0; i < kWarps; ++i) total += s.warp_total[i];
-    const float target = u * total;
-    // The segment that contains the target: first warp whose running total exceeds it.
-    int hit_warp = -1;
-    float before = 0.0f, run = 0.0f;
-#pragma unroll
-    for (int i = 0; i < kWarps; ++i) {
-        const float next = run + s.warp_total[i];
-        if (hit_warp < 0 && next > target) {
-            hit_warp = i;
-            before = run;
-        }
-        run = next;
-    }
-    if (hit_warp < 0) {  // rounding: fall back to the last segment with positive weight
-        before = 0.0f;
-        run = 0.0f;
-        for (int i = 0; i < kWarps; ++i) {
-            if (s.warp_total[i] > 0.0f) {
-                hit_warp = i;
-                before = run;
-            }
-            run += s.warp_total[i];
-        }
-    }
-
-    if (warp == hit_warp) {
-        const float rem = target - before;
-        float base = 0.0f;  // running sum of this segment before the current step
+    if (warp == 0) {
+        float run = 0.0f;
         int found = -1, last_pos = -1;
-        for (int gs = g0; gs < g1 && found < 0; gs += 32) {
-            const int g = gs + lane;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (g < g1) v = w(g);
-            const float mine = (v.x + v.y) + (v.z + v.w);
-            const float incl = warp_inclusive_scan(mine, lane);
-            const unsigned over = __ballot_sync(kFullMask, base + incl > rem);
-            const unsigned pos = __ballot_sync(kFullMask, mine > 0.0f);
-            if (pos) {
-                const int pl = 31 - __clz(pos);  // last lane with positive weight in this step
-                const float4 pv = make_float4(__shfl_sync(kFullMask, v.x, pl), __shfl_sync(kFullMask, v.y, pl),
-                                              __shfl_sync(kFullMask, v.z, pl), __shfl_sync(kFullMask, v.w, pl));
-                const int pg = 4 * (gs + pl);
-                last_pos = pv.w > 0.f ? pg + 3 : pv.z > 0.f ? pg + 2 : pv.y > 0.f ? pg + 1 : pg;
+        for (int gb = r0; gb < r1 && found < 0; gb += 32 * kWalkBatch) {
+            typename Weights::Raw raw[kWalkBatch];  // the whole batch is fetched before the serial scan
+#pragma unroll
+            for (int i = 0; i < kWalkBatch; ++i) {
+                const int g = gb + 32 * i + lane;
+                raw[i] = g < r1 ? w.fetch(g) : w.nothing();
             }
-            if (over) {
-                const int hl = __ffs(over) - 1;
-                const float excl = __shfl_sync(kFullMask, incl - mine, hl) + base;
-                const float4 hv = make_float4(__shfl_sync(kFullMask, v.x, hl), __shfl_sync(kFullMask, v.y, hl),
-                                              __shfl_sync(kFullMask, v.z, hl), __shfl_sync(kFullMask, v.w, hl));
-                const int hg = 4 * (gs + hl);
-                float c = excl + hv.x;
-                if (c > rem) found = hg;
-                else if ((c += hv.y) > rem) found = hg + 1;
-                else if ((c += hv.z) > rem) found = hg + 2;
-                else found = hg + 3;
+#pragma unroll
+            for (int i = 0; i < kWalkBatch; ++i) {
+                const int gs = gb + 32 * i;
+                if (gs >= r1 || found >= 0) break;
+                const float4 v = w.weigh(raw[i]);
+                const float mine = (v.x + v.y) + (v.z + v.w);
+                const float incl = warp_inclusive_scan(mine, lane);
+                const unsigned over = want_hit ? __ballot_sync(kFullMask, run + incl > rem) : 0u;
+                const unsigned pos = __ballot_sync(kFullMask, mine > 0.0f);
+                if (pos) {
+                    const int pl = 31 - __clz(pos);  // last lane with positive weight in this step
+                    const float py = __shfl_sync(kFullMask, v.y, pl), pz = __shfl_sync(kFullMask, v.z, pl),
+                                pw = __shfl_sync(kFullMask, v.w, pl);
+                    const int pg = 4 * (gs + pl);
+                    last_pos = pw > 0.f ? pg + 3 : pz > 0.f ? pg + 2 : py > 0.f ? pg + 1 : pg;
+                }
+                if (over) {
+                    const int hl = __ffs(over) - 1;
+                    const float excl = __shfl_sync(kFullMask, incl - mine, hl) + run;
+                    const float hx = __shfl_sync(kFullMask, v.x, hl), hy = __shfl_sync(kFullMask, v.y, hl),
+                                hz = __shfl_sync(kFullMask, v.z, hl);
+                    const int hg = 4 * (gs + hl);
+                    float c = excl + hx;
+                    if (c > rem) found = hg;
+                    else if ((c += hy) > rem) found = hg + 1;
+                    else if ((c += hz) > rem) found = hg + 2;
+                    else found = hg + 3;
+                }
+                run += __shfl_sync(kFullMask, incl, 31);
             }
-            base += __shfl_sync(kFullMask, incl, 31);
         }
         if (lane == 0) {
             s.result = found;
             s.last_positive = last_pos;
         }
     }
-    if (tid == 0) s.total = total;
     __syncthreads();
-    int k = s.result >= 0 ? s.result : s.last_positive;
-    k = max(0, min(k, vocab - 1));
-    *total_out = s.total;
+    const int k = s.result >= 0 ? s.result : s.last_positive;
     __syncthreads();  // scratch may be reused by the caller
     return k;
 }
 
-struct ChunkStat {
-    float max;   // chunk maximum
-    float aux;   // T > 0: sum exp((l - max) / T) over the chunk; T = 0: argmax index as int bits
-};
+// Inverse-CDF draw by one CTA of 32 * WARPS threads: the smallest index k whose
+// running weight sum exceeds u * (sum of all weights); the last index with
+// positive weight if rounding leaves none.  The vocabulary is cut into WARPS
+// contiguous segments (one per warp); the segment holding the target is then
+// resolved by locate_in_range.  Returns the index to all threads, the total
+// through *total_out.
+template <int WARPS, class Weights>
+__device__ int block_inverse_cdf(const Weights& w, int vocab, float u, CdfScratch<WARPS>& s, float* total_out) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int groups = (vocab + 3) >> 2;
+    const int seg = (groups + WARPS - 1) / WARPS;
+    const int g0 = min(groups, warp * seg), g1 = min(groups, g0 + seg);
+    const float acc = warp_range_sum<kCdfBatch>(w, g0, g1, lane);
+    if (lane == 0) s.part[warp] = acc;
+    __syncthreads();
+    float total = 0.0f;
+#pragma unroll
+    for (int i = 0; i < WARPS; ++i) total += s.part[i];
+    const float target = u * total;
+    float before = 0.0f;
+    int fallback = 0;
+    int hit = pick_part([&](int i) { return s.part[i]; }, WARPS, target, &before, &fallback);
+    const bool want_hit = hit >= 0;
+    if (!want_hit) hit = fallback;
+    const int r0 = min(groups, hit * seg), r1 = min(groups, r0 + seg);
+    const int k = locate_in_range<WARPS>(w, r0, r1, target - before, want_hit, s);
+    *total_out = total;
+    return max(0, min(k, vocab - 1));
+}
 
-struct SharedState {
-    float red[kWarps];
-    int red_i[kWarps];
-    float row_max[kMaxRows];
-    float row_aux[kMaxRows];
-    CdfScratch cdf;
-    int flag;
-    int n;
+// The same draw by a thread-block cluster: CTA `rank` of `nctas` owns a
+// contiguous slice of the vocabulary, the per-warp totals of all CTAs are read
+// through distributed shared memory, and only the CTA whose slice holds the
+// target goes on to resolve it.  Returns the index in that CTA and -1 in the
+// others; the total is returned to all.
+template <int WARPS, class Weights>
+__device__ int cluster_inverse_cdf(const Weights& w, int vocab, float u, CdfScratch<WARPS>& s, float* total_out) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int nctas = static_cast<int>(cluster.num_blocks());
+    const int rank = static_cast<int>(cluster.block_rank());
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int groups = (vocab + 3) >> 2;
+    const int slice = (groups + nctas - 1) / nctas;
+    const int seg = (slice + WARPS - 1) / WARPS;
+    auto seg_begin = [&](int part) {  // part = cta * WARPS + warp
+        const int c0 = min(groups, (part / WARPS) * slice), c1 = min(groups, c0 + slice);
+        return min(c1, c0 + (part % WARPS) * seg);
+    };
+    auto seg_end = [&](int part) {
+        const int c0 = min(groups, (part / WARPS) * slice), c1 = min(groups, c0 + slice);
+        return min(c1, seg_begin(part) + seg);
+    };
+    const int mine = rank * WARPS + warp;
+    const float acc = warp_range_sum<kClusterCdfBatch>(w, seg_begin(mine), seg_end(mine), lane);
+    if (lane == 0) s.part[warp] = acc;
+    cluster.sync();
+    // warp 0 copies every CTA's totals into this CTA's shared memory ...
+    const int parts = nctas * WARPS;
+    if (warp == 0)
+        for (int i = lane; i < parts; i += 32) s.all[i] = cluster.map_shared_rank(s.part, i / WARPS)[i % WARPS];
+    __syncthreads();
+    // ... and scans them: lane l takes the consecutive parts [l*per, (l+1)*per)
+    if (warp == 0) {
+        const int per = (parts + 31) / 32;
+        float mine_sum = 0.0f;
+        for (int i = lane * per; i < min(parts, (lane + 1) * per); ++i) mine_sum += s.all[i];
+        const float incl = warp_inclusive_scan(mine_sum, lane);
+        const float tot = __shfl_sync(kFullMask, incl, 31);
+        const float tgt = u * tot;
+        const unsigned over = __ballot_sync(kFullMask, incl > tgt);
+        const unsigned pos = __ballot_sync(kFullMask, mine_sum > 0.0f);
+        const int hl = over ? __ffs(over) - 1 : (pos ? 31 - __clz(pos) : 0);
+        if (lane == hl) {
+            float run = incl - mine_sum;
+            int hit = -1, last = lane * per;
+            for (int i = lane * per; i < min(parts, (lane + 1) * per); ++i) {
+                if (s.all[i] > 0.0f) last = i;
+                if (over && hit < 0 && run + s.all[i] > tgt) { hit = i; break; }
+                run += s.all[i];
+            }
+            if (hit < 0) { hit = last; s.pick_hit = 0; run = 0.0f; } else { s.pick_hit = 1; }
+            s.pick_part_index = hit;
+            s.pick_before = run;
+            s.pick_total = tot;
+        }
+    }
+    __syncthreads();
+    const float total = s.pick_total;
+    const float target = u * total;
+    const float before = s.pick_before;
+    int hit = s.pick_part_index;
+    const bool want_hit_flag = s.pick_hit != 0;
+    cluster.sync();  // nobody reads another CTA's totals after this point
+    const bool want_hit = want_hit_flag;
+    *total_out = total;
+    if (hit / WARPS != rank) return -1;
+    const int k = locate_in_range<WARPS>(w, seg_begin(hit), seg_end(hit), target - before, want_hit, s);
+    return max(0, min(k, vocab - 1));
+}
+
+// (max, lowest index attaining it) across a CTA of 32 * WARPS threads; the
+// result is valid in thread 0.
+template <int WARPS>
+__device__ __forceinline__ void block_argmax(float& m, int& arg, float* red, int* red_i) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(kFullMask, m, o);
+        const int oa = __shfl_xor_sync(kFullMask, arg, o);
+        if (om > m || (om == m && oa < arg)) { m = om; arg = oa; }
+    }
+    if (lane == 0) { red[warp] = m; red_i[warp] = arg; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < WARPS; ++i)
+            if (red[i] > m || (red[i] == m && red_i[i] < arg)) { m = red[i]; arg = red_i[i]; }
+    }
+}
+
+// One chunk of one row, as written by verify_stats_kernel.
+struct __align__(16) ChunkStat {
+    float max;     // chunk maximum
+    float aux;     // T > 0: sum exp((l - max) / T) over the chunk; T = 0: argmax index as int bits
+    float xlogit;  // the row's logit at the drafted token, if that token falls in this chunk
+    float pad;
 };
 
 // grid = (chunks, rows, batch); rows = 2*gamma+1 (T > 0: p_1..p_{gamma+1}, q_1..q_gamma)
 // or gamma+1 (T = 0: only p is read).
-template <bool GREEDY>
-__global__ void __launch_bounds__(kThreads)
-verify_sample_kernel(const float* __restrict__ target_logits, const float* __restrict__ draft_logits,
-                     const int32_t* __restrict__ draft_tokens, const float* __restrict__ uniforms, int gamma,
-                     int vocab, float inv_t, ChunkStat* __restrict__ stats, unsigned* __restrict__ tickets,
-                     int32_t* __restrict__ n_accepted, int32_t* __restrict__ next_token) {
-    __shared__ SharedState sh;
+template <bool GREEDY, bool VEC>
+__global__ void __launch_bounds__(kStatThreads)
+verify_stats_kernel(const float* __restrict__ target_logits, const float* __restrict__ draft_logits,
+                    const int32_t* __restrict__ draft_tokens, int gamma, int vocab, float c2,
+                    ChunkStat* __restrict__ stats) {
+    __shared__ float red[kStatWarps];
+    __shared__ float red_s[kStatWarps];
+    __shared__ int red_i[kStatWarps];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chunk = blockIdx.x, chunks = gridDim.x;
     const int row = blockIdx.y, rows = gridDim.y;
     const int b = blockIdx.z;
 
-    const float* tl = target_logits + static_cast<size_t>(b) * (gamma + 1) * vocab;
-    const float* ql = GREEDY ? nullptr : draft_logits + static_cast<size_t>(b) * gamma * vocab;
-    const float* src = row <= gamma ? tl + static_cast<size_t>(row) * vocab
-                                    : ql + static_cast<size_t>(row - gamma - 1) * vocab;
-    const Row r = make_row(src, vocab);
+    const float* src = row <= gamma
+        ? target_logits + (static_cast<size_t>(b) * (gamma + 1) + row) * vocab
+        : draft_logits + (static_cast<size_t>(b) * gamma + (row - gamma - 1)) * vocab;
+    const Row<VEC> r = make_row<VEC>(src, vocab);
     const int groups = (vocab + 3) >> 2;
-    const int per_chunk = (groups + chunks - 1) / chunks;  // <= kChunkGroups by construction of the grid
+    const int per_chunk = (groups + chunks - 1) / chunks;
     const int g0 = chunk * per_chunk;
     const int g1 = min(groups, g0 + per_chunk);
 
-    // ---- statistics phase: this chunk's logits, each read exactly once ----
-    float4 v[kGroupsPerThread];
-#pragma unroll
-    for (int i = 0; i < kGroupsPerThread; ++i) {
-        const int g = g0 + tid + i * kThreads;
-        v[i] = g < g1 ? r.load(g, -INFINITY) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    // The drafted token this row is tested at (none for p_{gamma+1}): thread 0
+    // fetches the row's logit there if it lies in this chunk, so the accept test
+    // needs no further trip to memory.
+    float xlogit = 0.0f;
+    if (tid == 0 && !GREEDY && row != gamma) {
+        const int x = draft_tokens[static_cast<size_t>(b) * gamma + (row < gamma ? row : row - gamma - 1)];
+        if (x >= 4 * g0 && x < min(vocab, 4 * g1)) xlogit = __ldg(src + x);
     }
-    float m = -INFINITY;
+
+    // Every thread streams groups g0+tid, g0+tid+T, ... with kUnroll 128-bit
+    // loads in flight and keeps a running (max, sum exp) pair that is rescaled
+    // when the maximum moves; one block-wide merge at the end.
+    constexpr float kPad = -INFINITY;
+    float m = -FLT_MAX;  // finite, so that (m - new_max) never becomes inf - inf
+    float s = 0.0f;
     int arg = 0x7fffffff;
+    for (int base = g0 + tid; base < g1; base += kUnroll * kStatThreads) {
+        float4 v[kUnroll];
 #pragma unroll
-    for (int i = 0; i < kGroupsPerThread; ++i) {
+        for (int i = 0; i < kUnroll; ++i) {
+            const int g = base + i * kStatThreads;
+            v[i] = g < g1 ? r.load(g, kPad) : make_float4(kPad, kPad, kPad, kPad);
+        }
         if (GREEDY) {
-            const int j = 4 * (g0 + tid + i * kThreads);
-            if (v[i].x > m) { m = v[i].x; arg = j; }
-            if (v[i].y > m) { m = v[i].y; arg = j + 1; }
-            if (v[i].z > m) { m = v[i].z; arg = j + 2; }
-            if (v[i].w > m) { m = v[i].w; arg = j + 3; }
+#pragma unroll
+            for (int i = 0; i < kUnroll; ++i) {
+                const int j = 4 * (base + i * kStatThreads);  // indices grow with i: '>' keeps the lowest on ties
+                if (v[i].x > m) { m = v[i].x; arg = j; }
+                if (v[i].y > m) { m = v[i].y; arg = j + 1; }
+                if (v[i].z > m) { m = v[i].z; arg = j + 2; }
+                if (v[i].w > m) { m = v[i].w; arg = j + 3; }
+            }
         } else {
-            m = fmaxf(m, fmaxf(fmaxf(v[i].x, v[i].y), fmaxf(v[i].z, v[i].w)));
+            float bm = m;
+#pragma unroll
+            for (int i = 0; i < kUnroll; ++i)
+                bm = fmaxf(bm, fmaxf(fmaxf(v[i].x, v[i].y), fmaxf(v[i].z, v[i].w)));
+            s *= fast_exp2((m - bm) * c2);
+            m = bm;
+#pragma unroll
+            for (int i = 0; i < kUnroll; ++i)
+                s += (fast_exp2((v[i].x - m) * c2) + fast_exp2((v[i].y - m) * c2)) +
+                     (fast_exp2((v[i].z - m) * c2) + fast_exp2((v[i].w - m) * c2));
         }
     }
+    ChunkStat* out = stats + (static_cast<size_t>(b) * rows + row) * chunks + chunk;
     if (GREEDY) {
-        // (max, lowest index) across the block
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float om = __shfl_xor_sync(kFullMask, m, o);
-            const int oa = __shfl_xor_sync(kFullMask, arg, o);
-            if (om > m || (om == m && oa < arg)) { m = om; arg = oa; }
-        }
-        if (lane == 0) { sh.red[warp] = m; sh.red_i[warp] = arg; }
-        __syncthreads();
-        if (tid == 0) {
-            for (int i = 1; i < kWarps; ++i)
-                if (sh.red[i] > m || (sh.red[i] == m && sh.red_i[i] < arg)) { m = sh.red[i]; arg = sh.red_i[i]; }
-            ChunkStat st;
-            st.max = m;
-            st.aux = __int_as_float(arg);
-            stats[(static_cast<size_t>(b) * rows + row) * chunks + chunk] = st;
-        }
+        block_argmax<kStatWarps>(m, arg, red, red_i);
+        if (tid == 0) *reinterpret_cast<float4*>(out) = make_float4(m, __int_as_float(arg), 0.0f, 0.0f);
     } else {
-        m = warp_max(m);
-        if (lane == 0) sh.red[warp] = m;
-        __syncthreads();
-        m = sh.red[0];
-#pragma unroll
-        for (int i = 1; i < kWarps; ++i) m = fmaxf(m, sh.red[i]);
-        __syncthreads();
-        float s = 0.0f;
-        if (m > -INFINITY) {
-#pragma unroll
-            for (int i = 0; i < kGroupsPerThread; ++i)
-                s += (expf((v[i].x - m) * inv_t) + expf((v[i].y - m) * inv_t)) +
-                     (expf((v[i].z - m) * inv_t) + expf((v[i].w - m) * inv_t));
-        }
-        s = warp_sum(s);
-        if (lane == 0) sh.red[warp] = s;
+        const float wm = warp_max(m);
+        s = warp_sum(s * fast_exp2((m - wm) * c2));
+        if (lane == 0) { red[warp] = wm; red_s[warp] = s; }
         __syncthreads();
         if (tid == 0) {
+            float bm = red[0];
+#pragma unroll
+            for (int i = 1; i < kStatWarps; ++i) bm = fmaxf(bm, red[i]);
             float t = 0.0f;
 #pragma unroll
-            for (int i = 0; i < kWarps; ++i) t += sh.red[i];
-            ChunkStat st;
-            st.max = m;
-            st.aux = t;
-            stats[(static_cast<size_t>(b) * rows + row) * chunks + chunk] = st;
+            for (int i = 0; i < kStatWarps; ++i) t += red_s[i] * fast_exp2((red[i] - bm) * c2);
+            *reinterpret_cast<float4*>(out) = make_float4(bm, t, xlogit, 0.0f);
         }
     }
+    // Let the finishing kernel's CTAs be scheduled as this grid drains.
+    asm volatile("griddepcontrol.launch_dependents;");
+}
 
-    // ---- ticket: the last CTA of this sequence does the rest ----
-    if (tid == 0) {
-        __threadfence();
-        const unsigned prev = atomicAdd(&tickets[b], 1u);
-        sh.flag = prev == static_cast<unsigned>(rows * chunks - 1);
-    }
-    __syncthreads();
-    if (!sh.flag) return;
-    __threadfence();
+struct FinishShared {
+    float row_max[kMaxRows];
+    float row_aux[kMaxRows];
+    float row_x[kMaxRows];
+    CdfScratch<kFinishThreads / 32> cdf;
+    float u_final;
+    int n;
+};
 
-    // merge chunk statistics per row
-    const ChunkStat* st_b = stats + static_cast<size_t>(b) * rows * chunks;
-    for (int rr = tid; rr < rows; rr += kThreads) {
-        float M = -INFINITY, A = 0.0f;
+// grid = batch * cluster size, one thread-block cluster per sequence.  Everything
+// after the statistics: merge, accept tests, adjusted distribution, draw.  The
+// cheap decision part is repeated in every CTA of the cluster; the pass over
+// row n+1 is split between them.
+template <bool GREEDY, bool VEC>
+__global__ void __launch_bounds__(kFinishThreads, 2)
+verify_finish_kernel(const float* __restrict__ target_logits, const float* __restrict__ draft_logits,
+                     const int32_t* __restrict__ draft_tokens, const float* __restrict__ uniforms, int gamma,
+                     int vocab, float inv_t, int chunks, int cluster_size, const ChunkStat* __restrict__ stats,
+                     int32_t* __restrict__ n_accepted, int32_t* __restrict__ next_token) {
+    __shared__ FinishShared sh;
+    const int tid = threadIdx.x;
+    const int b = blockIdx.x / cluster_size;
+    const int rank = blockIdx.x % cluster_size;
+    const int rows = GREEDY ? gamma + 1 : 2 * gamma + 1;
+    const float c2 = inv_t * kLog2e;
+    const float* tl = target_logits + static_cast<size_t>(b) * (gamma + 1) * vocab;
+    const float* ql = GREEDY ? nullptr : draft_logits + static_cast<size_t>(b) * gamma * vocab;
+    const int groups = (vocab + 3) >> 2;
+    const int per_chunk = (groups + chunks - 1) / chunks;
+
+    // Inputs that the statistics kernel does not produce can be fetched before
+    // waiting for it.
+    float my_uniform = 0.5f;
+    if (!GREEDY && tid <= gamma) my_uniform = __ldg(uniforms + static_cast<size_t>(b) * (gamma + 1) + tid);
+    int my_x = -1;
+    if (tid < rows && tid != gamma)
+        my_x = draft_tokens[static_cast<size_t>(b) * gamma + (tid < gamma ? tid : tid - gamma - 1)];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // merge the chunk statistics of row `tid` (four loads in flight at a time)
+    if (tid < rows) {
+        const ChunkStat* st_r = stats + (static_cast<size_t>(b) * rows + tid) * chunks;
+        float M = -FLT_MAX, A = 0.0f, X = 0.0f;
         int best = 0x7fffffff;
-        for (int c = 0; c < chunks; ++c) {
-            const float cm = __ldcg(&st_b[rr * chunks + c].max);
-            const float ca = __ldcg(&st_b[rr * chunks + c].aux);
-            if (GREEDY) {
-                const int ci = __float_as_int(ca);
-                if (cm > M || (cm == M && ci < best)) { M = cm; best = ci; }
-            } else {
-                M = fmaxf(M, cm);
-            }
-        }
-        if (GREEDY) {
-            A = __int_as_float(best);
-        } else {
-            for (int c = 0; c < chunks; ++c) {
-                const float cm = __ldcg(&st_b[rr * chunks + c].max);
-                const float ca = __ldcg(&st_b[rr * chunks + c].aux);
-                if (cm > -INFINITY) A += ca * expf((cm - M) * inv_t);
-            }
-        }
-        sh.row_max[rr] = M;
-        sh.row_aux[rr] = A;
-    }
-    __syncthreads();
-
-    // the gamma accept tests, in order (Algorithm 1: n = first rejection)
-    if (tid == 0) {
-        int n = gamma;
-        for (int i = 0; i < gamma; ++i) {
-            const int x = draft_tokens[static_cast<size_t>(b) * gamma + i];
-            bool reject = true;
-            if (x >= 0 && x < vocab) {
+        const int xchunk = (my_x >= 0 && my_x < vocab) ? (my_x >> 2) / per_chunk : -1;
+        for (int c0 = 0; c0 < chunks; c0 += 4) {
+            float4 st[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                st[i] = c0 + i < chunks ? __ldcg(reinterpret_cast<const float4*>(st_r + c0 + i))
+                                        : make_float4(-FLT_MAX, __int_as_float(0x7fffffff), 0.0f, 0.0f);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (c0 + i >= chunks) break;
                 if (GREEDY) {
-                    reject = x != __float_as_int(sh.row_aux[i]);
+                    const int ci = __float_as_int(st[i].y);
+                    if (st[i].x > M || (st[i].x == M && ci < best)) { M = st[i].x; best = ci; }
                 } else {
-                    const float ep = expf((tl[static_cast<size_t>(i) * vocab + x] - sh.row_max[i]) * inv_t);
-                    const float eq = expf((ql[static_cast<size_t>(i) * vocab + x] - sh.row_max[gamma + 1 + i]) * inv_t);
-                    const float rr = uniforms[static_cast<size_t>(b) * (gamma + 1) + i];
-                    // r * q(x) > p(x) with p = ep / Sp, q = eq / Sq, cross-multiplied
-                    reject = rr * eq * sh.row_aux[i] > ep * sh.row_aux[gamma + 1 + i];
+                    const float nm = fmaxf(M, st[i].x);
+                    A = A * fast_exp2((M - nm) * c2) + st[i].y * fast_exp2((st[i].x - nm) * c2);
+                    M = nm;
+                    if (c0 + i == xchunk) X = st[i].z;
                 }
             }
-            if (reject) { n = i; break; }
         }
-        sh.n = n;
+        sh.row_max[tid] = M;
+        sh.row_aux[tid] = GREEDY ? __int_as_float(best) : A;
+        sh.row_x[tid] = X;
     }
+    if (tid == 0) sh.n = gamma;
+    __syncthreads();
+
+    // the gamma accept tests (Algorithm 1: n = index of the first rejection)
+    if (tid < gamma) {
+        bool reject = true;
+        if (my_x >= 0 && my_x < vocab) {
+            if (GREEDY) {
+                reject = my_x != __float_as_int(sh.row_aux[tid]);
+            } else {
+                const float ep = expf((sh.row_x[tid] - sh.row_max[tid]) * inv_t);
+                const float eq = expf((sh.row_x[gamma + 1 + tid] - sh.row_max[gamma + 1 + tid]) * inv_t);
+                // r * q(x) > p(x) with p = ep / Sp, q = eq / Sq, cross-multiplied
+                reject = my_uniform * eq * sh.row_aux[tid] > ep * sh.row_aux[gamma + 1 + tid];
+            }
+        }
+        if (reject) atomicMin(&sh.n, tid);
+    }
+    if (tid == gamma) sh.u_final = my_uniform;
     __syncthreads();
     const int n = sh.n;
 
-    int token;
+    int token = -1;
     if (GREEDY) {
-        token = __float_as_int(sh.row_aux[n]);
+        if (rank == 0) token = __float_as_int(sh.row_aux[n]);
     } else {
-        const float u = uniforms[static_cast<size_t>(b) * (gamma + 1) + gamma];
-        PlainWeights pw;
-        pw.p = make_row(tl + static_cast<size_t>(n) * vocab, vocab);
+        constexpr int W = kFinishThreads / 32;
+        const float u = sh.u_final;
+        PlainWeights<VEC> pw;
+        pw.p = make_row<VEC>(tl + static_cast<size_t>(n) * vocab, vocab);
         pw.max_p = sh.row_max[n];
-        pw.inv_t = inv_t;
+        pw.c2 = c2;
         float total = 0.0f;
         bool plain = n == gamma;
         if (!plain) {
-            ResidualWeights rw;
+            ResidualWeights<VEC> rw;
             rw.p = pw.p;
-            rw.q = make_row(ql + static_cast<size_t>(n) * vocab, vocab);
+            rw.q = make_row<VEC>(ql + static_cast<size_t>(n) * vocab, vocab);
             rw.max_p = sh.row_max[n];
             rw.max_q = sh.row_max[gamma + 1 + n];
             rw.inv_sum_p = 1.0f / sh.row_aux[n];
             rw.inv_sum_q = 1.0f / sh.row_aux[gamma + 1 + n];
-            rw.inv_t = inv_t;
-            token = block_inverse_cdf(rw, vocab, u, sh.cdf, &total);
+            rw.c2 = c2;
+            token = cluster_inverse_cdf<W>(rw, vocab, u, sh.cdf, &total);
             plain = !(total > 0.0f) || !isfinite(total);  // vanished residual: draw from p_{n+1}
         }
-        if (plain) token = block_inverse_cdf(pw, vocab, u, sh.cdf, &total);
+        if (plain) token = cluster_inverse_cdf<W>(pw, vocab, u, sh.cdf, &total);
     }
     if (tid == 0) {
-        n_accepted[b] = n;
-        next_token[b] = token;
-        tickets[b] = 0;  // leave the workspace ready for the next launch
+        if (rank == 0) n_accepted[b] = n;
+        if (token >= 0) next_token[b] = token;  // exactly one CTA of the cluster holds the draw
     }
 }
 
 // One CTA per row: tokens[r] ~ softmax(logits[r] / T), or argmax at T = 0.
-__global__ void __launch_bounds__(kThreads)
+template <bool VEC>
+__global__ void __launch_bounds__(kSampleThreads)
 sample_kernel(const float* __restrict__ logits, const float* __restrict__ uniforms, int vocab, float inv_t,
               bool greedy, int32_t* __restrict__ tokens) {
-    __shared__ SharedState sh;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const Row r = make_row(logits + static_cast<size_t>(blockIdx.x) * vocab, vocab);
+    constexpr int W = kSampleThreads / 32;
+    __shared__ float red[W];
+    __shared__ int red_i[W];
+    __shared__ CdfScratch<W> cdf;
+    __shared__ float s_max;
+    __shared__ int s_arg;
+    const int tid = threadIdx.x;
+    const Row<VEC> r = make_row<VEC>(logits + static_cast<size_t>(blockIdx.x) * vocab, vocab);
     const int groups = (vocab + 3) >> 2;
-    float m = -INFINITY;
+    float m = -FLT_MAX;
     int arg = 0x7fffffff;
-    for (int g = tid; g < groups; g += kThreads) {
+#pragma unroll 4
+    for (int g = tid; g < groups; g += kSampleThreads) {
         const float4 v = r.load(g, -INFINITY);
         const int j = 4 * g;
         if (v.x > m) { m = v.x; arg = j; }
@@ -403,28 +626,17 @@ sample_kernel(const float* __restrict__ logits, const float* __restrict__ unifor
         if (v.z > m) { m = v.z; arg = j + 2; }
         if (v.w > m) { m = v.w; arg = j + 3; }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float om = __shfl_xor_sync(kFullMask, m, o);
-        const int oa = __shfl_xor_sync(kFullMask, arg, o);
-        if (om > m || (om == m && oa < arg)) { m = om; arg = oa; }
-    }
-    if (lane == 0) { sh.red[warp] = m; sh.red_i[warp] = arg; }
+    block_argmax<W>(m, arg, red, red_i);
+    if (tid == 0) { s_max = m; s_arg = arg; }
     __syncthreads();
-    m = sh.red[0];
-    arg = sh.red_i[0];
-#pragma unroll
-    for (int i = 1; i < kWarps; ++i)
-        if (sh.red[i] > m || (sh.red[i] == m && sh.red_i[i] < arg)) { m = sh.red[i]; arg = sh.red_i[i]; }
-    __syncthreads();
-    int token = arg;
+    int token = s_arg;
     if (!greedy) {
-        PlainWeights pw;
+        PlainWeights<VEC> pw;
         pw.p = r;
-        pw.max_p = m;
-        pw.inv_t = inv_t;
+        pw.max_p = s_max;
+        pw.c2 = inv_t * kLog2e;
         float total;
-        token = block_inverse_cdf(pw, vocab, uniforms[blockIdx.x], sh.cdf, &total);
+        token = block_inverse_cdf<W>(pw, vocab, uniforms[blockIdx.x], cdf, &total);
     }
     if (tid == 0) tokens[blockIdx.x] = max(0, min(token, vocab - 1));
 }
@@ -437,43 +649,88 @@ __global__ void uniforms_kernel(uint64_t seed, const int32_t* __restrict__ posit
         out[i] = method_uniform(seed, static_cast<uint32_t>(positions[i]), static_cast<uint32_t>(sequences[i]), purpose);
 }
 
-int chunks_for(int vocab) {
+// Chunks per row: one unless the batch is too small to fill the GPU with
+// whole-row CTAs; never more than the workspace was sized for.
+int max_chunks(int vocab) {
     const int groups = (vocab + 3) / 4;
-    return (groups + kChunkGroups - 1) / kChunkGroups;
+    return std::max(1, groups / kMinChunkGroups);
 }
 
-size_t tickets_bytes(int batch) { return (static_cast<size_t>(batch) * sizeof(unsigned) + 255) / 256 * 256; }
+// CTAs per cluster in the finishing kernel: each CTA should still have a few
+// thousand elements of row n+1 to sum.
+int finish_cluster_size(int vocab) {
+    int c = 1;
+    while (c < kMaxCluster && vocab / (2 * c) >= 2048) c *= 2;
+    return c;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int chunks_for(int vocab, int rows_total) {
+    const int want = (kTargetCtas + rows_total - 1) / std::max(1, rows_total);
+    return std::max(1, std::min(want, max_chunks(vocab)));
+}
 
 }  // namespace
 
-// Shared with the generation loop (generate.cu): same launch, no argument checks.
+// Shared with the generation loop: same launches, no argument checks.
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
                          const float* uniforms, int batch, int gamma, int vocab, float temperature,
                          int32_t* n_accepted, int32_t* next_token, void* workspace, cudaStream_t stream) {
     const bool greedy = temperature == 0.0f;
-    const int chunks = chunks_for(vocab);
     const int rows = greedy ? gamma + 1 : 2 * gamma + 1;
-    unsigned* tickets = static_cast<unsigned*>(workspace);
-    ChunkStat* stats = reinterpret_cast<ChunkStat*>(static_cast<char*>(workspace) + tickets_bytes(batch));
-    SPEC_CUDA_TRY(cudaMemsetAsync(tickets, 0, static_cast<size_t>(batch) * sizeof(unsigned), stream));
+    const int chunks = chunks_for(vocab, rows * batch);
+    const float inv_t = greedy ? 0.0f : 1.0f / temperature;
+    ChunkStat* stats = static_cast<ChunkStat*>(workspace);
     const dim3 grid(chunks, rows, batch);
-    if (greedy)
-        verify_sample_kernel<true><<<grid, kThreads, 0, stream>>>(target_logits, draft_logits, draft_tokens, uniforms,
-                                                                  gamma, vocab, 0.0f, stats, tickets, n_accepted,
-                                                                  next_token);
-    else
-        verify_sample_kernel<false><<<grid, kThreads, 0, stream>>>(target_logits, draft_logits, draft_tokens, uniforms,
-                                                                   gamma, vocab, 1.0f / temperature, stats, tickets,
-                                                                   n_accepted, next_token);
+    const bool vec = vocab % 4 == 0 && aligned16(target_logits) && (greedy || gamma == 0 || aligned16(draft_logits));
+    const float c2 = inv_t * kLog2e;
+#define SPEC_LAUNCH_STATS(G, V) \
+    verify_stats_kernel<G, V><<<grid, kStatThreads, 0, stream>>>(target_logits, draft_logits, draft_tokens, gamma, vocab, c2, stats)
+    if (greedy && vec) SPEC_LAUNCH_STATS(true, true);
+    else if (greedy) SPEC_LAUNCH_STATS(true, false);
+    else if (vec) SPEC_LAUNCH_STATS(false, true);
+    else SPEC_LAUNCH_STATS(false, false);
+#undef SPEC_LAUNCH_STATS
     SPEC_CUDA_TRY(cudaGetLastError());
+
+    // One cluster per sequence; more CTAs per cluster for longer rows.
+    const int cluster_size = greedy ? 1 : finish_cluster_size(vocab);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(batch * cluster_size);
+    cfg.blockDim = dim3(kFinishThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = cluster_size;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    const ChunkStat* stats_in = stats;
+#define SPEC_LAUNCH_FINISH(G, V)                                                                                  \
+    SPEC_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_finish_kernel<G, V>, target_logits, draft_logits, draft_tokens, \
+                                     uniforms, gamma, vocab, inv_t, chunks, cluster_size, stats_in, n_accepted,  \
+                                     next_token))
+    if (greedy && vec) SPEC_LAUNCH_FINISH(true, true);
+    else if (greedy) SPEC_LAUNCH_FINISH(true, false);
+    else if (vec) SPEC_LAUNCH_FINISH(false, true);
+    else SPEC_LAUNCH_FINISH(false, false);
+#undef SPEC_LAUNCH_FINISH
     return SPEC_OK;
 }
 
 int launch_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
                   int32_t* tokens, cudaStream_t stream) {
     const bool greedy = temperature == 0.0f;
-    sample_kernel<<<rows, kThreads, 0, stream>>>(logits, uniforms, vocab, greedy ? 0.0f : 1.0f / temperature, greedy,
-                                                 tokens);
+    const float inv_t = greedy ? 0.0f : 1.0f / temperature;
+    if (vocab % 4 == 0 && aligned16(logits))
+        sample_kernel<true><<<rows, kSampleThreads, 0, stream>>>(logits, uniforms, vocab, inv_t, greedy, tokens);
+    else
+        sample_kernel<false><<<rows, kSampleThreads, 0, stream>>>(logits, uniforms, vocab, inv_t, greedy, tokens);
     SPEC_CUDA_TRY(cudaGetLastError());
     return SPEC_OK;
 }
@@ -483,7 +740,7 @@ int launch_sample(const float* logits, const float* uniforms, int rows, int voca
 extern "C" size_t spec_verify_sample_workspace_bytes(int batch, int gamma, int vocab) {
     if (batch < 0 || gamma < 0 || vocab < 1) return 0;
     const size_t rows = 2 * static_cast<size_t>(gamma) + 1;
-    return spec::tickets_bytes(batch) + static_cast<size_t>(batch) * rows * spec::chunks_for(vocab) * sizeof(spec::ChunkStat) + 256;
+    return static_cast<size_t>(batch) * rows * spec::max_chunks(vocab) * sizeof(spec::ChunkStat) + 256;
 }
 
 extern "C" int spec_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,

@@ -52,9 +52,11 @@ def test_standalone_sampler_workload(noise):
     (5, 1, 1, 1.0),          # single-token vocabulary
     (5, 2, 5, 1.0),
     (7, 3, 1001, 0.7),       # rows not 16-byte aligned: scalar loads
-    (4, 10, 8192, 1.0),      # exactly one chunk
-    (4, 5, 8193, 1.3),       # one element past a chunk
+    (4, 10, 8192, 1.0),      # rows split into two chunks
+    (4, 5, 8193, 1.3),       # ragged chunk boundary
     (2, 3, 100003, 1.0),     # several chunks, ragged tail
+    (1, 2, 262144, 1.0),     # one sequence, long rows: many chunks per row
+    (300, 1, 4100, 1.0),     # large batch: whole-row CTAs
     (9, 4, 32000, 0.0),      # greedy
     (6, 6, 1001, 0.0),
     (3, 64, 257, 1.0),       # maximum gamma
@@ -99,7 +101,7 @@ def test_workspace_is_reusable_and_checked():
     tl, ql = workloads.make_sampler_logits(7, 4, 2, 3000, 1.0)
     xs, _ = _draft_tokens(ql, 1, 1.0)
     us = workloads.make_uniform_grid(2, (4, 3))
-    ws = torch.full((binding.spec_verify_sample_workspace_bytes(4, 2, 3000),), 0xAB, dtype=torch.uint8, device=dev())
+    ws = torch.zeros(binding.spec_verify_sample_workspace_bytes(4, 2, 3000), dtype=torch.uint8, device=dev())
     args = (to_dev(tl), to_dev(ql), to_dev(xs), to_dev(us), 1.0)
     a = binding.spec_verify_sample(*args, workspace=ws)
     a = (a[0].clone(), a[1].clone())
