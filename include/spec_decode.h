@@ -115,6 +115,141 @@ int spec_sample(const float* logits, const float* uniforms, int rows, int vocab,
 int spec_uniforms(uint64_t seed, const int32_t* positions, const int32_t* sequences,
                   int purpose, int count, float* out, void* stream);
 
+/* ------------------------------------------------------------------------- *
+ * Models.  The paper treats M_p and M_q as black boxes that map a prefix to a
+ * next-token distribution (Section 2.1) and fixes only their sizes (Section 4:
+ * GPT-like decoders, T5).  This library runs decoder-only Transformers:
+ * pre-RMSNorm blocks, no biases, causal attention scaled by 1/sqrt(d_head),
+ * n_heads query heads over n_kv_heads key/value heads.
+ *   SPEC_ARCH_GPT:   token + learned position embeddings, FFN per `ffn`.
+ *   SPEC_ARCH_LLAMA: rotary positions (rotate-half pairing j, j + d_head/2,
+ *                    angle position * rope_base^(-2j/d_head)) on q and k.
+ *   FFN: SPEC_FFN_GELU (tanh approximation) with W_in [d_ff, d_model];
+ *        SPEC_FFN_GATED_GELU / SPEC_FFN_SWIGLU with W_in [2*d_ff, d_model],
+ *        rows 0..d_ff-1 the gate, rows d_ff..2*d_ff-1 the up projection.
+ * Matrices are row-major [out_features, in_features] in `dtype` (fp32, or
+ * bf16 as raw 16-bit patterns); gains are fp32.  The residual stream, softmax,
+ * normalisation and logits are fp32 in every configuration.
+ * ------------------------------------------------------------------------- */
+enum { SPEC_ARCH_GPT = 0, SPEC_ARCH_LLAMA = 1 };
+enum { SPEC_FFN_GELU = 0, SPEC_FFN_GATED_GELU = 1, SPEC_FFN_SWIGLU = 2 };
+enum { SPEC_DTYPE_FP32 = 0, SPEC_DTYPE_BF16 = 1 };
+
+typedef struct spec_model_cfg {
+    int arch;             /* SPEC_ARCH_* */
+    int n_layers;
+    int d_model;
+    int n_heads;
+    int n_kv_heads;       /* divides n_heads */
+    int d_head;           /* 64 or 128 */
+    int d_ff;
+    int ffn;              /* SPEC_FFN_* */
+    int vocab;
+    int max_positions;    /* rows of pos_emb (GPT); upper bound on positions */
+    int tied_embeddings;  /* 1: the LM head is tok_emb */
+    int dtype;            /* SPEC_DTYPE_* of every matrix */
+    float rms_eps;
+    float rope_base;
+} spec_model_cfg;
+
+typedef struct spec_layer_weights {
+    const float* ln1;     /* [d_model] */
+    const void* wqkv;     /* [(n_heads + 2 n_kv_heads) d_head, d_model]: q rows, k rows, v rows */
+    const void* wo;       /* [d_model, n_heads d_head] */
+    const float* ln2;     /* [d_model] */
+    const void* w_in;     /* [d_ff or 2 d_ff, d_model] */
+    const void* w_out;    /* [d_model, d_ff] */
+} spec_layer_weights;
+
+/* All pointers are DEVICE pointers that the caller keeps alive until
+ * spec_free(); `layers` itself is a HOST array of n_layers entries that is
+ * copied during spec_init. */
+typedef struct spec_weights {
+    const void* tok_emb;  /* [vocab, d_model] */
+    const void* pos_emb;  /* [max_positions, d_model], GPT only */
+    const float* ln_f;    /* [d_model] */
+    const void* head;     /* [vocab, d_model]; ignored when tied_embeddings */
+    const spec_layer_weights* layers;
+} spec_weights;
+
+typedef struct spec_runtime_cfg {
+    int max_batch;        /* sequences decoded together */
+    int max_len;          /* tokens per sequence the KV caches can hold (prompt + new + gamma) */
+    int page_size;        /* tokens per KV page (power of two, 16..256) */
+    int max_gamma;        /* largest gamma spec_generate will be asked for */
+    int kv_dtype;         /* SPEC_DTYPE_FP32 or SPEC_DTYPE_BF16: element type of the cached K,V rows.
+                             bf16 halves the KV traffic but rounds every cached row to 8 mantissa
+                             bits, which on deep models moves logits by more than 2e-2. */
+} spec_runtime_cfg;
+
+typedef struct spec_ctx spec_ctx;
+
+/* Counters of one spec_generate call (Section 3: what alpha, E[#tokens] and the
+ * walltime analysis are computed from). */
+typedef struct spec_stats {
+    int64_t iterations;       /* runs of Algorithm 1, summed over sequences */
+    int64_t tokens;           /* tokens emitted by those runs (before truncation to n_new) */
+    int64_t tests_evaluated;  /* accept tests that were reached (i <= n + 1) */
+    int64_t tests_passed;     /* drafted tokens accepted */
+    int64_t target_passes;    /* batched forward passes of M_p inside the decode loop */
+    int64_t draft_passes;     /* batched forward passes of M_q inside the decode loop */
+    double prefill_ms;        /* device time of the prompt pass */
+    double decode_ms;         /* device time of the decode loop */
+} spec_stats;
+
+/* Creates a context for a target model and (optionally, draft_cfg == NULL for
+ * target-only decoding) a draft model with the same vocabulary.  Allocates the
+ * paged KV caches, activations and logits buffers with cudaMalloc on the
+ * current device and creates a private stream; weights are borrowed.
+ * Errors: SPEC_ERR_BAD_ARG (null), SPEC_ERR_BAD_CONFIG (unsupported shapes,
+ * vocabularies differ), SPEC_ERR_OOM, SPEC_ERR_CUDA. */
+int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg* draft_cfg,
+              const spec_weights* target_weights, const spec_weights* draft_weights,
+              const spec_runtime_cfg* runtime, spec_ctx** out);
+
+/* Releases everything spec_init allocated (not the weights). NULL is allowed. */
+void spec_free(spec_ctx* ctx);
+
+/* Generation by speculative decoding (Algorithm 1 repeated): for each of
+ * `batch` sequences, emits exactly n_new tokens after its prompt.
+ *   prompt      HOST int32 [batch, prompt_stride]; sequence b uses the first
+ *               prompt_len[b] >= 1 entries of its row
+ *   prompt_len  HOST int32 [batch]
+ *   gamma       drafted tokens per iteration; 0 = plain autoregressive
+ *               decoding from the target alone with the same kernels
+ *   temperature 0 = greedy (argmax, lowest index on ties)
+ *   seed        key of the counter-based generator (see spec_uniforms): the
+ *               draft's draw of the token at position s uses purpose 0, its
+ *               accept test purpose 1, the final draw of an iteration purpose
+ *               2, each with counter (s, sequence index)
+ *   out_tokens  HOST int32 [batch, n_new]
+ *   stats       HOST, may be NULL
+ * Both models first consume the prompt; then each iteration runs the draft
+ * gamma times (one row per sequence; two in the first step, which re-feeds
+ * the previous token so that the draft catches up after an iteration that
+ * accepted every guess), the target once over gamma+1 rows per sequence, the
+ * speculative-sampling rule, and the roll-back of both caches to the accepted
+ * length.  The last iteration's surplus tokens are dropped.  The call blocks
+ * until the tokens are on the host.
+ * Errors: SPEC_ERR_BAD_ARG; SPEC_ERR_CAPACITY if prompt_len + n_new + gamma + 1
+ * exceeds max_len or a model's max_positions, batch > max_batch or
+ * gamma > max_gamma; SPEC_ERR_BAD_CONFIG if gamma > 0 without a draft model. */
+int spec_generate(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride,
+                  int batch, int n_new, int gamma, float temperature, uint64_t seed,
+                  int32_t* out_tokens, spec_stats* stats);
+
+/* Diagnostics for parity tests: teacher-forced forward passes on the KV caches.
+ * spec_reset forgets every cached row.  spec_forward_logits feeds, for each
+ * of `batch` sequences, `rows` tokens at positions cached_len[b].. of model
+ * `which` (0 target, 1 draft), appends their K,V rows and writes fp32 logits
+ * [batch, rows, vocab] to the DEVICE buffer `logits`; tokens is HOST int32
+ * [batch, rows].  spec_truncate sets the cached length of every sequence of
+ * the model (HOST int32 [batch]); later passes overwrite the dropped rows.
+ * All three synchronise. */
+int spec_reset(spec_ctx* ctx);
+int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* tokens, int batch, int rows, float* logits);
+int spec_truncate(spec_ctx* ctx, int which, const int32_t* lengths, int batch);
+
 #ifdef __cplusplus
 }
 #endif

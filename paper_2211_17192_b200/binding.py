@@ -144,3 +144,164 @@ def spec_uniforms(seed, positions, sequences, purpose, out=None):
                                _ptr(sequences, torch.int32, "sequences"), int(purpose), count,
                                _ptr(out, torch.float32, "out"), _stream()))
     return out
+
+
+# --------------------------------------------------------------------------- #
+# models and generation
+# --------------------------------------------------------------------------- #
+class _ModelCfg(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("arch", "n_layers", "d_model", "n_heads", "n_kv_heads", "d_head", "d_ff",
+                                            "ffn", "vocab", "max_positions", "tied_embeddings", "dtype")] + \
+               [("rms_eps", ctypes.c_float), ("rope_base", ctypes.c_float)]
+
+
+class _LayerWeights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("ln1", "wqkv", "wo", "ln2", "w_in", "w_out")]
+
+
+class _Weights(ctypes.Structure):
+    _fields_ = [("tok_emb", ctypes.c_void_p), ("pos_emb", ctypes.c_void_p), ("ln_f", ctypes.c_void_p),
+                ("head", ctypes.c_void_p), ("layers", ctypes.POINTER(_LayerWeights))]
+
+
+class _RuntimeCfg(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("max_batch", "max_len", "page_size", "max_gamma", "kv_dtype")]
+
+
+class _Stats(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in ("iterations", "tokens", "tests_evaluated", "tests_passed",
+                                              "target_passes", "draft_passes")] + \
+               [("prefill_ms", ctypes.c_double), ("decode_ms", ctypes.c_double)]
+
+
+_ARCH = {"gpt": 0, "llama": 1}
+_FFN = {"gelu": 0, "gated_gelu": 1, "swiglu": 2}
+_DTYPE = {"fp32": 0, "bf16": 1}
+_engine_declared = False
+
+
+def _declare_engine(h):
+    global _engine_declared
+    if _engine_declared:
+        return
+    c = ctypes
+    vp = c.c_void_p
+    h.spec_init.restype = c.c_int
+    h.spec_init.argtypes = [c.POINTER(_ModelCfg), c.POINTER(_ModelCfg), c.POINTER(_Weights), c.POINTER(_Weights),
+                            c.POINTER(_RuntimeCfg), c.POINTER(vp)]
+    h.spec_free.restype = None
+    h.spec_free.argtypes = [vp]
+    h.spec_generate.restype = c.c_int
+    h.spec_generate.argtypes = [vp, vp, vp, c.c_int, c.c_int, c.c_int, c.c_int, c.c_float, c.c_uint64, vp,
+                                c.POINTER(_Stats)]
+    h.spec_reset.restype = c.c_int
+    h.spec_reset.argtypes = [vp]
+    h.spec_truncate.restype = c.c_int
+    h.spec_truncate.argtypes = [vp, c.c_int, vp, c.c_int]
+    h.spec_forward_logits.restype = c.c_int
+    h.spec_forward_logits.argtypes = [vp, c.c_int, vp, c.c_int, c.c_int, vp]
+    _engine_declared = True
+
+
+def _cfg_struct(cfg):
+    return _ModelCfg(_ARCH[cfg["arch"]], cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["n_kv_heads"],
+                     cfg["d_head"], cfg["d_ff"], _FFN[cfg["ffn"]], cfg["vocab"], cfg["max_positions"],
+                     1 if cfg["tied"] else 0, _DTYPE[cfg["dtype"]], cfg["rms_eps"], cfg["rope_base"])
+
+
+class Engine:
+    """A target model, an optional draft model and their KV caches on one GPU.
+
+    `*_cfg` are the dicts of `workloads.model_config`, `*_weights` dicts of
+    arrays (numpy or CUDA tensors) by the names of `workloads.tensor_shapes`.
+    Weights are uploaded once (bf16 models as bf16) and kept alive here; the
+    library borrows the pointers.
+    """
+
+    def __init__(self, target_cfg, target_weights, draft_cfg=None, draft_weights=None, max_batch=1, max_len=256,
+                 page_size=64, max_gamma=8, kv_dtype="fp32", device=None):
+        import numpy as np
+        self._np = np
+        h = lib()
+        _declare_engine(h)
+        self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+        self.cfgs = [target_cfg, draft_cfg]
+        self._keep = []
+        structs = []
+        for cfg, weights in ((target_cfg, target_weights), (draft_cfg, draft_weights)):
+            structs.append(None if cfg is None else self._upload(cfg, weights))
+        rt = _RuntimeCfg(max_batch, max_len, page_size, max_gamma, _DTYPE[kv_dtype])
+        self.max_batch, self.max_len, self.max_gamma = max_batch, max_len, max_gamma
+        ctx = ctypes.c_void_p()
+        tc = _cfg_struct(target_cfg)
+        dc = _cfg_struct(draft_cfg) if draft_cfg is not None else None
+        _check(h.spec_init(ctypes.byref(tc), ctypes.byref(dc) if dc is not None else None,
+                           ctypes.byref(structs[0]), ctypes.byref(structs[1]) if structs[1] is not None else None,
+                           ctypes.byref(rt), ctypes.byref(ctx)))
+        self._ctx = ctx
+
+    def _upload(self, cfg, weights):
+        bf16 = cfg["dtype"] == "bf16"
+
+        def dev(name, matrix):
+            a = weights[name]
+            t = a if isinstance(a, torch.Tensor) else torch.from_numpy(self._np.ascontiguousarray(a))
+            t = t.to(self.device)
+            t = t.to(torch.bfloat16 if (bf16 and matrix) else torch.float32).contiguous()
+            self._keep.append(t)
+            return t.data_ptr()
+
+        layers = (_LayerWeights * cfg["n_layers"])()
+        for l in range(cfg["n_layers"]):
+            layers[l] = _LayerWeights(dev(f"l{l}.ln1", False), dev(f"l{l}.wqkv", True), dev(f"l{l}.wo", True),
+                                      dev(f"l{l}.ln2", False), dev(f"l{l}.w_in", True), dev(f"l{l}.w_out", True))
+        self._keep.append(layers)
+        return _Weights(dev("tok_emb", True), dev("pos_emb", True) if cfg["arch"] == "gpt" else None,
+                        dev("ln_f", False), None if cfg["tied"] else dev("head", True), layers)
+
+    def close(self):
+        if getattr(self, "_ctx", None):
+            lib().spec_free(self._ctx)
+            self._ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def generate(self, prompts, n_new, gamma, temperature, seed):
+        """Speculative decoding (gamma = 0: target-only decoding).  `prompts` is a
+        list of 1-D int arrays; returns (tokens [B, n_new] int32 numpy, stats dict)."""
+        np = self._np
+        batch = len(prompts)
+        stride = max(len(p) for p in prompts)
+        flat = np.zeros((batch, stride), dtype=np.int32)
+        lens = np.zeros(batch, dtype=np.int32)
+        for b, p in enumerate(prompts):
+            flat[b, : len(p)] = p
+            lens[b] = len(p)
+        out = np.zeros((batch, n_new), dtype=np.int32)
+        st = _Stats()
+        _check(lib().spec_generate(self._ctx, flat.ctypes.data, lens.ctypes.data, stride, batch, n_new, gamma,
+                                   float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF, out.ctypes.data,
+                                   ctypes.byref(st)))
+        return out, {name: getattr(st, name) for name, _ in _Stats._fields_}
+
+    def reset(self):
+        _check(lib().spec_reset(self._ctx))
+
+    def truncate(self, which, lengths):
+        a = self._np.ascontiguousarray(lengths, dtype=self._np.int32)
+        _check(lib().spec_truncate(self._ctx, which, a.ctypes.data, a.shape[0]))
+
+    def forward_logits(self, which, tokens):
+        """Teacher-forced pass: tokens [B, rows] are appended at the cached
+        lengths of model `which` (0 target, 1 draft); returns fp32 logits
+        [B, rows, vocab] as a CUDA tensor."""
+        a = self._np.ascontiguousarray(tokens, dtype=self._np.int32)
+        batch, rows = a.shape
+        vocab = self.cfgs[which]["vocab"]
+        out = torch.empty((batch, rows, vocab), dtype=torch.float32, device=self.device)
+        _check(lib().spec_forward_logits(self._ctx, which, a.ctypes.data, batch, rows, out.data_ptr()))
+        return out

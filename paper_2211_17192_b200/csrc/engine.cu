@@ -1,0 +1,561 @@
+// Decoder engine: context set-up, the forward pass over a set of rows, the
+// device-resident generation loop of Algorithm 1 (draft steps, parallel
+// verification, speculative sampling, commit + roll-back) replayed as a CUDA
+// graph, and the teacher-forced diagnostics used by the parity tests.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "model.cuh"
+
+struct spec_ctx {
+    spec::Model model[2];  // 0 target, 1 draft
+    bool has_draft = false;
+    spec_runtime_cfg rt{};
+    cudaStream_t stream = nullptr;
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+    int max_rows = 0;
+    int pages_per_seq = 0;
+
+    // activations (sized for the wider model)
+    float *h = nullptr, *a = nullptr, *qkv = nullptr, *att = nullptr, *u = nullptr, *f = nullptr;
+    float *target_logits = nullptr, *draft_logits = nullptr;
+    int32_t *row_token = nullptr, *row_pos = nullptr, *row_seq = nullptr, *logit_src = nullptr, *logit_dst = nullptr;
+    int32_t* page_table = nullptr;
+
+    // generation state (device)
+    int32_t *tokens = nullptr, *length = nullptr, *prompt_len = nullptr, *draft_tokens = nullptr;
+    int32_t *n_accepted = nullptr, *next_token = nullptr;
+    float *draft_u = nullptr, *accept_u = nullptr, *final_u = nullptr;
+    unsigned long long* counters = nullptr;  // iterations, tokens, tests evaluated, tests passed
+    void* sampler_ws = nullptr;
+    struct Params { unsigned long long seed; int n_new; int pad; }* params = nullptr;
+
+    // cached iteration graph
+    cudaGraphExec_t graph = nullptr;
+    int graph_batch = -1, graph_gamma = -1;
+    float graph_temperature = -1.0f;
+
+    // host-side cached lengths for the diagnostics
+    std::vector<int32_t> cached[2];
+    std::vector<void*> allocations;
+};
+
+namespace spec {
+namespace {
+
+int check_cfg(const spec_model_cfg& c, const char* which) {
+    if (c.arch != SPEC_ARCH_GPT && c.arch != SPEC_ARCH_LLAMA) return fail(SPEC_ERR_BAD_CONFIG, "%s: unknown arch %d", which, c.arch);
+    if (c.n_layers < 1 || c.d_model < 8 || c.n_heads < 1 || c.n_kv_heads < 1 || c.d_ff < 8 || c.vocab < 1 || c.max_positions < 1)
+        return fail(SPEC_ERR_BAD_CONFIG, "%s: non-positive dimension", which);
+    if (c.d_head != 64 && c.d_head != 128) return fail(SPEC_ERR_BAD_CONFIG, "%s: d_head %d (64 or 128 supported)", which, c.d_head);
+    if (c.n_heads % c.n_kv_heads) return fail(SPEC_ERR_BAD_CONFIG, "%s: n_kv_heads must divide n_heads", which);
+    if (c.d_model % 8 || c.d_ff % 8) return fail(SPEC_ERR_BAD_CONFIG, "%s: d_model and d_ff must be multiples of 8", which);
+    if (c.ffn < SPEC_FFN_GELU || c.ffn > SPEC_FFN_SWIGLU) return fail(SPEC_ERR_BAD_CONFIG, "%s: unknown ffn %d", which, c.ffn);
+    if (c.dtype != SPEC_DTYPE_FP32 && c.dtype != SPEC_DTYPE_BF16) return fail(SPEC_ERR_BAD_CONFIG, "%s: unknown dtype %d", which, c.dtype);
+    if (!(c.rms_eps >= 0.0f)) return fail(SPEC_ERR_BAD_CONFIG, "%s: rms_eps", which);
+    return SPEC_OK;
+}
+
+template <typename T>
+int dev_alloc(spec_ctx* ctx, T** out, size_t count) {
+    void* p = nullptr;
+    const cudaError_t err = cudaMalloc(&p, std::max<size_t>(count, 1) * sizeof(T));
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return fail(SPEC_ERR_OOM, "cudaMalloc of %zu bytes failed: %s", count * sizeof(T), cudaGetErrorString(err));
+    }
+    ctx->allocations.push_back(p);
+    *out = static_cast<T*>(p);
+    return SPEC_OK;
+}
+
+#define SPEC_TRY(expr)                    \
+    do {                                  \
+        const int status__ = (expr);      \
+        if (status__ != SPEC_OK) return status__; \
+    } while (0)
+
+// One forward pass of `m` over the rows described by ctx->row_*; K,V rows of
+// active rows are appended to the cache.  If n_logit_rows > 0 the final norm and
+// LM head run on rows logit_src[i] and write logits rows logit_dst[i].
+int forward(spec_ctx* ctx, const Model& m, int n_rows, int n_logit_rows, const int32_t* logit_src,
+            const int32_t* logit_dst, float* logits) {
+    cudaStream_t st = ctx->stream;
+    const spec_model_cfg& c = m.cfg;
+    const RowMeta rows{ctx->row_token, ctx->row_pos, ctx->row_seq};
+    const bool bf = m.bf16();
+    SPEC_TRY(launch_embed(m, rows, n_rows, ctx->h, st));
+    for (int l = 0; l < c.n_layers; ++l) {
+        const spec_layer_weights& w = m.layers[l];
+        SPEC_TRY(launch_rmsnorm(ctx->h, w.ln1, nullptr, n_rows, c.d_model, c.rms_eps, ctx->a, st));
+        SPEC_TRY(launch_gemm_rows(ctx->a, w.wqkv, bf, nullptr, nullptr, n_rows, m.qkv_dim(), c.d_model, ctx->qkv, st));
+        SPEC_TRY(launch_rope_append(m, l, rows, n_rows, ctx->qkv, ctx->page_table, ctx->pages_per_seq, ctx->rt.page_size, st));
+        SPEC_TRY(launch_attention(m, l, rows, n_rows, ctx->qkv, ctx->att, ctx->page_table, ctx->pages_per_seq, ctx->rt.page_size, st));
+        SPEC_TRY(launch_gemm_rows(ctx->att, w.wo, bf, ctx->h, nullptr, n_rows, c.d_model, m.q_dim(), ctx->h, st));
+        SPEC_TRY(launch_rmsnorm(ctx->h, w.ln2, nullptr, n_rows, c.d_model, c.rms_eps, ctx->a, st));
+        SPEC_TRY(launch_gemm_rows(ctx->a, w.w_in, bf, nullptr, nullptr, n_rows, m.ffn_in_dim(), c.d_model, ctx->u, st));
+        SPEC_TRY(launch_ffn_act(ctx->u, n_rows, c.d_ff, c.ffn, ctx->f, st));
+        SPEC_TRY(launch_gemm_rows(ctx->f, w.w_out, bf, ctx->h, nullptr, n_rows, c.d_model, c.d_ff, ctx->h, st));
+    }
+    if (n_logit_rows > 0) {
+        SPEC_TRY(launch_rmsnorm(ctx->h, m.ln_f, logit_src, n_logit_rows, c.d_model, c.rms_eps, ctx->a, st));
+        SPEC_TRY(launch_gemm_rows(ctx->a, m.head, bf, nullptr, logit_dst, n_logit_rows, c.vocab, c.d_model, logits, st));
+    }
+    return SPEC_OK;
+}
+
+// ---- generation-loop kernels (one thread per sequence; tiny) ----------------
+
+// Uniforms of one iteration (the paper leaves the consumption of randomness
+// open; here every draw is keyed by the position it decides):
+//   draft_u[b, i]  draw of x_{i+1} at position L+i           (purpose 0)
+//   accept_u[b, i] accept test of x_{i+1} at position L+i     (purpose 1)
+//   final_u[b, n]  final draw t at position L+n, n = 0..gamma (purpose 2)
+__global__ void iteration_uniforms_kernel(const spec_ctx::Params* __restrict__ params,
+                                          const int32_t* __restrict__ length, int batch, int gamma,
+                                          float* __restrict__ draft_u, float* __restrict__ accept_u,
+                                          float* __restrict__ final_u) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= batch * (gamma + 1)) return;
+    const int b = i / (gamma + 1), j = i % (gamma + 1);
+    const uint32_t pos = static_cast<uint32_t>(length[b] + j);
+    const unsigned long long seed = params->seed;
+    final_u[i] = method_uniform(seed, pos, b, kPurposeFinal);
+    accept_u[i] = method_uniform(seed, pos, b, kPurposeAccept);  // entry j = gamma is unused
+    if (j < gamma) draft_u[b * gamma + j] = method_uniform(seed, pos, b, kPurposeDraft);
+}
+
+// First draft step of an iteration: two rows per sequence, positions L-2 and
+// L-1.  Position L-2 is already cached unless the previous iteration accepted
+// every guess (x_gamma was never fed to the draft); feeding it again rewrites
+// the same K,V row, so the shape of the step never changes.
+__global__ void prep_draft_first_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ length,
+                                        int batch, int gamma, int max_len, int32_t* row_token, int32_t* row_pos,
+                                        int32_t* row_seq, int32_t* logit_src, int32_t* logit_dst) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch) return;
+    const int L = length[b];
+    const int p0 = max(L - 2, 0), p1 = L - 1;
+    row_token[2 * b] = tokens[static_cast<size_t>(b) * max_len + p0];
+    row_token[2 * b + 1] = tokens[static_cast<size_t>(b) * max_len + p1];
+    row_pos[2 * b] = p0;
+    row_pos[2 * b + 1] = p1;
+    row_seq[2 * b] = row_seq[2 * b + 1] = b;
+    logit_src[b] = 2 * b + 1;
+    logit_dst[b] = b * gamma;  // q_1
+}
+
+// Draft step i (2..gamma): one row per sequence, the previous guess x_{i-1} at position L+i-2.
+__global__ void prep_draft_step_kernel(const int32_t* __restrict__ draft_tokens, const int32_t* __restrict__ length,
+                                       int batch, int gamma, int step, int32_t* row_token, int32_t* row_pos,
+                                       int32_t* row_seq, int32_t* logit_src, int32_t* logit_dst) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch) return;
+    row_token[b] = draft_tokens[b * gamma + step - 2];
+    row_pos[b] = length[b] + step - 2;
+    row_seq[b] = b;
+    logit_src[b] = b;
+    logit_dst[b] = b * gamma + step - 1;
+}
+
+// The target's parallel pass: rows [last committed token, x_1..x_gamma] at positions L-1..L-1+gamma.
+__global__ void prep_verify_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ draft_tokens,
+                                   const int32_t* __restrict__ length, int batch, int gamma, int max_len,
+                                   int32_t* row_token, int32_t* row_pos, int32_t* row_seq) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= batch * (gamma + 1)) return;
+    const int b = i / (gamma + 1), j = i % (gamma + 1);
+    const int L = length[b];
+    row_token[i] = j == 0 ? tokens[static_cast<size_t>(b) * max_len + L - 1] : draft_tokens[b * gamma + j - 1];
+    row_pos[i] = L - 1 + j;
+    row_seq[i] = b;
+}
+
+// Commit x_1..x_n and t, advance L.  Rolling the caches back needs no data
+// movement: both caches are valid up to position L_new - 2 by construction and
+// whatever lies beyond is overwritten by the next iteration.  A sequence that
+// already has its n_new tokens is frozen.
+__global__ void commit_kernel(const spec_ctx::Params* __restrict__ params, const int32_t* __restrict__ draft_tokens,
+                              const int32_t* __restrict__ n_accepted, const int32_t* __restrict__ next_token,
+                              const int32_t* __restrict__ prompt_len, int batch, int gamma, int max_len,
+                              int32_t* tokens, int32_t* length, unsigned long long* counters) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch) return;
+    const int L = length[b];
+    if (L - prompt_len[b] >= params->n_new) return;
+    const int n = n_accepted[b];
+    int32_t* seq_tokens = tokens + static_cast<size_t>(b) * max_len;
+    for (int i = 0; i < n; ++i) seq_tokens[L + i] = draft_tokens[b * gamma + i];
+    seq_tokens[L + n] = next_token[b];
+    length[b] = L + n + 1;
+    atomicAdd(&counters[0], 1ull);
+    atomicAdd(&counters[1], static_cast<unsigned long long>(n + 1));
+    atomicAdd(&counters[2], static_cast<unsigned long long>(min(n + 1, gamma)));
+    atomicAdd(&counters[3], static_cast<unsigned long long>(n));
+}
+
+// Enqueues one iteration of Algorithm 1 for the whole batch on ctx->stream.
+int enqueue_iteration(spec_ctx* ctx, int batch, int gamma, float temperature) {
+    cudaStream_t st = ctx->stream;
+    const int vocab = ctx->model[0].cfg.vocab;
+    const int threads = 128;
+    const int blocks_b = (batch + threads - 1) / threads;
+    const int blocks_bg = (batch * (gamma + 1) + threads - 1) / threads;
+    iteration_uniforms_kernel<<<blocks_bg, threads, 0, st>>>(ctx->params, ctx->length, batch, gamma, ctx->draft_u,
+                                                             ctx->accept_u, ctx->final_u);
+    for (int step = 1; step <= gamma; ++step) {
+        int rows;
+        if (step == 1) {
+            prep_draft_first_kernel<<<blocks_b, threads, 0, st>>>(ctx->tokens, ctx->length, batch, gamma,
+                                                                  ctx->rt.max_len, ctx->row_token, ctx->row_pos,
+                                                                  ctx->row_seq, ctx->logit_src, ctx->logit_dst);
+            rows = 2 * batch;
+        } else {
+            prep_draft_step_kernel<<<blocks_b, threads, 0, st>>>(ctx->draft_tokens, ctx->length, batch, gamma, step,
+                                                                 ctx->row_token, ctx->row_pos, ctx->row_seq,
+                                                                 ctx->logit_src, ctx->logit_dst);
+            rows = batch;
+        }
+        SPEC_CUDA_TRY(cudaGetLastError());
+        SPEC_TRY(forward(ctx, ctx->model[1], rows, batch, ctx->logit_src, ctx->logit_dst, ctx->draft_logits));
+        // x_step ~ q_step for every sequence
+        SPEC_TRY(launch_sample_strided(ctx->draft_logits + static_cast<size_t>(step - 1) * vocab,
+                                       static_cast<size_t>(gamma) * vocab, ctx->draft_u + (step - 1), gamma, batch,
+                                       vocab, temperature, ctx->draft_tokens + (step - 1), gamma, st));
+    }
+    prep_verify_kernel<<<blocks_bg, threads, 0, st>>>(ctx->tokens, ctx->draft_tokens, ctx->length, batch, gamma,
+                                                      ctx->rt.max_len, ctx->row_token, ctx->row_pos, ctx->row_seq);
+    SPEC_CUDA_TRY(cudaGetLastError());
+    SPEC_TRY(forward(ctx, ctx->model[0], batch * (gamma + 1), batch * (gamma + 1), nullptr, nullptr, ctx->target_logits));
+    SPEC_TRY(launch_verify_sample(ctx->target_logits, ctx->draft_logits, ctx->draft_tokens, ctx->accept_u, ctx->final_u,
+                                  batch, gamma, vocab, temperature, ctx->n_accepted, ctx->next_token, ctx->sampler_ws, st));
+    commit_kernel<<<blocks_b, threads, 0, st>>>(ctx->params, ctx->draft_tokens, ctx->n_accepted, ctx->next_token,
+                                                ctx->prompt_len, batch, gamma, ctx->rt.max_len, ctx->tokens,
+                                                ctx->length, ctx->counters);
+    SPEC_CUDA_TRY(cudaGetLastError());
+    return SPEC_OK;
+}
+
+int build_graph(spec_ctx* ctx, int batch, int gamma, float temperature) {
+    if (ctx->graph && ctx->graph_batch == batch && ctx->graph_gamma == gamma && ctx->graph_temperature == temperature)
+        return SPEC_OK;
+    if (ctx->graph) {
+        cudaGraphExecDestroy(ctx->graph);
+        ctx->graph = nullptr;
+    }
+    SPEC_CUDA_TRY(cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
+    const int status = enqueue_iteration(ctx, batch, gamma, temperature);
+    cudaGraph_t g = nullptr;
+    const cudaError_t err = cudaStreamEndCapture(ctx->stream, &g);
+    if (status != SPEC_OK) {
+        if (g) cudaGraphDestroy(g);
+        return status;
+    }
+    SPEC_CUDA_TRY(err);
+    const cudaError_t ierr = cudaGraphInstantiate(&ctx->graph, g, 0);
+    cudaGraphDestroy(g);
+    SPEC_CUDA_TRY(ierr);
+    ctx->graph_batch = batch;
+    ctx->graph_gamma = gamma;
+    ctx->graph_temperature = temperature;
+    return SPEC_OK;
+}
+
+// Feeds, for every sequence, positions [from[b], to[b]) of host tokens through
+// model `which` in chunks (no logits): the prompt pass.
+int feed_host_tokens(spec_ctx* ctx, int which, const int32_t* tokens, int stride, const std::vector<int>& from,
+                     const std::vector<int>& to, int batch) {
+    const int chunk = std::max(1, ctx->max_rows / batch);
+    int longest = 0;
+    for (int b = 0; b < batch; ++b) longest = std::max(longest, to[b] - from[b]);
+    std::vector<int32_t> tok(static_cast<size_t>(batch) * chunk), pos(tok.size()), seq(tok.size());
+    for (int c0 = 0; c0 < longest; c0 += chunk) {
+        for (int b = 0; b < batch; ++b)
+            for (int j = 0; j < chunk; ++j) {
+                const int p = from[b] + c0 + j;
+                const size_t r = static_cast<size_t>(b) * chunk + j;
+                const bool active = p < to[b];
+                tok[r] = active ? tokens[static_cast<size_t>(b) * stride + p] : 0;
+                pos[r] = active ? p : -1;
+                seq[r] = b;
+            }
+        const size_t bytes = tok.size() * sizeof(int32_t);
+        SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_token, tok.data(), bytes, cudaMemcpyHostToDevice, ctx->stream));
+        SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_pos, pos.data(), bytes, cudaMemcpyHostToDevice, ctx->stream));
+        SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_seq, seq.data(), bytes, cudaMemcpyHostToDevice, ctx->stream));
+        SPEC_TRY(forward(ctx, ctx->model[which], batch * chunk, 0, nullptr, nullptr, nullptr));
+        SPEC_CUDA_TRY(cudaStreamSynchronize(ctx->stream));  // the host vectors are reused
+    }
+    return SPEC_OK;
+}
+
+int init_model(spec_ctx* ctx, int which, const spec_model_cfg& cfg, const spec_weights& w) {
+    Model& m = ctx->model[which];
+    m.cfg = cfg;
+    if (!w.tok_emb || !w.ln_f || !w.layers || (cfg.arch == SPEC_ARCH_GPT && !w.pos_emb) || (!cfg.tied_embeddings && !w.head))
+        return fail(SPEC_ERR_BAD_ARG, "spec_init: missing weight pointer");
+    m.tok_emb = w.tok_emb;
+    m.pos_emb = w.pos_emb;
+    m.ln_f = w.ln_f;
+    m.head = cfg.tied_embeddings ? w.tok_emb : w.head;
+    m.layers.assign(w.layers, w.layers + cfg.n_layers);
+    for (const spec_layer_weights& l : m.layers)
+        if (!l.ln1 || !l.wqkv || !l.wo || !l.ln2 || !l.w_in || !l.w_out)
+            return fail(SPEC_ERR_BAD_ARG, "spec_init: missing layer weight pointer");
+    m.kv_elem_bytes = ctx->rt.kv_dtype == SPEC_DTYPE_BF16 ? 2 : 4;
+    const size_t n_pages = static_cast<size_t>(ctx->rt.max_batch) * ctx->pages_per_seq;
+    m.layer_stride = n_pages * 2 * cfg.n_kv_heads * ctx->rt.page_size * cfg.d_head * m.kv_elem_bytes;
+    char* kv = nullptr;
+    SPEC_TRY(dev_alloc(ctx, &kv, m.layer_stride * cfg.n_layers));
+    m.kv = kv;
+    return SPEC_OK;
+}
+
+}  // namespace
+}  // namespace spec
+
+using namespace spec;
+
+extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg* draft_cfg,
+                         const spec_weights* target_weights, const spec_weights* draft_weights,
+                         const spec_runtime_cfg* runtime, spec_ctx** out) {
+    if (!target_cfg || !target_weights || !runtime || !out) return fail(SPEC_ERR_BAD_ARG, "spec_init: null pointer");
+    if (draft_cfg && !draft_weights) return fail(SPEC_ERR_BAD_ARG, "spec_init: draft config without weights");
+    *out = nullptr;
+    SPEC_TRY(check_cfg(*target_cfg, "target"));
+    if (draft_cfg) {
+        SPEC_TRY(check_cfg(*draft_cfg, "draft"));
+        if (draft_cfg->vocab != target_cfg->vocab) return fail(SPEC_ERR_BAD_CONFIG, "spec_init: vocabularies differ");
+    }
+    const spec_runtime_cfg& rt = *runtime;
+    if (rt.max_batch < 1 || rt.max_batch > 4096 || rt.max_len < 2 || rt.max_gamma < 0 || rt.max_gamma > 64 ||
+        rt.page_size < 16 || rt.page_size > 256 || (rt.page_size & (rt.page_size - 1)) ||
+        (rt.kv_dtype != SPEC_DTYPE_FP32 && rt.kv_dtype != SPEC_DTYPE_BF16))
+        return fail(SPEC_ERR_BAD_CONFIG, "spec_init: runtime config out of range");
+    int device_count = 0;
+    if (cudaGetDeviceCount(&device_count) != cudaSuccess || device_count == 0) {
+        cudaGetLastError();
+        return fail(SPEC_ERR_CUDA, "spec_init: no CUDA device (this library has no CPU path)");
+    }
+    spec_ctx* ctx = new (std::nothrow) spec_ctx();
+    if (!ctx) return fail(SPEC_ERR_OOM, "spec_init: host allocation failed");
+    ctx->rt = rt;
+    ctx->has_draft = draft_cfg != nullptr;
+    ctx->pages_per_seq = (rt.max_len + rt.page_size - 1) / rt.page_size;
+    ctx->max_rows = std::max(rt.max_batch * std::max(rt.max_gamma + 1, 2), 64);
+    auto cleanup = [&](int status) {
+        spec_free(ctx);
+        return status;
+    };
+    cudaError_t err = cudaStreamCreateWithFlags(&ctx->stream, cudaStreamNonBlocking);
+    if (err != cudaSuccess) return cleanup(fail(SPEC_ERR_CUDA, "cudaStreamCreate: %s", cudaGetErrorString(err)));
+    for (auto& e : ctx->ev)
+        if (cudaEventCreate(&e) != cudaSuccess) return cleanup(fail(SPEC_ERR_CUDA, "cudaEventCreate failed"));
+
+    int status = init_model(ctx, 0, *target_cfg, *target_weights);
+    if (status == SPEC_OK && draft_cfg) status = init_model(ctx, 1, *draft_cfg, *draft_weights);
+    if (status != SPEC_OK) return cleanup(status);
+
+    size_t d = 0, qkv = 0, att = 0, fin = 0, ff = 0;
+    for (int i = 0; i < (ctx->has_draft ? 2 : 1); ++i) {
+        const Model& m = ctx->model[i];
+        d = std::max<size_t>(d, m.cfg.d_model);
+        qkv = std::max<size_t>(qkv, m.qkv_dim());
+        att = std::max<size_t>(att, m.q_dim());
+        fin = std::max<size_t>(fin, m.ffn_in_dim());
+        ff = std::max<size_t>(ff, m.cfg.d_ff);
+    }
+    const size_t R = ctx->max_rows, B = rt.max_batch, G = rt.max_gamma, V = target_cfg->vocab;
+#define SPEC_ALLOC(ptr, count) \
+    if ((status = dev_alloc(ctx, &ctx->ptr, (count))) != SPEC_OK) return cleanup(status)
+    SPEC_ALLOC(h, R * d);
+    SPEC_ALLOC(a, R * d);
+    SPEC_ALLOC(qkv, R * qkv);
+    SPEC_ALLOC(att, R * att);
+    SPEC_ALLOC(u, R * fin);
+    SPEC_ALLOC(f, R * ff);
+    SPEC_ALLOC(target_logits, R * V);
+    SPEC_ALLOC(draft_logits, std::max<size_t>(B * G, 1) * V);
+    SPEC_ALLOC(row_token, R);
+    SPEC_ALLOC(row_pos, R);
+    SPEC_ALLOC(row_seq, R);
+    SPEC_ALLOC(logit_src, R);
+    SPEC_ALLOC(logit_dst, R);
+    SPEC_ALLOC(page_table, B * ctx->pages_per_seq);
+    SPEC_ALLOC(tokens, B * rt.max_len);
+    SPEC_ALLOC(length, B);
+    SPEC_ALLOC(prompt_len, B);
+    SPEC_ALLOC(draft_tokens, std::max<size_t>(B * G, 1));
+    SPEC_ALLOC(n_accepted, B);
+    SPEC_ALLOC(next_token, B);
+    SPEC_ALLOC(draft_u, std::max<size_t>(B * G, 1));
+    SPEC_ALLOC(accept_u, B * (G + 1));
+    SPEC_ALLOC(final_u, B * (G + 1));
+    SPEC_ALLOC(counters, 4);
+    SPEC_ALLOC(params, 1);
+    {
+        char* ws = nullptr;
+        if ((status = dev_alloc(ctx, &ws, verify_sample_workspace_bytes(static_cast<int>(B), static_cast<int>(G), static_cast<int>(V)))) != SPEC_OK)
+            return cleanup(status);
+        ctx->sampler_ws = ws;
+    }
+#undef SPEC_ALLOC
+    // Page j of sequence b is pool page j * max_batch + b: consecutive pages of a
+    // sequence are not adjacent in memory, so every access goes through the table.
+    std::vector<int32_t> table(B * ctx->pages_per_seq);
+    for (size_t b = 0; b < B; ++b)
+        for (int j = 0; j < ctx->pages_per_seq; ++j) table[b * ctx->pages_per_seq + j] = static_cast<int32_t>(j * B + b);
+    err = cudaMemcpy(ctx->page_table, table.data(), table.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+    if (err != cudaSuccess) return cleanup(fail(SPEC_ERR_CUDA, "page table upload: %s", cudaGetErrorString(err)));
+    ctx->cached[0].assign(B, 0);
+    ctx->cached[1].assign(B, 0);
+    *out = ctx;
+    return SPEC_OK;
+}
+
+extern "C" void spec_free(spec_ctx* ctx) {
+    if (!ctx) return;
+    if (ctx->stream) cudaStreamSynchronize(ctx->stream);
+    if (ctx->graph) cudaGraphExecDestroy(ctx->graph);
+    for (void* p : ctx->allocations) cudaFree(p);
+    for (auto& e : ctx->ev)
+        if (e) cudaEventDestroy(e);
+    if (ctx->stream) cudaStreamDestroy(ctx->stream);
+    delete ctx;
+}
+
+extern "C" int spec_generate(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride,
+                             int batch, int n_new, int gamma, float temperature, uint64_t seed, int32_t* out_tokens,
+                             spec_stats* stats) {
+    if (!ctx || !prompt || !prompt_len || !out_tokens) return fail(SPEC_ERR_BAD_ARG, "spec_generate: null pointer");
+    if (batch < 1 || n_new < 1 || gamma < 0 || prompt_stride < 1 || !(temperature >= 0.0f) || !std::isfinite(temperature))
+        return fail(SPEC_ERR_BAD_ARG, "spec_generate: batch=%d n_new=%d gamma=%d temperature=%g", batch, n_new, gamma, temperature);
+    if (batch > ctx->rt.max_batch || gamma > ctx->rt.max_gamma)
+        return fail(SPEC_ERR_CAPACITY, "spec_generate: batch %d / gamma %d exceed the context's limits (%d / %d)", batch, gamma, ctx->rt.max_batch, ctx->rt.max_gamma);
+    if (gamma > 0 && !ctx->has_draft) return fail(SPEC_ERR_BAD_CONFIG, "spec_generate: gamma > 0 needs a draft model");
+    int limit = std::min(ctx->rt.max_len, ctx->model[0].cfg.max_positions);
+    if (gamma > 0) limit = std::min(limit, ctx->model[1].cfg.max_positions);
+    for (int b = 0; b < batch; ++b) {
+        if (prompt_len[b] < 1 || prompt_len[b] > prompt_stride) return fail(SPEC_ERR_BAD_ARG, "spec_generate: prompt_len[%d]=%d", b, prompt_len[b]);
+        if (prompt_len[b] + n_new + gamma + 1 > limit)
+            return fail(SPEC_ERR_CAPACITY, "spec_generate: sequence %d needs %d positions, limit %d", b, prompt_len[b] + n_new + gamma + 1, limit);
+        for (int i = 0; i < prompt_len[b]; ++i) {
+            const int32_t t = prompt[static_cast<size_t>(b) * prompt_stride + i];
+            if (t < 0 || t >= ctx->model[0].cfg.vocab) return fail(SPEC_ERR_BAD_ARG, "spec_generate: token %d out of range", t);
+        }
+    }
+    cudaStream_t st = ctx->stream;
+    const int max_len = ctx->rt.max_len;
+
+    // upload prompts and state
+    std::vector<int32_t> host_tokens(static_cast<size_t>(batch) * max_len, 0);
+    for (int b = 0; b < batch; ++b)
+        std::memcpy(&host_tokens[static_cast<size_t>(b) * max_len], prompt + static_cast<size_t>(b) * prompt_stride, prompt_len[b] * sizeof(int32_t));
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->tokens, host_tokens.data(), host_tokens.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->length, prompt_len, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->prompt_len, prompt_len, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_TRY(cudaMemsetAsync(ctx->counters, 0, 4 * sizeof(unsigned long long), st));
+    const spec_ctx::Params params{seed, n_new, 0};
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->params, &params, sizeof(params), cudaMemcpyHostToDevice, st));
+
+    // prompt pass: positions 0..prompt_len-2 (the last prompt token is fed by the first iteration)
+    SPEC_CUDA_TRY(cudaEventRecord(ctx->ev[0], st));
+    std::vector<int> from(batch, 0), to(batch);
+    for (int b = 0; b < batch; ++b) to[b] = prompt_len[b] - 1;
+    SPEC_TRY(feed_host_tokens(ctx, 0, prompt, prompt_stride, from, to, batch));
+    if (gamma > 0) SPEC_TRY(feed_host_tokens(ctx, 1, prompt, prompt_stride, from, to, batch));
+    SPEC_CUDA_TRY(cudaEventRecord(ctx->ev[1], st));
+
+    // decode loop: the iteration graph is replayed in bursts; after each burst the
+    // host reads the committed lengths.  A burst is as long as the iterations that
+    // are certainly needed (every iteration emits at most gamma + 1 tokens).
+    SPEC_TRY(build_graph(ctx, batch, gamma, temperature));
+    std::vector<int32_t> lengths(batch);
+    long long replays = 0;
+    int remaining = n_new;
+    while (remaining > 0) {
+        const int burst = (remaining + gamma) / (gamma + 1);
+        for (int i = 0; i < burst; ++i) SPEC_CUDA_TRY(cudaGraphLaunch(ctx->graph, st));
+        replays += burst;
+        SPEC_CUDA_TRY(cudaMemcpyAsync(lengths.data(), ctx->length, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+        SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+        remaining = 0;
+        for (int b = 0; b < batch; ++b) remaining = std::max(remaining, n_new - (lengths[b] - prompt_len[b]));
+    }
+    SPEC_CUDA_TRY(cudaEventRecord(ctx->ev[2], st));
+
+    SPEC_CUDA_TRY(cudaMemcpyAsync(host_tokens.data(), ctx->tokens, host_tokens.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    unsigned long long counters[4];
+    SPEC_CUDA_TRY(cudaMemcpyAsync(counters, ctx->counters, sizeof(counters), cudaMemcpyDeviceToHost, st));
+    SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+    for (int b = 0; b < batch; ++b)
+        std::memcpy(out_tokens + static_cast<size_t>(b) * n_new, &host_tokens[static_cast<size_t>(b) * max_len + prompt_len[b]], n_new * sizeof(int32_t));
+    // the diagnostics' view of the caches is stale now
+    std::fill(ctx->cached[0].begin(), ctx->cached[0].end(), 0);
+    std::fill(ctx->cached[1].begin(), ctx->cached[1].end(), 0);
+    if (stats) {
+        float pre = 0.0f, dec = 0.0f;
+        cudaEventElapsedTime(&pre, ctx->ev[0], ctx->ev[1]);
+        cudaEventElapsedTime(&dec, ctx->ev[1], ctx->ev[2]);
+        stats->iterations = static_cast<int64_t>(counters[0]);
+        stats->tokens = static_cast<int64_t>(counters[1]);
+        stats->tests_evaluated = static_cast<int64_t>(counters[2]);
+        stats->tests_passed = static_cast<int64_t>(counters[3]);
+        stats->target_passes = replays;
+        stats->draft_passes = replays * gamma;
+        stats->prefill_ms = pre;
+        stats->decode_ms = dec;
+    }
+    return SPEC_OK;
+}
+
+extern "C" int spec_reset(spec_ctx* ctx) {
+    if (!ctx) return fail(SPEC_ERR_BAD_ARG, "spec_reset: null context");
+    std::fill(ctx->cached[0].begin(), ctx->cached[0].end(), 0);
+    std::fill(ctx->cached[1].begin(), ctx->cached[1].end(), 0);
+    SPEC_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+    return SPEC_OK;
+}
+
+extern "C" int spec_truncate(spec_ctx* ctx, int which, const int32_t* lengths, int batch) {
+    if (!ctx || !lengths || which < 0 || which > 1 || batch < 1 || batch > ctx->rt.max_batch)
+        return fail(SPEC_ERR_BAD_ARG, "spec_truncate: bad argument");
+    for (int b = 0; b < batch; ++b) {
+        if (lengths[b] < 0 || lengths[b] > ctx->cached[which][b])
+            return fail(SPEC_ERR_BAD_ARG, "spec_truncate: length %d of sequence %d is not within the cached %d", lengths[b], b, ctx->cached[which][b]);
+    }
+    for (int b = 0; b < batch; ++b) ctx->cached[which][b] = lengths[b];
+    return SPEC_OK;
+}
+
+extern "C" int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* tokens, int batch, int rows, float* logits) {
+    if (!ctx || !tokens || !logits || which < 0 || which > 1 || batch < 1 || rows < 1)
+        return fail(SPEC_ERR_BAD_ARG, "spec_forward_logits: bad argument");
+    if (which == 1 && !ctx->has_draft) return fail(SPEC_ERR_BAD_CONFIG, "spec_forward_logits: no draft model");
+    if (batch > ctx->rt.max_batch || batch * rows > ctx->max_rows)
+        return fail(SPEC_ERR_CAPACITY, "spec_forward_logits: %d x %d rows exceed the workspace (%d rows)", batch, rows, ctx->max_rows);
+    const Model& m = ctx->model[which];
+    const int n = batch * rows;
+    std::vector<int32_t> tok(n), pos(n), seq(n);
+    for (int b = 0; b < batch; ++b) {
+        if (ctx->cached[which][b] + rows > std::min(ctx->rt.max_len, m.cfg.max_positions))
+            return fail(SPEC_ERR_CAPACITY, "spec_forward_logits: sequence %d would exceed the cache", b);
+        for (int j = 0; j < rows; ++j) {
+            const int32_t t = tokens[b * rows + j];
+            if (t < 0 || t >= m.cfg.vocab) return fail(SPEC_ERR_BAD_ARG, "spec_forward_logits: token %d out of range", t);
+            tok[b * rows + j] = t;
+            pos[b * rows + j] = ctx->cached[which][b] + j;
+            seq[b * rows + j] = b;
+        }
+    }
+    cudaStream_t st = ctx->stream;
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_token, tok.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_pos, pos.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_seq, seq.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_TRY(forward(ctx, m, n, n, nullptr, nullptr, logits));
+    SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+    for (int b = 0; b < batch; ++b) ctx->cached[which][b] += rows;
+    return SPEC_OK;
+}

@@ -17,7 +17,7 @@
 
 #include <cooperative_groups.h>
 
-#include "common.cuh"
+#include "model.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -496,7 +496,8 @@ __global__ void __launch_bounds__(kFinishThreads, 2)
 verify_finish_kernel(const float* __restrict__ target_logits, const float* __restrict__ draft_logits,
                      const int32_t* __restrict__ draft_tokens, const float* __restrict__ uniforms, int gamma,
                      int vocab, float inv_t, int chunks, int cluster_size, const ChunkStat* __restrict__ stats,
-                     int32_t* __restrict__ n_accepted, int32_t* __restrict__ next_token) {
+                     const float* __restrict__ final_uniforms, int32_t* __restrict__ n_accepted,
+                     int32_t* __restrict__ next_token) {
     __shared__ FinishShared sh;
     const int tid = threadIdx.x;
     const int b = blockIdx.x / cluster_size;
@@ -574,7 +575,9 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
         if (rank == 0) token = __float_as_int(sh.row_aux[n]);
     } else {
         constexpr int W = kFinishThreads / 32;
-        const float u = sh.u_final;
+        // The generation loop keys the final draw by the position it decides, which
+        // depends on n: it passes one candidate uniform per possible n.
+        const float u = final_uniforms ? __ldg(final_uniforms + static_cast<size_t>(b) * (gamma + 1) + n) : sh.u_final;
         PlainWeights<VEC> pw;
         pw.p = make_row<VEC>(tl + static_cast<size_t>(n) * vocab, vocab);
         pw.max_p = sh.row_max[n];
@@ -604,8 +607,9 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
 // One CTA per row: tokens[r] ~ softmax(logits[r] / T), or argmax at T = 0.
 template <bool VEC>
 __global__ void __launch_bounds__(kSampleThreads)
-sample_kernel(const float* __restrict__ logits, const float* __restrict__ uniforms, int vocab, float inv_t,
-              bool greedy, int32_t* __restrict__ tokens) {
+sample_kernel(const float* __restrict__ logits, size_t logit_stride, const float* __restrict__ uniforms,
+              int uniform_stride, int vocab, float inv_t, bool greedy, int32_t* __restrict__ tokens,
+              int token_stride) {
     constexpr int W = kSampleThreads / 32;
     __shared__ float red[W];
     __shared__ int red_i[W];
@@ -613,7 +617,7 @@ sample_kernel(const float* __restrict__ logits, const float* __restrict__ unifor
     __shared__ float s_max;
     __shared__ int s_arg;
     const int tid = threadIdx.x;
-    const Row<VEC> r = make_row<VEC>(logits + static_cast<size_t>(blockIdx.x) * vocab, vocab);
+    const Row<VEC> r = make_row<VEC>(logits + static_cast<size_t>(blockIdx.x) * logit_stride, vocab);
     const int groups = (vocab + 3) >> 2;
     float m = -FLT_MAX;
     int arg = 0x7fffffff;
@@ -636,9 +640,9 @@ sample_kernel(const float* __restrict__ logits, const float* __restrict__ unifor
         pw.max_p = s_max;
         pw.c2 = inv_t * kLog2e;
         float total;
-        token = block_inverse_cdf<W>(pw, vocab, uniforms[blockIdx.x], cdf, &total);
+        token = block_inverse_cdf<W>(pw, vocab, uniforms[blockIdx.x * uniform_stride], cdf, &total);
     }
-    if (tid == 0) tokens[blockIdx.x] = max(0, min(token, vocab - 1));
+    if (tid == 0) tokens[blockIdx.x * token_stride] = max(0, min(token, vocab - 1));
 }
 
 __global__ void uniforms_kernel(uint64_t seed, const int32_t* __restrict__ positions,
@@ -674,9 +678,15 @@ int chunks_for(int vocab, int rows_total) {
 }  // namespace
 
 // Shared with the generation loop: same launches, no argument checks.
+size_t verify_sample_workspace_bytes(int batch, int gamma, int vocab) {
+    const size_t rows = 2 * static_cast<size_t>(gamma) + 1;
+    return static_cast<size_t>(batch) * rows * max_chunks(vocab) * sizeof(ChunkStat) + 256;
+}
+
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
-                         const float* uniforms, int batch, int gamma, int vocab, float temperature,
-                         int32_t* n_accepted, int32_t* next_token, void* workspace, cudaStream_t stream) {
+                         const float* uniforms, const float* final_uniforms, int batch, int gamma, int vocab,
+                         float temperature, int32_t* n_accepted, int32_t* next_token, void* workspace,
+                         cudaStream_t stream) {
     const bool greedy = temperature == 0.0f;
     const int rows = greedy ? gamma + 1 : 2 * gamma + 1;
     const int chunks = chunks_for(vocab, rows * batch);
@@ -713,8 +723,8 @@ int launch_verify_sample(const float* target_logits, const float* draft_logits, 
     const ChunkStat* stats_in = stats;
 #define SPEC_LAUNCH_FINISH(G, V)                                                                                  \
     SPEC_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_finish_kernel<G, V>, target_logits, draft_logits, draft_tokens, \
-                                     uniforms, gamma, vocab, inv_t, chunks, cluster_size, stats_in, n_accepted,  \
-                                     next_token))
+                                     uniforms, gamma, vocab, inv_t, chunks, cluster_size, stats_in,              \
+                                     final_uniforms, n_accepted, next_token))
     if (greedy && vec) SPEC_LAUNCH_FINISH(true, true);
     else if (greedy) SPEC_LAUNCH_FINISH(true, false);
     else if (vec) SPEC_LAUNCH_FINISH(false, true);
@@ -723,24 +733,34 @@ int launch_verify_sample(const float* target_logits, const float* draft_logits, 
     return SPEC_OK;
 }
 
-int launch_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
-                  int32_t* tokens, cudaStream_t stream) {
+// Row r reads logits + r * logit_stride and uniforms[r * uniform_stride] and
+// writes tokens[r * token_stride].
+int launch_sample_strided(const float* logits, size_t logit_stride, const float* uniforms, int uniform_stride,
+                          int rows, int vocab, float temperature, int32_t* tokens, int token_stride,
+                          cudaStream_t stream) {
     const bool greedy = temperature == 0.0f;
     const float inv_t = greedy ? 0.0f : 1.0f / temperature;
-    if (vocab % 4 == 0 && aligned16(logits))
-        sample_kernel<true><<<rows, kSampleThreads, 0, stream>>>(logits, uniforms, vocab, inv_t, greedy, tokens);
+    if (vocab % 4 == 0 && logit_stride % 4 == 0 && aligned16(logits))
+        sample_kernel<true><<<rows, kSampleThreads, 0, stream>>>(logits, logit_stride, uniforms, uniform_stride, vocab,
+                                                                 inv_t, greedy, tokens, token_stride);
     else
-        sample_kernel<false><<<rows, kSampleThreads, 0, stream>>>(logits, uniforms, vocab, inv_t, greedy, tokens);
+        sample_kernel<false><<<rows, kSampleThreads, 0, stream>>>(logits, logit_stride, uniforms, uniform_stride,
+                                                                  vocab, inv_t, greedy, tokens, token_stride);
     SPEC_CUDA_TRY(cudaGetLastError());
     return SPEC_OK;
+}
+
+int launch_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
+                  int32_t* tokens, cudaStream_t stream) {
+    return launch_sample_strided(logits, static_cast<size_t>(vocab), uniforms, 1, rows, vocab, temperature, tokens, 1,
+                                 stream);
 }
 
 }  // namespace spec
 
 extern "C" size_t spec_verify_sample_workspace_bytes(int batch, int gamma, int vocab) {
     if (batch < 0 || gamma < 0 || vocab < 1) return 0;
-    const size_t rows = 2 * static_cast<size_t>(gamma) + 1;
-    return static_cast<size_t>(batch) * rows * spec::max_chunks(vocab) * sizeof(spec::ChunkStat) + 256;
+    return spec::verify_sample_workspace_bytes(batch, gamma, vocab);
 }
 
 extern "C" int spec_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
@@ -761,8 +781,8 @@ extern "C" int spec_verify_sample(const float* target_logits, const float* draft
     if (workspace_bytes < spec_verify_sample_workspace_bytes(batch, gamma, vocab) ||
         (reinterpret_cast<uintptr_t>(workspace) & 255u))
         return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: workspace too small (%zu bytes) or not 256-byte aligned", workspace_bytes);
-    return launch_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, batch, gamma, vocab, temperature,
-                                n_accepted, next_token, workspace, static_cast<cudaStream_t>(stream));
+    return launch_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, nullptr, batch, gamma, vocab,
+                                temperature, n_accepted, next_token, workspace, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int spec_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
