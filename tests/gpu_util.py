@@ -31,3 +31,38 @@ def compare_verify(n_gpu, t_gpu, tl, ql, xs, us, temperature):
                        f"t={ref.next_token}) margins {ref.accept_margin:.3g} {ref.cdf_margin:.3g}")
         flagged += 1
     return flagged, tl.shape[0]
+
+
+def compare_generation(engine, oracle_target, oracle_draft, prompt, n_new, gamma, temperature, seed, margin,
+                       logit_tol, sequence=0):
+    """Free-running comparison of token streams.  At the first difference the
+    oracle's own margins decide whether the decision was within tolerance of a
+    boundary (then it is counted, both sides restart from the oracle's prefix at
+    the end of that iteration, which the position-keyed randomness allows);
+    any other difference raises.  Returns (flagged, iterations)."""
+    from oracle import generate as oracle_generate
+
+    assert sequence == 0
+    ref = oracle_generate.speculative_generate(oracle_target, oracle_draft, prompt, n_new, gamma, temperature, seed)
+    prompt = [int(t) for t in prompt]
+    done = 0
+    flagged = 0
+    while done < n_new:
+        got, _ = engine.generate([np.array(prompt + ref.tokens[:done], dtype=np.int32)], n_new - done, gamma,
+                                 temperature, seed)
+        got = got[0].tolist()
+        want = ref.tokens[done:]
+        diff = next((k for k in range(len(want)) if got[k] != want[k]), None)
+        if diff is None:
+            break
+        index = len(prompt) + done + diff  # absolute position of the first differing token
+        it = next(i for i in ref.iterations if i.start_len <= index <= i.start_len + i.n_accepted)
+        if temperature > 0:
+            close = min([it.accept_margin, it.cdf_margin] + list(it.draft_cdf_margins)) < margin
+        else:
+            close = it.top2_gap <= 2 * logit_tol
+        assert close, (f"token {index}: gpu {got[diff]} oracle {want[diff]}; iteration margins accept "
+                       f"{it.accept_margin:.3g} cdf {it.cdf_margin:.3g} draft {it.draft_cdf_margins} gap {it.top2_gap:.3g}")
+        flagged += 1
+        done = it.start_len + it.n_accepted + 1 - len(prompt)
+    return flagged, len(ref.iterations)

@@ -1,0 +1,114 @@
+"""End-to-end generation through the C ABI against the CPU oracle: Algorithm 1
+with both decoders, free-running, plus the properties the paper fixes."""
+import numpy as np
+import pytest
+
+from gpu_util import compare_generation
+from oracle import generate as oracle_generate
+from oracle.decoder import Decoder
+from paper_2211_17192_b200 import binding, workloads
+
+pytestmark = pytest.mark.gpu
+
+
+def _models(target_name, draft_name, **overrides):
+    tcfg = workloads.scaled_config(workloads.model_config(target_name), **overrides)
+    dcfg = workloads.scaled_config(workloads.model_config(draft_name), **overrides)
+    return tcfg, workloads.make_weights(tcfg, 1), dcfg, workloads.make_weights(dcfg, 2)
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    tcfg, tw, dcfg, dw = _models("tiny_target", "tiny_draft")
+    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=4, max_len=128, page_size=16, max_gamma=8)
+    yield eng, Decoder(tcfg, tw), Decoder(dcfg, dw), tcfg
+    eng.close()
+
+
+@pytest.mark.parametrize("temperature", [1.0, 0.0])
+def test_tiny_pair_matches_the_oracle(tiny, temperature):
+    """Tiny fp32 pair, gamma = 3, 16-token prompt, 64 new tokens."""
+    eng, target, draft, cfg = tiny
+    prompt = workloads.make_prompt(7, 16, cfg["vocab"])
+    flagged, iters = compare_generation(eng, target, draft, prompt, 64, 3, temperature, seed=11, margin=1e-3,
+                                        logit_tol=1e-3)
+    assert flagged <= 2, f"{flagged} decisions within tolerance of a boundary in {iters} iterations"
+
+
+@pytest.mark.parametrize("gamma", [1, 2, 5, 8])
+def test_temperature_zero_equals_target_only_greedy(tiny, gamma):
+    eng, target, _, cfg = tiny
+    prompt = workloads.make_prompt(8, 9, cfg["vocab"])
+    greedy, _ = eng.generate([prompt], 40, 0, 0.0, 0)
+    spec, stats = eng.generate([prompt], 40, gamma, 0.0, 0)
+    assert np.array_equal(greedy, spec)
+    ref, rows, _ = oracle_generate.target_only_generate(target, prompt, 40, 0.0, 0, keep_logits=True)
+    gaps = [np.sort(r)[-1] - np.sort(r)[-2] for r in rows]
+    for k in range(40):
+        if greedy[0, k] != ref[k]:
+            assert gaps[k] < 2e-3  # an argmax tie within the logit tolerance; the runs diverge from here
+            break
+    assert stats["iterations"] >= 40 / (gamma + 1)
+
+
+def test_target_only_sampling_matches_the_oracle(tiny):
+    eng, target, _, cfg = tiny
+    prompt = workloads.make_prompt(9, 5, cfg["vocab"])
+    got, stats = eng.generate([prompt], 48, 0, 1.0, 5)
+    ref, _, margins = oracle_generate.target_only_generate(target, prompt, 48, 1.0, 5)
+    for k in range(48):
+        if got[0, k] != ref[k]:
+            assert margins[k] < 1e-3
+            break
+    assert stats["iterations"] == 48 and stats["tests_evaluated"] == 0 and stats["draft_passes"] == 0
+
+
+def test_draft_equal_to_target_accepts_everything():
+    tcfg, tw, _, _ = _models("tiny_target", "tiny_draft", n_layers=2)
+    eng = binding.Engine(tcfg, tw, tcfg, tw, max_batch=1, max_len=128, page_size=32, max_gamma=4)
+    prompt = workloads.make_prompt(3, 10, tcfg["vocab"])
+    out, stats = eng.generate([prompt], 50, 4, 1.0, 3)
+    assert stats["tests_passed"] == stats["tests_evaluated"] == 4 * stats["iterations"]
+    assert stats["iterations"] == 10 and stats["tokens"] == 50
+    eng.close()
+
+
+def test_ragged_batch_equals_per_sequence_oracle(tiny):
+    eng, target, draft, cfg = tiny
+    prompts = [workloads.make_prompt(20 + b, n, cfg["vocab"]) for b, n in enumerate([3, 16, 9, 1])]
+    out, stats = eng.generate(prompts, 24, 3, 1.0, 17)
+    assert stats["tokens"] >= 4 * 24
+    for b, prompt in enumerate(prompts):
+        ref = oracle_generate.speculative_generate(target, draft, prompt, 24, 3, 1.0, 17, sequence=b)
+        got = out[b].tolist()
+        diff = next((k for k in range(24) if got[k] != ref.tokens[k]), None)
+        if diff is not None:
+            index = len(prompt) + diff
+            it = next(i for i in ref.iterations if i.start_len <= index <= i.start_len + i.n_accepted)
+            assert min([it.accept_margin, it.cdf_margin] + list(it.draft_cdf_margins)) < 1e-3
+
+
+def test_bf16_llama_pair_matches_the_oracle():
+    tcfg, tw, dcfg, dw = _models("llama_test_target", "llama_test_draft")
+    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=1, max_len=256, page_size=16, max_gamma=4)
+    prompt = workloads.make_prompt(2, 24, tcfg["vocab"])
+    for temperature in (1.0, 0.0):
+        flagged, iters = compare_generation(eng, Decoder(tcfg, tw), Decoder(dcfg, dw), prompt, 48, 4, temperature,
+                                            seed=5, margin=5e-3, logit_tol=5e-3)
+        assert flagged <= 3, f"{flagged} flagged of {iters}"
+    eng.close()
+
+
+def test_statistics_are_consistent(tiny):
+    eng, _, _, cfg = tiny
+    prompt = workloads.make_prompt(4, 12, cfg["vocab"])
+    out, st = eng.generate([prompt], 60, 3, 1.0, 1)
+    assert out.shape == (1, 60) and out.min() >= 0 and out.max() < cfg["vocab"]
+    assert st["tokens"] == st["iterations"] + st["tests_passed"]          # n + 1 tokens per iteration
+    assert st["tests_passed"] <= st["tests_evaluated"] <= 3 * st["iterations"]
+    assert 60 <= st["tokens"] <= 60 + 3 and st["target_passes"] >= st["iterations"]
+    assert st["decode_ms"] > 0 and st["prefill_ms"] >= 0
+    again, _ = eng.generate([prompt], 60, 3, 1.0, 1)
+    assert np.array_equal(out, again)  # same seed, same tokens
+    other, _ = eng.generate([prompt], 60, 3, 1.0, 2)
+    assert not np.array_equal(out, other)
