@@ -175,7 +175,7 @@ typedef struct spec_weights {
 typedef struct spec_runtime_cfg {
     int max_batch;        /* sequences decoded together */
     int max_len;          /* tokens per sequence the KV caches can hold (prompt + new + gamma) */
-    int page_size;        /* tokens per KV page (power of two, 16..256) */
+    int page_size;        /* tokens per KV page (power of two, 32..256) */
     int max_gamma;        /* largest gamma spec_generate will be asked for */
     int kv_dtype;         /* SPEC_DTYPE_FP32 or SPEC_DTYPE_BF16: element type of the cached K,V rows.
                              bf16 halves the KV traffic but rounds every cached row to 8 mantissa

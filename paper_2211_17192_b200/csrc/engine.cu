@@ -331,7 +331,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     }
     const spec_runtime_cfg& rt = *runtime;
     if (rt.max_batch < 1 || rt.max_batch > 4096 || rt.max_len < 2 || rt.max_gamma < 0 || rt.max_gamma > 64 ||
-        rt.page_size < 16 || rt.page_size > 256 || (rt.page_size & (rt.page_size - 1)) ||
+        rt.page_size < 32 || rt.page_size > 256 || (rt.page_size & (rt.page_size - 1)) ||
         (rt.kv_dtype != SPEC_DTYPE_FP32 && rt.kv_dtype != SPEC_DTYPE_BF16))
         return fail(SPEC_ERR_BAD_CONFIG, "spec_init: runtime config out of range");
     int device_count = 0;

@@ -42,7 +42,7 @@ def _pair(name, seed=1, **overrides):
 def test_teacher_forced_logits_with_rollback(name, overrides):
     cfg, w = _pair(name, **overrides)
     oracle = Decoder(cfg, w)
-    eng = binding.Engine(cfg, w, max_batch=1, max_len=128, page_size=16, max_gamma=10)
+    eng = binding.Engine(cfg, w, max_batch=1, max_len=128, page_size=32, max_gamma=10)
     tokens = workloads.make_prompt(3, 40, cfg["vocab"])
     ref = oracle.forward_full(tokens)  # cache-free: cannot carry a stale row
     eng.reset()
@@ -68,7 +68,7 @@ def test_bf16_kv_cache_option_stays_close():
     cfg, w = _pair("llama_test_target")
     tokens = workloads.make_prompt(3, 40, cfg["vocab"])
     ref = Decoder(cfg, w).forward_full(tokens)
-    eng = binding.Engine(cfg, w, max_batch=1, max_len=64, page_size=16, max_gamma=3, kv_dtype="bf16")
+    eng = binding.Engine(cfg, w, max_batch=1, max_len=64, page_size=32, max_gamma=3, kv_dtype="bf16")
     eng.reset()
     got = eng.forward_logits(0, tokens[None, :]).cpu().numpy()[0]
     err = np.abs(got - ref).max()
@@ -81,7 +81,7 @@ def test_batched_sequences_are_independent_and_page_size_is_invisible():
     seqs = [workloads.make_prompt(10 + b, 30, cfg["vocab"]) for b in range(3)]
     ref = [Decoder(cfg, w).forward_full(s) for s in seqs]
     outs = []
-    for page in (16, 64):
+    for page in (32, 128):
         eng = binding.Engine(cfg, w, max_batch=3, max_len=64, page_size=page, max_gamma=7)
         eng.reset()
         a = eng.forward_logits(0, np.stack([s[:8] for s in seqs])).cpu().numpy()
@@ -102,7 +102,7 @@ def test_batched_sequences_are_independent_and_page_size_is_invisible():
 def test_both_models_of_a_pair_share_a_context():
     tcfg, tw = _pair("tiny_target")
     dcfg, dw = _pair("tiny_draft", seed=2)
-    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=2, max_len=64, page_size=16, max_gamma=3)
+    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=2, max_len=64, page_size=32, max_gamma=3)
     tokens = np.stack([workloads.make_prompt(5, 12, 8192), workloads.make_prompt(6, 12, 8192)])
     eng.reset()
     t = eng.forward_logits(0, tokens).cpu().numpy()
@@ -118,7 +118,7 @@ def test_errors_are_reported():
     with pytest.raises(binding.SpecError) as e:
         binding.Engine(workloads.scaled_config(cfg, d_head=48), w)
     assert e.value.status == -2
-    eng = binding.Engine(cfg, w, max_batch=1, max_len=32, page_size=16, max_gamma=2)
+    eng = binding.Engine(cfg, w, max_batch=1, max_len=32, page_size=32, max_gamma=2)
     with pytest.raises(binding.SpecError) as e:
         eng.forward_logits(0, np.zeros((1, 40), dtype=np.int32))
     assert e.value.status == -4

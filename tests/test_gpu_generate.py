@@ -20,7 +20,7 @@ def _models(target_name, draft_name, **overrides):
 @pytest.fixture(scope="module")
 def tiny():
     tcfg, tw, dcfg, dw = _models("tiny_target", "tiny_draft")
-    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=4, max_len=128, page_size=16, max_gamma=8)
+    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=4, max_len=128, page_size=32, max_gamma=8)
     yield eng, Decoder(tcfg, tw), Decoder(dcfg, dw), tcfg
     eng.close()
 
@@ -90,7 +90,7 @@ def test_ragged_batch_equals_per_sequence_oracle(tiny):
 
 def test_bf16_llama_pair_matches_the_oracle():
     tcfg, tw, dcfg, dw = _models("llama_test_target", "llama_test_draft")
-    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=1, max_len=256, page_size=16, max_gamma=4)
+    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=1, max_len=256, page_size=32, max_gamma=4)
     prompt = workloads.make_prompt(2, 24, tcfg["vocab"])
     for temperature in (1.0, 0.0):
         flagged, iters = compare_generation(eng, Decoder(tcfg, tw), Decoder(dcfg, dw), prompt, 48, 4, temperature,
