@@ -250,6 +250,28 @@ int spec_reset(spec_ctx* ctx);
 int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* tokens, int batch, int rows, float* logits);
 int spec_truncate(spec_ctx* ctx, int which, const int32_t* lengths, int batch);
 
+/* ------------------------------------------------------------------------- *
+ * One linear layer y = x . W^T, the building block of the verification pass
+ * (the paper's premise, Section 1 and Section 3.4: the pass is bound by
+ * streaming W from memory, and gamma+1 rows share one stream of the weights).
+ *   x [rows, k] fp32 device; w [n_out, k] device in w_dtype (SPEC_DTYPE_*);
+ *   y [rows, n_out] fp32 device out; k a multiple of 8.
+ *   path 0: the path the engine would choose (tensor cores for bf16 weights,
+ *           FMA pipes for fp32); 1: FMA pipes; 2: tensor cores (bf16 only).
+ * The tensor-core path splits x into two bf16 terms and sums split-K partial
+ * results in a fixed order; it needs `workspace` (device, 256-byte aligned, at
+ * least spec_linear_workspace_bytes(rows, n_out, k) bytes, contents arbitrary,
+ * not shared by overlapping calls).  The FMA path ignores the workspace.
+ * Asynchronous on `stream`; allocates nothing.
+ * spec_device_error() returns non-zero (and clears it) if a kernel of this
+ * library gave up on a bounded device-side wait since the last call; it
+ * synchronises with the device.
+ * ------------------------------------------------------------------------- */
+size_t spec_linear_workspace_bytes(int rows, int n_out, int k);
+int spec_linear(const float* x, const void* w, int w_dtype, int rows, int n_out, int k, int path,
+                float* y, void* workspace, size_t workspace_bytes, void* stream);
+int spec_device_error(void);
+
 #ifdef __cplusplus
 }
 #endif

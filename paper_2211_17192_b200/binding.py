@@ -59,6 +59,12 @@ def _declare(h):
     h.spec_sample.argtypes = [vp, vp, i32, i32, f32, vp, vp]
     h.spec_uniforms.restype = i32
     h.spec_uniforms.argtypes = [u64, vp, vp, i32, i32, vp, vp]
+    h.spec_linear_workspace_bytes.restype = sz
+    h.spec_linear_workspace_bytes.argtypes = [i32, i32, i32]
+    h.spec_linear.restype = i32
+    h.spec_linear.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp]
+    h.spec_device_error.restype = i32
+    h.spec_device_error.argtypes = []
 
 
 def _check(status):
@@ -144,6 +150,38 @@ def spec_uniforms(seed, positions, sequences, purpose, out=None):
                                _ptr(sequences, torch.int32, "sequences"), int(purpose), count,
                                _ptr(out, torch.float32, "out"), _stream()))
     return out
+
+
+PATHS = {"auto": 0, "alu": 1, "tensor": 2}
+
+
+def spec_linear_workspace_bytes(rows, n_out, k):
+    return int(lib().spec_linear_workspace_bytes(rows, n_out, k))
+
+
+def spec_linear(x, w, path="auto", y=None, workspace=None):
+    """y = x . W^T; x [rows, k] fp32 CUDA, w [n_out, k] fp32 or bf16 CUDA -> y [rows, n_out] fp32."""
+    rows, k = x.shape
+    n_out = w.shape[0]
+    if w.shape[1] != k:
+        raise ValueError("inner dimensions differ")
+    if w.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("w must be fp32 or bf16")
+    if y is None:
+        y = torch.empty((rows, n_out), dtype=torch.float32, device=x.device)
+    need = spec_linear_workspace_bytes(rows, n_out, k)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+    if not w.is_cuda or not w.is_contiguous():
+        raise ValueError("w must be a contiguous CUDA tensor")
+    _check(lib().spec_linear(_ptr(x, torch.float32, "x"), w.data_ptr(), 1 if w.dtype == torch.bfloat16 else 0,
+                             rows, n_out, k, PATHS[path], _ptr(y, torch.float32, "y"),
+                             _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()))
+    return y
+
+
+def spec_device_error():
+    return int(lib().spec_device_error())
 
 
 # --------------------------------------------------------------------------- #

@@ -4,6 +4,7 @@
 // graph, and the teacher-forced diagnostics used by the parity tests.
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -21,6 +22,11 @@ struct spec_ctx {
     // activations (sized for the wider model)
     float *h = nullptr, *a = nullptr, *qkv = nullptr, *att = nullptr, *u = nullptr, *f = nullptr;
     float *target_logits = nullptr, *draft_logits = nullptr;
+    // tensor-core GEMM path: bf16 hi/lo copies of the GEMM input, split-K partial sums
+    __nv_bfloat16 *x_hi = nullptr, *x_lo = nullptr;
+    float* partials = nullptr;
+    int hi_rows = 0;
+    bool tensor_cores = true;
     int32_t *row_token = nullptr, *row_pos = nullptr, *row_seq = nullptr, *logit_src = nullptr, *logit_dst = nullptr;
     int32_t* page_table = nullptr;
 
@@ -80,28 +86,38 @@ int dev_alloc(spec_ctx* ctx, T** out, size_t count) {
 // One forward pass of `m` over the rows described by ctx->row_*; K,V rows of
 // active rows are appended to the cache.  If n_logit_rows > 0 the final norm and
 // LM head run on rows logit_src[i] and write logits rows logit_dst[i].
+// y[dst(r)] = x[r] . W^T (+ residual[r]): tensor cores for bf16 weights, FMA pipes otherwise.
+int gemm(spec_ctx* ctx, const Model& m, const float* x, const void* w, const float* residual, const int32_t* dst_rows,
+         int n_rows, int n_out, int k, float* y) {
+    if (m.bf16() && ctx->tensor_cores) {
+        SPEC_TRY(launch_split_bf16(x, static_cast<size_t>(n_rows) * k, ctx->x_hi, ctx->x_lo, ctx->stream));
+        return launch_gemm_tc(ctx->x_hi, ctx->x_lo, ctx->hi_rows, w, residual, dst_rows, n_rows, n_out, k,
+                              ctx->partials, y, ctx->stream);
+    }
+    return launch_gemm_rows(x, w, m.bf16(), residual, dst_rows, n_rows, n_out, k, y, ctx->stream);
+}
+
 int forward(spec_ctx* ctx, const Model& m, int n_rows, int n_logit_rows, const int32_t* logit_src,
             const int32_t* logit_dst, float* logits) {
     cudaStream_t st = ctx->stream;
     const spec_model_cfg& c = m.cfg;
     const RowMeta rows{ctx->row_token, ctx->row_pos, ctx->row_seq};
-    const bool bf = m.bf16();
     SPEC_TRY(launch_embed(m, rows, n_rows, ctx->h, st));
     for (int l = 0; l < c.n_layers; ++l) {
         const spec_layer_weights& w = m.layers[l];
         SPEC_TRY(launch_rmsnorm(ctx->h, w.ln1, nullptr, n_rows, c.d_model, c.rms_eps, ctx->a, st));
-        SPEC_TRY(launch_gemm_rows(ctx->a, w.wqkv, bf, nullptr, nullptr, n_rows, m.qkv_dim(), c.d_model, ctx->qkv, st));
+        SPEC_TRY(gemm(ctx, m, ctx->a, w.wqkv, nullptr, nullptr, n_rows, m.qkv_dim(), c.d_model, ctx->qkv));
         SPEC_TRY(launch_rope_append(m, l, rows, n_rows, ctx->qkv, ctx->page_table, ctx->pages_per_seq, ctx->rt.page_size, st));
         SPEC_TRY(launch_attention(m, l, rows, n_rows, ctx->qkv, ctx->att, ctx->page_table, ctx->pages_per_seq, ctx->rt.page_size, st));
-        SPEC_TRY(launch_gemm_rows(ctx->att, w.wo, bf, ctx->h, nullptr, n_rows, c.d_model, m.q_dim(), ctx->h, st));
+        SPEC_TRY(gemm(ctx, m, ctx->att, w.wo, ctx->h, nullptr, n_rows, c.d_model, m.q_dim(), ctx->h));
         SPEC_TRY(launch_rmsnorm(ctx->h, w.ln2, nullptr, n_rows, c.d_model, c.rms_eps, ctx->a, st));
-        SPEC_TRY(launch_gemm_rows(ctx->a, w.w_in, bf, nullptr, nullptr, n_rows, m.ffn_in_dim(), c.d_model, ctx->u, st));
+        SPEC_TRY(gemm(ctx, m, ctx->a, w.w_in, nullptr, nullptr, n_rows, m.ffn_in_dim(), c.d_model, ctx->u));
         SPEC_TRY(launch_ffn_act(ctx->u, n_rows, c.d_ff, c.ffn, ctx->f, st));
-        SPEC_TRY(launch_gemm_rows(ctx->f, w.w_out, bf, ctx->h, nullptr, n_rows, c.d_model, c.d_ff, ctx->h, st));
+        SPEC_TRY(gemm(ctx, m, ctx->f, w.w_out, ctx->h, nullptr, n_rows, c.d_model, c.d_ff, ctx->h));
     }
     if (n_logit_rows > 0) {
         SPEC_TRY(launch_rmsnorm(ctx->h, m.ln_f, logit_src, n_logit_rows, c.d_model, c.rms_eps, ctx->a, st));
-        SPEC_TRY(launch_gemm_rows(ctx->a, m.head, bf, nullptr, logit_dst, n_logit_rows, c.vocab, c.d_model, logits, st));
+        SPEC_TRY(gemm(ctx, m, ctx->a, m.head, nullptr, logit_dst, n_logit_rows, c.vocab, c.d_model, logits));
     }
     return SPEC_OK;
 }
@@ -378,6 +394,32 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     SPEC_ALLOC(f, R * ff);
     SPEC_ALLOC(target_logits, R * V);
     SPEC_ALLOC(draft_logits, std::max<size_t>(B * G, 1) * V);
+    {
+        // Tensor-core path (any bf16 model): inputs as two bf16 terms, split-K partial sums.
+        const char* path = std::getenv("SPEC_GEMM_PATH");
+        ctx->tensor_cores = !(path && std::strcmp(path, "alu") == 0);
+        size_t max_k = 0, partial = 0;
+        bool any_bf16 = false;
+        for (int i = 0; i < (ctx->has_draft ? 2 : 1); ++i) {
+            const Model& m = ctx->model[i];
+            if (!m.bf16()) continue;
+            any_bf16 = true;
+            max_k = std::max<size_t>({max_k, static_cast<size_t>(m.cfg.d_model), static_cast<size_t>(m.q_dim()), static_cast<size_t>(m.cfg.d_ff)});
+            const int shapes[5][2] = {{m.qkv_dim(), m.cfg.d_model}, {m.cfg.d_model, m.q_dim()}, {m.ffn_in_dim(), m.cfg.d_model},
+                                      {m.cfg.d_model, m.cfg.d_ff}, {m.cfg.vocab, m.cfg.d_model}};
+            for (const auto& sh : shapes)
+                for (int rows = 1; rows <= ctx->max_rows; ++rows)
+                    partial = std::max(partial, gemm_tc_partial_elems(sh[0], sh[1], rows));
+        }
+        if (any_bf16 && ctx->tensor_cores) {
+            ctx->hi_rows = (ctx->max_rows + 127) / 128 * 128;
+            SPEC_ALLOC(x_hi, static_cast<size_t>(ctx->hi_rows) * max_k);
+            SPEC_ALLOC(x_lo, static_cast<size_t>(ctx->hi_rows) * max_k);
+            SPEC_ALLOC(partials, partial);
+            cudaMemset(ctx->x_hi, 0, static_cast<size_t>(ctx->hi_rows) * max_k * 2);
+            cudaMemset(ctx->x_lo, 0, static_cast<size_t>(ctx->hi_rows) * max_k * 2);
+        }
+    }
     SPEC_ALLOC(row_token, R);
     SPEC_ALLOC(row_pos, R);
     SPEC_ALLOC(row_seq, R);
@@ -490,6 +532,7 @@ extern "C" int spec_generate(spec_ctx* ctx, const int32_t* prompt, const int32_t
     unsigned long long counters[4];
     SPEC_CUDA_TRY(cudaMemcpyAsync(counters, ctx->counters, sizeof(counters), cudaMemcpyDeviceToHost, st));
     SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+    if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
     for (int b = 0; b < batch; ++b)
         std::memcpy(out_tokens + static_cast<size_t>(b) * n_new, &host_tokens[static_cast<size_t>(b) * max_len + prompt_len[b]], n_new * sizeof(int32_t));
     // the diagnostics' view of the caches is stale now
@@ -556,6 +599,7 @@ extern "C" int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* toke
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_seq, seq.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SPEC_TRY(forward(ctx, m, n, n, nullptr, nullptr, logits));
     SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+    if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
     for (int b = 0; b < batch; ++b) ctx->cached[which][b] += rows;
     return SPEC_OK;
 }

@@ -1,0 +1,460 @@
+// Skinny weight-streaming GEMM on the 5th-generation tensor cores:
+//   partial[s][r][n] = sum over the k-range of split s of x[r][k] * W[n][k]
+// for a few activation rows against a bf16 weight matrix W [n_out, k] that is
+// streamed from HBM exactly once.
+//
+// The weights take the M side of the MMA ("swap A/B"): a CTA owns 128 output
+// features, TMA brings [128 x 64] bf16 weight tiles (128-byte swizzle) into a
+// ring of shared-memory stages, and one thread issues tcgen05.mma (kind::f16,
+// M = 128, N = padded token count, K = 16) into an fp32 accumulator in tensor
+// memory.  The token side carries the activations split into two bf16 terms,
+// x = hi + lo, issued as two MMAs into the same accumulator, so that the
+// result keeps ~16 mantissa bits of the fp32 activations while the weight
+// tile is still read once.  Split-K over the grid keeps every SM streaming for
+// matrices with few 128-row tiles; partial sums go to a workspace and are added
+// up in a fixed order by reduce_partials_kernel (no atomics, bit-reproducible).
+//
+// Every wait on an mbarrier is bounded; on expiry the kernel records an error
+// code and unwinds (tensor memory is freed on every path).
+#include <cuda.h>
+
+#include <map>
+#include <mutex>
+#include <tuple>
+
+#include "model.cuh"
+
+namespace spec {
+namespace {
+
+constexpr int kTileM = 128;     // output features per CTA (MMA M)
+constexpr int kTileK = 64;      // bf16 elements per k-block: one 128-byte swizzle row
+constexpr int kMmaK = 16;       // K of one tcgen05.mma.kind::f16
+constexpr int kThreads = 128;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+__device__ int g_gemm_error;  // first device-side time-out (0 = none)
+
+// ---- PTX wrappers ----------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+// Bounded wait for the phase with the given parity; false on time-out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t"
+            "}"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes
+// long and 128-byte swizzled: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr & 0x3FFFF) >> 4);   // start address, 16-byte units
+    d |= static_cast<uint64_t>(1) << 16;                 // leading byte offset (unused with swizzle)
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;         // stride byte offset between 8-row groups
+    d |= static_cast<uint64_t>(1) << 46;                 // descriptor version of this architecture
+    d |= static_cast<uint64_t>(2) << 61;                 // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128.
+__host__ __device__ constexpr uint32_t instr_desc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+           (static_cast<uint32_t>(kTileM >> 4) << 24);
+}
+
+__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+        "}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// The mbarrier gets one arrival once every MMA issued so far has finished.
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+template <int N_TOK>
+struct Smem {
+    static constexpr int kStages = N_TOK <= 16 ? 5 : N_TOK == 64 ? 3 : 4;
+    static constexpr int kABytes = kTileM * kTileK * 2;   // 16 KB
+    static constexpr int kBBytes = N_TOK * kTileK * 2;     // one of hi / lo
+    static constexpr int kStageBytes = kABytes + 2 * kBBytes;
+    static constexpr int kTotal = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+};
+
+// grid = (tiles of 128 features, splits, token tiles), block = 128.
+template <int N_TOK>
+__global__ void __launch_bounds__(kThreads)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_hi,
+               const __grid_constant__ CUtensorMap map_lo, float* __restrict__ partial, int n_out, int n_rows,
+               int k_blocks) {
+    using S = Smem<N_TOK>;
+    constexpr int kTmemCols = N_TOK < 32 ? 32 : N_TOK;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + S::kStages * S::kStageBytes);
+    uint64_t* empty_bar = full_bar + S::kStages;
+    uint64_t* acc_bar = empty_bar + S::kStages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_bar + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x, split = blockIdx.y, splits = gridDim.y, tok0 = blockIdx.z * N_TOK;
+    const int kb0 = static_cast<int>(static_cast<long long>(k_blocks) * split / splits);
+    const int kb1 = static_cast<int>(static_cast<long long>(k_blocks) * (split + 1) / splits);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S::kStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        mbar_init(acc_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {  // one warp owns the tensor-memory allocation
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(kTmemCols));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_acc = *tmem_slot;
+    bool ok = true;
+
+    if (warp == 0 && lane == 0) {
+        // ---- producer: weights and both activation terms of one k-block per stage ----
+        for (int kb = kb0; kb < kb1; ++kb) {
+            const int it = kb - kb0, s = it % S::kStages;
+            if (it >= S::kStages && !mbar_wait(&empty_bar[s], ((it / S::kStages) - 1) & 1)) { ok = false; break; }
+            uint8_t* stage = smem + s * S::kStageBytes;
+            mbar_expect_tx(&full_bar[s], S::kStageBytes);
+            tma_load_2d(stage, &map_w, kb * kTileK, tile * kTileM, &full_bar[s]);
+            tma_load_2d(stage + S::kABytes, &map_hi, kb * kTileK, tok0, &full_bar[s]);
+            tma_load_2d(stage + S::kABytes + S::kBBytes, &map_lo, kb * kTileK, tok0, &full_bar[s]);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---- MMA issuer ----
+        constexpr uint32_t idesc = instr_desc(N_TOK);
+        for (int kb = kb0; kb < kb1; ++kb) {
+            const int it = kb - kb0, s = it % S::kStages;
+            if (!mbar_wait(&full_bar[s], (it / S::kStages) & 1)) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_addr = smem_u32(smem + s * S::kStageBytes);
+            const uint64_t a_desc = smem_desc_sw128(a_addr);
+            const uint64_t hi_desc = smem_desc_sw128(a_addr + S::kABytes);
+            const uint64_t lo_desc = smem_desc_sw128(a_addr + S::kABytes + S::kBBytes);
+#pragma unroll
+            for (int k = 0; k < kTileK / kMmaK; ++k) {
+                const uint64_t step = static_cast<uint64_t>((k * kMmaK * 2) >> 4);  // 32 bytes along K, in 16-byte units
+                mma_f16(tmem_acc, a_desc + step, hi_desc + step, idesc, (it > 0 || k > 0) ? 1u : 0u);
+                mma_f16(tmem_acc, a_desc + step, lo_desc + step, idesc, 1u);
+            }
+            mma_commit(&empty_bar[s]);  // the stage may be refilled once these MMAs have read it
+        }
+        mma_commit(acc_bar);  // accumulator complete
+    }
+    __syncwarp();
+
+    // ---- epilogue: all four warps, warp w reads accumulator lanes 32w .. 32w+31 ----
+    if (kb1 > kb0) {
+        if (!mbar_wait(acc_bar, 0)) ok = false;
+    }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int feature = tile * kTileM + warp * 32 + lane;
+    float* out = partial + (static_cast<size_t>(split) * n_rows) * n_out + feature;
+    if (ok) {
+#pragma unroll
+        for (int c0 = 0; c0 < N_TOK; c0 += 16) {
+            if (tok0 + c0 < n_rows) {  // uniform across the warp
+                float v[16];
+                if (kb1 > kb0) {
+                    tmem_ld16(tmem_acc + (static_cast<uint32_t>(warp * 32) << 16) + c0, v);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] = 0.0f;
+                }
+                if (feature < n_out) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int r = tok0 + c0 + i;
+                        if (r < n_rows) out[static_cast<size_t>(r) * n_out] = v[i];
+                    }
+                }
+            }
+        }
+    } else {
+        atomicCAS(&g_gemm_error, 0, 1 + warp);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(kTmemCols));
+    }
+}
+
+// x (fp32) -> hi = bf16(x), lo = bf16(x - hi); grid-stride, 4 elements per thread
+__global__ void split_bf16_kernel(const float* __restrict__ x, size_t n, __nv_bfloat16* __restrict__ hi,
+                                  __nv_bfloat16* __restrict__ lo) {
+    for (size_t i = (blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x) * 4; i < n;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x * 4) {
+        const float4 v = *reinterpret_cast<const float4*>(x + i);
+        const float f[4] = {v.x, v.y, v.z, v.w};
+        __nv_bfloat16 h[4], l[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            h[j] = __float2bfloat16_rn(f[j]);
+            l[j] = __float2bfloat16_rn(f[j] - __bfloat162float(h[j]));
+        }
+        *reinterpret_cast<uint2*>(hi + i) = *reinterpret_cast<const uint2*>(h);
+        *reinterpret_cast<uint2*>(lo + i) = *reinterpret_cast<const uint2*>(l);
+    }
+}
+
+// y[dst(r)][n] = sum_s partial[s][r][n] (+ residual[r][n]), splits added in index order
+__global__ void reduce_partials_kernel(const float* __restrict__ partial, int splits, int n_rows, int n_out,
+                                       const float* residual, const int32_t* __restrict__ dst_rows, float* y) {
+    const size_t total = static_cast<size_t>(n_rows) * n_out;
+    for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        float acc = partial[i];
+        for (int s = 1; s < splits; ++s) acc += partial[static_cast<size_t>(s) * total + i];
+        if (residual) acc += residual[i];
+        const size_t r = i / n_out, n = i % n_out;
+        y[(dst_rows ? static_cast<size_t>(dst_rows[r]) : r) * n_out + n] = acc;
+    }
+}
+
+// ---- host side ----------------------------------------------------------------
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+    static EncodeFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeFn>(p);
+    }();
+    return fn;
+}
+
+// A bf16 matrix [rows, cols] row-major, fetched in boxes of [box_rows, 64] with 128-byte swizzle.
+int make_map(const void* base, int rows, int cols, int box_rows, CUtensorMap* out) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return fail(SPEC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * 2};
+    const cuuint32_t box[2] = {kTileK, static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t elem[2] = {1, 1};
+    const CUresult res = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (res != CUDA_SUCCESS) return fail(SPEC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", static_cast<int>(res));
+    return SPEC_OK;
+}
+
+struct MapKey {
+    const void* base;
+    int rows, cols, box_rows;
+    bool operator<(const MapKey& o) const {
+        return std::tie(base, rows, cols, box_rows) < std::tie(o.base, o.rows, o.cols, o.box_rows);
+    }
+};
+
+// Tensor maps are pure functions of (address, shape, box): cached process-wide.
+int cached_map(const void* base, int rows, int cols, int box_rows, CUtensorMap* out) {
+    static std::mutex mu;
+    static std::map<MapKey, CUtensorMap> cache;
+    std::lock_guard<std::mutex> lock(mu);
+    const MapKey key{base, rows, cols, box_rows};
+    auto it = cache.find(key);
+    if (it == cache.end()) {
+        CUtensorMap m;
+        const int status = make_map(base, rows, cols, box_rows, &m);
+        if (status != SPEC_OK) return status;
+        it = cache.emplace(key, m).first;
+    }
+    *out = it->second;
+    return SPEC_OK;
+}
+
+template <int N_TOK>
+int launch_tc(const CUtensorMap& mw, const CUtensorMap& mhi, const CUtensorMap& mlo, float* partial, int n_out,
+              int n_rows, int k_blocks, int splits, cudaStream_t stream) {
+    static bool configured = false;
+    if (!configured) {
+        SPEC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<N_TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           Smem<N_TOK>::kTotal));
+        configured = true;
+    }
+    const dim3 grid((n_out + kTileM - 1) / kTileM, splits, (n_rows + N_TOK - 1) / N_TOK);
+    gemm_tc_kernel<N_TOK><<<grid, kThreads, Smem<N_TOK>::kTotal, stream>>>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks);
+    SPEC_CUDA_TRY(cudaGetLastError());
+    return SPEC_OK;
+}
+
+}  // namespace
+
+int gemm_tc_token_tile(int n_rows) { return n_rows <= 16 ? 16 : n_rows <= 32 ? 32 : n_rows <= 64 ? 64 : 128; }
+
+// Split-K factor: the smallest one that fills the last wave of CTAs to 85 %, with
+// at least two k-blocks per split.
+int gemm_tc_splits(int n_out, int k, int n_rows) {
+    const int n_tok = gemm_tc_token_tile(n_rows);
+    const int tiles = ((n_out + kTileM - 1) / kTileM) * ((n_rows + n_tok - 1) / n_tok);
+    const int k_blocks = (k + kTileK - 1) / kTileK;
+    const int resident = 148 * (n_tok <= 64 ? 2 : 1);
+    const int max_splits = std::max(1, std::min(k_blocks / 2, 16));
+    int best = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= max_splits; ++s) {
+        const int ctas = tiles * s;
+        const int waves = (ctas + resident - 1) / resident;
+        const double eff = static_cast<double>(ctas) / (static_cast<double>(waves) * resident);
+        if (eff > best_eff + 1e-9) {
+            best_eff = eff;
+            best = s;
+        }
+        if (eff >= 0.85) return s;
+    }
+    return best;
+}
+
+size_t gemm_tc_partial_elems(int n_out, int k, int n_rows) {
+    return static_cast<size_t>(gemm_tc_splits(n_out, k, n_rows)) * n_rows * n_out;
+}
+
+int launch_split_bf16(const float* x, size_t n, __nv_bfloat16* hi, __nv_bfloat16* lo, cudaStream_t stream) {
+    const int blocks = static_cast<int>(std::min<size_t>((n / 4 + 255) / 256, 148 * 8));
+    split_bf16_kernel<<<std::max(blocks, 1), 256, 0, stream>>>(x, n, hi, lo);
+    SPEC_CUDA_TRY(cudaGetLastError());
+    return SPEC_OK;
+}
+
+// y[dst(r)] = x[r] . W^T (+ residual[r]) with x already split into hi + lo
+// (both [hi_rows, k] bf16, the first n_rows rows valid).
+int launch_gemm_tc(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, const float* residual,
+                   const int32_t* dst_rows, int n_rows, int n_out, int k, float* partial, float* y,
+                   cudaStream_t stream) {
+    if (n_rows <= 0) return SPEC_OK;
+    if (k % 8 != 0) return fail(SPEC_ERR_BAD_CONFIG, "gemm: inner dimension %d is not a multiple of 8", k);
+    const int n_tok = gemm_tc_token_tile(n_rows);
+    const int splits = gemm_tc_splits(n_out, k, n_rows);
+    const int k_blocks = (k + kTileK - 1) / kTileK;
+    CUtensorMap mw, mhi, mlo;
+    int status = cached_map(w, n_out, k, kTileM, &mw);
+    if (status == SPEC_OK) status = cached_map(hi, hi_rows, k, n_tok, &mhi);
+    if (status == SPEC_OK) status = cached_map(lo, hi_rows, k, n_tok, &mlo);
+    if (status != SPEC_OK) return status;
+    switch (n_tok) {
+        case 16: status = launch_tc<16>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream); break;
+        case 32: status = launch_tc<32>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream); break;
+        case 64: status = launch_tc<64>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream); break;
+        default: status = launch_tc<128>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream); break;
+    }
+    if (status != SPEC_OK) return status;
+    const size_t total = static_cast<size_t>(n_rows) * n_out;
+    const int blocks = static_cast<int>(std::min<size_t>((total + 255) / 256, 148 * 8));
+    reduce_partials_kernel<<<blocks, 256, 0, stream>>>(partial, splits, n_rows, n_out, residual, dst_rows, y);
+    SPEC_CUDA_TRY(cudaGetLastError());
+    return SPEC_OK;
+}
+
+// Non-zero if a tensor-core GEMM gave up on a bounded wait since the last call.
+int gemm_tc_take_error() {
+    int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_gemm_error, sizeof(int)) != cudaSuccess) return -1;
+    if (v) cudaMemcpyToSymbol(g_gemm_error, &zero, sizeof(int));
+    return v;
+}
+
+}  // namespace spec
+
+// ---- C ABI: one linear layer, for tests and benchmarks of the GEMM kernels ----
+namespace {
+size_t align256(size_t v) { return (v + 255) / 256 * 256; }
+int padded_rows(int rows) { return (rows + 127) / 128 * 128; }
+}  // namespace
+
+extern "C" size_t spec_linear_workspace_bytes(int rows, int n_out, int k) {
+    if (rows < 1 || n_out < 1 || k < 1) return 0;
+    const size_t split_bytes = align256(static_cast<size_t>(padded_rows(rows)) * k * 2);
+    return 2 * split_bytes + align256(spec::gemm_tc_partial_elems(n_out, k, rows) * sizeof(float)) + 256;
+}
+
+extern "C" int spec_linear(const float* x, const void* w, int w_dtype, int rows, int n_out, int k, int path, float* y,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+    using namespace spec;
+    if (!x || !w || !y) return fail(SPEC_ERR_BAD_ARG, "spec_linear: null pointer");
+    if (rows < 1 || n_out < 1 || k < 8 || k % 8) return fail(SPEC_ERR_BAD_ARG, "spec_linear: rows=%d n_out=%d k=%d (k must be a multiple of 8)", rows, n_out, k);
+    if (w_dtype != SPEC_DTYPE_FP32 && w_dtype != SPEC_DTYPE_BF16) return fail(SPEC_ERR_BAD_ARG, "spec_linear: dtype %d", w_dtype);
+    if (path < 0 || path > 2) return fail(SPEC_ERR_BAD_ARG, "spec_linear: path %d", path);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool tensor = w_dtype == SPEC_DTYPE_BF16 && path != 1;
+    if (path == 2 && w_dtype != SPEC_DTYPE_BF16) return fail(SPEC_ERR_BAD_CONFIG, "spec_linear: the tensor-core path needs bf16 weights");
+    if (!tensor) return launch_gemm_rows(x, w, w_dtype == SPEC_DTYPE_BF16, nullptr, nullptr, rows, n_out, k, y, st);
+    if (!workspace || workspace_bytes < spec_linear_workspace_bytes(rows, n_out, k) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return fail(SPEC_ERR_BAD_ARG, "spec_linear: workspace missing, too small or not 256-byte aligned");
+    const size_t split_bytes = align256(static_cast<size_t>(padded_rows(rows)) * k * 2);
+    char* base = static_cast<char*>(workspace);
+    __nv_bfloat16* hi = reinterpret_cast<__nv_bfloat16*>(base);
+    __nv_bfloat16* lo = reinterpret_cast<__nv_bfloat16*>(base + split_bytes);
+    float* partial = reinterpret_cast<float*>(base + 2 * split_bytes);
+    // rows past `rows` of the padded tile are read by the MMA (their results are discarded): keep them finite
+    SPEC_CUDA_TRY(cudaMemsetAsync(base, 0, 2 * split_bytes, st));
+    int status = launch_split_bf16(x, static_cast<size_t>(rows) * k, hi, lo, st);
+    if (status != SPEC_OK) return status;
+    return launch_gemm_tc(hi, lo, padded_rows(rows), w, nullptr, nullptr, rows, n_out, k, partial, y, st);
+}
+
+extern "C" int spec_device_error(void) { return spec::gemm_tc_take_error(); }

@@ -53,6 +53,16 @@ int launch_rmsnorm(const float* in, const float* gain, const int32_t* src_rows, 
 int launch_gemm_rows(const float* x, const void* w, bool w_bf16, const float* residual, const int32_t* dst_rows,
                      int n_rows, int n_out, int k, float* y, cudaStream_t stream);
 
+// Tensor-core path for bf16 weights (gemm_tc.cu): x is first split into two bf16
+// terms, partial sums of the split-K grid are reduced in a fixed order.
+int gemm_tc_splits(int n_out, int k, int n_rows);
+size_t gemm_tc_partial_elems(int n_out, int k, int n_rows);
+int launch_split_bf16(const float* x, size_t n, __nv_bfloat16* hi, __nv_bfloat16* lo, cudaStream_t stream);
+int launch_gemm_tc(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, const float* residual,
+                   const int32_t* dst_rows, int n_rows, int n_out, int k, float* partial, float* y,
+                   cudaStream_t stream);
+int gemm_tc_take_error();
+
 // Rotary positions on q and k (Llama), then K,V rows of every active row into the paged cache.
 int launch_rope_append(const Model& m, int layer, const RowMeta& rows, int n_rows, float* qkv,
                        const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream);
