@@ -1,15 +1,21 @@
 // Causal attention of the new rows against the paged KV cache.
 //
-// One CTA per (row, query head); its warps split the keys between them in tiles
-// of 32 (tile t goes to warp t mod kAttnWarps) and merge their partial softmax
-// states at the end.  Inside a tile each lane owns one key: it reads that key's
-// d_head values with 16-byte loads (a page stores the keys of one head back to
-// back, so a warp's loads cover one contiguous span), takes the dot product
-// with the query held in shared memory, and the warp keeps an online softmax
-// (running max and sum, fp32).  For P.V the lanes turn to the head dimension:
-// lane l owns d_head/32 output elements, the tile's V rows are fetched eight at
-// a time, and every key's probability is broadcast with a shuffle.  A tile
+// Work is cut by (sequence, KV head, slice of the keys).  A CTA owns one such
+// piece and runs one warp per query that reads this KV head: the G query heads
+// of the group times the m new rows of the sequence.  All warps of the CTA walk
+// the same 32-key tiles, so the K and V rows come from HBM/L2 once per CTA and
+// from L1 for the other queries.  Inside a tile each lane owns one key: it reads
+// the key's d_head values with 16-byte loads (a page stores the keys of one head
+// back to back, so a warp's loads cover one contiguous span), takes the dot
+// product with the query held in shared memory, and the warp keeps an online
+// softmax (running max and sum, fp32).  For P.V the lanes turn to the head
+// dimension: lane l owns d_head/32 output elements, V rows are fetched sixteen
+// at a time, and every key's probability is broadcast with a shuffle.  A tile
 // never straddles a page (pages hold a multiple of 32 tokens).
+//
+// Each CTA writes an unnormalised partial state (max, sum, accumulator) per
+// query; attention_combine_kernel merges the key slices and emits the
+// out-projection's input (fp32 and/or split into two bf16 terms).
 #include <cfloat>
 
 #include "model.cuh"
@@ -17,7 +23,8 @@
 namespace spec {
 namespace {
 
-constexpr int kAttnWarps = 8;
+constexpr int kMaxAttnWarps = 16;
+constexpr int kVBatch = 16;
 
 template <typename KV>
 struct KvLoad;
@@ -29,7 +36,15 @@ struct KvLoad<float> {
         const float4 t = *reinterpret_cast<const float4*>(p);
         out[0] = t.x; out[1] = t.y; out[2] = t.z; out[3] = t.w;
     }
-    __device__ static __forceinline__ float one(const float* p) { return *p; }
+    template <int N>
+    __device__ static __forceinline__ void load_n(const float* p, float* out) {
+        if (N == 4) {
+            load(p, out);
+        } else {
+            const float2 t = *reinterpret_cast<const float2*>(p);
+            out[0] = t.x; out[1] = t.y;
+        }
+    }
 };
 
 template <>
@@ -44,116 +59,189 @@ struct KvLoad<__nv_bfloat16> {
             out[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
         }
     }
-    __device__ static __forceinline__ float one(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    template <int N>
+    __device__ static __forceinline__ void load_n(const __nv_bfloat16* p, float* out) {
+        if (N == 4) {
+            const uint2 t = *reinterpret_cast<const uint2*>(p);
+            out[0] = __uint_as_float(t.x << 16); out[1] = __uint_as_float(t.x & 0xffff0000u);
+            out[2] = __uint_as_float(t.y << 16); out[3] = __uint_as_float(t.y & 0xffff0000u);
+        } else {
+            const uint32_t t = *reinterpret_cast<const uint32_t*>(p);
+            out[0] = __uint_as_float(t << 16); out[1] = __uint_as_float(t & 0xffff0000u);
+        }
+    }
 };
 
-// grid = rows * n_heads, block = 32 * kAttnWarps
+// grid = (slices, n_kv_heads, batch), block = 32 * warps (warps <= kMaxAttnWarps).
+// Rows of sequence b are rows b*m .. b*m+m-1 of the pass.
 template <typename KV, int DH>
-__global__ void __launch_bounds__(32 * kAttnWarps)
+__global__ void __launch_bounds__(32 * kMaxAttnWarps)
 attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos, const int32_t* __restrict__ seq,
-                 int n_heads, int n_kv_heads, const KV* __restrict__ kv_layer,
+                 int m_rows, int n_heads, int n_kv_heads, const KV* __restrict__ kv_layer,
                  const int32_t* __restrict__ page_table, int pages_per_seq, int page_size, float scale,
-                 float* __restrict__ att) {
+                 float* __restrict__ part) {
     constexpr int PER_LANE = DH / 32;
-    __shared__ float q_sh[DH];
-    __shared__ float part_m[kAttnWarps], part_l[kAttnWarps];
-    __shared__ float part_acc[kAttnWarps][DH];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int r = blockIdx.x / n_heads, head = blockIdx.x % n_heads;
-    const int p = pos[r];
-    float* out = att + (static_cast<size_t>(r) * n_heads + head) * DH;
-    if (p < 0) {  // inactive row
-        for (int i = threadIdx.x; i < DH; i += blockDim.x) out[i] = 0.0f;
-        return;
-    }
-    const int kv_head = head / (n_heads / n_kv_heads);
+    __shared__ float q_sh[kMaxAttnWarps][DH];
+    pdl_trigger();
+    pdl_wait();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
+    const int slice = blockIdx.x, slices = gridDim.x, kv_head = blockIdx.y, b = blockIdx.z;
+    const int group = n_heads / n_kv_heads;
+    const int queries = group * m_rows;
     const int qkv_dim = (n_heads + 2 * n_kv_heads) * DH;
-    const float* q = qkv + static_cast<size_t>(r) * qkv_dim + head * DH;
-    for (int i = threadIdx.x; i < DH; i += blockDim.x) q_sh[i] = q[i] * scale;
-    __syncthreads();
 
-    const int32_t* pages = page_table + seq[r] * pages_per_seq;
+    // the key range of this slice: whole tiles, same for every query of the sequence
+    int max_pos = -1;
+    for (int j = 0; j < m_rows; ++j) max_pos = max(max_pos, pos[b * m_rows + j]);
+    const int tiles = (max_pos + 1 + 31) / 32;
+    const int t0 = static_cast<int>(static_cast<long long>(tiles) * slice / slices);
+    const int t1 = static_cast<int>(static_cast<long long>(tiles) * (slice + 1) / slices);
+
     const size_t head_stride = static_cast<size_t>(page_size) * DH;               // one head inside a page
     const size_t page_stride = 2 * static_cast<size_t>(n_kv_heads) * head_stride;  // K block + V block
     const size_t v_offset = static_cast<size_t>(n_kv_heads) * head_stride;
 
-    float m = -FLT_MAX, l = 0.0f;
-    float acc[PER_LANE];
-#pragma unroll
-    for (int i = 0; i < PER_LANE; ++i) acc[i] = 0.0f;
+    for (int q = warp; q < queries; q += warps) {
+        const int j = q / group, head = kv_head * group + q % group;
+        const int r = b * m_rows + j;
+        const int p = pos[r];
+        const int32_t* pages = page_table + seq[r] * pages_per_seq;
+        __syncwarp();
+        const float* qp = qkv + static_cast<size_t>(r) * qkv_dim + head * DH;
+        for (int i = lane; i < DH; i += 32) q_sh[warp][i] = qp[i] * scale;
+        __syncwarp();
 
-    const int n_keys = p + 1;  // causal: positions 0..p
-    for (int k0 = 32 * warp; k0 < n_keys; k0 += 32 * kAttnWarps) {
-        // the whole tile lives in one page
-        const KV* tile = kv_layer + pages[k0 / page_size] * page_stride + kv_head * head_stride +
-                         static_cast<size_t>(k0 % page_size) * DH;
-        const int in_tile = min(32, n_keys - k0);
-        float s = -FLT_MAX;
-        if (lane < in_tile) {
-            const KV* kp = tile + static_cast<size_t>(lane) * DH;
-            float dot = 0.0f;
+        float mx = -FLT_MAX, l = 0.0f;
+        float acc[PER_LANE];
 #pragma unroll
-            for (int d0 = 0; d0 < DH; d0 += KvLoad<KV>::kVec) {
-                float kvv[KvLoad<KV>::kVec];
-                KvLoad<KV>::load(kp + d0, kvv);
+        for (int i = 0; i < PER_LANE; ++i) acc[i] = 0.0f;
+        const int n_keys = p + 1;  // causal: positions 0..p (p < 0: inactive row, no keys)
+        for (int t = t0; t < t1; ++t) {
+            const int k0 = 32 * t;
+            if (k0 >= n_keys) break;
+            // the whole tile lives in one page
+            const KV* tile = kv_layer + pages[k0 / page_size] * page_stride + kv_head * head_stride +
+                             static_cast<size_t>(k0 % page_size) * DH;
+            const int in_tile = min(32, n_keys - k0);
+            float s = -FLT_MAX;
+            if (lane < in_tile) {
+                const KV* kp = tile + static_cast<size_t>(lane) * DH;
+                float dot = 0.0f;
 #pragma unroll
-                for (int e = 0; e < KvLoad<KV>::kVec; ++e) dot = fmaf(q_sh[d0 + e], kvv[e], dot);
+                for (int d0 = 0; d0 < DH; d0 += KvLoad<KV>::kVec) {
+                    float kvv[KvLoad<KV>::kVec];
+                    KvLoad<KV>::load(kp + d0, kvv);
+#pragma unroll
+                    for (int e = 0; e < KvLoad<KV>::kVec; ++e) dot = fmaf(q_sh[warp][d0 + e], kvv[e], dot);
+                }
+                s = dot;
             }
-            s = dot;
-        }
-        const float m_new = fmaxf(m, warp_max(s));
-        const float pr = lane < in_tile ? expf(s - m_new) : 0.0f;
-        const float rescale = expf(m - m_new);
-        l = l * rescale + warp_sum(pr);
-        m = m_new;
+            const float m_new = fmaxf(mx, warp_max(s));
+            const float pr = lane < in_tile ? expf(s - m_new) : 0.0f;
+            const float rescale = expf(mx - m_new);
+            l = l * rescale + warp_sum(pr);
+            mx = m_new;
 #pragma unroll
-        for (int i = 0; i < PER_LANE; ++i) acc[i] *= rescale;
-        const KV* vt = tile + v_offset + lane * PER_LANE;
-        for (int j0 = 0; j0 < in_tile; j0 += 8) {
-            float vv[8][PER_LANE];
+            for (int i = 0; i < PER_LANE; ++i) acc[i] *= rescale;
+            const KV* vt = tile + v_offset + lane * PER_LANE;
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
+            for (int j0 = 0; j0 < 32; j0 += kVBatch) {
+                if (j0 < in_tile) {
+                    float vv[kVBatch][PER_LANE];
 #pragma unroll
-                for (int i = 0; i < PER_LANE; ++i)
-                    vv[j][i] = j0 + j < in_tile ? KvLoad<KV>::one(vt + static_cast<size_t>(j0 + j) * DH + i) : 0.0f;
+                    for (int jj = 0; jj < kVBatch; ++jj) {
+                        if (j0 + jj < in_tile) {
+                            KvLoad<KV>::template load_n<PER_LANE>(vt + static_cast<size_t>(j0 + jj) * DH, vv[jj]);
+                        } else {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float pj = __shfl_sync(kFullMask, pr, (j0 + j) & 31);
+                            for (int i = 0; i < PER_LANE; ++i) vv[jj][i] = 0.0f;
+                        }
+                    }
 #pragma unroll
-                for (int i = 0; i < PER_LANE; ++i) acc[i] = fmaf(pj, vv[j][i], acc[i]);
+                    for (int jj = 0; jj < kVBatch; ++jj) {
+                        const float pj = __shfl_sync(kFullMask, pr, j0 + jj);
+#pragma unroll
+                        for (int i = 0; i < PER_LANE; ++i) acc[i] = fmaf(pj, vv[jj][i], acc[i]);
+                    }
+                }
             }
         }
+        // partial state of (row r, head, slice): [max, sum, acc[DH]]
+        float* out = part + ((static_cast<size_t>(r) * n_heads + head) * slices + slice) * (DH + 2);
+        if (lane == 0) {
+            out[0] = mx;
+            out[1] = l;
+        }
+#pragma unroll
+        for (int i = 0; i < PER_LANE; ++i) out[2 + lane * PER_LANE + i] = acc[i];
     }
-    // merge the warps' partial states
-    if (lane == 0) { part_m[warp] = m; part_l[warp] = l; }
-#pragma unroll
-    for (int i = 0; i < PER_LANE; ++i) part_acc[warp][lane * PER_LANE + i] = acc[i];
+}
+
+// grid = rows * n_heads, block = DH: merge the key slices of one (row, head).
+template <int DH>
+__global__ void attention_combine_kernel(const float* __restrict__ part, int slices, float* __restrict__ att,
+                                         __nv_bfloat16* __restrict__ att_hi, __nv_bfloat16* __restrict__ att_lo) {
+    __shared__ float w_sh[64];  // weight of every slice, then their normaliser at [slices]
+    pdl_trigger();
+    pdl_wait();
+    const float* in = part + static_cast<size_t>(blockIdx.x) * slices * (DH + 2);
+    if (threadIdx.x < 32) {  // slices <= 32: one lane per slice
+        const int s = threadIdx.x;
+        const float ms = s < slices ? in[s * (DH + 2)] : -FLT_MAX;
+        const float ls = s < slices ? in[s * (DH + 2) + 1] : 0.0f;
+        const float mm = warp_max(ms);
+        const float w = s < slices ? expf(ms - mm) : 0.0f;
+        const float l = warp_sum(ls * w);
+        if (s < slices) w_sh[s] = w;
+        if (s == 0) w_sh[32] = l;
+    }
     __syncthreads();
-    float mm = part_m[0];
-#pragma unroll
-    for (int w = 1; w < kAttnWarps; ++w) mm = fmaxf(mm, part_m[w]);
-    float ll = 0.0f;
-#pragma unroll
-    for (int w = 0; w < kAttnWarps; ++w) ll += part_l[w] * expf(part_m[w] - mm);
-    for (int i = threadIdx.x; i < DH; i += blockDim.x) {
-        float o = 0.0f;
-#pragma unroll
-        for (int w = 0; w < kAttnWarps; ++w) o += part_acc[w][i] * expf(part_m[w] - mm);
-        out[i] = o / ll;
+    float o = 0.0f;
+#pragma unroll 8
+    for (int s = 0; s < slices; ++s) o += in[s * (DH + 2) + 2 + threadIdx.x] * w_sh[s];
+    const float l = w_sh[32];
+    const float y = l > 0.0f ? o / l : 0.0f;  // an inactive row has no keys
+    const size_t i = static_cast<size_t>(blockIdx.x) * DH + threadIdx.x;
+    if (att) att[i] = y;
+    if (att_hi) {
+        const __nv_bfloat16 h = __float2bfloat16_rn(y);
+        att_hi[i] = h;
+        att_lo[i] = __float2bfloat16_rn(y - __bfloat162float(h));
     }
 }
 
 }  // namespace
 
-int launch_attention(const Model& m, int layer, const RowMeta& rows, int n_rows, const float* qkv, float* att,
+// Key slices per (sequence, KV head): enough CTAs for two per SM, at least 64 keys each.
+int attention_slices(int batch, int n_kv_heads, int max_len) {
+    const int want = (2 * 148 + batch * n_kv_heads - 1) / (batch * n_kv_heads);
+    const int most = std::max(1, max_len / 64);
+    return std::max(1, std::min(std::min(want, most), 32));
+}
+
+size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices) {
+    return static_cast<size_t>(rows) * n_heads * slices * (d_head + 2);
+}
+
+int launch_attention(const Model& m, int layer, const RowMeta& rows, int batch, int m_rows, int slices,
+                     const float* qkv, float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo,
                      const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream) {
     const char* kv_layer = static_cast<const char*>(m.kv) + static_cast<size_t>(layer) * m.layer_stride;
-    const int grid = n_rows * m.cfg.n_heads;
+    const int group = m.cfg.n_heads / m.cfg.n_kv_heads;
+    const int warps = std::min(kMaxAttnWarps, std::max(1, group * m_rows));
+    const dim3 grid(slices, m.cfg.n_kv_heads, batch);
     const float scale = 1.0f / sqrtf(static_cast<float>(m.cfg.d_head));
-#define SPEC_ATTN(KV, DH)                                                                                       \
-    attention_kernel<KV, DH><<<grid, 32 * kAttnWarps, 0, stream>>>(                                             \
-        qkv, rows.pos, rows.seq, m.cfg.n_heads, m.cfg.n_kv_heads, reinterpret_cast<const KV*>(kv_layer),         \
-        page_table, pages_per_seq, page_size, scale, att)
+    const int n_rows = batch * m_rows;
+#define SPEC_ATTN(KV, DH)                                                                                         \
+    do {                                                                                                          \
+        int status = launch_pdl(attention_kernel<KV, DH>, grid, dim3(32 * warps), 0, stream, qkv, rows.pos,       \
+                                rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads,                                \
+                                reinterpret_cast<const KV*>(kv_layer), page_table, pages_per_seq, page_size,      \
+                                scale, part);                                                                     \
+        if (status != SPEC_OK) return status;                                                                     \
+        return launch_pdl(attention_combine_kernel<DH>, dim3(n_rows * m.cfg.n_heads), dim3(DH), 0, stream,         \
+                          static_cast<const float*>(part), slices, att, att_hi, att_lo);                          \
+    } while (0)
     if (m.kv_elem_bytes == 2) {
         if (m.cfg.d_head == 64) SPEC_ATTN(__nv_bfloat16, 64);
         else SPEC_ATTN(__nv_bfloat16, 128);
@@ -162,7 +250,6 @@ int launch_attention(const Model& m, int layer, const RowMeta& rows, int n_rows,
         else SPEC_ATTN(float, 128);
     }
 #undef SPEC_ATTN
-    SPEC_CUDA_TRY(cudaGetLastError());
     return SPEC_OK;
 }
 

@@ -31,6 +31,38 @@ inline int fail(int status, const char* fmt, ...) {
                                 cudaGetErrorString(err__), __FILE__, __LINE__);         \
     } while (0)
 
+// ---- programmatic dependent launch -------------------------------------------
+// Every kernel of the decode path is launched with programmatic stream
+// serialization and follows one rule: it may start while its predecessor in the
+// stream is still running, it calls pdl_wait() before it reads or writes
+// anything another kernel touches, and it calls pdl_trigger() as early as it
+// can so that its successor can start its own independent prologue (for a GEMM:
+// streaming the first weight tiles).  pdl_wait() returns once the predecessor
+// grid has completed and its writes are visible; because every kernel waits,
+// completion is transitive along the stream.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// SPEC_NO_PDL=1 in the environment launches every kernel fully serialised (for debugging).
+bool pdl_enabled();  // api.cu
+
+template <typename... KArgs, typename... Args>
+inline int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    if (err != cudaSuccess) return fail(SPEC_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(err));
+    return SPEC_OK;
+}
+
 // ---- warp / block primitives ----------------------------------------------
 constexpr unsigned kFullMask = 0xffffffffu;
 

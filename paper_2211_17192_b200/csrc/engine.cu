@@ -25,6 +25,7 @@ struct spec_ctx {
     // tensor-core GEMM path: bf16 hi/lo copies of the GEMM input, split-K partial sums
     __nv_bfloat16 *x_hi = nullptr, *x_lo = nullptr;
     float* partials = nullptr;
+    float* attn_part = nullptr;  // per key slice: (max, sum, accumulator) of every (row, head)
     int hi_rows = 0;
     bool tensor_cores = true;
     int32_t *row_token = nullptr, *row_pos = nullptr, *row_seq = nullptr, *logit_src = nullptr, *logit_dst = nullptr;
@@ -86,38 +87,67 @@ int dev_alloc(spec_ctx* ctx, T** out, size_t count) {
 // One forward pass of `m` over the rows described by ctx->row_*; K,V rows of
 // active rows are appended to the cache.  If n_logit_rows > 0 the final norm and
 // LM head run on rows logit_src[i] and write logits rows logit_dst[i].
-// y[dst(r)] = x[r] . W^T (+ residual[r]): tensor cores for bf16 weights, FMA pipes otherwise.
-int gemm(spec_ctx* ctx, const Model& m, const float* x, const void* w, const float* residual, const int32_t* dst_rows,
-         int n_rows, int n_out, int k, float* y) {
-    if (m.bf16() && ctx->tensor_cores) {
-        SPEC_TRY(launch_split_bf16(x, static_cast<size_t>(n_rows) * k, ctx->x_hi, ctx->x_lo, ctx->stream));
-        return launch_gemm_tc(ctx->x_hi, ctx->x_lo, ctx->hi_rows, w, residual, dst_rows, n_rows, n_out, k,
-                              ctx->partials, y, ctx->stream);
-    }
-    return launch_gemm_rows(x, w, m.bf16(), residual, dst_rows, n_rows, n_out, k, y, ctx->stream);
-}
-
-int forward(spec_ctx* ctx, const Model& m, int n_rows, int n_logit_rows, const int32_t* logit_src,
+// One forward pass of `m` over batch * m_rows rows (rows of sequence b are rows
+// b*m_rows .. of ctx->row_*); K,V rows of active rows are appended to the cache.
+// If n_logit_rows > 0 the final norm and LM head run on rows logit_src[i] and
+// write logits rows logit_dst[i].
+//
+// bf16 models take the tensor-core path: every GEMM leaves split-K partial sums
+// that the next small kernel adds up, and every GEMM input is produced directly
+// as two bf16 terms.  fp32 models run the same kernels with fp32 hand-offs and
+// the FMA-pipe GEMM.
+int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_rows, const int32_t* logit_src,
             const int32_t* logit_dst, float* logits) {
     cudaStream_t st = ctx->stream;
     const spec_model_cfg& c = m.cfg;
+    const int n_rows = batch * m_rows;
     const RowMeta rows{ctx->row_token, ctx->row_pos, ctx->row_seq};
+    const bool tc = m.bf16() && ctx->tensor_cores;
+    __nv_bfloat16 *hi = tc ? ctx->x_hi : nullptr, *lo = tc ? ctx->x_lo : nullptr;
+    float* part = ctx->partials;
+    const int d = c.d_model, pages = ctx->pages_per_seq, page = ctx->rt.page_size;
+    const int slices = attention_slices(batch, c.n_kv_heads, ctx->rt.max_len);
+    // split-K factors of the four GEMM shapes of a block at this row count
+    const int s_qkv = tc ? gemm_tc_splits(m.qkv_dim(), d, n_rows) : 0;
+    const int s_o = tc ? gemm_tc_splits(d, m.q_dim(), n_rows) : 0;
+    const int s_in = tc ? gemm_tc_splits(m.ffn_in_dim(), d, n_rows) : 0;
+    const int s_out = tc ? gemm_tc_splits(d, c.d_ff, n_rows) : 0;
+
     SPEC_TRY(launch_embed(m, rows, n_rows, ctx->h, st));
     for (int l = 0; l < c.n_layers; ++l) {
         const spec_layer_weights& w = m.layers[l];
-        SPEC_TRY(launch_rmsnorm(ctx->h, w.ln1, nullptr, n_rows, c.d_model, c.rms_eps, ctx->a, st));
-        SPEC_TRY(gemm(ctx, m, ctx->a, w.wqkv, nullptr, nullptr, n_rows, m.qkv_dim(), c.d_model, ctx->qkv));
-        SPEC_TRY(launch_rope_append(m, l, rows, n_rows, ctx->qkv, ctx->page_table, ctx->pages_per_seq, ctx->rt.page_size, st));
-        SPEC_TRY(launch_attention(m, l, rows, n_rows, ctx->qkv, ctx->att, ctx->page_table, ctx->pages_per_seq, ctx->rt.page_size, st));
-        SPEC_TRY(gemm(ctx, m, ctx->att, w.wo, ctx->h, nullptr, n_rows, c.d_model, m.q_dim(), ctx->h));
-        SPEC_TRY(launch_rmsnorm(ctx->h, w.ln2, nullptr, n_rows, c.d_model, c.rms_eps, ctx->a, st));
-        SPEC_TRY(gemm(ctx, m, ctx->a, w.w_in, nullptr, nullptr, n_rows, m.ffn_in_dim(), c.d_model, ctx->u));
-        SPEC_TRY(launch_ffn_act(ctx->u, n_rows, c.d_ff, c.ffn, ctx->f, st));
-        SPEC_TRY(gemm(ctx, m, ctx->f, w.w_out, ctx->h, nullptr, n_rows, c.d_model, c.d_ff, ctx->h));
+        if (tc) {
+            // (the FFN-out partial sums of the previous block are added into h by this norm)
+            SPEC_TRY(launch_norm(ctx->h, l ? part : nullptr, s_out, n_rows, w.ln1, nullptr, n_rows, d, c.rms_eps, nullptr, hi, lo, st));
+            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, w.wqkv, n_rows, m.qkv_dim(), d, part, st));
+            SPEC_TRY(launch_qkv(m, l, rows, n_rows, ctx->qkv, part, s_qkv, ctx->page_table, pages, page, st));
+            SPEC_TRY(launch_attention(m, l, rows, batch, m_rows, slices, ctx->qkv, ctx->attn_part, nullptr, hi, lo, ctx->page_table, pages, page, st));
+            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, w.wo, n_rows, d, m.q_dim(), part, st));
+            SPEC_TRY(launch_norm(ctx->h, part, s_o, n_rows, w.ln2, nullptr, n_rows, d, c.rms_eps, nullptr, hi, lo, st));
+            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, w.w_in, n_rows, m.ffn_in_dim(), d, part, st));
+            SPEC_TRY(launch_ffn_act(nullptr, part, s_in, n_rows, c.d_ff, c.ffn, nullptr, hi, lo, st));
+            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, w.w_out, n_rows, d, c.d_ff, part, st));
+        } else {
+            const bool bf = m.bf16();
+            SPEC_TRY(launch_norm(ctx->h, nullptr, 0, n_rows, w.ln1, nullptr, n_rows, d, c.rms_eps, ctx->a, nullptr, nullptr, st));
+            SPEC_TRY(launch_gemm_rows(ctx->a, w.wqkv, bf, nullptr, nullptr, n_rows, m.qkv_dim(), d, ctx->qkv, st));
+            SPEC_TRY(launch_qkv(m, l, rows, n_rows, ctx->qkv, nullptr, 0, ctx->page_table, pages, page, st));
+            SPEC_TRY(launch_attention(m, l, rows, batch, m_rows, slices, ctx->qkv, ctx->attn_part, ctx->att, nullptr, nullptr, ctx->page_table, pages, page, st));
+            SPEC_TRY(launch_gemm_rows(ctx->att, w.wo, bf, ctx->h, nullptr, n_rows, d, m.q_dim(), ctx->h, st));
+            SPEC_TRY(launch_norm(ctx->h, nullptr, 0, n_rows, w.ln2, nullptr, n_rows, d, c.rms_eps, ctx->a, nullptr, nullptr, st));
+            SPEC_TRY(launch_gemm_rows(ctx->a, w.w_in, bf, nullptr, nullptr, n_rows, m.ffn_in_dim(), d, ctx->u, st));
+            SPEC_TRY(launch_ffn_act(ctx->u, nullptr, 0, n_rows, c.d_ff, c.ffn, ctx->f, nullptr, nullptr, st));
+            SPEC_TRY(launch_gemm_rows(ctx->f, w.w_out, bf, ctx->h, nullptr, n_rows, d, c.d_ff, ctx->h, st));
+        }
     }
     if (n_logit_rows > 0) {
-        SPEC_TRY(launch_rmsnorm(ctx->h, m.ln_f, logit_src, n_logit_rows, c.d_model, c.rms_eps, ctx->a, st));
-        SPEC_TRY(gemm(ctx, m, ctx->a, m.head, nullptr, logit_dst, n_logit_rows, c.vocab, c.d_model, logits));
+        if (tc) {
+            SPEC_TRY(launch_norm(ctx->h, part, s_out, n_rows, m.ln_f, logit_src, n_logit_rows, d, c.rms_eps, nullptr, hi, lo, st));
+            SPEC_TRY(launch_gemm_tc(hi, lo, ctx->hi_rows, m.head, nullptr, logit_dst, n_logit_rows, c.vocab, d, part, logits, st));
+        } else {
+            SPEC_TRY(launch_norm(ctx->h, nullptr, 0, n_rows, m.ln_f, logit_src, n_logit_rows, d, c.rms_eps, ctx->a, nullptr, nullptr, st));
+            SPEC_TRY(launch_gemm_rows(ctx->a, m.head, m.bf16(), nullptr, logit_dst, n_logit_rows, c.vocab, d, logits, st));
+        }
     }
     return SPEC_OK;
 }
@@ -133,6 +163,8 @@ __global__ void iteration_uniforms_kernel(const spec_ctx::Params* __restrict__ p
                                           const int32_t* __restrict__ length, int batch, int gamma,
                                           float* __restrict__ draft_u, float* __restrict__ accept_u,
                                           float* __restrict__ final_u) {
+    pdl_trigger();
+    pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= batch * (gamma + 1)) return;
     const int b = i / (gamma + 1), j = i % (gamma + 1);
@@ -150,6 +182,8 @@ __global__ void iteration_uniforms_kernel(const spec_ctx::Params* __restrict__ p
 __global__ void prep_draft_first_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ length,
                                         int batch, int gamma, int max_len, int32_t* row_token, int32_t* row_pos,
                                         int32_t* row_seq, int32_t* logit_src, int32_t* logit_dst) {
+    pdl_trigger();
+    pdl_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch) return;
     const int L = length[b];
@@ -167,6 +201,8 @@ __global__ void prep_draft_first_kernel(const int32_t* __restrict__ tokens, cons
 __global__ void prep_draft_step_kernel(const int32_t* __restrict__ draft_tokens, const int32_t* __restrict__ length,
                                        int batch, int gamma, int step, int32_t* row_token, int32_t* row_pos,
                                        int32_t* row_seq, int32_t* logit_src, int32_t* logit_dst) {
+    pdl_trigger();
+    pdl_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch) return;
     row_token[b] = draft_tokens[b * gamma + step - 2];
@@ -180,6 +216,8 @@ __global__ void prep_draft_step_kernel(const int32_t* __restrict__ draft_tokens,
 __global__ void prep_verify_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ draft_tokens,
                                    const int32_t* __restrict__ length, int batch, int gamma, int max_len,
                                    int32_t* row_token, int32_t* row_pos, int32_t* row_seq) {
+    pdl_trigger();
+    pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= batch * (gamma + 1)) return;
     const int b = i / (gamma + 1), j = i % (gamma + 1);
@@ -197,6 +235,8 @@ __global__ void commit_kernel(const spec_ctx::Params* __restrict__ params, const
                               const int32_t* __restrict__ n_accepted, const int32_t* __restrict__ next_token,
                               const int32_t* __restrict__ prompt_len, int batch, int gamma, int max_len,
                               int32_t* tokens, int32_t* length, unsigned long long* counters) {
+    pdl_trigger();
+    pdl_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch) return;
     const int L = length[b];
@@ -219,39 +259,35 @@ int enqueue_iteration(spec_ctx* ctx, int batch, int gamma, float temperature) {
     const int threads = 128;
     const int blocks_b = (batch + threads - 1) / threads;
     const int blocks_bg = (batch * (gamma + 1) + threads - 1) / threads;
-    iteration_uniforms_kernel<<<blocks_bg, threads, 0, st>>>(ctx->params, ctx->length, batch, gamma, ctx->draft_u,
-                                                             ctx->accept_u, ctx->final_u);
+    SPEC_TRY(launch_pdl(iteration_uniforms_kernel, dim3(blocks_bg), dim3(threads), 0, st, ctx->params, ctx->length,
+                        batch, gamma, ctx->draft_u, ctx->accept_u, ctx->final_u));
     for (int step = 1; step <= gamma; ++step) {
         int rows;
         if (step == 1) {
-            prep_draft_first_kernel<<<blocks_b, threads, 0, st>>>(ctx->tokens, ctx->length, batch, gamma,
-                                                                  ctx->rt.max_len, ctx->row_token, ctx->row_pos,
-                                                                  ctx->row_seq, ctx->logit_src, ctx->logit_dst);
+            SPEC_TRY(launch_pdl(prep_draft_first_kernel, dim3(blocks_b), dim3(threads), 0, st, ctx->tokens, ctx->length,
+                                batch, gamma, ctx->rt.max_len, ctx->row_token, ctx->row_pos, ctx->row_seq,
+                                ctx->logit_src, ctx->logit_dst));
             rows = 2 * batch;
         } else {
-            prep_draft_step_kernel<<<blocks_b, threads, 0, st>>>(ctx->draft_tokens, ctx->length, batch, gamma, step,
-                                                                 ctx->row_token, ctx->row_pos, ctx->row_seq,
-                                                                 ctx->logit_src, ctx->logit_dst);
+            SPEC_TRY(launch_pdl(prep_draft_step_kernel, dim3(blocks_b), dim3(threads), 0, st, ctx->draft_tokens,
+                                ctx->length, batch, gamma, step, ctx->row_token, ctx->row_pos, ctx->row_seq,
+                                ctx->logit_src, ctx->logit_dst));
             rows = batch;
         }
-        SPEC_CUDA_TRY(cudaGetLastError());
-        SPEC_TRY(forward(ctx, ctx->model[1], rows, batch, ctx->logit_src, ctx->logit_dst, ctx->draft_logits));
+        SPEC_TRY(forward(ctx, ctx->model[1], batch, rows / batch, batch, ctx->logit_src, ctx->logit_dst, ctx->draft_logits));
         // x_step ~ q_step for every sequence
         SPEC_TRY(launch_sample_strided(ctx->draft_logits + static_cast<size_t>(step - 1) * vocab,
                                        static_cast<size_t>(gamma) * vocab, ctx->draft_u + (step - 1), gamma, batch,
                                        vocab, temperature, ctx->draft_tokens + (step - 1), gamma, st));
     }
-    prep_verify_kernel<<<blocks_bg, threads, 0, st>>>(ctx->tokens, ctx->draft_tokens, ctx->length, batch, gamma,
-                                                      ctx->rt.max_len, ctx->row_token, ctx->row_pos, ctx->row_seq);
-    SPEC_CUDA_TRY(cudaGetLastError());
-    SPEC_TRY(forward(ctx, ctx->model[0], batch * (gamma + 1), batch * (gamma + 1), nullptr, nullptr, ctx->target_logits));
+    SPEC_TRY(launch_pdl(prep_verify_kernel, dim3(blocks_bg), dim3(threads), 0, st, ctx->tokens, ctx->draft_tokens,
+                        ctx->length, batch, gamma, ctx->rt.max_len, ctx->row_token, ctx->row_pos, ctx->row_seq));
+    SPEC_TRY(forward(ctx, ctx->model[0], batch, gamma + 1, batch * (gamma + 1), nullptr, nullptr, ctx->target_logits));
     SPEC_TRY(launch_verify_sample(ctx->target_logits, ctx->draft_logits, ctx->draft_tokens, ctx->accept_u, ctx->final_u,
                                   batch, gamma, vocab, temperature, ctx->n_accepted, ctx->next_token, ctx->sampler_ws, st));
-    commit_kernel<<<blocks_b, threads, 0, st>>>(ctx->params, ctx->draft_tokens, ctx->n_accepted, ctx->next_token,
-                                                ctx->prompt_len, batch, gamma, ctx->rt.max_len, ctx->tokens,
-                                                ctx->length, ctx->counters);
-    SPEC_CUDA_TRY(cudaGetLastError());
-    return SPEC_OK;
+    return launch_pdl(commit_kernel, dim3(blocks_b), dim3(threads), 0, st, ctx->params, ctx->draft_tokens,
+                      ctx->n_accepted, ctx->next_token, ctx->prompt_len, batch, gamma, ctx->rt.max_len, ctx->tokens,
+                      ctx->length, ctx->counters);
 }
 
 int build_graph(spec_ctx* ctx, int batch, int gamma, float temperature) {
@@ -301,7 +337,7 @@ int feed_host_tokens(spec_ctx* ctx, int which, const int32_t* tokens, int stride
         SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_token, tok.data(), bytes, cudaMemcpyHostToDevice, ctx->stream));
         SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_pos, pos.data(), bytes, cudaMemcpyHostToDevice, ctx->stream));
         SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_seq, seq.data(), bytes, cudaMemcpyHostToDevice, ctx->stream));
-        SPEC_TRY(forward(ctx, ctx->model[which], batch * chunk, 0, nullptr, nullptr, nullptr));
+        SPEC_TRY(forward(ctx, ctx->model[which], batch, chunk, 0, nullptr, nullptr, nullptr));
         SPEC_CUDA_TRY(cudaStreamSynchronize(ctx->stream));  // the host vectors are reused
     }
     return SPEC_OK;
@@ -326,6 +362,14 @@ int init_model(spec_ctx* ctx, int which, const spec_model_cfg& cfg, const spec_w
     char* kv = nullptr;
     SPEC_TRY(dev_alloc(ctx, &kv, m.layer_stride * cfg.n_layers));
     m.kv = kv;
+    if (cfg.arch == SPEC_ARCH_LLAMA) {
+        std::vector<float2> table;
+        fill_rope_table(table, std::min(ctx->rt.max_len, cfg.max_positions), cfg.d_head, cfg.rope_base);
+        float2* dev = nullptr;
+        SPEC_TRY(dev_alloc(ctx, &dev, table.size()));
+        SPEC_CUDA_TRY(cudaMemcpy(dev, table.data(), table.size() * sizeof(float2), cudaMemcpyHostToDevice));
+        m.rope_table = dev;
+    }
     return SPEC_OK;
 }
 
@@ -392,6 +436,16 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     SPEC_ALLOC(att, R * att);
     SPEC_ALLOC(u, R * fin);
     SPEC_ALLOC(f, R * ff);
+    {
+        size_t attn = 0;
+        for (int i = 0; i < (ctx->has_draft ? 2 : 1); ++i) {
+            const Model& m = ctx->model[i];
+            for (int b = 1; b <= rt.max_batch; ++b)
+                attn = std::max(attn, attention_partial_elems(ctx->max_rows, m.cfg.n_heads, m.cfg.d_head,
+                                                              attention_slices(b, m.cfg.n_kv_heads, rt.max_len)));
+        }
+        SPEC_ALLOC(attn_part, attn);
+    }
     SPEC_ALLOC(target_logits, R * V);
     SPEC_ALLOC(draft_logits, std::max<size_t>(B * G, 1) * V);
     {
@@ -597,7 +651,7 @@ extern "C" int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* toke
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_token, tok.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_pos, pos.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_seq, seq.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
-    SPEC_TRY(forward(ctx, m, n, n, nullptr, nullptr, logits));
+    SPEC_TRY(forward(ctx, m, batch, rows, n, nullptr, nullptr, logits));
     SPEC_CUDA_TRY(cudaStreamSynchronize(st));
     if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
     for (int b = 0; b < batch; ++b) ctx->cached[which][b] += rows;

@@ -50,6 +50,8 @@ __global__ void __launch_bounds__(32 * kGemmWarps)
 gemm_rows_kernel(const float* __restrict__ x, const WT* __restrict__ w, const float* residual,
                  const int32_t* __restrict__ dst_rows, int n_rows, int n_out, int k, float* y) {
     constexpr int E = WVec<WT>::kElems;
+    pdl_trigger();
+    pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n0 = (blockIdx.x * kGemmWarps + warp) * NPW;
     const int r0 = blockIdx.y * MT;
@@ -97,20 +99,20 @@ gemm_rows_kernel(const float* __restrict__ x, const WT* __restrict__ w, const fl
 }
 
 template <typename WT, int MT, int NPW>
-void launch(const float* x, const void* w, const float* residual, const int32_t* dst_rows, int n_rows, int n_out,
+int launch(const float* x, const void* w, const float* residual, const int32_t* dst_rows, int n_rows, int n_out,
             int k, float* y, cudaStream_t stream) {
     const dim3 grid((n_out + kGemmWarps * NPW - 1) / (kGemmWarps * NPW), (n_rows + MT - 1) / MT);
-    gemm_rows_kernel<WT, MT, NPW><<<grid, 32 * kGemmWarps, 0, stream>>>(x, static_cast<const WT*>(w), residual,
-                                                                       dst_rows, n_rows, n_out, k, y);
+    return launch_pdl(gemm_rows_kernel<WT, MT, NPW>, grid, dim3(32 * kGemmWarps), 0, stream, x,
+                      static_cast<const WT*>(w), residual, dst_rows, n_rows, n_out, k, y);
 }
 
 template <typename WT>
-void dispatch(const float* x, const void* w, const float* residual, const int32_t* dst_rows, int n_rows, int n_out,
+int dispatch(const float* x, const void* w, const float* residual, const int32_t* dst_rows, int n_rows, int n_out,
               int k, float* y, cudaStream_t stream) {
-    if (n_rows <= 2) launch<WT, 2, 4>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
-    else if (n_rows <= 4) launch<WT, 4, 4>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
-    else if (n_rows <= 8) launch<WT, 8, 4>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
-    else launch<WT, 16, 2>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
+    if (n_rows <= 2) return launch<WT, 2, 4>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
+    if (n_rows <= 4) return launch<WT, 4, 4>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
+    if (n_rows <= 8) return launch<WT, 8, 4>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
+    return launch<WT, 16, 2>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
 }
 
 }  // namespace
@@ -119,10 +121,8 @@ int launch_gemm_rows(const float* x, const void* w, bool w_bf16, const float* re
                      int n_rows, int n_out, int k, float* y, cudaStream_t stream) {
     if (n_rows <= 0) return SPEC_OK;
     if (k % 8 != 0) return fail(SPEC_ERR_BAD_CONFIG, "gemm: inner dimension %d is not a multiple of 8", k);
-    if (w_bf16) dispatch<__nv_bfloat16>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
-    else dispatch<float>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
-    SPEC_CUDA_TRY(cudaGetLastError());
-    return SPEC_OK;
+    if (w_bf16) return dispatch<__nv_bfloat16>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
+    return dispatch<float>(x, w, residual, dst_rows, n_rows, n_out, k, y, stream);
 }
 
 }  // namespace spec

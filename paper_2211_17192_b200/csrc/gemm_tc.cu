@@ -144,6 +144,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     uint64_t* acc_bar = empty_bar + S::kStages;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_bar + 1);
 
+    pdl_trigger();  // the next kernel may start its own prologue
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x, split = blockIdx.y, splits = gridDim.y, tok0 = blockIdx.z * N_TOK;
     const int kb0 = static_cast<int>(static_cast<long long>(k_blocks) * split / splits);
@@ -170,9 +171,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
     if (warp == 0 && lane == 0) {
         // ---- producer: weights and both activation terms of one k-block per stage ----
-        for (int kb = kb0; kb < kb1; ++kb) {
-            const int it = kb - kb0, s = it % S::kStages;
-            if (it >= S::kStages && !mbar_wait(&empty_bar[s], ((it / S::kStages) - 1) & 1)) { ok = false; break; }
+        // The weights do not depend on the kernel before this one: the first
+        // ring of weight tiles is already streaming while that kernel finishes.
+        const int total = kb1 - kb0;
+        const int ahead = min(total, S::kStages);
+        for (int it = 0; it < ahead; ++it) {
+            mbar_expect_tx(&full_bar[it], S::kStageBytes);
+            tma_load_2d(smem + it * S::kStageBytes, &map_w, (kb0 + it) * kTileK, tile * kTileM, &full_bar[it]);
+        }
+        pdl_wait();  // the activations are written by the previous kernel
+        for (int it = 0; it < ahead; ++it) {
+            uint8_t* stage = smem + it * S::kStageBytes;
+            tma_load_2d(stage + S::kABytes, &map_hi, (kb0 + it) * kTileK, tok0, &full_bar[it]);
+            tma_load_2d(stage + S::kABytes + S::kBBytes, &map_lo, (kb0 + it) * kTileK, tok0, &full_bar[it]);
+        }
+        for (int it = ahead; it < total; ++it) {
+            const int kb = kb0 + it, s = it % S::kStages;
+            if (!mbar_wait(&empty_bar[s], ((it / S::kStages) - 1) & 1)) { ok = false; break; }
             uint8_t* stage = smem + s * S::kStageBytes;
             mbar_expect_tx(&full_bar[s], S::kStageBytes);
             tma_load_2d(stage, &map_w, kb * kTileK, tile * kTileM, &full_bar[s]);
@@ -201,6 +216,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         mma_commit(acc_bar);  // accumulator complete
     }
     __syncwarp();
+    pdl_wait();  // (already satisfied for the producer) nothing below may overtake the previous kernel
 
     // ---- epilogue: all four warps, warp w reads accumulator lanes 32w .. 32w+31 ----
     if (kb1 > kb0) {
@@ -242,6 +258,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 // x (fp32) -> hi = bf16(x), lo = bf16(x - hi); grid-stride, 4 elements per thread
 __global__ void split_bf16_kernel(const float* __restrict__ x, size_t n, __nv_bfloat16* __restrict__ hi,
                                   __nv_bfloat16* __restrict__ lo) {
+    pdl_trigger();
+    pdl_wait();
     for (size_t i = (blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x) * 4; i < n;
          i += static_cast<size_t>(gridDim.x) * blockDim.x * 4) {
         const float4 v = *reinterpret_cast<const float4*>(x + i);
@@ -260,6 +278,8 @@ __global__ void split_bf16_kernel(const float* __restrict__ x, size_t n, __nv_bf
 // y[dst(r)][n] = sum_s partial[s][r][n] (+ residual[r][n]), splits added in index order
 __global__ void reduce_partials_kernel(const float* __restrict__ partial, int splits, int n_rows, int n_out,
                                        const float* residual, const int32_t* __restrict__ dst_rows, float* y) {
+    pdl_trigger();
+    pdl_wait();
     const size_t total = static_cast<size_t>(n_rows) * n_out;
     for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < total;
          i += static_cast<size_t>(gridDim.x) * blockDim.x) {
@@ -338,9 +358,8 @@ int launch_tc(const CUtensorMap& mw, const CUtensorMap& mhi, const CUtensorMap& 
         configured = true;
     }
     const dim3 grid((n_out + kTileM - 1) / kTileM, splits, (n_rows + N_TOK - 1) / N_TOK);
-    gemm_tc_kernel<N_TOK><<<grid, kThreads, Smem<N_TOK>::kTotal, stream>>>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks);
-    SPEC_CUDA_TRY(cudaGetLastError());
-    return SPEC_OK;
+    return launch_pdl(gemm_tc_kernel<N_TOK>, grid, dim3(kThreads), Smem<N_TOK>::kTotal, stream, mw, mhi, mlo, partial,
+                      n_out, n_rows, k_blocks);
 }
 
 }  // namespace
@@ -376,16 +395,13 @@ size_t gemm_tc_partial_elems(int n_out, int k, int n_rows) {
 
 int launch_split_bf16(const float* x, size_t n, __nv_bfloat16* hi, __nv_bfloat16* lo, cudaStream_t stream) {
     const int blocks = static_cast<int>(std::min<size_t>((n / 4 + 255) / 256, 148 * 8));
-    split_bf16_kernel<<<std::max(blocks, 1), 256, 0, stream>>>(x, n, hi, lo);
-    SPEC_CUDA_TRY(cudaGetLastError());
-    return SPEC_OK;
+    return launch_pdl(split_bf16_kernel, dim3(std::max(blocks, 1)), dim3(256), 0, stream, x, n, hi, lo);
 }
 
-// y[dst(r)] = x[r] . W^T (+ residual[r]) with x already split into hi + lo
-// (both [hi_rows, k] bf16, the first n_rows rows valid).
-int launch_gemm_tc(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, const float* residual,
-                   const int32_t* dst_rows, int n_rows, int n_out, int k, float* partial, float* y,
-                   cudaStream_t stream) {
+// partial[s][r][n] for x already split into hi + lo (both [hi_rows, k] bf16, the
+// first n_rows rows valid); s < gemm_tc_splits(n_out, k, n_rows).
+int launch_gemm_tc_partials(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, int n_rows,
+                            int n_out, int k, float* partial, cudaStream_t stream) {
     if (n_rows <= 0) return SPEC_OK;
     if (k % 8 != 0) return fail(SPEC_ERR_BAD_CONFIG, "gemm: inner dimension %d is not a multiple of 8", k);
     const int n_tok = gemm_tc_token_tile(n_rows);
@@ -397,17 +413,25 @@ int launch_gemm_tc(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows
     if (status == SPEC_OK) status = cached_map(lo, hi_rows, k, n_tok, &mlo);
     if (status != SPEC_OK) return status;
     switch (n_tok) {
-        case 16: status = launch_tc<16>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream); break;
-        case 32: status = launch_tc<32>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream); break;
-        case 64: status = launch_tc<64>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream); break;
-        default: status = launch_tc<128>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream); break;
+        case 16: return launch_tc<16>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream);
+        case 32: return launch_tc<32>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream);
+        case 64: return launch_tc<64>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream);
+        default: return launch_tc<128>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream);
     }
+}
+
+// y[dst(r)] = x[r] . W^T (+ residual[r]): the partial sums, then their reduction.
+int launch_gemm_tc(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, const float* residual,
+                   const int32_t* dst_rows, int n_rows, int n_out, int k, float* partial, float* y,
+                   cudaStream_t stream) {
+    if (n_rows <= 0) return SPEC_OK;
+    const int status = launch_gemm_tc_partials(hi, lo, hi_rows, w, n_rows, n_out, k, partial, stream);
     if (status != SPEC_OK) return status;
+    const int splits = gemm_tc_splits(n_out, k, n_rows);
     const size_t total = static_cast<size_t>(n_rows) * n_out;
     const int blocks = static_cast<int>(std::min<size_t>((total + 255) / 256, 148 * 8));
-    reduce_partials_kernel<<<blocks, 256, 0, stream>>>(partial, splits, n_rows, n_out, residual, dst_rows, y);
-    SPEC_CUDA_TRY(cudaGetLastError());
-    return SPEC_OK;
+    return launch_pdl(reduce_partials_kernel, dim3(blocks), dim3(256), 0, stream, static_cast<const float*>(partial),
+                      splits, n_rows, n_out, residual, dst_rows, y);
 }
 
 // Non-zero if a tensor-core GEMM gave up on a bounded wait since the last call.

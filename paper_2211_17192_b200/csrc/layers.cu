@@ -1,7 +1,11 @@
-// The small kernels of a decoder block: embedding gather, RMSNorm, rotary
-// positions + K/V append into the paged cache, FFN activations.  All of them
-// move O(rows * d) bytes and exist to keep the residual stream in fp32 around
-// the weight-streaming GEMMs.
+// The small kernels between the weight-streaming GEMMs of a decoder block.
+// Each one also finishes the GEMM before it (adds up the split-K partial sums
+// in a fixed order, adds the residual) and prepares the input of the GEMM after
+// it (fp32, and/or split into two bf16 terms for the tensor-core path), so that
+// a block is nine launches: norm, qkv GEMM, rope + KV append, attention,
+// out-projection GEMM, norm, FFN-in GEMM, activation, FFN-out GEMM.
+#include <cmath>
+
 #include "model.cuh"
 
 namespace spec {
@@ -11,10 +15,26 @@ __device__ __forceinline__ float load_elem(const void* base, size_t i, bool bf16
     return bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(base)[i]) : static_cast<const float*>(base)[i];
 }
 
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi): 16 mantissa bits survive.
+__device__ __forceinline__ void store_split(__nv_bfloat16* hi, __nv_bfloat16* lo, size_t i, float x) {
+    const __nv_bfloat16 h = __float2bfloat16_rn(x);
+    hi[i] = h;
+    lo[i] = __float2bfloat16_rn(x - __bfloat162float(h));
+}
+
+// sum of the split-K partial results of element i, in split order
+__device__ __forceinline__ float sum_partials(const float* __restrict__ partial, int splits, size_t stride, size_t i) {
+    float acc = partial[i];
+    for (int s = 1; s < splits; ++s) acc += partial[static_cast<size_t>(s) * stride + i];
+    return acc;
+}
+
 // grid = rows, block = 128
 __global__ void embed_kernel(const void* __restrict__ tok_emb, const void* __restrict__ pos_emb, bool bf16,
                              bool add_pos, const int32_t* __restrict__ token, const int32_t* __restrict__ pos, int d,
                              int vocab, int max_positions, float* __restrict__ h) {
+    pdl_trigger();
+    pdl_wait();
     const int r = blockIdx.x;
     const int t = min(max(token[r], 0), vocab - 1);
     const int p = min(max(pos[r], 0), max_positions - 1);
@@ -25,73 +45,112 @@ __global__ void embed_kernel(const void* __restrict__ tok_emb, const void* __res
     }
 }
 
-// grid = rows, block = 256; d is a multiple of 4
-__global__ void rmsnorm_kernel(const float* __restrict__ in, const float* __restrict__ gain,
-                               const int32_t* __restrict__ src_rows, int d, float eps, float* __restrict__ out) {
-    __shared__ float red[8];
+// grid = rows, block = kNormThreads; d is a multiple of 4.  Row r of the output is
+// RMSNorm(h[src(r)]) * gain.  If `partial` is given, h[r] += sum of the partial
+// results first (the residual add of the GEMM that produced them) and the new h
+// is stored.  A thread holds up to kNormPerThread float4 of the row in registers,
+// so every load of the row and of its partial sums is in flight at once.
+constexpr int kNormThreads = 1024;
+constexpr int kNormPerThread = 4;  // rows up to 16384 wide
+
+__global__ void __launch_bounds__(kNormThreads)
+norm_kernel(float* h, const float* __restrict__ partial, int splits, int n_rows, const float* __restrict__ gain,
+            const int32_t* __restrict__ src_rows, int d, float eps, float* __restrict__ out,
+            __nv_bfloat16* __restrict__ out_hi, __nv_bfloat16* __restrict__ out_lo) {
+    __shared__ float red[kNormThreads / 32];
+    pdl_trigger();
+    pdl_wait();
     const int r = blockIdx.x;
-    const float4* x = reinterpret_cast<const float4*>(in + static_cast<size_t>(src_rows ? src_rows[r] : r) * d);
-    const float4* g = reinterpret_cast<const float4*>(gain);
-    float4* y = reinterpret_cast<float4*>(out + static_cast<size_t>(r) * d);
+    const size_t src = static_cast<size_t>(src_rows ? src_rows[r] : r) * d;
+    const size_t stride = static_cast<size_t>(n_rows) * d;
+    const int groups = d / 4;
+    float4 v[kNormPerThread];
     float ss = 0.0f;
-    for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
-        const float4 v = x[i];
-        ss += (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
+#pragma unroll
+    for (int j = 0; j < kNormPerThread; ++j) {
+        const int g = threadIdx.x + j * kNormThreads;
+        v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (g < groups) {
+            v[j] = *reinterpret_cast<const float4*>(h + src + 4 * g);
+            if (partial) {
+                for (int s = 0; s < splits; ++s) {
+                    const float4 p = *reinterpret_cast<const float4*>(partial + s * stride + src + 4 * g);
+                    v[j].x += p.x; v[j].y += p.y; v[j].z += p.z; v[j].w += p.w;
+                }
+                *reinterpret_cast<float4*>(h + src + 4 * g) = v[j];
+            }
+            ss += (v[j].x * v[j].x + v[j].y * v[j].y) + (v[j].z * v[j].z + v[j].w * v[j].w);
+        }
     }
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
     __syncthreads();
     float total = 0.0f;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) total += red[i];
+    for (int i = 0; i < kNormThreads / 32; ++i) total += red[i];
     const float scale = rsqrtf(total / static_cast<float>(d) + eps);
-    for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
-        const float4 v = x[i];
-        const float4 gg = g[i];
-        y[i] = make_float4(v.x * scale * gg.x, v.y * scale * gg.y, v.z * scale * gg.z, v.w * scale * gg.w);
+    const size_t dst = static_cast<size_t>(r) * d;
+#pragma unroll
+    for (int j = 0; j < kNormPerThread; ++j) {
+        const int g = threadIdx.x + j * kNormThreads;
+        if (g < groups) {
+            const float4 gg = *reinterpret_cast<const float4*>(gain + 4 * g);
+            const float y[4] = {v[j].x * scale * gg.x, v[j].y * scale * gg.y, v[j].z * scale * gg.z, v[j].w * scale * gg.w};
+            if (out) *reinterpret_cast<float4*>(out + dst + 4 * g) = make_float4(y[0], y[1], y[2], y[3]);
+            if (out_hi) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) store_split(out_hi, out_lo, dst + 4 * g + e, y[e]);
+            }
+        }
     }
 }
 
-// grid = rows, block = 128.  qkv row layout: [q heads | k heads | v heads], d_head each.
+// grid = (n_heads + 2 n_kv_heads, rows), block = d_head / 2.  qkv row layout:
+// [q heads | k heads | v heads], d_head each.  A CTA finishes one head of one row
+// of the qkv GEMM (optional partial sums), applies rotary positions (q and k
+// heads; thread j owns the pair j, j + d_head/2), leaves q in `qkv` for the
+// attention kernel, and appends K or V to the paged cache.
 template <typename KV>
-__global__ void rope_append_kernel(float* __restrict__ qkv, const int32_t* __restrict__ pos,
-                                   const int32_t* __restrict__ seq, int n_heads, int n_kv_heads, int d_head,
-                                   bool rotary, float rope_base, KV* __restrict__ kv_layer,
-                                   const int32_t* __restrict__ page_table, int pages_per_seq, int page_size) {
-    const int r = blockIdx.x;
+__global__ void qkv_kernel(float* __restrict__ qkv, const float* __restrict__ partial, int splits, int n_rows,
+                           const int32_t* __restrict__ pos, const int32_t* __restrict__ seq, int n_heads,
+                           int n_kv_heads, int d_head, const float2* __restrict__ rope_table,
+                           KV* __restrict__ kv_layer, const int32_t* __restrict__ page_table, int pages_per_seq,
+                           int page_size) {
+    pdl_trigger();
+    pdl_wait();
+    const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x;
     const int p = pos[r];
-    if (p < 0) return;
     const int half = d_head / 2;
-    float* row = qkv + static_cast<size_t>(r) * (n_heads + 2 * n_kv_heads) * d_head;
-    if (rotary) {
-        // q heads and k heads are contiguous: (n_heads + n_kv_heads) * half rotations
-        const int pairs = (n_heads + n_kv_heads) * half;
-        for (int i = threadIdx.x; i < pairs; i += blockDim.x) {
-            const int head = i / half, j = i % half;
-            // angle = position * base^(-2j / d_head), evaluated in double so that
-            // large positions do not lose the fractional turn
-            const double inv_freq = pow(static_cast<double>(rope_base), -2.0 * j / static_cast<double>(d_head));
-            double s, c;
-            sincos(static_cast<double>(p) * inv_freq, &s, &c);
-            float* hp = row + head * d_head;
-            const float x1 = hp[j], x2 = hp[j + half];
-            hp[j] = x1 * static_cast<float>(c) - x2 * static_cast<float>(s);
-            hp[j + half] = x2 * static_cast<float>(c) + x1 * static_cast<float>(s);
-        }
-        __syncthreads();
+    const int width = (n_heads + 2 * n_kv_heads) * d_head;
+    const size_t at = static_cast<size_t>(r) * width + head * d_head;
+    float x1, x2;
+    if (partial) {
+        const size_t stride = static_cast<size_t>(n_rows) * width;
+        x1 = sum_partials(partial, splits, stride, at + j);
+        x2 = sum_partials(partial, splits, stride, at + j + half);
+    } else {
+        x1 = qkv[at + j];
+        x2 = qkv[at + j + half];
     }
+    const bool is_q = head < n_heads, is_k = !is_q && head < n_heads + n_kv_heads;
+    if (rope_table && p >= 0 && (is_q || is_k)) {
+        const float2 t = rope_table[static_cast<size_t>(p) * half + j];  // (cos, sin) of position p
+        const float y1 = x1 * t.x - x2 * t.y, y2 = x2 * t.x + x1 * t.y;
+        x1 = y1;
+        x2 = y2;
+    }
+    if (is_q) {
+        qkv[at + j] = x1;
+        qkv[at + j + half] = x2;
+        return;
+    }
+    if (p < 0) return;  // inactive row: nothing is cached
+    const int kv_head = is_k ? head - n_heads : head - n_heads - n_kv_heads;
     const int page = page_table[seq[r] * pages_per_seq + p / page_size];
-    const int slot = p % page_size;
-    const int kv_dim = n_kv_heads * d_head;
-    const float* k = row + n_heads * d_head;
-    const float* v = k + kv_dim;
-    for (int i = threadIdx.x; i < kv_dim; i += blockDim.x) {
-        const int head = i / d_head, e = i % d_head;
-        const size_t base = ((static_cast<size_t>(page) * 2) * n_kv_heads + head) * page_size + slot;
-        const size_t v_off = static_cast<size_t>(n_kv_heads) * page_size;
-        kv_layer[base * d_head + e] = static_cast<KV>(k[i]);
-        kv_layer[(base + v_off) * d_head + e] = static_cast<KV>(v[i]);
-    }
+    const size_t block = (static_cast<size_t>(page) * 2 + (is_k ? 0 : 1)) * n_kv_heads + kv_head;
+    KV* dst = kv_layer + (block * page_size + p % page_size) * d_head;
+    dst[j] = static_cast<KV>(x1);
+    dst[j + half] = static_cast<KV>(x2);
 }
 
 __device__ __forceinline__ float gelu_tanh(float x) {
@@ -101,58 +160,85 @@ __device__ __forceinline__ float gelu_tanh(float x) {
 
 __device__ __forceinline__ float silu(float x) { return x / (1.0f + expf(-x)); }
 
-__global__ void ffn_act_kernel(const float* __restrict__ u, int n_rows, int d_ff, int ffn, float* __restrict__ f) {
+// f = gelu(u)  |  gelu(gate) * up  |  silu(gate) * up, with u either given in
+// full or as the partial sums of the FFN-in GEMM.
+__global__ void ffn_act_kernel(const float* __restrict__ u, const float* __restrict__ partial, int splits, int n_rows,
+                               int d_ff, int ffn, float* __restrict__ f, __nv_bfloat16* __restrict__ f_hi,
+                               __nv_bfloat16* __restrict__ f_lo) {
+    pdl_trigger();
+    pdl_wait();
     const size_t total = static_cast<size_t>(n_rows) * d_ff;
+    const int width = ffn == SPEC_FFN_GELU ? d_ff : 2 * d_ff;
+    const size_t stride = static_cast<size_t>(n_rows) * width;
     for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < total;
          i += static_cast<size_t>(gridDim.x) * blockDim.x) {
         const size_t r = i / d_ff, c = i % d_ff;
+        const size_t a = r * width + c;
+        float y;
         if (ffn == SPEC_FFN_GELU) {
-            f[i] = gelu_tanh(u[i]);
+            y = gelu_tanh(partial ? sum_partials(partial, splits, stride, a) : u[a]);
         } else {
-            const float gate = u[r * 2 * d_ff + c], up = u[r * 2 * d_ff + d_ff + c];
-            f[i] = (ffn == SPEC_FFN_SWIGLU ? silu(gate) : gelu_tanh(gate)) * up;
+            const float gate = partial ? sum_partials(partial, splits, stride, a) : u[a];
+            const float up = partial ? sum_partials(partial, splits, stride, a + d_ff) : u[a + d_ff];
+            y = (ffn == SPEC_FFN_SWIGLU ? silu(gate) : gelu_tanh(gate)) * up;
         }
+        if (f) f[i] = y;
+        if (f_hi) store_split(f_hi, f_lo, i, y);
     }
 }
 
 }  // namespace
 
 int launch_embed(const Model& m, const RowMeta& rows, int n_rows, float* h, cudaStream_t stream) {
-    embed_kernel<<<n_rows, 128, 0, stream>>>(m.tok_emb, m.pos_emb, m.bf16(), m.cfg.arch == SPEC_ARCH_GPT, rows.token,
-                                             rows.pos, m.cfg.d_model, m.cfg.vocab, m.cfg.max_positions, h);
-    SPEC_CUDA_TRY(cudaGetLastError());
-    return SPEC_OK;
+    return launch_pdl(embed_kernel, dim3(n_rows), dim3(128), 0, stream, m.tok_emb, m.pos_emb, m.bf16(),
+                      m.cfg.arch == SPEC_ARCH_GPT, rows.token, rows.pos, m.cfg.d_model, m.cfg.vocab,
+                      m.cfg.max_positions, h);
 }
 
-int launch_rmsnorm(const float* in, const float* gain, const int32_t* src_rows, int n_rows, int d, float eps,
-                   float* out, cudaStream_t stream) {
-    rmsnorm_kernel<<<n_rows, 256, 0, stream>>>(in, gain, src_rows, d, eps, out);
-    SPEC_CUDA_TRY(cudaGetLastError());
-    return SPEC_OK;
+int launch_norm(float* h, const float* partial, int splits, int rows_total, const float* gain, const int32_t* src_rows,
+                int n_rows, int d, float eps, float* out, __nv_bfloat16* out_hi, __nv_bfloat16* out_lo,
+                cudaStream_t stream) {
+    if (d % 4 || d > 4 * kNormThreads * kNormPerThread)
+        return fail(SPEC_ERR_BAD_CONFIG, "norm: width %d is not a multiple of 4 or exceeds %d", d, 4 * kNormThreads * kNormPerThread);
+    return launch_pdl(norm_kernel, dim3(n_rows), dim3(kNormThreads), 0, stream, h, partial, splits, rows_total, gain,
+                      src_rows, d, eps, out, out_hi, out_lo);
 }
 
-int launch_rope_append(const Model& m, int layer, const RowMeta& rows, int n_rows, float* qkv,
-                       const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream) {
+int launch_qkv(const Model& m, int layer, const RowMeta& rows, int n_rows, float* qkv, const float* partial,
+               int splits, const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream) {
     char* kv_layer = static_cast<char*>(m.kv) + static_cast<size_t>(layer) * m.layer_stride;
-    const bool rotary = m.cfg.arch == SPEC_ARCH_LLAMA;
+    const float2* table = m.cfg.arch == SPEC_ARCH_LLAMA ? m.rope_table : nullptr;
+    const dim3 grid(m.cfg.n_heads + 2 * m.cfg.n_kv_heads, n_rows);
+    const dim3 block(m.cfg.d_head / 2);
     if (m.kv_elem_bytes == 2)
-        rope_append_kernel<__nv_bfloat16><<<n_rows, 128, 0, stream>>>(
-            qkv, rows.pos, rows.seq, m.cfg.n_heads, m.cfg.n_kv_heads, m.cfg.d_head, rotary, m.cfg.rope_base,
-            reinterpret_cast<__nv_bfloat16*>(kv_layer), page_table, pages_per_seq, page_size);
-    else
-        rope_append_kernel<float><<<n_rows, 128, 0, stream>>>(
-            qkv, rows.pos, rows.seq, m.cfg.n_heads, m.cfg.n_kv_heads, m.cfg.d_head, rotary, m.cfg.rope_base,
-            reinterpret_cast<float*>(kv_layer), page_table, pages_per_seq, page_size);
-    SPEC_CUDA_TRY(cudaGetLastError());
-    return SPEC_OK;
+        return launch_pdl(qkv_kernel<__nv_bfloat16>, grid, block, 0, stream, qkv, partial, splits, n_rows, rows.pos,
+                          rows.seq, m.cfg.n_heads, m.cfg.n_kv_heads, m.cfg.d_head, table,
+                          reinterpret_cast<__nv_bfloat16*>(kv_layer), page_table, pages_per_seq, page_size);
+    return launch_pdl(qkv_kernel<float>, grid, block, 0, stream, qkv, partial, splits, n_rows, rows.pos, rows.seq,
+                      m.cfg.n_heads, m.cfg.n_kv_heads, m.cfg.d_head, table, reinterpret_cast<float*>(kv_layer),
+                      page_table, pages_per_seq, page_size);
 }
 
-int launch_ffn_act(const float* u, int n_rows, int d_ff, int ffn, float* f, cudaStream_t stream) {
+int launch_ffn_act(const float* u, const float* partial, int splits, int n_rows, int d_ff, int ffn, float* f,
+                   __nv_bfloat16* f_hi, __nv_bfloat16* f_lo, cudaStream_t stream) {
     const size_t total = static_cast<size_t>(n_rows) * d_ff;
     const int blocks = static_cast<int>(std::min<size_t>((total + 255) / 256, 148 * 8));
-    ffn_act_kernel<<<blocks, 256, 0, stream>>>(u, n_rows, d_ff, ffn, f);
-    SPEC_CUDA_TRY(cudaGetLastError());
-    return SPEC_OK;
+    return launch_pdl(ffn_act_kernel, dim3(blocks), dim3(256), 0, stream, u, partial, splits, n_rows, d_ff, ffn, f,
+                      f_hi, f_lo);
+}
+
+// (cos, sin) of position * base^(-2j / d_head), evaluated in double precision on
+// the host and rounded once to fp32: [positions][d_head / 2].
+void fill_rope_table(std::vector<float2>& table, int positions, int d_head, double base) {
+    const int half = d_head / 2;
+    table.resize(static_cast<size_t>(positions) * half);
+    for (int j = 0; j < half; ++j) {
+        const double inv_freq = std::pow(base, -2.0 * j / static_cast<double>(d_head));
+        for (int p = 0; p < positions; ++p) {
+            const double a = static_cast<double>(p) * inv_freq;
+            table[static_cast<size_t>(p) * half + j] = make_float2(static_cast<float>(std::cos(a)), static_cast<float>(std::sin(a)));
+        }
+    }
 }
 
 }  // namespace spec

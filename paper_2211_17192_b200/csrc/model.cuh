@@ -23,6 +23,7 @@ struct Model {
     void* kv = nullptr;
     size_t layer_stride = 0;
     int kv_elem_bytes = 4;
+    const float2* rope_table = nullptr;  // Llama: (cos, sin) [positions][d_head / 2], owned
 
     int q_dim() const { return cfg.n_heads * cfg.d_head; }
     int kv_dim() const { return cfg.n_kv_heads * cfg.d_head; }
@@ -44,35 +45,48 @@ struct RowMeta {
 // h[r] = tok_emb[token[r]] (+ pos_emb[pos[r]] for GPT), fp32.
 int launch_embed(const Model& m, const RowMeta& rows, int n_rows, float* h, cudaStream_t stream);
 
-// out[i] = in[src[i]] / sqrt(mean(in[src[i]]^2) + eps) * gain   (src == nullptr: identity)
-int launch_rmsnorm(const float* in, const float* gain, const int32_t* src_rows, int n_rows, int d, float eps,
-                   float* out, cudaStream_t stream);
+// Row i of the output = RMSNorm(h[src(i)]) * gain, as fp32 (`out`) and/or as two
+// bf16 terms (`out_hi`, `out_lo`).  If `partial` is given (split-K results of
+// the GEMM before, [splits][rows_total][d]) it is first added into h.
+int launch_norm(float* h, const float* partial, int splits, int rows_total, const float* gain, const int32_t* src_rows,
+                int n_rows, int d, float eps, float* out, __nv_bfloat16* out_hi, __nv_bfloat16* out_lo,
+                cudaStream_t stream);
 
-// y[dst(r)] = x[r] . W^T (+ residual[r]);  W is [n_out, k] row-major in fp32 or bf16.
+// y[dst(r)] = x[r] . W^T (+ residual[r]) on the FMA pipes;  W is [n_out, k] row-major in fp32 or bf16.
 // dst(r) = dst_rows ? dst_rows[r] : r.  y and residual may alias.
 int launch_gemm_rows(const float* x, const void* w, bool w_bf16, const float* residual, const int32_t* dst_rows,
                      int n_rows, int n_out, int k, float* y, cudaStream_t stream);
 
-// Tensor-core path for bf16 weights (gemm_tc.cu): x is first split into two bf16
-// terms, partial sums of the split-K grid are reduced in a fixed order.
+// Tensor-core path for bf16 weights (gemm_tc.cu): x arrives as two bf16 terms;
+// launch_gemm_tc_partials leaves the split-K partial sums [splits][n_rows][n_out]
+// for the next kernel to add up, launch_gemm_tc adds them up itself.
 int gemm_tc_splits(int n_out, int k, int n_rows);
 size_t gemm_tc_partial_elems(int n_out, int k, int n_rows);
 int launch_split_bf16(const float* x, size_t n, __nv_bfloat16* hi, __nv_bfloat16* lo, cudaStream_t stream);
+int launch_gemm_tc_partials(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, int n_rows,
+                            int n_out, int k, float* partial, cudaStream_t stream);
 int launch_gemm_tc(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, const float* residual,
                    const int32_t* dst_rows, int n_rows, int n_out, int k, float* partial, float* y,
                    cudaStream_t stream);
 int gemm_tc_take_error();
 
-// Rotary positions on q and k (Llama), then K,V rows of every active row into the paged cache.
-int launch_rope_append(const Model& m, int layer, const RowMeta& rows, int n_rows, float* qkv,
-                       const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream);
+// Finishes the qkv GEMM (optional partial sums), rotary positions on q and k
+// (Llama), K,V rows of every active row into the paged cache; q stays in `qkv`.
+int launch_qkv(const Model& m, int layer, const RowMeta& rows, int n_rows, float* qkv, const float* partial,
+               int splits, const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream);
+void fill_rope_table(std::vector<float2>& table, int positions, int d_head, double base);
 
-// att[r, h] = softmax(q_r,h . K / sqrt(d_head)) V over cached positions <= pos[r] of sequence seq[r].
-int launch_attention(const Model& m, int layer, const RowMeta& rows, int n_rows, const float* qkv, float* att,
+// att[r, h] = softmax(q_r,h . K / sqrt(d_head)) V over cached positions <= pos[r];
+// rows of sequence b are rows b*m_rows .. of the pass.  Output as fp32 and/or two bf16 terms.
+int attention_slices(int batch, int n_kv_heads, int max_len);
+size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices);
+int launch_attention(const Model& m, int layer, const RowMeta& rows, int batch, int m_rows, int slices,
+                     const float* qkv, float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo,
                      const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream);
 
-// f = gelu(u)  |  gelu(u[:, :F]) * u[:, F:]  |  silu(u[:, :F]) * u[:, F:]
-int launch_ffn_act(const float* u, int n_rows, int d_ff, int ffn, float* f, cudaStream_t stream);
+// f = gelu(u)  |  gelu(u[:, :F]) * u[:, F:]  |  silu(u[:, :F]) * u[:, F:], u given in full or as partial sums.
+int launch_ffn_act(const float* u, const float* partial, int splits, int n_rows, int d_ff, int ffn, float* f,
+                   __nv_bfloat16* f_hi, __nv_bfloat16* f_lo, cudaStream_t stream);
 
 // sampling.cu
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,

@@ -396,6 +396,8 @@ verify_stats_kernel(const float* __restrict__ target_logits, const float* __rest
     __shared__ float red[kStatWarps];
     __shared__ float red_s[kStatWarps];
     __shared__ int red_i[kStatWarps];
+    pdl_trigger();  // the finishing kernel's CTAs may take their places as this grid drains
+    pdl_wait();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chunk = blockIdx.x, chunks = gridDim.x;
     const int row = blockIdx.y, rows = gridDim.y;
@@ -474,8 +476,6 @@ verify_stats_kernel(const float* __restrict__ target_logits, const float* __rest
             *reinterpret_cast<float4*>(out) = make_float4(bm, t, xlogit, 0.0f);
         }
     }
-    // Let the finishing kernel's CTAs be scheduled as this grid drains.
-    asm volatile("griddepcontrol.launch_dependents;");
 }
 
 struct FinishShared {
@@ -516,7 +516,8 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
     int my_x = -1;
     if (tid < rows && tid != gamma)
         my_x = draft_tokens[static_cast<size_t>(b) * gamma + (tid < gamma ? tid : tid - gamma - 1)];
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    pdl_trigger();
+    pdl_wait();
 
     // merge the chunk statistics of row `tid` (four loads in flight at a time)
     if (tid < rows) {
@@ -616,6 +617,8 @@ sample_kernel(const float* __restrict__ logits, size_t logit_stride, const float
     __shared__ CdfScratch<W> cdf;
     __shared__ float s_max;
     __shared__ int s_arg;
+    pdl_trigger();
+    pdl_wait();
     const int tid = threadIdx.x;
     const Row<VEC> r = make_row<VEC>(logits + static_cast<size_t>(blockIdx.x) * logit_stride, vocab);
     const int groups = (vocab + 3) >> 2;
@@ -695,14 +698,16 @@ int launch_verify_sample(const float* target_logits, const float* draft_logits, 
     const dim3 grid(chunks, rows, batch);
     const bool vec = vocab % 4 == 0 && aligned16(target_logits) && (greedy || gamma == 0 || aligned16(draft_logits));
     const float c2 = inv_t * kLog2e;
-#define SPEC_LAUNCH_STATS(G, V) \
-    verify_stats_kernel<G, V><<<grid, kStatThreads, 0, stream>>>(target_logits, draft_logits, draft_tokens, gamma, vocab, c2, stats)
+    int status;
+#define SPEC_LAUNCH_STATS(G, V)                                                                                  \
+    status = launch_pdl(verify_stats_kernel<G, V>, grid, dim3(kStatThreads), 0, stream, target_logits, draft_logits, \
+                        draft_tokens, gamma, vocab, c2, stats)
     if (greedy && vec) SPEC_LAUNCH_STATS(true, true);
     else if (greedy) SPEC_LAUNCH_STATS(true, false);
     else if (vec) SPEC_LAUNCH_STATS(false, true);
     else SPEC_LAUNCH_STATS(false, false);
 #undef SPEC_LAUNCH_STATS
-    SPEC_CUDA_TRY(cudaGetLastError());
+    if (status != SPEC_OK) return status;
 
     // One cluster per sequence; more CTAs per cluster for longer rows.
     const int cluster_size = greedy ? 1 : finish_cluster_size(vocab);
@@ -741,13 +746,10 @@ int launch_sample_strided(const float* logits, size_t logit_stride, const float*
     const bool greedy = temperature == 0.0f;
     const float inv_t = greedy ? 0.0f : 1.0f / temperature;
     if (vocab % 4 == 0 && logit_stride % 4 == 0 && aligned16(logits))
-        sample_kernel<true><<<rows, kSampleThreads, 0, stream>>>(logits, logit_stride, uniforms, uniform_stride, vocab,
-                                                                 inv_t, greedy, tokens, token_stride);
-    else
-        sample_kernel<false><<<rows, kSampleThreads, 0, stream>>>(logits, logit_stride, uniforms, uniform_stride,
-                                                                  vocab, inv_t, greedy, tokens, token_stride);
-    SPEC_CUDA_TRY(cudaGetLastError());
-    return SPEC_OK;
+        return launch_pdl(sample_kernel<true>, dim3(rows), dim3(kSampleThreads), 0, stream, logits, logit_stride,
+                          uniforms, uniform_stride, vocab, inv_t, greedy, tokens, token_stride);
+    return launch_pdl(sample_kernel<false>, dim3(rows), dim3(kSampleThreads), 0, stream, logits, logit_stride, uniforms,
+                      uniform_stride, vocab, inv_t, greedy, tokens, token_stride);
 }
 
 int launch_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
