@@ -1,12 +1,18 @@
 """Benchmark of the speculative-decoding hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--batch B] [--gamma G] [--impl reference]
 
 Prints ONE JSON line (rank 0).  For N > 1 it is launched with torchrun, one
 process per GPU; ranks are independent replicas (the path has no exchange
 step), timed between barriers, max over ranks.
 
-Workloads
+Workloads (--workload)
+  llama7b   (default) Llama-7B-shaped bf16 target with a 160M-shaped draft, random
+            init, 1024-token prompts, batch --batch (1), gamma --gamma (2), T = 1.
+            A step is one iteration of Algorithm 1 for the whole batch: gamma
+            draft passes, one target pass over gamma+1 rows, speculative sampling,
+            commit and KV roll-back.
+  gpt97m    the paper-shaped GPT-like 97M target with its 6M draft, 8k vocabulary.
   sampler   the standalone speculative-sampling kernel: batch 64 x
             (gamma+1 = 8) x vocab 32000, T = 1, draft logits = target + N(0, s^2)
             with s rotating over {0.5, 1, 2}.  A step is one call of
@@ -180,18 +186,202 @@ class SamplerWorkload:
         xs = np.zeros((self.batch, self.gamma), dtype=np.int32)
         t0 = time.perf_counter()
         done = tokens = 0
-        while done < self.batch and (time.perf_counter() - t0 < budget_s or done < 2):
-            b = done
+        while time.perf_counter() - t0 < budget_s or done < 2:
+            b = done % self.batch
             for i in range(self.gamma):
                 xs[b, i] = oracle_sampling.sample_token(ql[b, i], draw[b * self.gamma + i], self.temperature)[0]
             res = oracle_sampling.verify_step(tl[b], ql[b], xs[b], us[b], self.temperature)
             tokens += res.n_accepted + 1
             done += 1
         dt = time.perf_counter() - t0
-        return tokens / dt, f"{done} of {self.batch} sequences of one batch (draft draws + verify), {dt:.1f} s"
+        return tokens / dt, f"{done} sequences drawn from one batch of {self.batch} (draft draws + verify), {dt:.1f} s"
 
 
-WORKLOADS = {"sampler": SamplerWorkload}
+# --------------------------------------------------------------------------- #
+# workload: speculative decoding of a model pair (Algorithm 1, device-resident loop)
+# --------------------------------------------------------------------------- #
+def gpu_weights(cfg, seed, device):
+    """Seeded random-init weights drawn on the GPU with torch's generator (matrices
+    N(0, 0.02^2), head N(0, head_std^2), gains 1; bf16 models stored as bf16)."""
+    import torch
+    from paper_2211_17192_b200 import workloads
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    out = {}
+    for name, shape, kind in workloads.tensor_shapes(cfg):
+        if kind == "gain":
+            out[name] = torch.ones(shape, device=device)
+            continue
+        std = cfg["head_std"] if kind == "head" else workloads.INIT_STD
+        t = torch.randn(shape, device=device, generator=g, dtype=torch.float32) * std
+        out[name] = t.to(torch.bfloat16) if cfg["dtype"] == "bf16" else t
+    return out
+
+
+def weight_stream_bytes(cfg):
+    """Bytes of one pass over the model: every block matrix and the LM head once."""
+    from paper_2211_17192_b200 import workloads
+    elem = 2 if cfg["dtype"] == "bf16" else 4
+    total = 0
+    for name, shape, kind in workloads.tensor_shapes(cfg):
+        if kind == "gain" or name in ("pos_emb",) or (name == "tok_emb" and not cfg["tied"]):
+            continue
+        total += int(np.prod(shape)) * elem
+    return total
+
+
+class GenerationWorkload:
+    dtype = "bf16"
+
+    def __init__(self, name, target, draft, batch, prompt_len, n_new, gamma, temperature=1.0):
+        self.name, self.target_name, self.draft_name = name, target, draft
+        self.batch, self.prompt_len, self.n_new, self.gamma, self.temperature = batch, prompt_len, n_new, gamma, temperature
+
+    def description(self):
+        return {"workload": self.name, "target": self.target_name, "draft": self.draft_name, "batch": self.batch,
+                "prompt_len": self.prompt_len, "n_new": self.n_new, "gamma": self.gamma,
+                "temperature": self.temperature, "kv_dtype": "fp32",
+                "l2": "one pass streams the target's weights (>> 126 MB L2) from HBM",
+                "parallelism": "replicas"}
+
+    def prepare(self, rank, device, iterations):
+        import torch
+        from paper_2211_17192_b200 import binding, workloads
+        self.torch, self.binding, self.device = torch, binding, device
+        self.tcfg = workloads.model_config(self.target_name)
+        self.dcfg = workloads.model_config(self.draft_name)
+        self.dtype = "bf16" if self.tcfg["dtype"] == "bf16" else "f32"
+        self.tw = gpu_weights(self.tcfg, 100 + rank, device)
+        self.dw = gpu_weights(self.dcfg, 200 + rank, device)
+        grow = max(self.n_new, iterations * (self.gamma + 1) + 64)
+        self.max_len = self.prompt_len + grow + self.gamma + 2
+        self.engine = binding.Engine(self.tcfg, self.tw, self.dcfg, self.dw, max_batch=self.batch, max_len=self.max_len,
+                                     page_size=64, max_gamma=max(self.gamma, 1))
+        self.prompts = [workloads.make_prompt(1000 * rank + b, self.prompt_len, self.tcfg["vocab"]) for b in range(self.batch)]
+        self.budget_tokens = grow
+
+    def launches_per_iteration(self):
+        fwd = lambda cfg: 1 + 10 * cfg["n_layers"] + 3
+        return 1 + self.gamma * (1 + fwd(self.dcfg) + 1) + 1 + fwd(self.tcfg) + 2 + 1
+
+    def timed_decode(self, warmup, steps, gamma):
+        """Device time of `steps` iterations after `warmup` untimed ones (prompt pass untimed)."""
+        self.engine.begin(self.prompts, self.budget_tokens, gamma, self.temperature, 7)
+        _, before = self.engine.step(warmup)
+        _, after = self.engine.step(steps)
+        tokens = after["tokens"] - before["tokens"]
+        stats = {k: after[k] - before[k] for k in ("iterations", "tokens", "tests_evaluated", "tests_passed")}
+        return tokens, after["decode_ms"], stats
+
+    def e2e(self, calls):
+        """The public call with host buffers: prompts in, tokens out, prompt pass included."""
+        t0 = time.perf_counter()
+        tokens = 0
+        for i in range(calls):
+            out, _ = self.engine.generate(self.prompts, self.n_new, self.gamma, self.temperature, 11 + i)
+            tokens += out.size
+        return tokens, time.perf_counter() - t0
+
+    def e2e_bytes(self):
+        return self.batch * self.prompt_len * 4 + self.batch * 4, self.batch * self.n_new * 4
+
+    def pass_times(self, repeats=20):
+        """Wall time of single passes through the teacher-forced entry point: the target
+        on 1 and on gamma+1 rows, the draft on 1 row, at the prompt's context length."""
+        eng, torch = self.engine, self.torch
+        tok = np.stack([p[: self.prompt_len - 1] for p in self.prompts])
+        def timed(which, rows):
+            best = []
+            for _ in range(repeats):
+                eng.truncate(which, [self.prompt_len - 1] * self.batch)
+                t0 = time.perf_counter()
+                eng.forward_logits(which, np.zeros((self.batch, rows), dtype=np.int32))
+                best.append(time.perf_counter() - t0)
+            return statistics.median(best) * 1e3
+        eng.reset()
+        chunk = 64
+        for which in (0, 1):
+            for c0 in range(0, tok.shape[1], chunk):
+                eng.forward_logits(which, tok[:, c0:c0 + chunk])
+        return {"target_1row_ms": timed(0, 1), "target_rows_ms": timed(0, self.gamma + 1), "draft_1row_ms": timed(1, 1)}
+
+    def gemm_roofline(self, rows):
+        """The weight-streaming GEMM alone: every block matrix and the head of the
+        target once through spec_linear at `rows` rows, captured in a CUDA graph and
+        timed with events on its stream."""
+        torch, binding = self.torch, self.binding
+        mats = [(n, t) for n, t in self.tw.items() if t.dim() == 2 and n not in ("tok_emb", "pos_emb")]
+        if self.tcfg["tied"]:
+            mats.append(("head", self.tw["tok_emb"]))
+        kmax = max(t.shape[1] for _, t in mats)
+        x = torch.randn(rows, kmax, device=self.device)
+        ys = {n: torch.empty(rows, t.shape[0], device=self.device) for n, t in mats}
+        need = max(binding.spec_linear_workspace_bytes(rows, t.shape[0], t.shape[1]) for _, t in mats)
+        ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        xs = {k: x[:, :k].contiguous() for k in {t.shape[1] for _, t in mats}}
+        stream = torch.cuda.Stream(self.device)
+        with torch.cuda.stream(stream):
+            def sweep():
+                for n, t in mats:
+                    binding.spec_linear(xs[t.shape[1]], t, "auto", ys[n], ws)
+            sweep()
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                sweep()
+            graph.replay()
+            stream.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            graph.replay()
+            b.record(stream)
+            stream.synchronize()
+        nbytes = sum(t.numel() * t.element_size() for _, t in mats)
+        return nbytes, a.elapsed_time(b), len(mats)
+
+    def cpu_sample(self, budget_s):
+        """The oracle on a bounded sample: both models at full width and reduced depth
+        (2 layers each), a short prompt, a few iterations; extrapolated to the full
+        depth by streamed weight bytes."""
+        from oracle import generate as oracle_generate
+        from oracle.decoder import Decoder
+        from paper_2211_17192_b200 import workloads
+        small_t = workloads.scaled_config(self.tcfg, n_layers=min(2, self.tcfg["n_layers"]))
+        small_d = workloads.scaled_config(self.dcfg, n_layers=min(2, self.dcfg["n_layers"]))
+        dtype = np.float32 if self.tcfg["d_model"] >= 2048 else np.float64
+        target = Decoder(small_t, workloads.make_weights(small_t, 1), dtype=dtype)
+        draft = Decoder(small_d, workloads.make_weights(small_d, 2), dtype=dtype)
+        prompt = workloads.make_prompt(3, 32, self.tcfg["vocab"])
+        t0 = time.perf_counter()
+        tokens = iters = 0
+        n_new = 4 * (self.gamma + 1)
+        while time.perf_counter() - t0 < budget_s or iters == 0:
+            res = oracle_generate.speculative_generate(target, draft, prompt, n_new, self.gamma, self.temperature, seed=iters)
+            tokens += len(res.tokens)
+            iters += len(res.iterations)
+        dt = time.perf_counter() - t0
+        full = weight_stream_bytes(self.tcfg) + self.gamma * weight_stream_bytes(self.dcfg)
+        small = weight_stream_bytes(small_t) + self.gamma * weight_stream_bytes(small_d)
+        value = tokens / dt * small / full
+        sample = (f"{iters} iterations of Algorithm 1, batch 1, 32-token prompt, both models at full width and "
+                  f"{small_t['n_layers']}+{small_d['n_layers']} layers in {np.dtype(dtype).name}, {dt:.1f} s; "
+                  f"scaled by streamed weight bytes ({small / full:.3f}) to the full depth")
+        return value, sample
+
+
+def make_workload(args):
+    if args.workload == "sampler":
+        return SamplerWorkload()
+    batch = args.batch or 1
+    if args.workload == "gpt97m":
+        return GenerationWorkload("gpt97m_6m_b1", "gpt97m_target", "gpt6m_draft", batch, 128, 512, args.gamma or 5,
+                                  args.temperature)
+    gamma = args.gamma or 2
+    return GenerationWorkload(f"llama7b_160m_b{batch}_g{gamma}", "llama7b_target", "llama160m_draft", batch, 1024, 256,
+                              gamma, args.temperature)
+
+
+WORKLOAD_NAMES = ["llama7b", "gpt97m", "sampler"]
 
 
 # --------------------------------------------------------------------------- #
@@ -220,11 +410,12 @@ def run_reference(args, wl):
         return
     values = []
     sample = ""
+    per_step = max(1.0, 60.0 / max(1, args.steps + args.warmup))
     for _ in range(args.warmup):
-        wl.cpu_sample(0.5)
+        wl.cpu_sample(per_step)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        v, sample = wl.cpu_sample(max(1.0, 60.0 / max(1, args.steps)))
+        v, sample = wl.cpu_sample(per_step)
         values.append(v)
     dt = time.perf_counter() - t0
     value = statistics.mean(values)
@@ -233,24 +424,144 @@ def run_reference(args, wl):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1000.0 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": wl.description(),
-        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cpu_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(out))
 
 
+def run_sampler(args, wl, torch, device, local, barrier):
+    """Timed region: K calls of spec_verify_sample captured in one CUDA graph."""
+    wl.prepare(int(os.environ.get("RANK", "0")), device)
+    stream = torch.cuda.Stream(device)
+    with torch.cuda.stream(stream):
+        for i in range(args.warmup):
+            wl.step(i)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        launches = 0
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(args.steps):
+                launches += wl.step(args.warmup + i)
+        graph.replay()  # untimed: uploads the graph
+        stream.synchronize()
+        clocks = ClockSampler(local)
+        clocks.start()
+        time.sleep(0.15)
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        w0 = time.time()
+        start.record(stream)
+        graph.replay()
+        stop.record(stream)
+        barrier()
+        elapsed_ms = start.elapsed_time(stop)
+        t_end = time.time() + 0.5  # keep the GPU under this load while the clocks are sampled
+        while time.time() < t_end:
+            graph.replay()
+        stream.synchronize()
+        clock_info = clocks.stop(w0, time.time())
+        tokens = wl.tokens_emitted(args.warmup, args.steps)
+    for i in range(3):
+        wl.e2e_step(i)
+    barrier()
+    e0 = time.perf_counter()
+    e2e_tokens = 0
+    for i in range(args.steps):
+        e2e_tokens += wl.e2e_step(i)
+    barrier()
+    e2e_s = time.perf_counter() - e0
+    peak, peak_kind = load_peaks()
+    launch_s = elapsed_ms / args.steps / 1e3
+    achieved = wl.algorithmic_bytes() / launch_s / 1e9
+    extras = {
+        "roofline": {"bound": "hbm", "kernel": "verify_stats_kernel+verify_finish_kernel", "achieved": achieved,
+                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "frac_of_nominal_8tbs": achieved / 8000.0, "traffic": 122.98e6,
+                     "traffic_note": "dram bytes read per launch from the ncu capture under profiles/",
+                     "algorithmic_bytes_per_launch": wl.algorithmic_bytes(), "launch_us": 1e6 * launch_s},
+    }
+    return dict(tokens=tokens, elapsed_ms=elapsed_ms, e2e_tokens=e2e_tokens, e2e_s=e2e_s, launches=launches,
+                clocks=clock_info, extras=extras)
+
+
+def run_generation(args, wl, torch, device, local, barrier):
+    """Timed region: K iterations of Algorithm 1 (gamma draft passes, one target pass
+    over gamma+1 rows, speculative sampling, commit and roll-back), replayed as a
+    CUDA graph per iteration by the library and timed with events on its stream."""
+    from oracle import analysis  # closed forms only, for the report (rank 0)
+    rank = int(os.environ.get("RANK", "0"))
+    wl.prepare(rank, device, args.warmup + args.steps)
+    clocks = ClockSampler(local)
+    clocks.start()
+    time.sleep(0.15)
+    barrier()
+    w0 = time.time()
+    tokens, elapsed_ms, stats = wl.timed_decode(args.warmup, args.steps, wl.gamma)
+    barrier()
+    clock_info = clocks.stop(w0, time.time())
+    base_tokens, base_ms, _ = wl.timed_decode(args.warmup, args.steps, 0)  # target-only, same kernels
+    for _ in range(1):
+        wl.e2e(1)
+    barrier()
+    e2e_tokens, e2e_s = wl.e2e(3)
+    barrier()
+    extras = {}
+    if rank == 0:
+        peak, peak_kind = load_peaks()
+        rows = wl.batch * (wl.gamma + 1)
+        nbytes, gemm_ms, n_mats = wl.gemm_roofline(rows)
+        achieved = nbytes / (gemm_ms / 1e3) / 1e9
+        times = wl.pass_times()
+        alpha = stats["tests_passed"] / max(1, stats["tests_evaluated"])
+        tok_per_iter = stats["tokens"] / max(1, stats["iterations"])
+        c = times["draft_1row_ms"] / times["target_1row_ms"]
+        kv_bytes = wl.batch * wl.prompt_len * 2 * wl.tcfg["n_layers"] * wl.tcfg["n_kv_heads"] * wl.tcfg["d_head"] * 4
+        pass_bytes = weight_stream_bytes(wl.tcfg) + kv_bytes
+        extras = {
+            "speedup_vs_target_only": (tokens / elapsed_ms) / (base_tokens / base_ms),
+            "target_only_tokens_per_s": base_tokens / (base_ms / 1e3),
+            "alpha": alpha, "tokens_per_iteration": tok_per_iter, "c": c,
+            "kappa": times["target_rows_ms"] / times["target_1row_ms"],
+            "closed_form": {"theorem_3_8": analysis.walltime_improvement(alpha, wl.gamma, c),
+                            "expected_tokens_eq_1": analysis.expected_tokens(alpha, wl.gamma),
+                            "generalised": analysis.generalised_speedup(tok_per_iter, times["target_1row_ms"],
+                                                                        times["target_rows_ms"], times["draft_1row_ms"],
+                                                                        wl.gamma)},
+            "pass_ms": times,
+            "verify_pass": {"bytes": pass_bytes, "ms": times["target_rows_ms"],
+                            "gbs": pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9,
+                            "frac": pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9 / peak,
+                            "note": "weights + fp32 KV of the prompt, one pass over gamma+1 rows, host-timed call"},
+            "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbs": achieved / 8000.0,
+                         "traffic": None, "algorithmic_bytes_per_launch": nbytes / n_mats,
+                         "launch_us": 1e3 * gemm_ms / n_mats,
+                         "note": f"all {n_mats} weight matrices of the target once at {rows} rows through spec_linear "
+                                 "(bf16 split + GEMM + split-K reduction), CUDA graph, events on its stream"},
+        }
+    launches = wl.launches_per_iteration() * args.steps
+    return dict(tokens=tokens, elapsed_ms=elapsed_ms, e2e_tokens=e2e_tokens, e2e_s=e2e_s, launches=launches,
+                clocks=clock_info, extras=extras)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=6)
-    ap.add_argument("--workload", default="sampler", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="llama7b", choices=WORKLOAD_NAMES)
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--gamma", type=int, default=None)
+    ap.add_argument("--temperature", type=float, default=1.0)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
-    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for cpu_baseline")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 300 if args.workload == "sampler" else 100
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
-    wl = WORKLOADS[args.workload]()
+    wl = make_workload(args)
 
     if args.impl == "reference":
         run_reference(args, wl)
@@ -280,54 +591,9 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    wl.prepare(rank, device)
-    stream = torch.cuda.Stream(device)
-    with torch.cuda.stream(stream):
-        for i in range(args.warmup):
-            wl.step(i)
-        stream.synchronize()
-        # The K timed steps are captured once in a CUDA graph so that the device
-        # never waits for the Python launch loop; the timed region is one replay.
-        graph = torch.cuda.CUDAGraph()
-        launches = 0
-        with torch.cuda.graph(graph, stream=stream):
-            for i in range(args.steps):
-                launches += wl.step(args.warmup + i)
-        graph.replay()  # untimed: uploads the graph
-        stream.synchronize()
-
-        clocks = ClockSampler(local)
-        clocks.start()
-        time.sleep(0.15)
-        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        w0 = time.time()
-        start.record(stream)
-        graph.replay()
-        stop.record(stream)
-        barrier()
-        w1 = time.time()
-        elapsed_ms = start.elapsed_time(stop)
-        # keep the clocks sampler busy long enough to see the GPU under this load
-        t_end = time.time() + 0.5
-        while time.time() < t_end:
-            graph.replay()
-        stream.synchronize()
-        w1 = time.time()
-        clock_info = clocks.stop(w0, w1)
-        tokens = wl.tokens_emitted(args.warmup, args.steps)
-    kernel_ms = [elapsed_ms / args.steps]
-
-    # end-to-end leg: pinned host buffers in, host results out
-    for i in range(3):
-        wl.e2e_step(i)
-    barrier()
-    e0 = time.perf_counter()
-    e2e_tokens = 0
-    for i in range(args.steps):
-        e2e_tokens += wl.e2e_step(i)
-    barrier()
-    e2e_s = time.perf_counter() - e0
+    runner = run_sampler if args.workload == "sampler" else run_generation
+    res = runner(args, wl, torch, device, local, barrier)
+    tokens, elapsed_ms, e2e_tokens, e2e_s, launches = (res[k] for k in ("tokens", "elapsed_ms", "e2e_tokens", "e2e_s", "launches"))
 
     if world > 1:
         t = torch.tensor([elapsed_ms, e2e_s], dtype=torch.float64, device=device)
@@ -338,9 +604,6 @@ def main():
         tokens, e2e_tokens, launches = int(c[0]), int(c[1]), int(c[2])
 
     if rank == 0:
-        peak, peak_kind = load_peaks()
-        avg_kernel_s = statistics.mean(kernel_ms) / 1000.0
-        achieved = wl.algorithmic_bytes() / avg_kernel_s / 1e9
         cpu_value, cpu_sample = wl.cpu_sample(args.cpu_budget) if world == 1 else (None, "skipped for N > 1")
         h2d, d2h = wl.e2e_bytes()
         out = {
@@ -348,19 +611,14 @@ def main():
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
             "data": "synthetic", "config": wl.description(),
-            "clocks": clock_info,
+            "clocks": res["clocks"],
             "e2e": {"value": e2e_tokens / e2e_s, "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h},
             "gpu_launches": launches,
-            "roofline": {"bound": "hbm", "kernel": "verify_stats_kernel+verify_finish_kernel", "achieved": achieved,
-                         "peak": peak,
-                         "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                         "frac_of_nominal_8tbs": achieved / 8000.0, "traffic": None,
-                         "algorithmic_bytes_per_launch": wl.algorithmic_bytes(),
-                         "launch_us": 1e3 * statistics.mean(kernel_ms)},
-            "cpu_baseline": {"value": cpu_value, "unit": "tokens/s", "cores": 1, "kind": "oracle",
-                             "sample": cpu_sample},
         }
+        out.update(res["extras"])
+        out["cpu_baseline"] = {"value": cpu_value, "unit": "tokens/s", "cores": cpu_threads(), "kind": "oracle",
+                               "sample": cpu_sample}
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

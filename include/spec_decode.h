@@ -238,6 +238,22 @@ int spec_generate(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_le
                   int batch, int n_new, int gamma, float temperature, uint64_t seed,
                   int32_t* out_tokens, spec_stats* stats);
 
+/* The same generation in phases, for callers that interleave other work or
+ * time the decode loop: spec_begin validates the request, uploads the prompts
+ * and runs the prompt pass (arguments as for spec_generate); spec_step runs
+ * `iterations` iterations of Algorithm 1 for the whole batch (sequences that
+ * already have n_new tokens are frozen), blocks until they are done and reports
+ * in *remaining (may be NULL) the largest number of tokens any sequence still
+ * lacks; *stats (may be NULL) gets the counters since spec_begin, with
+ * decode_ms the device time of this call alone.  spec_read_tokens copies the
+ * n_new tokens of every sequence to HOST int32 [batch, n_new] (entries not yet
+ * generated are unspecified).  A teacher-forced diagnostic call ends the
+ * generation in progress. */
+int spec_begin(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride,
+               int batch, int n_new, int gamma, float temperature, uint64_t seed);
+int spec_step(spec_ctx* ctx, int iterations, int* remaining, spec_stats* stats);
+int spec_read_tokens(spec_ctx* ctx, int32_t* out_tokens);
+
 /* Diagnostics for parity tests: teacher-forced forward passes on the KV caches.
  * spec_reset forgets every cached row.  spec_forward_logits feeds, for each
  * of `batch` sequences, `rows` tokens at positions cached_len[b].. of model

@@ -232,6 +232,12 @@ def _declare_engine(h):
     h.spec_generate.restype = c.c_int
     h.spec_generate.argtypes = [vp, vp, vp, c.c_int, c.c_int, c.c_int, c.c_int, c.c_float, c.c_uint64, vp,
                                 c.POINTER(_Stats)]
+    h.spec_begin.restype = c.c_int
+    h.spec_begin.argtypes = [vp, vp, vp, c.c_int, c.c_int, c.c_int, c.c_int, c.c_float, c.c_uint64]
+    h.spec_step.restype = c.c_int
+    h.spec_step.argtypes = [vp, c.c_int, c.POINTER(c.c_int), c.POINTER(_Stats)]
+    h.spec_read_tokens.restype = c.c_int
+    h.spec_read_tokens.argtypes = [vp, vp]
     h.spec_reset.restype = c.c_int
     h.spec_reset.argtypes = [vp]
     h.spec_truncate.restype = c.c_int
@@ -307,6 +313,36 @@ class Engine:
             self.close()
         except Exception:
             pass
+
+    def _pack_prompts(self, prompts):
+        np = self._np
+        stride = max(len(p) for p in prompts)
+        flat = np.zeros((len(prompts), stride), dtype=np.int32)
+        lens = np.zeros(len(prompts), dtype=np.int32)
+        for b, p in enumerate(prompts):
+            flat[b, : len(p)] = p
+            lens[b] = len(p)
+        return flat, lens, stride
+
+    def begin(self, prompts, n_new, gamma, temperature, seed):
+        """Prompt pass of a generation that `step` then advances."""
+        flat, lens, stride = self._pack_prompts(prompts)
+        _check(lib().spec_begin(self._ctx, flat.ctypes.data, lens.ctypes.data, stride, len(prompts), n_new, gamma,
+                                float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF))
+        self._session = (len(prompts), n_new)
+
+    def step(self, iterations):
+        """`iterations` iterations of Algorithm 1; returns (remaining, stats dict)."""
+        left = ctypes.c_int()
+        st = _Stats()
+        _check(lib().spec_step(self._ctx, iterations, ctypes.byref(left), ctypes.byref(st)))
+        return left.value, {name: getattr(st, name) for name, _ in _Stats._fields_}
+
+    def read_tokens(self):
+        batch, n_new = self._session
+        out = self._np.zeros((batch, n_new), dtype=self._np.int32)
+        _check(lib().spec_read_tokens(self._ctx, out.ctypes.data))
+        return out
 
     def generate(self, prompts, n_new, gamma, temperature, seed):
         """Speculative decoding (gamma = 0: target-only decoding).  `prompts` is a

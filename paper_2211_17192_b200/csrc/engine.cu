@@ -44,6 +44,12 @@ struct spec_ctx {
     int graph_batch = -1, graph_gamma = -1;
     float graph_temperature = -1.0f;
 
+    // generation in progress (spec_begin / spec_generate)
+    int session_batch = 0, session_gamma = 0, session_n_new = 0;
+    long long session_replays = 0;
+    float session_prefill_ms = 0.0f;
+    std::vector<int32_t> session_prompt_len;
+
     // host-side cached lengths for the diagnostics
     std::vector<int32_t> cached[2];
     std::vector<void*> allocations;
@@ -522,28 +528,32 @@ extern "C" void spec_free(spec_ctx* ctx) {
     delete ctx;
 }
 
-extern "C" int spec_generate(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride,
-                             int batch, int n_new, int gamma, float temperature, uint64_t seed, int32_t* out_tokens,
-                             spec_stats* stats) {
-    if (!ctx || !prompt || !prompt_len || !out_tokens) return fail(SPEC_ERR_BAD_ARG, "spec_generate: null pointer");
+namespace {
+
+// Validates a generation request, uploads the prompts, runs the prompt pass of
+// both models and prepares the iteration graph.
+int begin_session(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride, int batch,
+                  int n_new, int gamma, float temperature, uint64_t seed) {
+    if (!ctx || !prompt || !prompt_len) return fail(SPEC_ERR_BAD_ARG, "generation: null pointer");
     if (batch < 1 || n_new < 1 || gamma < 0 || prompt_stride < 1 || !(temperature >= 0.0f) || !std::isfinite(temperature))
-        return fail(SPEC_ERR_BAD_ARG, "spec_generate: batch=%d n_new=%d gamma=%d temperature=%g", batch, n_new, gamma, temperature);
+        return fail(SPEC_ERR_BAD_ARG, "generation: batch=%d n_new=%d gamma=%d temperature=%g", batch, n_new, gamma, temperature);
     if (batch > ctx->rt.max_batch || gamma > ctx->rt.max_gamma)
-        return fail(SPEC_ERR_CAPACITY, "spec_generate: batch %d / gamma %d exceed the context's limits (%d / %d)", batch, gamma, ctx->rt.max_batch, ctx->rt.max_gamma);
-    if (gamma > 0 && !ctx->has_draft) return fail(SPEC_ERR_BAD_CONFIG, "spec_generate: gamma > 0 needs a draft model");
+        return fail(SPEC_ERR_CAPACITY, "generation: batch %d / gamma %d exceed the context's limits (%d / %d)", batch, gamma, ctx->rt.max_batch, ctx->rt.max_gamma);
+    if (gamma > 0 && !ctx->has_draft) return fail(SPEC_ERR_BAD_CONFIG, "generation: gamma > 0 needs a draft model");
     int limit = std::min(ctx->rt.max_len, ctx->model[0].cfg.max_positions);
     if (gamma > 0) limit = std::min(limit, ctx->model[1].cfg.max_positions);
     for (int b = 0; b < batch; ++b) {
-        if (prompt_len[b] < 1 || prompt_len[b] > prompt_stride) return fail(SPEC_ERR_BAD_ARG, "spec_generate: prompt_len[%d]=%d", b, prompt_len[b]);
+        if (prompt_len[b] < 1 || prompt_len[b] > prompt_stride) return fail(SPEC_ERR_BAD_ARG, "generation: prompt_len[%d]=%d", b, prompt_len[b]);
         if (prompt_len[b] + n_new + gamma + 1 > limit)
-            return fail(SPEC_ERR_CAPACITY, "spec_generate: sequence %d needs %d positions, limit %d", b, prompt_len[b] + n_new + gamma + 1, limit);
+            return fail(SPEC_ERR_CAPACITY, "generation: sequence %d needs %d positions, limit %d", b, prompt_len[b] + n_new + gamma + 1, limit);
         for (int i = 0; i < prompt_len[b]; ++i) {
             const int32_t t = prompt[static_cast<size_t>(b) * prompt_stride + i];
-            if (t < 0 || t >= ctx->model[0].cfg.vocab) return fail(SPEC_ERR_BAD_ARG, "spec_generate: token %d out of range", t);
+            if (t < 0 || t >= ctx->model[0].cfg.vocab) return fail(SPEC_ERR_BAD_ARG, "generation: token %d out of range", t);
         }
     }
     cudaStream_t st = ctx->stream;
     const int max_len = ctx->rt.max_len;
+    ctx->session_batch = 0;
 
     // upload prompts and state
     std::vector<int32_t> host_tokens(static_cast<size_t>(batch) * max_len, 0);
@@ -563,48 +573,103 @@ extern "C" int spec_generate(spec_ctx* ctx, const int32_t* prompt, const int32_t
     SPEC_TRY(feed_host_tokens(ctx, 0, prompt, prompt_stride, from, to, batch));
     if (gamma > 0) SPEC_TRY(feed_host_tokens(ctx, 1, prompt, prompt_stride, from, to, batch));
     SPEC_CUDA_TRY(cudaEventRecord(ctx->ev[1], st));
-
-    // decode loop: the iteration graph is replayed in bursts; after each burst the
-    // host reads the committed lengths.  A burst is as long as the iterations that
-    // are certainly needed (every iteration emits at most gamma + 1 tokens).
     SPEC_TRY(build_graph(ctx, batch, gamma, temperature));
-    std::vector<int32_t> lengths(batch);
-    long long replays = 0;
-    int remaining = n_new;
-    while (remaining > 0) {
-        const int burst = (remaining + gamma) / (gamma + 1);
-        for (int i = 0; i < burst; ++i) SPEC_CUDA_TRY(cudaGraphLaunch(ctx->graph, st));
-        replays += burst;
-        SPEC_CUDA_TRY(cudaMemcpyAsync(lengths.data(), ctx->length, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-        SPEC_CUDA_TRY(cudaStreamSynchronize(st));
-        remaining = 0;
-        for (int b = 0; b < batch; ++b) remaining = std::max(remaining, n_new - (lengths[b] - prompt_len[b]));
-    }
-    SPEC_CUDA_TRY(cudaEventRecord(ctx->ev[2], st));
-
-    SPEC_CUDA_TRY(cudaMemcpyAsync(host_tokens.data(), ctx->tokens, host_tokens.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-    unsigned long long counters[4];
-    SPEC_CUDA_TRY(cudaMemcpyAsync(counters, ctx->counters, sizeof(counters), cudaMemcpyDeviceToHost, st));
-    SPEC_CUDA_TRY(cudaStreamSynchronize(st));
-    if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
-    for (int b = 0; b < batch; ++b)
-        std::memcpy(out_tokens + static_cast<size_t>(b) * n_new, &host_tokens[static_cast<size_t>(b) * max_len + prompt_len[b]], n_new * sizeof(int32_t));
+    SPEC_CUDA_TRY(cudaStreamSynchronize(st));  // host_tokens goes out of scope
+    float pre = 0.0f;
+    cudaEventElapsedTime(&pre, ctx->ev[0], ctx->ev[1]);
+    ctx->session_prefill_ms = pre;
+    ctx->session_batch = batch;
+    ctx->session_gamma = gamma;
+    ctx->session_n_new = n_new;
+    ctx->session_replays = 0;
+    ctx->session_prompt_len.assign(prompt_len, prompt_len + batch);
     // the diagnostics' view of the caches is stale now
     std::fill(ctx->cached[0].begin(), ctx->cached[0].end(), 0);
     std::fill(ctx->cached[1].begin(), ctx->cached[1].end(), 0);
-    if (stats) {
-        float pre = 0.0f, dec = 0.0f;
-        cudaEventElapsedTime(&pre, ctx->ev[0], ctx->ev[1]);
-        cudaEventElapsedTime(&dec, ctx->ev[1], ctx->ev[2]);
-        stats->iterations = static_cast<int64_t>(counters[0]);
-        stats->tokens = static_cast<int64_t>(counters[1]);
-        stats->tests_evaluated = static_cast<int64_t>(counters[2]);
-        stats->tests_passed = static_cast<int64_t>(counters[3]);
-        stats->target_passes = replays;
-        stats->draft_passes = replays * gamma;
-        stats->prefill_ms = pre;
-        stats->decode_ms = dec;
+    return SPEC_OK;
+}
+
+// Replays the iteration graph `iterations` times; returns the device time and
+// the largest number of tokens any sequence still lacks.
+int run_iterations(spec_ctx* ctx, int iterations, float* elapsed_ms, int* remaining) {
+    cudaStream_t st = ctx->stream;
+    const int batch = ctx->session_batch;
+    std::vector<int32_t> lengths(batch);
+    SPEC_CUDA_TRY(cudaEventRecord(ctx->ev[1], st));
+    for (int i = 0; i < iterations; ++i) SPEC_CUDA_TRY(cudaGraphLaunch(ctx->graph, st));
+    SPEC_CUDA_TRY(cudaEventRecord(ctx->ev[2], st));
+    ctx->session_replays += iterations;
+    SPEC_CUDA_TRY(cudaMemcpyAsync(lengths.data(), ctx->length, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+    if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
+    SPEC_CUDA_TRY(cudaEventElapsedTime(elapsed_ms, ctx->ev[1], ctx->ev[2]));
+    *remaining = 0;
+    for (int b = 0; b < batch; ++b)
+        *remaining = std::max(*remaining, ctx->session_n_new - (lengths[b] - ctx->session_prompt_len[b]));
+    return SPEC_OK;
+}
+
+int fill_stats(spec_ctx* ctx, double decode_ms, spec_stats* stats) {
+    unsigned long long counters[4];
+    SPEC_CUDA_TRY(cudaMemcpy(counters, ctx->counters, sizeof(counters), cudaMemcpyDeviceToHost));
+    stats->iterations = static_cast<int64_t>(counters[0]);
+    stats->tokens = static_cast<int64_t>(counters[1]);
+    stats->tests_evaluated = static_cast<int64_t>(counters[2]);
+    stats->tests_passed = static_cast<int64_t>(counters[3]);
+    stats->target_passes = ctx->session_replays;
+    stats->draft_passes = ctx->session_replays * ctx->session_gamma;
+    stats->prefill_ms = ctx->session_prefill_ms;
+    stats->decode_ms = decode_ms;
+    return SPEC_OK;
+}
+
+}  // namespace
+
+extern "C" int spec_generate(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride,
+                             int batch, int n_new, int gamma, float temperature, uint64_t seed, int32_t* out_tokens,
+                             spec_stats* stats) {
+    if (!out_tokens) return fail(SPEC_ERR_BAD_ARG, "spec_generate: null pointer");
+    SPEC_TRY(begin_session(ctx, prompt, prompt_len, prompt_stride, batch, n_new, gamma, temperature, seed));
+    // decode loop: the iteration graph is replayed in bursts; after each burst the
+    // host reads the committed lengths.  A burst is as long as the iterations that
+    // are certainly needed (every iteration emits at most gamma + 1 tokens).
+    double decode_ms = 0.0;
+    int remaining = n_new;
+    while (remaining > 0) {
+        float ms = 0.0f;
+        SPEC_TRY(run_iterations(ctx, (remaining + gamma) / (gamma + 1), &ms, &remaining));
+        decode_ms += ms;
     }
+    SPEC_TRY(spec_read_tokens(ctx, out_tokens));
+    if (stats) SPEC_TRY(fill_stats(ctx, decode_ms, stats));
+    return SPEC_OK;
+}
+
+extern "C" int spec_begin(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride,
+                          int batch, int n_new, int gamma, float temperature, uint64_t seed) {
+    return begin_session(ctx, prompt, prompt_len, prompt_stride, batch, n_new, gamma, temperature, seed);
+}
+
+extern "C" int spec_step(spec_ctx* ctx, int iterations, int* remaining, spec_stats* stats) {
+    if (!ctx || iterations < 1) return fail(SPEC_ERR_BAD_ARG, "spec_step: bad argument");
+    if (ctx->session_batch < 1) return fail(SPEC_ERR_BAD_ARG, "spec_step: no generation in progress (call spec_begin)");
+    float ms = 0.0f;
+    int left = 0;
+    SPEC_TRY(run_iterations(ctx, iterations, &ms, &left));
+    if (remaining) *remaining = left;
+    if (stats) SPEC_TRY(fill_stats(ctx, ms, stats));
+    return SPEC_OK;
+}
+
+extern "C" int spec_read_tokens(spec_ctx* ctx, int32_t* out_tokens) {
+    if (!ctx || !out_tokens) return fail(SPEC_ERR_BAD_ARG, "spec_read_tokens: null pointer");
+    if (ctx->session_batch < 1) return fail(SPEC_ERR_BAD_ARG, "spec_read_tokens: no generation in progress");
+    const int batch = ctx->session_batch, n_new = ctx->session_n_new, max_len = ctx->rt.max_len;
+    std::vector<int32_t> host_tokens(static_cast<size_t>(batch) * max_len);
+    SPEC_CUDA_TRY(cudaMemcpyAsync(host_tokens.data(), ctx->tokens, host_tokens.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
+    SPEC_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+    for (int b = 0; b < batch; ++b)
+        std::memcpy(out_tokens + static_cast<size_t>(b) * n_new, &host_tokens[static_cast<size_t>(b) * max_len + ctx->session_prompt_len[b]], n_new * sizeof(int32_t));
     return SPEC_OK;
 }
 
@@ -612,6 +677,7 @@ extern "C" int spec_reset(spec_ctx* ctx) {
     if (!ctx) return fail(SPEC_ERR_BAD_ARG, "spec_reset: null context");
     std::fill(ctx->cached[0].begin(), ctx->cached[0].end(), 0);
     std::fill(ctx->cached[1].begin(), ctx->cached[1].end(), 0);
+    ctx->session_batch = 0;  // the diagnostics reuse the caches
     SPEC_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
     return SPEC_OK;
 }
@@ -635,6 +701,7 @@ extern "C" int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* toke
         return fail(SPEC_ERR_CAPACITY, "spec_forward_logits: %d x %d rows exceed the workspace (%d rows)", batch, rows, ctx->max_rows);
     const Model& m = ctx->model[which];
     const int n = batch * rows;
+    ctx->session_batch = 0;  // the diagnostics reuse the caches
     std::vector<int32_t> tok(n), pos(n), seq(n);
     for (int b = 0; b < batch; ++b) {
         if (ctx->cached[which][b] + rows > std::min(ctx->rt.max_len, m.cfg.max_positions))

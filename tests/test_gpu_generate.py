@@ -112,3 +112,21 @@ def test_statistics_are_consistent(tiny):
     assert np.array_equal(out, again)  # same seed, same tokens
     other, _ = eng.generate([prompt], 60, 3, 1.0, 2)
     assert not np.array_equal(out, other)
+
+
+def test_phased_generation_equals_the_single_call(tiny):
+    eng, _, _, cfg = tiny
+    prompts = [workloads.make_prompt(31, 7, cfg["vocab"]), workloads.make_prompt(32, 12, cfg["vocab"])]
+    whole, st = eng.generate(prompts, 30, 3, 1.0, 9)
+    eng.begin(prompts, 30, 3, 1.0, 9)
+    remaining, steps = 30, 0
+    while remaining > 0:
+        remaining, part = eng.step(2)
+        steps += 2
+        assert part["target_passes"] == steps and part["decode_ms"] > 0
+    assert np.array_equal(eng.read_tokens(), whole)
+    assert part["tokens"] == st["tokens"] and part["tests_passed"] == st["tests_passed"]
+    # a diagnostic call ends the generation in progress
+    eng.reset()
+    with pytest.raises(binding.SpecError):
+        eng.step(1)
