@@ -233,14 +233,16 @@ def weight_stream_bytes(cfg):
 class GenerationWorkload:
     dtype = "bf16"
 
-    def __init__(self, name, target, draft, batch, prompt_len, n_new, gamma, temperature=1.0):
+    def __init__(self, name, target, draft, batch, prompt_len, n_new, gamma, temperature=1.0, layers=None):
         self.name, self.target_name, self.draft_name = name, target, draft
+        self.layers = layers
         self.batch, self.prompt_len, self.n_new, self.gamma, self.temperature = batch, prompt_len, n_new, gamma, temperature
 
     def description(self):
         return {"workload": self.name, "target": self.target_name, "draft": self.draft_name, "batch": self.batch,
                 "prompt_len": self.prompt_len, "n_new": self.n_new, "gamma": self.gamma,
                 "temperature": self.temperature, "kv_dtype": "fp32",
+                **({"target_layers_override": self.layers} if self.layers else {}),
                 "l2": "one pass streams the target's weights (>> 126 MB L2) from HBM",
                 "parallelism": "replicas"}
 
@@ -249,6 +251,8 @@ class GenerationWorkload:
         from paper_2211_17192_b200 import binding, workloads
         self.torch, self.binding, self.device = torch, binding, device
         self.tcfg = workloads.model_config(self.target_name)
+        if self.layers:
+            self.tcfg = workloads.scaled_config(self.tcfg, n_layers=self.layers)
         self.dcfg = workloads.model_config(self.draft_name)
         self.dtype = "bf16" if self.tcfg["dtype"] == "bf16" else "f32"
         self.tw = gpu_weights(self.tcfg, 100 + rank, device)
@@ -374,11 +378,11 @@ def make_workload(args):
         return SamplerWorkload()
     batch = args.batch or 1
     if args.workload == "gpt97m":
-        return GenerationWorkload("gpt97m_6m_b1", "gpt97m_target", "gpt6m_draft", batch, 128, 512, args.gamma or 5,
-                                  args.temperature)
+        return GenerationWorkload("gpt97m_6m_b1", "gpt97m_target", "gpt6m_draft", batch, args.prompt_len or 128, 512,
+                                  args.gamma or 5, args.temperature, args.layers)
     gamma = args.gamma or 2
-    return GenerationWorkload(f"llama7b_160m_b{batch}_g{gamma}", "llama7b_target", "llama160m_draft", batch, 1024, 256,
-                              gamma, args.temperature)
+    return GenerationWorkload(f"llama7b_160m_b{batch}_g{gamma}", "llama7b_target", "llama160m_draft", batch,
+                              args.prompt_len or 1024, 256, gamma, args.temperature, args.layers)
 
 
 WORKLOAD_NAMES = ["llama7b", "gpt97m", "sampler"]
@@ -555,6 +559,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--gamma", type=int, default=None)
     ap.add_argument("--temperature", type=float, default=1.0)
+    ap.add_argument("--prompt-len", type=int, default=None, help="override the workload's prompt length (profiling)")
+    ap.add_argument("--layers", type=int, default=None, help="override the target's depth, full width (profiling)")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for cpu_baseline")
     args = ap.parse_args()

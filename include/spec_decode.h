@@ -200,7 +200,9 @@ typedef struct spec_stats {
 /* Creates a context for a target model and (optionally, draft_cfg == NULL for
  * target-only decoding) a draft model with the same vocabulary.  Allocates the
  * paged KV caches, activations and logits buffers with cudaMalloc on the
- * current device and creates a private stream; weights are borrowed.
+ * current device and creates a private stream.  Weights are borrowed; for bf16
+ * models the library also makes its own tile-major copies of the block matrices
+ * and the LM head (see spec_pack_weight), which doubles their footprint.
  * Errors: SPEC_ERR_BAD_ARG (null), SPEC_ERR_BAD_CONFIG (unsupported shapes,
  * vocabularies differ), SPEC_ERR_OOM, SPEC_ERR_CUDA. */
 int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg* draft_cfg,
@@ -272,8 +274,13 @@ int spec_truncate(spec_ctx* ctx, int which, const int32_t* lengths, int batch);
  * streaming W from memory, and gamma+1 rows share one stream of the weights).
  *   x [rows, k] fp32 device; w [n_out, k] device in w_dtype (SPEC_DTYPE_*);
  *   y [rows, n_out] fp32 device out; k a multiple of 8.
- *   path 0: the path the engine would choose (tensor cores for bf16 weights,
- *           FMA pipes for fp32); 1: FMA pipes; 2: tensor cores (bf16 only).
+ *   path 0: tensor cores for bf16 weights, FMA pipes for fp32; 1: FMA pipes;
+ *        2: tensor cores (bf16 only); 3: tensor cores with `w` in the
+ *           tile-major layout that spec_pack_weight produces, which is what
+ *           the engine streams: every [128 x 64] tile of W is contiguous
+ *           (tiles ordered by 128-row band, then by 64-column block; rows and
+ *           columns past the matrix are zero), so that a CTA's weight stream
+ *           is one sequential run of HBM.
  * The tensor-core path splits x into two bf16 terms and sums split-K partial
  * results in a fixed order; it needs `workspace` (device, 256-byte aligned, at
  * least spec_linear_workspace_bytes(rows, n_out, k) bytes, contents arbitrary,
@@ -284,6 +291,10 @@ int spec_truncate(spec_ctx* ctx, int which, const int32_t* lengths, int batch);
  * synchronises with the device.
  * ------------------------------------------------------------------------- */
 size_t spec_linear_workspace_bytes(int rows, int n_out, int k);
+/* Bytes of the tile-major copy of a bf16 matrix [n_out, k], and the copy itself
+ * (device pointers, asynchronous on `stream`). */
+size_t spec_packed_weight_bytes(int n_out, int k);
+int spec_pack_weight(const void* w, int n_out, int k, void* packed, void* stream);
 int spec_linear(const float* x, const void* w, int w_dtype, int rows, int n_out, int k, int path,
                 float* y, void* workspace, size_t workspace_bytes, void* stream);
 int spec_device_error(void);

@@ -63,6 +63,10 @@ def _declare(h):
     h.spec_linear_workspace_bytes.argtypes = [i32, i32, i32]
     h.spec_linear.restype = i32
     h.spec_linear.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp]
+    h.spec_packed_weight_bytes.restype = sz
+    h.spec_packed_weight_bytes.argtypes = [i32, i32]
+    h.spec_pack_weight.restype = i32
+    h.spec_pack_weight.argtypes = [vp, i32, i32, vp, vp]
     h.spec_device_error.restype = i32
     h.spec_device_error.argtypes = []
 
@@ -152,21 +156,34 @@ def spec_uniforms(seed, positions, sequences, purpose, out=None):
     return out
 
 
-PATHS = {"auto": 0, "alu": 1, "tensor": 2}
+PATHS = {"auto": 0, "alu": 1, "tensor": 2, "tensor_packed": 3}
+
+
+def spec_pack_weight(w):
+    """Tile-major copy of a bf16 CUDA matrix [n_out, k] (see the header); returns a uint8 tensor."""
+    n_out, k = w.shape
+    out = torch.empty(int(lib().spec_packed_weight_bytes(n_out, k)), dtype=torch.uint8, device=w.device)
+    _check(lib().spec_pack_weight(_ptr(w, torch.bfloat16, "w"), n_out, k, out.data_ptr(), _stream()))
+    return out
 
 
 def spec_linear_workspace_bytes(rows, n_out, k):
     return int(lib().spec_linear_workspace_bytes(rows, n_out, k))
 
 
-def spec_linear(x, w, path="auto", y=None, workspace=None):
-    """y = x . W^T; x [rows, k] fp32 CUDA, w [n_out, k] fp32 or bf16 CUDA -> y [rows, n_out] fp32."""
+def spec_linear(x, w, path="auto", y=None, workspace=None, n_out=None):
+    """y = x . W^T; x [rows, k] fp32 CUDA, w [n_out, k] fp32 or bf16 CUDA -> y [rows, n_out] fp32.
+    With path "tensor_packed", w is the uint8 tensor from spec_pack_weight and n_out must be given."""
     rows, k = x.shape
-    n_out = w.shape[0]
-    if w.shape[1] != k:
-        raise ValueError("inner dimensions differ")
-    if w.dtype not in (torch.float32, torch.bfloat16):
-        raise ValueError("w must be fp32 or bf16")
+    if path == "tensor_packed":
+        if n_out is None:
+            raise ValueError("n_out is required with packed weights")
+    else:
+        n_out = w.shape[0]
+        if w.shape[1] != k:
+            raise ValueError("inner dimensions differ")
+        if w.dtype not in (torch.float32, torch.bfloat16):
+            raise ValueError("w must be fp32 or bf16")
     if y is None:
         y = torch.empty((rows, n_out), dtype=torch.float32, device=x.device)
     need = spec_linear_workspace_bytes(rows, n_out, k)
@@ -174,7 +191,8 @@ def spec_linear(x, w, path="auto", y=None, workspace=None):
         workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
     if not w.is_cuda or not w.is_contiguous():
         raise ValueError("w must be a contiguous CUDA tensor")
-    _check(lib().spec_linear(_ptr(x, torch.float32, "x"), w.data_ptr(), 1 if w.dtype == torch.bfloat16 else 0,
+    _check(lib().spec_linear(_ptr(x, torch.float32, "x"), w.data_ptr(),
+                             1 if (w.dtype == torch.bfloat16 or path == "tensor_packed") else 0,
                              rows, n_out, k, PATHS[path], _ptr(y, torch.float32, "y"),
                              _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()))
     return y

@@ -123,16 +123,17 @@ int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_ro
     for (int l = 0; l < c.n_layers; ++l) {
         const spec_layer_weights& w = m.layers[l];
         if (tc) {
+            const spec_layer_weights& pw = m.packed[l];
             // (the FFN-out partial sums of the previous block are added into h by this norm)
             SPEC_TRY(launch_norm(ctx->h, l ? part : nullptr, s_out, n_rows, w.ln1, nullptr, n_rows, d, c.rms_eps, nullptr, hi, lo, st));
-            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, w.wqkv, n_rows, m.qkv_dim(), d, part, st));
+            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, pw.wqkv, true, n_rows, m.qkv_dim(), d, part, st));
             SPEC_TRY(launch_qkv(m, l, rows, n_rows, ctx->qkv, part, s_qkv, ctx->page_table, pages, page, st));
             SPEC_TRY(launch_attention(m, l, rows, batch, m_rows, slices, ctx->qkv, ctx->attn_part, nullptr, hi, lo, ctx->page_table, pages, page, st));
-            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, w.wo, n_rows, d, m.q_dim(), part, st));
+            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, pw.wo, true, n_rows, d, m.q_dim(), part, st));
             SPEC_TRY(launch_norm(ctx->h, part, s_o, n_rows, w.ln2, nullptr, n_rows, d, c.rms_eps, nullptr, hi, lo, st));
-            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, w.w_in, n_rows, m.ffn_in_dim(), d, part, st));
+            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, pw.w_in, true, n_rows, m.ffn_in_dim(), d, part, st));
             SPEC_TRY(launch_ffn_act(nullptr, part, s_in, n_rows, c.d_ff, c.ffn, nullptr, hi, lo, st));
-            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, w.w_out, n_rows, d, c.d_ff, part, st));
+            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, pw.w_out, true, n_rows, d, c.d_ff, part, st));
         } else {
             const bool bf = m.bf16();
             SPEC_TRY(launch_norm(ctx->h, nullptr, 0, n_rows, w.ln1, nullptr, n_rows, d, c.rms_eps, ctx->a, nullptr, nullptr, st));
@@ -149,7 +150,7 @@ int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_ro
     if (n_logit_rows > 0) {
         if (tc) {
             SPEC_TRY(launch_norm(ctx->h, part, s_out, n_rows, m.ln_f, logit_src, n_logit_rows, d, c.rms_eps, nullptr, hi, lo, st));
-            SPEC_TRY(launch_gemm_tc(hi, lo, ctx->hi_rows, m.head, nullptr, logit_dst, n_logit_rows, c.vocab, d, part, logits, st));
+            SPEC_TRY(launch_gemm_tc(hi, lo, ctx->hi_rows, m.packed_head, true, nullptr, logit_dst, n_logit_rows, c.vocab, d, part, logits, st));
         } else {
             SPEC_TRY(launch_norm(ctx->h, nullptr, 0, n_rows, m.ln_f, logit_src, n_logit_rows, d, c.rms_eps, ctx->a, nullptr, nullptr, st));
             SPEC_TRY(launch_gemm_rows(ctx->a, m.head, m.bf16(), nullptr, logit_dst, n_logit_rows, c.vocab, d, logits, st));
@@ -349,6 +350,28 @@ int feed_host_tokens(spec_ctx* ctx, int which, const int32_t* tokens, int stride
     return SPEC_OK;
 }
 
+// Tile-major copies of every matrix the tensor-core GEMM streams.
+int pack_model(spec_ctx* ctx, Model& m) {
+    const spec_model_cfg& c = m.cfg;
+    auto pack = [&](const void* w, int n_out, int k, const void** out) -> int {
+        __nv_bfloat16* dst = nullptr;
+        SPEC_TRY(dev_alloc(ctx, &dst, packed_weight_elems(n_out, k)));
+        SPEC_TRY(launch_pack_weight(w, n_out, k, dst, ctx->stream));
+        *out = dst;
+        return SPEC_OK;
+    };
+    m.packed.assign(c.n_layers, spec_layer_weights{});
+    for (int l = 0; l < c.n_layers; ++l) {
+        SPEC_TRY(pack(m.layers[l].wqkv, m.qkv_dim(), c.d_model, &m.packed[l].wqkv));
+        SPEC_TRY(pack(m.layers[l].wo, c.d_model, m.q_dim(), &m.packed[l].wo));
+        SPEC_TRY(pack(m.layers[l].w_in, m.ffn_in_dim(), c.d_model, &m.packed[l].w_in));
+        SPEC_TRY(pack(m.layers[l].w_out, c.d_model, c.d_ff, &m.packed[l].w_out));
+    }
+    SPEC_TRY(pack(m.head, c.vocab, c.d_model, &m.packed_head));
+    SPEC_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+    return SPEC_OK;
+}
+
 int init_model(spec_ctx* ctx, int which, const spec_model_cfg& cfg, const spec_weights& w) {
     Model& m = ctx->model[which];
     m.cfg = cfg;
@@ -472,6 +495,8 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
                     partial = std::max(partial, gemm_tc_partial_elems(sh[0], sh[1], rows));
         }
         if (any_bf16 && ctx->tensor_cores) {
+            for (int i = 0; i < (ctx->has_draft ? 2 : 1); ++i)
+                if (ctx->model[i].bf16() && (status = pack_model(ctx, ctx->model[i])) != SPEC_OK) return cleanup(status);
             ctx->hi_rows = (ctx->max_rows + 127) / 128 * 128;
             SPEC_ALLOC(x_hi, static_cast<size_t>(ctx->hi_rows) * max_k);
             SPEC_ALLOC(x_lo, static_cast<size_t>(ctx->hi_rows) * max_k);

@@ -134,7 +134,7 @@ template <int N_TOK>
 __global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_hi,
                const __grid_constant__ CUtensorMap map_lo, float* __restrict__ partial, int n_out, int n_rows,
-               int k_blocks) {
+               int k_blocks, int packed) {
     using S = Smem<N_TOK>;
     constexpr int kTmemCols = N_TOK < 32 ? 32 : N_TOK;
     extern __shared__ uint8_t smem_raw[];
@@ -173,11 +173,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // ---- producer: weights and both activation terms of one k-block per stage ----
         // The weights do not depend on the kernel before this one: the first
         // ring of weight tiles is already streaming while that kernel finishes.
+        // Weight tile of k-block kb: in the row-major matrix the box at (kb*64, tile*128);
+        // in the tile-major copy the 128 consecutive 128-byte rows of tile (tile, kb).
+        auto load_w = [&](void* dst, int kb, uint64_t* bar) {
+            if (packed) tma_load_2d(dst, &map_w, 0, (tile * k_blocks + kb) * kTileM, bar);
+            else tma_load_2d(dst, &map_w, kb * kTileK, tile * kTileM, bar);
+        };
         const int total = kb1 - kb0;
         const int ahead = min(total, S::kStages);
         for (int it = 0; it < ahead; ++it) {
             mbar_expect_tx(&full_bar[it], S::kStageBytes);
-            tma_load_2d(smem + it * S::kStageBytes, &map_w, (kb0 + it) * kTileK, tile * kTileM, &full_bar[it]);
+            load_w(smem + it * S::kStageBytes, kb0 + it, &full_bar[it]);
         }
         pdl_wait();  // the activations are written by the previous kernel
         for (int it = 0; it < ahead; ++it) {
@@ -190,7 +196,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if (!mbar_wait(&empty_bar[s], ((it / S::kStages) - 1) & 1)) { ok = false; break; }
             uint8_t* stage = smem + s * S::kStageBytes;
             mbar_expect_tx(&full_bar[s], S::kStageBytes);
-            tma_load_2d(stage, &map_w, kb * kTileK, tile * kTileM, &full_bar[s]);
+            load_w(stage, kb, &full_bar[s]);
             tma_load_2d(stage + S::kABytes, &map_hi, kb * kTileK, tok0, &full_bar[s]);
             tma_load_2d(stage + S::kABytes + S::kBBytes, &map_lo, kb * kTileK, tok0, &full_bar[s]);
         }
@@ -252,6 +258,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(kTmemCols));
+    }
+}
+
+// Tile-major copy of a row-major bf16 matrix W [n_out, k]: tile (t, kb) holds rows
+// t*128 .. t*128+127, columns kb*64 .. kb*64+63 as 128 consecutive 128-byte rows,
+// tiles ordered (t, kb); rows and columns past the matrix are zero.  One 16-byte
+// vector (8 elements) per thread.
+__global__ void pack_weight_kernel(const __nv_bfloat16* __restrict__ w, int n_out, int k, int k_blocks, size_t vectors,
+                                   __nv_bfloat16* __restrict__ out) {
+    for (size_t v = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; v < vectors;
+         v += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        const size_t tile_index = v / (kTileM * kTileK / 8);
+        const int within = static_cast<int>(v % (kTileM * kTileK / 8));
+        const int r = within / (kTileK / 8), c8 = within % (kTileK / 8);
+        const int row = static_cast<int>(tile_index / k_blocks) * kTileM + r;
+        const int col = static_cast<int>(tile_index % k_blocks) * kTileK + c8 * 8;
+        uint4 val = make_uint4(0u, 0u, 0u, 0u);
+        if (row < n_out && col < k) val = *reinterpret_cast<const uint4*>(w + static_cast<size_t>(row) * k + col);
+        *reinterpret_cast<uint4*>(out + v * 8) = val;
     }
 }
 
@@ -350,7 +375,7 @@ int cached_map(const void* base, int rows, int cols, int box_rows, CUtensorMap* 
 
 template <int N_TOK>
 int launch_tc(const CUtensorMap& mw, const CUtensorMap& mhi, const CUtensorMap& mlo, float* partial, int n_out,
-              int n_rows, int k_blocks, int splits, cudaStream_t stream) {
+              int n_rows, int k_blocks, int splits, int packed, cudaStream_t stream) {
     static bool configured = false;
     if (!configured) {
         SPEC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<N_TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -359,7 +384,7 @@ int launch_tc(const CUtensorMap& mw, const CUtensorMap& mhi, const CUtensorMap& 
     }
     const dim3 grid((n_out + kTileM - 1) / kTileM, splits, (n_rows + N_TOK - 1) / N_TOK);
     return launch_pdl(gemm_tc_kernel<N_TOK>, grid, dim3(kThreads), Smem<N_TOK>::kTotal, stream, mw, mhi, mlo, partial,
-                      n_out, n_rows, k_blocks);
+                      n_out, n_rows, k_blocks, packed);
 }
 
 }  // namespace
@@ -393,6 +418,20 @@ size_t gemm_tc_partial_elems(int n_out, int k, int n_rows) {
     return static_cast<size_t>(gemm_tc_splits(n_out, k, n_rows)) * n_rows * n_out;
 }
 
+size_t packed_weight_elems(int n_out, int k) {
+    return static_cast<size_t>((n_out + kTileM - 1) / kTileM) * ((k + kTileK - 1) / kTileK) * kTileM * kTileK;
+}
+
+int launch_pack_weight(const void* w, int n_out, int k, void* out, cudaStream_t stream) {
+    if (k % 8 != 0) return fail(SPEC_ERR_BAD_CONFIG, "pack: inner dimension %d is not a multiple of 8", k);
+    const size_t vectors = packed_weight_elems(n_out, k) / 8;
+    const int blocks = static_cast<int>(std::min<size_t>((vectors + 255) / 256, 148 * 16));
+    pack_weight_kernel<<<blocks, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(w), n_out, k, (k + kTileK - 1) / kTileK,
+                                                   vectors, static_cast<__nv_bfloat16*>(out));
+    SPEC_CUDA_TRY(cudaGetLastError());
+    return SPEC_OK;
+}
+
 int launch_split_bf16(const float* x, size_t n, __nv_bfloat16* hi, __nv_bfloat16* lo, cudaStream_t stream) {
     const int blocks = static_cast<int>(std::min<size_t>((n / 4 + 255) / 256, 148 * 8));
     return launch_pdl(split_bf16_kernel, dim3(std::max(blocks, 1)), dim3(256), 0, stream, x, n, hi, lo);
@@ -400,32 +439,35 @@ int launch_split_bf16(const float* x, size_t n, __nv_bfloat16* hi, __nv_bfloat16
 
 // partial[s][r][n] for x already split into hi + lo (both [hi_rows, k] bf16, the
 // first n_rows rows valid); s < gemm_tc_splits(n_out, k, n_rows).
-int launch_gemm_tc_partials(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, int n_rows,
-                            int n_out, int k, float* partial, cudaStream_t stream) {
+int launch_gemm_tc_partials(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, bool packed,
+                            int n_rows, int n_out, int k, float* partial, cudaStream_t stream) {
     if (n_rows <= 0) return SPEC_OK;
     if (k % 8 != 0) return fail(SPEC_ERR_BAD_CONFIG, "gemm: inner dimension %d is not a multiple of 8", k);
     const int n_tok = gemm_tc_token_tile(n_rows);
     const int splits = gemm_tc_splits(n_out, k, n_rows);
     const int k_blocks = (k + kTileK - 1) / kTileK;
     CUtensorMap mw, mhi, mlo;
-    int status = cached_map(w, n_out, k, kTileM, &mw);
+    const int tiles = (n_out + kTileM - 1) / kTileM;
+    // tile-major weights are one long [tiles * k_blocks * 128, 64] matrix of 128-byte rows
+    int status = packed ? cached_map(w, tiles * k_blocks * kTileM, kTileK, kTileM, &mw) : cached_map(w, n_out, k, kTileM, &mw);
     if (status == SPEC_OK) status = cached_map(hi, hi_rows, k, n_tok, &mhi);
     if (status == SPEC_OK) status = cached_map(lo, hi_rows, k, n_tok, &mlo);
     if (status != SPEC_OK) return status;
+    const int pk = packed ? 1 : 0;
     switch (n_tok) {
-        case 16: return launch_tc<16>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream);
-        case 32: return launch_tc<32>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream);
-        case 64: return launch_tc<64>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream);
-        default: return launch_tc<128>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, stream);
+        case 16: return launch_tc<16>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
+        case 32: return launch_tc<32>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
+        case 64: return launch_tc<64>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
+        default: return launch_tc<128>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
     }
 }
 
 // y[dst(r)] = x[r] . W^T (+ residual[r]): the partial sums, then their reduction.
-int launch_gemm_tc(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, const float* residual,
-                   const int32_t* dst_rows, int n_rows, int n_out, int k, float* partial, float* y,
-                   cudaStream_t stream) {
+int launch_gemm_tc(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, bool packed,
+                   const float* residual, const int32_t* dst_rows, int n_rows, int n_out, int k, float* partial,
+                   float* y, cudaStream_t stream) {
     if (n_rows <= 0) return SPEC_OK;
-    const int status = launch_gemm_tc_partials(hi, lo, hi_rows, w, n_rows, n_out, k, partial, stream);
+    const int status = launch_gemm_tc_partials(hi, lo, hi_rows, w, packed, n_rows, n_out, k, partial, stream);
     if (status != SPEC_OK) return status;
     const int splits = gemm_tc_splits(n_out, k, n_rows);
     const size_t total = static_cast<size_t>(n_rows) * n_out;
@@ -462,10 +504,10 @@ extern "C" int spec_linear(const float* x, const void* w, int w_dtype, int rows,
     if (!x || !w || !y) return fail(SPEC_ERR_BAD_ARG, "spec_linear: null pointer");
     if (rows < 1 || n_out < 1 || k < 8 || k % 8) return fail(SPEC_ERR_BAD_ARG, "spec_linear: rows=%d n_out=%d k=%d (k must be a multiple of 8)", rows, n_out, k);
     if (w_dtype != SPEC_DTYPE_FP32 && w_dtype != SPEC_DTYPE_BF16) return fail(SPEC_ERR_BAD_ARG, "spec_linear: dtype %d", w_dtype);
-    if (path < 0 || path > 2) return fail(SPEC_ERR_BAD_ARG, "spec_linear: path %d", path);
+    if (path < 0 || path > 3) return fail(SPEC_ERR_BAD_ARG, "spec_linear: path %d", path);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool tensor = w_dtype == SPEC_DTYPE_BF16 && path != 1;
-    if (path == 2 && w_dtype != SPEC_DTYPE_BF16) return fail(SPEC_ERR_BAD_CONFIG, "spec_linear: the tensor-core path needs bf16 weights");
+    if (path >= 2 && w_dtype != SPEC_DTYPE_BF16) return fail(SPEC_ERR_BAD_CONFIG, "spec_linear: the tensor-core path needs bf16 weights");
     if (!tensor) return launch_gemm_rows(x, w, w_dtype == SPEC_DTYPE_BF16, nullptr, nullptr, rows, n_out, k, y, st);
     if (!workspace || workspace_bytes < spec_linear_workspace_bytes(rows, n_out, k) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
         return fail(SPEC_ERR_BAD_ARG, "spec_linear: workspace missing, too small or not 256-byte aligned");
@@ -478,7 +520,18 @@ extern "C" int spec_linear(const float* x, const void* w, int w_dtype, int rows,
     SPEC_CUDA_TRY(cudaMemsetAsync(base, 0, 2 * split_bytes, st));
     int status = launch_split_bf16(x, static_cast<size_t>(rows) * k, hi, lo, st);
     if (status != SPEC_OK) return status;
-    return launch_gemm_tc(hi, lo, padded_rows(rows), w, nullptr, nullptr, rows, n_out, k, partial, y, st);
+    return launch_gemm_tc(hi, lo, padded_rows(rows), w, path == 3, nullptr, nullptr, rows, n_out, k, partial, y, st);
+}
+
+extern "C" size_t spec_packed_weight_bytes(int n_out, int k) {
+    if (n_out < 1 || k < 1) return 0;
+    return spec::packed_weight_elems(n_out, k) * 2;
+}
+
+extern "C" int spec_pack_weight(const void* w, int n_out, int k, void* packed, void* stream) {
+    using namespace spec;
+    if (!w || !packed || n_out < 1 || k < 8 || k % 8) return fail(SPEC_ERR_BAD_ARG, "spec_pack_weight: bad argument");
+    return launch_pack_weight(w, n_out, k, packed, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int spec_device_error(void) { return spec::gemm_tc_take_error(); }

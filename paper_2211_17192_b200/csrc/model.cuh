@@ -17,6 +17,10 @@ struct Model {
     const float* ln_f = nullptr;
     const void* head = nullptr;  // == tok_emb when tied
     std::vector<spec_layer_weights> layers;
+    // Tensor-core path: the library's own tile-major copies of the block matrices
+    // and of the LM head (ln1 / ln2 of these entries are unused).
+    std::vector<spec_layer_weights> packed;
+    const void* packed_head = nullptr;
 
     // KV pool of layer l: kv + l * layer_stride bytes, laid out
     // [n_pages][2 (K, V)][n_kv_heads][page_size][d_head] in kv_elem_bytes-wide elements.
@@ -63,11 +67,15 @@ int launch_gemm_rows(const float* x, const void* w, bool w_bf16, const float* re
 int gemm_tc_splits(int n_out, int k, int n_rows);
 size_t gemm_tc_partial_elems(int n_out, int k, int n_rows);
 int launch_split_bf16(const float* x, size_t n, __nv_bfloat16* hi, __nv_bfloat16* lo, cudaStream_t stream);
-int launch_gemm_tc_partials(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, int n_rows,
-                            int n_out, int k, float* partial, cudaStream_t stream);
-int launch_gemm_tc(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, const float* residual,
-                   const int32_t* dst_rows, int n_rows, int n_out, int k, float* partial, float* y,
-                   cudaStream_t stream);
+// `packed`: w is the tile-major copy made by launch_pack_weight (every [128 x 64]
+// tile contiguous, so a CTA's weight stream is one sequential run of HBM).
+size_t packed_weight_elems(int n_out, int k);
+int launch_pack_weight(const void* w, int n_out, int k, void* out, cudaStream_t stream);
+int launch_gemm_tc_partials(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, bool packed,
+                            int n_rows, int n_out, int k, float* partial, cudaStream_t stream);
+int launch_gemm_tc(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows, const void* w, bool packed,
+                   const float* residual, const int32_t* dst_rows, int n_rows, int n_out, int k, float* partial,
+                   float* y, cudaStream_t stream);
 int gemm_tc_take_error();
 
 // Finishes the qkv GEMM (optional partial sums), rotary positions on q and k

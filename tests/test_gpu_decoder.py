@@ -132,3 +132,28 @@ def test_errors_are_reported():
         eng.generate([np.array([1, 2, 3])], 40, 0, 1.0, 0)  # does not fit max_len
     assert e.value.status == -4
     eng.close()
+
+
+@pytest.mark.parametrize("rows,n_out,k", [(1, 128, 64), (5, 300, 200), (3, 768, 768), (11, 2304, 768), (16, 704, 256),
+                                          (17, 256, 512), (70, 384, 256), (130, 256, 192), (7, 8192, 768)])
+def test_linear_layer_paths_agree_with_the_plain_definition(rows, n_out, k):
+    """y = x W^T on the FMA pipes, on the tensor cores (row-major and tile-major
+    weights) against numpy in fp64; the two tensor-core layouts are bit-identical."""
+    rng = np.random.default_rng(rows * 1000 + k)
+    x = rng.standard_normal((rows, k)).astype(np.float32)
+    w = workloads.round_to_bf16(rng.standard_normal((n_out, k)).astype(np.float32) * 0.05)
+    ref = x.astype(np.float64) @ w.astype(np.float64).T
+    xd = torch.from_numpy(x).cuda()
+    wd = torch.from_numpy(w).cuda().to(torch.bfloat16)
+    scale = np.abs(ref).max()
+    alu = binding.spec_linear(xd, wd, "alu").cpu().numpy()
+    tc = binding.spec_linear(xd, wd, "tensor")
+    packed = binding.spec_linear(xd, binding.spec_pack_weight(wd), "tensor_packed", n_out=n_out)
+    f32 = binding.spec_linear(xd, torch.from_numpy(w).cuda(), "auto").cpu().numpy()
+    torch.cuda.synchronize()
+    assert binding.spec_device_error() == 0
+    assert np.abs(alu - ref).max() <= 1e-5 * scale
+    assert np.abs(f32 - ref).max() <= 1e-5 * scale
+    # two bf16 terms keep 16 mantissa bits of x: relative error ~ 2^-16 per product
+    assert np.abs(tc.cpu().numpy() - ref).max() <= 1e-4 * scale
+    assert torch.equal(tc, packed)
