@@ -92,6 +92,44 @@ int spec_verify_sample(const float* target_logits, const float* draft_logits,
                        void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------- *
+ * spec_verify_sample for callers that cannot allocate device memory.  (The
+ * paper has no counterpart: this is a property of the library, not of the
+ * method.)
+ *
+ * Some hosts of this library may not call cudaMalloc when they need to sample:
+ * a serving process that handed all device memory to its own pool at start-up,
+ * a real-time loop that forbids allocation after warm-up, a plugin that is only
+ * given input and output buffers.  They have nowhere to put the workspace that
+ * spec_verify_sample asks for.  This entry point computes the same result with
+ * the same kernels but keeps the per-chunk softmax statistics in a fixed array
+ * of spec_verify_sample_static_capacity() bytes (1 MiB) that is part of the
+ * library image: every GPU that loads the library holds that array until the
+ * process exits, and the call itself allocates nothing (no cudaMalloc, no
+ * cudaFree, no allocating library routine).
+ *
+ * Arguments, layouts, asynchrony and errors are those of spec_verify_sample,
+ * without the workspace.  In addition:
+ *   - SPEC_ERR_CAPACITY if spec_verify_sample_workspace_bytes(batch, gamma,
+ *     vocab) exceeds the built-in array (for example batch 64, gamma 7, vocab
+ *     32000 needs about 105 KB; batch 1024 at the same shape does not fit).
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current); make that first call
+ *     before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps whatever the
+ *     last call left in it.  Nothing in it has to start at zero: each call
+ *     overwrites every entry it later reads.  Two calls that may overlap on
+ *     the device (different streams, no ordering between them) race on the
+ *     array and corrupt each other's results; order them, or give one of them
+ *     a workspace through spec_verify_sample.
+ * ------------------------------------------------------------------------- */
+size_t spec_verify_sample_static_capacity(void);
+
+int spec_verify_sample_static(const float* target_logits, const float* draft_logits,
+                              const int32_t* draft_tokens, const float* uniforms,
+                              int batch, int gamma, int vocab, float temperature,
+                              int32_t* n_accepted, int32_t* next_token, void* stream);
+
+/* ------------------------------------------------------------------------- *
  * Plain standardised sampling (Section 2.2): one token per row of logits,
  * tokens[r] ~ softmax(logits[r] / T) by the same inverse-CDF rule, or the
  * lowest-index argmax at T = 0.  This is the draft model's x_i ~ q_i

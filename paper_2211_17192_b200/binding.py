@@ -55,6 +55,10 @@ def _declare(h):
     h.spec_verify_sample_workspace_bytes.argtypes = [i32, i32, i32]
     h.spec_verify_sample.restype = i32
     h.spec_verify_sample.argtypes = [vp, vp, vp, vp, i32, i32, i32, f32, vp, vp, vp, sz, vp]
+    h.spec_verify_sample_static_capacity.restype = sz
+    h.spec_verify_sample_static_capacity.argtypes = []
+    h.spec_verify_sample_static.restype = i32
+    h.spec_verify_sample_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, f32, vp, vp, vp]
     h.spec_sample.restype = i32
     h.spec_sample.argtypes = [vp, vp, i32, i32, f32, vp, vp]
     h.spec_uniforms.restype = i32
@@ -131,6 +135,23 @@ def spec_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, temp
         batch, gamma, vocab, float(temperature),
         _ptr(n_accepted, torch.int32, "n_accepted"), _ptr(next_token, torch.int32, "next_token"),
         _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()))
+    return n_accepted, next_token
+
+
+def spec_verify_sample_static(target_logits, draft_logits, draft_tokens, uniforms, temperature, n_accepted, next_token):
+    """`spec_verify_sample` for callers that cannot allocate: same inputs and
+    results, the scratch lives in a fixed 1 MiB array inside the library, and the
+    outputs must be passed in (nothing is allocated here either).  Shapes whose
+    statistics do not fit raise SpecError (SPEC_ERR_CAPACITY).  Calls that may
+    overlap on the device must not both use this entry point."""
+    batch, rows, vocab = target_logits.shape
+    _check(lib().spec_verify_sample_static(
+        _ptr(target_logits, torch.float32, "target_logits"),
+        _ptr(draft_logits, torch.float32, "draft_logits", optional=True),
+        _ptr(draft_tokens, torch.int32, "draft_tokens", optional=True),
+        _ptr(uniforms, torch.float32, "uniforms", optional=True),
+        batch, rows - 1, vocab, float(temperature),
+        _ptr(n_accepted, torch.int32, "n_accepted"), _ptr(next_token, torch.int32, "next_token"), _stream()))
     return n_accepted, next_token
 
 

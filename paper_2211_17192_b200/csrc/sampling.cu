@@ -14,6 +14,7 @@
 //      launch latency and prologue overlap the tail of the first kernel.
 #include <algorithm>
 #include <cfloat>
+#include <mutex>
 
 #include <cooperative_groups.h>
 
@@ -785,6 +786,68 @@ extern "C" int spec_verify_sample(const float* target_logits, const float* draft
         return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: workspace too small (%zu bytes) or not 256-byte aligned", workspace_bytes);
     return launch_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, nullptr, batch, gamma, vocab,
                                 temperature, n_accepted, next_token, workspace, static_cast<cudaStream_t>(stream));
+}
+
+// ---- spec_verify_sample without any allocation ---------------------------------
+// The chunk statistics that the two kernels hand to each other normally live in a
+// caller-provided workspace.  This variant keeps them in a fixed array inside the
+// library image instead, so the call needs no device memory beyond its inputs and
+// outputs.  Every GPU that loads the library holds the array until the process
+// exits.
+namespace {
+
+constexpr size_t kStaticStatsBytes = 1u << 20;  // 65536 chunk statistics
+static __device__ __align__(256) unsigned char g_static_stats[kStaticStatsBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};  // device address of g_static_stats, per device
+
+// The array's name is only a host-side handle; kernels need its device address,
+// which differs per device and is looked up once per device.
+int static_stats_address(void** out) {
+    int device = -1;
+    SPEC_CUDA_TRY(cudaGetDevice(&device));
+    if (device < 0 || device >= kMaxDevices) return spec::fail(SPEC_ERR_BAD_CONFIG, "device ordinal %d not supported", device);
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {
+        void* p = nullptr;
+        SPEC_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_stats));
+        g_static_ptr[device] = p;
+    }
+    *out = g_static_ptr[device];
+    return SPEC_OK;
+}
+
+}  // namespace
+
+extern "C" size_t spec_verify_sample_static_capacity(void) { return kStaticStatsBytes; }
+
+extern "C" int spec_verify_sample_static(const float* target_logits, const float* draft_logits,
+                                         const int32_t* draft_tokens, const float* uniforms, int batch, int gamma,
+                                         int vocab, float temperature, int32_t* n_accepted, int32_t* next_token,
+                                         void* stream) {
+    using namespace spec;
+    if (batch < 0 || gamma < 0 || gamma > kMaxGamma || vocab < 1)
+        return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample_static: batch=%d gamma=%d (max %d) vocab=%d", batch, gamma, kMaxGamma, vocab);
+    if (!(temperature >= 0.0f) || !isfinite(temperature))
+        return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample_static: temperature must be finite and >= 0");
+    if (batch == 0) return SPEC_OK;
+    if (batch > 65535) return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample_static: batch %d exceeds 65535", batch);
+    const bool greedy = temperature == 0.0f;
+    if (!target_logits || !n_accepted || !next_token || (gamma > 0 && !draft_tokens) ||
+        (!greedy && (!uniforms || (gamma > 0 && !draft_logits))))
+        return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample_static: null pointer");
+    const size_t need = verify_sample_workspace_bytes(batch, gamma, vocab);
+    if (need > kStaticStatsBytes)
+        return fail(SPEC_ERR_CAPACITY,
+                    "spec_verify_sample_static: batch %d x gamma %d x vocab %d needs %zu bytes of statistics, the built-in "
+                    "array holds %zu; use spec_verify_sample with a workspace", batch, gamma, vocab, need, kStaticStatsBytes);
+    void* scratch = nullptr;
+    const int status = static_stats_address(&scratch);
+    if (status != SPEC_OK) return status;
+    return launch_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, nullptr, batch, gamma, vocab,
+                                temperature, n_accepted, next_token, scratch, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int spec_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
