@@ -4,14 +4,14 @@
 // piece and runs one warp per query that reads this KV head: the G query heads
 // of the group times the m new rows of the sequence.  All warps of the CTA walk
 // the same 32-key tiles, so the K and V rows come from HBM/L2 once per CTA and
-// from L1 for the other queries.  Inside a tile each lane owns one key: it reads
-// the key's d_head values with 16-byte loads (a page stores the keys of one head
-// back to back, so a warp's loads cover one contiguous span), takes the dot
-// product with the query held in shared memory, and the warp keeps an online
-// softmax (running max and sum, fp32).  For P.V the lanes turn to the head
-// dimension: lane l owns d_head/32 output elements, V rows are fetched sixteen
-// at a time, and every key's probability is broadcast with a shuffle.  A tile
-// never straddles a page (pages hold a multiple of 32 tokens).
+// from L1 for the other queries.  Lane l owns d_head/32 consecutive elements of
+// the head dimension throughout, so every load of a K or V row is one coalesced
+// span (a page stores the rows of one head back to back).  For Q.K^T each lane
+// forms its share of the 32 dot products of a tile and a 31-shuffle butterfly
+// (reduce-scatter) leaves the score of key l in lane l; the warp keeps an online
+// softmax (running max and sum, fp32).  For P.V every key's probability is
+// broadcast with a shuffle.  A tile never straddles a page (pages hold a
+// multiple of 32 tokens).
 //
 // Each CTA writes an unnormalised partial state (max, sum, accumulator) per
 // query; attention_combine_kernel merges the key slices and emits the
@@ -24,7 +24,7 @@ namespace spec {
 namespace {
 
 constexpr int kMaxAttnWarps = 16;
-constexpr int kVBatch = 16;
+constexpr int kVBatch = 8;
 
 template <typename KV>
 struct KvLoad;
@@ -81,7 +81,6 @@ attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
                  const int32_t* __restrict__ page_table, int pages_per_seq, int page_size, float scale,
                  float* __restrict__ part) {
     constexpr int PER_LANE = DH / 32;
-    __shared__ float q_sh[kMaxAttnWarps][DH];
     pdl_trigger();
     pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
@@ -106,10 +105,10 @@ attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
         const int r = b * m_rows + j;
         const int p = pos[r];
         const int32_t* pages = page_table + seq[r] * pages_per_seq;
-        __syncwarp();
-        const float* qp = qkv + static_cast<size_t>(r) * qkv_dim + head * DH;
-        for (int i = lane; i < DH; i += 32) q_sh[warp][i] = qp[i] * scale;
-        __syncwarp();
+        float qv[PER_LANE];  // this lane's share of the (scaled) query
+        KvLoad<float>::template load_n<PER_LANE>(qkv + static_cast<size_t>(r) * qkv_dim + head * DH + lane * PER_LANE, qv);
+#pragma unroll
+        for (int i = 0; i < PER_LANE; ++i) qv[i] *= scale;
 
         float mx = -FLT_MAX, l = 0.0f;
         float acc[PER_LANE];
@@ -123,19 +122,36 @@ attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
             const KV* tile = kv_layer + pages[k0 / page_size] * page_stride + kv_head * head_stride +
                              static_cast<size_t>(k0 % page_size) * DH;
             const int in_tile = min(32, n_keys - k0);
-            float s = -FLT_MAX;
-            if (lane < in_tile) {
-                const KV* kp = tile + static_cast<size_t>(lane) * DH;
-                float dot = 0.0f;
+            // partial dot products of all 32 keys over this lane's elements ...
+            float pd[32];
+            const KV* kt = tile + lane * PER_LANE;
 #pragma unroll
-                for (int d0 = 0; d0 < DH; d0 += KvLoad<KV>::kVec) {
-                    float kvv[KvLoad<KV>::kVec];
-                    KvLoad<KV>::load(kp + d0, kvv);
+            for (int k = 0; k < 32; ++k) {
+                float kv[PER_LANE];
+                if (k < in_tile) {
+                    KvLoad<KV>::template load_n<PER_LANE>(kt + static_cast<size_t>(k) * DH, kv);
+                } else {
 #pragma unroll
-                    for (int e = 0; e < KvLoad<KV>::kVec; ++e) dot = fmaf(q_sh[warp][d0 + e], kvv[e], dot);
+                    for (int i = 0; i < PER_LANE; ++i) kv[i] = 0.0f;
                 }
-                s = dot;
+                float d = 0.0f;
+#pragma unroll
+                for (int i = 0; i < PER_LANE; ++i) d = fmaf(qv[i], kv[i], d);
+                pd[k] = d;
             }
+            // ... summed over the lanes by a butterfly that halves the live values
+            // at every step: lane l ends with the full score of key l
+#pragma unroll
+            for (int step = 16; step > 0; step >>= 1) {
+                const bool upper = (lane & step) != 0;
+#pragma unroll
+                for (int i = 0; i < step; ++i) {
+                    const float keep = upper ? pd[i + step] : pd[i];
+                    const float send = upper ? pd[i] : pd[i + step];
+                    pd[i] = keep + __shfl_xor_sync(kFullMask, send, step);
+                }
+            }
+            const float s = lane < in_tile ? pd[0] : -FLT_MAX;
             const float m_new = fmaxf(mx, warp_max(s));
             const float pr = lane < in_tile ? expf(s - m_new) : 0.0f;
             const float rescale = expf(mx - m_new);
