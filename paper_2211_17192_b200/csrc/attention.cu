@@ -24,7 +24,7 @@ namespace spec {
 namespace {
 
 constexpr int kMaxAttnWarps = 16;
-constexpr int kVBatch = 8;
+constexpr int kVBatch = 16;
 
 template <typename KV>
 struct KvLoad;
@@ -77,10 +77,11 @@ struct KvLoad<__nv_bfloat16> {
 template <typename KV, int DH>
 __global__ void __launch_bounds__(32 * kMaxAttnWarps)
 attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos, const int32_t* __restrict__ seq,
-                 int m_rows, int n_heads, int n_kv_heads, const KV* __restrict__ kv_layer,
+                 int m_rows, int n_heads, int n_kv_heads, int ks, const KV* __restrict__ kv_layer,
                  const int32_t* __restrict__ page_table, int pages_per_seq, int page_size, float scale,
                  float* __restrict__ part) {
     constexpr int PER_LANE = DH / 32;
+    __shared__ float share[kMaxAttnWarps][DH + 2];  // states of the warps that share a query (ks > 1)
     pdl_trigger();
     pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
@@ -100,7 +101,11 @@ attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
     const size_t page_stride = 2 * static_cast<size_t>(n_kv_heads) * head_stride;  // K block + V block
     const size_t v_offset = static_cast<size_t>(n_kv_heads) * head_stride;
 
-    for (int q = warp; q < queries; q += warps) {
+    // Work unit u = (query q, sub-slice sub): with ks > 1 the ks warps q, q + queries,
+    // ... share query q and take every ks-th tile of the slice (then the block has
+    // exactly queries * ks warps and this loop runs once).
+    for (int u = warp; u < queries * ks; u += warps) {
+        const int q = u % queries, sub = u / queries;
         const int j = q / group, head = kv_head * group + q % group;
         const int r = b * m_rows + j;
         const int p = pos[r];
@@ -115,7 +120,7 @@ attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
 #pragma unroll
         for (int i = 0; i < PER_LANE; ++i) acc[i] = 0.0f;
         const int n_keys = p + 1;  // causal: positions 0..p (p < 0: inactive row, no keys)
-        for (int t = t0; t < t1; ++t) {
+        for (int t = t0 + sub; t < t1; t += ks) {
             const int k0 = 32 * t;
             if (k0 >= n_keys) break;
             // the whole tile lives in one page
@@ -182,14 +187,50 @@ attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
                 }
             }
         }
-        // partial state of (row r, head, slice): [max, sum, acc[DH]]
-        float* out = part + ((static_cast<size_t>(r) * n_heads + head) * slices + slice) * (DH + 2);
-        if (lane == 0) {
-            out[0] = mx;
-            out[1] = l;
-        }
+        if (ks > 1) {  // park the state; warp `q` merges the ks of them below
+            if (lane == 0) {
+                share[warp][0] = mx;
+                share[warp][1] = l;
+            }
 #pragma unroll
-        for (int i = 0; i < PER_LANE; ++i) out[2 + lane * PER_LANE + i] = acc[i];
+            for (int i = 0; i < PER_LANE; ++i) share[warp][2 + lane * PER_LANE + i] = acc[i];
+        } else {
+            // partial state of (row r, head, slice): [max, sum, acc[DH]]
+            float* out = part + ((static_cast<size_t>(r) * n_heads + head) * slices + slice) * (DH + 2);
+            if (lane == 0) {
+                out[0] = mx;
+                out[1] = l;
+            }
+#pragma unroll
+            for (int i = 0; i < PER_LANE; ++i) out[2 + lane * PER_LANE + i] = acc[i];
+        }
+    }
+    if (ks > 1) {
+        __syncthreads();
+        if (warp < queries) {
+            const int q = warp;
+            const int j = q / group, head = kv_head * group + q % group;
+            const int r = b * m_rows + j;
+            float mm = -FLT_MAX;
+            for (int s = 0; s < ks; ++s) mm = fmaxf(mm, share[q + s * queries][0]);
+            float l = 0.0f, acc[PER_LANE];
+#pragma unroll
+            for (int i = 0; i < PER_LANE; ++i) acc[i] = 0.0f;
+            for (int s = 0; s < ks; ++s) {  // sub-slices in index order
+                const float* st = share[q + s * queries];
+                const float w = expf(st[0] - mm);
+                l += st[1] * w;
+#pragma unroll
+                for (int i = 0; i < PER_LANE; ++i) acc[i] += st[2 + lane * PER_LANE + i] * w;
+            }
+            float* out = part + ((static_cast<size_t>(r) * n_heads + head) * slices + slice) * (DH + 2);
+            if (lane == 0) {
+                out[0] = mm;
+                out[1] = l;
+            }
+#pragma unroll
+            for (int i = 0; i < PER_LANE; ++i) out[2 + lane * PER_LANE + i] = acc[i];
+        }
     }
 }
 
@@ -228,10 +269,18 @@ __global__ void attention_combine_kernel(const float* __restrict__ part, int sli
 
 }  // namespace
 
-// Key slices per (sequence, KV head): enough CTAs for two per SM, at least 64 keys each.
-int attention_slices(int batch, int n_kv_heads, int max_len) {
+// Warps that share one query inside a CTA (only when all queries then fit the
+// block in one round), and key slices (CTAs) per (sequence, KV head): about one
+// 32-key tile per warp when the batch is small, about two CTAs per SM at most.
+int attention_sub_slices(int queries) {
+    return queries * 2 <= kMaxAttnWarps ? kMaxAttnWarps / queries : 1;
+}
+
+int attention_slices(int batch, int n_kv_heads, int queries, int max_len) {
     const int want = (2 * 148 + batch * n_kv_heads - 1) / (batch * n_kv_heads);
-    const int most = std::max(1, max_len / 64);
+    const int tiles = (max_len + 31) / 32;
+    const int ks = attention_sub_slices(queries);
+    const int most = std::max(1, (tiles + ks - 1) / ks);
     return std::max(1, std::min(std::min(want, most), 32));
 }
 
@@ -244,14 +293,15 @@ int launch_attention(const Model& m, int layer, const RowMeta& rows, int batch, 
                      const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream) {
     const char* kv_layer = static_cast<const char*>(m.kv) + static_cast<size_t>(layer) * m.layer_stride;
     const int group = m.cfg.n_heads / m.cfg.n_kv_heads;
-    const int warps = std::min(kMaxAttnWarps, std::max(1, group * m_rows));
+    const int ks = attention_sub_slices(group * m_rows);
+    const int warps = std::min(kMaxAttnWarps, std::max(1, group * m_rows * ks));
     const dim3 grid(slices, m.cfg.n_kv_heads, batch);
     const float scale = 1.0f / sqrtf(static_cast<float>(m.cfg.d_head));
     const int n_rows = batch * m_rows;
 #define SPEC_ATTN(KV, DH)                                                                                         \
     do {                                                                                                          \
         int status = launch_pdl(attention_kernel<KV, DH>, grid, dim3(32 * warps), 0, stream, qkv, rows.pos,       \
-                                rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads,                                \
+                                rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads, ks,                            \
                                 reinterpret_cast<const KV*>(kv_layer), page_table, pages_per_seq, page_size,      \
                                 scale, part);                                                                     \
         if (status != SPEC_OK) return status;                                                                     \

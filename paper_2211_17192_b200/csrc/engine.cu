@@ -112,7 +112,7 @@ int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_ro
     __nv_bfloat16 *hi = tc ? ctx->x_hi : nullptr, *lo = tc ? ctx->x_lo : nullptr;
     float* part = ctx->partials;
     const int d = c.d_model, pages = ctx->pages_per_seq, page = ctx->rt.page_size;
-    const int slices = attention_slices(batch, c.n_kv_heads, ctx->rt.max_len);
+    const int slices = attention_slices(batch, c.n_kv_heads, (c.n_heads / c.n_kv_heads) * m_rows, ctx->rt.max_len);
     // split-K factors of the four GEMM shapes of a block at this row count
     const int s_qkv = tc ? gemm_tc_splits(m.qkv_dim(), d, n_rows) : 0;
     const int s_o = tc ? gemm_tc_splits(d, m.q_dim(), n_rows) : 0;
@@ -470,8 +470,9 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
         for (int i = 0; i < (ctx->has_draft ? 2 : 1); ++i) {
             const Model& m = ctx->model[i];
             for (int b = 1; b <= rt.max_batch; ++b)
-                attn = std::max(attn, attention_partial_elems(ctx->max_rows, m.cfg.n_heads, m.cfg.d_head,
-                                                              attention_slices(b, m.cfg.n_kv_heads, rt.max_len)));
+                for (int mr = 1; b * mr <= ctx->max_rows; ++mr)
+                    attn = std::max(attn, attention_partial_elems(b * mr, m.cfg.n_heads, m.cfg.d_head,
+                                                                  attention_slices(b, m.cfg.n_kv_heads, (m.cfg.n_heads / m.cfg.n_kv_heads) * mr, rt.max_len)));
         }
         SPEC_ALLOC(attn_part, attn);
     }

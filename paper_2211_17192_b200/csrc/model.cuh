@@ -86,7 +86,7 @@ void fill_rope_table(std::vector<float2>& table, int positions, int d_head, doub
 
 // att[r, h] = softmax(q_r,h . K / sqrt(d_head)) V over cached positions <= pos[r];
 // rows of sequence b are rows b*m_rows .. of the pass.  Output as fp32 and/or two bf16 terms.
-int attention_slices(int batch, int n_kv_heads, int max_len);
+int attention_slices(int batch, int n_kv_heads, int queries, int max_len);
 size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices);
 int launch_attention(const Model& m, int layer, const RowMeta& rows, int batch, int m_rows, int slices,
                      const float* qkv, float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo,
