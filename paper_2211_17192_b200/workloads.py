@@ -18,7 +18,8 @@ INIT_STD = 0.02
 
 def model_config(name):
     """Shapes of the synthetic models, by config name."""
-    base = dict(rms_eps=1e-6, rope_base=10000.0, tied=False, arch="gpt", ffn="gelu")
+    base = dict(rms_eps=1e-6, rope_base=10000.0, tied=False, arch="gpt", ffn="gelu", n_enc_layers=0,
+                rel_buckets=32, rel_max_distance=128, bias_std=0.5)
     table = {
         # tiny fp32 pair (correctness config)
         "tiny_target": dict(n_layers=4, d_model=256, n_heads=4, n_kv_heads=4, d_head=64, d_ff=1024,
@@ -44,6 +45,26 @@ def model_config(name):
         "llama_test_draft": dict(arch="llama", ffn="swiglu", n_layers=1, d_model=128, n_heads=2, n_kv_heads=1,
                                  d_head=64, d_ff=384, vocab=2048, max_positions=512, dtype="bf16",
                                  head_std=INIT_STD),
+        # T5-shaped encoder-decoder pair (XXL-shaped target, small-shaped draft), bf16
+        "t5xxl_target": dict(arch="t5", ffn="gated_gelu", n_layers=24, n_enc_layers=24, d_model=4096, n_heads=64,
+                             n_kv_heads=64, d_head=64, d_ff=10240, vocab=32128, max_positions=1024, dtype="bf16",
+                             head_std=INIT_STD),
+        "t5small_draft": dict(arch="t5", ffn="gated_gelu", n_layers=8, n_enc_layers=8, d_model=512, n_heads=6,
+                              n_kv_heads=6, d_head=64, d_ff=1024, vocab=32128, max_positions=1024, dtype="bf16",
+                              head_std=INIT_STD),
+        # small encoder-decoder pairs for tests
+        "t5_test_target": dict(arch="t5", ffn="gated_gelu", n_layers=2, n_enc_layers=2, d_model=256, n_heads=4,
+                               n_kv_heads=4, d_head=64, d_ff=512, vocab=2048, max_positions=512, dtype="bf16",
+                               head_std=INIT_STD),
+        "t5_test_draft": dict(arch="t5", ffn="gated_gelu", n_layers=1, n_enc_layers=1, d_model=128, n_heads=2,
+                              n_kv_heads=2, d_head=64, d_ff=256, vocab=2048, max_positions=512, dtype="bf16",
+                              head_std=INIT_STD),
+        "t5_tiny_target": dict(arch="t5", ffn="gated_gelu", n_layers=2, n_enc_layers=2, d_model=128, n_heads=2,
+                               n_kv_heads=2, d_head=64, d_ff=256, vocab=512, max_positions=256, dtype="fp32",
+                               head_std=3.0 / np.sqrt(128.0)),
+        "t5_tiny_draft": dict(arch="t5", ffn="gated_gelu", n_layers=1, n_enc_layers=1, d_model=64, n_heads=1,
+                              n_kv_heads=1, d_head=64, d_ff=128, vocab=512, max_positions=256, dtype="fp32",
+                              head_std=3.0 / 8.0),
     }
     cfg = dict(base)
     cfg.update(table[name])
@@ -59,21 +80,39 @@ def scaled_config(cfg, **overrides):
 
 
 def tensor_shapes(cfg):
-    """Ordered (name, shape, kind) of a model's tensors; kind is 'gain' or 'matrix'."""
+    """Ordered (name, shape, kind) of a model's tensors; kind is 'gain', 'matrix', 'bias' or 'head'."""
     d, H, Hkv, dh, F = cfg["d_model"], cfg["n_heads"], cfg["n_kv_heads"], cfg["d_head"], cfg["d_ff"]
     f_in = F if cfg["ffn"] == "gelu" else 2 * F
+    t5 = cfg["arch"] == "t5"
     out = [("tok_emb", (cfg["vocab"], d), "matrix")]
     if cfg["arch"] == "gpt":
         out.append(("pos_emb", (cfg["max_positions"], d), "matrix"))
-    for l in range(cfg["n_layers"]):
-        out += [
-            (f"l{l}.ln1", (d,), "gain"),
-            (f"l{l}.wqkv", ((H + 2 * Hkv) * dh, d), "matrix"),
-            (f"l{l}.wo", (d, H * dh), "matrix"),
-            (f"l{l}.ln2", (d,), "gain"),
-            (f"l{l}.w_in", (f_in, d), "matrix"),
-            (f"l{l}.w_out", (d, F), "matrix"),
+
+    def block(prefix):
+        return [
+            (prefix + "ln1", (d,), "gain"),
+            (prefix + "wqkv", ((H + 2 * Hkv) * dh, d), "matrix"),
+            (prefix + "wo", (d, H * dh), "matrix"),
+            (prefix + "ln2", (d,), "gain"),
+            (prefix + "w_in", (f_in, d), "matrix"),
+            (prefix + "w_out", (d, F), "matrix"),
         ]
+
+    if t5:  # encoder stack, then the decoder's bias table
+        out.append(("enc.rel_bias", (cfg["rel_buckets"], H), "bias"))
+        for l in range(cfg["n_enc_layers"]):
+            out += block(f"enc.l{l}.")
+        out.append(("enc.ln_f", (d,), "gain"))
+        out.append(("rel_bias", (cfg["rel_buckets"], H), "bias"))
+    for l in range(cfg["n_layers"]):
+        out += block(f"l{l}.")
+        if t5:  # cross-attention
+            out += [
+                (f"l{l}.lnx", (d,), "gain"),
+                (f"l{l}.wq_x", (H * dh, d), "matrix"),
+                (f"l{l}.wkv_x", (2 * H * dh, d), "matrix"),
+                (f"l{l}.wo_x", (d, H * dh), "matrix"),
+            ]
     out.append(("ln_f", (d,), "gain"))
     if not cfg["tied"]:
         out.append(("head", (cfg["vocab"], d), "head"))
@@ -93,7 +132,8 @@ def bf16_bits(a):
 
 
 def make_weights(cfg, seed):
-    """Random-init weights: matrices N(0, 0.02^2), head N(0, head_std^2), gains 1.
+    """Random-init weights: matrices N(0, 0.02^2), head N(0, head_std^2), relative-position
+    bias tables N(0, bias_std^2) (always fp32), gains 1.
 
     Every tensor has its own generator keyed by (seed, index in tensor_shapes),
     so a tensor's values do not depend on the others.  For dtype "bf16" the
@@ -106,9 +146,9 @@ def make_weights(cfg, seed):
             weights[name] = np.ones(shape, dtype=np.float32)
             continue
         rng = np.random.default_rng([int(seed), index])
-        std = cfg["head_std"] if kind == "head" else INIT_STD
+        std = cfg["head_std"] if kind == "head" else cfg["bias_std"] if kind == "bias" else INIT_STD
         a = rng.standard_normal(shape, dtype=np.float32) * np.float32(std)
-        if cfg["dtype"] == "bf16":
+        if cfg["dtype"] == "bf16" and kind != "bias":
             a = round_to_bf16(a)
         weights[name] = a
     return weights
