@@ -162,6 +162,20 @@ int spec_uniforms(uint64_t seed, const int32_t* positions, const int32_t* sequen
  *   SPEC_ARCH_GPT:   token + learned position embeddings, FFN per `ffn`.
  *   SPEC_ARCH_LLAMA: rotary positions (rotate-half pairing j, j + d_head/2,
  *                    angle position * rope_base^(-2j/d_head)) on q and k.
+ *   SPEC_ARCH_T5:    encoder-decoder (the T5-shaped pairs of Section 4.1; the
+ *                    paper fixes only their sizes).  No absolute positions;
+ *                    self-attention scores get, after scaling, an additive
+ *                    bias table[bucket(key pos - query pos)][head] with the
+ *                    usual log-spaced buckets (rel_buckets of them up to
+ *                    rel_max_distance; two mirrored halves in the encoder,
+ *                    backwards only in the decoder), one table per stack.
+ *                    The encoder (n_enc_layers blocks, every source position
+ *                    sees every other, output RMS-normalised with enc_ln_f)
+ *                    runs once per source.  A decoder block is causal
+ *                    self-attention, cross-attention (q = Wq_x . rmsnorm(h)
+ *                    with gain lnx; [K; V] = Wkv_x . encoder output, computed
+ *                    once; no bias; out-projection Wo_x) and the FFN.
+ *                    n_kv_heads == n_heads; decoding starts from token id 0.
  *   FFN: SPEC_FFN_GELU (tanh approximation) with W_in [d_ff, d_model];
  *        SPEC_FFN_GATED_GELU / SPEC_FFN_SWIGLU with W_in [2*d_ff, d_model],
  *        rows 0..d_ff-1 the gate, rows d_ff..2*d_ff-1 the up projection.
@@ -169,7 +183,7 @@ int spec_uniforms(uint64_t seed, const int32_t* positions, const int32_t* sequen
  * bf16 as raw 16-bit patterns); gains are fp32.  The residual stream, softmax,
  * normalisation and logits are fp32 in every configuration.
  * ------------------------------------------------------------------------- */
-enum { SPEC_ARCH_GPT = 0, SPEC_ARCH_LLAMA = 1 };
+enum { SPEC_ARCH_GPT = 0, SPEC_ARCH_LLAMA = 1, SPEC_ARCH_T5 = 2 };
 enum { SPEC_FFN_GELU = 0, SPEC_FFN_GATED_GELU = 1, SPEC_FFN_SWIGLU = 2 };
 enum { SPEC_DTYPE_FP32 = 0, SPEC_DTYPE_BF16 = 1 };
 
@@ -188,6 +202,9 @@ typedef struct spec_model_cfg {
     int dtype;            /* SPEC_DTYPE_* of every matrix */
     float rms_eps;
     float rope_base;
+    int n_enc_layers;     /* T5: encoder blocks (0 otherwise) */
+    int rel_buckets;      /* T5: rows of the bias tables (even, 2..256) */
+    int rel_max_distance; /* T5: distance from which the last bucket is used */
 } spec_model_cfg;
 
 typedef struct spec_layer_weights {
@@ -197,6 +214,11 @@ typedef struct spec_layer_weights {
     const float* ln2;     /* [d_model] */
     const void* w_in;     /* [d_ff or 2 d_ff, d_model] */
     const void* w_out;    /* [d_model, d_ff] */
+    /* T5 decoder blocks only (NULL otherwise): cross-attention */
+    const float* lnx;     /* [d_model] */
+    const void* wq_x;     /* [n_heads d_head, d_model] */
+    const void* wkv_x;    /* [2 n_heads d_head, d_model]: k rows, v rows */
+    const void* wo_x;     /* [d_model, n_heads d_head] */
 } spec_layer_weights;
 
 /* All pointers are DEVICE pointers that the caller keeps alive until
@@ -208,6 +230,11 @@ typedef struct spec_weights {
     const float* ln_f;    /* [d_model] */
     const void* head;     /* [vocab, d_model]; ignored when tied_embeddings */
     const spec_layer_weights* layers;
+    /* T5 only (NULL otherwise) */
+    const spec_layer_weights* enc_layers; /* HOST array of n_enc_layers entries */
+    const float* enc_ln_f;                /* [d_model] */
+    const float* enc_rel_bias;            /* fp32 [rel_buckets, n_heads] */
+    const float* rel_bias;                /* fp32 [rel_buckets, n_heads], decoder */
 } spec_weights;
 
 typedef struct spec_runtime_cfg {
@@ -218,6 +245,7 @@ typedef struct spec_runtime_cfg {
     int kv_dtype;         /* SPEC_DTYPE_FP32 or SPEC_DTYPE_BF16: element type of the cached K,V rows.
                              bf16 halves the KV traffic but rounds every cached row to 8 mantissa
                              bits, which on deep models moves logits by more than 2e-2. */
+    int max_src_len;      /* T5: longest source the encoders are given (0 for decoder-only models) */
 } spec_runtime_cfg;
 
 typedef struct spec_ctx spec_ctx;
@@ -278,6 +306,12 @@ int spec_generate(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_le
                   int batch, int n_new, int gamma, float temperature, uint64_t seed,
                   int32_t* out_tokens, spec_stats* stats);
 
+/* Encoder-decoder models (SPEC_ARCH_T5): `prompt` holds the SOURCE of every
+ * sequence.  spec_generate / spec_begin run both encoders over it once, keep
+ * the cross-attention K,V of every decoder block, and then decode n_new tokens
+ * from the start token 0 exactly as above (the decoder's "prompt" is that one
+ * token).  SPEC_ERR_CAPACITY also if a source is longer than max_src_len. */
+
 /* The same generation in phases, for callers that interleave other work or
  * time the decode loop: spec_begin validates the request, uploads the prompts
  * and runs the prompt pass (arguments as for spec_generate); spec_step runs
@@ -291,6 +325,22 @@ int spec_generate(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_le
  * generation in progress. */
 int spec_begin(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride,
                int batch, int n_new, int gamma, float temperature, uint64_t seed);
+
+/* Encoder-decoder models only: runs the encoder of every model of the context
+ * over the sources (HOST int32 [batch, source_stride], source_len[b] >= 1
+ * entries used) and stores the cross-attention K,V; forgets every cached
+ * decoder row.  spec_generate and spec_begin call it themselves; the
+ * teacher-forced diagnostics below need it called first.  Blocks until done.
+ * Errors: SPEC_ERR_BAD_ARG, SPEC_ERR_BAD_CONFIG (not an encoder-decoder
+ * context), SPEC_ERR_CAPACITY (batch > max_batch, a source longer than
+ * max_src_len). */
+int spec_encode(spec_ctx* ctx, const int32_t* source, const int32_t* source_len, int source_stride, int batch);
+
+/* The relative-position bucket of SPEC_ARCH_T5 for delta = key position - query
+ * position (host arithmetic only; exported so that it can be checked without a
+ * GPU).  Negative return: SPEC_ERR_BAD_ARG for a table shape spec_init would
+ * reject. */
+int spec_rel_bucket(int delta, int bidirectional, int n_buckets, int max_distance);
 int spec_step(spec_ctx* ctx, int iterations, int* remaining, spec_stats* stats);
 int spec_read_tokens(spec_ctx* ctx, int32_t* out_tokens);
 

@@ -229,20 +229,25 @@ def spec_device_error():
 class _ModelCfg(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("arch", "n_layers", "d_model", "n_heads", "n_kv_heads", "d_head", "d_ff",
                                             "ffn", "vocab", "max_positions", "tied_embeddings", "dtype")] + \
-               [("rms_eps", ctypes.c_float), ("rope_base", ctypes.c_float)]
+               [("rms_eps", ctypes.c_float), ("rope_base", ctypes.c_float)] + \
+               [(n, ctypes.c_int) for n in ("n_enc_layers", "rel_buckets", "rel_max_distance")]
 
 
 class _LayerWeights(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_void_p) for n in ("ln1", "wqkv", "wo", "ln2", "w_in", "w_out")]
+    _fields_ = [(n, ctypes.c_void_p) for n in ("ln1", "wqkv", "wo", "ln2", "w_in", "w_out",
+                                               "lnx", "wq_x", "wkv_x", "wo_x")]
 
 
 class _Weights(ctypes.Structure):
     _fields_ = [("tok_emb", ctypes.c_void_p), ("pos_emb", ctypes.c_void_p), ("ln_f", ctypes.c_void_p),
-                ("head", ctypes.c_void_p), ("layers", ctypes.POINTER(_LayerWeights))]
+                ("head", ctypes.c_void_p), ("layers", ctypes.POINTER(_LayerWeights)),
+                ("enc_layers", ctypes.POINTER(_LayerWeights)), ("enc_ln_f", ctypes.c_void_p),
+                ("enc_rel_bias", ctypes.c_void_p), ("rel_bias", ctypes.c_void_p)]
 
 
 class _RuntimeCfg(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int) for n in ("max_batch", "max_len", "page_size", "max_gamma", "kv_dtype")]
+    _fields_ = [(n, ctypes.c_int) for n in ("max_batch", "max_len", "page_size", "max_gamma", "kv_dtype",
+                                            "max_src_len")]
 
 
 class _Stats(ctypes.Structure):
@@ -251,7 +256,7 @@ class _Stats(ctypes.Structure):
                [("prefill_ms", ctypes.c_double), ("decode_ms", ctypes.c_double)]
 
 
-_ARCH = {"gpt": 0, "llama": 1}
+_ARCH = {"gpt": 0, "llama": 1, "t5": 2}
 _FFN = {"gelu": 0, "gated_gelu": 1, "swiglu": 2}
 _DTYPE = {"fp32": 0, "bf16": 1}
 _engine_declared = False
@@ -283,13 +288,16 @@ def _declare_engine(h):
     h.spec_truncate.argtypes = [vp, c.c_int, vp, c.c_int]
     h.spec_forward_logits.restype = c.c_int
     h.spec_forward_logits.argtypes = [vp, c.c_int, vp, c.c_int, c.c_int, vp]
+    h.spec_encode.restype = c.c_int
+    h.spec_encode.argtypes = [vp, vp, vp, c.c_int, c.c_int]
     _engine_declared = True
 
 
 def _cfg_struct(cfg):
     return _ModelCfg(_ARCH[cfg["arch"]], cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["n_kv_heads"],
                      cfg["d_head"], cfg["d_ff"], _FFN[cfg["ffn"]], cfg["vocab"], cfg["max_positions"],
-                     1 if cfg["tied"] else 0, _DTYPE[cfg["dtype"]], cfg["rms_eps"], cfg["rope_base"])
+                     1 if cfg["tied"] else 0, _DTYPE[cfg["dtype"]], cfg["rms_eps"], cfg["rope_base"],
+                     cfg.get("n_enc_layers", 0), cfg.get("rel_buckets", 0), cfg.get("rel_max_distance", 0))
 
 
 class Engine:
@@ -302,7 +310,7 @@ class Engine:
     """
 
     def __init__(self, target_cfg, target_weights, draft_cfg=None, draft_weights=None, max_batch=1, max_len=256,
-                 page_size=64, max_gamma=8, kv_dtype="fp32", device=None):
+                 page_size=64, max_gamma=8, kv_dtype="fp32", device=None, max_src_len=0):
         import numpy as np
         self._np = np
         h = lib()
@@ -313,7 +321,7 @@ class Engine:
         structs = []
         for cfg, weights in ((target_cfg, target_weights), (draft_cfg, draft_weights)):
             structs.append(None if cfg is None else self._upload(cfg, weights))
-        rt = _RuntimeCfg(max_batch, max_len, page_size, max_gamma, _DTYPE[kv_dtype])
+        rt = _RuntimeCfg(max_batch, max_len, page_size, max_gamma, _DTYPE[kv_dtype], max_src_len)
         self.max_batch, self.max_len, self.max_gamma = max_batch, max_len, max_gamma
         ctx = ctypes.c_void_p()
         tc = _cfg_struct(target_cfg)
@@ -334,13 +342,28 @@ class Engine:
             self._keep.append(t)
             return t.data_ptr()
 
+        t5 = cfg["arch"] == "t5"
+
+        def block(p, cross):
+            extra = (dev(p + "lnx", False), dev(p + "wq_x", True), dev(p + "wkv_x", True), dev(p + "wo_x", True)) \
+                if cross else (None, None, None, None)
+            return _LayerWeights(dev(p + "ln1", False), dev(p + "wqkv", True), dev(p + "wo", True),
+                                 dev(p + "ln2", False), dev(p + "w_in", True), dev(p + "w_out", True), *extra)
+
         layers = (_LayerWeights * cfg["n_layers"])()
         for l in range(cfg["n_layers"]):
-            layers[l] = _LayerWeights(dev(f"l{l}.ln1", False), dev(f"l{l}.wqkv", True), dev(f"l{l}.wo", True),
-                                      dev(f"l{l}.ln2", False), dev(f"l{l}.w_in", True), dev(f"l{l}.w_out", True))
+            layers[l] = block(f"l{l}.", t5)
         self._keep.append(layers)
+        enc_layers = None
+        if t5:
+            enc_layers = (_LayerWeights * cfg["n_enc_layers"])()
+            for l in range(cfg["n_enc_layers"]):
+                enc_layers[l] = block(f"enc.l{l}.", False)
+            self._keep.append(enc_layers)
         return _Weights(dev("tok_emb", True), dev("pos_emb", True) if cfg["arch"] == "gpt" else None,
-                        dev("ln_f", False), None if cfg["tied"] else dev("head", True), layers)
+                        dev("ln_f", False), None if cfg["tied"] else dev("head", True), layers,
+                        enc_layers, dev("enc.ln_f", False) if t5 else None,
+                        dev("enc.rel_bias", False) if t5 else None, dev("rel_bias", False) if t5 else None)
 
     def close(self):
         if getattr(self, "_ctx", None):
@@ -400,6 +423,12 @@ class Engine:
                                    float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF, out.ctypes.data,
                                    ctypes.byref(st)))
         return out, {name: getattr(st, name) for name, _ in _Stats._fields_}
+
+    def encode(self, sources):
+        """Encoder-decoder models: run the encoders over `sources` (list of 1-D int
+        arrays) and keep the cross-attention K,V; clears the decoder caches."""
+        flat, lens, stride = self._pack_prompts(sources)
+        _check(lib().spec_encode(self._ctx, flat.ctypes.data, lens.ctypes.data, stride, len(sources)))
 
     def reset(self):
         _check(lib().spec_reset(self._ctx))

@@ -1,4 +1,7 @@
-// Causal attention of the new rows against the paged KV cache.
+// Attention of the rows of a pass against paged K,V rows: causal over the
+// decoder cache (row at position p sees keys 0..p), or over a fixed set of keys
+// per sequence (the encoder's own rows; the cross-attention rows of an
+// encoder-decoder), optionally with an additive relative-position bias.
 //
 // Work is cut by (sequence, KV head, slice of the keys).  A CTA owns one such
 // piece and runs one warp per query that reads this KV head: the G query heads
@@ -76,10 +79,11 @@ struct KvLoad<__nv_bfloat16> {
 // Rows of sequence b are rows b*m .. b*m+m-1 of the pass.
 template <typename KV, int DH>
 __global__ void __launch_bounds__(32 * kMaxAttnWarps)
-attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos, const int32_t* __restrict__ seq,
-                 int m_rows, int n_heads, int n_kv_heads, int ks, const KV* __restrict__ kv_layer,
-                 const int32_t* __restrict__ page_table, int pages_per_seq, int page_size, float scale,
-                 float* __restrict__ part) {
+attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __restrict__ pos,
+                 const int32_t* __restrict__ seq, int m_rows, int n_heads, int n_kv_heads, int ks,
+                 const KV* __restrict__ kv_layer, const int32_t* __restrict__ page_table, int pages_per_seq,
+                 int page_size, const int32_t* __restrict__ kv_len, const float* __restrict__ bias, int bias_span,
+                 int bias_zero, float scale, float* __restrict__ part) {
     constexpr int PER_LANE = DH / 32;
     __shared__ float share[kMaxAttnWarps][DH + 2];  // states of the warps that share a query (ks > 1)
     pdl_trigger();
@@ -88,12 +92,15 @@ attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
     const int slice = blockIdx.x, slices = gridDim.x, kv_head = blockIdx.y, b = blockIdx.z;
     const int group = n_heads / n_kv_heads;
     const int queries = group * m_rows;
-    const int qkv_dim = (n_heads + 2 * n_kv_heads) * DH;
 
     // the key range of this slice: whole tiles, same for every query of the sequence
-    int max_pos = -1;
-    for (int j = 0; j < m_rows; ++j) max_pos = max(max_pos, pos[b * m_rows + j]);
-    const int tiles = (max_pos + 1 + 31) / 32;
+    int seq_keys = 0;
+    if (kv_len) {
+        seq_keys = kv_len[seq[b * m_rows]];
+    } else {
+        for (int j = 0; j < m_rows; ++j) seq_keys = max(seq_keys, pos[b * m_rows + j] + 1);
+    }
+    const int tiles = (seq_keys + 31) / 32;
     const int t0 = static_cast<int>(static_cast<long long>(tiles) * slice / slices);
     const int t1 = static_cast<int>(static_cast<long long>(tiles) * (slice + 1) / slices);
 
@@ -111,7 +118,7 @@ attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
         const int p = pos[r];
         const int32_t* pages = page_table + seq[r] * pages_per_seq;
         float qv[PER_LANE];  // this lane's share of the (scaled) query
-        KvLoad<float>::template load_n<PER_LANE>(qkv + static_cast<size_t>(r) * qkv_dim + head * DH + lane * PER_LANE, qv);
+        KvLoad<float>::template load_n<PER_LANE>(qkv + static_cast<size_t>(r) * q_stride + head * DH + lane * PER_LANE, qv);
 #pragma unroll
         for (int i = 0; i < PER_LANE; ++i) qv[i] *= scale;
 
@@ -119,7 +126,9 @@ attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
         float acc[PER_LANE];
 #pragma unroll
         for (int i = 0; i < PER_LANE; ++i) acc[i] = 0.0f;
-        const int n_keys = p + 1;  // causal: positions 0..p (p < 0: inactive row, no keys)
+        // causal: positions 0..p; otherwise the sequence's key set (p < 0: inactive row, no keys)
+        const int n_keys = kv_len ? (p >= 0 ? seq_keys : 0) : p + 1;
+        const float* bias_row = bias ? bias + static_cast<size_t>(head) * bias_span + (bias_zero - p) : nullptr;
         for (int t = t0 + sub; t < t1; t += ks) {
             const int k0 = 32 * t;
             if (k0 >= n_keys) break;
@@ -156,7 +165,8 @@ attention_kernel(const float* __restrict__ qkv, const int32_t* __restrict__ pos,
                     pd[i] = keep + __shfl_xor_sync(kFullMask, send, step);
                 }
             }
-            const float s = lane < in_tile ? pd[0] : -FLT_MAX;
+            float s = -FLT_MAX;
+            if (lane < in_tile) s = bias_row ? pd[0] + bias_row[k0 + lane] : pd[0];
             const float m_new = fmaxf(mx, warp_max(s));
             const float pr = lane < in_tile ? expf(s - m_new) : 0.0f;
             const float rescale = expf(mx - m_new);
@@ -288,10 +298,8 @@ size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices) {
     return static_cast<size_t>(rows) * n_heads * slices * (d_head + 2);
 }
 
-int launch_attention(const Model& m, int layer, const RowMeta& rows, int batch, int m_rows, int slices,
-                     const float* qkv, float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo,
-                     const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream) {
-    const char* kv_layer = static_cast<const char*>(m.kv) + static_cast<size_t>(layer) * m.layer_stride;
+int launch_attention(const Model& m, const AttnSource& src, const RowMeta& rows, int batch, int m_rows, int slices,
+                     float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo, cudaStream_t stream) {
     const int group = m.cfg.n_heads / m.cfg.n_kv_heads;
     const int ks = attention_sub_slices(group * m_rows);
     const int warps = std::min(kMaxAttnWarps, std::max(1, group * m_rows * ks));
@@ -300,15 +308,16 @@ int launch_attention(const Model& m, int layer, const RowMeta& rows, int batch, 
     const int n_rows = batch * m_rows;
 #define SPEC_ATTN(KV, DH)                                                                                         \
     do {                                                                                                          \
-        int status = launch_pdl(attention_kernel<KV, DH>, grid, dim3(32 * warps), 0, stream, qkv, rows.pos,       \
-                                rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads, ks,                            \
-                                reinterpret_cast<const KV*>(kv_layer), page_table, pages_per_seq, page_size,      \
-                                scale, part);                                                                     \
+        int status = launch_pdl(attention_kernel<KV, DH>, grid, dim3(32 * warps), 0, stream, src.q, src.q_stride, \
+                                rows.pos, rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads, ks,                  \
+                                static_cast<const KV*>(src.pool.kv), src.pool.page_table, src.pool.pages_per_seq,     \
+                                src.pool.page_size,                                                               \
+                                src.kv_len, src.bias, src.bias_span, src.bias_zero, scale, part);                 \
         if (status != SPEC_OK) return status;                                                                     \
         return launch_pdl(attention_combine_kernel<DH>, dim3(n_rows * m.cfg.n_heads), dim3(DH), 0, stream,         \
                           static_cast<const float*>(part), slices, att, att_hi, att_lo);                          \
     } while (0)
-    if (m.kv_elem_bytes == 2) {
+    if (src.pool.elem_bytes == 2) {
         if (m.cfg.d_head == 64) SPEC_ATTN(__nv_bfloat16, 64);
         else SPEC_ATTN(__nv_bfloat16, 128);
     } else {

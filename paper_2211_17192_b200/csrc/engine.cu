@@ -16,8 +16,14 @@ struct spec_ctx {
     spec_runtime_cfg rt{};
     cudaStream_t stream = nullptr;
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
-    int max_rows = 0;
+    int max_rows = 0;       // rows of any pass (activations)
+    int max_logit_rows = 0;  // rows of the generation loop's logits buffers
     int pages_per_seq = 0;
+    // encoder-decoder contexts: the sources' own page table and lengths
+    int src_pages_per_seq = 0;
+    int32_t *src_page_table = nullptr, *src_len = nullptr;
+    bool encoded = false;
+    int encoded_batch = 0;
 
     // activations (sized for the wider model)
     float *h = nullptr, *a = nullptr, *qkv = nullptr, *att = nullptr, *u = nullptr, *f = nullptr;
@@ -59,7 +65,14 @@ namespace spec {
 namespace {
 
 int check_cfg(const spec_model_cfg& c, const char* which) {
-    if (c.arch != SPEC_ARCH_GPT && c.arch != SPEC_ARCH_LLAMA) return fail(SPEC_ERR_BAD_CONFIG, "%s: unknown arch %d", which, c.arch);
+    if (c.arch != SPEC_ARCH_GPT && c.arch != SPEC_ARCH_LLAMA && c.arch != SPEC_ARCH_T5)
+        return fail(SPEC_ERR_BAD_CONFIG, "%s: unknown arch %d", which, c.arch);
+    if (c.arch == SPEC_ARCH_T5) {
+        if (c.n_enc_layers < 1 || c.n_kv_heads != c.n_heads || c.tied_embeddings)
+            return fail(SPEC_ERR_BAD_CONFIG, "%s: encoder-decoder needs n_enc_layers >= 1, n_kv_heads == n_heads, an untied head", which);
+        if (c.rel_buckets < 4 || c.rel_buckets > 256 || c.rel_buckets % 4 || c.rel_max_distance <= c.rel_buckets / 2)
+            return fail(SPEC_ERR_BAD_CONFIG, "%s: rel_buckets %d (multiple of 4, 4..256) / rel_max_distance %d", which, c.rel_buckets, c.rel_max_distance);
+    }
     if (c.n_layers < 1 || c.d_model < 8 || c.n_heads < 1 || c.n_kv_heads < 1 || c.d_ff < 8 || c.vocab < 1 || c.max_positions < 1)
         return fail(SPEC_ERR_BAD_CONFIG, "%s: non-positive dimension", which);
     if (c.d_head != 64 && c.d_head != 128) return fail(SPEC_ERR_BAD_CONFIG, "%s: d_head %d (64 or 128 supported)", which, c.d_head);
@@ -90,71 +103,157 @@ int dev_alloc(spec_ctx* ctx, T** out, size_t count) {
         if (status__ != SPEC_OK) return status__; \
     } while (0)
 
-// One forward pass of `m` over the rows described by ctx->row_*; K,V rows of
-// active rows are appended to the cache.  If n_logit_rows > 0 the final norm and
-// LM head run on rows logit_src[i] and write logits rows logit_dst[i].
+// The GEMMs and hand-offs of a pass on either path.  bf16 models take the
+// tensor-core path: every GEMM leaves split-K partial sums that the next small
+// kernel adds up (a GEMM that closes a residual branch leaves them pending until
+// the next norm adds them into h), and every GEMM input is produced directly as
+// two bf16 terms.  fp32 models run the same kernels with fp32 hand-offs and the
+// FMA-pipe GEMM.
+struct Pass {
+    spec_ctx* ctx;
+    const Model& m;
+    int n_rows;
+    bool tc;
+    cudaStream_t st;
+    int pending = 0;      // split count of partial sums not yet added into h
+    int last_splits = 0;  // split count of the last projection
+
+    __nv_bfloat16* hi() const { return ctx->x_hi; }
+    __nv_bfloat16* lo() const { return ctx->x_lo; }
+
+    // a (fp32) or hi/lo = rmsnorm(h[src(i)]) * gain for i < n
+    int norm(const float* gain, const int32_t* src_rows, int n) {
+        const int d = m.cfg.d_model;
+        const int status = tc ? launch_norm(ctx->h, pending ? ctx->partials : nullptr, pending, n_rows, gain, src_rows, n, d,
+                                            m.cfg.rms_eps, nullptr, hi(), lo(), st)
+                              : launch_norm(ctx->h, nullptr, 0, n_rows, gain, src_rows, n, d, m.cfg.rms_eps, ctx->a, nullptr,
+                                            nullptr, st);
+        pending = 0;
+        return status;
+    }
+    // y = x . W^T for a consumer that is not the residual stream: partial sums (tc) or `y` (fp32 path, input `x`)
+    int proj(const void* w, const void* pw, int n_out, int k, const float* x, float* y) {
+        if (tc) {
+            last_splits = gemm_tc_splits(n_out, k, n_rows);
+            return launch_gemm_tc_partials(hi(), lo(), ctx->hi_rows, pw, true, n_rows, n_out, k, ctx->partials, st);
+        }
+        return launch_gemm_rows(x, w, m.bf16(), nullptr, nullptr, n_rows, n_out, k, y, st);
+    }
+    // h += x . W^T
+    int residual(const void* w, const void* pw, int k, const float* x) {
+        const int d = m.cfg.d_model;
+        if (tc) {
+            pending = gemm_tc_splits(d, k, n_rows);
+            return launch_gemm_tc_partials(hi(), lo(), ctx->hi_rows, pw, true, n_rows, d, k, ctx->partials, st);
+        }
+        return launch_gemm_rows(x, w, m.bf16(), ctx->h, nullptr, n_rows, d, k, ctx->h, st);
+    }
+    const float* partials() const { return tc ? ctx->partials : nullptr; }
+    // h += FFN(rmsnorm(h) * gain)
+    int ffn(const spec_layer_weights& w, const spec_layer_weights& pw) {
+        const spec_model_cfg& c = m.cfg;
+        SPEC_TRY(norm(w.ln2, nullptr, n_rows));
+        SPEC_TRY(proj(w.w_in, pw.w_in, m.ffn_in_dim(), c.d_model, ctx->a, ctx->u));
+        SPEC_TRY(launch_ffn_act(tc ? nullptr : ctx->u, partials(), last_splits, n_rows, c.d_ff, c.ffn, tc ? nullptr : ctx->f,
+                                tc ? hi() : nullptr, tc ? lo() : nullptr, st));
+        return residual(w.w_out, pw.w_out, c.d_ff, ctx->f);
+    }
+    // h += Wo . attention(projection of rmsnorm(h) * gain) over `pool`
+    int self_attention(const spec_layer_weights& w, const spec_layer_weights& pw, const RowMeta& rows, int batch, int m_rows,
+                       const KvPool& pool, const int32_t* kv_len, const float* bias, int bias_span, int bias_zero,
+                       int max_keys) {
+        const spec_model_cfg& c = m.cfg;
+        SPEC_TRY(norm(w.ln1, nullptr, n_rows));
+        SPEC_TRY(proj(w.wqkv, pw.wqkv, m.qkv_dim(), c.d_model, ctx->a, ctx->qkv));
+        SPEC_TRY(launch_qkv(c.n_heads, c.n_kv_heads, c.d_head, c.arch == SPEC_ARCH_LLAMA ? m.rope_table : nullptr, pool, rows,
+                            n_rows, ctx->qkv, partials(), last_splits, st));
+        const int slices = attention_slices(batch, c.n_kv_heads, (c.n_heads / c.n_kv_heads) * m_rows, max_keys);
+        const AttnSource src{ctx->qkv, m.qkv_dim(), pool, kv_len, bias, bias_span, bias_zero};
+        SPEC_TRY(launch_attention(m, src, rows, batch, m_rows, slices, ctx->attn_part, tc ? nullptr : ctx->att,
+                                  tc ? hi() : nullptr, tc ? lo() : nullptr, st));
+        return residual(w.wo, pw.wo, m.q_dim(), ctx->att);
+    }
+};
+
+KvPool layer_pool(const spec_ctx* ctx, const Model& m, int layer) {
+    return KvPool{static_cast<char*>(m.kv) + static_cast<size_t>(layer) * m.layer_stride, m.kv_elem_bytes, ctx->page_table,
+                  ctx->pages_per_seq, ctx->rt.page_size};
+}
+
+KvPool source_pool(const spec_ctx* ctx, const Model& m, void* base) {
+    return KvPool{base, m.kv_elem_bytes, ctx->src_page_table, ctx->src_pages_per_seq, ctx->rt.page_size};
+}
+
 // One forward pass of `m` over batch * m_rows rows (rows of sequence b are rows
 // b*m_rows .. of ctx->row_*); K,V rows of active rows are appended to the cache.
 // If n_logit_rows > 0 the final norm and LM head run on rows logit_src[i] and
-// write logits rows logit_dst[i].
-//
-// bf16 models take the tensor-core path: every GEMM leaves split-K partial sums
-// that the next small kernel adds up, and every GEMM input is produced directly
-// as two bf16 terms.  fp32 models run the same kernels with fp32 hand-offs and
-// the FMA-pipe GEMM.
+// write logits rows logit_dst[i] (all rows in order if both are null).
 int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_rows, const int32_t* logit_src,
             const int32_t* logit_dst, float* logits) {
-    cudaStream_t st = ctx->stream;
     const spec_model_cfg& c = m.cfg;
     const int n_rows = batch * m_rows;
     const RowMeta rows{ctx->row_token, ctx->row_pos, ctx->row_seq};
-    const bool tc = m.bf16() && ctx->tensor_cores;
-    __nv_bfloat16 *hi = tc ? ctx->x_hi : nullptr, *lo = tc ? ctx->x_lo : nullptr;
-    float* part = ctx->partials;
-    const int d = c.d_model, pages = ctx->pages_per_seq, page = ctx->rt.page_size;
-    const int slices = attention_slices(batch, c.n_kv_heads, (c.n_heads / c.n_kv_heads) * m_rows, ctx->rt.max_len);
-    // split-K factors of the four GEMM shapes of a block at this row count
-    const int s_qkv = tc ? gemm_tc_splits(m.qkv_dim(), d, n_rows) : 0;
-    const int s_o = tc ? gemm_tc_splits(d, m.q_dim(), n_rows) : 0;
-    const int s_in = tc ? gemm_tc_splits(m.ffn_in_dim(), d, n_rows) : 0;
-    const int s_out = tc ? gemm_tc_splits(d, c.d_ff, n_rows) : 0;
+    Pass pass{ctx, m, n_rows, m.bf16() && ctx->tensor_cores, ctx->stream};
+    const int d = c.d_model;
+    const float* bias = m.t5() ? m.dec_bias : nullptr;
 
-    SPEC_TRY(launch_embed(m, rows, n_rows, ctx->h, st));
+    SPEC_TRY(launch_embed(m, rows, n_rows, ctx->h, ctx->stream));
     for (int l = 0; l < c.n_layers; ++l) {
         const spec_layer_weights& w = m.layers[l];
-        if (tc) {
-            const spec_layer_weights& pw = m.packed[l];
-            // (the FFN-out partial sums of the previous block are added into h by this norm)
-            SPEC_TRY(launch_norm(ctx->h, l ? part : nullptr, s_out, n_rows, w.ln1, nullptr, n_rows, d, c.rms_eps, nullptr, hi, lo, st));
-            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, pw.wqkv, true, n_rows, m.qkv_dim(), d, part, st));
-            SPEC_TRY(launch_qkv(m, l, rows, n_rows, ctx->qkv, part, s_qkv, ctx->page_table, pages, page, st));
-            SPEC_TRY(launch_attention(m, l, rows, batch, m_rows, slices, ctx->qkv, ctx->attn_part, nullptr, hi, lo, ctx->page_table, pages, page, st));
-            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, pw.wo, true, n_rows, d, m.q_dim(), part, st));
-            SPEC_TRY(launch_norm(ctx->h, part, s_o, n_rows, w.ln2, nullptr, n_rows, d, c.rms_eps, nullptr, hi, lo, st));
-            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, pw.w_in, true, n_rows, m.ffn_in_dim(), d, part, st));
-            SPEC_TRY(launch_ffn_act(nullptr, part, s_in, n_rows, c.d_ff, c.ffn, nullptr, hi, lo, st));
-            SPEC_TRY(launch_gemm_tc_partials(hi, lo, ctx->hi_rows, pw.w_out, true, n_rows, d, c.d_ff, part, st));
-        } else {
-            const bool bf = m.bf16();
-            SPEC_TRY(launch_norm(ctx->h, nullptr, 0, n_rows, w.ln1, nullptr, n_rows, d, c.rms_eps, ctx->a, nullptr, nullptr, st));
-            SPEC_TRY(launch_gemm_rows(ctx->a, w.wqkv, bf, nullptr, nullptr, n_rows, m.qkv_dim(), d, ctx->qkv, st));
-            SPEC_TRY(launch_qkv(m, l, rows, n_rows, ctx->qkv, nullptr, 0, ctx->page_table, pages, page, st));
-            SPEC_TRY(launch_attention(m, l, rows, batch, m_rows, slices, ctx->qkv, ctx->attn_part, ctx->att, nullptr, nullptr, ctx->page_table, pages, page, st));
-            SPEC_TRY(launch_gemm_rows(ctx->att, w.wo, bf, ctx->h, nullptr, n_rows, d, m.q_dim(), ctx->h, st));
-            SPEC_TRY(launch_norm(ctx->h, nullptr, 0, n_rows, w.ln2, nullptr, n_rows, d, c.rms_eps, ctx->a, nullptr, nullptr, st));
-            SPEC_TRY(launch_gemm_rows(ctx->a, w.w_in, bf, nullptr, nullptr, n_rows, m.ffn_in_dim(), d, ctx->u, st));
-            SPEC_TRY(launch_ffn_act(ctx->u, nullptr, 0, n_rows, c.d_ff, c.ffn, ctx->f, nullptr, nullptr, st));
-            SPEC_TRY(launch_gemm_rows(ctx->f, w.w_out, bf, ctx->h, nullptr, n_rows, d, c.d_ff, ctx->h, st));
+        const spec_layer_weights& pw = pass.tc ? m.packed[l] : w;
+        SPEC_TRY(pass.self_attention(w, pw, rows, batch, m_rows, layer_pool(ctx, m, l), nullptr, bias, ctx->rt.max_len,
+                                     ctx->rt.max_len - 1, ctx->rt.max_len));
+        if (m.t5()) {  // cross-attention over the source's K,V (every row sees every source position)
+            SPEC_TRY(pass.norm(w.lnx, nullptr, n_rows));
+            SPEC_TRY(pass.proj(w.wq_x, pw.wq_x, m.q_dim(), d, ctx->a, ctx->qkv));
+            if (pass.tc)  // the partial sums become the query rows
+                SPEC_TRY(launch_qkv(c.n_heads, 0, c.d_head, nullptr, KvPool{}, rows, n_rows, ctx->qkv, ctx->partials,
+                                    pass.last_splits, ctx->stream));
+            const KvPool pool = source_pool(ctx, m, static_cast<char*>(m.cross_kv) + static_cast<size_t>(l) * m.cross_stride);
+            const int slices = attention_slices(batch, c.n_kv_heads, m_rows, ctx->rt.max_src_len);
+            const AttnSource src{ctx->qkv, m.q_dim(), pool, ctx->src_len, nullptr, 0, 0};
+            SPEC_TRY(launch_attention(m, src, rows, batch, m_rows, slices, ctx->attn_part, pass.tc ? nullptr : ctx->att,
+                                      pass.tc ? pass.hi() : nullptr, pass.tc ? pass.lo() : nullptr, ctx->stream));
+            SPEC_TRY(pass.residual(w.wo_x, pw.wo_x, m.q_dim(), ctx->att));
         }
+        SPEC_TRY(pass.ffn(w, pw));
     }
     if (n_logit_rows > 0) {
-        if (tc) {
-            SPEC_TRY(launch_norm(ctx->h, part, s_out, n_rows, m.ln_f, logit_src, n_logit_rows, d, c.rms_eps, nullptr, hi, lo, st));
-            SPEC_TRY(launch_gemm_tc(hi, lo, ctx->hi_rows, m.packed_head, true, nullptr, logit_dst, n_logit_rows, c.vocab, d, part, logits, st));
-        } else {
-            SPEC_TRY(launch_norm(ctx->h, nullptr, 0, n_rows, m.ln_f, logit_src, n_logit_rows, d, c.rms_eps, ctx->a, nullptr, nullptr, st));
-            SPEC_TRY(launch_gemm_rows(ctx->a, m.head, m.bf16(), nullptr, logit_dst, n_logit_rows, c.vocab, d, logits, st));
-        }
+        SPEC_TRY(pass.norm(m.ln_f, logit_src, n_logit_rows));
+        if (pass.tc)
+            SPEC_TRY(launch_gemm_tc(pass.hi(), pass.lo(), ctx->hi_rows, m.packed_head, true, nullptr, logit_dst, n_logit_rows,
+                                    c.vocab, d, ctx->partials, logits, ctx->stream));
+        else
+            SPEC_TRY(launch_gemm_rows(ctx->a, m.head, m.bf16(), nullptr, logit_dst, n_logit_rows, c.vocab, d, logits, ctx->stream));
+    }
+    return SPEC_OK;
+}
+
+// The encoder of `m` over batch * m_rows source rows described by ctx->row_*
+// (inactive rows pad short sources), then the cross-attention K,V of every
+// decoder block from its output.
+int encode(spec_ctx* ctx, const Model& m, int batch, int m_rows) {
+    const spec_model_cfg& c = m.cfg;
+    const int n_rows = batch * m_rows;
+    const RowMeta rows{ctx->row_token, ctx->row_pos, ctx->row_seq};
+    Pass pass{ctx, m, n_rows, m.bf16() && ctx->tensor_cores, ctx->stream};
+    const int S = ctx->rt.max_src_len;
+    SPEC_TRY(launch_embed(m, rows, n_rows, ctx->h, ctx->stream));
+    for (int l = 0; l < c.n_enc_layers; ++l) {
+        const spec_layer_weights& w = m.enc_layers[l];
+        const spec_layer_weights& pw = pass.tc ? m.enc_packed[l] : w;
+        SPEC_TRY(pass.self_attention(w, pw, rows, batch, m_rows, source_pool(ctx, m, m.enc_kv), ctx->src_len, m.enc_bias,
+                                     2 * S - 1, S - 1, S));
+        SPEC_TRY(pass.ffn(w, pw));
+    }
+    SPEC_TRY(pass.norm(m.enc_ln_f, nullptr, n_rows));  // the encoder output, input of every Wkv_x
+    for (int l = 0; l < c.n_layers; ++l) {
+        const spec_layer_weights& w = m.layers[l];
+        const spec_layer_weights& pw = pass.tc ? m.packed[l] : w;
+        SPEC_TRY(pass.proj(w.wkv_x, pw.wkv_x, 2 * m.kv_dim(), c.d_model, ctx->a, ctx->qkv));
+        const KvPool pool = source_pool(ctx, m, static_cast<char*>(m.cross_kv) + static_cast<size_t>(l) * m.cross_stride);
+        SPEC_TRY(launch_qkv(0, c.n_kv_heads, c.d_head, nullptr, pool, rows, n_rows, ctx->qkv, pass.partials(),
+                            pass.last_splits, ctx->stream));
     }
     return SPEC_OK;
 }
@@ -360,13 +459,24 @@ int pack_model(spec_ctx* ctx, Model& m) {
         *out = dst;
         return SPEC_OK;
     };
+    auto pack_block = [&](const spec_layer_weights& w, spec_layer_weights& out) -> int {
+        SPEC_TRY(pack(w.wqkv, m.qkv_dim(), c.d_model, &out.wqkv));
+        SPEC_TRY(pack(w.wo, c.d_model, m.q_dim(), &out.wo));
+        SPEC_TRY(pack(w.w_in, m.ffn_in_dim(), c.d_model, &out.w_in));
+        SPEC_TRY(pack(w.w_out, c.d_model, c.d_ff, &out.w_out));
+        return SPEC_OK;
+    };
     m.packed.assign(c.n_layers, spec_layer_weights{});
     for (int l = 0; l < c.n_layers; ++l) {
-        SPEC_TRY(pack(m.layers[l].wqkv, m.qkv_dim(), c.d_model, &m.packed[l].wqkv));
-        SPEC_TRY(pack(m.layers[l].wo, c.d_model, m.q_dim(), &m.packed[l].wo));
-        SPEC_TRY(pack(m.layers[l].w_in, m.ffn_in_dim(), c.d_model, &m.packed[l].w_in));
-        SPEC_TRY(pack(m.layers[l].w_out, c.d_model, c.d_ff, &m.packed[l].w_out));
+        SPEC_TRY(pack_block(m.layers[l], m.packed[l]));
+        if (m.t5()) {
+            SPEC_TRY(pack(m.layers[l].wq_x, m.q_dim(), c.d_model, &m.packed[l].wq_x));
+            SPEC_TRY(pack(m.layers[l].wkv_x, 2 * m.kv_dim(), c.d_model, &m.packed[l].wkv_x));
+            SPEC_TRY(pack(m.layers[l].wo_x, c.d_model, m.q_dim(), &m.packed[l].wo_x));
+        }
     }
+    m.enc_packed.assign(m.enc_layers.size(), spec_layer_weights{});
+    for (size_t l = 0; l < m.enc_layers.size(); ++l) SPEC_TRY(pack_block(m.enc_layers[l], m.enc_packed[l]));
     SPEC_TRY(pack(m.head, c.vocab, c.d_model, &m.packed_head));
     SPEC_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
     return SPEC_OK;
@@ -385,6 +495,18 @@ int init_model(spec_ctx* ctx, int which, const spec_model_cfg& cfg, const spec_w
     for (const spec_layer_weights& l : m.layers)
         if (!l.ln1 || !l.wqkv || !l.wo || !l.ln2 || !l.w_in || !l.w_out)
             return fail(SPEC_ERR_BAD_ARG, "spec_init: missing layer weight pointer");
+    if (m.t5()) {
+        if (!w.enc_layers || !w.enc_ln_f || !w.enc_rel_bias || !w.rel_bias)
+            return fail(SPEC_ERR_BAD_ARG, "spec_init: missing encoder weight pointer");
+        m.enc_layers.assign(w.enc_layers, w.enc_layers + cfg.n_enc_layers);
+        m.enc_ln_f = w.enc_ln_f;
+        for (const spec_layer_weights& l : m.enc_layers)
+            if (!l.ln1 || !l.wqkv || !l.wo || !l.ln2 || !l.w_in || !l.w_out)
+                return fail(SPEC_ERR_BAD_ARG, "spec_init: missing encoder layer weight pointer");
+        for (const spec_layer_weights& l : m.layers)
+            if (!l.lnx || !l.wq_x || !l.wkv_x || !l.wo_x)
+                return fail(SPEC_ERR_BAD_ARG, "spec_init: missing cross-attention weight pointer");
+    }
     m.kv_elem_bytes = ctx->rt.kv_dtype == SPEC_DTYPE_BF16 ? 2 : 4;
     const size_t n_pages = static_cast<size_t>(ctx->rt.max_batch) * ctx->pages_per_seq;
     m.layer_stride = n_pages * 2 * cfg.n_kv_heads * ctx->rt.page_size * cfg.d_head * m.kv_elem_bytes;
@@ -399,6 +521,37 @@ int init_model(spec_ctx* ctx, int which, const spec_model_cfg& cfg, const spec_w
         SPEC_CUDA_TRY(cudaMemcpy(dev, table.data(), table.size() * sizeof(float2), cudaMemcpyHostToDevice));
         m.rope_table = dev;
     }
+    if (m.t5()) {
+        // pools of the source positions: the encoder block in flight and every decoder block's cross K,V
+        const size_t src_pages = static_cast<size_t>(ctx->rt.max_batch) * ctx->src_pages_per_seq;
+        m.cross_stride = src_pages * 2 * cfg.n_kv_heads * ctx->rt.page_size * cfg.d_head * m.kv_elem_bytes;
+        char *enc_kv = nullptr, *cross = nullptr;
+        SPEC_TRY(dev_alloc(ctx, &enc_kv, m.cross_stride));
+        SPEC_TRY(dev_alloc(ctx, &cross, m.cross_stride * cfg.n_layers));
+        m.enc_kv = enc_kv;
+        m.cross_kv = cross;
+        // bias tables by relative position, from the bucket tables
+        const int H = cfg.n_heads, B = cfg.rel_buckets, S = ctx->rt.max_src_len, L = ctx->rt.max_len;
+        std::vector<float> enc_table(static_cast<size_t>(B) * H), dec_table(enc_table.size());
+        SPEC_CUDA_TRY(cudaMemcpy(enc_table.data(), w.enc_rel_bias, enc_table.size() * sizeof(float), cudaMemcpyDeviceToHost));
+        SPEC_CUDA_TRY(cudaMemcpy(dec_table.data(), w.rel_bias, dec_table.size() * sizeof(float), cudaMemcpyDeviceToHost));
+        std::vector<float> enc_bias(static_cast<size_t>(H) * (2 * S - 1)), dec_bias(static_cast<size_t>(H) * L);
+        for (int h = 0; h < H; ++h) {
+            for (int delta = -(S - 1); delta <= S - 1; ++delta)
+                enc_bias[static_cast<size_t>(h) * (2 * S - 1) + delta + S - 1] =
+                    enc_table[static_cast<size_t>(spec_rel_bucket(delta, 1, B, cfg.rel_max_distance)) * H + h];
+            for (int delta = -(L - 1); delta <= 0; ++delta)
+                dec_bias[static_cast<size_t>(h) * L + delta + L - 1] =
+                    dec_table[static_cast<size_t>(spec_rel_bucket(delta, 0, B, cfg.rel_max_distance)) * H + h];
+        }
+        float *enc_dev = nullptr, *dec_dev = nullptr;
+        SPEC_TRY(dev_alloc(ctx, &enc_dev, enc_bias.size()));
+        SPEC_TRY(dev_alloc(ctx, &dec_dev, dec_bias.size()));
+        SPEC_CUDA_TRY(cudaMemcpy(enc_dev, enc_bias.data(), enc_bias.size() * sizeof(float), cudaMemcpyHostToDevice));
+        SPEC_CUDA_TRY(cudaMemcpy(dec_dev, dec_bias.data(), dec_bias.size() * sizeof(float), cudaMemcpyHostToDevice));
+        m.enc_bias = enc_dev;
+        m.dec_bias = dec_dev;
+    }
     return SPEC_OK;
 }
 
@@ -406,6 +559,22 @@ int init_model(spec_ctx* ctx, int which, const spec_model_cfg& cfg, const spec_w
 }  // namespace spec
 
 using namespace spec;
+
+extern "C" int spec_rel_bucket(int delta, int bidirectional, int n_buckets, int max_distance) {
+    if (n_buckets < 4 || n_buckets % 4 || max_distance <= n_buckets / 2) return fail(SPEC_ERR_BAD_ARG, "spec_rel_bucket: bad table shape");
+    int n = n_buckets, base = 0, dist;
+    if (bidirectional) {
+        n /= 2;
+        base = delta > 0 ? n : 0;  // keys after the query use the upper half
+        dist = std::abs(delta);
+    } else {
+        dist = std::max(-delta, 0);  // only keys at or before the query matter
+    }
+    const int exact = n / 2;  // distances below this have a bucket each
+    if (dist < exact) return base + dist;
+    const double spread = std::log(static_cast<double>(dist) / exact) / std::log(static_cast<double>(max_distance) / exact) * (n - exact);
+    return base + std::min(exact + static_cast<int>(std::floor(spread)), n - 1);
+}
 
 extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg* draft_cfg,
                          const spec_weights* target_weights, const spec_weights* draft_weights,
@@ -417,7 +586,13 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     if (draft_cfg) {
         SPEC_TRY(check_cfg(*draft_cfg, "draft"));
         if (draft_cfg->vocab != target_cfg->vocab) return fail(SPEC_ERR_BAD_CONFIG, "spec_init: vocabularies differ");
+        if ((draft_cfg->arch == SPEC_ARCH_T5) != (target_cfg->arch == SPEC_ARCH_T5))
+            return fail(SPEC_ERR_BAD_CONFIG, "spec_init: an encoder-decoder target needs an encoder-decoder draft and vice versa");
     }
+    const bool t5 = target_cfg->arch == SPEC_ARCH_T5;
+    if (t5 && (runtime->max_src_len < 1 || runtime->max_src_len > (1 << 16) ||
+               static_cast<long long>(runtime->max_src_len) * runtime->max_batch > (1 << 20)))
+        return fail(SPEC_ERR_BAD_CONFIG, "spec_init: max_src_len %d out of range for an encoder-decoder context", runtime->max_src_len);
     const spec_runtime_cfg& rt = *runtime;
     if (rt.max_batch < 1 || rt.max_batch > 4096 || rt.max_len < 2 || rt.max_gamma < 0 || rt.max_gamma > 64 ||
         rt.page_size < 32 || rt.page_size > 256 || (rt.page_size & (rt.page_size - 1)) ||
@@ -433,7 +608,12 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     ctx->rt = rt;
     ctx->has_draft = draft_cfg != nullptr;
     ctx->pages_per_seq = (rt.max_len + rt.page_size - 1) / rt.page_size;
-    ctx->max_rows = std::max(rt.max_batch * std::max(rt.max_gamma + 1, 2), 64);
+    ctx->max_logit_rows = std::max(rt.max_batch * std::max(rt.max_gamma + 1, 2), 64);
+    ctx->max_rows = ctx->max_logit_rows;
+    if (t5) {  // an encoder pass takes every source row of the batch at once
+        ctx->src_pages_per_seq = (rt.max_src_len + rt.page_size - 1) / rt.page_size;
+        ctx->max_rows = std::max(ctx->max_rows, rt.max_batch * rt.max_src_len);
+    }
     auto cleanup = [&](int status) {
         spec_free(ctx);
         return status;
@@ -457,11 +637,12 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
         ff = std::max<size_t>(ff, m.cfg.d_ff);
     }
     const size_t R = ctx->max_rows, B = rt.max_batch, G = rt.max_gamma, V = target_cfg->vocab;
+    const size_t RL = ctx->max_logit_rows;
 #define SPEC_ALLOC(ptr, count) \
     if ((status = dev_alloc(ctx, &ctx->ptr, (count))) != SPEC_OK) return cleanup(status)
     SPEC_ALLOC(h, R * d);
     SPEC_ALLOC(a, R * d);
-    SPEC_ALLOC(qkv, R * qkv);
+    SPEC_ALLOC(qkv, R * std::max(qkv, 2 * att));
     SPEC_ALLOC(att, R * att);
     SPEC_ALLOC(u, R * fin);
     SPEC_ALLOC(f, R * ff);
@@ -471,12 +652,14 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
             const Model& m = ctx->model[i];
             for (int b = 1; b <= rt.max_batch; ++b)
                 for (int mr = 1; b * mr <= ctx->max_rows; ++mr)
-                    attn = std::max(attn, attention_partial_elems(b * mr, m.cfg.n_heads, m.cfg.d_head,
-                                                                  attention_slices(b, m.cfg.n_kv_heads, (m.cfg.n_heads / m.cfg.n_kv_heads) * mr, rt.max_len)));
+                    for (int keys : {rt.max_len, rt.max_src_len})
+                        if (keys > 0)
+                            attn = std::max(attn, attention_partial_elems(b * mr, m.cfg.n_heads, m.cfg.d_head,
+                                                                          attention_slices(b, m.cfg.n_kv_heads, (m.cfg.n_heads / m.cfg.n_kv_heads) * mr, keys)));
         }
         SPEC_ALLOC(attn_part, attn);
     }
-    SPEC_ALLOC(target_logits, R * V);
+    SPEC_ALLOC(target_logits, RL * V);
     SPEC_ALLOC(draft_logits, std::max<size_t>(B * G, 1) * V);
     {
         // Tensor-core path (any bf16 model): inputs as two bf16 terms, split-K partial sums.
@@ -489,11 +672,15 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
             if (!m.bf16()) continue;
             any_bf16 = true;
             max_k = std::max<size_t>({max_k, static_cast<size_t>(m.cfg.d_model), static_cast<size_t>(m.q_dim()), static_cast<size_t>(m.cfg.d_ff)});
-            const int shapes[5][2] = {{m.qkv_dim(), m.cfg.d_model}, {m.cfg.d_model, m.q_dim()}, {m.ffn_in_dim(), m.cfg.d_model},
-                                      {m.cfg.d_model, m.cfg.d_ff}, {m.cfg.vocab, m.cfg.d_model}};
-            for (const auto& sh : shapes)
-                for (int rows = 1; rows <= ctx->max_rows; ++rows)
-                    partial = std::max(partial, gemm_tc_partial_elems(sh[0], sh[1], rows));
+            const int shapes[7][2] = {{m.qkv_dim(), m.cfg.d_model}, {m.cfg.d_model, m.q_dim()}, {m.ffn_in_dim(), m.cfg.d_model},
+                                      {m.cfg.d_model, m.cfg.d_ff}, {m.q_dim(), m.cfg.d_model}, {2 * m.kv_dim(), m.cfg.d_model},
+                                      {m.cfg.vocab, m.cfg.d_model}};
+            for (int s = 0; s < 7; ++s) {
+                if (!m.t5() && (s == 4 || s == 5)) continue;  // cross-attention projections
+                const int most = s == 6 ? ctx->max_logit_rows : ctx->max_rows;  // the head only sees decode rows
+                for (int rows = 1; rows <= most; ++rows)
+                    partial = std::max(partial, gemm_tc_partial_elems(shapes[s][0], shapes[s][1], rows));
+            }
         }
         if (any_bf16 && ctx->tensor_cores) {
             for (int i = 0; i < (ctx->has_draft ? 2 : 1); ++i)
@@ -512,6 +699,10 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     SPEC_ALLOC(logit_src, R);
     SPEC_ALLOC(logit_dst, R);
     SPEC_ALLOC(page_table, B * ctx->pages_per_seq);
+    if (t5) {
+        SPEC_ALLOC(src_page_table, B * ctx->src_pages_per_seq);
+        SPEC_ALLOC(src_len, B);
+    }
     SPEC_ALLOC(tokens, B * rt.max_len);
     SPEC_ALLOC(length, B);
     SPEC_ALLOC(prompt_len, B);
@@ -537,6 +728,13 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
         for (int j = 0; j < ctx->pages_per_seq; ++j) table[b * ctx->pages_per_seq + j] = static_cast<int32_t>(j * B + b);
     err = cudaMemcpy(ctx->page_table, table.data(), table.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
     if (err != cudaSuccess) return cleanup(fail(SPEC_ERR_CUDA, "page table upload: %s", cudaGetErrorString(err)));
+    if (t5) {
+        std::vector<int32_t> src_table(B * ctx->src_pages_per_seq);
+        for (size_t b = 0; b < B; ++b)
+            for (int j = 0; j < ctx->src_pages_per_seq; ++j) src_table[b * ctx->src_pages_per_seq + j] = static_cast<int32_t>(j * B + b);
+        err = cudaMemcpy(ctx->src_page_table, src_table.data(), src_table.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+        if (err != cudaSuccess) return cleanup(fail(SPEC_ERR_CUDA, "source page table upload: %s", cudaGetErrorString(err)));
+    }
     ctx->cached[0].assign(B, 0);
     ctx->cached[1].assign(B, 0);
     *out = ctx;
@@ -556,6 +754,44 @@ extern "C" void spec_free(spec_ctx* ctx) {
 
 namespace {
 
+// Encoder pass of the first n_models models over the sources of `batch` sequences.
+int encode_sources(spec_ctx* ctx, const int32_t* source, const int32_t* source_len, int stride, int batch, int n_models) {
+    if (!ctx->model[0].t5()) return fail(SPEC_ERR_BAD_CONFIG, "encode: not an encoder-decoder context");
+    if (!source || !source_len || stride < 1 || batch < 1) return fail(SPEC_ERR_BAD_ARG, "encode: bad argument");
+    if (batch > ctx->rt.max_batch) return fail(SPEC_ERR_CAPACITY, "encode: batch %d exceeds max_batch %d", batch, ctx->rt.max_batch);
+    int longest = 0;
+    for (int b = 0; b < batch; ++b) {
+        if (source_len[b] < 1 || source_len[b] > stride) return fail(SPEC_ERR_BAD_ARG, "encode: source_len[%d]=%d", b, source_len[b]);
+        if (source_len[b] > ctx->rt.max_src_len)
+            return fail(SPEC_ERR_CAPACITY, "encode: source %d has %d tokens, max_src_len is %d", b, source_len[b], ctx->rt.max_src_len);
+        for (int i = 0; i < source_len[b]; ++i) {
+            const int32_t t = source[static_cast<size_t>(b) * stride + i];
+            if (t < 0 || t >= ctx->model[0].cfg.vocab) return fail(SPEC_ERR_BAD_ARG, "encode: token %d out of range", t);
+        }
+        longest = std::max(longest, source_len[b]);
+    }
+    const size_t n = static_cast<size_t>(batch) * longest;
+    std::vector<int32_t> tok(n), pos(n), seq(n);
+    for (int b = 0; b < batch; ++b)
+        for (int j = 0; j < longest; ++j) {
+            const bool active = j < source_len[b];
+            tok[static_cast<size_t>(b) * longest + j] = active ? source[static_cast<size_t>(b) * stride + j] : 0;
+            pos[static_cast<size_t>(b) * longest + j] = active ? j : -1;
+            seq[static_cast<size_t>(b) * longest + j] = b;
+        }
+    cudaStream_t st = ctx->stream;
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_token, tok.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_pos, pos.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_seq, seq.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->src_len, source_len, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    for (int which = 0; which < n_models; ++which) SPEC_TRY(encode(ctx, ctx->model[which], batch, longest));
+    SPEC_CUDA_TRY(cudaStreamSynchronize(st));  // the host vectors go out of scope
+    if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
+    ctx->encoded = true;
+    ctx->encoded_batch = batch;
+    return SPEC_OK;
+}
+
 // Validates a generation request, uploads the prompts, runs the prompt pass of
 // both models and prepares the iteration graph.
 int begin_session(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride, int batch,
@@ -568,6 +804,16 @@ int begin_session(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_le
     if (gamma > 0 && !ctx->has_draft) return fail(SPEC_ERR_BAD_CONFIG, "generation: gamma > 0 needs a draft model");
     int limit = std::min(ctx->rt.max_len, ctx->model[0].cfg.max_positions);
     if (gamma > 0) limit = std::min(limit, ctx->model[1].cfg.max_positions);
+    // Encoder-decoder: `prompt` is the source; the decoder's own prompt is the start token.
+    const bool t5 = ctx->model[0].t5();
+    const int32_t *source = prompt, *source_len = prompt_len;
+    const int source_stride = prompt_stride;
+    std::vector<int32_t> start_tokens(batch, 0), start_len(batch, 1);
+    if (t5) {
+        prompt = start_tokens.data();
+        prompt_len = start_len.data();
+        prompt_stride = 1;
+    }
     for (int b = 0; b < batch; ++b) {
         if (prompt_len[b] < 1 || prompt_len[b] > prompt_stride) return fail(SPEC_ERR_BAD_ARG, "generation: prompt_len[%d]=%d", b, prompt_len[b]);
         if (prompt_len[b] + n_new + gamma + 1 > limit)
@@ -594,6 +840,7 @@ int begin_session(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_le
 
     // prompt pass: positions 0..prompt_len-2 (the last prompt token is fed by the first iteration)
     SPEC_CUDA_TRY(cudaEventRecord(ctx->ev[0], st));
+    if (t5) SPEC_TRY(encode_sources(ctx, source, source_len, source_stride, batch, gamma > 0 ? 2 : 1));
     std::vector<int> from(batch, 0), to(batch);
     for (int b = 0; b < batch; ++b) to[b] = prompt_len[b] - 1;
     SPEC_TRY(feed_host_tokens(ctx, 0, prompt, prompt_stride, from, to, batch));
@@ -699,6 +946,15 @@ extern "C" int spec_read_tokens(spec_ctx* ctx, int32_t* out_tokens) {
     return SPEC_OK;
 }
 
+extern "C" int spec_encode(spec_ctx* ctx, const int32_t* source, const int32_t* source_len, int source_stride, int batch) {
+    if (!ctx) return fail(SPEC_ERR_BAD_ARG, "spec_encode: null context");
+    ctx->session_batch = 0;
+    SPEC_TRY(encode_sources(ctx, source, source_len, source_stride, batch, ctx->has_draft ? 2 : 1));
+    std::fill(ctx->cached[0].begin(), ctx->cached[0].end(), 0);
+    std::fill(ctx->cached[1].begin(), ctx->cached[1].end(), 0);
+    return SPEC_OK;
+}
+
 extern "C" int spec_reset(spec_ctx* ctx) {
     if (!ctx) return fail(SPEC_ERR_BAD_ARG, "spec_reset: null context");
     std::fill(ctx->cached[0].begin(), ctx->cached[0].end(), 0);
@@ -723,8 +979,10 @@ extern "C" int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* toke
     if (!ctx || !tokens || !logits || which < 0 || which > 1 || batch < 1 || rows < 1)
         return fail(SPEC_ERR_BAD_ARG, "spec_forward_logits: bad argument");
     if (which == 1 && !ctx->has_draft) return fail(SPEC_ERR_BAD_CONFIG, "spec_forward_logits: no draft model");
-    if (batch > ctx->rt.max_batch || batch * rows > ctx->max_rows)
-        return fail(SPEC_ERR_CAPACITY, "spec_forward_logits: %d x %d rows exceed the workspace (%d rows)", batch, rows, ctx->max_rows);
+    if (batch > ctx->rt.max_batch || batch * rows > ctx->max_logit_rows)
+        return fail(SPEC_ERR_CAPACITY, "spec_forward_logits: %d x %d rows exceed the workspace (%d rows)", batch, rows, ctx->max_logit_rows);
+    if (ctx->model[which].t5() && (!ctx->encoded || batch > ctx->encoded_batch))
+        return fail(SPEC_ERR_BAD_ARG, "spec_forward_logits: call spec_encode for these sequences first");
     const Model& m = ctx->model[which];
     const int n = batch * rows;
     ctx->session_batch = 0;  // the diagnostics reuse the caches

@@ -204,19 +204,17 @@ int launch_norm(float* h, const float* partial, int splits, int rows_total, cons
                       src_rows, d, eps, out, out_hi, out_lo);
 }
 
-int launch_qkv(const Model& m, int layer, const RowMeta& rows, int n_rows, float* qkv, const float* partial,
-               int splits, const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream) {
-    char* kv_layer = static_cast<char*>(m.kv) + static_cast<size_t>(layer) * m.layer_stride;
-    const float2* table = m.cfg.arch == SPEC_ARCH_LLAMA ? m.rope_table : nullptr;
-    const dim3 grid(m.cfg.n_heads + 2 * m.cfg.n_kv_heads, n_rows);
-    const dim3 block(m.cfg.d_head / 2);
-    if (m.kv_elem_bytes == 2)
+int launch_qkv(int n_heads, int n_kv_heads, int d_head, const float2* rope, const KvPool& pool, const RowMeta& rows,
+               int n_rows, float* qkv, const float* partial, int splits, cudaStream_t stream) {
+    const dim3 grid(n_heads + 2 * n_kv_heads, n_rows);
+    const dim3 block(d_head / 2);
+    if (pool.elem_bytes == 2)
         return launch_pdl(qkv_kernel<__nv_bfloat16>, grid, block, 0, stream, qkv, partial, splits, n_rows, rows.pos,
-                          rows.seq, m.cfg.n_heads, m.cfg.n_kv_heads, m.cfg.d_head, table,
-                          reinterpret_cast<__nv_bfloat16*>(kv_layer), page_table, pages_per_seq, page_size);
+                          rows.seq, n_heads, n_kv_heads, d_head, rope, static_cast<__nv_bfloat16*>(pool.kv),
+                          pool.page_table, pool.pages_per_seq, pool.page_size);
     return launch_pdl(qkv_kernel<float>, grid, block, 0, stream, qkv, partial, splits, n_rows, rows.pos, rows.seq,
-                      m.cfg.n_heads, m.cfg.n_kv_heads, m.cfg.d_head, table, reinterpret_cast<float*>(kv_layer),
-                      page_table, pages_per_seq, page_size);
+                      n_heads, n_kv_heads, d_head, rope, static_cast<float*>(pool.kv), pool.page_table,
+                      pool.pages_per_seq, pool.page_size);
 }
 
 int launch_ffn_act(const float* u, const float* partial, int splits, int n_rows, int d_ff, int ffn, float* f,

@@ -29,6 +29,17 @@ struct Model {
     int kv_elem_bytes = 4;
     const float2* rope_table = nullptr;  // Llama: (cos, sin) [positions][d_head / 2], owned
 
+    // Encoder-decoder (T5) only.  The bias tables are the bucket tables expanded by
+    // relative position: [n_heads][span], entry (key pos - query pos) + zero.
+    std::vector<spec_layer_weights> enc_layers, enc_packed;
+    const float* enc_ln_f = nullptr;
+    const float* enc_bias = nullptr;  // span 2 * max_src_len - 1, zero max_src_len - 1, owned
+    const float* dec_bias = nullptr;  // span max_len, zero max_len - 1 (only keys at or before the query), owned
+    void* enc_kv = nullptr;           // K,V of the encoder block being computed (one layer's pool), owned
+    void* cross_kv = nullptr;         // cross-attention K,V of decoder layer l: cross_kv + l * cross_stride, owned
+    size_t cross_stride = 0;
+    bool t5() const { return cfg.arch == SPEC_ARCH_T5; }
+
     int q_dim() const { return cfg.n_heads * cfg.d_head; }
     int kv_dim() const { return cfg.n_kv_heads * cfg.d_head; }
     int qkv_dim() const { return q_dim() + 2 * kv_dim(); }
@@ -78,19 +89,47 @@ int launch_gemm_tc(const __nv_bfloat16* hi, const __nv_bfloat16* lo, int hi_rows
                    float* y, cudaStream_t stream);
 int gemm_tc_take_error();
 
-// Finishes the qkv GEMM (optional partial sums), rotary positions on q and k
-// (Llama), K,V rows of every active row into the paged cache; q stays in `qkv`.
-int launch_qkv(const Model& m, int layer, const RowMeta& rows, int n_rows, float* qkv, const float* partial,
-               int splits, const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream);
+// Where the K,V rows of a pass go / come from: one layer's pool
+// [n_pages][2 (K, V)][n_kv_heads][page_size][d_head] and the table that maps
+// (sequence slot, position / page_size) to a pool page.
+struct KvPool {
+    void* kv;
+    int elem_bytes;  // 4 (fp32) or 2 (bf16)
+    const int32_t* page_table;
+    int pages_per_seq;
+    int page_size;
+};
+
+// Finishes a projection GEMM whose output row is [n_heads q heads | n_kv_heads k
+// heads | n_kv_heads v heads] (optional split-K partial sums): rotary positions
+// on q and k when `rope` is given, q heads left in `qkv`, K,V heads of every
+// active row appended to the pool.  n_kv_heads = 0: queries only; n_heads = 0:
+// K,V only.
+int launch_qkv(int n_heads, int n_kv_heads, int d_head, const float2* rope, const KvPool& pool, const RowMeta& rows,
+               int n_rows, float* qkv, const float* partial, int splits, cudaStream_t stream);
 void fill_rope_table(std::vector<float2>& table, int positions, int d_head, double base);
 
-// att[r, h] = softmax(q_r,h . K / sqrt(d_head)) V over cached positions <= pos[r];
-// rows of sequence b are rows b*m_rows .. of the pass.  Output as fp32 and/or two bf16 terms.
+// One attention call: head h of query row r is at q + r * q_stride + h * d_head.
+// kv_len == nullptr: causal over the pool (row at position p sees keys 0..p);
+// otherwise every active row of sequence slot s sees keys 0..kv_len[s]-1.
+// bias (optional): score of (row at position p, key at position k, head h) gets
+// bias[h * bias_span + (k - p) + bias_zero] added after scaling.
+struct AttnSource {
+    const float* q;
+    int q_stride;
+    KvPool pool;
+    const int32_t* kv_len;
+    const float* bias;
+    int bias_span;
+    int bias_zero;
+};
+
+// att[r, h] = softmax(scores) V for the rows of a pass; rows of sequence b are
+// rows b*m_rows .. of the pass.  Output as fp32 and/or two bf16 terms.
 int attention_slices(int batch, int n_kv_heads, int queries, int max_len);
 size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices);
-int launch_attention(const Model& m, int layer, const RowMeta& rows, int batch, int m_rows, int slices,
-                     const float* qkv, float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo,
-                     const int32_t* page_table, int pages_per_seq, int page_size, cudaStream_t stream);
+int launch_attention(const Model& m, const AttnSource& src, const RowMeta& rows, int batch, int m_rows, int slices,
+                     float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo, cudaStream_t stream);
 
 // f = gelu(u)  |  gelu(u[:, :F]) * u[:, F:]  |  silu(u[:, :F]) * u[:, F:], u given in full or as partial sums.
 int launch_ffn_act(const float* u, const float* partial, int splits, int n_rows, int d_ff, int ffn, float* f,
