@@ -12,6 +12,9 @@ Workloads (--workload)
             A step is one iteration of Algorithm 1 for the whole batch: gamma
             draft passes, one target pass over gamma+1 rows, speculative sampling,
             commit and KV roll-back.
+  t5xxl     T5-XXL-shaped bf16 encoder-decoder target with a T5-small-shaped draft,
+            512-token sources (encoders run once, in the prompt pass), 128 decoded
+            tokens, gamma --gamma (5).
   gpt97m    the paper-shaped GPT-like 97M target with its 6M draft, 8k vocabulary.
   sampler   the standalone speculative-sampling kernel: batch 64 x
             (gamma+1 = 8) x vocab 32000, T = 1, draft logits = target + N(0, s^2)
@@ -212,10 +215,16 @@ def gpu_weights(cfg, seed, device):
         if kind == "gain":
             out[name] = torch.ones(shape, device=device)
             continue
-        std = cfg["head_std"] if kind == "head" else workloads.INIT_STD
+        std = cfg["head_std"] if kind == "head" else cfg["bias_std"] if kind == "bias" else workloads.INIT_STD
         t = torch.randn(shape, device=device, generator=g, dtype=torch.float32) * std
-        out[name] = t.to(torch.bfloat16) if cfg["dtype"] == "bf16" else t
+        out[name] = t.to(torch.bfloat16) if cfg["dtype"] == "bf16" and kind != "bias" else t
     return out
+
+
+def decode_stream(name):
+    """Whether a tensor is streamed by a decoder pass (encoder-decoder models: not the
+    encoder stack, nor the projections of the encoder output, which run once per source)."""
+    return not (name.startswith("enc.") or name.endswith(("wkv_x", "rel_bias")))
 
 
 def weight_stream_bytes(cfg):
@@ -224,7 +233,7 @@ def weight_stream_bytes(cfg):
     elem = 2 if cfg["dtype"] == "bf16" else 4
     total = 0
     for name, shape, kind in workloads.tensor_shapes(cfg):
-        if kind == "gain" or name in ("pos_emb",) or (name == "tok_emb" and not cfg["tied"]):
+        if kind == "gain" or name in ("pos_emb",) or (name == "tok_emb" and not cfg["tied"]) or not decode_stream(name):
             continue
         total += int(np.prod(shape)) * elem
     return total
@@ -234,8 +243,10 @@ class GenerationWorkload:
     dtype = "bf16"
 
     def __init__(self, name, target, draft, batch, prompt_len, n_new, gamma, temperature=1.0, layers=None):
+        from paper_2211_17192_b200 import workloads
         self.name, self.target_name, self.draft_name = name, target, draft
         self.layers = layers
+        self.tcfg, self.dcfg = workloads.model_config(target), workloads.model_config(draft)  # (prepare applies --layers)
         self.batch, self.prompt_len, self.n_new, self.gamma, self.temperature = batch, prompt_len, n_new, gamma, temperature
 
     def description(self):
@@ -314,7 +325,7 @@ class GenerationWorkload:
         target once through spec_linear at `rows` rows, captured in a CUDA graph and
         timed with events on its stream."""
         torch, binding = self.torch, self.binding
-        mats = [(n, t) for n, t in self.tw.items() if t.dim() == 2 and n not in ("tok_emb", "pos_emb")]
+        mats = [(n, t) for n, t in self.tw.items() if t.dim() == 2 and n not in ("tok_emb", "pos_emb") and decode_stream(n)]
         if self.tcfg["tied"]:
             mats.append(("head", self.tw["tok_emb"]))
         kmax = max(t.shape[1] for _, t in mats)
@@ -353,8 +364,10 @@ class GenerationWorkload:
         small_t = workloads.scaled_config(self.tcfg, n_layers=min(2, self.tcfg["n_layers"]))
         small_d = workloads.scaled_config(self.dcfg, n_layers=min(2, self.dcfg["n_layers"]))
         dtype = np.float32 if self.tcfg["d_model"] >= 2048 else np.float64
-        target = Decoder(small_t, workloads.make_weights(small_t, 1), dtype=dtype)
-        draft = Decoder(small_d, workloads.make_weights(small_d, 2), dtype=dtype)
+        if not hasattr(self, "_cpu_models"):  # built once, outside every timed sample
+            self._cpu_models = (Decoder(small_t, workloads.make_weights(small_t, 1), dtype=dtype),
+                                Decoder(small_d, workloads.make_weights(small_d, 2), dtype=dtype))
+        target, draft = self._cpu_models
         prompt = workloads.make_prompt(3, 32, self.tcfg["vocab"])
         t0 = time.perf_counter()
         tokens = iters = 0
@@ -373,10 +386,106 @@ class GenerationWorkload:
         return value, sample
 
 
+class EncDecWorkload(GenerationWorkload):
+    """Encoder-decoder pair: `prompt_len` is the source length; the encoders run once
+    per source (inside the prompt pass, untimed in `value`, timed in `e2e`) and the
+    decoders start from the start token."""
+
+    def description(self):
+        d = super().description()
+        d["source_len"] = d.pop("prompt_len")
+        d["l2"] = "one pass streams the target decoder's weights (>> 126 MB L2) from HBM"
+        return d
+
+    def prepare(self, rank, device, iterations):
+        import torch
+        from paper_2211_17192_b200 import binding, workloads
+        self.torch, self.binding, self.device = torch, binding, device
+        self.tcfg = workloads.model_config(self.target_name)
+        if self.layers:
+            self.tcfg = workloads.scaled_config(self.tcfg, n_layers=self.layers, n_enc_layers=self.layers)
+        self.dcfg = workloads.model_config(self.draft_name)
+        self.dtype = "bf16"
+        self.tw = gpu_weights(self.tcfg, 100 + rank, device)
+        self.dw = gpu_weights(self.dcfg, 200 + rank, device)
+        grow = max(self.n_new, iterations * (self.gamma + 1) + 64)
+        self.max_len = 1 + grow + self.gamma + 2
+        self.engine = binding.Engine(self.tcfg, self.tw, self.dcfg, self.dw, max_batch=self.batch, max_len=self.max_len,
+                                     page_size=64, max_gamma=max(self.gamma, 1), max_src_len=self.prompt_len)
+        self.prompts = [workloads.make_prompt(1000 * rank + b, self.prompt_len, self.tcfg["vocab"]) for b in range(self.batch)]
+        self.budget_tokens = grow
+
+    def launches_per_iteration(self):
+        fwd = lambda cfg: 1 + 16 * cfg["n_layers"] + 3
+        return 1 + self.gamma * (1 + fwd(self.dcfg) + 1) + 1 + fwd(self.tcfg) + 2 + 1
+
+    def kv_bytes(self, context):
+        c = self.tcfg
+        per_position = 2 * c["n_layers"] * c["n_kv_heads"] * c["d_head"] * 4
+        return self.batch * (context + self.prompt_len) * per_position  # self-attention rows + cross-attention rows
+
+    def pass_times(self, repeats=20):
+        """Single passes through the teacher-forced entry point at a decoder context
+        of n_new / 2 tokens: the target on 1 and gamma+1 rows, the draft on 1 row."""
+        eng = self.engine
+        context = max(1, self.n_new // 2)
+        self.pass_context = context
+        def timed(which, rows):
+            best = []
+            for _ in range(repeats):
+                eng.truncate(which, [context] * self.batch)
+                t0 = time.perf_counter()
+                eng.forward_logits(which, np.zeros((self.batch, rows), dtype=np.int32))
+                best.append(time.perf_counter() - t0)
+            return statistics.median(best) * 1e3
+        eng.encode(self.prompts)
+        for which in (0, 1):
+            for c0 in range(0, context, 32):
+                eng.forward_logits(which, np.zeros((self.batch, min(32, context - c0)), dtype=np.int32))
+        return {"target_1row_ms": timed(0, 1), "target_rows_ms": timed(0, self.gamma + 1), "draft_1row_ms": timed(1, 1)}
+
+    def cpu_sample(self, budget_s):
+        """The oracle on a bounded sample: both models at full width with one encoder and
+        one decoder block each, a 32-token source; extrapolated to the full decoder depth
+        by streamed weight bytes."""
+        from oracle import generate as oracle_generate
+        from oracle.encdec import START_TOKEN, EncoderDecoder
+        from paper_2211_17192_b200 import workloads
+        small_t = workloads.scaled_config(self.tcfg, n_layers=1, n_enc_layers=1)
+        small_d = workloads.scaled_config(self.dcfg, n_layers=1, n_enc_layers=1)
+        if not hasattr(self, "_cpu_models"):  # built and encoded once, outside every timed sample
+            target = EncoderDecoder(small_t, workloads.make_weights(small_t, 1), dtype=np.float32)
+            draft = EncoderDecoder(small_d, workloads.make_weights(small_d, 2), dtype=np.float32)
+            source = workloads.make_prompt(3, 32, self.tcfg["vocab"])
+            target.encode(source)
+            draft.encode(source)
+            self._cpu_models = (target, draft)
+        target, draft = self._cpu_models
+        t0 = time.perf_counter()
+        tokens = iters = 0
+        n_new = self.gamma + 1
+        while time.perf_counter() - t0 < budget_s or iters == 0:
+            res = oracle_generate.speculative_generate(target, draft, [START_TOKEN], n_new, self.gamma, self.temperature, seed=iters)
+            tokens += len(res.tokens)
+            iters += len(res.iterations)
+        dt = time.perf_counter() - t0
+        full = weight_stream_bytes(self.tcfg) + self.gamma * weight_stream_bytes(self.dcfg)
+        small = weight_stream_bytes(small_t) + self.gamma * weight_stream_bytes(small_d)
+        value = tokens / dt * small / full
+        sample = (f"{iters} iterations of Algorithm 1 (decode only, encoders run before the clock), batch 1, 32-token "
+                  f"source, both models at full width and 1 decoder layer in float32, {dt:.1f} s; scaled by "
+                  f"streamed weight bytes ({small / full:.3f}) to the full depth")
+        return value, sample
+
+
 def make_workload(args):
     if args.workload == "sampler":
         return SamplerWorkload()
     batch = args.batch or 1
+    if args.workload == "t5xxl":
+        gamma = args.gamma or 5
+        return EncDecWorkload(f"t5xxl_small_b{batch}_g{gamma}", "t5xxl_target", "t5small_draft", batch,
+                              args.prompt_len or 512, 128, gamma, args.temperature, args.layers)
     if args.workload == "gpt97m":
         return GenerationWorkload("gpt97m_6m_b1", "gpt97m_target", "gpt6m_draft", batch, args.prompt_len or 128, 512,
                                   args.gamma or 5, args.temperature, args.layers)
@@ -385,7 +494,7 @@ def make_workload(args):
                               args.prompt_len or 1024, 256, gamma, args.temperature, args.layers)
 
 
-WORKLOAD_NAMES = ["llama7b", "gpt97m", "sampler"]
+WORKLOAD_NAMES = ["llama7b", "t5xxl", "gpt97m", "sampler"]
 
 
 # --------------------------------------------------------------------------- #
@@ -521,7 +630,10 @@ def run_generation(args, wl, torch, device, local, barrier):
         alpha = stats["tests_passed"] / max(1, stats["tests_evaluated"])
         tok_per_iter = stats["tokens"] / max(1, stats["iterations"])
         c = times["draft_1row_ms"] / times["target_1row_ms"]
-        kv_bytes = wl.batch * wl.prompt_len * 2 * wl.tcfg["n_layers"] * wl.tcfg["n_kv_heads"] * wl.tcfg["d_head"] * 4
+        if hasattr(wl, "kv_bytes"):
+            kv_bytes = wl.kv_bytes(wl.pass_context)
+        else:
+            kv_bytes = wl.batch * wl.prompt_len * 2 * wl.tcfg["n_layers"] * wl.tcfg["n_kv_heads"] * wl.tcfg["d_head"] * 4
         pass_bytes = weight_stream_bytes(wl.tcfg) + kv_bytes
         extras = {
             "speedup_vs_target_only": (tokens / elapsed_ms) / (base_tokens / base_ms),
@@ -537,7 +649,7 @@ def run_generation(args, wl, torch, device, local, barrier):
             "verify_pass": {"bytes": pass_bytes, "ms": times["target_rows_ms"],
                             "gbs": pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9,
                             "frac": pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9 / peak,
-                            "note": "weights + fp32 KV of the prompt, one pass over gamma+1 rows, host-timed call"},
+                            "note": "weights + fp32 K,V rows read (context; for encoder-decoders also the source), one pass over gamma+1 rows, host-timed call"},
             "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbs": achieved / 8000.0,
                          "traffic": None, "algorithmic_bytes_per_launch": nbytes / n_mats,

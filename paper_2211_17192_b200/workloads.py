@@ -49,8 +49,8 @@ def model_config(name):
         "t5xxl_target": dict(arch="t5", ffn="gated_gelu", n_layers=24, n_enc_layers=24, d_model=4096, n_heads=64,
                              n_kv_heads=64, d_head=64, d_ff=10240, vocab=32128, max_positions=1024, dtype="bf16",
                              head_std=INIT_STD),
-        "t5small_draft": dict(arch="t5", ffn="gated_gelu", n_layers=8, n_enc_layers=8, d_model=512, n_heads=6,
-                              n_kv_heads=6, d_head=64, d_ff=1024, vocab=32128, max_positions=1024, dtype="bf16",
+        "t5small_draft": dict(arch="t5", ffn="gated_gelu", n_layers=6, n_enc_layers=6, d_model=512, n_heads=8,
+                              n_kv_heads=8, d_head=64, d_ff=2048, vocab=32128, max_positions=1024, dtype="bf16",
                               head_std=INIT_STD),
         # small encoder-decoder pairs for tests
         "t5_test_target": dict(arch="t5", ffn="gated_gelu", n_layers=2, n_enc_layers=2, d_model=256, n_heads=4,
