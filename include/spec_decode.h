@@ -326,6 +326,16 @@ int spec_generate(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_le
 int spec_begin(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride,
                int batch, int n_new, int gamma, float temperature, uint64_t seed);
 
+/* Timing instrument (no counterpart in Algorithm 1): from the next spec_begin /
+ * spec_generate on, the accept decision of every drafted token is replaced by
+ * "r_i < alpha" with the same uniforms r_i, i.e. an i.i.d. Bernoulli(alpha)
+ * acceptance as the analysis of Section 3.1-3.2 assumes, whatever p and q say;
+ * the final token is still drawn by the sampler.  The emitted tokens are then
+ * NOT distributed as the target's: use it only to time iterations at a chosen
+ * acceptance rate (random-init model pairs sit at one uncontrolled alpha).
+ * alpha < 0 restores Algorithm 1.  Errors: SPEC_ERR_BAD_ARG (alpha > 1 or NaN). */
+int spec_set_imposed_acceptance(spec_ctx* ctx, float alpha);
+
 /* Encoder-decoder models only: runs the encoder of every model of the context
  * over the sources (HOST int32 [batch, source_stride], source_len[b] >= 1
  * entries used) and stores the cross-attention K,V; forgets every cached

@@ -288,6 +288,8 @@ def _declare_engine(h):
     h.spec_truncate.argtypes = [vp, c.c_int, vp, c.c_int]
     h.spec_forward_logits.restype = c.c_int
     h.spec_forward_logits.argtypes = [vp, c.c_int, vp, c.c_int, c.c_int, vp]
+    h.spec_set_imposed_acceptance.restype = c.c_int
+    h.spec_set_imposed_acceptance.argtypes = [vp, c.c_float]
     h.spec_encode.restype = c.c_int
     h.spec_encode.argtypes = [vp, vp, vp, c.c_int, c.c_int]
     _engine_declared = True
@@ -423,6 +425,12 @@ class Engine:
                                    float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF, out.ctypes.data,
                                    ctypes.byref(st)))
         return out, {name: getattr(st, name) for name, _ in _Stats._fields_}
+
+    def set_imposed_acceptance(self, alpha):
+        """Timing instrument: accept every drafted token with probability `alpha`
+        (i.i.d., from the same uniforms) instead of by Algorithm 1's test; None or a
+        negative value restores the algorithm."""
+        _check(lib().spec_set_imposed_acceptance(self._ctx, -1.0 if alpha is None else float(alpha)))
 
     def encode(self, sources):
         """Encoder-decoder models: run the encoders over `sources` (list of 1-D int

@@ -43,7 +43,8 @@ struct spec_ctx {
     float *draft_u = nullptr, *accept_u = nullptr, *final_u = nullptr;
     unsigned long long* counters = nullptr;  // iterations, tokens, tests evaluated, tests passed
     void* sampler_ws = nullptr;
-    struct Params { unsigned long long seed; int n_new; int pad; }* params = nullptr;
+    struct Params { unsigned long long seed; int n_new; float imposed_alpha; }* params = nullptr;
+    float imposed_alpha = -1.0f;  // >= 0: timing instrument, see spec_set_imposed_acceptance
 
     // cached iteration graph
     cudaGraphExec_t graph = nullptr;
@@ -339,15 +340,20 @@ __global__ void prep_verify_kernel(const int32_t* __restrict__ tokens, const int
 // already has its n_new tokens is frozen.
 __global__ void commit_kernel(const spec_ctx::Params* __restrict__ params, const int32_t* __restrict__ draft_tokens,
                               const int32_t* __restrict__ n_accepted, const int32_t* __restrict__ next_token,
-                              const int32_t* __restrict__ prompt_len, int batch, int gamma, int max_len,
-                              int32_t* tokens, int32_t* length, unsigned long long* counters) {
+                              const float* __restrict__ accept_u, const int32_t* __restrict__ prompt_len, int batch,
+                              int gamma, int max_len, int32_t* tokens, int32_t* length, unsigned long long* counters) {
     pdl_trigger();
     pdl_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch) return;
     const int L = length[b];
     if (L - prompt_len[b] >= params->n_new) return;
-    const int n = n_accepted[b];
+    int n = n_accepted[b];
+    const float imposed = params->imposed_alpha;
+    if (imposed >= 0.0f) {  // timing instrument: accept x_i iff r_i < alpha, whatever p and q say
+        n = 0;
+        while (n < gamma && accept_u[b * (gamma + 1) + n] < imposed) ++n;
+    }
     int32_t* seq_tokens = tokens + static_cast<size_t>(b) * max_len;
     for (int i = 0; i < n; ++i) seq_tokens[L + i] = draft_tokens[b * gamma + i];
     seq_tokens[L + n] = next_token[b];
@@ -392,8 +398,8 @@ int enqueue_iteration(spec_ctx* ctx, int batch, int gamma, float temperature) {
     SPEC_TRY(launch_verify_sample(ctx->target_logits, ctx->draft_logits, ctx->draft_tokens, ctx->accept_u, ctx->final_u,
                                   batch, gamma, vocab, temperature, ctx->n_accepted, ctx->next_token, ctx->sampler_ws, st));
     return launch_pdl(commit_kernel, dim3(blocks_b), dim3(threads), 0, st, ctx->params, ctx->draft_tokens,
-                      ctx->n_accepted, ctx->next_token, ctx->prompt_len, batch, gamma, ctx->rt.max_len, ctx->tokens,
-                      ctx->length, ctx->counters);
+                      ctx->n_accepted, ctx->next_token, ctx->accept_u, ctx->prompt_len, batch, gamma, ctx->rt.max_len,
+                      ctx->tokens, ctx->length, ctx->counters);
 }
 
 int build_graph(spec_ctx* ctx, int batch, int gamma, float temperature) {
@@ -835,7 +841,7 @@ int begin_session(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_le
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->length, prompt_len, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->prompt_len, prompt_len, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SPEC_CUDA_TRY(cudaMemsetAsync(ctx->counters, 0, 4 * sizeof(unsigned long long), st));
-    const spec_ctx::Params params{seed, n_new, 0};
+    const spec_ctx::Params params{seed, n_new, ctx->imposed_alpha};
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->params, &params, sizeof(params), cudaMemcpyHostToDevice, st));
 
     // prompt pass: positions 0..prompt_len-2 (the last prompt token is fed by the first iteration)
@@ -943,6 +949,12 @@ extern "C" int spec_read_tokens(spec_ctx* ctx, int32_t* out_tokens) {
     SPEC_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
     for (int b = 0; b < batch; ++b)
         std::memcpy(out_tokens + static_cast<size_t>(b) * n_new, &host_tokens[static_cast<size_t>(b) * max_len + ctx->session_prompt_len[b]], n_new * sizeof(int32_t));
+    return SPEC_OK;
+}
+
+extern "C" int spec_set_imposed_acceptance(spec_ctx* ctx, float alpha) {
+    if (!ctx || !(alpha <= 1.0f)) return fail(SPEC_ERR_BAD_ARG, "spec_set_imposed_acceptance: alpha must be <= 1 (negative: off)");
+    ctx->imposed_alpha = alpha < 0.0f ? -1.0f : alpha;
     return SPEC_OK;
 }
 

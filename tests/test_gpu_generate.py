@@ -130,3 +130,33 @@ def test_phased_generation_equals_the_single_call(tiny):
     eng.reset()
     with pytest.raises(binding.SpecError):
         eng.step(1)
+
+
+def test_imposed_acceptance_is_iid_with_the_chosen_rate(tiny):
+    """The timing instrument: n follows the capped geometric law of Section 3.1
+    (Eq. 1) for the imposed alpha, independent of the models."""
+    from oracle import analysis
+    eng, _, _, cfg = tiny
+    prompt = workloads.make_prompt(10, 6, cfg["vocab"])
+    gamma = 4
+    try:
+        for alpha in (0.0, 0.7, 1.0):
+            eng.set_imposed_acceptance(alpha)
+            total = {"iterations": 0, "tokens": 0, "tests_evaluated": 0, "tests_passed": 0}
+            for seed in range(8):
+                _, stats = eng.generate([prompt], 100, gamma, 1.0, seed)
+                for k in total:
+                    total[k] += stats[k]
+            per_iteration = total["tokens"] / total["iterations"]
+            if alpha in (0.0, 1.0):
+                assert per_iteration == (1 if alpha == 0.0 else gamma + 1)
+                continue
+            rate = total["tests_passed"] / total["tests_evaluated"]
+            sigma = (alpha * (1 - alpha) / total["tests_evaluated"]) ** 0.5
+            assert abs(rate - alpha) < 4 * sigma
+            assert abs(per_iteration - analysis.expected_tokens(alpha, gamma)) < 0.25
+    finally:
+        eng.set_imposed_acceptance(None)
+    a, _ = eng.generate([prompt], 20, gamma, 1.0, 3)
+    b, _ = eng.generate([prompt], 20, gamma, 1.0, 3)
+    assert np.array_equal(a, b)
