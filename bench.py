@@ -301,18 +301,12 @@ class GenerationWorkload:
         return self.batch * self.prompt_len * 4 + self.batch * 4, self.batch * self.n_new * 4
 
     def pass_times(self, repeats=20):
-        """Wall time of single passes through the teacher-forced entry point: the target
-        on 1 and on gamma+1 rows, the draft on 1 row, at the prompt's context length."""
+        """Device time of single passes (graph-replayed, events on the library's stream):
+        the target on 1 and on gamma+1 rows, the draft on 1 row, at the prompt's context length."""
         eng, torch = self.engine, self.torch
         tok = np.stack([p[: self.prompt_len - 1] for p in self.prompts])
         def timed(which, rows):
-            best = []
-            for _ in range(repeats):
-                eng.truncate(which, [self.prompt_len - 1] * self.batch)
-                t0 = time.perf_counter()
-                eng.forward_logits(which, np.zeros((self.batch, rows), dtype=np.int32))
-                best.append(time.perf_counter() - t0)
-            return statistics.median(best) * 1e3
+            return eng.time_forward(which, self.batch, rows, repeats)
         eng.reset()
         chunk = 64
         for which in (0, 1):
@@ -425,19 +419,13 @@ class EncDecWorkload(GenerationWorkload):
         return self.batch * (context + self.prompt_len) * per_position  # self-attention rows + cross-attention rows
 
     def pass_times(self, repeats=20):
-        """Single passes through the teacher-forced entry point at a decoder context
-        of n_new / 2 tokens: the target on 1 and gamma+1 rows, the draft on 1 row."""
+        """Device time of single passes (graph-replayed) at a decoder context of
+        n_new / 2 tokens: the target on 1 and gamma+1 rows, the draft on 1 row."""
         eng = self.engine
         context = max(1, self.n_new // 2)
         self.pass_context = context
         def timed(which, rows):
-            best = []
-            for _ in range(repeats):
-                eng.truncate(which, [context] * self.batch)
-                t0 = time.perf_counter()
-                eng.forward_logits(which, np.zeros((self.batch, rows), dtype=np.int32))
-                best.append(time.perf_counter() - t0)
-            return statistics.median(best) * 1e3
+            return eng.time_forward(which, self.batch, rows, repeats)
         eng.encode(self.prompts)
         for which in (0, 1):
             for c0 in range(0, context, 32):
@@ -666,7 +654,7 @@ def run_generation(args, wl, torch, device, local, barrier):
             "verify_pass": {"bytes": pass_bytes, "ms": times["target_rows_ms"],
                             "gbs": pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9,
                             "frac": pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9 / peak,
-                            "note": "weights + fp32 K,V rows read (context; for encoder-decoders also the source), one pass over gamma+1 rows, host-timed call"},
+                            "note": "weights + fp32 K,V rows read (context; for encoder-decoders also the source), one pass over gamma+1 rows, graph replays timed with events"},
             "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbs": achieved / 8000.0,
                          "traffic": None, "algorithmic_bytes_per_launch": nbytes / n_mats,

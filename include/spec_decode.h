@@ -366,6 +366,17 @@ int spec_reset(spec_ctx* ctx);
 int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* tokens, int batch, int rows, float* logits);
 int spec_truncate(spec_ctx* ctx, int which, const int32_t* lengths, int batch);
 
+/* Device time of one forward pass of model `which` over `rows` rows per
+ * sequence for `batch` sequences, at the cached lengths the diagnostics above
+ * have built up (the quantities c and the cost of gamma+1 parallel rows in the
+ * walltime analysis of Section 3.3 are ratios of such times).  The pass (token
+ * 0 in every row, logits of every row computed and discarded) is captured in a
+ * CUDA graph once and replayed `repeats` times between two events on the
+ * context's stream; *ms_per_pass gets the mean.  The cached lengths do not
+ * change (the rows are written beyond them).  Synchronises.
+ * Errors as spec_forward_logits. */
+int spec_time_forward(spec_ctx* ctx, int which, int batch, int rows, int repeats, float* ms_per_pass);
+
 /* ------------------------------------------------------------------------- *
  * One linear layer y = x . W^T, the building block of the verification pass
  * (the paper's premise, Section 1 and Section 3.4: the pass is bound by

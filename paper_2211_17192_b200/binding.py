@@ -290,6 +290,8 @@ def _declare_engine(h):
     h.spec_forward_logits.argtypes = [vp, c.c_int, vp, c.c_int, c.c_int, vp]
     h.spec_set_imposed_acceptance.restype = c.c_int
     h.spec_set_imposed_acceptance.argtypes = [vp, c.c_float]
+    h.spec_time_forward.restype = c.c_int
+    h.spec_time_forward.argtypes = [vp, c.c_int, c.c_int, c.c_int, c.c_int, c.POINTER(c.c_float)]
     h.spec_encode.restype = c.c_int
     h.spec_encode.argtypes = [vp, vp, vp, c.c_int, c.c_int]
     _engine_declared = True
@@ -444,6 +446,13 @@ class Engine:
     def truncate(self, which, lengths):
         a = self._np.ascontiguousarray(lengths, dtype=self._np.int32)
         _check(lib().spec_truncate(self._ctx, which, a.ctypes.data, a.shape[0]))
+
+    def time_forward(self, which, batch, rows, repeats=20):
+        """Device time (ms) of one pass of model `which` over `rows` rows per sequence at
+        the current cached lengths, graph-replayed `repeats` times; the caches keep their lengths."""
+        ms = ctypes.c_float()
+        _check(lib().spec_time_forward(self._ctx, which, batch, rows, repeats, ctypes.byref(ms)))
+        return ms.value
 
     def forward_logits(self, which, tokens):
         """Teacher-forced pass: tokens [B, rows] are appended at the cached

@@ -987,6 +987,58 @@ extern "C" int spec_truncate(spec_ctx* ctx, int which, const int32_t* lengths, i
     return SPEC_OK;
 }
 
+extern "C" int spec_time_forward(spec_ctx* ctx, int which, int batch, int rows, int repeats, float* ms_per_pass) {
+    if (!ctx || !ms_per_pass || which < 0 || which > 1 || batch < 1 || rows < 1 || repeats < 1)
+        return fail(SPEC_ERR_BAD_ARG, "spec_time_forward: bad argument");
+    if (which == 1 && !ctx->has_draft) return fail(SPEC_ERR_BAD_CONFIG, "spec_time_forward: no draft model");
+    if (batch > ctx->rt.max_batch || batch * rows > ctx->max_logit_rows)
+        return fail(SPEC_ERR_CAPACITY, "spec_time_forward: %d x %d rows exceed the workspace (%d rows)", batch, rows, ctx->max_logit_rows);
+    const Model& m = ctx->model[which];
+    if (m.t5() && (!ctx->encoded || batch > ctx->encoded_batch))
+        return fail(SPEC_ERR_BAD_ARG, "spec_time_forward: call spec_encode for these sequences first");
+    const int n = batch * rows;
+    ctx->session_batch = 0;
+    std::vector<int32_t> tok(n, 0), pos(n), seq(n);
+    for (int b = 0; b < batch; ++b) {
+        if (ctx->cached[which][b] + rows > std::min(ctx->rt.max_len, m.cfg.max_positions))
+            return fail(SPEC_ERR_CAPACITY, "spec_time_forward: sequence %d would exceed the cache", b);
+        for (int j = 0; j < rows; ++j) {
+            pos[b * rows + j] = ctx->cached[which][b] + j;
+            seq[b * rows + j] = b;
+        }
+    }
+    cudaStream_t st = ctx->stream;
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_token, tok.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_pos, pos.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_seq, seq.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+    SPEC_CUDA_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+    const int status = forward(ctx, m, batch, rows, n, nullptr, nullptr, ctx->target_logits);
+    cudaGraph_t g = nullptr;
+    const cudaError_t end = cudaStreamEndCapture(st, &g);
+    if (status != SPEC_OK) {
+        if (g) cudaGraphDestroy(g);
+        return status;
+    }
+    SPEC_CUDA_TRY(end);
+    cudaGraphExec_t exec = nullptr;
+    const cudaError_t inst = cudaGraphInstantiate(&exec, g, 0);
+    cudaGraphDestroy(g);
+    SPEC_CUDA_TRY(inst);
+    cudaError_t err = cudaGraphLaunch(exec, st);  // untimed: uploads the graph, warms the caches
+    if (err == cudaSuccess) err = cudaEventRecord(ctx->ev[1], st);
+    for (int i = 0; i < repeats && err == cudaSuccess; ++i) err = cudaGraphLaunch(exec, st);
+    if (err == cudaSuccess) err = cudaEventRecord(ctx->ev[2], st);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(st);
+    cudaGraphExecDestroy(exec);
+    SPEC_CUDA_TRY(err);
+    if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
+    float ms = 0.0f;
+    SPEC_CUDA_TRY(cudaEventElapsedTime(&ms, ctx->ev[1], ctx->ev[2]));
+    *ms_per_pass = ms / static_cast<float>(repeats);
+    return SPEC_OK;
+}
+
 extern "C" int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* tokens, int batch, int rows, float* logits) {
     if (!ctx || !tokens || !logits || which < 0 || which > 1 || batch < 1 || rows < 1)
         return fail(SPEC_ERR_BAD_ARG, "spec_forward_logits: bad argument");

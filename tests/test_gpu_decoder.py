@@ -157,3 +157,20 @@ def test_linear_layer_paths_agree_with_the_plain_definition(rows, n_out, k):
     # two bf16 terms keep 16 mantissa bits of x: relative error ~ 2^-16 per product
     assert np.abs(tc.cpu().numpy() - ref).max() <= 1e-4 * scale
     assert torch.equal(tc, packed)
+
+
+def test_timing_a_pass_leaves_the_caches_alone():
+    """spec_time_forward replays a pass beyond the cached rows: positive device time,
+    and the teacher-forced logits that follow are those of the untouched prefix."""
+    cfg, w = _pair("llama_test_target")
+    tokens = workloads.make_prompt(5, 30, cfg["vocab"])
+    ref = Decoder(cfg, w).forward_full(tokens)
+    eng = binding.Engine(cfg, w, max_batch=1, max_len=64, page_size=32, max_gamma=3)
+    eng.forward_logits(0, tokens[None, :20])
+    one, four = eng.time_forward(0, 1, 1, repeats=5), eng.time_forward(0, 1, 4, repeats=5)
+    assert 0.0 < one < 50.0 and 0.0 < four < 50.0
+    got = eng.forward_logits(0, tokens[None, 20:30]).cpu().numpy()[0]
+    _check_logits(got, ref[20:30], cfg["dtype"])
+    with pytest.raises(binding.SpecError):
+        eng.time_forward(1, 1, 1)  # no draft model
+    eng.close()
