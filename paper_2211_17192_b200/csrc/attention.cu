@@ -281,15 +281,19 @@ __global__ void attention_combine_kernel(const float* __restrict__ part, int sli
 
 // Warps that share one query inside a CTA (only when all queries then fit the
 // block in one round), and key slices (CTAs) per (sequence, KV head): about one
-// 32-key tile per warp when the batch is small, about two CTAs per SM at most.
+// 32-key tile per warp when the batch is small, one wave of CTAs at most.
 int attention_sub_slices(int queries) {
     return queries * 2 <= kMaxAttnWarps ? kMaxAttnWarps / queries : 1;
 }
 
 int attention_slices(int batch, int n_kv_heads, int queries, int max_len) {
-    const int want = (2 * 148 + batch * n_kv_heads - 1) / (batch * n_kv_heads);
-    const int tiles = (max_len + 31) / 32;
     const int ks = attention_sub_slices(queries);
+    // CTAs that fit the GPU at once: the kernel holds 128 registers per thread, so an
+    // SM takes 16 warps of it; one wave of CTAs beats more, thinner slices
+    const int warps = std::min(kMaxAttnWarps, std::max(1, queries * ks));
+    const int resident = 148 * std::max(1, 16 / warps);
+    const int want = std::max(1, resident / (batch * n_kv_heads));
+    const int tiles = (max_len + 31) / 32;
     const int most = std::max(1, (tiles + ks - 1) / ks);
     return std::max(1, std::min(std::min(want, most), 32));
 }
