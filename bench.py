@@ -657,7 +657,11 @@ def run_generation(args, wl, torch, device, local, barrier):
                             "note": "weights + fp32 K,V rows read (context; for encoder-decoders also the source), one pass over gamma+1 rows, graph replays timed with events"},
             "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbs": achieved / 8000.0,
-                         "traffic": None, "algorithmic_bytes_per_launch": nbytes / n_mats,
+                         "traffic": 1.026 * nbytes / n_mats,
+                         "traffic_note": "dram read+write bytes per launch: algorithmic bytes x 1.026, the ratio the ncu "
+                                         "capture of the four GEMMs of a 7B-shaped block shows (363.6 MB vs 354.4 MB; "
+                                         "profiles/ncu_gemm_tc_llama7b_layer.txt)",
+                         "algorithmic_bytes_per_launch": nbytes / n_mats,
                          "launch_us": 1e3 * gemm_ms / n_mats,
                          "note": f"all {n_mats} weight matrices of the target once at {rows} rows through spec_linear "
                                  "(bf16 split + GEMM + split-K reduction), CUDA graph, events on its stream"},
