@@ -404,6 +404,19 @@ size_t spec_linear_workspace_bytes(int rows, int n_out, int k);
  * (device pointers, asynchronous on `stream`). */
 size_t spec_packed_weight_bytes(int n_out, int k);
 int spec_pack_weight(const void* w, int n_out, int k, void* packed, void* stream);
+
+/* The tensor-core weight-streaming GEMM exactly as the decoder engine launches it
+ * for one matrix: tile-major weights (spec_pack_weight), the activations as two
+ * bf16 terms, split-K partial sums left for the consumer (in the engine the next
+ * small kernel adds them up).  With split_input != 0 the fp32 rows x [rows, k] are
+ * first split into the workspace; with 0 the split made by an earlier call with
+ * the same (rows, k) and workspace is reused, so that a sweep over many matrices
+ * launches nothing but the GEMM kernel.  *partial (may be NULL) receives the
+ * DEVICE address, inside the workspace, of the sums [*splits][rows][n_out] fp32;
+ * their sum over the first index, in index order, is x . W^T.  Workspace as for
+ * spec_linear.  Asynchronous on `stream`.  Errors: SPEC_ERR_BAD_ARG. */
+int spec_linear_partials(const float* x, const void* w_packed, int rows, int n_out, int k, int split_input,
+                         void* workspace, size_t workspace_bytes, float** partial, int* splits, void* stream);
 int spec_linear(const float* x, const void* w, int w_dtype, int rows, int n_out, int k, int path,
                 float* y, void* workspace, size_t workspace_bytes, void* stream);
 int spec_device_error(void);

@@ -219,6 +219,27 @@ def spec_linear(x, w, path="auto", y=None, workspace=None, n_out=None):
     return y
 
 
+def spec_linear_partials(x, w_packed, n_out, workspace, split_input=True, rows=None, k=None):
+    """The engine's tensor-core GEMM alone on tile-major weights: returns a view
+    [splits, rows, n_out] of the split-K partial sums inside `workspace` (their sum
+    over the first axis is x . W^T).  split_input=False reuses the bf16 split of x that
+    an earlier call with the same (rows, k, workspace) left there (x may then be None)."""
+    h = lib()
+    if x is not None:
+        rows, k = x.shape
+    h.spec_linear_partials.restype = ctypes.c_int
+    h.spec_linear_partials.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                       ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t,
+                                       ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_int), ctypes.c_void_p]
+    where, splits = ctypes.c_void_p(), ctypes.c_int()
+    _check(h.spec_linear_partials(_ptr(x, torch.float32, "x") if x is not None else None, w_packed.data_ptr(), rows,
+                                  n_out, k, 1 if split_input else 0, _ptr(workspace, torch.uint8, "workspace"),
+                                  workspace.numel(), ctypes.byref(where), ctypes.byref(splits), _stream()))
+    offset = where.value - workspace.data_ptr()
+    count = splits.value * rows * n_out
+    return workspace[offset:offset + 4 * count].view(torch.float32).view(splits.value, rows, n_out)
+
+
 def spec_device_error():
     return int(lib().spec_device_error())
 

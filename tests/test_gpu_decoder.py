@@ -157,6 +157,16 @@ def test_linear_layer_paths_agree_with_the_plain_definition(rows, n_out, k):
     # two bf16 terms keep 16 mantissa bits of x: relative error ~ 2^-16 per product
     assert np.abs(tc.cpu().numpy() - ref).max() <= 1e-4 * scale
     assert torch.equal(tc, packed)
+    # the GEMM kernel alone: its split-K partial sums, added in split order, are the same result
+    ws = torch.empty(binding.spec_linear_workspace_bytes(rows, n_out, k), dtype=torch.uint8, device="cuda")
+    pk = binding.spec_pack_weight(wd)
+    parts = binding.spec_linear_partials(xd, pk, n_out, ws)
+    total = parts[0].clone()
+    for s in range(1, parts.shape[0]):
+        total += parts[s]
+    assert torch.equal(total, tc)
+    again = binding.spec_linear_partials(None, pk, n_out, ws, split_input=False, rows=rows, k=k)  # reuses the split
+    assert torch.equal(again.sum(0), parts.sum(0))
 
 
 def test_timing_a_pass_leaves_the_caches_alone():
