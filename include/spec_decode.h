@@ -91,6 +91,24 @@ int spec_verify_sample(const float* target_logits, const float* draft_logits,
                        int32_t* n_accepted, int32_t* next_token,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same with the lenience factor of Appendix A.5, `lenience` in (0, 1]:
+ * q_i(x_i) is multiplied by it before the comparison, i.e. x_i is rejected iff
+ * r_i * lenience * q_i(x_i) > p_i(x_i); the adjusted distribution after a
+ * rejection stays norm(max(0, p - q)) (the appendix changes only the
+ * comparison).  The output is then no longer distributed as the target's, but
+ * no token is emitted with probability above p(x) / lenience.  At T = 0 lenience
+ * is applied before standardising: x_i is accepted iff
+ * logit(x_i) >= max logit + ln(lenience) on the target's row (p(x_i) >= lenience
+ * * max p for the T = 1 softmax); the appendix prints this inequality the other
+ * way round, which would accept everything at lenience 1.  lenience == 1 is
+ * spec_verify_sample exactly.  Errors as above, plus SPEC_ERR_BAD_ARG for a
+ * lenience outside (0, 1]. */
+int spec_verify_sample_lenient(const float* target_logits, const float* draft_logits,
+                               const int32_t* draft_tokens, const float* uniforms,
+                               int batch, int gamma, int vocab, float temperature, float lenience,
+                               int32_t* n_accepted, int32_t* next_token,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
 /* ------------------------------------------------------------------------- *
  * spec_verify_sample for callers that cannot allocate device memory.  (The
  * paper has no counterpart: this is a property of the library, not of the
@@ -325,6 +343,11 @@ int spec_generate(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_le
  * generation in progress. */
 int spec_begin(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride,
                int batch, int n_new, int gamma, float temperature, uint64_t seed);
+
+/* Lenience factor (Appendix A.5; see spec_verify_sample_lenient) used by the
+ * generations that start after this call; 1 (the default) is Algorithm 1 as
+ * printed.  Errors: SPEC_ERR_BAD_ARG outside (0, 1]. */
+int spec_set_lenience(spec_ctx* ctx, float lenience);
 
 /* Timing instrument (no counterpart in Algorithm 1): from the next spec_begin /
  * spec_generate on, the accept decision of every drafted token is replaced by

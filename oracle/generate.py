@@ -65,7 +65,8 @@ class GenerationResult:
         return sum(it.n_accepted for it in self.iterations)
 
 
-def speculative_generate(target, draft, prompt, n_new, gamma, temperature, seed, sequence=0, cached=True, keep_logits=False):
+def speculative_generate(target, draft, prompt, n_new, gamma, temperature, seed, sequence=0, cached=True, keep_logits=False,
+                         lenience=1.0):
     """Algorithm 1 repeated until n_new tokens are emitted.
 
     `target` and `draft` are model objects with forward_rows / forward_full /
@@ -107,9 +108,9 @@ def speculative_generate(target, draft, prompt, n_new, gamma, temperature, seed,
         q_arr = np.stack(q_logits) if gamma else np.zeros((0, p_logits.shape[1]))
         # The final draw decides the token at position L + n, known only after
         # the accept tests: evaluate once with a placeholder to find n.
-        probe = verify_step(p_logits, q_arr, xs, uniforms + [0.5], temperature)
+        probe = verify_step(p_logits, q_arr, xs, uniforms + [0.5], temperature, lenience)
         u_final = philox.uniform(seed, L + probe.n_accepted, sequence, philox.PURPOSE_FINAL)
-        res = verify_step(p_logits, q_arr, xs, uniforms + [u_final], temperature)
+        res = verify_step(p_logits, q_arr, xs, uniforms + [u_final], temperature, lenience)
         n = res.n_accepted
         committed.extend(xs[:n])
         committed.append(res.next_token)

@@ -23,8 +23,23 @@ What follows the paper, and where it is silent:
   order on unnormalised weights w: the smallest k with w_0 + ... + w_k > u * W,
   W the total; if rounding leaves none, the last k with w_k > 0.
 
+* Appendix A.5 (lenience l in (0, 1]): q(x) is multiplied by l before it is
+  compared with p(x): reject iff r_i * l * q_i(x_i) > p_i(x_i).  The text
+  changes only the comparison; reading: the adjusted distribution after a
+  rejection stays norm(max(0, p - q)) (a rejection still implies q(x) > p(x),
+  so it is well defined, and no token is then emitted with probability above
+  p(x) / l).  At T = 0 the paper applies lenience before standardising; its
+  printed condition "p(x) <= l * max(p)" would accept everything at l = 1, so
+  the inequality is read the other way round: x_i is accepted iff
+  p(x_i) >= l * max p with p the T = 1 softmax of the target's logits, i.e.
+  logit(x_i) >= max logit + ln l; l = 1 keeps the strict rule (x_i accepted
+  iff it is the lowest-index maximum).
+
 Pins (tests/test_oracle_sampling.py): emitted-token law equals p over 10^6
-seeded trials (Appendix A.1); acceptance frequency equals sum min(p, q)
+seeded trials (Appendix A.1); with lenience the acceptance frequency equals
+sum min(p / l, q) (Appendix A.5), the emitted law equals min(q, p / l) +
+(1 - alpha_l) * max(0, p - q) / (1 - beta) and never exceeds p / l, and
+l = 1 is the strict algorithm; acceptance frequency equals sum min(p, q)
 (Theorem 3.5); rejected-branch law equals max(0, p - q) / (1 - beta);
 p = q always accepts, disjoint supports never accept (Corollary 3.4); exact
 measures of every outcome on an (r, u) grid for vocabularies <= 8; gamma = 0
@@ -74,15 +89,15 @@ def inverse_cdf(weights, u):
     return k, float(margin)
 
 
-def speculative_sampling(p, q, x, r, u):
+def speculative_sampling(p, q, x, r, u, lenience=1.0):
     """Section 2.3 for one token: x was drawn from q; returns (accepted, token).
 
-    Keeps x unless r > p(x) / q(x); otherwise draws from norm(max(0, p - q))
-    with the uniform u.
+    Keeps x unless r > p(x) / (l q(x)) (l = 1: the paper's algorithm; l < 1:
+    Appendix A.5); otherwise draws from norm(max(0, p - q)) with the uniform u.
     """
     p = np.asarray(p, dtype=np.float64)
     q = np.asarray(q, dtype=np.float64)
-    if not (r * q[x] > p[x]):
+    if not (r * lenience * q[x] > p[x]):
         return True, int(x)
     residual = np.maximum(0.0, p - q)
     if not residual.sum() > 0.0:
@@ -104,7 +119,16 @@ class VerifyResult:
     betas: list = field(default_factory=list)  # sum min(p_i, q_i), tests evaluated
 
 
-def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature):
+def lenient_greedy_accepts(target_row, x, lenience):
+    """Appendix A.5 at T = 0: (accepted, margin).  l = 1: x must be the lowest-index
+    maximum; l < 1: logit(x) >= max logit + ln l (p(x) >= l max p before standardising)."""
+    if lenience >= 1.0:
+        return int(x) == int(np.argmax(target_row)), float("inf")
+    slack = float(target_row[int(x)] - target_row.max() - np.log(lenience))
+    return slack >= 0.0, abs(slack)
+
+
+def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0):
     """Algorithm 1 from "determine the number of accepted guesses" to the end.
 
     target_logits [gamma+1, V]: row i-1 gives p_i (i = 1..gamma+1).
@@ -130,9 +154,16 @@ def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature
         r = float(uniforms[i])
         betas.append(float(np.minimum(p[i], q[i]).sum()))
         top2_gap = min(top2_gap, _top2_gap(tl[i]))
+        if temperature == 0 and lenience < 1.0:
+            accepted, slack = lenient_greedy_accepts(tl[i], x, lenience)
+            accept_margin = min(accept_margin, slack)
+            if not accepted:
+                n = i
+                break
+            continue
         if q[i][x] > 0.0:
-            accept_margin = min(accept_margin, abs(r - p[i][x] / q[i][x]))
-        if r * q[i][x] > p[i][x]:
+            accept_margin = min(accept_margin, abs(r - p[i][x] / (lenience * q[i][x])))
+        if r * lenience * q[i][x] > p[i][x]:
             n = i
             break
 
@@ -149,10 +180,10 @@ def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature
     return VerifyResult(n, t, accept_margin, cdf_margin, top2_gap, fallback, betas)
 
 
-def verify_batch(target_logits, draft_logits, draft_tokens, uniforms, temperature):
+def verify_batch(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0):
     """`verify_step` for every sequence of a batch: [B, ...] inputs -> list."""
     return [
-        verify_step(target_logits[b], draft_logits[b], draft_tokens[b], uniforms[b], temperature)
+        verify_step(target_logits[b], draft_logits[b], draft_tokens[b], uniforms[b], temperature, lenience)
         for b in range(len(target_logits))
     ]
 
@@ -184,7 +215,7 @@ def sample_trials(logits, uniforms, temperature):
     return np.where(k >= w.shape[0], positive[-1], k).astype(np.int64)
 
 
-def verify_trials(target_logits, draft_logits, draft_tokens, uniforms, temperature):
+def verify_trials(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0):
     """Many independent trials of `verify_step` that share one set of logits.
 
     target_logits [gamma+1, V] and draft_logits [gamma, V] are fixed;
@@ -206,7 +237,10 @@ def verify_trials(target_logits, draft_logits, draft_tokens, uniforms, temperatu
     undecided = np.ones(trials, dtype=bool)
     for i in range(gamma):
         x = xs[:, i]
-        rejected = us[:, i] * q[i][x] > p[i][x]
+        if temperature == 0 and lenience < 1.0:
+            rejected = ~(tl[i][x] - tl[i].max() - np.log(lenience) >= 0.0)
+        else:
+            rejected = us[:, i] * lenience * q[i][x] > p[i][x]
         first = undecided & rejected
         n[first] = i
         undecided &= ~rejected

@@ -103,8 +103,9 @@ def spec_verify_sample_workspace_bytes(batch, gamma, vocab):
 
 
 def spec_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, temperature,
-                       n_accepted=None, next_token=None, workspace=None):
-    """Speculative sampling for a batch; see `spec_verify_sample` in the header.
+                       n_accepted=None, next_token=None, workspace=None, lenience=1.0):
+    """Speculative sampling for a batch; see `spec_verify_sample` (and, for
+    lenience < 1, `spec_verify_sample_lenient`) in the header.
 
     target_logits [B, gamma+1, V] fp32, draft_logits [B, gamma, V] fp32,
     draft_tokens [B, gamma] int32, uniforms [B, gamma+1] fp32, all CUDA.
@@ -127,14 +128,20 @@ def spec_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, temp
         raise ValueError("draft_tokens must be [B, gamma]")
     if uniforms is not None and tuple(uniforms.shape) != (batch, gamma + 1):
         raise ValueError("uniforms must be [B, gamma+1]")
-    _check(lib().spec_verify_sample(
-        _ptr(target_logits, torch.float32, "target_logits"),
-        _ptr(draft_logits, torch.float32, "draft_logits", optional=True),
-        _ptr(draft_tokens, torch.int32, "draft_tokens", optional=True),
-        _ptr(uniforms, torch.float32, "uniforms", optional=True),
-        batch, gamma, vocab, float(temperature),
-        _ptr(n_accepted, torch.int32, "n_accepted"), _ptr(next_token, torch.int32, "next_token"),
-        _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()))
+    pointers = (_ptr(target_logits, torch.float32, "target_logits"),
+                _ptr(draft_logits, torch.float32, "draft_logits", optional=True),
+                _ptr(draft_tokens, torch.int32, "draft_tokens", optional=True),
+                _ptr(uniforms, torch.float32, "uniforms", optional=True))
+    outputs = (_ptr(n_accepted, torch.int32, "n_accepted"), _ptr(next_token, torch.int32, "next_token"),
+               _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream())
+    if lenience == 1.0:
+        _check(lib().spec_verify_sample(*pointers, batch, gamma, vocab, float(temperature), *outputs))
+    else:
+        h = lib()
+        h.spec_verify_sample_lenient.restype = ctypes.c_int
+        h.spec_verify_sample_lenient.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int] * 3 + [ctypes.c_float] * 2 + \
+            [ctypes.c_void_p] * 3 + [ctypes.c_size_t, ctypes.c_void_p]
+        _check(h.spec_verify_sample_lenient(*pointers, batch, gamma, vocab, float(temperature), float(lenience), *outputs))
     return n_accepted, next_token
 
 
@@ -309,6 +316,8 @@ def _declare_engine(h):
     h.spec_truncate.argtypes = [vp, c.c_int, vp, c.c_int]
     h.spec_forward_logits.restype = c.c_int
     h.spec_forward_logits.argtypes = [vp, c.c_int, vp, c.c_int, c.c_int, vp]
+    h.spec_set_lenience.restype = c.c_int
+    h.spec_set_lenience.argtypes = [vp, c.c_float]
     h.spec_set_imposed_acceptance.restype = c.c_int
     h.spec_set_imposed_acceptance.argtypes = [vp, c.c_float]
     h.spec_time_forward.restype = c.c_int
@@ -448,6 +457,10 @@ class Engine:
                                    float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF, out.ctypes.data,
                                    ctypes.byref(st)))
         return out, {name: getattr(st, name) for name, _ in _Stats._fields_}
+
+    def set_lenience(self, lenience):
+        """Lenience factor of Appendix A.5 for the generations that follow (1 = Algorithm 1)."""
+        _check(lib().spec_set_lenience(self._ctx, float(lenience)))
 
     def set_imposed_acceptance(self, alpha):
         """Timing instrument: accept every drafted token with probability `alpha`

@@ -45,11 +45,12 @@ struct spec_ctx {
     void* sampler_ws = nullptr;
     struct Params { unsigned long long seed; int n_new; float imposed_alpha; }* params = nullptr;
     float imposed_alpha = -1.0f;  // >= 0: timing instrument, see spec_set_imposed_acceptance
+    float lenience = 1.0f;        // Appendix A.5; 1 = Algorithm 1 as printed
 
     // cached iteration graph
     cudaGraphExec_t graph = nullptr;
     int graph_batch = -1, graph_gamma = -1;
-    float graph_temperature = -1.0f;
+    float graph_temperature = -1.0f, graph_lenience = 1.0f;
 
     // generation in progress (spec_begin / spec_generate)
     int session_batch = 0, session_gamma = 0, session_n_new = 0;
@@ -396,14 +397,16 @@ int enqueue_iteration(spec_ctx* ctx, int batch, int gamma, float temperature) {
                         ctx->length, batch, gamma, ctx->rt.max_len, ctx->row_token, ctx->row_pos, ctx->row_seq));
     SPEC_TRY(forward(ctx, ctx->model[0], batch, gamma + 1, batch * (gamma + 1), nullptr, nullptr, ctx->target_logits));
     SPEC_TRY(launch_verify_sample(ctx->target_logits, ctx->draft_logits, ctx->draft_tokens, ctx->accept_u, ctx->final_u,
-                                  batch, gamma, vocab, temperature, ctx->n_accepted, ctx->next_token, ctx->sampler_ws, st));
+                                  batch, gamma, vocab, temperature, ctx->lenience, ctx->n_accepted, ctx->next_token,
+                                  ctx->sampler_ws, st));
     return launch_pdl(commit_kernel, dim3(blocks_b), dim3(threads), 0, st, ctx->params, ctx->draft_tokens,
                       ctx->n_accepted, ctx->next_token, ctx->accept_u, ctx->prompt_len, batch, gamma, ctx->rt.max_len,
                       ctx->tokens, ctx->length, ctx->counters);
 }
 
 int build_graph(spec_ctx* ctx, int batch, int gamma, float temperature) {
-    if (ctx->graph && ctx->graph_batch == batch && ctx->graph_gamma == gamma && ctx->graph_temperature == temperature)
+    if (ctx->graph && ctx->graph_batch == batch && ctx->graph_gamma == gamma && ctx->graph_temperature == temperature &&
+        ctx->graph_lenience == ctx->lenience)
         return SPEC_OK;
     if (ctx->graph) {
         cudaGraphExecDestroy(ctx->graph);
@@ -424,6 +427,7 @@ int build_graph(spec_ctx* ctx, int batch, int gamma, float temperature) {
     ctx->graph_batch = batch;
     ctx->graph_gamma = gamma;
     ctx->graph_temperature = temperature;
+    ctx->graph_lenience = ctx->lenience;
     return SPEC_OK;
 }
 
@@ -949,6 +953,12 @@ extern "C" int spec_read_tokens(spec_ctx* ctx, int32_t* out_tokens) {
     SPEC_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
     for (int b = 0; b < batch; ++b)
         std::memcpy(out_tokens + static_cast<size_t>(b) * n_new, &host_tokens[static_cast<size_t>(b) * max_len + ctx->session_prompt_len[b]], n_new * sizeof(int32_t));
+    return SPEC_OK;
+}
+
+extern "C" int spec_set_lenience(spec_ctx* ctx, float lenience) {
+    if (!ctx || !(lenience > 0.0f) || !(lenience <= 1.0f)) return fail(SPEC_ERR_BAD_ARG, "spec_set_lenience: lenience must be in (0, 1]");
+    ctx->lenience = lenience;
     return SPEC_OK;
 }
 

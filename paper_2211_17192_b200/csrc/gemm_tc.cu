@@ -523,6 +523,29 @@ extern "C" int spec_linear(const float* x, const void* w, int w_dtype, int rows,
     return launch_gemm_tc(hi, lo, padded_rows(rows), w, path == 3, nullptr, nullptr, rows, n_out, k, partial, y, st);
 }
 
+extern "C" int spec_linear_partials(const float* x, const void* w_packed, int rows, int n_out, int k, int split_input,
+                                    void* workspace, size_t workspace_bytes, float** partial, int* splits, void* stream) {
+    using namespace spec;
+    if (!w_packed || (split_input && !x)) return fail(SPEC_ERR_BAD_ARG, "spec_linear_partials: null pointer");
+    if (rows < 1 || n_out < 1 || k < 8 || k % 8) return fail(SPEC_ERR_BAD_ARG, "spec_linear_partials: rows=%d n_out=%d k=%d (k must be a multiple of 8)", rows, n_out, k);
+    if (!workspace || workspace_bytes < spec_linear_workspace_bytes(rows, n_out, k) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return fail(SPEC_ERR_BAD_ARG, "spec_linear_partials: workspace missing, too small or not 256-byte aligned");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t split_bytes = align256(static_cast<size_t>(padded_rows(rows)) * k * 2);
+    char* base = static_cast<char*>(workspace);
+    __nv_bfloat16* hi = reinterpret_cast<__nv_bfloat16*>(base);
+    __nv_bfloat16* lo = reinterpret_cast<__nv_bfloat16*>(base + split_bytes);
+    float* sums = reinterpret_cast<float*>(base + 2 * split_bytes);
+    if (split_input) {
+        SPEC_CUDA_TRY(cudaMemsetAsync(base, 0, 2 * split_bytes, st));
+        const int status = launch_split_bf16(x, static_cast<size_t>(rows) * k, hi, lo, st);
+        if (status != SPEC_OK) return status;
+    }
+    if (partial) *partial = sums;
+    if (splits) *splits = gemm_tc_splits(n_out, k, rows);
+    return launch_gemm_tc_partials(hi, lo, padded_rows(rows), w_packed, true, rows, n_out, k, sums, st);
+}
+
 extern "C" size_t spec_packed_weight_bytes(int n_out, int k) {
     if (n_out < 1 || k < 1) return 0;
     return spec::packed_weight_elems(n_out, k) * 2;

@@ -138,7 +138,7 @@ int launch_ffn_act(const float* u, const float* partial, int splits, int n_rows,
 // sampling.cu
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
                          const float* uniforms, const float* final_uniforms, int batch, int gamma, int vocab,
-                         float temperature, int32_t* n_accepted, int32_t* next_token, void* workspace,
+                         float temperature, float lenience, int32_t* n_accepted, int32_t* next_token, void* workspace,
                          cudaStream_t stream);
 int launch_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
                   int32_t* tokens, cudaStream_t stream);

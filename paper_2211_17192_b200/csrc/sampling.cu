@@ -497,7 +497,7 @@ __global__ void __launch_bounds__(kFinishThreads, 2)
 verify_finish_kernel(const float* __restrict__ target_logits, const float* __restrict__ draft_logits,
                      const int32_t* __restrict__ draft_tokens, const float* __restrict__ uniforms, int gamma,
                      int vocab, float inv_t, int chunks, int cluster_size, const ChunkStat* __restrict__ stats,
-                     const float* __restrict__ final_uniforms, int32_t* __restrict__ n_accepted,
+                     const float* __restrict__ final_uniforms, float lenience, int32_t* __restrict__ n_accepted,
                      int32_t* __restrict__ next_token) {
     __shared__ FinishShared sh;
     const int tid = threadIdx.x;
@@ -517,6 +517,9 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
     int my_x = -1;
     if (tid < rows && tid != gamma)
         my_x = draft_tokens[static_cast<size_t>(b) * gamma + (tid < gamma ? tid : tid - gamma - 1)];
+    // lenient argmax decoding compares the target's logit at the drafted token with the row maximum
+    float my_xlogit = 0.0f;
+    if (GREEDY && lenience < 1.0f && tid < gamma && my_x >= 0 && my_x < vocab) my_xlogit = __ldg(tl + static_cast<size_t>(tid) * vocab + my_x);
     pdl_trigger();
     pdl_wait();
 
@@ -558,12 +561,15 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
         bool reject = true;
         if (my_x >= 0 && my_x < vocab) {
             if (GREEDY) {
-                reject = my_x != __float_as_int(sh.row_aux[tid]);
+                // strict: x must be the lowest-index maximum; lenient (Appendix A.5 at T = 0):
+                // p(x) >= l max p before standardising, i.e. logit(x) >= max logit + ln l
+                reject = lenience < 1.0f ? !(my_xlogit - sh.row_max[tid] - logf(lenience) >= 0.0f)
+                                         : my_x != __float_as_int(sh.row_aux[tid]);
             } else {
                 const float ep = expf((sh.row_x[tid] - sh.row_max[tid]) * inv_t);
                 const float eq = expf((sh.row_x[gamma + 1 + tid] - sh.row_max[gamma + 1 + tid]) * inv_t);
-                // r * q(x) > p(x) with p = ep / Sp, q = eq / Sq, cross-multiplied
-                reject = my_uniform * eq * sh.row_aux[tid] > ep * sh.row_aux[gamma + 1 + tid];
+                // r * l * q(x) > p(x) with p = ep / Sp, q = eq / Sq, cross-multiplied (l = 1: Algorithm 1)
+                reject = my_uniform * lenience * eq * sh.row_aux[tid] > ep * sh.row_aux[gamma + 1 + tid];
             }
         }
         if (reject) atomicMin(&sh.n, tid);
@@ -689,7 +695,7 @@ size_t verify_sample_workspace_bytes(int batch, int gamma, int vocab) {
 
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
                          const float* uniforms, const float* final_uniforms, int batch, int gamma, int vocab,
-                         float temperature, int32_t* n_accepted, int32_t* next_token, void* workspace,
+                         float temperature, float lenience, int32_t* n_accepted, int32_t* next_token, void* workspace,
                          cudaStream_t stream) {
     const bool greedy = temperature == 0.0f;
     const int rows = greedy ? gamma + 1 : 2 * gamma + 1;
@@ -730,7 +736,7 @@ int launch_verify_sample(const float* target_logits, const float* draft_logits, 
 #define SPEC_LAUNCH_FINISH(G, V)                                                                                  \
     SPEC_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_finish_kernel<G, V>, target_logits, draft_logits, draft_tokens, \
                                      uniforms, gamma, vocab, inv_t, chunks, cluster_size, stats_in,              \
-                                     final_uniforms, n_accepted, next_token))
+                                     final_uniforms, lenience, n_accepted, next_token))
     if (greedy && vec) SPEC_LAUNCH_FINISH(true, true);
     else if (greedy) SPEC_LAUNCH_FINISH(true, false);
     else if (vec) SPEC_LAUNCH_FINISH(false, true);
@@ -766,11 +772,12 @@ extern "C" size_t spec_verify_sample_workspace_bytes(int batch, int gamma, int v
     return spec::verify_sample_workspace_bytes(batch, gamma, vocab);
 }
 
-extern "C" int spec_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
-                                  const float* uniforms, int batch, int gamma, int vocab, float temperature,
-                                  int32_t* n_accepted, int32_t* next_token, void* workspace, size_t workspace_bytes,
-                                  void* stream) {
+extern "C" int spec_verify_sample_lenient(const float* target_logits, const float* draft_logits,
+                                          const int32_t* draft_tokens, const float* uniforms, int batch, int gamma,
+                                          int vocab, float temperature, float lenience, int32_t* n_accepted,
+                                          int32_t* next_token, void* workspace, size_t workspace_bytes, void* stream) {
     using namespace spec;
+    if (!(lenience > 0.0f) || !(lenience <= 1.0f)) return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: lenience must be in (0, 1]");
     if (batch < 0 || gamma < 0 || gamma > kMaxGamma || vocab < 1)
         return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: batch=%d gamma=%d (max %d) vocab=%d", batch, gamma, kMaxGamma, vocab);
     if (!(temperature >= 0.0f) || !isfinite(temperature))
@@ -785,7 +792,15 @@ extern "C" int spec_verify_sample(const float* target_logits, const float* draft
         (reinterpret_cast<uintptr_t>(workspace) & 255u))
         return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: workspace too small (%zu bytes) or not 256-byte aligned", workspace_bytes);
     return launch_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, nullptr, batch, gamma, vocab,
-                                temperature, n_accepted, next_token, workspace, static_cast<cudaStream_t>(stream));
+                                temperature, lenience, n_accepted, next_token, workspace, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int spec_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
+                                  const float* uniforms, int batch, int gamma, int vocab, float temperature,
+                                  int32_t* n_accepted, int32_t* next_token, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+    return spec_verify_sample_lenient(target_logits, draft_logits, draft_tokens, uniforms, batch, gamma, vocab, temperature,
+                                      1.0f, n_accepted, next_token, workspace, workspace_bytes, stream);
 }
 
 // ---- spec_verify_sample without any allocation ---------------------------------
@@ -847,7 +862,7 @@ extern "C" int spec_verify_sample_static(const float* target_logits, const float
     const int status = static_stats_address(&scratch);
     if (status != SPEC_OK) return status;
     return launch_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, nullptr, batch, gamma, vocab,
-                                temperature, n_accepted, next_token, scratch, static_cast<cudaStream_t>(stream));
+                                temperature, 1.0f, n_accepted, next_token, scratch, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int spec_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature,

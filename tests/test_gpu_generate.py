@@ -160,3 +160,26 @@ def test_imposed_acceptance_is_iid_with_the_chosen_rate(tiny):
     a, _ = eng.generate([prompt], 20, gamma, 1.0, 3)
     b, _ = eng.generate([prompt], 20, gamma, 1.0, 3)
     assert np.array_equal(a, b)
+
+
+def test_lenient_generation_matches_the_oracle_and_accepts_more(tiny):
+    """Appendix A.5 through the whole loop: token stream equal to the oracle's with the
+    same lenience, and a higher acceptance rate than the strict run."""
+    eng, target, draft, cfg = tiny
+    prompt = workloads.make_prompt(12, 10, cfg["vocab"])
+    try:
+        eng.set_lenience(0.2)
+        ref = oracle_generate.speculative_generate(target, draft, prompt, 48, 3, 1.0, seed=21, lenience=0.2)
+        got, lenient = eng.generate([prompt], 48, 3, 1.0, 21)
+        got = got[0].tolist()
+        diff = next((k for k in range(48) if got[k] != ref.tokens[k]), None)
+        if diff is not None:  # a decision within tolerance of a boundary ends the comparison
+            index = len(prompt) + diff
+            it = next(i for i in ref.iterations if i.start_len <= index <= i.start_len + i.n_accepted)
+            assert min([it.accept_margin, it.cdf_margin] + list(it.draft_cdf_margins)) < 1e-3
+        with pytest.raises(binding.SpecError):
+            eng.set_lenience(1.5)
+    finally:
+        eng.set_lenience(1.0)
+    _, strict = eng.generate([prompt], 48, 3, 1.0, 21)
+    assert lenient["tests_passed"] / lenient["tests_evaluated"] > strict["tests_passed"] / strict["tests_evaluated"]

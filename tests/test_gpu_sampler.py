@@ -24,9 +24,9 @@ def _draft_tokens(ql, seed, temperature):
     return xs, draw
 
 
-def _run(tl, ql, xs, us, temperature):
+def _run(tl, ql, xs, us, temperature, lenience=1.0):
     n, t = binding.spec_verify_sample(to_dev(tl), to_dev(ql) if ql.size else None,
-                                      to_dev(xs) if xs.size else None, to_dev(us), temperature)
+                                      to_dev(xs) if xs.size else None, to_dev(us), temperature, lenience=lenience)
     torch.cuda.synchronize()
     return n, t
 
@@ -68,6 +68,26 @@ def test_shapes_and_edges(batch, gamma, vocab, temperature):
     n, t = _run(tl, ql, xs, us, temperature)
     flagged, _ = compare_verify(n, t, tl, ql, xs, us, temperature)
     assert flagged <= 1
+
+
+@pytest.mark.parametrize("temperature", [1.0, 0.0])
+@pytest.mark.parametrize("lenience", [0.5, 0.1])
+def test_lenience(temperature, lenience):
+    """Appendix A.5: decisions and tokens identical to the oracle; more drafted tokens
+    survive than under the strict rule."""
+    batch, gamma, vocab = 48, 5, 8192
+    tl, ql = workloads.make_sampler_logits(77, batch, gamma, vocab, 2.0)
+    xs, _ = _draft_tokens(ql, 5, 1.0)  # drafted by sampling, also for the argmax case: a spread of logits at x
+    us = workloads.make_uniform_grid(6, (batch, gamma + 1))
+    n, t = _run(tl, ql, xs, us, temperature, lenience)
+    flagged, _ = compare_verify(n, t, tl, ql, xs, us, temperature, lenience)
+    assert flagged <= 1
+    strict, _ = _run(tl, ql, xs, us, temperature)
+    assert n.sum().item() >= strict.sum().item()
+    if temperature > 0:
+        assert n.sum().item() > strict.sum().item()
+    with pytest.raises(binding.SpecError):
+        _run(tl, ql, xs, us, temperature, 0.0)
 
 
 def test_identical_and_disjoint_distributions():

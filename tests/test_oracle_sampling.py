@@ -244,3 +244,67 @@ def test_speculative_sampling_single_token_rule():
     # rejected: residual = [0.3, 0.1, 0] / 0.4 -> boundary at 0.75
     assert sampling.speculative_sampling(p, q, 2, 0.34, 0.74) == (False, 0)
     assert sampling.speculative_sampling(p, q, 2, 0.34, 0.76) == (False, 1)
+
+
+@pytest.mark.parametrize("lenience", [0.5, 0.3, 0.1])
+def test_lenience_acceptance_and_emitted_law(lenience):
+    """Appendix A.5: alpha_l = sum min(p / l, q); no token is emitted with probability above p / l."""
+    tl, ql = _fixed_pair(2.0)
+    p = sampling.standardise(tl[0], 1.0)
+    q = sampling.standardise(ql[0], 1.0)
+    idx = np.arange(TRIALS)
+    x = sampling.sample_trials(ql[0], philox.uniforms_vec(6, idx, 0, philox.PURPOSE_DRAFT), 1.0)
+    r = philox.uniforms_vec(6, idx, 0, philox.PURPOSE_ACCEPT)
+    u = philox.uniforms_vec(6, idx, 0, philox.PURPOSE_FINAL)
+    n, t = sampling.verify_trials(tl, ql, x[:, None], np.stack([r, u], axis=1), 1.0, lenience)
+    alpha_l = analysis.beta_lenient(p, q, lenience)
+    assert alpha_l > analysis.beta(p, q)
+    assert abs((n == 1).mean() - alpha_l) <= 4 * np.sqrt(alpha_l * (1 - alpha_l) / TRIALS)
+    # exact law of the first emitted token under the reading taken for the adjusted distribution
+    residual = np.maximum(0, p - q)
+    law = np.minimum(q, p / lenience) + (1 - alpha_l) * residual / residual.sum()
+    assert law.sum() == pytest.approx(1.0, abs=1e-12)
+    assert np.all(law <= p / lenience + 1e-15)
+    first = np.where(n == 1, x, t)
+    assert _chi_square_p(np.bincount(first, minlength=VOCAB), law) > 1e-3
+    # and it is no longer p
+    assert _chi_square_p(np.bincount(first, minlength=VOCAB), p) < 1e-6
+
+
+def test_lenience_one_is_the_strict_algorithm_and_scalar_equals_vectorised():
+    tl, ql = _fixed_pair(2.0)
+    idx = np.arange(2000)
+    x = sampling.sample_trials(ql[0], philox.uniforms_vec(7, idx, 0, philox.PURPOSE_DRAFT), 1.0)
+    us = np.stack([philox.uniforms_vec(7, idx, 0, philox.PURPOSE_ACCEPT), philox.uniforms_vec(7, idx, 0, philox.PURPOSE_FINAL)], axis=1)
+    strict = sampling.verify_trials(tl, ql, x[:, None], us, 1.0)
+    same = sampling.verify_trials(tl, ql, x[:, None], us, 1.0, 1.0)
+    assert np.array_equal(strict[0], same[0]) and np.array_equal(strict[1], same[1])
+    for temperature in (1.0, 0.0):
+        n, t = sampling.verify_trials(tl, ql, x[:, None], us, temperature, 0.3)
+        for k in range(0, 2000, 37):
+            ref = sampling.verify_step(tl, ql, x[k : k + 1], us[k], temperature, 0.3)
+            assert (ref.n_accepted, ref.next_token) == (n[k], t[k])
+
+
+def test_lenience_at_temperature_zero():
+    """Accept x iff p(x) >= l * max p with p the T = 1 softmax of the target row; a rejected slot gets argmax p."""
+    rng = np.random.default_rng(3)
+    tl = rng.standard_normal((2, 16)) * 2.0
+    ql = rng.standard_normal((1, 16))
+    p = sampling.standardise(tl[0], 1.0)
+    best = int(np.argmax(tl[0]))
+    for lenience in (0.5, 0.3, 0.1, 1e-9):
+        for x in range(16):
+            res = sampling.verify_step(tl, ql, [x], [0.5, 0.5], 0.0, lenience)
+            assert (res.n_accepted == 1) == bool(p[x] >= lenience * p.max() * (1 - 1e-12))
+            if res.n_accepted == 0:
+                assert res.next_token == best
+            else:
+                assert res.next_token == int(np.argmax(tl[1]))
+    # strict rule at l = 1: the draft's own argmax x is accepted only if it is the target's argmax
+    accepted = []
+    for x in range(16):
+        draft = np.zeros((1, 16))
+        draft[0, x] = 5.0
+        accepted.append(sampling.verify_step(tl, draft, [x], [0.5, 0.5], 0.0, 1.0).n_accepted)
+    assert accepted == [1 if x == best else 0 for x in range(16)]
