@@ -308,7 +308,7 @@ class GenerationWorkload:
         def timed(which, rows):
             return eng.time_forward(which, self.batch, rows, repeats)
         eng.reset()
-        chunk = 64
+        chunk = max(1, 64 // self.batch)  # the teacher-forced entry point takes 64 rows per call
         for which in (0, 1):
             for c0 in range(0, tok.shape[1], chunk):
                 eng.forward_logits(which, tok[:, c0:c0 + chunk])
@@ -356,171 +356,6 @@ class GenerationWorkload:
         del packed
         torch.cuda.empty_cache()
         return nbytes, ms, len(mats)
-
-    def cpu_sample(self, budget_s):
-        from oracle import sampling as oracle_sampling
-        tl, ql, us, draw = self.host[1] if hasattr(self, "host") else self.host_inputs(0)[1]
-        xs = np.zeros((self.batch, self.gamma), dtype=np.int32)
-        t0 = time.perf_counter()
-        done = tokens = 0
-        while time.perf_counter() - t0 < budget_s or done < 2:
-            b = done % self.batch
-            for i in range(self.gamma):
-                xs[b, i] = oracle_sampling.sample_token(ql[b, i], draw[b * self.gamma + i], self.temperature)[0]
-            res = oracle_sampling.verify_step(tl[b], ql[b], xs[b], us[b], self.temperature)
-            tokens += res.n_accepted + 1
-            done += 1
-        dt = time.perf_counter() - t0
-        return tokens / dt, f"{done} sequences drawn from one batch of {self.batch} (draft draws + verify), {dt:.1f} s"
-
-
-# --------------------------------------------------------------------------- #
-# workload: speculative decoding of a model pair (Algorithm 1, device-resident loop)
-# --------------------------------------------------------------------------- #
-def gpu_weights(cfg, seed, device):
-    """Seeded random-init weights drawn on the GPU with torch's generator (matrices
-    N(0, 0.02^2), head N(0, head_std^2), gains 1; bf16 models stored as bf16)."""
-    import torch
-    from paper_2211_17192_b200 import workloads
-    g = torch.Generator(device=device)
-    g.manual_seed(int(seed))
-    out = {}
-    for name, shape, kind in workloads.tensor_shapes(cfg):
-        if kind == "gain":
-            out[name] = torch.ones(shape, device=device)
-            continue
-        std = cfg["head_std"] if kind == "head" else cfg["bias_std"] if kind == "bias" else workloads.INIT_STD
-        t = torch.randn(shape, device=device, generator=g, dtype=torch.float32) * std
-        out[name] = t.to(torch.bfloat16) if cfg["dtype"] == "bf16" and kind != "bias" else t
-    return out
-
-
-def decode_stream(name):
-    """Whether a tensor is streamed by a decoder pass (encoder-decoder models: not the
-    encoder stack, nor the projections of the encoder output, which run once per source)."""
-    return not (name.startswith("enc.") or name.endswith(("wkv_x", "rel_bias")))
-
-
-def weight_stream_bytes(cfg):
-    """Bytes of one pass over the model: every block matrix and the LM head once."""
-    from paper_2211_17192_b200 import workloads
-    elem = 2 if cfg["dtype"] == "bf16" else 4
-    total = 0
-    for name, shape, kind in workloads.tensor_shapes(cfg):
-        if kind == "gain" or name in ("pos_emb",) or (name == "tok_emb" and not cfg["tied"]) or not decode_stream(name):
-            continue
-        total += int(np.prod(shape)) * elem
-    return total
-
-
-class GenerationWorkload:
-    dtype = "bf16"
-
-    def __init__(self, name, target, draft, batch, prompt_len, n_new, gamma, temperature=1.0, layers=None):
-        from paper_2211_17192_b200 import workloads
-        self.name, self.target_name, self.draft_name = name, target, draft
-        self.layers = layers
-        self.tcfg, self.dcfg = workloads.model_config(target), workloads.model_config(draft)  # (prepare applies --layers)
-        self.batch, self.prompt_len, self.n_new, self.gamma, self.temperature = batch, prompt_len, n_new, gamma, temperature
-
-    def description(self):
-        return {"workload": self.name, "target": self.target_name, "draft": self.draft_name, "batch": self.batch,
-                "prompt_len": self.prompt_len, "n_new": self.n_new, "gamma": self.gamma,
-                "temperature": self.temperature, "kv_dtype": "fp32",
-                **({"target_layers_override": self.layers} if self.layers else {}),
-                "l2": "one pass streams the target's weights (>> 126 MB L2) from HBM",
-                "parallelism": "replicas"}
-
-    def prepare(self, rank, device, iterations):
-        import torch
-        from paper_2211_17192_b200 import binding, workloads
-        self.torch, self.binding, self.device = torch, binding, device
-        self.tcfg = workloads.model_config(self.target_name)
-        if self.layers:
-            self.tcfg = workloads.scaled_config(self.tcfg, n_layers=self.layers)
-        self.dcfg = workloads.model_config(self.draft_name)
-        self.dtype = "bf16" if self.tcfg["dtype"] == "bf16" else "f32"
-        self.tw = gpu_weights(self.tcfg, 100 + rank, device)
-        self.dw = gpu_weights(self.dcfg, 200 + rank, device)
-        grow = max(self.n_new, iterations * (self.gamma + 1) + 64)
-        self.max_len = self.prompt_len + grow + self.gamma + 2
-        self.engine = binding.Engine(self.tcfg, self.tw, self.dcfg, self.dw, max_batch=self.batch, max_len=self.max_len,
-                                     page_size=64, max_gamma=max(self.gamma, 1))
-        self.prompts = [workloads.make_prompt(1000 * rank + b, self.prompt_len, self.tcfg["vocab"]) for b in range(self.batch)]
-        self.budget_tokens = grow
-
-    def launches_per_iteration(self):
-        fwd = lambda cfg: 1 + 10 * cfg["n_layers"] + 3
-        return 1 + self.gamma * (1 + fwd(self.dcfg) + 1) + 1 + fwd(self.tcfg) + 2 + 1
-
-    def timed_decode(self, warmup, steps, gamma):
-        """Device time of `steps` iterations after `warmup` untimed ones (prompt pass untimed)."""
-        self.engine.begin(self.prompts, self.budget_tokens, gamma, self.temperature, 7)
-        _, before = self.engine.step(warmup)
-        _, after = self.engine.step(steps)
-        tokens = after["tokens"] - before["tokens"]
-        stats = {k: after[k] - before[k] for k in ("iterations", "tokens", "tests_evaluated", "tests_passed")}
-        return tokens, after["decode_ms"], stats
-
-    def e2e(self, calls):
-        """The public call with host buffers: prompts in, tokens out, prompt pass included."""
-        t0 = time.perf_counter()
-        tokens = 0
-        for i in range(calls):
-            out, _ = self.engine.generate(self.prompts, self.n_new, self.gamma, self.temperature, 11 + i)
-            tokens += out.size
-        return tokens, time.perf_counter() - t0
-
-    def e2e_bytes(self):
-        return self.batch * self.prompt_len * 4 + self.batch * 4, self.batch * self.n_new * 4
-
-    def pass_times(self, repeats=20):
-        """Device time of single passes (graph-replayed, events on the library's stream):
-        the target on 1 and on gamma+1 rows, the draft on 1 row, at the prompt's context length."""
-        eng, torch = self.engine, self.torch
-        tok = np.stack([p[: self.prompt_len - 1] for p in self.prompts])
-        def timed(which, rows):
-            return eng.time_forward(which, self.batch, rows, repeats)
-        eng.reset()
-        chunk = 64
-        for which in (0, 1):
-            for c0 in range(0, tok.shape[1], chunk):
-                eng.forward_logits(which, tok[:, c0:c0 + chunk])
-        return {"target_1row_ms": timed(0, 1), "target_rows_ms": timed(0, self.gamma + 1), "draft_1row_ms": timed(1, 1)}
-
-    def gemm_roofline(self, rows):
-        """The weight-streaming GEMM alone: every block matrix and the head of the
-        target once through spec_linear at `rows` rows, captured in a CUDA graph and
-        timed with events on its stream."""
-        torch, binding = self.torch, self.binding
-        mats = [(n, t) for n, t in self.tw.items() if t.dim() == 2 and n not in ("tok_emb", "pos_emb") and decode_stream(n)]
-        if self.tcfg["tied"]:
-            mats.append(("head", self.tw["tok_emb"]))
-        kmax = max(t.shape[1] for _, t in mats)
-        x = torch.randn(rows, kmax, device=self.device)
-        ys = {n: torch.empty(rows, t.shape[0], device=self.device) for n, t in mats}
-        need = max(binding.spec_linear_workspace_bytes(rows, t.shape[0], t.shape[1]) for _, t in mats)
-        ws = torch.empty(need, dtype=torch.uint8, device=self.device)
-        xs = {k: x[:, :k].contiguous() for k in {t.shape[1] for _, t in mats}}
-        stream = torch.cuda.Stream(self.device)
-        with torch.cuda.stream(stream):
-            def sweep():
-                for n, t in mats:
-                    binding.spec_linear(xs[t.shape[1]], t, "auto", ys[n], ws)
-            sweep()
-            stream.synchronize()
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=stream):
-                sweep()
-            graph.replay()
-            stream.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            graph.replay()
-            b.record(stream)
-            stream.synchronize()
-        nbytes = sum(t.numel() * t.element_size() for _, t in mats)
-        return nbytes, a.elapsed_time(b), len(mats)
 
     def cpu_sample(self, budget_s):
         """The oracle on a bounded sample: both models at full width and reduced depth

@@ -20,6 +20,7 @@
 // query; attention_combine_kernel merges the key slices and emits the
 // out-projection's input (fp32 and/or split into two bf16 terms).
 #include <cfloat>
+#include <cstdlib>
 
 #include "model.cuh"
 
@@ -244,6 +245,281 @@ attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __r
     }
 }
 
+// ---- the same attention on the tensor cores, for many queries per KV head ----
+//
+// With grouped query heads, several new rows per sequence and a batch of
+// sequences, the kernel above re-reads every K,V tile from L1 once per query.
+// Here the (up to 16) queries that share a KV head form the M side of
+// mma.sync.m16n8k8 (tf32, fp32 accumulate): a warp stages a 32-key tile of K and
+// of V in shared memory once (cp.async, both in flight together), computes
+// S = Q K^T for all queries, keeps the online softmax in the accumulator layout
+// (a row's maximum and sum live in a quad of lanes), and accumulates O += P V.
+// The warps of a CTA take the tiles of its key slice in turn and merge their
+// states at the end; the partial state per (row, head, slice) has the same
+// format as above, so attention_combine_kernel serves both.
+constexpr int kMmaWarps = 4;
+
+__device__ __forceinline__ uint32_t to_tf32(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid) {
+    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(dst));
+    const int bytes = valid ? 16 : 0;  // 0: the 16 bytes are zero-filled
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// A 32-key tile of one KV head ([key][DH] in the pool) into shared memory rows of
+// DH + 4 floats; keys at or beyond n_valid become zeros.
+template <int DH>
+__device__ __forceinline__ void stage_tile(const float* tile, int n_valid, float* dst, int lane) {
+    constexpr int kChunks = DH / 4;
+    for (int i = lane; i < 32 * kChunks; i += 32) {
+        const int row = i / kChunks, c = i % kChunks;
+        const bool valid = row < n_valid;
+        cp_async16(dst + row * (DH + 4) + 4 * c, tile + static_cast<size_t>(valid ? row : 0) * DH + 4 * c, valid);
+    }
+}
+template <int DH>
+__device__ __forceinline__ void stage_tile(const __nv_bfloat16* tile, int n_valid, float* dst, int lane) {
+    constexpr int kChunks = DH / 8;
+    for (int i = lane; i < 32 * kChunks; i += 32) {
+        const int row = i / kChunks, c = i % kChunks;
+        float v[8];
+        if (row < n_valid) {
+            KvLoad<__nv_bfloat16>::load(tile + static_cast<size_t>(row) * DH + 8 * c, v);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) v[e] = 0.0f;
+        }
+        float* d = dst + row * (DH + 4) + 8 * c;
+        *reinterpret_cast<float4*>(d) = make_float4(v[0], v[1], v[2], v[3]);
+        *reinterpret_cast<float4*>(d + 4) = make_float4(v[4], v[5], v[6], v[7]);
+    }
+}
+
+template <int DH>
+struct MmaSmem {
+    static constexpr int kRow = DH + 4;              // floats per staged row (bank-conflict-free fragments)
+    static constexpr int kQ = 16 * kRow;             // the queries, scaled and rounded to tf32
+    static constexpr int kTile = 32 * kRow;          // one staged K or V tile
+    static constexpr int kP = 16 * 36;               // probabilities of one tile
+    static constexpr int kPerWarp = 2 * kTile + kP;
+    static constexpr size_t kBytes = static_cast<size_t>(kQ + kMmaWarps * kPerWarp) * sizeof(float);
+};
+
+// grid = (slices, n_kv_heads * m_blocks, batch), block = 32 * kMmaWarps.
+template <typename KV, int DH>
+__global__ void __launch_bounds__(32 * kMmaWarps)
+attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __restrict__ pos,
+                     const int32_t* __restrict__ seq, int m_rows, int n_heads, int n_kv_heads, int m_blocks,
+                     const KV* __restrict__ kv_layer, const int32_t* __restrict__ page_table, int pages_per_seq,
+                     int page_size, const int32_t* __restrict__ kv_len, const float* __restrict__ bias, int bias_span,
+                     int bias_zero, float scale, float* __restrict__ part) {
+    using S = MmaSmem<DH>;
+    extern __shared__ __align__(16) float smem_f[];
+    __shared__ int q_pos[16], q_row[16], q_head[16];
+    pdl_trigger();
+    pdl_wait();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int slice = blockIdx.x, slices = gridDim.x, b = blockIdx.z;
+    const int kv_head = blockIdx.y / m_blocks, mb = blockIdx.y % m_blocks;
+    const int group = n_heads / n_kv_heads;
+    const int queries = group * m_rows;
+    float* Qs = smem_f;
+    float* Kt = smem_f + S::kQ + warp * S::kPerWarp;
+    float* Vt = Kt + S::kTile;
+    float* Ps = Vt + S::kTile;
+
+    if (tid < 16) {
+        const int q = mb * 16 + tid;
+        const bool live = q < queries;
+        const int j = live ? q / group : 0;
+        q_row[tid] = b * m_rows + j;
+        q_head[tid] = kv_head * group + (live ? q % group : 0);
+        q_pos[tid] = live ? pos[b * m_rows + j] : -1;
+    }
+    __syncthreads();
+    for (int i = tid; i < 16 * DH; i += 32 * kMmaWarps) {
+        const int qi = i / DH, e = i % DH;
+        const float v = q_pos[qi] >= 0 ? qkv[static_cast<size_t>(q_row[qi]) * q_stride + q_head[qi] * DH + e] * scale : 0.0f;
+        Qs[qi * S::kRow + e] = __uint_as_float(to_tf32(v));
+    }
+    int seq_keys = 0;
+    if (kv_len) {
+        seq_keys = kv_len[seq[b * m_rows]];
+    } else {
+        for (int j = 0; j < m_rows; ++j) seq_keys = max(seq_keys, pos[b * m_rows + j] + 1);
+    }
+    const int tiles = (seq_keys + 31) / 32;
+    const int t0 = static_cast<int>(static_cast<long long>(tiles) * slice / slices);
+    const int t1 = static_cast<int>(static_cast<long long>(tiles) * (slice + 1) / slices);
+    const size_t head_stride = static_cast<size_t>(page_size) * DH;
+    const size_t page_stride = 2 * static_cast<size_t>(n_kv_heads) * head_stride;
+    const size_t v_offset = static_cast<size_t>(n_kv_heads) * head_stride;
+    const int32_t* pages = page_table + seq[b * m_rows] * pages_per_seq;
+    __syncthreads();
+
+    // the two query rows of this lane: g and g + 8
+    const int p_lo = q_pos[g], p_hi = q_pos[g + 8];
+    const int keys_lo = p_lo < 0 ? 0 : kv_len ? seq_keys : p_lo + 1;
+    const int keys_hi = p_hi < 0 ? 0 : kv_len ? seq_keys : p_hi + 1;
+    const float* bias_lo = bias ? bias + static_cast<size_t>(q_head[g]) * bias_span + (bias_zero - p_lo) : nullptr;
+    const float* bias_hi = bias ? bias + static_cast<size_t>(q_head[g + 8]) * bias_span + (bias_zero - p_hi) : nullptr;
+    float m_lo = -FLT_MAX, m_hi = -FLT_MAX, l_lo = 0.0f, l_hi = 0.0f;
+    float o[DH / 8][4];
+#pragma unroll
+    for (int n = 0; n < DH / 8; ++n)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[n][i] = 0.0f;
+
+    for (int tile_i = t0 + warp; tile_i < t1; tile_i += kMmaWarps) {
+        const int k0 = 32 * tile_i;
+        const KV* tile = kv_layer + pages[k0 / page_size] * page_stride + kv_head * head_stride +
+                         static_cast<size_t>(k0 % page_size) * DH;
+        const int n_valid = min(32, seq_keys - k0);
+        stage_tile<DH>(tile, n_valid, Kt, lane);
+        cp_async_commit();
+        stage_tile<DH>(tile + v_offset, n_valid, Vt, lane);
+        cp_async_commit();
+        cp_async_wait<1>();  // K has landed (V may still be in flight)
+        __syncwarp();
+
+        // S = Q K^T: four blocks of 8 keys
+        float s[4][4];
+#pragma unroll
+        for (int nb = 0; nb < 4; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) s[nb][i] = 0.0f;
+#pragma unroll 4
+        for (int ks = 0; ks < DH / 8; ++ks) {
+            uint32_t a[4];
+            a[0] = __float_as_uint(Qs[g * S::kRow + ks * 8 + t]);
+            a[1] = __float_as_uint(Qs[(g + 8) * S::kRow + ks * 8 + t]);
+            a[2] = __float_as_uint(Qs[g * S::kRow + ks * 8 + t + 4]);
+            a[3] = __float_as_uint(Qs[(g + 8) * S::kRow + ks * 8 + t + 4]);
+#pragma unroll
+            for (int nb = 0; nb < 4; ++nb) {
+                const float* kr = Kt + (nb * 8 + g) * S::kRow + ks * 8 + t;
+                mma_tf32(s[nb], a, __float_as_uint(kr[0]), __float_as_uint(kr[4]));
+            }
+        }
+        // mask, bias, online softmax (rows g and g + 8; a row's 32 scores sit in its quad of lanes)
+        float tmax_lo = -FLT_MAX, tmax_hi = -FLT_MAX;
+#pragma unroll
+        for (int nb = 0; nb < 4; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int key = k0 + nb * 8 + 2 * t + (i & 1);
+                const bool hi_row = i >= 2;
+                const bool valid = key < (hi_row ? keys_hi : keys_lo);
+                float v = s[nb][i];
+                if (valid && bias) v += hi_row ? bias_hi[key] : bias_lo[key];
+                s[nb][i] = valid ? v : -FLT_MAX;
+                if (hi_row) tmax_hi = fmaxf(tmax_hi, s[nb][i]);
+                else tmax_lo = fmaxf(tmax_lo, s[nb][i]);
+            }
+        tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(kFullMask, tmax_lo, 1));
+        tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(kFullMask, tmax_lo, 2));
+        tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(kFullMask, tmax_hi, 1));
+        tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(kFullMask, tmax_hi, 2));
+        const float new_lo = fmaxf(m_lo, tmax_lo), new_hi = fmaxf(m_hi, tmax_hi);
+        const float r_lo = expf(m_lo - new_lo), r_hi = expf(m_hi - new_hi);
+        float sum_lo = 0.0f, sum_hi = 0.0f;
+#pragma unroll
+        for (int nb = 0; nb < 4; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const bool hi_row = i >= 2;
+                const float pv = s[nb][i] > -FLT_MAX ? expf(s[nb][i] - (hi_row ? new_hi : new_lo)) : 0.0f;
+                if (hi_row) sum_hi += pv;
+                else sum_lo += pv;
+                Ps[(hi_row ? g + 8 : g) * 36 + nb * 8 + 2 * t + (i & 1)] = __uint_as_float(to_tf32(pv));
+            }
+        sum_lo += __shfl_xor_sync(kFullMask, sum_lo, 1);
+        sum_lo += __shfl_xor_sync(kFullMask, sum_lo, 2);
+        sum_hi += __shfl_xor_sync(kFullMask, sum_hi, 1);
+        sum_hi += __shfl_xor_sync(kFullMask, sum_hi, 2);
+        l_lo = l_lo * r_lo + sum_lo;
+        l_hi = l_hi * r_hi + sum_hi;
+        m_lo = new_lo;
+        m_hi = new_hi;
+        cp_async_wait<0>();  // V has landed
+        __syncwarp();        // ... and every lane's probabilities are in shared memory
+
+        // O = O * rescale + P V
+        uint32_t pa[4][4];
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+            pa[ks][0] = __float_as_uint(Ps[g * 36 + ks * 8 + t]);
+            pa[ks][1] = __float_as_uint(Ps[(g + 8) * 36 + ks * 8 + t]);
+            pa[ks][2] = __float_as_uint(Ps[g * 36 + ks * 8 + t + 4]);
+            pa[ks][3] = __float_as_uint(Ps[(g + 8) * 36 + ks * 8 + t + 4]);
+        }
+#pragma unroll
+        for (int n = 0; n < DH / 8; ++n) {
+            o[n][0] *= r_lo; o[n][1] *= r_lo; o[n][2] *= r_hi; o[n][3] *= r_hi;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                const float* vr = Vt + (ks * 8 + t) * S::kRow + n * 8 + g;
+                mma_tf32(o[n], pa[ks], __float_as_uint(vr[0]), __float_as_uint(vr[4 * S::kRow]));
+            }
+        }
+        __syncwarp();  // the tile buffers are free for the next tile
+    }
+
+    // park this warp's state in its own tile buffer: [query][max, sum, O[DH]]
+    __syncthreads();
+    float* st = Kt;  // 16 * (DH + 2) floats <= one tile
+#pragma unroll
+    for (int n = 0; n < DH / 8; ++n) {
+        st[g * (DH + 2) + 2 + n * 8 + 2 * t] = o[n][0];
+        st[g * (DH + 2) + 2 + n * 8 + 2 * t + 1] = o[n][1];
+        st[(g + 8) * (DH + 2) + 2 + n * 8 + 2 * t] = o[n][2];
+        st[(g + 8) * (DH + 2) + 2 + n * 8 + 2 * t + 1] = o[n][3];
+    }
+    if (t == 0) {
+        st[g * (DH + 2)] = m_lo;
+        st[g * (DH + 2) + 1] = l_lo;
+        st[(g + 8) * (DH + 2)] = m_hi;
+        st[(g + 8) * (DH + 2) + 1] = l_hi;
+    }
+    __syncthreads();
+    // merge the warps (in warp order) and write the slice's partial state of every live query
+    for (int i = tid; i < 16 * (DH + 2); i += 32 * kMmaWarps) {
+        const int qi = i / (DH + 2), e = i % (DH + 2);
+        if (mb * 16 + qi >= queries) continue;
+        float mm = -FLT_MAX;
+#pragma unroll
+        for (int w = 0; w < kMmaWarps; ++w) mm = fmaxf(mm, smem_f[S::kQ + w * S::kPerWarp + qi * (DH + 2)]);
+        float out;
+        if (e == 0) {
+            out = mm;
+        } else {
+            out = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kMmaWarps; ++w) {
+                const float* sw = smem_f + S::kQ + w * S::kPerWarp + qi * (DH + 2);
+                out += sw[e] * expf(sw[0] - mm);
+            }
+        }
+        part[((static_cast<size_t>(q_row[qi]) * n_heads + q_head[qi]) * slices + slice) * (DH + 2) + e] = out;
+    }
+}
+
 // grid = rows * n_heads, block = DH: merge the key slices of one (row, head).
 template <int DH>
 __global__ void attention_combine_kernel(const float* __restrict__ part, int slices, float* __restrict__ att,
@@ -286,14 +562,32 @@ int attention_sub_slices(int queries) {
     return queries * 2 <= kMaxAttnWarps ? kMaxAttnWarps / queries : 1;
 }
 
-int attention_slices(int batch, int n_kv_heads, int queries, int max_len) {
+// The tensor-core kernel serves bf16 models (its tf32 products stay far inside
+// their 2e-2 logit bar, not inside the 1e-4 bar of fp32 models) once a KV head
+// has enough queries to fill a good part of a 16-row block.
+bool attention_uses_mma(const Model& m, int m_rows) {
+    static const bool disabled = [] { const char* e = std::getenv("SPEC_NO_MMA_ATTENTION"); return e && e[0] == '1'; }();
+    return !disabled && m.bf16() && (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows >= 5;  // below that the warp-per-query kernel wins
+}
+
+int attention_slices(const Model& m, int batch, int m_rows, int max_len) {
+    const int n_kv_heads = m.cfg.n_kv_heads;
+    const int queries = (m.cfg.n_heads / n_kv_heads) * m_rows;
+    const int tiles = (max_len + 31) / 32;
+    if (attention_uses_mma(m, m_rows)) {
+        // one wave of CTAs (shared memory allows one per SM at d_head 128, two at 64); a tile per warp at least
+        const int m_blocks = (queries + 15) / 16;
+        const int resident = 148 * (m.cfg.d_head == 64 ? 2 : 1);
+        const int want = std::max(1, resident / (batch * n_kv_heads * m_blocks));
+        const int most = std::max(1, (tiles + kMmaWarps - 1) / kMmaWarps);
+        return std::max(1, std::min(std::min(want, most), 32));
+    }
     const int ks = attention_sub_slices(queries);
     // CTAs that fit the GPU at once: the kernel holds 128 registers per thread, so an
     // SM takes 16 warps of it; one wave of CTAs beats more, thinner slices
     const int warps = std::min(kMaxAttnWarps, std::max(1, queries * ks));
     const int resident = 148 * std::max(1, 16 / warps);
     const int want = std::max(1, resident / (batch * n_kv_heads));
-    const int tiles = (max_len + 31) / 32;
     const int most = std::max(1, (tiles + ks - 1) / ks);
     return std::max(1, std::min(std::min(want, most), 32));
 }
@@ -310,6 +604,35 @@ int launch_attention(const Model& m, const AttnSource& src, const RowMeta& rows,
     const dim3 grid(slices, m.cfg.n_kv_heads, batch);
     const float scale = 1.0f / sqrtf(static_cast<float>(m.cfg.d_head));
     const int n_rows = batch * m_rows;
+    if (attention_uses_mma(m, m_rows)) {
+        const int m_blocks = (group * m_rows + 15) / 16;
+        const dim3 mma_grid(slices, m.cfg.n_kv_heads * m_blocks, batch);
+#define SPEC_ATTN_MMA(KV, DH)                                                                                       \
+    do {                                                                                                            \
+        static bool configured = false;                                                                             \
+        if (!configured) {                                                                                          \
+            SPEC_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<KV, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                               static_cast<int>(MmaSmem<DH>::kBytes)));                            \
+            configured = true;                                                                                      \
+        }                                                                                                           \
+        int status = launch_pdl(attention_mma_kernel<KV, DH>, mma_grid, dim3(32 * kMmaWarps), MmaSmem<DH>::kBytes,  \
+                                stream, src.q, src.q_stride, rows.pos, rows.seq, m_rows, m.cfg.n_heads,            \
+                                m.cfg.n_kv_heads, m_blocks, static_cast<const KV*>(src.pool.kv), src.pool.page_table, \
+                                src.pool.pages_per_seq, src.pool.page_size, src.kv_len, src.bias, src.bias_span,    \
+                                src.bias_zero, scale, part);                                                        \
+        if (status != SPEC_OK) return status;                                                                       \
+        return launch_pdl(attention_combine_kernel<DH>, dim3(n_rows * m.cfg.n_heads), dim3(DH), 0, stream,           \
+                          static_cast<const float*>(part), slices, att, att_hi, att_lo);                            \
+    } while (0)
+        if (src.pool.elem_bytes == 2) {
+            if (m.cfg.d_head == 64) SPEC_ATTN_MMA(__nv_bfloat16, 64);
+            else SPEC_ATTN_MMA(__nv_bfloat16, 128);
+        } else {
+            if (m.cfg.d_head == 64) SPEC_ATTN_MMA(float, 64);
+            else SPEC_ATTN_MMA(float, 128);
+        }
+#undef SPEC_ATTN_MMA
+    }
 #define SPEC_ATTN(KV, DH)                                                                                         \
     do {                                                                                                          \
         int status = launch_pdl(attention_kernel<KV, DH>, grid, dim3(32 * warps), 0, stream, src.q, src.q_stride, \

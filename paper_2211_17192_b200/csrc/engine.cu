@@ -169,7 +169,7 @@ struct Pass {
         SPEC_TRY(proj(w.wqkv, pw.wqkv, m.qkv_dim(), c.d_model, ctx->a, ctx->qkv));
         SPEC_TRY(launch_qkv(c.n_heads, c.n_kv_heads, c.d_head, c.arch == SPEC_ARCH_LLAMA ? m.rope_table : nullptr, pool, rows,
                             n_rows, ctx->qkv, partials(), last_splits, st));
-        const int slices = attention_slices(batch, c.n_kv_heads, (c.n_heads / c.n_kv_heads) * m_rows, max_keys);
+        const int slices = attention_slices(m, batch, m_rows, max_keys);
         const AttnSource src{ctx->qkv, m.qkv_dim(), pool, kv_len, bias, bias_span, bias_zero};
         SPEC_TRY(launch_attention(m, src, rows, batch, m_rows, slices, ctx->attn_part, tc ? nullptr : ctx->att,
                                   tc ? hi() : nullptr, tc ? lo() : nullptr, st));
@@ -212,7 +212,7 @@ int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_ro
                 SPEC_TRY(launch_qkv(c.n_heads, 0, c.d_head, nullptr, KvPool{}, rows, n_rows, ctx->qkv, ctx->partials,
                                     pass.last_splits, ctx->stream));
             const KvPool pool = source_pool(ctx, m, static_cast<char*>(m.cross_kv) + static_cast<size_t>(l) * m.cross_stride);
-            const int slices = attention_slices(batch, c.n_kv_heads, m_rows, ctx->rt.max_src_len);
+            const int slices = attention_slices(m, batch, m_rows, ctx->rt.max_src_len);
             const AttnSource src{ctx->qkv, m.q_dim(), pool, ctx->src_len, nullptr, 0, 0};
             SPEC_TRY(launch_attention(m, src, rows, batch, m_rows, slices, ctx->attn_part, pass.tc ? nullptr : ctx->att,
                                       pass.tc ? pass.hi() : nullptr, pass.tc ? pass.lo() : nullptr, ctx->stream));
@@ -665,7 +665,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
                     for (int keys : {rt.max_len, rt.max_src_len})
                         if (keys > 0)
                             attn = std::max(attn, attention_partial_elems(b * mr, m.cfg.n_heads, m.cfg.d_head,
-                                                                          attention_slices(b, m.cfg.n_kv_heads, (m.cfg.n_heads / m.cfg.n_kv_heads) * mr, keys)));
+                                                                          attention_slices(m, b, mr, keys)));
         }
         SPEC_ALLOC(attn_part, attn);
     }

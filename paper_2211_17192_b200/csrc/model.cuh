@@ -126,7 +126,7 @@ struct AttnSource {
 
 // att[r, h] = softmax(scores) V for the rows of a pass; rows of sequence b are
 // rows b*m_rows .. of the pass.  Output as fp32 and/or two bf16 terms.
-int attention_slices(int batch, int n_kv_heads, int queries, int max_len);
+int attention_slices(const Model& m, int batch, int m_rows, int max_len);
 size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices);
 int launch_attention(const Model& m, const AttnSource& src, const RowMeta& rows, int batch, int m_rows, int slices,
                      float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo, cudaStream_t stream);
