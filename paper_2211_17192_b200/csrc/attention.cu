@@ -76,15 +76,85 @@ struct KvLoad<__nv_bfloat16> {
     }
 };
 
+// ---- merging the key slices inside a thread-block cluster ---------------------
+// The CTAs of one (sequence, KV head) - one per key slice - are launched as a
+// cluster.  Each leaves the states of its queries, [query][max, sum, O[DH]], in
+// its own shared memory; after a cluster barrier the CTAs share out the queries,
+// read the slices' states through distributed shared memory, merge them in
+// slice order and write the attention output.  No partial state goes through
+// global memory and no second kernel is needed.
+struct AttnOut {
+    float* att;             // fp32 [rows][n_heads * DH] or nullptr
+    __nv_bfloat16 *hi, *lo;  // the same as two bf16 terms, or nullptr
+};
+
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ld_peer_f32(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    float v;
+    asm("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote));
+    return v;
+}
+
+constexpr int kMaxClusterSlices = 8;  // portable cluster size; larger clusters of these fat CTAs schedule too slowly
+
+// `fin`: this CTA's states of queries q_base .. q_base + n_q - 1 of the (sequence b,
+// KV head) group; query q is row b * m_rows + q / group, head kv_head * group + q % group.
+template <int DH>
+__device__ __forceinline__ void cluster_merge_write(const float* fin, int n_q, int q_base, int queries, int b, int m_rows,
+                                                    int group, int kv_head, int n_heads, int slices, const AttnOut& out) {
+    cluster_arrive();
+    cluster_wait();  // every slice's states are in place
+    const uint32_t base = static_cast<uint32_t>(__cvta_generic_to_shared(fin));
+    const int rank = blockIdx.x;  // the cluster spans the slice dimension of the grid
+    for (int qi = rank; qi < n_q && q_base + qi < queries; qi += slices) {
+        const int q = q_base + qi;
+        const size_t at = (static_cast<size_t>(b * m_rows + q / group) * n_heads + kv_head * group + q % group) * DH;
+        const uint32_t state = base + static_cast<uint32_t>(qi * (DH + 2) * 4);
+        for (int e = threadIdx.x; e < DH; e += blockDim.x) {
+            float ms[kMaxClusterSlices], ls[kMaxClusterSlices], os[kMaxClusterSlices];
+#pragma unroll
+            for (int s = 0; s < kMaxClusterSlices; ++s) {
+                ms[s] = s < slices ? ld_peer_f32(state, s) : -FLT_MAX;
+                ls[s] = s < slices ? ld_peer_f32(state + 4, s) : 0.0f;
+                os[s] = s < slices ? ld_peer_f32(state + 8 + 4 * e, s) : 0.0f;
+            }
+            float mm = -FLT_MAX;
+#pragma unroll
+            for (int s = 0; s < kMaxClusterSlices; ++s) mm = fmaxf(mm, ms[s]);
+            float l = 0.0f, o = 0.0f;
+#pragma unroll
+            for (int s = 0; s < kMaxClusterSlices; ++s) {  // slices in index order
+                const float w = s < slices ? expf(ms[s] - mm) : 0.0f;
+                l += ls[s] * w;
+                o += os[s] * w;
+            }
+            const float y = l > 0.0f ? o / l : 0.0f;  // an inactive row has no keys
+            if (out.att) out.att[at + e] = y;
+            if (out.hi) {
+                const __nv_bfloat16 h = __float2bfloat16_rn(y);
+                out.hi[at + e] = h;
+                out.lo[at + e] = __float2bfloat16_rn(y - __bfloat162float(h));
+            }
+        }
+    }
+    cluster_arrive();
+    cluster_wait();  // nobody leaves while a peer may still read its shared memory
+}
+
 // grid = (slices, n_kv_heads, batch), block = 32 * warps (warps <= kMaxAttnWarps).
 // Rows of sequence b are rows b*m .. b*m+m-1 of the pass.
-template <typename KV, int DH>
+// FUSED (needs queries * ks <= kMaxAttnWarps, i.e. one round of work units): the
+// grid is launched as clusters over the slice dimension and writes `out` itself.
+template <typename KV, int DH, bool FUSED>
 __global__ void __launch_bounds__(32 * kMaxAttnWarps)
 attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __restrict__ pos,
                  const int32_t* __restrict__ seq, int m_rows, int n_heads, int n_kv_heads, int ks,
                  const KV* __restrict__ kv_layer, const int32_t* __restrict__ page_table, int pages_per_seq,
                  int page_size, const int32_t* __restrict__ kv_len, const float* __restrict__ bias, int bias_span,
-                 int bias_zero, float scale, float* __restrict__ part) {
+                 int bias_zero, float scale, float* __restrict__ part, const AttnOut out) {
     constexpr int PER_LANE = DH / 32;
     __shared__ float share[kMaxAttnWarps][DH + 2];  // states of the warps that share a query (ks > 1)
     pdl_trigger();
@@ -198,7 +268,7 @@ attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __r
                 }
             }
         }
-        if (ks > 1) {  // park the state; warp `q` merges the ks of them below
+        if (ks > 1 || FUSED) {  // park the state (ks > 1: warp `q` merges the ks of them below)
             if (lane == 0) {
                 share[warp][0] = mx;
                 share[warp][1] = l;
@@ -207,13 +277,13 @@ attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __r
             for (int i = 0; i < PER_LANE; ++i) share[warp][2 + lane * PER_LANE + i] = acc[i];
         } else {
             // partial state of (row r, head, slice): [max, sum, acc[DH]]
-            float* out = part + ((static_cast<size_t>(r) * n_heads + head) * slices + slice) * (DH + 2);
+            float* dst = part + ((static_cast<size_t>(r) * n_heads + head) * slices + slice) * (DH + 2);
             if (lane == 0) {
-                out[0] = mx;
-                out[1] = l;
+                dst[0] = mx;
+                dst[1] = l;
             }
 #pragma unroll
-            for (int i = 0; i < PER_LANE; ++i) out[2 + lane * PER_LANE + i] = acc[i];
+            for (int i = 0; i < PER_LANE; ++i) dst[2 + lane * PER_LANE + i] = acc[i];
         }
     }
     if (ks > 1) {
@@ -234,14 +304,20 @@ attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __r
 #pragma unroll
                 for (int i = 0; i < PER_LANE; ++i) acc[i] += st[2 + lane * PER_LANE + i] * w;
             }
-            float* out = part + ((static_cast<size_t>(r) * n_heads + head) * slices + slice) * (DH + 2);
+            // (warp q is the only reader of the rows it merged, so it may reuse row q)
+            float* dst = FUSED ? share[q] : part + ((static_cast<size_t>(r) * n_heads + head) * slices + slice) * (DH + 2);
+            __syncwarp();
             if (lane == 0) {
-                out[0] = mm;
-                out[1] = l;
+                dst[0] = mm;
+                dst[1] = l;
             }
 #pragma unroll
-            for (int i = 0; i < PER_LANE; ++i) out[2 + lane * PER_LANE + i] = acc[i];
+            for (int i = 0; i < PER_LANE; ++i) dst[2 + lane * PER_LANE + i] = acc[i];
         }
+    }
+    if (FUSED) {
+        __syncthreads();
+        cluster_merge_write<DH>(&share[0][0], queries, 0, queries, b, m_rows, group, kv_head, n_heads, slices, out);
     }
 }
 
@@ -321,13 +397,13 @@ struct MmaSmem {
 };
 
 // grid = (slices, n_kv_heads * m_blocks, batch), block = 32 * kMmaWarps.
-template <typename KV, int DH>
+template <typename KV, int DH, bool FUSED>
 __global__ void __launch_bounds__(32 * kMmaWarps)
 attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __restrict__ pos,
                      const int32_t* __restrict__ seq, int m_rows, int n_heads, int n_kv_heads, int m_blocks,
                      const KV* __restrict__ kv_layer, const int32_t* __restrict__ page_table, int pages_per_seq,
                      int page_size, const int32_t* __restrict__ kv_len, const float* __restrict__ bias, int bias_span,
-                     int bias_zero, float scale, float* __restrict__ part) {
+                     int bias_zero, float scale, float* __restrict__ part, const AttnOut out) {
     using S = MmaSmem<DH>;
     extern __shared__ __align__(16) float smem_f[];
     __shared__ int q_pos[16], q_row[16], q_head[16];
@@ -499,24 +575,30 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     }
     __syncthreads();
     // merge the warps (in warp order) and write the slice's partial state of every live query
+    // (fused: into the queries' buffer, which nobody needs any more, for the cluster merge)
     for (int i = tid; i < 16 * (DH + 2); i += 32 * kMmaWarps) {
         const int qi = i / (DH + 2), e = i % (DH + 2);
         if (mb * 16 + qi >= queries) continue;
         float mm = -FLT_MAX;
 #pragma unroll
         for (int w = 0; w < kMmaWarps; ++w) mm = fmaxf(mm, smem_f[S::kQ + w * S::kPerWarp + qi * (DH + 2)]);
-        float out;
+        float merged;
         if (e == 0) {
-            out = mm;
+            merged = mm;
         } else {
-            out = 0.0f;
+            merged = 0.0f;
 #pragma unroll
             for (int w = 0; w < kMmaWarps; ++w) {
                 const float* sw = smem_f + S::kQ + w * S::kPerWarp + qi * (DH + 2);
-                out += sw[e] * expf(sw[0] - mm);
+                merged += sw[e] * expf(sw[0] - mm);
             }
         }
-        part[((static_cast<size_t>(q_row[qi]) * n_heads + q_head[qi]) * slices + slice) * (DH + 2) + e] = out;
+        if (FUSED) Qs[i] = merged;
+        else part[((static_cast<size_t>(q_row[qi]) * n_heads + q_head[qi]) * slices + slice) * (DH + 2) + e] = merged;
+    }
+    if (FUSED) {
+        __syncthreads();
+        cluster_merge_write<DH>(Qs, 16, mb * 16, queries, b, m_rows, group, kv_head, n_heads, slices, out);
     }
 }
 
@@ -570,7 +652,19 @@ bool attention_uses_mma(const Model& m, int m_rows) {
     return !disabled && m.bf16() && (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows >= 5;  // below that the warp-per-query kernel wins
 }
 
+// The key slices can be merged inside a cluster (no second kernel) whenever a CTA
+// holds all its queries' states at once: always on the tensor-core path, and on
+// the warp-per-query path when the queries fit one round of warps.  It is done
+// when the slice count that balances the keys is at most 8: long contexts want
+// more slices than a cluster schedules well, and keep the separate combine kernel.
+bool attention_merges_in_cluster(const Model& m, int m_rows) {
+    static const bool disabled = [] { const char* e = std::getenv("SPEC_NO_CLUSTER_MERGE"); return e && e[0] == '1'; }();
+    if (disabled) return false;
+    return attention_uses_mma(m, m_rows) || (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows <= kMaxAttnWarps;
+}
+
 int attention_slices(const Model& m, int batch, int m_rows, int max_len) {
+    const int cap = 32;
     const int n_kv_heads = m.cfg.n_kv_heads;
     const int queries = (m.cfg.n_heads / n_kv_heads) * m_rows;
     const int tiles = (max_len + 31) / 32;
@@ -580,7 +674,7 @@ int attention_slices(const Model& m, int batch, int m_rows, int max_len) {
         const int resident = 148 * (m.cfg.d_head == 64 ? 2 : 1);
         const int want = std::max(1, resident / (batch * n_kv_heads * m_blocks));
         const int most = std::max(1, (tiles + kMmaWarps - 1) / kMmaWarps);
-        return std::max(1, std::min(std::min(want, most), 32));
+        return std::max(1, std::min(std::min(want, most), cap));
     }
     const int ks = attention_sub_slices(queries);
     // CTAs that fit the GPU at once: the kernel holds 128 registers per thread, so an
@@ -589,70 +683,104 @@ int attention_slices(const Model& m, int batch, int m_rows, int max_len) {
     const int resident = 148 * std::max(1, 16 / warps);
     const int want = std::max(1, resident / (batch * n_kv_heads));
     const int most = std::max(1, (tiles + ks - 1) / ks);
-    return std::max(1, std::min(std::min(want, most), 32));
+    return std::max(1, std::min(std::min(want, most), cap));
 }
 
 size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices) {
     return static_cast<size_t>(rows) * n_heads * slices * (d_head + 2);
 }
 
-int launch_attention(const Model& m, const AttnSource& src, const RowMeta& rows, int batch, int m_rows, int slices,
-                     float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo, cudaStream_t stream) {
+namespace {
+
+// A launch with programmatic stream serialization and, if cluster_x > 0, clusters of
+// cluster_x CTAs along x.
+template <typename... KArgs, typename... Args>
+int launch_attn(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, int cluster_x, cudaStream_t stream,
+                Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (cluster_x > 0) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = static_cast<unsigned>(cluster_x);
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    if (pdl_enabled()) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    if (err != cudaSuccess) return fail(SPEC_ERR_CUDA, "attention launch failed: %s", cudaGetErrorString(err));
+    return SPEC_OK;
+}
+
+template <typename KV, int DH>
+int launch_attention_variant(const Model& m, const AttnSource& src, const RowMeta& rows, int batch, int m_rows, int slices,
+                             float* part, const AttnOut& out, cudaStream_t stream) {
     const int group = m.cfg.n_heads / m.cfg.n_kv_heads;
-    const int ks = attention_sub_slices(group * m_rows);
-    const int warps = std::min(kMaxAttnWarps, std::max(1, group * m_rows * ks));
-    const dim3 grid(slices, m.cfg.n_kv_heads, batch);
+    const int queries = group * m_rows;
     const float scale = 1.0f / sqrtf(static_cast<float>(m.cfg.d_head));
     const int n_rows = batch * m_rows;
+    const bool fused = attention_merges_in_cluster(m, m_rows) && slices <= kMaxClusterSlices;
+    const KV* pool = static_cast<const KV*>(src.pool.kv);
+    int status;
     if (attention_uses_mma(m, m_rows)) {
-        const int m_blocks = (group * m_rows + 15) / 16;
-        const dim3 mma_grid(slices, m.cfg.n_kv_heads * m_blocks, batch);
-#define SPEC_ATTN_MMA(KV, DH)                                                                                       \
-    do {                                                                                                            \
-        static bool configured = false;                                                                             \
-        if (!configured) {                                                                                          \
-            SPEC_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<KV, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                               static_cast<int>(MmaSmem<DH>::kBytes)));                            \
-            configured = true;                                                                                      \
-        }                                                                                                           \
-        int status = launch_pdl(attention_mma_kernel<KV, DH>, mma_grid, dim3(32 * kMmaWarps), MmaSmem<DH>::kBytes,  \
-                                stream, src.q, src.q_stride, rows.pos, rows.seq, m_rows, m.cfg.n_heads,            \
-                                m.cfg.n_kv_heads, m_blocks, static_cast<const KV*>(src.pool.kv), src.pool.page_table, \
-                                src.pool.pages_per_seq, src.pool.page_size, src.kv_len, src.bias, src.bias_span,    \
-                                src.bias_zero, scale, part);                                                        \
-        if (status != SPEC_OK) return status;                                                                       \
-        return launch_pdl(attention_combine_kernel<DH>, dim3(n_rows * m.cfg.n_heads), dim3(DH), 0, stream,           \
-                          static_cast<const float*>(part), slices, att, att_hi, att_lo);                            \
-    } while (0)
-        if (src.pool.elem_bytes == 2) {
-            if (m.cfg.d_head == 64) SPEC_ATTN_MMA(__nv_bfloat16, 64);
-            else SPEC_ATTN_MMA(__nv_bfloat16, 128);
-        } else {
-            if (m.cfg.d_head == 64) SPEC_ATTN_MMA(float, 64);
-            else SPEC_ATTN_MMA(float, 128);
+        static bool configured = false;
+        if (!configured) {
+            SPEC_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<KV, DH, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               static_cast<int>(MmaSmem<DH>::kBytes)));
+            SPEC_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<KV, DH, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               static_cast<int>(MmaSmem<DH>::kBytes)));
+            configured = true;
         }
-#undef SPEC_ATTN_MMA
-    }
-#define SPEC_ATTN(KV, DH)                                                                                         \
-    do {                                                                                                          \
-        int status = launch_pdl(attention_kernel<KV, DH>, grid, dim3(32 * warps), 0, stream, src.q, src.q_stride, \
-                                rows.pos, rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads, ks,                  \
-                                static_cast<const KV*>(src.pool.kv), src.pool.page_table, src.pool.pages_per_seq,     \
-                                src.pool.page_size,                                                               \
-                                src.kv_len, src.bias, src.bias_span, src.bias_zero, scale, part);                 \
-        if (status != SPEC_OK) return status;                                                                     \
-        return launch_pdl(attention_combine_kernel<DH>, dim3(n_rows * m.cfg.n_heads), dim3(DH), 0, stream,         \
-                          static_cast<const float*>(part), slices, att, att_hi, att_lo);                          \
-    } while (0)
-    if (src.pool.elem_bytes == 2) {
-        if (m.cfg.d_head == 64) SPEC_ATTN(__nv_bfloat16, 64);
-        else SPEC_ATTN(__nv_bfloat16, 128);
+        const int m_blocks = (queries + 15) / 16;
+        const dim3 grid(slices, m.cfg.n_kv_heads * m_blocks, batch);
+        status = fused ? launch_attn(attention_mma_kernel<KV, DH, true>, grid, dim3(32 * kMmaWarps), MmaSmem<DH>::kBytes, slices,
+                                     stream, src.q, src.q_stride, rows.pos, rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads,
+                                     m_blocks, pool, src.pool.page_table, src.pool.pages_per_seq, src.pool.page_size, src.kv_len,
+                                     src.bias, src.bias_span, src.bias_zero, scale, part, out)
+                       : launch_attn(attention_mma_kernel<KV, DH, false>, grid, dim3(32 * kMmaWarps), MmaSmem<DH>::kBytes, 0,
+                                     stream, src.q, src.q_stride, rows.pos, rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads,
+                                     m_blocks, pool, src.pool.page_table, src.pool.pages_per_seq, src.pool.page_size, src.kv_len,
+                                     src.bias, src.bias_span, src.bias_zero, scale, part, out);
     } else {
-        if (m.cfg.d_head == 64) SPEC_ATTN(float, 64);
-        else SPEC_ATTN(float, 128);
+        const int ks = attention_sub_slices(queries);
+        const int warps = std::min(kMaxAttnWarps, std::max(1, queries * ks));
+        const dim3 grid(slices, m.cfg.n_kv_heads, batch);
+        status = fused ? launch_attn(attention_kernel<KV, DH, true>, grid, dim3(32 * warps), 0, slices, stream, src.q, src.q_stride,
+                                     rows.pos, rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads, ks, pool, src.pool.page_table,
+                                     src.pool.pages_per_seq, src.pool.page_size, src.kv_len, src.bias, src.bias_span,
+                                     src.bias_zero, scale, part, out)
+                       : launch_attn(attention_kernel<KV, DH, false>, grid, dim3(32 * warps), 0, 0, stream, src.q, src.q_stride,
+                                     rows.pos, rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads, ks, pool, src.pool.page_table,
+                                     src.pool.pages_per_seq, src.pool.page_size, src.kv_len, src.bias, src.bias_span,
+                                     src.bias_zero, scale, part, out);
     }
-#undef SPEC_ATTN
-    return SPEC_OK;
+    if (status != SPEC_OK || fused) return status;
+    return launch_pdl(attention_combine_kernel<DH>, dim3(n_rows * m.cfg.n_heads), dim3(DH), 0, stream,
+                      static_cast<const float*>(part), slices, out.att, out.hi, out.lo);
+}
+
+}  // namespace
+
+int launch_attention(const Model& m, const AttnSource& src, const RowMeta& rows, int batch, int m_rows, int slices,
+                     float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo, cudaStream_t stream) {
+    const AttnOut out{att, att_hi, att_lo};
+    if (src.pool.elem_bytes == 2) {
+        if (m.cfg.d_head == 64) return launch_attention_variant<__nv_bfloat16, 64>(m, src, rows, batch, m_rows, slices, part, out, stream);
+        return launch_attention_variant<__nv_bfloat16, 128>(m, src, rows, batch, m_rows, slices, part, out, stream);
+    }
+    if (m.cfg.d_head == 64) return launch_attention_variant<float, 64>(m, src, rows, batch, m_rows, slices, part, out, stream);
+    return launch_attention_variant<float, 128>(m, src, rows, batch, m_rows, slices, part, out, stream);
 }
 
 }  // namespace spec
