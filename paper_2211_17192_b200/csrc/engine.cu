@@ -619,7 +619,12 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     ctx->has_draft = draft_cfg != nullptr;
     ctx->pages_per_seq = (rt.max_len + rt.page_size - 1) / rt.page_size;
     ctx->max_logit_rows = std::max(rt.max_batch * std::max(rt.max_gamma + 1, 2), 64);
-    ctx->max_rows = ctx->max_logit_rows;
+    // The prompt pass takes up to 256 rows at a time (weights streamed once per chunk).
+    {
+        const char* e = std::getenv("SPEC_PREFILL_ROWS");
+        const int prefill_rows = e ? std::max(1, std::atoi(e)) : 256;
+        ctx->max_rows = std::max(ctx->max_logit_rows, std::min(prefill_rows, rt.max_batch * rt.max_len));
+    }
     if (t5) {  // an encoder pass takes every source row of the batch at once
         ctx->src_pages_per_seq = (rt.max_src_len + rt.page_size - 1) / rt.page_size;
         ctx->max_rows = std::max(ctx->max_rows, rt.max_batch * rt.max_src_len);
