@@ -326,14 +326,15 @@ attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __r
 // With grouped query heads, several new rows per sequence and a batch of
 // sequences, the kernel above re-reads every K,V tile from L1 once per query.
 // Here the (up to 16) queries that share a KV head form the M side of
-// mma.sync.m16n8k8 (tf32, fp32 accumulate): a warp stages a 32-key tile of K and
-// of V in shared memory once (cp.async, both in flight together), computes
-// S = Q K^T for all queries, keeps the online softmax in the accumulator layout
-// (a row's maximum and sum live in a quad of lanes), and accumulates O += P V.
-// The warps of a CTA take the tiles of its key slice in turn and merge their
-// states at the end; the partial state per (row, head, slice) has the same
+// mma.sync.m16n8k8 (tf32, fp32 accumulate): a warp stages 16-key tiles of K and
+// of V in shared memory once (cp.async, two tiles in flight: the next one loads
+// while this one is multiplied), computes S = Q K^T for all queries, keeps the
+// online softmax in the accumulator layout (a row's maximum and sum live in a
+// quad of lanes), and accumulates O += P V.  The warps of a CTA take the 32-key
+// blocks of its key slice in turn and merge their states at the end; the partial state per (row, head, slice) has the same
 // format as above, so attention_combine_kernel serves both.
-constexpr int kMmaWarps = 4;
+constexpr int kMmaWarps = 8;
+constexpr int kMmaStages = 1;  // staged tiles per warp (2: the next tile loads while this one is multiplied)
 
 __device__ __forceinline__ uint32_t to_tf32(float x) {
     uint32_t r;
@@ -357,12 +358,14 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// A 32-key tile of one KV head ([key][DH] in the pool) into shared memory rows of
+constexpr int kTileKeys = 16;  // keys per staged tile of the tensor-core kernel
+
+// A 16-key tile of one KV head ([key][DH] in the pool) into shared memory rows of
 // DH + 4 floats; keys at or beyond n_valid become zeros.
 template <int DH>
 __device__ __forceinline__ void stage_tile(const float* tile, int n_valid, float* dst, int lane) {
     constexpr int kChunks = DH / 4;
-    for (int i = lane; i < 32 * kChunks; i += 32) {
+    for (int i = lane; i < kTileKeys * kChunks; i += 32) {
         const int row = i / kChunks, c = i % kChunks;
         const bool valid = row < n_valid;
         cp_async16(dst + row * (DH + 4) + 4 * c, tile + static_cast<size_t>(valid ? row : 0) * DH + 4 * c, valid);
@@ -371,7 +374,7 @@ __device__ __forceinline__ void stage_tile(const float* tile, int n_valid, float
 template <int DH>
 __device__ __forceinline__ void stage_tile(const __nv_bfloat16* tile, int n_valid, float* dst, int lane) {
     constexpr int kChunks = DH / 8;
-    for (int i = lane; i < 32 * kChunks; i += 32) {
+    for (int i = lane; i < kTileKeys * kChunks; i += 32) {
         const int row = i / kChunks, c = i % kChunks;
         float v[8];
         if (row < n_valid) {
@@ -390,9 +393,11 @@ template <int DH>
 struct MmaSmem {
     static constexpr int kRow = DH + 4;              // floats per staged row (bank-conflict-free fragments)
     static constexpr int kQ = 16 * kRow;             // the queries, scaled and rounded to tf32
-    static constexpr int kTile = 32 * kRow;          // one staged K or V tile
-    static constexpr int kP = 16 * 36;               // probabilities of one tile
-    static constexpr int kPerWarp = 2 * kTile + kP;
+    static constexpr int kTile = kTileKeys * kRow;   // one staged K or V tile
+    static constexpr int kStage = 2 * kTile;         // K and V of one tile
+    static constexpr int kPStride = 20;              // floats per row of the probabilities (bank-conflict-free)
+    static constexpr int kP = 16 * kPStride;         // probabilities of one tile
+    static constexpr int kPerWarp = kMmaStages * kStage + kP;
     static constexpr size_t kBytes = static_cast<size_t>(kQ + kMmaWarps * kPerWarp) * sizeof(float);
 };
 
@@ -416,9 +421,8 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     const int group = n_heads / n_kv_heads;
     const int queries = group * m_rows;
     float* Qs = smem_f;
-    float* Kt = smem_f + S::kQ + warp * S::kPerWarp;
-    float* Vt = Kt + S::kTile;
-    float* Ps = Vt + S::kTile;
+    float* stage0 = smem_f + S::kQ + warp * S::kPerWarp;  // stage s: K tile, then V tile
+    float* Ps = stage0 + kMmaStages * S::kStage;
 
     if (tid < 16) {
         const int q = mb * 16 + tid;
@@ -462,104 +466,130 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 #pragma unroll
         for (int i = 0; i < 4; ++i) o[n][i] = 0.0f;
 
-    for (int tile_i = t0 + warp; tile_i < t1; tile_i += kMmaWarps) {
-        const int k0 = 32 * tile_i;
-        const KV* tile = kv_layer + pages[k0 / page_size] * page_stride + kv_head * head_stride +
-                         static_cast<size_t>(k0 % page_size) * DH;
-        const int n_valid = min(32, seq_keys - k0);
-        stage_tile<DH>(tile, n_valid, Kt, lane);
+    // This warp's tiles: the 16-key halves of the 32-key blocks t0 + warp, t0 + warp + 4, ...
+    const int my_blocks = t0 + warp < t1 ? (t1 - t0 - warp + kMmaWarps - 1) / kMmaWarps : 0;
+    const int my_tiles = 2 * my_blocks;
+    auto first_key = [&](int i) { return 32 * (t0 + warp + (i >> 1) * kMmaWarps) + 16 * (i & 1); };  // (kMmaWarps blocks apart)
+    auto issue = [&](int i) {  // tile i into stage i & 1 (an empty group if there is no such tile)
+        if (i < my_tiles) {
+            const int k0 = first_key(i);
+            const int n_valid = min(kTileKeys, seq_keys - k0);
+            if (n_valid > 0) {
+                const KV* tile = kv_layer + pages[k0 / page_size] * page_stride + kv_head * head_stride +
+                                 static_cast<size_t>(k0 % page_size) * DH;
+                float* st = stage0 + (i % kMmaStages) * S::kStage;
+                stage_tile<DH>(tile, n_valid, st, lane);
+                stage_tile<DH>(tile + v_offset, n_valid, st + S::kTile, lane);
+            }
+        }
         cp_async_commit();
-        stage_tile<DH>(tile + v_offset, n_valid, Vt, lane);
-        cp_async_commit();
-        cp_async_wait<1>();  // K has landed (V may still be in flight)
+    };
+#pragma unroll
+    for (int i = 0; i < kMmaStages; ++i) issue(i);
+    for (int i = 0; i < my_tiles; ++i) {
+        const int k0 = first_key(i);
+        cp_async_wait<kMmaStages - 1>();  // tile i has landed (later tiles may still be in flight)
         __syncwarp();
-
-        // S = Q K^T: four blocks of 8 keys
-        float s[4][4];
+        if (k0 < seq_keys) {
+            const float* Kt = stage0 + (i % kMmaStages) * S::kStage;
+            const float* Vt = Kt + S::kTile;
+            // S = Q K^T: two blocks of 8 keys; even and odd k-steps go to separate accumulators
+            // (four independent MMA chains instead of two), added at the end
+            float s[2][4], s_odd[2][4];
 #pragma unroll
-        for (int nb = 0; nb < 4; ++nb)
+            for (int nb = 0; nb < 2; ++nb)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) s[nb][i] = 0.0f;
+                for (int j = 0; j < 4; ++j) s[nb][j] = s_odd[nb][j] = 0.0f;
 #pragma unroll 4
-        for (int ks = 0; ks < DH / 8; ++ks) {
-            uint32_t a[4];
-            a[0] = __float_as_uint(Qs[g * S::kRow + ks * 8 + t]);
-            a[1] = __float_as_uint(Qs[(g + 8) * S::kRow + ks * 8 + t]);
-            a[2] = __float_as_uint(Qs[g * S::kRow + ks * 8 + t + 4]);
-            a[3] = __float_as_uint(Qs[(g + 8) * S::kRow + ks * 8 + t + 4]);
+            for (int ks = 0; ks < DH / 8; ks += 2) {
+                uint32_t a[2][4];
 #pragma unroll
-            for (int nb = 0; nb < 4; ++nb) {
-                const float* kr = Kt + (nb * 8 + g) * S::kRow + ks * 8 + t;
-                mma_tf32(s[nb], a, __float_as_uint(kr[0]), __float_as_uint(kr[4]));
+                for (int h = 0; h < 2; ++h) {
+                    a[h][0] = __float_as_uint(Qs[g * S::kRow + (ks + h) * 8 + t]);
+                    a[h][1] = __float_as_uint(Qs[(g + 8) * S::kRow + (ks + h) * 8 + t]);
+                    a[h][2] = __float_as_uint(Qs[g * S::kRow + (ks + h) * 8 + t + 4]);
+                    a[h][3] = __float_as_uint(Qs[(g + 8) * S::kRow + (ks + h) * 8 + t + 4]);
+                }
+#pragma unroll
+                for (int nb = 0; nb < 2; ++nb) {
+                    const float* kr = Kt + (nb * 8 + g) * S::kRow + ks * 8 + t;
+                    mma_tf32(s[nb], a[0], __float_as_uint(kr[0]), __float_as_uint(kr[4]));
+                    mma_tf32(s_odd[nb], a[1], __float_as_uint(kr[8]), __float_as_uint(kr[12]));
+                }
             }
-        }
-        // mask, bias, online softmax (rows g and g + 8; a row's 32 scores sit in its quad of lanes)
-        float tmax_lo = -FLT_MAX, tmax_hi = -FLT_MAX;
 #pragma unroll
-        for (int nb = 0; nb < 4; ++nb)
+            for (int nb = 0; nb < 2; ++nb)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int key = k0 + nb * 8 + 2 * t + (i & 1);
-                const bool hi_row = i >= 2;
-                const bool valid = key < (hi_row ? keys_hi : keys_lo);
-                float v = s[nb][i];
-                if (valid && bias) v += hi_row ? bias_hi[key] : bias_lo[key];
-                s[nb][i] = valid ? v : -FLT_MAX;
-                if (hi_row) tmax_hi = fmaxf(tmax_hi, s[nb][i]);
-                else tmax_lo = fmaxf(tmax_lo, s[nb][i]);
-            }
-        tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(kFullMask, tmax_lo, 1));
-        tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(kFullMask, tmax_lo, 2));
-        tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(kFullMask, tmax_hi, 1));
-        tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(kFullMask, tmax_hi, 2));
-        const float new_lo = fmaxf(m_lo, tmax_lo), new_hi = fmaxf(m_hi, tmax_hi);
-        const float r_lo = expf(m_lo - new_lo), r_hi = expf(m_hi - new_hi);
-        float sum_lo = 0.0f, sum_hi = 0.0f;
+                for (int j = 0; j < 4; ++j) s[nb][j] += s_odd[nb][j];
+            // mask, bias, online softmax (rows g and g + 8; a row's 16 scores sit in its quad of lanes)
+            float tmax_lo = -FLT_MAX, tmax_hi = -FLT_MAX;
 #pragma unroll
-        for (int nb = 0; nb < 4; ++nb)
+            for (int nb = 0; nb < 2; ++nb)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const bool hi_row = i >= 2;
-                const float pv = s[nb][i] > -FLT_MAX ? expf(s[nb][i] - (hi_row ? new_hi : new_lo)) : 0.0f;
-                if (hi_row) sum_hi += pv;
-                else sum_lo += pv;
-                Ps[(hi_row ? g + 8 : g) * 36 + nb * 8 + 2 * t + (i & 1)] = __uint_as_float(to_tf32(pv));
-            }
-        sum_lo += __shfl_xor_sync(kFullMask, sum_lo, 1);
-        sum_lo += __shfl_xor_sync(kFullMask, sum_lo, 2);
-        sum_hi += __shfl_xor_sync(kFullMask, sum_hi, 1);
-        sum_hi += __shfl_xor_sync(kFullMask, sum_hi, 2);
-        l_lo = l_lo * r_lo + sum_lo;
-        l_hi = l_hi * r_hi + sum_hi;
-        m_lo = new_lo;
-        m_hi = new_hi;
-        cp_async_wait<0>();  // V has landed
-        __syncwarp();        // ... and every lane's probabilities are in shared memory
+                for (int j = 0; j < 4; ++j) {
+                    const int key = k0 + nb * 8 + 2 * t + (j & 1);
+                    const bool hi_row = j >= 2;
+                    const bool valid = key < (hi_row ? keys_hi : keys_lo);
+                    float v = s[nb][j];
+                    if (valid && bias) v += hi_row ? bias_hi[key] : bias_lo[key];
+                    s[nb][j] = valid ? v : -FLT_MAX;
+                    if (hi_row) tmax_hi = fmaxf(tmax_hi, s[nb][j]);
+                    else tmax_lo = fmaxf(tmax_lo, s[nb][j]);
+                }
+            tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(kFullMask, tmax_lo, 1));
+            tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(kFullMask, tmax_lo, 2));
+            tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(kFullMask, tmax_hi, 1));
+            tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(kFullMask, tmax_hi, 2));
+            const float new_lo = fmaxf(m_lo, tmax_lo), new_hi = fmaxf(m_hi, tmax_hi);
+            const float r_lo = expf(m_lo - new_lo), r_hi = expf(m_hi - new_hi);
+            float sum_lo = 0.0f, sum_hi = 0.0f;
+#pragma unroll
+            for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const bool hi_row = j >= 2;
+                    const float pv = s[nb][j] > -FLT_MAX ? expf(s[nb][j] - (hi_row ? new_hi : new_lo)) : 0.0f;
+                    if (hi_row) sum_hi += pv;
+                    else sum_lo += pv;
+                    Ps[(hi_row ? g + 8 : g) * S::kPStride + nb * 8 + 2 * t + (j & 1)] = __uint_as_float(to_tf32(pv));
+                }
+            sum_lo += __shfl_xor_sync(kFullMask, sum_lo, 1);
+            sum_lo += __shfl_xor_sync(kFullMask, sum_lo, 2);
+            sum_hi += __shfl_xor_sync(kFullMask, sum_hi, 1);
+            sum_hi += __shfl_xor_sync(kFullMask, sum_hi, 2);
+            l_lo = l_lo * r_lo + sum_lo;
+            l_hi = l_hi * r_hi + sum_hi;
+            m_lo = new_lo;
+            m_hi = new_hi;
+            __syncwarp();  // every lane's probabilities are in shared memory
 
-        // O = O * rescale + P V
-        uint32_t pa[4][4];
+            // O = O * rescale + P V
+            uint32_t pa[2][4];
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-            pa[ks][0] = __float_as_uint(Ps[g * 36 + ks * 8 + t]);
-            pa[ks][1] = __float_as_uint(Ps[(g + 8) * 36 + ks * 8 + t]);
-            pa[ks][2] = __float_as_uint(Ps[g * 36 + ks * 8 + t + 4]);
-            pa[ks][3] = __float_as_uint(Ps[(g + 8) * 36 + ks * 8 + t + 4]);
-        }
+            for (int ks = 0; ks < 2; ++ks) {
+                pa[ks][0] = __float_as_uint(Ps[g * S::kPStride + ks * 8 + t]);
+                pa[ks][1] = __float_as_uint(Ps[(g + 8) * S::kPStride + ks * 8 + t]);
+                pa[ks][2] = __float_as_uint(Ps[g * S::kPStride + ks * 8 + t + 4]);
+                pa[ks][3] = __float_as_uint(Ps[(g + 8) * S::kPStride + ks * 8 + t + 4]);
+            }
 #pragma unroll
-        for (int n = 0; n < DH / 8; ++n) {
-            o[n][0] *= r_lo; o[n][1] *= r_lo; o[n][2] *= r_hi; o[n][3] *= r_hi;
+            for (int n = 0; n < DH / 8; ++n) {
+                o[n][0] *= r_lo; o[n][1] *= r_lo; o[n][2] *= r_hi; o[n][3] *= r_hi;
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                const float* vr = Vt + (ks * 8 + t) * S::kRow + n * 8 + g;
-                mma_tf32(o[n], pa[ks], __float_as_uint(vr[0]), __float_as_uint(vr[4 * S::kRow]));
+                for (int ks = 0; ks < 2; ++ks) {
+                    const float* vr = Vt + (ks * 8 + t) * S::kRow + n * 8 + g;
+                    mma_tf32(o[n], pa[ks], __float_as_uint(vr[0]), __float_as_uint(vr[4 * S::kRow]));
+                }
             }
         }
-        __syncwarp();  // the tile buffers are free for the next tile
+        __syncwarp();  // this stage (and the probabilities) are free again
+        issue(i + kMmaStages);
     }
+    cp_async_wait<0>();
 
     // park this warp's state in its own tile buffer: [query][max, sum, O[DH]]
     __syncthreads();
-    float* st = Kt;  // 16 * (DH + 2) floats <= one tile
+    float* st = stage0;  // 16 * (DH + 2) floats fit a stage
 #pragma unroll
     for (int n = 0; n < DH / 8; ++n) {
         st[g * (DH + 2) + 2 + n * 8 + 2 * t] = o[n][0];
