@@ -276,8 +276,13 @@ class GenerationWorkload:
         self.budget_tokens = grow
 
     def launches_per_iteration(self):
-        fwd = lambda cfg: 1 + 10 * cfg["n_layers"] + 3
-        return 1 + self.gamma * (1 + fwd(self.dcfg) + 1) + 1 + fwd(self.tcfg) + 2 + 1
+        # per block: 4 GEMMs, 2 norms, RoPE/append, attention, activation (+ the combine kernel when the
+        # key slices are not merged inside a cluster: long contexts); embed, final norm, head, its reduction
+        long_context = self.prompt_len > 256
+        fwd = lambda cfg, combine: 1 + (9 + combine) * cfg["n_layers"] + 3
+        draft = fwd(self.dcfg, 0)  # one or two rows against few slices: merged in the cluster
+        target = fwd(self.tcfg, 1 if long_context else 0)
+        return 1 + self.gamma * (1 + draft + 1) + 1 + target + 2 + 1
 
     def timed_decode(self, warmup, steps, gamma):
         """Device time of `steps` iterations after `warmup` untimed ones (prompt pass untimed)."""
@@ -419,7 +424,8 @@ class EncDecWorkload(GenerationWorkload):
         self.budget_tokens = grow
 
     def launches_per_iteration(self):
-        fwd = lambda cfg: 1 + 16 * cfg["n_layers"] + 3
+        # per decoder block: 7 GEMMs, 3 norms, K/V append, cross-attention queries, 2 attentions, activation
+        fwd = lambda cfg: 1 + 15 * cfg["n_layers"] + 3
         return 1 + self.gamma * (1 + fwd(self.dcfg) + 1) + 1 + fwd(self.tcfg) + 2 + 1
 
     def kv_bytes(self, context):
@@ -659,6 +665,13 @@ def run_generation(args, wl, torch, device, local, barrier):
                                                                         times["target_rows_ms"], times["draft_1row_ms"],
                                                                         wl.gamma)},
             "pass_ms": times,
+            # Section 3.5: the gamma that maximises Theorem 3.8 for the measured alpha and c, and the one that
+            # maximises the generalised form when every extra verified row costs what the measured kappa implies
+            "best_gamma": {"theorem_3_8": analysis.best_gamma(alpha, c, 32) if 0.0 < alpha < 1.0 else None,
+                           "generalised": max(range(1, 33), key=lambda g_: analysis.generalised_speedup(
+                               analysis.expected_tokens(alpha, g_), times["target_1row_ms"],
+                               times["target_1row_ms"] * (1.0 + (times["target_rows_ms"] / times["target_1row_ms"] - 1.0) * g_ / max(wl.gamma, 1)),
+                               times["draft_1row_ms"], g_)) if 0.0 < alpha < 1.0 else None},
             "imposed_acceptance_sweep": sweep,
             "verify_pass": {"bytes": pass_bytes, "ms": times["target_rows_ms"],
                             "gbs": pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9,
