@@ -231,6 +231,8 @@ def weight_stream_bytes(cfg):
     """Bytes of one pass over the model: every block matrix and the LM head once."""
     from paper_2211_17192_b200 import workloads
     elem = 2 if cfg["dtype"] == "bf16" else 4
+    if cfg["arch"] == "bigram":
+        return cfg["vocab"] * elem  # one row of the table
     total = 0
     for name, shape, kind in workloads.tensor_shapes(cfg):
         if kind == "gain" or name in ("pos_emb",) or (name == "tok_emb" and not cfg["tied"]) or not decode_stream(name):
@@ -280,7 +282,7 @@ class GenerationWorkload:
         # key slices are not merged inside a cluster: long contexts); embed, final norm, head, its reduction
         long_context = self.prompt_len > 256
         fwd = lambda cfg, combine: 1 + (9 + combine) * cfg["n_layers"] + 3
-        draft = fwd(self.dcfg, 0)  # one or two rows against few slices: merged in the cluster
+        draft = 1 if self.dcfg["arch"] == "bigram" else fwd(self.dcfg, 0)  # (few slices: merged in the cluster)
         target = fwd(self.tcfg, 1 if long_context else 0)
         return 1 + self.gamma * (1 + draft + 1) + 1 + target + 2 + 1
 
@@ -370,11 +372,15 @@ class GenerationWorkload:
         from oracle.decoder import Decoder
         from paper_2211_17192_b200 import workloads
         small_t = workloads.scaled_config(self.tcfg, n_layers=min(2, self.tcfg["n_layers"]))
-        small_d = workloads.scaled_config(self.dcfg, n_layers=min(2, self.dcfg["n_layers"]))
+        small_d = self.dcfg if self.dcfg["arch"] == "bigram" else workloads.scaled_config(self.dcfg, n_layers=min(2, self.dcfg["n_layers"]))
         dtype = np.float32 if self.tcfg["d_model"] >= 2048 else np.float64
         if not hasattr(self, "_cpu_models"):  # built once, outside every timed sample
-            self._cpu_models = (Decoder(small_t, workloads.make_weights(small_t, 1), dtype=dtype),
-                                Decoder(small_d, workloads.make_weights(small_d, 2), dtype=dtype))
+            if self.dcfg["arch"] == "bigram":
+                from oracle.ngram import BigramTable
+                draft_model = BigramTable(workloads.make_weights(self.dcfg, 2)["table"], dtype=np.float32)
+            else:
+                draft_model = Decoder(small_d, workloads.make_weights(small_d, 2), dtype=dtype)
+            self._cpu_models = (Decoder(small_t, workloads.make_weights(small_t, 1), dtype=dtype), draft_model)
         target, draft = self._cpu_models
         prompt = workloads.make_prompt(3, 32, self.tcfg["vocab"])
         t0 = time.perf_counter()
@@ -389,7 +395,7 @@ class GenerationWorkload:
         small = weight_stream_bytes(small_t) + self.gamma * weight_stream_bytes(small_d)
         value = tokens / dt * small / full
         sample = (f"{iters} iterations of Algorithm 1, batch 1, 32-token prompt, both models at full width and "
-                  f"{small_t['n_layers']}+{small_d['n_layers']} layers in {np.dtype(dtype).name}, {dt:.1f} s; "
+                  f"{small_t['n_layers']}+{small_d.get('n_layers', 0)} layers in {np.dtype(dtype).name}, {dt:.1f} s; "
                   f"scaled by streamed weight bytes ({small / full:.3f}) to the full depth")
         return value, sample
 
@@ -493,6 +499,9 @@ def make_workload(args):
         return GenerationWorkload("gpt97m_6m_b1", "gpt97m_target", "gpt6m_draft", batch, args.prompt_len or 128, 512,
                                   args.gamma or 5, args.temperature, args.layers)
     gamma = args.gamma or 2
+    if args.draft == "bigram":  # a negligible-cost draft: one table row per step instead of a model pass
+        return GenerationWorkload(f"llama7b_bigram_b{batch}_g{gamma}", "llama7b_target", "bigram_32k", batch,
+                                  args.prompt_len or 1024, 256, gamma, args.temperature, args.layers)
     return GenerationWorkload(f"llama7b_160m_b{batch}_g{gamma}", "llama7b_target", "llama160m_draft", batch,
                               args.prompt_len or 1024, 256, gamma, args.temperature, args.layers)
 
@@ -704,6 +713,8 @@ def main():
     ap.add_argument("--gamma", type=int, default=None)
     ap.add_argument("--temperature", type=float, default=1.0)
     ap.add_argument("--prompt-len", type=int, default=None, help="override the workload's prompt length (profiling)")
+    ap.add_argument("--draft", default="model", choices=["model", "bigram"],
+                    help="llama7b workload: the 160M-shaped draft model, or a bigram table (negligible-cost draft)")
     ap.add_argument("--layers", type=int, default=None, help="override the target's depth, full width (profiling)")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for cpu_baseline")

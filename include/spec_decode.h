@@ -194,6 +194,13 @@ int spec_uniforms(uint64_t seed, const int32_t* positions, const int32_t* sequen
  *                    with gain lnx; [K; V] = Wkv_x . encoder output, computed
  *                    once; no bias; out-projection Wo_x) and the FFN.
  *                    n_kv_heads == n_heads; decoding starts from token id 0.
+ *   SPEC_ARCH_BIGRAM: a negligible-cost approximation model (the paper's
+ *                    Section 4 evaluates unigram and bigram drafts): the next-token logits depend
+ *                    on the last token only, logits = table[token].  Only
+ *                    valid as the DRAFT.  tok_emb points at the table
+ *                    [vocab, vocab] (row = last token) in `dtype`; only `arch`,
+ *                    `vocab` and `dtype` of the config are read, no other
+ *                    weight pointer is used, and it keeps no K,V rows.
  *   FFN: SPEC_FFN_GELU (tanh approximation) with W_in [d_ff, d_model];
  *        SPEC_FFN_GATED_GELU / SPEC_FFN_SWIGLU with W_in [2*d_ff, d_model],
  *        rows 0..d_ff-1 the gate, rows d_ff..2*d_ff-1 the up projection.
@@ -201,7 +208,7 @@ int spec_uniforms(uint64_t seed, const int32_t* positions, const int32_t* sequen
  * bf16 as raw 16-bit patterns); gains are fp32.  The residual stream, softmax,
  * normalisation and logits are fp32 in every configuration.
  * ------------------------------------------------------------------------- */
-enum { SPEC_ARCH_GPT = 0, SPEC_ARCH_LLAMA = 1, SPEC_ARCH_T5 = 2 };
+enum { SPEC_ARCH_GPT = 0, SPEC_ARCH_LLAMA = 1, SPEC_ARCH_T5 = 2, SPEC_ARCH_BIGRAM = 3 };
 enum { SPEC_FFN_GELU = 0, SPEC_FFN_GATED_GELU = 1, SPEC_FFN_SWIGLU = 2 };
 enum { SPEC_DTYPE_FP32 = 0, SPEC_DTYPE_BF16 = 1 };
 

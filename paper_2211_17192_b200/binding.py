@@ -284,7 +284,7 @@ class _Stats(ctypes.Structure):
                [("prefill_ms", ctypes.c_double), ("decode_ms", ctypes.c_double)]
 
 
-_ARCH = {"gpt": 0, "llama": 1, "t5": 2}
+_ARCH = {"gpt": 0, "llama": 1, "t5": 2, "bigram": 3}
 _FFN = {"gelu": 0, "gated_gelu": 1, "swiglu": 2}
 _DTYPE = {"fp32": 0, "bf16": 1}
 _engine_declared = False
@@ -328,6 +328,8 @@ def _declare_engine(h):
 
 
 def _cfg_struct(cfg):
+    if cfg["arch"] == "bigram":  # only arch, vocab and dtype are read
+        return _ModelCfg(_ARCH["bigram"], 0, 0, 0, 0, 0, 0, 0, cfg["vocab"], 0, 0, _DTYPE[cfg["dtype"]], 0.0, 0.0, 0, 0, 0)
     return _ModelCfg(_ARCH[cfg["arch"]], cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["n_kv_heads"],
                      cfg["d_head"], cfg["d_ff"], _FFN[cfg["ffn"]], cfg["vocab"], cfg["max_positions"],
                      1 if cfg["tied"] else 0, _DTYPE[cfg["dtype"]], cfg["rms_eps"], cfg["rope_base"],
@@ -376,6 +378,8 @@ class Engine:
             self._keep.append(t)
             return t.data_ptr()
 
+        if cfg["arch"] == "bigram":
+            return _Weights(dev("table", True), None, None, None, None, None, None, None, None)
         t5 = cfg["arch"] == "t5"
 
         def block(p, cross):

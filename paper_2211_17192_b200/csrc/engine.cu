@@ -67,6 +67,11 @@ namespace spec {
 namespace {
 
 int check_cfg(const spec_model_cfg& c, const char* which) {
+    if (c.arch == SPEC_ARCH_BIGRAM) {
+        if (c.vocab < 1 || (c.dtype != SPEC_DTYPE_FP32 && c.dtype != SPEC_DTYPE_BF16))
+            return fail(SPEC_ERR_BAD_CONFIG, "%s: a table model needs vocab >= 1 and a known dtype", which);
+        return SPEC_OK;
+    }
     if (c.arch != SPEC_ARCH_GPT && c.arch != SPEC_ARCH_LLAMA && c.arch != SPEC_ARCH_T5)
         return fail(SPEC_ERR_BAD_CONFIG, "%s: unknown arch %d", which, c.arch);
     if (c.arch == SPEC_ARCH_T5) {
@@ -195,6 +200,10 @@ int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_ro
     const spec_model_cfg& c = m.cfg;
     const int n_rows = batch * m_rows;
     const RowMeta rows{ctx->row_token, ctx->row_pos, ctx->row_seq};
+    if (c.arch == SPEC_ARCH_BIGRAM)  // logits = table[last token]: one gather
+        return n_logit_rows > 0 ? launch_table_logits(m.tok_emb, m.bf16(), c.vocab, rows.token, logit_src, logit_dst, n_logit_rows,
+                                                       logits, ctx->stream)
+                                : SPEC_OK;
     Pass pass{ctx, m, n_rows, m.bf16() && ctx->tensor_cores, ctx->stream};
     const int d = c.d_model;
     const float* bias = m.t5() ? m.dec_bias : nullptr;
@@ -495,6 +504,19 @@ int pack_model(spec_ctx* ctx, Model& m) {
 int init_model(spec_ctx* ctx, int which, const spec_model_cfg& cfg, const spec_weights& w) {
     Model& m = ctx->model[which];
     m.cfg = cfg;
+    if (cfg.arch == SPEC_ARCH_BIGRAM) {  // a table: no blocks, no cache; the sizes below only keep the buffer arithmetic valid
+        if (which != 1) return fail(SPEC_ERR_BAD_CONFIG, "spec_init: a table model can only be the draft");
+        if (!w.tok_emb) return fail(SPEC_ERR_BAD_ARG, "spec_init: missing table pointer");
+        m.tok_emb = w.tok_emb;
+        m.cfg.n_layers = 0;
+        m.cfg.d_model = m.cfg.d_ff = 8;
+        m.cfg.n_heads = m.cfg.n_kv_heads = 1;
+        m.cfg.d_head = 64;
+        m.cfg.ffn = SPEC_FFN_GELU;
+        m.cfg.max_positions = 1 << 30;
+        m.cfg.tied_embeddings = 1;
+        return SPEC_OK;
+    }
     if (!w.tok_emb || !w.ln_f || !w.layers || (cfg.arch == SPEC_ARCH_GPT && !w.pos_emb) || (!cfg.tied_embeddings && !w.head))
         return fail(SPEC_ERR_BAD_ARG, "spec_init: missing weight pointer");
     m.tok_emb = w.tok_emb;
@@ -596,7 +618,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     if (draft_cfg) {
         SPEC_TRY(check_cfg(*draft_cfg, "draft"));
         if (draft_cfg->vocab != target_cfg->vocab) return fail(SPEC_ERR_BAD_CONFIG, "spec_init: vocabularies differ");
-        if ((draft_cfg->arch == SPEC_ARCH_T5) != (target_cfg->arch == SPEC_ARCH_T5))
+        if (draft_cfg->arch != SPEC_ARCH_BIGRAM && (draft_cfg->arch == SPEC_ARCH_T5) != (target_cfg->arch == SPEC_ARCH_T5))
             return fail(SPEC_ERR_BAD_CONFIG, "spec_init: an encoder-decoder target needs an encoder-decoder draft and vice versa");
     }
     const bool t5 = target_cfg->arch == SPEC_ARCH_T5;
@@ -684,7 +706,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
         bool any_bf16 = false;
         for (int i = 0; i < (ctx->has_draft ? 2 : 1); ++i) {
             const Model& m = ctx->model[i];
-            if (!m.bf16()) continue;
+            if (!m.bf16() || m.cfg.arch == SPEC_ARCH_BIGRAM) continue;
             any_bf16 = true;
             max_k = std::max<size_t>({max_k, static_cast<size_t>(m.cfg.d_model), static_cast<size_t>(m.q_dim()), static_cast<size_t>(m.cfg.d_ff)});
             const int shapes[7][2] = {{m.qkv_dim(), m.cfg.d_model}, {m.cfg.d_model, m.q_dim()}, {m.ffn_in_dim(), m.cfg.d_model},
@@ -699,7 +721,9 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
         }
         if (any_bf16 && ctx->tensor_cores) {
             for (int i = 0; i < (ctx->has_draft ? 2 : 1); ++i)
-                if (ctx->model[i].bf16() && (status = pack_model(ctx, ctx->model[i])) != SPEC_OK) return cleanup(status);
+                if (ctx->model[i].bf16() && ctx->model[i].cfg.arch != SPEC_ARCH_BIGRAM &&
+                    (status = pack_model(ctx, ctx->model[i])) != SPEC_OK)
+                    return cleanup(status);
             ctx->hi_rows = (ctx->max_rows + 127) / 128 * 128;
             SPEC_ALLOC(x_hi, static_cast<size_t>(ctx->hi_rows) * max_k);
             SPEC_ALLOC(x_lo, static_cast<size_t>(ctx->hi_rows) * max_k);
@@ -799,7 +823,8 @@ int encode_sources(spec_ctx* ctx, const int32_t* source, const int32_t* source_l
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_pos, pos.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_seq, seq.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->src_len, source_len, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
-    for (int which = 0; which < n_models; ++which) SPEC_TRY(encode(ctx, ctx->model[which], batch, longest));
+    for (int which = 0; which < n_models; ++which)
+        if (ctx->model[which].t5()) SPEC_TRY(encode(ctx, ctx->model[which], batch, longest));  // (a table draft has no encoder)
     SPEC_CUDA_TRY(cudaStreamSynchronize(st));  // the host vectors go out of scope
     if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
     ctx->encoded = true;

@@ -153,6 +153,19 @@ __global__ void qkv_kernel(float* __restrict__ qkv, const float* __restrict__ pa
     dst[j + half] = static_cast<KV>(x2);
 }
 
+// logits[dst(i)] = table[token[src(i)]] for a table model: grid = (chunks, rows), block = 256.
+__global__ void table_logits_kernel(const void* __restrict__ table, bool bf16, int vocab, const int32_t* __restrict__ token,
+                                    const int32_t* __restrict__ src_rows, const int32_t* __restrict__ dst_rows,
+                                    float* __restrict__ logits) {
+    pdl_trigger();
+    pdl_wait();
+    const int i = blockIdx.y;
+    const int t = min(max(token[src_rows ? src_rows[i] : i], 0), vocab - 1);
+    float* out = logits + static_cast<size_t>(dst_rows ? dst_rows[i] : i) * vocab;
+    for (int v = blockIdx.x * blockDim.x + threadIdx.x; v < vocab; v += gridDim.x * blockDim.x)
+        out[v] = load_elem(table, static_cast<size_t>(t) * vocab + v, bf16);
+}
+
 __device__ __forceinline__ float gelu_tanh(float x) {
     const float k = 0.7978845608028654f;  // sqrt(2 / pi)
     return 0.5f * x * (1.0f + tanhf(k * (x + 0.044715f * x * x * x)));
@@ -193,6 +206,13 @@ int launch_embed(const Model& m, const RowMeta& rows, int n_rows, float* h, cuda
     return launch_pdl(embed_kernel, dim3(n_rows), dim3(128), 0, stream, m.tok_emb, m.pos_emb, m.bf16(),
                       m.cfg.arch == SPEC_ARCH_GPT, rows.token, rows.pos, m.cfg.d_model, m.cfg.vocab,
                       m.cfg.max_positions, h);
+}
+
+int launch_table_logits(const void* table, bool bf16, int vocab, const int32_t* token, const int32_t* src_rows,
+                        const int32_t* dst_rows, int n_rows, float* logits, cudaStream_t stream) {
+    const int chunks = std::max(1, std::min((vocab + 255) / 256, 32));
+    return launch_pdl(table_logits_kernel, dim3(chunks, n_rows), dim3(256), 0, stream, table, bf16, vocab, token, src_rows,
+                      dst_rows, logits);
 }
 
 int launch_norm(float* h, const float* partial, int splits, int rows_total, const float* gain, const int32_t* src_rows,

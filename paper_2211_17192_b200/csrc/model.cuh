@@ -60,6 +60,10 @@ struct RowMeta {
 // h[r] = tok_emb[token[r]] (+ pos_emb[pos[r]] for GPT), fp32.
 int launch_embed(const Model& m, const RowMeta& rows, int n_rows, float* h, cudaStream_t stream);
 
+// A table model's logits: logits[dst(i)] = table[token[src(i)]] (table [vocab, vocab], fp32 or bf16).
+int launch_table_logits(const void* table, bool bf16, int vocab, const int32_t* token, const int32_t* src_rows,
+                        const int32_t* dst_rows, int n_rows, float* logits, cudaStream_t stream);
+
 // Row i of the output = RMSNorm(h[src(i)]) * gain, as fp32 (`out`) and/or as two
 // bf16 terms (`out_hi`, `out_lo`).  If `partial` is given (split-K results of
 // the GEMM before, [splits][rows_total][d]) it is first added into h.

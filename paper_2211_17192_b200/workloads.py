@@ -45,6 +45,9 @@ def model_config(name):
         "llama_test_draft": dict(arch="llama", ffn="swiglu", n_layers=1, d_model=128, n_heads=2, n_kv_heads=1,
                                  d_head=64, d_ff=384, vocab=2048, max_positions=512, dtype="bf16",
                                  head_std=INIT_STD),
+        # bigram tables: negligible-cost drafts (next-token logits from the last token alone)
+        "bigram_8k": dict(arch="bigram", vocab=8192, dtype="fp32", head_std=1.0),
+        "bigram_32k": dict(arch="bigram", vocab=32000, dtype="bf16", head_std=0.3),
         # T5-shaped encoder-decoder pair (XXL-shaped target, small-shaped draft), bf16
         "t5xxl_target": dict(arch="t5", ffn="gated_gelu", n_layers=24, n_enc_layers=24, d_model=4096, n_heads=64,
                              n_kv_heads=64, d_head=64, d_ff=10240, vocab=32128, max_positions=1024, dtype="bf16",
@@ -81,6 +84,8 @@ def scaled_config(cfg, **overrides):
 
 def tensor_shapes(cfg):
     """Ordered (name, shape, kind) of a model's tensors; kind is 'gain', 'matrix', 'bias' or 'head'."""
+    if cfg["arch"] == "bigram":
+        return [("table", (cfg["vocab"], cfg["vocab"]), "head")]
     d, H, Hkv, dh, F = cfg["d_model"], cfg["n_heads"], cfg["n_kv_heads"], cfg["d_head"], cfg["d_ff"]
     f_in = F if cfg["ffn"] == "gelu" else 2 * F
     t5 = cfg["arch"] == "t5"

@@ -183,3 +183,26 @@ def test_lenient_generation_matches_the_oracle_and_accepts_more(tiny):
         eng.set_lenience(1.0)
     _, strict = eng.generate([prompt], 48, 3, 1.0, 21)
     assert lenient["tests_passed"] / lenient["tests_evaluated"] > strict["tests_passed"] / strict["tests_evaluated"]
+
+
+@pytest.mark.parametrize("temperature", [1.0, 0.0])
+def test_bigram_table_draft_matches_the_oracle(temperature):
+    """The tiny fp32 target with a bigram table as its draft (no draft passes at all)."""
+    from oracle.ngram import BigramTable
+    tcfg = workloads.model_config("tiny_target")
+    tw = workloads.make_weights(tcfg, 1)
+    dcfg = workloads.model_config("bigram_8k")
+    dw = workloads.make_weights(dcfg, 2)
+    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=2, max_len=96, page_size=32, max_gamma=4)
+    try:
+        prompt = workloads.make_prompt(13, 12, tcfg["vocab"])
+        flagged, iters = compare_generation(eng, Decoder(tcfg, tw), BigramTable(dw["table"]), prompt, 48, 3, temperature,
+                                            seed=17, margin=1e-3, logit_tol=1e-3)
+        assert flagged <= 2
+        # a ragged batch of two runs, and greedy equals target-only greedy
+        prompts = [prompt, workloads.make_prompt(14, 5, tcfg["vocab"])]
+        greedy, _ = eng.generate(prompts, 24, 0, 0.0, 0)
+        spec, stats = eng.generate(prompts, 24, 4, 0.0, 0)
+        assert np.array_equal(greedy, spec) and stats["draft_passes"] > 0
+    finally:
+        eng.close()

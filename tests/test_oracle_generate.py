@@ -150,3 +150,23 @@ def test_generation_is_position_keyed():
     done = cut - 2
     rest = generate.speculative_generate(target, draft, [3, 4] + full.tokens[:done], 30 - done, 3, 1.0, seed=9)
     assert rest.tokens == full.tokens[done:]
+
+
+def test_bigram_table_draft():
+    """A table look-up as M_q (the paper's negligible-cost drafts): logits depend on the
+    last token only; a target that is itself that table accepts everything; T = 0
+    output equals the target's greedy output whatever the table."""
+    from oracle.ngram import BigramTable
+    rng = np.random.default_rng(5)
+    table = rng.standard_normal((32, 32)) * 2.0
+    draft = BigramTable(table)
+    a = draft.forward_rows([3, 7, 7])
+    assert np.array_equal(a[1], a[2]) and np.array_equal(a[0], table[3]) and draft.cached_len == 3
+    draft.truncate(1)
+    assert draft.cached_len == 1
+    same = generate.speculative_generate(BigramTable(table), BigramTable(table), [1, 2], 30, 4, 1.0, seed=3)
+    assert same.tests_passed == same.tests_evaluated and all(it.n_accepted == 4 for it in same.iterations)
+    other = BigramTable(rng.standard_normal((32, 32)))
+    want, _, _ = generate.target_only_generate(BigramTable(table), [1, 2], 25, 0.0, seed=0)
+    got = generate.speculative_generate(BigramTable(table), other, [1, 2], 25, 3, 0.0, seed=0)
+    assert got.tokens == want
