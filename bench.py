@@ -528,6 +528,17 @@ def cpu_threads():
         return 1
 
 
+def aggregate_over_ranks(dist, device, times, counts):
+    """Replicas only: every rank ran the same job on its own sequences.  The job's time
+    is the slowest rank's (MAX), its work the sum over ranks (SUM); no other exchange."""
+    import torch
+    t = torch.tensor(list(times), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    c = torch.tensor(list(counts), dtype=torch.int64, device=device)
+    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return [float(v) for v in t], [int(v) for v in c]
+
+
 def run_reference(args, wl):
     """The reference arm: the CPU oracle as it stands, on the machine's host cores."""
     rank = int(os.environ.get("RANK", "0"))
@@ -535,7 +546,7 @@ def run_reference(args, wl):
         return
     values = []
     sample = ""
-    per_step = max(1.0, 60.0 / max(1, args.steps + args.warmup))
+    per_step = max(0.5, min(60.0 / max(1, args.steps + args.warmup), 4.0 * args.cpu_budget))  # about a minute in all by default
     for _ in range(args.warmup):
         wl.cpu_sample(per_step)
     t0 = time.perf_counter()
@@ -757,12 +768,8 @@ def main():
     tokens, elapsed_ms, e2e_tokens, e2e_s, launches = (res[k] for k in ("tokens", "elapsed_ms", "e2e_tokens", "e2e_s", "launches"))
 
     if world > 1:
-        t = torch.tensor([elapsed_ms, e2e_s], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms, e2e_s = float(t[0]), float(t[1])
-        c = torch.tensor([tokens, e2e_tokens, launches], dtype=torch.int64, device=device)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        tokens, e2e_tokens, launches = int(c[0]), int(c[1]), int(c[2])
+        (elapsed_ms, e2e_s), (tokens, e2e_tokens, launches) = aggregate_over_ranks(
+            dist, device, [elapsed_ms, e2e_s], [tokens, e2e_tokens, launches])
 
     if rank == 0:
         cpu_value, cpu_sample = wl.cpu_sample(args.cpu_budget) if world == 1 else (None, "skipped for N > 1")
