@@ -432,12 +432,6 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
         q_head[tid] = kv_head * group + (live ? q % group : 0);
         q_pos[tid] = live ? pos[b * m_rows + j] : -1;
     }
-    __syncthreads();
-    for (int i = tid; i < 16 * DH; i += 32 * kMmaWarps) {
-        const int qi = i / DH, e = i % DH;
-        const float v = q_pos[qi] >= 0 ? qkv[static_cast<size_t>(q_row[qi]) * q_stride + q_head[qi] * DH + e] * scale : 0.0f;
-        Qs[qi * S::kRow + e] = __uint_as_float(to_tf32(v));
-    }
     int seq_keys = 0;
     if (kv_len) {
         seq_keys = kv_len[seq[b * m_rows]];
@@ -451,7 +445,7 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     const size_t page_stride = 2 * static_cast<size_t>(n_kv_heads) * head_stride;
     const size_t v_offset = static_cast<size_t>(n_kv_heads) * head_stride;
     const int32_t* pages = page_table + seq[b * m_rows] * pages_per_seq;
-    __syncthreads();
+    __syncthreads();  // (the queries' positions)
 
     // the two query rows of this lane: g and g + 8
     const int p_lo = q_pos[g], p_hi = q_pos[g + 8];
@@ -484,8 +478,15 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
         }
         cp_async_commit();
     };
+    // the first tiles are requested before the queries are staged
 #pragma unroll
     for (int i = 0; i < kMmaStages; ++i) issue(i);
+    for (int i = tid; i < 16 * DH; i += 32 * kMmaWarps) {
+        const int qi = i / DH, e = i % DH;
+        const float v = q_pos[qi] >= 0 ? qkv[static_cast<size_t>(q_row[qi]) * q_stride + q_head[qi] * DH + e] * scale : 0.0f;
+        Qs[qi * S::kRow + e] = __uint_as_float(to_tf32(v));
+    }
+    __syncthreads();
     for (int i = 0; i < my_tiles; ++i) {
         const int k0 = first_key(i);
         cp_async_wait<kMmaStages - 1>();  // tile i has landed (later tiles may still be in flight)
@@ -640,6 +641,10 @@ __global__ void attention_combine_kernel(const float* __restrict__ part, int sli
     pdl_trigger();
     pdl_wait();
     const float* in = part + static_cast<size_t>(blockIdx.x) * slices * (DH + 2);
+    // every load of this kernel is requested at once: the accumulators do not depend on the weights
+    float acc[32];
+#pragma unroll
+    for (int s = 0; s < 32; ++s) acc[s] = s < slices ? in[s * (DH + 2) + 2 + threadIdx.x] : 0.0f;
     if (threadIdx.x < 32) {  // slices <= 32: one lane per slice
         const int s = threadIdx.x;
         const float ms = s < slices ? in[s * (DH + 2)] : -FLT_MAX;
@@ -652,8 +657,8 @@ __global__ void attention_combine_kernel(const float* __restrict__ part, int sli
     }
     __syncthreads();
     float o = 0.0f;
-#pragma unroll 8
-    for (int s = 0; s < slices; ++s) o += in[s * (DH + 2) + 2 + threadIdx.x] * w_sh[s];
+#pragma unroll
+    for (int s = 0; s < 32; ++s) o += s < slices ? acc[s] * w_sh[s] : 0.0f;  // slices in index order
     const float l = w_sh[32];
     const float y = l > 0.0f ? o / l : 0.0f;  // an inactive row has no keys
     const size_t i = static_cast<size_t>(blockIdx.x) * DH + threadIdx.x;

@@ -59,11 +59,18 @@ norm_kernel(float* h, const float* __restrict__ partial, int splits, int n_rows,
             __nv_bfloat16* __restrict__ out_hi, __nv_bfloat16* __restrict__ out_lo) {
     __shared__ float red[kNormThreads / 32];
     pdl_trigger();
-    pdl_wait();
     const int r = blockIdx.x;
+    const int groups = d / 4;
+    // the gains are constants: fetched while the kernel before this one is still finishing
+    float4 gg[kNormPerThread];
+#pragma unroll
+    for (int j = 0; j < kNormPerThread; ++j) {
+        const int g = threadIdx.x + j * kNormThreads;
+        gg[j] = g < groups ? *reinterpret_cast<const float4*>(gain + 4 * g) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    pdl_wait();
     const size_t src = static_cast<size_t>(src_rows ? src_rows[r] : r) * d;
     const size_t stride = static_cast<size_t>(n_rows) * d;
-    const int groups = d / 4;
     float4 v[kNormPerThread];
     float ss = 0.0f;
 #pragma unroll
@@ -94,8 +101,8 @@ norm_kernel(float* h, const float* __restrict__ partial, int splits, int n_rows,
     for (int j = 0; j < kNormPerThread; ++j) {
         const int g = threadIdx.x + j * kNormThreads;
         if (g < groups) {
-            const float4 gg = *reinterpret_cast<const float4*>(gain + 4 * g);
-            const float y[4] = {v[j].x * scale * gg.x, v[j].y * scale * gg.y, v[j].z * scale * gg.z, v[j].w * scale * gg.w};
+            const float y[4] = {v[j].x * scale * gg[j].x, v[j].y * scale * gg[j].y, v[j].z * scale * gg[j].z,
+                                v[j].w * scale * gg[j].w};
             if (out) *reinterpret_cast<float4*>(out + dst + 4 * g) = make_float4(y[0], y[1], y[2], y[3]);
             if (out_hi) {
 #pragma unroll
