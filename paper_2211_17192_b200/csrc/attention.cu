@@ -682,9 +682,13 @@ int attention_sub_slices(int queries) {
 // The tensor-core kernel serves bf16 models (its tf32 products stay far inside
 // their 2e-2 logit bar, not inside the 1e-4 bar of fp32 models) once a KV head
 // has enough queries to fill a good part of a 16-row block.
-bool attention_uses_mma(const Model& m, int m_rows) {
+bool attention_uses_mma(const Model& m, int batch, int m_rows, int max_keys) {
     static const bool disabled = [] { const char* e = std::getenv("SPEC_NO_MMA_ATTENTION"); return e && e[0] == '1'; }();
-    return !disabled && m.bf16() && (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows >= 5;  // below that the warp-per-query kernel wins
+    const int queries = (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows;
+    // With fewer than 5 queries per KV head, or little work in all (query-key pairs over the
+    // whole launch), the warp-per-query kernel wins: its CTAs are lighter to launch.
+    const long long pairs = static_cast<long long>(batch) * m.cfg.n_kv_heads * queries * max_keys;
+    return !disabled && m.bf16() && queries >= 5 && pairs >= 65536;
 }
 
 // The key slices can be merged inside a cluster (no second kernel) whenever a CTA
@@ -692,10 +696,10 @@ bool attention_uses_mma(const Model& m, int m_rows) {
 // the warp-per-query path when the queries fit one round of warps.  It is done
 // when the slice count that balances the keys is at most 8: long contexts want
 // more slices than a cluster schedules well, and keep the separate combine kernel.
-bool attention_merges_in_cluster(const Model& m, int m_rows) {
+bool attention_merges_in_cluster(const Model& m, int batch, int m_rows, int max_keys) {
     static const bool disabled = [] { const char* e = std::getenv("SPEC_NO_CLUSTER_MERGE"); return e && e[0] == '1'; }();
     if (disabled) return false;
-    return attention_uses_mma(m, m_rows) || (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows <= kMaxAttnWarps;
+    return attention_uses_mma(m, batch, m_rows, max_keys) || (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows <= kMaxAttnWarps;
 }
 
 int attention_slices(const Model& m, int batch, int m_rows, int max_len) {
@@ -703,7 +707,7 @@ int attention_slices(const Model& m, int batch, int m_rows, int max_len) {
     const int n_kv_heads = m.cfg.n_kv_heads;
     const int queries = (m.cfg.n_heads / n_kv_heads) * m_rows;
     const int tiles = (max_len + 31) / 32;
-    if (attention_uses_mma(m, m_rows)) {
+    if (attention_uses_mma(m, batch, m_rows, max_len)) {
         // one wave of CTAs (shared memory allows one per SM at d_head 128, two at 64); a tile per warp at least
         const int m_blocks = (queries + 15) / 16;
         const int resident = 148 * (m.cfg.d_head == 64 ? 2 : 1);
@@ -760,15 +764,15 @@ int launch_attn(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, in
 
 template <typename KV, int DH>
 int launch_attention_variant(const Model& m, const AttnSource& src, const RowMeta& rows, int batch, int m_rows, int slices,
-                             float* part, const AttnOut& out, cudaStream_t stream) {
+                             int max_keys, float* part, const AttnOut& out, cudaStream_t stream) {
     const int group = m.cfg.n_heads / m.cfg.n_kv_heads;
     const int queries = group * m_rows;
     const float scale = 1.0f / sqrtf(static_cast<float>(m.cfg.d_head));
     const int n_rows = batch * m_rows;
-    const bool fused = attention_merges_in_cluster(m, m_rows) && slices <= kMaxClusterSlices;
+    const bool fused = attention_merges_in_cluster(m, batch, m_rows, max_keys) && slices <= kMaxClusterSlices;
     const KV* pool = static_cast<const KV*>(src.pool.kv);
     int status;
-    if (attention_uses_mma(m, m_rows)) {
+    if (attention_uses_mma(m, batch, m_rows, max_keys)) {
         static bool configured = false;
         if (!configured) {
             SPEC_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<KV, DH, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -808,14 +812,14 @@ int launch_attention_variant(const Model& m, const AttnSource& src, const RowMet
 }  // namespace
 
 int launch_attention(const Model& m, const AttnSource& src, const RowMeta& rows, int batch, int m_rows, int slices,
-                     float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo, cudaStream_t stream) {
+                     int max_keys, float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo, cudaStream_t stream) {
     const AttnOut out{att, att_hi, att_lo};
     if (src.pool.elem_bytes == 2) {
-        if (m.cfg.d_head == 64) return launch_attention_variant<__nv_bfloat16, 64>(m, src, rows, batch, m_rows, slices, part, out, stream);
-        return launch_attention_variant<__nv_bfloat16, 128>(m, src, rows, batch, m_rows, slices, part, out, stream);
+        if (m.cfg.d_head == 64) return launch_attention_variant<__nv_bfloat16, 64>(m, src, rows, batch, m_rows, slices, max_keys, part, out, stream);
+        return launch_attention_variant<__nv_bfloat16, 128>(m, src, rows, batch, m_rows, slices, max_keys, part, out, stream);
     }
-    if (m.cfg.d_head == 64) return launch_attention_variant<float, 64>(m, src, rows, batch, m_rows, slices, part, out, stream);
-    return launch_attention_variant<float, 128>(m, src, rows, batch, m_rows, slices, part, out, stream);
+    if (m.cfg.d_head == 64) return launch_attention_variant<float, 64>(m, src, rows, batch, m_rows, slices, max_keys, part, out, stream);
+    return launch_attention_variant<float, 128>(m, src, rows, batch, m_rows, slices, max_keys, part, out, stream);
 }
 
 }  // namespace spec

@@ -176,7 +176,7 @@ struct Pass {
                             n_rows, ctx->qkv, partials(), last_splits, st));
         const int slices = attention_slices(m, batch, m_rows, max_keys);
         const AttnSource src{ctx->qkv, m.qkv_dim(), pool, kv_len, bias, bias_span, bias_zero};
-        SPEC_TRY(launch_attention(m, src, rows, batch, m_rows, slices, ctx->attn_part, tc ? nullptr : ctx->att,
+        SPEC_TRY(launch_attention(m, src, rows, batch, m_rows, slices, max_keys, ctx->attn_part, tc ? nullptr : ctx->att,
                                   tc ? hi() : nullptr, tc ? lo() : nullptr, st));
         return residual(w.wo, pw.wo, m.q_dim(), ctx->att);
     }
@@ -223,7 +223,7 @@ int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_ro
             const KvPool pool = source_pool(ctx, m, static_cast<char*>(m.cross_kv) + static_cast<size_t>(l) * m.cross_stride);
             const int slices = attention_slices(m, batch, m_rows, ctx->rt.max_src_len);
             const AttnSource src{ctx->qkv, m.q_dim(), pool, ctx->src_len, nullptr, 0, 0};
-            SPEC_TRY(launch_attention(m, src, rows, batch, m_rows, slices, ctx->attn_part, pass.tc ? nullptr : ctx->att,
+            SPEC_TRY(launch_attention(m, src, rows, batch, m_rows, slices, ctx->rt.max_src_len, ctx->attn_part, pass.tc ? nullptr : ctx->att,
                                       pass.tc ? pass.hi() : nullptr, pass.tc ? pass.lo() : nullptr, ctx->stream));
             SPEC_TRY(pass.residual(w.wo_x, pw.wo_x, m.q_dim(), ctx->att));
         }

@@ -132,8 +132,9 @@ struct AttnSource {
 // rows b*m_rows .. of the pass.  Output as fp32 and/or two bf16 terms.
 int attention_slices(const Model& m, int batch, int m_rows, int max_len);
 size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices);
+// (slices from attention_slices with the same batch, m_rows and max_keys, the capacity of the key set)
 int launch_attention(const Model& m, const AttnSource& src, const RowMeta& rows, int batch, int m_rows, int slices,
-                     float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo, cudaStream_t stream);
+                     int max_keys, float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo, cudaStream_t stream);
 
 // f = gelu(u)  |  gelu(u[:, :F]) * u[:, F:]  |  silu(u[:, :F]) * u[:, F:], u given in full or as partial sums.
 int launch_ffn_act(const float* u, const float* partial, int splits, int n_rows, int d_ff, int ffn, float* f,
