@@ -35,7 +35,18 @@ What follows the paper, and where it is silent:
   logit(x_i) >= max logit + ln l; l = 1 keeps the strict rule (x_i accepted
   iff it is the lowest-index maximum).
 
-Pins (tests/test_oracle_sampling.py): emitted-token law equals p over 10^6
+* Section 2.2 names top-k among the sampling methods that reduce to a draw
+  from an adjusted distribution and gives no definition.  Reading: with k > 0,
+  every logit below the k-th largest logit of its row is set to -inf before
+  the temperature softmax (entries equal to the k-th largest all stay, so
+  ties can keep more than k); k = 0 or k >= vocabulary changes nothing.  The
+  same k standardises p and q, as the section asks.  T = 0 ignores k (the
+  maximum is always kept).
+
+Pins (tests/test_oracle_sampling.py): top-k against a pick-the-maximum-k-times
+restatement, its support size, the preserved ratios inside the support, k = 1
+against argmax and k >= V against plain softmax, and the emitted-token law
+under top-k against the top-k target distribution; emitted-token law equals p over 10^6
 seeded trials (Appendix A.1); with lenience the acceptance frequency equals
 sum min(p / l, q) (Appendix A.5), the emitted law equals min(q, p / l) +
 (1 - alpha_l) * max(0, p - q) / (1 - beta) and never exceeds p / l, and
@@ -51,10 +62,25 @@ from dataclasses import dataclass, field
 import numpy as np
 
 
-def standardise(logits, temperature):
+def top_k_floor(logits, top_k):
+    """The k-th largest logit of a row (-inf when top-k is off: k = 0 or k >= V)."""
+    z = np.asarray(logits, dtype=np.float64)
+    if top_k <= 0 or top_k >= z.shape[0]:
+        return -np.inf
+    return float(np.sort(z)[z.shape[0] - top_k])
+
+
+def keep_top_k(logits, top_k):
+    """The row with every logit below its k-th largest replaced by -inf."""
+    z = np.asarray(logits, dtype=np.float64)
+    return np.where(z >= top_k_floor(z, top_k), z, -np.inf)
+
+
+def standardise(logits, temperature, top_k=0):
     """Section 2.2: logits -> the adjusted distribution that is sampled from.
 
-    T > 0: softmax(logits / T) with the maximum subtracted first.
+    T > 0: softmax(logits / T) over the top-k logits (all of them for k = 0),
+    with the maximum subtracted first.
     T = 0: one-hot at the maximum (lowest index on ties).
     """
     z = np.asarray(logits, dtype=np.float64)
@@ -62,7 +88,7 @@ def standardise(logits, temperature):
         out = np.zeros_like(z)
         out[int(np.argmax(z))] = 1.0  # numpy's argmax returns the first maximum
         return out
-    z = z / float(temperature)
+    z = keep_top_k(z, top_k) / float(temperature)
     z = z - z.max()
     e = np.exp(z)
     return e / e.sum()
@@ -128,7 +154,7 @@ def lenient_greedy_accepts(target_row, x, lenience):
     return slack >= 0.0, abs(slack)
 
 
-def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0):
+def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0, top_k=0):
     """Algorithm 1 from "determine the number of accepted guesses" to the end.
 
     target_logits [gamma+1, V]: row i-1 gives p_i (i = 1..gamma+1).
@@ -142,8 +168,8 @@ def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature
     assert ql.shape[0] == gamma and len(draft_tokens) == gamma
     assert len(uniforms) == gamma + 1
 
-    p = [standardise(tl[i], temperature) for i in range(gamma + 1)]
-    q = [standardise(ql[i], temperature) for i in range(gamma)]
+    p = [standardise(tl[i], temperature, top_k) for i in range(gamma + 1)]
+    q = [standardise(ql[i], temperature, top_k) for i in range(gamma)]
 
     accept_margin = float("inf")
     top2_gap = float("inf")
@@ -180,15 +206,15 @@ def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature
     return VerifyResult(n, t, accept_margin, cdf_margin, top2_gap, fallback, betas)
 
 
-def verify_batch(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0):
+def verify_batch(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0, top_k=0):
     """`verify_step` for every sequence of a batch: [B, ...] inputs -> list."""
     return [
-        verify_step(target_logits[b], draft_logits[b], draft_tokens[b], uniforms[b], temperature, lenience)
+        verify_step(target_logits[b], draft_logits[b], draft_tokens[b], uniforms[b], temperature, lenience, top_k)
         for b in range(len(target_logits))
     ]
 
 
-def sample_token(logits, u, temperature):
+def sample_token(logits, u, temperature, top_k=0):
     """A plain draw from the standardised distribution: (token, cdf margin).
 
     This is how the draft model draws x_i ~ q_i and how target-only decoding
@@ -198,24 +224,24 @@ def sample_token(logits, u, temperature):
     z = np.asarray(logits, dtype=np.float64)
     if temperature == 0:
         return int(np.argmax(z)), float("inf")
-    w = np.exp((z - z.max()) / float(temperature))
+    w = np.exp((keep_top_k(z, top_k) - z.max()) / float(temperature))
     return inverse_cdf(w, u)
 
 
-def sample_trials(logits, uniforms, temperature):
+def sample_trials(logits, uniforms, temperature, top_k=0):
     """`sample_token` for many uniforms that share one row of logits -> [N]."""
     z = np.asarray(logits, dtype=np.float64)
     us = np.asarray(uniforms, dtype=np.float64)
     if temperature == 0:
         return np.full(us.shape[0], int(np.argmax(z)), dtype=np.int64)
-    w = np.exp((z - z.max()) / float(temperature))
+    w = np.exp((keep_top_k(z, top_k) - z.max()) / float(temperature))
     running = np.cumsum(w)
     k = np.searchsorted(running, us * running[-1], side="right")
     positive = np.nonzero(w > 0.0)[0]
     return np.where(k >= w.shape[0], positive[-1], k).astype(np.int64)
 
 
-def verify_trials(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0):
+def verify_trials(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0, top_k=0):
     """Many independent trials of `verify_step` that share one set of logits.
 
     target_logits [gamma+1, V] and draft_logits [gamma, V] are fixed;
@@ -230,8 +256,8 @@ def verify_trials(target_logits, draft_logits, draft_tokens, uniforms, temperatu
     us = np.asarray(uniforms, dtype=np.float64)
     gamma = tl.shape[0] - 1
     trials = us.shape[0]
-    p = np.stack([standardise(tl[i], temperature) for i in range(gamma + 1)])
-    q = np.stack([standardise(ql[i], temperature) for i in range(gamma)]) if gamma else np.zeros((0, tl.shape[1]))
+    p = np.stack([standardise(tl[i], temperature, top_k) for i in range(gamma + 1)])
+    q = np.stack([standardise(ql[i], temperature, top_k) for i in range(gamma)]) if gamma else np.zeros((0, tl.shape[1]))
 
     n = np.full(trials, gamma, dtype=np.int64)
     undecided = np.ones(trials, dtype=bool)

@@ -308,3 +308,74 @@ def test_lenience_at_temperature_zero():
         draft[0, x] = 5.0
         accepted.append(sampling.verify_step(tl, draft, [x], [0.5, 0.5], 0.0, 1.0).n_accepted)
     assert accepted == [1 if x == best else 0 for x in range(16)]
+
+
+def _top_k_by_repeated_argmax(row, k):
+    """Indices of a top-k set found by taking the maximum k times (no sort, no threshold)."""
+    left = np.array(row, dtype=np.float64)
+    chosen = []
+    for _ in range(k):
+        i = int(np.argmax(left))
+        chosen.append(i)
+        left[i] = -np.inf
+    return chosen
+
+
+@pytest.mark.parametrize("k", [1, 2, 7, 63])
+def test_top_k_support_and_ratios(k):
+    tl, _ = _fixed_pair(1.0)
+    row = tl[0]  # drawn from a continuous law: no ties
+    for T in (1.0, 0.6):
+        p_all = sampling.standardise(row, T)
+        p_k = sampling.standardise(row, T, top_k=k)
+        chosen = _top_k_by_repeated_argmax(row, k)
+        assert sorted(np.nonzero(p_k)[0].tolist()) == sorted(chosen)
+        assert p_k.sum() == pytest.approx(1.0, abs=1e-12)
+        # inside the support the ratios of the plain softmax survive
+        assert np.allclose(p_k[chosen] / p_k[chosen[0]], p_all[chosen] / p_all[chosen[0]], rtol=1e-12)
+    assert sampling.top_k_floor(row, k) == row[chosen[-1]]
+
+
+def test_top_k_edge_cases():
+    tl, _ = _fixed_pair(1.0)
+    row = tl[0]
+    plain = sampling.standardise(row, 0.8)
+    for k in (0, VOCAB, VOCAB + 5):
+        assert np.array_equal(sampling.standardise(row, 0.8, top_k=k), plain)
+    one = sampling.standardise(row, 0.8, top_k=1)
+    assert np.array_equal(one, sampling.standardise(row, 0.0))
+    # entries tied with the k-th largest all stay
+    tied = np.array([0.0, 2.0, 1.0, 1.0, -1.0, 1.0])
+    assert np.nonzero(sampling.standardise(tied, 1.0, top_k=2))[0].tolist() == [1, 2, 3, 5]
+    assert np.nonzero(sampling.standardise(tied, 1.0, top_k=1))[0].tolist() == [1]
+    # T = 0 ignores k
+    assert np.array_equal(sampling.standardise(tied, 0.0, top_k=3), sampling.standardise(tied, 0.0))
+    # a plain draw never leaves the support
+    us = philox.uniforms_vec(9, np.arange(20000), 0, philox.PURPOSE_DRAFT)
+    drawn = sampling.sample_trials(row, us, 1.0, top_k=5)
+    assert set(drawn.tolist()) <= set(_top_k_by_repeated_argmax(row, 5))
+    assert [sampling.sample_token(row, float(u), 1.0, top_k=5)[0] for u in us[:200]] == drawn[:200].tolist()
+
+
+@pytest.mark.parametrize("k", [3, 12])
+def test_emitted_law_under_top_k_is_the_top_k_target_distribution(k):
+    """Section 2.2 with Appendix A.1: both models standardised the same way, output law = adjusted p."""
+    trials = 400_000
+    tl, ql = _fixed_pair(1.0)
+    p = sampling.standardise(tl[0], 1.0, top_k=k)
+    q = sampling.standardise(ql[0], 1.0, top_k=k)
+    idx = np.arange(trials)
+    x = sampling.sample_trials(ql[0], philox.uniforms_vec(6, idx, 0, philox.PURPOSE_DRAFT), 1.0, top_k=k)
+    r = philox.uniforms_vec(6, idx, 0, philox.PURPOSE_ACCEPT)
+    u = philox.uniforms_vec(6, idx, 0, philox.PURPOSE_FINAL)
+    n, t = sampling.verify_trials(tl, ql, x[:, None], np.stack([r, u], axis=1), 1.0, top_k=k)
+    assert _chi_square_p(np.bincount(x, minlength=VOCAB), q) > 1e-3
+    first = np.where(n == 1, x, t)
+    assert np.all(p[first] > 0)
+    assert _chi_square_p(np.bincount(first, minlength=VOCAB), p) > 1e-3
+    beta = analysis.beta(p, q)
+    assert abs((n == 1).mean() - beta) < 4 * np.sqrt(beta * (1 - beta) / trials)
+    # the vectorised trials are the scalar step
+    for i in range(300):
+        res = sampling.verify_step(tl, ql, x[i : i + 1], [r[i], u[i]], 1.0, top_k=k)
+        assert (res.n_accepted, res.next_token) == (n[i], t[i])
