@@ -109,6 +109,29 @@ int spec_verify_sample_lenient(const float* target_logits, const float* draft_lo
                                int32_t* n_accepted, int32_t* next_token,
                                void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same with top-k standardisation (Section 2.2 lists top-k among the
+ * sampling methods that are a draw from an adjusted distribution and asks that
+ * both models be standardised the same way; it gives no definition).  With
+ * 0 < top_k < vocab and T > 0, every logit below the top_k-th largest logit of
+ * its own row reads as -inf, for the target's rows and the draft's alike,
+ * before the temperature softmax; logits equal to the top_k-th largest all
+ * stay, so ties can keep more than top_k.  top_k == 0 or >= vocab, or T == 0
+ * (the maximum is always kept), is spec_verify_sample_lenient exactly.  A
+ * drafted token outside the target's top-k set has p_i(x_i) = 0 and is rejected
+ * unless q_i(x_i) is 0 too.  Enqueues one more kernel (the per-row selection)
+ * before the other two; same workspace, errors as above plus SPEC_ERR_BAD_ARG
+ * for top_k < 0. */
+int spec_verify_sample_topk(const float* target_logits, const float* draft_logits,
+                            const int32_t* draft_tokens, const float* uniforms,
+                            int batch, int gamma, int vocab, float temperature, float lenience,
+                            int top_k, int32_t* n_accepted, int32_t* next_token,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/* floors[r] = the top_k-th largest value of row r of logits [rows, vocab] (fp32
+ * device in, fp32 device out), 1 <= top_k <= vocab: the threshold that the
+ * top-k variants apply.  Exact (comparisons only).  One kernel on `stream`. */
+int spec_top_k_floors(const float* logits, int rows, int vocab, int top_k, float* floors, void* stream);
+
 /* ------------------------------------------------------------------------- *
  * spec_verify_sample for callers that cannot allocate device memory.  (The
  * paper has no counterpart: this is a property of the library, not of the
@@ -158,6 +181,13 @@ int spec_verify_sample_static(const float* target_logits, const float* draft_log
  * ------------------------------------------------------------------------- */
 int spec_sample(const float* logits, const float* uniforms, int rows, int vocab,
                 float temperature, int32_t* tokens, void* stream);
+
+/* The same over the top_k largest logits of each row (see
+ * spec_verify_sample_topk); floors [rows] fp32 device is scratch that receives
+ * the rows' thresholds (may be NULL when top_k == 0, top_k >= vocab or T == 0,
+ * where the call is spec_sample).  Two kernels. */
+int spec_sample_topk(const float* logits, const float* uniforms, int rows, int vocab,
+                     float temperature, int top_k, int32_t* tokens, float* floors, void* stream);
 
 /* ------------------------------------------------------------------------- *
  * Uniforms of the method's counter-based generator, on the device.
@@ -355,6 +385,13 @@ int spec_begin(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, 
  * generations that start after this call; 1 (the default) is Algorithm 1 as
  * printed.  Errors: SPEC_ERR_BAD_ARG outside (0, 1]. */
 int spec_set_lenience(spec_ctx* ctx, float lenience);
+
+/* top-k standardisation (see spec_verify_sample_topk) of both models in the
+ * generations that start after this call: the draft draws x_i from its top-k
+ * distribution, the accept tests and the final draw use the target's and the
+ * draft's top-k distributions, and gamma = 0 decodes from the target's.  0 (the
+ * default): the whole vocabulary.  Errors: SPEC_ERR_BAD_ARG for top_k < 0. */
+int spec_set_top_k(spec_ctx* ctx, int top_k);
 
 /* Timing instrument (no counterpart in Algorithm 1): from the next spec_begin /
  * spec_generate on, the accept decision of every drafted token is replaced by

@@ -46,11 +46,14 @@ struct spec_ctx {
     struct Params { unsigned long long seed; int n_new; float imposed_alpha; }* params = nullptr;
     float imposed_alpha = -1.0f;  // >= 0: timing instrument, see spec_set_imposed_acceptance
     float lenience = 1.0f;        // Appendix A.5; 1 = Algorithm 1 as printed
+    int top_k = 0;                // Section 2.2: both models standardised over their k largest logits; 0 = all
+    float* sample_floors = nullptr;  // the draft rows' k-th largest logits, one per sequence
 
     // cached iteration graph
     cudaGraphExec_t graph = nullptr;
     int graph_batch = -1, graph_gamma = -1;
     float graph_temperature = -1.0f, graph_lenience = 1.0f;
+    int graph_top_k = 0;
 
     // generation in progress (spec_begin / spec_generate)
     int session_batch = 0, session_gamma = 0, session_n_new = 0;
@@ -400,14 +403,15 @@ int enqueue_iteration(spec_ctx* ctx, int batch, int gamma, float temperature) {
         // x_step ~ q_step for every sequence
         SPEC_TRY(launch_sample_strided(ctx->draft_logits + static_cast<size_t>(step - 1) * vocab,
                                        static_cast<size_t>(gamma) * vocab, ctx->draft_u + (step - 1), gamma, batch,
-                                       vocab, temperature, ctx->draft_tokens + (step - 1), gamma, st));
+                                       vocab, temperature, ctx->top_k, ctx->sample_floors,
+                                       ctx->draft_tokens + (step - 1), gamma, st));
     }
     SPEC_TRY(launch_pdl(prep_verify_kernel, dim3(blocks_bg), dim3(threads), 0, st, ctx->tokens, ctx->draft_tokens,
                         ctx->length, batch, gamma, ctx->rt.max_len, ctx->row_token, ctx->row_pos, ctx->row_seq));
     SPEC_TRY(forward(ctx, ctx->model[0], batch, gamma + 1, batch * (gamma + 1), nullptr, nullptr, ctx->target_logits));
     SPEC_TRY(launch_verify_sample(ctx->target_logits, ctx->draft_logits, ctx->draft_tokens, ctx->accept_u, ctx->final_u,
-                                  batch, gamma, vocab, temperature, ctx->lenience, ctx->n_accepted, ctx->next_token,
-                                  ctx->sampler_ws, st));
+                                  batch, gamma, vocab, temperature, ctx->lenience, ctx->top_k, ctx->n_accepted,
+                                  ctx->next_token, ctx->sampler_ws, st));
     return launch_pdl(commit_kernel, dim3(blocks_b), dim3(threads), 0, st, ctx->params, ctx->draft_tokens,
                       ctx->n_accepted, ctx->next_token, ctx->accept_u, ctx->prompt_len, batch, gamma, ctx->rt.max_len,
                       ctx->tokens, ctx->length, ctx->counters);
@@ -415,7 +419,7 @@ int enqueue_iteration(spec_ctx* ctx, int batch, int gamma, float temperature) {
 
 int build_graph(spec_ctx* ctx, int batch, int gamma, float temperature) {
     if (ctx->graph && ctx->graph_batch == batch && ctx->graph_gamma == gamma && ctx->graph_temperature == temperature &&
-        ctx->graph_lenience == ctx->lenience)
+        ctx->graph_lenience == ctx->lenience && ctx->graph_top_k == ctx->top_k)
         return SPEC_OK;
     if (ctx->graph) {
         cudaGraphExecDestroy(ctx->graph);
@@ -437,6 +441,7 @@ int build_graph(spec_ctx* ctx, int batch, int gamma, float temperature) {
     ctx->graph_gamma = gamma;
     ctx->graph_temperature = temperature;
     ctx->graph_lenience = ctx->lenience;
+    ctx->graph_top_k = ctx->top_k;
     return SPEC_OK;
 }
 
@@ -753,6 +758,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     SPEC_ALLOC(final_u, B * (G + 1));
     SPEC_ALLOC(counters, 4);
     SPEC_ALLOC(params, 1);
+    SPEC_ALLOC(sample_floors, B);
     {
         char* ws = nullptr;
         if ((status = dev_alloc(ctx, &ws, verify_sample_workspace_bytes(static_cast<int>(B), static_cast<int>(G), static_cast<int>(V)))) != SPEC_OK)
@@ -989,6 +995,12 @@ extern "C" int spec_read_tokens(spec_ctx* ctx, int32_t* out_tokens) {
 extern "C" int spec_set_lenience(spec_ctx* ctx, float lenience) {
     if (!ctx || !(lenience > 0.0f) || !(lenience <= 1.0f)) return fail(SPEC_ERR_BAD_ARG, "spec_set_lenience: lenience must be in (0, 1]");
     ctx->lenience = lenience;
+    return SPEC_OK;
+}
+
+extern "C" int spec_set_top_k(spec_ctx* ctx, int top_k) {
+    if (!ctx || top_k < 0) return fail(SPEC_ERR_BAD_ARG, "spec_set_top_k: top_k must be >= 0 (0: the whole vocabulary)");
+    ctx->top_k = top_k;
     return SPEC_OK;
 }
 

@@ -51,13 +51,17 @@ __device__ __forceinline__ float fast_exp2(float x) {
 // A row of fp32 logits addressed in groups of four elements.  VEC: the vocabulary
 // is a multiple of four and every row starts on a 16-byte boundary, so a group
 // is one unconditional 128-bit load.  Otherwise four guarded scalar loads, with
-// elements past the end of the row reading as `pad`.
-template <bool VEC>
+// elements past the end of the row reading as `pad`.  Logits below `floor` read
+// as -inf: that is top-k standardisation (Section 2.2) with `floor` the row's
+// k-th largest logit, and no change with floor = -inf.
+template <bool VEC, bool CUT = false>
 struct Row {
     const float* base;
     int vocab;
+    float floor;  // used only with CUT, so that the usual path pays nothing for it
 
-    __device__ __forceinline__ float4 load(int g, float pad) const {
+    __device__ __forceinline__ float kept(float v) const { return (!CUT || v >= floor) ? v : -INFINITY; }
+    __device__ __forceinline__ float4 raw(int g, float pad) const {
         if (VEC) return __ldg(reinterpret_cast<const float4*>(base) + g);
         const int j = 4 * g;
         float4 v;
@@ -67,13 +71,19 @@ struct Row {
         v.w = j + 3 < vocab ? __ldg(base + j + 3) : pad;
         return v;
     }
+    __device__ __forceinline__ float4 load(int g, float pad) const {
+        const float4 v = raw(g, pad);
+        if (!CUT) return v;
+        return make_float4(kept(v.x), kept(v.y), kept(v.z), kept(v.w));
+    }
 };
 
-template <bool VEC>
-__device__ __forceinline__ Row<VEC> make_row(const float* base, int vocab) {
-    Row<VEC> r;
+template <bool VEC, bool CUT = false>
+__device__ __forceinline__ Row<VEC, CUT> make_row(const float* base, int vocab, float floor = -INFINITY) {
+    Row<VEC, CUT> r;
     r.base = base;
     r.vocab = vocab;
+    r.floor = floor;
     return r;
 }
 
@@ -82,10 +92,10 @@ __device__ __forceinline__ Row<VEC> make_row(const float* base, int vocab) {
 // consumes any of them.
 
 // Unnormalised softmax weights exp((l - max) / T) of one row; c2 = log2(e) / T.
-template <bool VEC>
+template <bool VEC, bool CUT = false>
 struct PlainWeights {
     struct Raw { float4 a; };
-    Row<VEC> p;
+    Row<VEC, CUT> p;
     float max_p, c2;
     __device__ __forceinline__ Raw fetch(int g) const { return Raw{p.load(g, -INFINITY)}; }
     __device__ __forceinline__ Raw nothing() const {
@@ -100,10 +110,10 @@ struct PlainWeights {
 
 // max(0, p - q) with p, q the normalised softmaxes of two rows (Algorithm 1's
 // adjusted distribution before normalisation).
-template <bool VEC>
+template <bool VEC, bool CUT = false>
 struct ResidualWeights {
     struct Raw { float4 a, b; };
-    Row<VEC> p, q;
+    Row<VEC, CUT> p, q;
     float max_p, max_q, inv_sum_p, inv_sum_q, c2;
     __device__ __forceinline__ Raw fetch(int g) const { return Raw{p.load(g, -INFINITY), q.load(g, -INFINITY)}; }
     __device__ __forceinline__ Raw nothing() const {
@@ -389,11 +399,11 @@ struct __align__(16) ChunkStat {
 
 // grid = (chunks, rows, batch); rows = 2*gamma+1 (T > 0: p_1..p_{gamma+1}, q_1..q_gamma)
 // or gamma+1 (T = 0: only p is read).
-template <bool GREEDY, bool VEC>
+template <bool GREEDY, bool VEC, bool CUT>
 __global__ void __launch_bounds__(kStatThreads)
 verify_stats_kernel(const float* __restrict__ target_logits, const float* __restrict__ draft_logits,
                     const int32_t* __restrict__ draft_tokens, int gamma, int vocab, float c2,
-                    ChunkStat* __restrict__ stats) {
+                    const float* __restrict__ floors, ChunkStat* __restrict__ stats) {
     __shared__ float red[kStatWarps];
     __shared__ float red_s[kStatWarps];
     __shared__ int red_i[kStatWarps];
@@ -407,7 +417,8 @@ verify_stats_kernel(const float* __restrict__ target_logits, const float* __rest
     const float* src = row <= gamma
         ? target_logits + (static_cast<size_t>(b) * (gamma + 1) + row) * vocab
         : draft_logits + (static_cast<size_t>(b) * gamma + (row - gamma - 1)) * vocab;
-    const Row<VEC> r = make_row<VEC>(src, vocab);
+    const float floor = CUT ? __ldcg(floors + static_cast<size_t>(b) * rows + row) : -INFINITY;
+    const Row<VEC, CUT> r = make_row<VEC, CUT>(src, vocab, floor);
     const int groups = (vocab + 3) >> 2;
     const int per_chunk = (groups + chunks - 1) / chunks;
     const int g0 = chunk * per_chunk;
@@ -419,7 +430,7 @@ verify_stats_kernel(const float* __restrict__ target_logits, const float* __rest
     float xlogit = 0.0f;
     if (tid == 0 && !GREEDY && row != gamma) {
         const int x = draft_tokens[static_cast<size_t>(b) * gamma + (row < gamma ? row : row - gamma - 1)];
-        if (x >= 4 * g0 && x < min(vocab, 4 * g1)) xlogit = __ldg(src + x);
+        if (x >= 4 * g0 && x < min(vocab, 4 * g1)) xlogit = r.kept(__ldg(src + x));
     }
 
     // Every thread streams groups g0+tid, g0+tid+T, ... with kUnroll 128-bit
@@ -492,13 +503,13 @@ struct FinishShared {
 // after the statistics: merge, accept tests, adjusted distribution, draw.  The
 // cheap decision part is repeated in every CTA of the cluster; the pass over
 // row n+1 is split between them.
-template <bool GREEDY, bool VEC>
+template <bool GREEDY, bool VEC, bool CUT>
 __global__ void __launch_bounds__(kFinishThreads, 2)
 verify_finish_kernel(const float* __restrict__ target_logits, const float* __restrict__ draft_logits,
                      const int32_t* __restrict__ draft_tokens, const float* __restrict__ uniforms, int gamma,
                      int vocab, float inv_t, int chunks, int cluster_size, const ChunkStat* __restrict__ stats,
-                     const float* __restrict__ final_uniforms, float lenience, int32_t* __restrict__ n_accepted,
-                     int32_t* __restrict__ next_token) {
+                     const float* __restrict__ final_uniforms, float lenience, const float* __restrict__ floors,
+                     int32_t* __restrict__ n_accepted, int32_t* __restrict__ next_token) {
     __shared__ FinishShared sh;
     const int tid = threadIdx.x;
     const int b = blockIdx.x / cluster_size;
@@ -586,16 +597,17 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
         // The generation loop keys the final draw by the position it decides, which
         // depends on n: it passes one candidate uniform per possible n.
         const float u = final_uniforms ? __ldg(final_uniforms + static_cast<size_t>(b) * (gamma + 1) + n) : sh.u_final;
-        PlainWeights<VEC> pw;
-        pw.p = make_row<VEC>(tl + static_cast<size_t>(n) * vocab, vocab);
+        PlainWeights<VEC, CUT> pw;
+        const float* fl = CUT ? floors + static_cast<size_t>(b) * rows : nullptr;
+        pw.p = make_row<VEC, CUT>(tl + static_cast<size_t>(n) * vocab, vocab, CUT ? __ldcg(fl + n) : -INFINITY);
         pw.max_p = sh.row_max[n];
         pw.c2 = c2;
         float total = 0.0f;
         bool plain = n == gamma;
         if (!plain) {
-            ResidualWeights<VEC> rw;
+            ResidualWeights<VEC, CUT> rw;
             rw.p = pw.p;
-            rw.q = make_row<VEC>(ql + static_cast<size_t>(n) * vocab, vocab);
+            rw.q = make_row<VEC, CUT>(ql + static_cast<size_t>(n) * vocab, vocab, CUT ? __ldcg(fl + gamma + 1 + n) : -INFINITY);
             rw.max_p = sh.row_max[n];
             rw.max_q = sh.row_max[gamma + 1 + n];
             rw.inv_sum_p = 1.0f / sh.row_aux[n];
@@ -613,11 +625,11 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
 }
 
 // One CTA per row: tokens[r] ~ softmax(logits[r] / T), or argmax at T = 0.
-template <bool VEC>
+template <bool VEC, bool CUT>
 __global__ void __launch_bounds__(kSampleThreads)
 sample_kernel(const float* __restrict__ logits, size_t logit_stride, const float* __restrict__ uniforms,
-              int uniform_stride, int vocab, float inv_t, bool greedy, int32_t* __restrict__ tokens,
-              int token_stride) {
+              int uniform_stride, int vocab, float inv_t, bool greedy, const float* __restrict__ floors,
+              int32_t* __restrict__ tokens, int token_stride) {
     constexpr int W = kSampleThreads / 32;
     __shared__ float red[W];
     __shared__ int red_i[W];
@@ -627,7 +639,8 @@ sample_kernel(const float* __restrict__ logits, size_t logit_stride, const float
     pdl_trigger();
     pdl_wait();
     const int tid = threadIdx.x;
-    const Row<VEC> r = make_row<VEC>(logits + static_cast<size_t>(blockIdx.x) * logit_stride, vocab);
+    const Row<VEC, CUT> r = make_row<VEC, CUT>(logits + static_cast<size_t>(blockIdx.x) * logit_stride, vocab,
+                                               CUT ? __ldcg(floors + blockIdx.x) : -INFINITY);
     const int groups = (vocab + 3) >> 2;
     float m = -FLT_MAX;
     int arg = 0x7fffffff;
@@ -645,7 +658,7 @@ sample_kernel(const float* __restrict__ logits, size_t logit_stride, const float
     __syncthreads();
     int token = s_arg;
     if (!greedy) {
-        PlainWeights<VEC> pw;
+        PlainWeights<VEC, CUT> pw;
         pw.p = r;
         pw.max_p = s_max;
         pw.c2 = inv_t * kLog2e;
@@ -653,6 +666,148 @@ sample_kernel(const float* __restrict__ logits, size_t logit_stride, const float
         token = block_inverse_cdf<W>(pw, vocab, uniforms[blockIdx.x * uniform_stride], cdf, &total);
     }
     if (tid == 0) tokens[blockIdx.x * token_stride] = max(0, min(token, vocab - 1));
+}
+
+// ---- top-k: the k-th largest logit of every row --------------------------------
+constexpr int kFloorThreads = 512;
+
+// Unsigned keys that order like the floats they come from.
+__device__ __forceinline__ uint32_t float_key(float v) {
+    const uint32_t u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
+}
+
+// One CTA per row.  The k-th largest key is the largest value t with
+// count(key >= t) >= k; its 32 bits are fixed from the top, one block-wide count
+// per bit.  Keys whose upper bits differ from the bits fixed so far are settled
+// (above: counted once and for all; below: out), so as soon as at most kLiveCap
+// keys remain undecided they are copied to shared memory and the remaining
+// bits look at those alone.  KPT > 0: the row (at most kFloorThreads * KPT
+// logits) is read once and its keys stay in registers; KPT = 0: any length,
+// re-read per bit until the copy (the row stays in L2).  Rows come from two
+// arrays: sequence s owns a_rows consecutive rows of `a`, then b_rows of `b`;
+// floors has the same order.
+constexpr int kLiveCap = 2048;
+
+template <bool VEC, int KPT>
+__global__ void __launch_bounds__(kFloorThreads, 1)
+topk_floor_kernel(const float* __restrict__ a, size_t a_stride, int a_rows, const float* __restrict__ b,
+                  size_t b_stride, int b_rows, int vocab, int top_k, float* __restrict__ floors) {
+    __shared__ unsigned counts[32];
+    __shared__ unsigned n_live;
+    __shared__ uint32_t live[kLiveCap];
+    pdl_trigger();
+    pdl_wait();
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int per_seq = a_rows + b_rows;
+    const int seq = blockIdx.x / per_seq, row = blockIdx.x % per_seq;
+    const float* src = row < a_rows ? a + (static_cast<size_t>(seq) * a_rows + row) * a_stride
+                                    : b + (static_cast<size_t>(seq) * b_rows + (row - a_rows)) * b_stride;
+    const Row<VEC> r = make_row<VEC>(src, vocab);
+    const int groups = (vocab + 3) >> 2;
+    if (tid < 32) counts[tid] = 0;
+    if (tid == 0) n_live = 0;
+
+    constexpr int G = KPT > 0 ? KPT / 4 : 1;
+    uint32_t keys[4 * G];
+    if (KPT > 0) {
+#pragma unroll
+        for (int i = 0; i < G; ++i) {
+            const int g = tid + i * kFloorThreads;
+            // past the end of the row: -inf, below every threshold that k <= vocab can give
+            const float4 v = g < groups ? r.raw(g, -INFINITY) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            keys[4 * i + 0] = float_key(v.x);
+            keys[4 * i + 1] = float_key(v.y);
+            keys[4 * i + 2] = float_key(v.z);
+            keys[4 * i + 3] = float_key(v.w);
+        }
+    }
+    __syncthreads();
+
+    const unsigned k = static_cast<unsigned>(top_k);
+    uint32_t prefix = 0;
+    // count(key >= prefix) and count(key >= prefix + 2^(bit+1)): the keys between the two are undecided
+    unsigned at_prefix = KPT > 0 ? 4u * G * kFloorThreads : 4u * groups;
+    unsigned above = 0;
+    int bit = 31;
+    for (; bit >= 0 && at_prefix - above > kLiveCap; --bit) {
+        const uint32_t cand = prefix | (1u << bit);
+        unsigned c = 0;
+        if (KPT > 0) {
+#pragma unroll
+            for (int i = 0; i < 4 * G; ++i) c += keys[i] >= cand;
+        } else {
+            for (int g = tid; g < groups; g += kFloorThreads) {
+                const float4 v = r.raw(g, -INFINITY);
+                c += (float_key(v.x) >= cand) + (float_key(v.y) >= cand) + (float_key(v.z) >= cand) +
+                     (float_key(v.w) >= cand);
+            }
+        }
+        c = __reduce_add_sync(0xffffffffu, c);
+        if (lane == 0 && c) atomicAdd(&counts[bit], c);
+        __syncthreads();
+        const unsigned total = counts[bit];
+        if (total >= k) { prefix = cand; at_prefix = total; } else { above = total; }
+    }
+    if (bit >= 0) {
+        // undecided: the keys that agree with `prefix` on every bit above `bit`
+        const int shift = bit + 1;
+        auto undecided = [&](uint32_t key) { return shift >= 32 || ((key ^ prefix) >> shift) == 0; };
+        // each thread counts its own, one scan per warp and one atomic per warp place them
+        unsigned mine = 0;
+        if (KPT > 0) {
+#pragma unroll
+            for (int i = 0; i < 4 * G; ++i) mine += undecided(keys[i]);
+        } else {
+            for (int g = tid; g < groups; g += kFloorThreads) {
+                const float4 v = r.raw(g, -INFINITY);
+                mine += undecided(float_key(v.x)) + undecided(float_key(v.y)) + undecided(float_key(v.z)) +
+                        undecided(float_key(v.w));
+            }
+        }
+        unsigned incl = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        unsigned base = 0;
+        if (lane == 31 && incl) base = atomicAdd(&n_live, incl);
+        unsigned pos = __shfl_sync(0xffffffffu, base, 31) + incl - mine;
+        auto keep = [&](uint32_t key) {
+            if (undecided(key)) {
+                if (pos < kLiveCap) live[pos] = key;
+                ++pos;
+            }
+        };
+        if (KPT > 0) {
+#pragma unroll
+            for (int i = 0; i < 4 * G; ++i) keep(keys[i]);
+        } else {
+            for (int g = tid; g < groups; g += kFloorThreads) {
+                const float4 v = r.raw(g, -INFINITY);
+                keep(float_key(v.x));
+                keep(float_key(v.y));
+                keep(float_key(v.z));
+                keep(float_key(v.w));
+            }
+        }
+        __syncthreads();
+        const int n = static_cast<int>(min(n_live, static_cast<unsigned>(kLiveCap)));  // = at_prefix - above
+        for (; bit >= 0; --bit) {
+            const uint32_t cand = prefix | (1u << bit);
+            unsigned c = 0;
+            for (int j = tid; j < n; j += kFloorThreads) c += live[j] >= cand;
+            c = __reduce_add_sync(0xffffffffu, c);
+            if (lane == 0 && c) atomicAdd(&counts[bit], c);
+            __syncthreads();
+            if (counts[bit] + above >= k) prefix = cand;
+        }
+    }
+    if (tid == 0) floors[blockIdx.x] = key_float(prefix);
 }
 
 __global__ void uniforms_kernel(uint64_t seed, const int32_t* __restrict__ positions,
@@ -685,34 +840,75 @@ int chunks_for(int vocab, int rows_total) {
     return std::max(1, std::min(want, max_chunks(vocab)));
 }
 
+size_t stats_bytes(int batch, int gamma, int vocab) {
+    const size_t rows = 2 * static_cast<size_t>(gamma) + 1;
+    return (static_cast<size_t>(batch) * rows * max_chunks(vocab) * sizeof(ChunkStat) + 255) & ~static_cast<size_t>(255);
+}
+
 }  // namespace
 
 // Shared with the generation loop: same launches, no argument checks.
+// Layout: chunk statistics, then one top-k floor per row.
 size_t verify_sample_workspace_bytes(int batch, int gamma, int vocab) {
     const size_t rows = 2 * static_cast<size_t>(gamma) + 1;
-    return static_cast<size_t>(batch) * rows * max_chunks(vocab) * sizeof(ChunkStat) + 256;
+    return stats_bytes(batch, gamma, vocab) + static_cast<size_t>(batch) * rows * sizeof(float) + 256;
+}
+
+// floors[s * (a_rows + b_rows) + r] = the top_k-th largest logit of sequence s's
+// row r (its a_rows rows of `a`, then its b_rows rows of `b`).  0 < top_k < vocab.
+int launch_topk_floors(const float* a, size_t a_stride, int a_rows, const float* b, size_t b_stride, int b_rows,
+                       int seqs, int vocab, int top_k, float* floors, cudaStream_t stream) {
+    const int total = seqs * (a_rows + b_rows);
+    if (total == 0) return SPEC_OK;
+    const bool vec = vocab % 4 == 0 && a_stride % 4 == 0 && aligned16(a) && (b_rows == 0 || (b_stride % 4 == 0 && aligned16(b)));
+#define SPEC_LAUNCH_FLOORS(V, K)                                                                              \
+    return launch_pdl(topk_floor_kernel<V, K>, dim3(total), dim3(kFloorThreads), 0, stream, a, a_stride, a_rows, b, \
+                      b_stride, b_rows, vocab, top_k, floors)
+    if (vocab <= kFloorThreads * 16) {
+        if (vec) SPEC_LAUNCH_FLOORS(true, 16);
+        SPEC_LAUNCH_FLOORS(false, 16);
+    }
+    if (vocab <= kFloorThreads * 64) {
+        if (vec) SPEC_LAUNCH_FLOORS(true, 64);
+        SPEC_LAUNCH_FLOORS(false, 64);
+    }
+    if (vec) SPEC_LAUNCH_FLOORS(true, 0);
+    SPEC_LAUNCH_FLOORS(false, 0);
+#undef SPEC_LAUNCH_FLOORS
 }
 
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
                          const float* uniforms, const float* final_uniforms, int batch, int gamma, int vocab,
-                         float temperature, float lenience, int32_t* n_accepted, int32_t* next_token, void* workspace,
-                         cudaStream_t stream) {
+                         float temperature, float lenience, int top_k, int32_t* n_accepted, int32_t* next_token,
+                         void* workspace, cudaStream_t stream) {
     const bool greedy = temperature == 0.0f;
     const int rows = greedy ? gamma + 1 : 2 * gamma + 1;
     const int chunks = chunks_for(vocab, rows * batch);
     const float inv_t = greedy ? 0.0f : 1.0f / temperature;
     ChunkStat* stats = static_cast<ChunkStat*>(workspace);
+    // top-k (Section 2.2): both models' rows are cut at their own k-th largest logit
+    const float* floors = nullptr;
+    if (!greedy && top_k > 0 && top_k < vocab) {
+        float* f = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + stats_bytes(batch, gamma, vocab));
+        const int st = launch_topk_floors(target_logits, static_cast<size_t>(vocab), gamma + 1, draft_logits,
+                                          static_cast<size_t>(vocab), gamma, batch, vocab, top_k, f, stream);
+        if (st != SPEC_OK) return st;
+        floors = f;
+    }
     const dim3 grid(chunks, rows, batch);
     const bool vec = vocab % 4 == 0 && aligned16(target_logits) && (greedy || gamma == 0 || aligned16(draft_logits));
     const float c2 = inv_t * kLog2e;
     int status;
-#define SPEC_LAUNCH_STATS(G, V)                                                                                  \
-    status = launch_pdl(verify_stats_kernel<G, V>, grid, dim3(kStatThreads), 0, stream, target_logits, draft_logits, \
-                        draft_tokens, gamma, vocab, c2, stats)
-    if (greedy && vec) SPEC_LAUNCH_STATS(true, true);
-    else if (greedy) SPEC_LAUNCH_STATS(true, false);
-    else if (vec) SPEC_LAUNCH_STATS(false, true);
-    else SPEC_LAUNCH_STATS(false, false);
+    const bool cut = floors != nullptr;  // never with greedy
+#define SPEC_LAUNCH_STATS(G, V, C)                                                                               \
+    status = launch_pdl(verify_stats_kernel<G, V, C>, grid, dim3(kStatThreads), 0, stream, target_logits, draft_logits, \
+                        draft_tokens, gamma, vocab, c2, floors, stats)
+    if (greedy && vec) SPEC_LAUNCH_STATS(true, true, false);
+    else if (greedy) SPEC_LAUNCH_STATS(true, false, false);
+    else if (vec && cut) SPEC_LAUNCH_STATS(false, true, true);
+    else if (vec) SPEC_LAUNCH_STATS(false, true, false);
+    else if (cut) SPEC_LAUNCH_STATS(false, false, true);
+    else SPEC_LAUNCH_STATS(false, false, false);
 #undef SPEC_LAUNCH_STATS
     if (status != SPEC_OK) return status;
 
@@ -733,36 +929,49 @@ int launch_verify_sample(const float* target_logits, const float* draft_logits, 
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     const ChunkStat* stats_in = stats;
-#define SPEC_LAUNCH_FINISH(G, V)                                                                                  \
-    SPEC_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_finish_kernel<G, V>, target_logits, draft_logits, draft_tokens, \
-                                     uniforms, gamma, vocab, inv_t, chunks, cluster_size, stats_in,              \
-                                     final_uniforms, lenience, n_accepted, next_token))
-    if (greedy && vec) SPEC_LAUNCH_FINISH(true, true);
-    else if (greedy) SPEC_LAUNCH_FINISH(true, false);
-    else if (vec) SPEC_LAUNCH_FINISH(false, true);
-    else SPEC_LAUNCH_FINISH(false, false);
+#define SPEC_LAUNCH_FINISH(G, V, C)                                                                                  \
+    SPEC_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_finish_kernel<G, V, C>, target_logits, draft_logits, draft_tokens, \
+                                     uniforms, gamma, vocab, inv_t, chunks, cluster_size, stats_in,                 \
+                                     final_uniforms, lenience, floors, n_accepted, next_token))
+    if (greedy && vec) SPEC_LAUNCH_FINISH(true, true, false);
+    else if (greedy) SPEC_LAUNCH_FINISH(true, false, false);
+    else if (vec && cut) SPEC_LAUNCH_FINISH(false, true, true);
+    else if (vec) SPEC_LAUNCH_FINISH(false, true, false);
+    else if (cut) SPEC_LAUNCH_FINISH(false, false, true);
+    else SPEC_LAUNCH_FINISH(false, false, false);
 #undef SPEC_LAUNCH_FINISH
     return SPEC_OK;
 }
 
 // Row r reads logits + r * logit_stride and uniforms[r * uniform_stride] and
 // writes tokens[r * token_stride].
+// With 0 < top_k < vocab (and T > 0) `floor_scratch` must hold `rows` floats.
 int launch_sample_strided(const float* logits, size_t logit_stride, const float* uniforms, int uniform_stride,
-                          int rows, int vocab, float temperature, int32_t* tokens, int token_stride,
-                          cudaStream_t stream) {
+                          int rows, int vocab, float temperature, int top_k, float* floor_scratch, int32_t* tokens,
+                          int token_stride, cudaStream_t stream) {
     const bool greedy = temperature == 0.0f;
     const float inv_t = greedy ? 0.0f : 1.0f / temperature;
-    if (vocab % 4 == 0 && logit_stride % 4 == 0 && aligned16(logits))
-        return launch_pdl(sample_kernel<true>, dim3(rows), dim3(kSampleThreads), 0, stream, logits, logit_stride,
-                          uniforms, uniform_stride, vocab, inv_t, greedy, tokens, token_stride);
-    return launch_pdl(sample_kernel<false>, dim3(rows), dim3(kSampleThreads), 0, stream, logits, logit_stride, uniforms,
-                      uniform_stride, vocab, inv_t, greedy, tokens, token_stride);
+    const float* floors = nullptr;
+    if (!greedy && top_k > 0 && top_k < vocab) {
+        const int st = launch_topk_floors(logits, logit_stride, 1, nullptr, 0, 0, rows, vocab, top_k, floor_scratch, stream);
+        if (st != SPEC_OK) return st;
+        floors = floor_scratch;
+    }
+    const bool vec = vocab % 4 == 0 && logit_stride % 4 == 0 && aligned16(logits);
+#define SPEC_LAUNCH_SAMPLE(V, C)                                                                                   \
+    return launch_pdl(sample_kernel<V, C>, dim3(rows), dim3(kSampleThreads), 0, stream, logits, logit_stride, uniforms, \
+                      uniform_stride, vocab, inv_t, greedy, floors, tokens, token_stride)
+    if (vec && floors) SPEC_LAUNCH_SAMPLE(true, true);
+    if (vec) SPEC_LAUNCH_SAMPLE(true, false);
+    if (floors) SPEC_LAUNCH_SAMPLE(false, true);
+    SPEC_LAUNCH_SAMPLE(false, false);
+#undef SPEC_LAUNCH_SAMPLE
 }
 
-int launch_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
-                  int32_t* tokens, cudaStream_t stream) {
-    return launch_sample_strided(logits, static_cast<size_t>(vocab), uniforms, 1, rows, vocab, temperature, tokens, 1,
-                                 stream);
+int launch_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature, int top_k,
+                  float* floor_scratch, int32_t* tokens, cudaStream_t stream) {
+    return launch_sample_strided(logits, static_cast<size_t>(vocab), uniforms, 1, rows, vocab, temperature, top_k,
+                                 floor_scratch, tokens, 1, stream);
 }
 
 }  // namespace spec
@@ -772,11 +981,12 @@ extern "C" size_t spec_verify_sample_workspace_bytes(int batch, int gamma, int v
     return spec::verify_sample_workspace_bytes(batch, gamma, vocab);
 }
 
-extern "C" int spec_verify_sample_lenient(const float* target_logits, const float* draft_logits,
-                                          const int32_t* draft_tokens, const float* uniforms, int batch, int gamma,
-                                          int vocab, float temperature, float lenience, int32_t* n_accepted,
-                                          int32_t* next_token, void* workspace, size_t workspace_bytes, void* stream) {
+extern "C" int spec_verify_sample_topk(const float* target_logits, const float* draft_logits,
+                                       const int32_t* draft_tokens, const float* uniforms, int batch, int gamma,
+                                       int vocab, float temperature, float lenience, int top_k, int32_t* n_accepted,
+                                       int32_t* next_token, void* workspace, size_t workspace_bytes, void* stream) {
     using namespace spec;
+    if (top_k < 0) return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: top_k must be >= 0");
     if (!(lenience > 0.0f) || !(lenience <= 1.0f)) return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: lenience must be in (0, 1]");
     if (batch < 0 || gamma < 0 || gamma > kMaxGamma || vocab < 1)
         return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: batch=%d gamma=%d (max %d) vocab=%d", batch, gamma, kMaxGamma, vocab);
@@ -792,7 +1002,16 @@ extern "C" int spec_verify_sample_lenient(const float* target_logits, const floa
         (reinterpret_cast<uintptr_t>(workspace) & 255u))
         return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: workspace too small (%zu bytes) or not 256-byte aligned", workspace_bytes);
     return launch_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, nullptr, batch, gamma, vocab,
-                                temperature, lenience, n_accepted, next_token, workspace, static_cast<cudaStream_t>(stream));
+                                temperature, lenience, top_k, n_accepted, next_token, workspace,
+                                static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int spec_verify_sample_lenient(const float* target_logits, const float* draft_logits,
+                                          const int32_t* draft_tokens, const float* uniforms, int batch, int gamma,
+                                          int vocab, float temperature, float lenience, int32_t* n_accepted,
+                                          int32_t* next_token, void* workspace, size_t workspace_bytes, void* stream) {
+    return spec_verify_sample_topk(target_logits, draft_logits, draft_tokens, uniforms, batch, gamma, vocab, temperature,
+                                   lenience, 0, n_accepted, next_token, workspace, workspace_bytes, stream);
 }
 
 extern "C" int spec_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
@@ -862,7 +1081,7 @@ extern "C" int spec_verify_sample_static(const float* target_logits, const float
     const int status = static_stats_address(&scratch);
     if (status != SPEC_OK) return status;
     return launch_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, nullptr, batch, gamma, vocab,
-                                temperature, 1.0f, n_accepted, next_token, scratch, static_cast<cudaStream_t>(stream));
+                                temperature, 1.0f, 0, n_accepted, next_token, scratch, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int spec_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
@@ -873,7 +1092,30 @@ extern "C" int spec_sample(const float* logits, const float* uniforms, int rows,
         return fail(SPEC_ERR_BAD_ARG, "spec_sample: temperature must be finite and >= 0");
     if (rows == 0) return SPEC_OK;
     if (!logits || !tokens || (temperature > 0.0f && !uniforms)) return fail(SPEC_ERR_BAD_ARG, "spec_sample: null pointer");
-    return launch_sample(logits, uniforms, rows, vocab, temperature, tokens, static_cast<cudaStream_t>(stream));
+    return launch_sample(logits, uniforms, rows, vocab, temperature, 0, nullptr, tokens, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int spec_sample_topk(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
+                                int top_k, int32_t* tokens, float* floors, void* stream) {
+    using namespace spec;
+    if (rows < 0 || vocab < 1 || top_k < 0) return fail(SPEC_ERR_BAD_ARG, "spec_sample_topk: rows=%d vocab=%d top_k=%d", rows, vocab, top_k);
+    if (!(temperature >= 0.0f) || !isfinite(temperature))
+        return fail(SPEC_ERR_BAD_ARG, "spec_sample_topk: temperature must be finite and >= 0");
+    if (rows == 0) return SPEC_OK;
+    const bool cut = temperature > 0.0f && top_k > 0 && top_k < vocab;
+    if (!logits || !tokens || (temperature > 0.0f && !uniforms) || (cut && !floors))
+        return fail(SPEC_ERR_BAD_ARG, "spec_sample_topk: null pointer");
+    return launch_sample(logits, uniforms, rows, vocab, temperature, top_k, floors, tokens, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int spec_top_k_floors(const float* logits, int rows, int vocab, int top_k, float* floors, void* stream) {
+    using namespace spec;
+    if (rows < 0 || vocab < 1 || top_k < 1 || top_k > vocab)
+        return fail(SPEC_ERR_BAD_ARG, "spec_top_k_floors: rows=%d vocab=%d top_k=%d", rows, vocab, top_k);
+    if (rows == 0) return SPEC_OK;
+    if (!logits || !floors) return fail(SPEC_ERR_BAD_ARG, "spec_top_k_floors: null pointer");
+    return launch_topk_floors(logits, static_cast<size_t>(vocab), 1, nullptr, 0, 0, rows, vocab, top_k, floors,
+                              static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int spec_uniforms(uint64_t seed, const int32_t* positions, const int32_t* sequences, int purpose, int count,

@@ -15,7 +15,7 @@ def to_dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).to(dev())
 
 
-def compare_verify(n_gpu, t_gpu, tl, ql, xs, us, temperature, lenience=1.0):
+def compare_verify(n_gpu, t_gpu, tl, ql, xs, us, temperature, lenience=1.0, top_k=0):
     """Element-by-element comparison with the oracle.  Returns (flagged, total):
     sequences whose decision sat within MARGIN of a boundary and differed.  Any
     other difference raises."""
@@ -23,7 +23,7 @@ def compare_verify(n_gpu, t_gpu, tl, ql, xs, us, temperature, lenience=1.0):
     flagged = 0
     for b in range(tl.shape[0]):
         q_rows = ql[b] if ql is not None else np.zeros((0, tl.shape[2]))
-        ref = oracle_sampling.verify_step(tl[b], q_rows, xs[b], us[b], temperature, lenience)
+        ref = oracle_sampling.verify_step(tl[b], q_rows, xs[b], us[b], temperature, lenience, top_k)
         if (int(n_gpu[b]), int(t_gpu[b])) == (ref.n_accepted, ref.next_token):
             continue
         if temperature > 0:

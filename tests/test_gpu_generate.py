@@ -185,6 +185,49 @@ def test_lenient_generation_matches_the_oracle_and_accepts_more(tiny):
     assert lenient["tests_passed"] / lenient["tests_evaluated"] > strict["tests_passed"] / strict["tests_evaluated"]
 
 
+@pytest.mark.parametrize("gamma", [3, 0])
+def test_top_k_generation_matches_the_oracle(tiny, gamma):
+    """Section 2.2's top-k through the whole loop (gamma = 0: target-only decoding from the
+    target's top-k distribution): token stream equal to the oracle's with the same k, every
+    emitted token inside the target's top-k set, and a stream that differs from the uncut one."""
+    eng, target, draft, cfg = tiny
+    prompt = workloads.make_prompt(14, 10, cfg["vocab"])
+    k = 6
+    try:
+        eng.set_top_k(k)
+        if gamma:
+            ref = oracle_generate.speculative_generate(target, draft, prompt, 48, gamma, 1.0, seed=23, top_k=k, keep_logits=True)
+            want, records = ref.tokens, ref.iterations
+        else:
+            want, rows, margins = oracle_generate.target_only_generate(target, prompt, 48, 1.0, seed=23, top_k=k, keep_logits=True)
+        got, _ = eng.generate([prompt], 48, gamma, 1.0, 23)
+        got = got[0].tolist()
+        diff = next((i for i in range(48) if got[i] != want[i]), None)
+        if diff is not None:  # a decision, or the k-th largest logit, within tolerance of a boundary
+            if gamma:
+                index = len(prompt) + diff
+                it = next(i for i in records if i.start_len <= index <= i.start_len + i.n_accepted)
+                logits = np.concatenate([it.target_logits, it.draft_logits])
+                margin = min([it.accept_margin, it.cdf_margin] + list(it.draft_cdf_margins))
+            else:
+                logits, margin = rows[diff][None], margins[diff]
+            ordered = np.sort(logits, axis=1)
+            cut_gap = float((ordered[:, -k] - ordered[:, -k - 1]).min())
+            assert margin < 1e-3 or cut_gap < 1e-3
+        checked = diff if diff is not None else 48
+        assert checked >= 8
+        # every token up to the first difference lies in the top-k set of the oracle's target row
+        if gamma == 0:
+            for i in range(checked):
+                assert rows[i][got[i]] >= np.sort(rows[i])[-k]
+        with pytest.raises(binding.SpecError):
+            eng.set_top_k(-1)
+    finally:
+        eng.set_top_k(0)
+    uncut, _ = eng.generate([prompt], 48, gamma, 1.0, 23)
+    assert uncut[0].tolist() != got
+
+
 @pytest.mark.parametrize("temperature", [1.0, 0.0])
 def test_bigram_table_draft_matches_the_oracle(temperature):
     """The tiny fp32 target with a bigram table as its draft (no draft passes at all)."""

@@ -13,20 +13,21 @@ from paper_2211_17192_b200 import binding, workloads
 pytestmark = pytest.mark.gpu
 
 
-def _draft_tokens(ql, seed, temperature):
+def _draft_tokens(ql, seed, temperature, top_k=0):
     """x_i ~ q_i drawn by the oracle with seeded uniforms."""
     batch, gamma, _ = ql.shape
     draw = workloads.make_uniform_grid(seed, (batch, max(gamma, 1)))
     xs = np.zeros((batch, gamma), dtype=np.int32)
     for b in range(batch):
         for i in range(gamma):
-            xs[b, i] = oracle_sampling.sample_token(ql[b, i], draw[b, i], temperature)[0]
+            xs[b, i] = oracle_sampling.sample_token(ql[b, i], draw[b, i], temperature, top_k)[0]
     return xs, draw
 
 
-def _run(tl, ql, xs, us, temperature, lenience=1.0):
+def _run(tl, ql, xs, us, temperature, lenience=1.0, top_k=0):
     n, t = binding.spec_verify_sample(to_dev(tl), to_dev(ql) if ql.size else None,
-                                      to_dev(xs) if xs.size else None, to_dev(us), temperature, lenience=lenience)
+                                      to_dev(xs) if xs.size else None, to_dev(us), temperature, lenience=lenience,
+                                      top_k=top_k)
     torch.cuda.synchronize()
     return n, t
 
@@ -189,3 +190,70 @@ def test_plain_sampler(rows, vocab, temperature):
             assert margin < MARGIN
             flagged += 1
     assert flagged <= 1
+
+
+@pytest.mark.parametrize("rows,vocab", [(6, 7), (5, 1001), (9, 8192), (16, 32000), (4, 32128), (3, 50257), (2, 100003)])
+def test_top_k_floors_are_bit_exact(rows, vocab):
+    """The k-th largest logit of every row, for k across the range; also with heavy ties."""
+    logits, _ = workloads.make_sampler_logits(rows * 7 + vocab, rows, 0, vocab, 1.0)
+    logits = np.ascontiguousarray(logits[:, 0])
+    tied = np.round(logits * 2).astype(np.float32) / 2  # a few dozen distinct values, both signs and zero
+    tied[0, : min(3, vocab)] = -0.0
+    for data in (logits, tied):
+        d = to_dev(data)
+        for k in sorted({1, 2, min(40, vocab), max(1, vocab // 2), vocab - 1, vocab} - {0}):
+            got = binding.spec_top_k_floors(d, k).cpu().numpy()
+            want = np.sort(data, axis=1)[:, vocab - k]
+            assert np.array_equal(got, want), (vocab, k)
+            if 0 < k < vocab:
+                assert [oracle_sampling.top_k_floor(data[r], k) for r in range(rows)] == want.astype(np.float64).tolist()
+
+
+@pytest.mark.parametrize("batch,gamma,vocab,temperature,top_k", [
+    (64, 7, 32000, 1.0, 40),
+    (64, 7, 32000, 1.0, 1),     # both models one-hot: accepted iff the two maxima coincide
+    (8, 3, 8192, 0.7, 5),
+    (5, 2, 1001, 1.0, 10),      # scalar loads
+    (2, 3, 100003, 1.0, 50),    # rows re-read per bit
+    (7, 4, 4096, 1.0, 4096),    # k = V: no cut
+    (7, 4, 4096, 1.0, 5000),    # k > V: no cut
+    (6, 0, 32128, 1.0, 20),     # gamma = 0: plain top-k draw from p
+    (9, 4, 32000, 0.0, 3),      # T = 0 ignores k
+])
+def test_top_k_verify(batch, gamma, vocab, temperature, top_k):
+    tl, ql = workloads.make_sampler_logits(batch + gamma + vocab, batch, gamma, vocab, 1.0)
+    xs, _ = _draft_tokens(ql, 3, temperature, top_k)
+    us = workloads.make_uniform_grid(4, (batch, gamma + 1))
+    n, t = _run(tl, ql, xs, us, temperature, top_k=top_k)
+    flagged, _ = compare_verify(n, t, tl, ql, xs, us, temperature, top_k=top_k)
+    assert flagged <= 1
+    if temperature > 0 and 0 < top_k < vocab:
+        # every emitted token lies in the target's top-k set of its row
+        ns, ts = n.cpu().numpy(), t.cpu().numpy()
+        for b in range(batch):
+            row = tl[b, ns[b]]
+            assert row[ts[b]] >= np.sort(row)[vocab - top_k]
+        plain_n, _ = _run(tl, ql, xs, us, temperature)
+        if top_k == 1:
+            same = (tl[:, :gamma].argmax(-1) == ql.argmax(-1)) if gamma else np.zeros((batch, 0), bool)
+            want = [int(np.argmin(np.append(same[b], False))) for b in range(batch)]
+            assert ns.tolist() == want
+        del plain_n
+
+
+@pytest.mark.parametrize("rows,vocab,temperature,top_k", [(64, 8192, 1.0, 50), (5, 1001, 0.5, 3), (3, 7, 1.0, 2),
+                                                          (16, 32000, 1.0, 1), (2, 100003, 1.0, 40), (4, 32000, 0.0, 5)])
+def test_plain_sampler_top_k(rows, vocab, temperature, top_k):
+    logits, _ = workloads.make_sampler_logits(rows + vocab, rows, 0, vocab, 1.0)
+    logits = logits[:, 0]
+    us = workloads.make_uniform_grid(12, (rows,))
+    got = binding.spec_sample(to_dev(logits), to_dev(us), temperature, top_k=top_k).cpu().numpy()
+    flagged = 0
+    for r in range(rows):
+        ref, margin = oracle_sampling.sample_token(logits[r], us[r], temperature, top_k)
+        if got[r] != ref:
+            assert margin < MARGIN
+            flagged += 1
+    assert flagged <= 1
+    if top_k == 1:
+        assert got.tolist() == logits.argmax(-1).tolist()
