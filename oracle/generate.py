@@ -66,7 +66,7 @@ class GenerationResult:
 
 
 def speculative_generate(target, draft, prompt, n_new, gamma, temperature, seed, sequence=0, cached=True, keep_logits=False,
-                         lenience=1.0, top_k=0):
+                         lenience=1.0, top_k=0, top_p=1.0):
     """Algorithm 1 repeated until n_new tokens are emitted.
 
     `target` and `draft` are model objects with forward_rows / forward_full /
@@ -94,7 +94,7 @@ def speculative_generate(target, draft, prompt, n_new, gamma, temperature, seed,
             else:
                 row = draft.forward_full(committed + xs)[-1]
             u = philox.uniform(seed, L + i - 1, sequence, philox.PURPOSE_DRAFT)
-            x, margin = sample_token(row, u, temperature, top_k)
+            x, margin = sample_token(row, u, temperature, top_k, top_p)
             xs.append(x)
             q_logits.append(row)
             draft_margins.append(margin)
@@ -108,9 +108,9 @@ def speculative_generate(target, draft, prompt, n_new, gamma, temperature, seed,
         q_arr = np.stack(q_logits) if gamma else np.zeros((0, p_logits.shape[1]))
         # The final draw decides the token at position L + n, known only after
         # the accept tests: evaluate once with a placeholder to find n.
-        probe = verify_step(p_logits, q_arr, xs, uniforms + [0.5], temperature, lenience, top_k)
+        probe = verify_step(p_logits, q_arr, xs, uniforms + [0.5], temperature, lenience, top_k, top_p)
         u_final = philox.uniform(seed, L + probe.n_accepted, sequence, philox.PURPOSE_FINAL)
-        res = verify_step(p_logits, q_arr, xs, uniforms + [u_final], temperature, lenience, top_k)
+        res = verify_step(p_logits, q_arr, xs, uniforms + [u_final], temperature, lenience, top_k, top_p)
         n = res.n_accepted
         committed.extend(xs[:n])
         committed.append(res.next_token)
@@ -128,7 +128,7 @@ def speculative_generate(target, draft, prompt, n_new, gamma, temperature, seed,
     return result
 
 
-def target_only_generate(target, prompt, n_new, temperature, seed, sequence=0, cached=True, keep_logits=False, top_k=0):
+def target_only_generate(target, prompt, n_new, temperature, seed, sequence=0, cached=True, keep_logits=False, top_k=0, top_p=1.0):
     """Standard autoregressive decoding from the target alone (cost T per token)."""
     committed = [int(t) for t in prompt]
     prompt_len = len(committed)
@@ -143,7 +143,7 @@ def target_only_generate(target, prompt, n_new, temperature, seed, sequence=0, c
         else:
             row = target.forward_full(committed)[-1]
         u = philox.uniform(seed, L, sequence, philox.PURPOSE_FINAL)
-        t, margin = sample_token(row, u, temperature, top_k)
+        t, margin = sample_token(row, u, temperature, top_k, top_p)
         committed.append(t)
         margins.append(margin)
         if keep_logits:

@@ -42,8 +42,19 @@ What follows the paper, and where it is silent:
   ties can keep more than k); k = 0 or k >= vocabulary changes nothing.  The
   same k standardises p and q, as the section asks.  T = 0 ignores k (the
   maximum is always kept).
+* Nucleus sampling is named in the same sentence, again without a definition.
+  Reading (the usual one): with 0 < top_p < 1, tokens are taken in order of
+  decreasing probability under the temperature softmax (of the top-k logits
+  when k is set: top-k first, then the nucleus of what is left) until their
+  mass first reaches top_p of the total; every logit below the last one taken
+  is set to -inf (logits equal to it all stay) and the rest is renormalised.
+  top_p >= 1 (or <= 0) changes nothing; T = 0 ignores it.
 
-Pins (tests/test_oracle_sampling.py): top-k against a pick-the-maximum-k-times
+Pins (tests/test_oracle_sampling.py): the nucleus against a
+take-the-maximum-until-the-mass-is-reached restatement, on a hand-computed
+four-token example, its limits (top_p -> 0 keeps the argmax, top_p = 1 keeps
+everything), its composition with top-k, and the emitted-token law under it;
+top-k against a pick-the-maximum-k-times
 restatement, its support size, the preserved ratios inside the support, k = 1
 against argmax and k >= V against plain softmax, and the emitted-token law
 under top-k against the top-k target distribution; emitted-token law equals p over 10^6
@@ -76,11 +87,41 @@ def keep_top_k(logits, top_k):
     return np.where(z >= top_k_floor(z, top_k), z, -np.inf)
 
 
-def standardise(logits, temperature, top_k=0):
+def nucleus_floor(logits, temperature, top_k=0, top_p=1.0):
+    """(floor, margin): the smallest logit that top-k followed by the nucleus keeps.
+
+    margin: distance, as a fraction of the total mass, between top_p and the
+    nearer of the two cumulative masses around the cut (inf when the nucleus is
+    off); a caller comparing with lower-precision arithmetic can tell from it
+    whether the cut was a close call.
+    """
+    z = keep_top_k(logits, top_k)
+    floor = top_k_floor(logits, top_k)
+    if not 0.0 < top_p < 1.0 or temperature == 0:
+        return floor, float("inf")
+    w = np.exp((z - z.max()) / float(temperature))
+    order = np.argsort(-z, kind="stable")  # decreasing probability
+    running = np.cumsum(w[order])
+    goal = top_p * running[-1]
+    taken = int(np.searchsorted(running, goal, side="left")) + 1  # first prefix whose mass reaches the goal
+    taken = min(taken, z.shape[0])
+    margin = abs(running[taken - 1] - goal)
+    if taken > 1:
+        margin = min(margin, abs(running[taken - 2] - goal))
+    return float(z[order[taken - 1]]), float(margin / running[-1])
+
+
+def keep_nucleus(logits, temperature, top_k=0, top_p=1.0):
+    """The row with everything outside top-k and the nucleus replaced by -inf."""
+    z = np.asarray(logits, dtype=np.float64)
+    return np.where(z >= nucleus_floor(z, temperature, top_k, top_p)[0], z, -np.inf)
+
+
+def standardise(logits, temperature, top_k=0, top_p=1.0):
     """Section 2.2: logits -> the adjusted distribution that is sampled from.
 
-    T > 0: softmax(logits / T) over the top-k logits (all of them for k = 0),
-    with the maximum subtracted first.
+    T > 0: softmax(logits / T) over the logits that top-k and then the nucleus
+    keep (all of them for k = 0, top_p = 1), with the maximum subtracted first.
     T = 0: one-hot at the maximum (lowest index on ties).
     """
     z = np.asarray(logits, dtype=np.float64)
@@ -88,7 +129,7 @@ def standardise(logits, temperature, top_k=0):
         out = np.zeros_like(z)
         out[int(np.argmax(z))] = 1.0  # numpy's argmax returns the first maximum
         return out
-    z = keep_top_k(z, top_k) / float(temperature)
+    z = keep_nucleus(z, temperature, top_k, top_p) / float(temperature)
     z = z - z.max()
     e = np.exp(z)
     return e / e.sum()
@@ -154,7 +195,7 @@ def lenient_greedy_accepts(target_row, x, lenience):
     return slack >= 0.0, abs(slack)
 
 
-def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0, top_k=0):
+def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0, top_k=0, top_p=1.0):
     """Algorithm 1 from "determine the number of accepted guesses" to the end.
 
     target_logits [gamma+1, V]: row i-1 gives p_i (i = 1..gamma+1).
@@ -168,8 +209,8 @@ def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature
     assert ql.shape[0] == gamma and len(draft_tokens) == gamma
     assert len(uniforms) == gamma + 1
 
-    p = [standardise(tl[i], temperature, top_k) for i in range(gamma + 1)]
-    q = [standardise(ql[i], temperature, top_k) for i in range(gamma)]
+    p = [standardise(tl[i], temperature, top_k, top_p) for i in range(gamma + 1)]
+    q = [standardise(ql[i], temperature, top_k, top_p) for i in range(gamma)]
 
     accept_margin = float("inf")
     top2_gap = float("inf")
@@ -206,15 +247,15 @@ def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature
     return VerifyResult(n, t, accept_margin, cdf_margin, top2_gap, fallback, betas)
 
 
-def verify_batch(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0, top_k=0):
+def verify_batch(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0, top_k=0, top_p=1.0):
     """`verify_step` for every sequence of a batch: [B, ...] inputs -> list."""
     return [
-        verify_step(target_logits[b], draft_logits[b], draft_tokens[b], uniforms[b], temperature, lenience, top_k)
+        verify_step(target_logits[b], draft_logits[b], draft_tokens[b], uniforms[b], temperature, lenience, top_k, top_p)
         for b in range(len(target_logits))
     ]
 
 
-def sample_token(logits, u, temperature, top_k=0):
+def sample_token(logits, u, temperature, top_k=0, top_p=1.0):
     """A plain draw from the standardised distribution: (token, cdf margin).
 
     This is how the draft model draws x_i ~ q_i and how target-only decoding
@@ -224,24 +265,24 @@ def sample_token(logits, u, temperature, top_k=0):
     z = np.asarray(logits, dtype=np.float64)
     if temperature == 0:
         return int(np.argmax(z)), float("inf")
-    w = np.exp((keep_top_k(z, top_k) - z.max()) / float(temperature))
+    w = np.exp((keep_nucleus(z, temperature, top_k, top_p) - z.max()) / float(temperature))
     return inverse_cdf(w, u)
 
 
-def sample_trials(logits, uniforms, temperature, top_k=0):
+def sample_trials(logits, uniforms, temperature, top_k=0, top_p=1.0):
     """`sample_token` for many uniforms that share one row of logits -> [N]."""
     z = np.asarray(logits, dtype=np.float64)
     us = np.asarray(uniforms, dtype=np.float64)
     if temperature == 0:
         return np.full(us.shape[0], int(np.argmax(z)), dtype=np.int64)
-    w = np.exp((keep_top_k(z, top_k) - z.max()) / float(temperature))
+    w = np.exp((keep_nucleus(z, temperature, top_k, top_p) - z.max()) / float(temperature))
     running = np.cumsum(w)
     k = np.searchsorted(running, us * running[-1], side="right")
     positive = np.nonzero(w > 0.0)[0]
     return np.where(k >= w.shape[0], positive[-1], k).astype(np.int64)
 
 
-def verify_trials(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0, top_k=0):
+def verify_trials(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0, top_k=0, top_p=1.0):
     """Many independent trials of `verify_step` that share one set of logits.
 
     target_logits [gamma+1, V] and draft_logits [gamma, V] are fixed;
@@ -256,8 +297,8 @@ def verify_trials(target_logits, draft_logits, draft_tokens, uniforms, temperatu
     us = np.asarray(uniforms, dtype=np.float64)
     gamma = tl.shape[0] - 1
     trials = us.shape[0]
-    p = np.stack([standardise(tl[i], temperature, top_k) for i in range(gamma + 1)])
-    q = np.stack([standardise(ql[i], temperature, top_k) for i in range(gamma)]) if gamma else np.zeros((0, tl.shape[1]))
+    p = np.stack([standardise(tl[i], temperature, top_k, top_p) for i in range(gamma + 1)])
+    q = np.stack([standardise(ql[i], temperature, top_k, top_p) for i in range(gamma)]) if gamma else np.zeros((0, tl.shape[1]))
 
     n = np.full(trials, gamma, dtype=np.int64)
     undecided = np.ones(trials, dtype=bool)

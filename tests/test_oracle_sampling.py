@@ -379,3 +379,91 @@ def test_emitted_law_under_top_k_is_the_top_k_target_distribution(k):
     for i in range(300):
         res = sampling.verify_step(tl, ql, x[i : i + 1], [r[i], u[i]], 1.0, top_k=k)
         assert (res.n_accepted, res.next_token) == (n[i], t[i])
+
+
+def _nucleus_by_repeated_argmax(probs, top_p):
+    """Indices taken by picking the most probable remaining token until the mass reaches top_p."""
+    left = np.array(probs, dtype=np.float64)
+    chosen, mass = [], 0.0
+    while mass < top_p * probs.sum() and len(chosen) < len(probs):
+        i = int(np.argmax(left))
+        chosen.append(i)
+        mass += probs[i]
+        left[i] = -1.0
+    return chosen
+
+
+def test_nucleus_on_a_hand_computed_example():
+    probs = np.array([0.05, 0.5, 0.15, 0.3])
+    logits = np.log(probs)
+    for top_p, kept in [(0.4, [1]), (0.6, [1, 3]), (0.75, [1, 3]), (0.85, [1, 2, 3]), (0.97, [0, 1, 2, 3])]:
+        got = sampling.standardise(logits, 1.0, top_p=top_p)
+        assert np.nonzero(got)[0].tolist() == kept
+        assert np.allclose(got[kept], probs[kept] / probs[kept].sum(), rtol=1e-12)
+    # the margin reports how close top_p came to a cumulative mass (0.5, 0.8, 0.95, 1.0)
+    assert sampling.nucleus_floor(logits, 1.0, 0, 0.6)[1] == pytest.approx(0.1, abs=1e-12)
+    assert sampling.nucleus_floor(logits, 1.0, 0, 0.94)[1] == pytest.approx(0.01, abs=1e-12)
+    # temperature enters before the cut: at T = 0.5 the probabilities are proportional to p^2
+    sharper = probs**2 / (probs**2).sum()  # 0.0068 0.68 0.061 0.245
+    assert np.nonzero(sampling.standardise(logits, 0.5, top_p=0.7))[0].tolist() == [1, 3]
+    assert np.allclose(sampling.standardise(logits, 0.5, top_p=0.7)[[1, 3]], sharper[[1, 3]] / sharper[[1, 3]].sum())
+
+
+@pytest.mark.parametrize("top_p", [0.05, 0.5, 0.9, 0.999])
+@pytest.mark.parametrize("temperature", [1.0, 0.6])
+def test_nucleus_equals_the_greedy_restatement(top_p, temperature):
+    tl, _ = _fixed_pair(2.0)
+    row = tl[0]
+    plain = sampling.standardise(row, temperature)
+    got = sampling.standardise(row, temperature, top_p=top_p)
+    chosen = _nucleus_by_repeated_argmax(plain, top_p)
+    assert sorted(np.nonzero(got)[0].tolist()) == sorted(chosen)
+    assert got.sum() == pytest.approx(1.0, abs=1e-12)
+    assert plain[chosen].sum() >= top_p and plain[chosen[:-1]].sum() < top_p  # the smallest such prefix
+    assert np.allclose(got[chosen] / got[chosen[0]], plain[chosen] / plain[chosen[0]], rtol=1e-12)
+    # with top-k first, the nucleus is taken of the renormalised top-k distribution
+    k = 9
+    top = sampling.standardise(row, temperature, top_k=k)
+    both = sampling.standardise(row, temperature, top_k=k, top_p=top_p)
+    assert sorted(np.nonzero(both)[0].tolist()) == sorted(_nucleus_by_repeated_argmax(top, top_p))
+
+
+def test_nucleus_limits_and_ties():
+    tl, _ = _fixed_pair(1.0)
+    row = tl[0]
+    plain = sampling.standardise(row, 0.8)
+    for off in (1.0, 1.5, 0.0, -0.1):
+        assert np.array_equal(sampling.standardise(row, 0.8, top_p=off), plain)
+    assert np.array_equal(sampling.standardise(row, 0.8, top_p=1e-9), sampling.standardise(row, 0.0))
+    assert np.array_equal(sampling.standardise(row, 0.0, top_p=0.3), sampling.standardise(row, 0.0))
+    # a tie at the cut stays whole: probabilities 0.4 0.2 0.2 0.2, top_p 0.5 reaches its mass inside the tie
+    tied = np.log(np.array([0.2, 0.4, 0.2, 0.2]))
+    assert np.nonzero(sampling.standardise(tied, 1.0, top_p=0.5))[0].tolist() == [0, 1, 2, 3]
+    assert np.nonzero(sampling.standardise(tied, 1.0, top_p=0.4 - 1e-9))[0].tolist() == [1]
+    us = philox.uniforms_vec(9, np.arange(20000), 0, philox.PURPOSE_DRAFT)
+    support = set(np.nonzero(sampling.standardise(row, 1.0, top_p=0.5))[0].tolist())
+    drawn = sampling.sample_trials(row, us, 1.0, top_p=0.5)
+    assert set(drawn.tolist()) <= support
+    assert [sampling.sample_token(row, float(u), 1.0, top_p=0.5)[0] for u in us[:200]] == drawn[:200].tolist()
+
+
+def test_emitted_law_under_the_nucleus_is_the_nucleus_target_distribution():
+    trials = 400_000
+    tl, ql = _fixed_pair(1.0)
+    kw = dict(top_k=20, top_p=0.8)
+    p = sampling.standardise(tl[0], 1.0, **kw)
+    q = sampling.standardise(ql[0], 1.0, **kw)
+    assert 1 < np.count_nonzero(p) < 20 and 1 < np.count_nonzero(q) < 20
+    idx = np.arange(trials)
+    x = sampling.sample_trials(ql[0], philox.uniforms_vec(8, idx, 0, philox.PURPOSE_DRAFT), 1.0, **kw)
+    r = philox.uniforms_vec(8, idx, 0, philox.PURPOSE_ACCEPT)
+    u = philox.uniforms_vec(8, idx, 0, philox.PURPOSE_FINAL)
+    n, t = sampling.verify_trials(tl, ql, x[:, None], np.stack([r, u], axis=1), 1.0, **kw)
+    first = np.where(n == 1, x, t)
+    assert np.all(p[first] > 0)
+    assert _chi_square_p(np.bincount(first, minlength=VOCAB), p) > 1e-3
+    beta = analysis.beta(p, q)
+    assert abs((n == 1).mean() - beta) < 4 * np.sqrt(beta * (1 - beta) / trials)
+    for i in range(300):
+        res = sampling.verify_step(tl, ql, x[i : i + 1], [r[i], u[i]], 1.0, **kw)
+        assert (res.n_accepted, res.next_token) == (n[i], t[i])
