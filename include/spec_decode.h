@@ -109,28 +109,38 @@ int spec_verify_sample_lenient(const float* target_logits, const float* draft_lo
                                int32_t* n_accepted, int32_t* next_token,
                                void* workspace, size_t workspace_bytes, void* stream);
 
-/* The same with top-k standardisation (Section 2.2 lists top-k among the
- * sampling methods that are a draw from an adjusted distribution and asks that
- * both models be standardised the same way; it gives no definition).  With
- * 0 < top_k < vocab and T > 0, every logit below the top_k-th largest logit of
- * its own row reads as -inf, for the target's rows and the draft's alike,
- * before the temperature softmax; logits equal to the top_k-th largest all
- * stay, so ties can keep more than top_k.  top_k == 0 or >= vocab, or T == 0
- * (the maximum is always kept), is spec_verify_sample_lenient exactly.  A
- * drafted token outside the target's top-k set has p_i(x_i) = 0 and is rejected
- * unless q_i(x_i) is 0 too.  Enqueues one more kernel (the per-row selection)
- * before the other two; same workspace, errors as above plus SPEC_ERR_BAD_ARG
- * for top_k < 0. */
-int spec_verify_sample_topk(const float* target_logits, const float* draft_logits,
-                            const int32_t* draft_tokens, const float* uniforms,
-                            int batch, int gamma, int vocab, float temperature, float lenience,
-                            int top_k, int32_t* n_accepted, int32_t* next_token,
-                            void* workspace, size_t workspace_bytes, void* stream);
+/* The same with top-k and nucleus (top-p) standardisation.  Section 2.2 lists
+ * both among the sampling methods that are a draw from an adjusted
+ * distribution and asks that both models be standardised the same way; it
+ * defines neither.  Here, for T > 0:
+ *   0 < top_k < vocab: every logit below the top_k-th largest logit of its own
+ *     row reads as -inf before the temperature softmax (logits equal to the
+ *     top_k-th largest all stay, so ties can keep more than top_k);
+ *   0 < top_p < 1: of what top-k left, tokens are taken in order of decreasing
+ *     probability until their mass first reaches top_p of the total; every
+ *     logit below the last one taken reads as -inf (ties with it stay);
+ * for the target's rows and the draft's alike.  top_k == 0 or >= vocab switches
+ * the first off, top_p <= 0 or >= 1 the second; with both off, or at T == 0 (the
+ * maximum is always kept), this is spec_verify_sample_lenient exactly.  A
+ * drafted token outside the target's kept set has p_i(x_i) = 0 and is rejected
+ * unless q_i(x_i) is 0 too.  Enqueues one more kernel per active cut (the
+ * per-row selections) before the other two; same workspace.  The nucleus sums
+ * fp32 weights in a fixed order: a row always gives the same cut, and a cut
+ * whose mass comes within rounding of top_p may differ from exact arithmetic
+ * by one token.  Errors as above plus SPEC_ERR_BAD_ARG for top_k < 0 or a NaN
+ * top_p. */
+int spec_verify_sample_truncated(const float* target_logits, const float* draft_logits,
+                                 const int32_t* draft_tokens, const float* uniforms,
+                                 int batch, int gamma, int vocab, float temperature, float lenience,
+                                 int top_k, float top_p, int32_t* n_accepted, int32_t* next_token,
+                                 void* workspace, size_t workspace_bytes, void* stream);
 
-/* floors[r] = the top_k-th largest value of row r of logits [rows, vocab] (fp32
- * device in, fp32 device out), 1 <= top_k <= vocab: the threshold that the
- * top-k variants apply.  Exact (comparisons only).  One kernel on `stream`. */
-int spec_top_k_floors(const float* logits, int rows, int vocab, int top_k, float* floors, void* stream);
+/* floors[r] = the lowest logit of row r that the cuts above keep, for logits
+ * [rows, vocab] fp32 device and T > 0 (fp32 device out): what the truncated
+ * variants apply.  With top-k alone the result is exact (comparisons only).
+ * Errors: SPEC_ERR_BAD_ARG if neither cut is active or T <= 0. */
+int spec_truncation_floors(const float* logits, int rows, int vocab, float temperature,
+                           int top_k, float top_p, float* floors, void* stream);
 
 /* ------------------------------------------------------------------------- *
  * spec_verify_sample for callers that cannot allocate device memory.  (The
@@ -182,12 +192,13 @@ int spec_verify_sample_static(const float* target_logits, const float* draft_log
 int spec_sample(const float* logits, const float* uniforms, int rows, int vocab,
                 float temperature, int32_t* tokens, void* stream);
 
-/* The same over the top_k largest logits of each row (see
- * spec_verify_sample_topk); floors [rows] fp32 device is scratch that receives
- * the rows' thresholds (may be NULL when top_k == 0, top_k >= vocab or T == 0,
- * where the call is spec_sample).  Two kernels. */
-int spec_sample_topk(const float* logits, const float* uniforms, int rows, int vocab,
-                     float temperature, int top_k, int32_t* tokens, float* floors, void* stream);
+/* The same over what top-k and the nucleus keep of each row (see
+ * spec_verify_sample_truncated); floors [rows] fp32 device is scratch that
+ * receives the rows' thresholds (may be NULL when both cuts are off or T == 0,
+ * where the call is spec_sample).  One more kernel per active cut. */
+int spec_sample_truncated(const float* logits, const float* uniforms, int rows, int vocab,
+                          float temperature, int top_k, float top_p, int32_t* tokens,
+                          float* floors, void* stream);
 
 /* ------------------------------------------------------------------------- *
  * Uniforms of the method's counter-based generator, on the device.
@@ -386,12 +397,13 @@ int spec_begin(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, 
  * printed.  Errors: SPEC_ERR_BAD_ARG outside (0, 1]. */
 int spec_set_lenience(spec_ctx* ctx, float lenience);
 
-/* top-k standardisation (see spec_verify_sample_topk) of both models in the
- * generations that start after this call: the draft draws x_i from its top-k
- * distribution, the accept tests and the final draw use the target's and the
- * draft's top-k distributions, and gamma = 0 decodes from the target's.  0 (the
- * default): the whole vocabulary.  Errors: SPEC_ERR_BAD_ARG for top_k < 0. */
-int spec_set_top_k(spec_ctx* ctx, int top_k);
+/* top-k and nucleus standardisation (see spec_verify_sample_truncated) of both
+ * models in the generations that start after this call: the draft draws x_i
+ * from its truncated distribution, the accept tests and the final draw use the
+ * target's and the draft's truncated distributions, and gamma = 0 decodes from
+ * the target's.  top_k = 0 and top_p = 1 (the defaults): the whole vocabulary.
+ * Errors: SPEC_ERR_BAD_ARG for top_k < 0 or a NaN top_p. */
+int spec_set_truncation(spec_ctx* ctx, int top_k, float top_p);
 
 /* Timing instrument (no counterpart in Algorithm 1): from the next spec_begin /
  * spec_generate on, the accept decision of every drafted token is replaced by

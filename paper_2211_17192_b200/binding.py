@@ -103,10 +103,10 @@ def spec_verify_sample_workspace_bytes(batch, gamma, vocab):
 
 
 def spec_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, temperature,
-                       n_accepted=None, next_token=None, workspace=None, lenience=1.0, top_k=0):
+                       n_accepted=None, next_token=None, workspace=None, lenience=1.0, top_k=0, top_p=1.0):
     """Speculative sampling for a batch; see `spec_verify_sample` (and, for
-    lenience < 1, `spec_verify_sample_lenient`; for top_k > 0,
-    `spec_verify_sample_topk`) in the header.
+    lenience < 1, `spec_verify_sample_lenient`; for top_k > 0 or top_p < 1,
+    `spec_verify_sample_truncated`) in the header.
 
     target_logits [B, gamma+1, V] fp32, draft_logits [B, gamma, V] fp32,
     draft_tokens [B, gamma] int32, uniforms [B, gamma+1] fp32, all CUDA.
@@ -135,13 +135,13 @@ def spec_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, temp
                 _ptr(uniforms, torch.float32, "uniforms", optional=True))
     outputs = (_ptr(n_accepted, torch.int32, "n_accepted"), _ptr(next_token, torch.int32, "next_token"),
                _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream())
-    if top_k:
+    if top_k or top_p != 1.0:
         h = lib()
-        h.spec_verify_sample_topk.restype = ctypes.c_int
-        h.spec_verify_sample_topk.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int] * 3 + [ctypes.c_float] * 2 + \
-            [ctypes.c_int] + [ctypes.c_void_p] * 3 + [ctypes.c_size_t, ctypes.c_void_p]
-        _check(h.spec_verify_sample_topk(*pointers, batch, gamma, vocab, float(temperature), float(lenience),
-                                         int(top_k), *outputs))
+        h.spec_verify_sample_truncated.restype = ctypes.c_int
+        h.spec_verify_sample_truncated.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int] * 3 + [ctypes.c_float] * 2 + \
+            [ctypes.c_int, ctypes.c_float] + [ctypes.c_void_p] * 3 + [ctypes.c_size_t, ctypes.c_void_p]
+        _check(h.spec_verify_sample_truncated(*pointers, batch, gamma, vocab, float(temperature), float(lenience),
+                                              int(top_k), float(top_p), *outputs))
     elif lenience == 1.0:
         _check(lib().spec_verify_sample(*pointers, batch, gamma, vocab, float(temperature), *outputs))
     else:
@@ -170,35 +170,36 @@ def spec_verify_sample_static(target_logits, draft_logits, draft_tokens, uniform
     return n_accepted, next_token
 
 
-def spec_top_k_floors(logits, top_k, floors=None):
-    """floors[r] = the top_k-th largest value of row r; logits [R, V] fp32 CUDA."""
+def spec_truncation_floors(logits, temperature, top_k=0, top_p=1.0, floors=None):
+    """floors[r] = the lowest logit of row r that top-k and then the nucleus keep; logits [R, V] fp32 CUDA."""
     rows, vocab = logits.shape
     if floors is None:
         floors = torch.empty(rows, dtype=torch.float32, device=logits.device)
     h = lib()
-    h.spec_top_k_floors.restype = ctypes.c_int
-    h.spec_top_k_floors.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
-    _check(h.spec_top_k_floors(_ptr(logits, torch.float32, "logits"), rows, vocab, int(top_k),
-                               _ptr(floors, torch.float32, "floors"), _stream()))
+    h.spec_truncation_floors.restype = ctypes.c_int
+    h.spec_truncation_floors.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_float, ctypes.c_int,
+                                         ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p]
+    _check(h.spec_truncation_floors(_ptr(logits, torch.float32, "logits"), rows, vocab, float(temperature), int(top_k),
+                                    float(top_p), _ptr(floors, torch.float32, "floors"), _stream()))
     return floors
 
 
-def spec_sample(logits, uniforms, temperature, tokens=None, top_k=0):
-    """tokens[r] ~ softmax(logits[r] / T) (argmax at T = 0), over the top_k
-    largest logits of each row when top_k > 0; logits [R, V] fp32 CUDA."""
+def spec_sample(logits, uniforms, temperature, tokens=None, top_k=0, top_p=1.0):
+    """tokens[r] ~ softmax(logits[r] / T) (argmax at T = 0), over what top-k and the
+    nucleus keep of each row when top_k > 0 or top_p < 1; logits [R, V] fp32 CUDA."""
     rows, vocab = logits.shape
     if tokens is None:
         tokens = torch.empty(rows, dtype=torch.int32, device=logits.device)
-    if top_k:
+    if top_k or top_p != 1.0:
         floors = torch.empty(max(rows, 1), dtype=torch.float32, device=logits.device)
         h = lib()
-        h.spec_sample_topk.restype = ctypes.c_int
-        h.spec_sample_topk.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_float,
-                                       ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
-        _check(h.spec_sample_topk(_ptr(logits, torch.float32, "logits"),
-                                  _ptr(uniforms, torch.float32, "uniforms", optional=True), rows, vocab,
-                                  float(temperature), int(top_k), _ptr(tokens, torch.int32, "tokens"),
-                                  _ptr(floors, torch.float32, "floors"), _stream()))
+        h.spec_sample_truncated.restype = ctypes.c_int
+        h.spec_sample_truncated.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_float,
+                                            ctypes.c_int, ctypes.c_float, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        _check(h.spec_sample_truncated(_ptr(logits, torch.float32, "logits"),
+                                       _ptr(uniforms, torch.float32, "uniforms", optional=True), rows, vocab,
+                                       float(temperature), int(top_k), float(top_p), _ptr(tokens, torch.int32, "tokens"),
+                                       _ptr(floors, torch.float32, "floors"), _stream()))
         return tokens
     _check(lib().spec_sample(_ptr(logits, torch.float32, "logits"),
                              _ptr(uniforms, torch.float32, "uniforms", optional=True),
@@ -351,8 +352,8 @@ def _declare_engine(h):
     h.spec_forward_logits.argtypes = [vp, c.c_int, vp, c.c_int, c.c_int, vp]
     h.spec_set_lenience.restype = c.c_int
     h.spec_set_lenience.argtypes = [vp, c.c_float]
-    h.spec_set_top_k.restype = c.c_int
-    h.spec_set_top_k.argtypes = [vp, c.c_int]
+    h.spec_set_truncation.restype = c.c_int
+    h.spec_set_truncation.argtypes = [vp, c.c_int, c.c_float]
     h.spec_set_imposed_acceptance.restype = c.c_int
     h.spec_set_imposed_acceptance.argtypes = [vp, c.c_float]
     h.spec_time_forward.restype = c.c_int
@@ -501,9 +502,10 @@ class Engine:
         """Lenience factor of Appendix A.5 for the generations that follow (1 = Algorithm 1)."""
         _check(lib().spec_set_lenience(self._ctx, float(lenience)))
 
-    def set_top_k(self, top_k):
-        """Top-k standardisation (Section 2.2) of both models for the generations that follow (0 = off)."""
-        _check(lib().spec_set_top_k(self._ctx, int(top_k)))
+    def set_truncation(self, top_k=0, top_p=1.0):
+        """Top-k and nucleus standardisation (Section 2.2) of both models for the generations
+        that follow; top_k = 0 and top_p = 1 switch them off."""
+        _check(lib().spec_set_truncation(self._ctx, int(top_k), float(top_p)))
 
     def set_imposed_acceptance(self, alpha):
         """Timing instrument: accept every drafted token with probability `alpha`

@@ -47,6 +47,7 @@ struct spec_ctx {
     float imposed_alpha = -1.0f;  // >= 0: timing instrument, see spec_set_imposed_acceptance
     float lenience = 1.0f;        // Appendix A.5; 1 = Algorithm 1 as printed
     int top_k = 0;                // Section 2.2: both models standardised over their k largest logits; 0 = all
+    float top_p = 1.0f;           // and then over the nucleus of mass top_p; 1 = all
     float* sample_floors = nullptr;  // the draft rows' k-th largest logits, one per sequence
 
     // cached iteration graph
@@ -54,6 +55,7 @@ struct spec_ctx {
     int graph_batch = -1, graph_gamma = -1;
     float graph_temperature = -1.0f, graph_lenience = 1.0f;
     int graph_top_k = 0;
+    float graph_top_p = 1.0f;
 
     // generation in progress (spec_begin / spec_generate)
     int session_batch = 0, session_gamma = 0, session_n_new = 0;
@@ -403,14 +405,14 @@ int enqueue_iteration(spec_ctx* ctx, int batch, int gamma, float temperature) {
         // x_step ~ q_step for every sequence
         SPEC_TRY(launch_sample_strided(ctx->draft_logits + static_cast<size_t>(step - 1) * vocab,
                                        static_cast<size_t>(gamma) * vocab, ctx->draft_u + (step - 1), gamma, batch,
-                                       vocab, temperature, ctx->top_k, ctx->sample_floors,
+                                       vocab, temperature, ctx->top_k, ctx->top_p, ctx->sample_floors,
                                        ctx->draft_tokens + (step - 1), gamma, st));
     }
     SPEC_TRY(launch_pdl(prep_verify_kernel, dim3(blocks_bg), dim3(threads), 0, st, ctx->tokens, ctx->draft_tokens,
                         ctx->length, batch, gamma, ctx->rt.max_len, ctx->row_token, ctx->row_pos, ctx->row_seq));
     SPEC_TRY(forward(ctx, ctx->model[0], batch, gamma + 1, batch * (gamma + 1), nullptr, nullptr, ctx->target_logits));
     SPEC_TRY(launch_verify_sample(ctx->target_logits, ctx->draft_logits, ctx->draft_tokens, ctx->accept_u, ctx->final_u,
-                                  batch, gamma, vocab, temperature, ctx->lenience, ctx->top_k, ctx->n_accepted,
+                                  batch, gamma, vocab, temperature, ctx->lenience, ctx->top_k, ctx->top_p, ctx->n_accepted,
                                   ctx->next_token, ctx->sampler_ws, st));
     return launch_pdl(commit_kernel, dim3(blocks_b), dim3(threads), 0, st, ctx->params, ctx->draft_tokens,
                       ctx->n_accepted, ctx->next_token, ctx->accept_u, ctx->prompt_len, batch, gamma, ctx->rt.max_len,
@@ -419,7 +421,7 @@ int enqueue_iteration(spec_ctx* ctx, int batch, int gamma, float temperature) {
 
 int build_graph(spec_ctx* ctx, int batch, int gamma, float temperature) {
     if (ctx->graph && ctx->graph_batch == batch && ctx->graph_gamma == gamma && ctx->graph_temperature == temperature &&
-        ctx->graph_lenience == ctx->lenience && ctx->graph_top_k == ctx->top_k)
+        ctx->graph_lenience == ctx->lenience && ctx->graph_top_k == ctx->top_k && ctx->graph_top_p == ctx->top_p)
         return SPEC_OK;
     if (ctx->graph) {
         cudaGraphExecDestroy(ctx->graph);
@@ -442,6 +444,7 @@ int build_graph(spec_ctx* ctx, int batch, int gamma, float temperature) {
     ctx->graph_temperature = temperature;
     ctx->graph_lenience = ctx->lenience;
     ctx->graph_top_k = ctx->top_k;
+    ctx->graph_top_p = ctx->top_p;
     return SPEC_OK;
 }
 
@@ -998,9 +1001,11 @@ extern "C" int spec_set_lenience(spec_ctx* ctx, float lenience) {
     return SPEC_OK;
 }
 
-extern "C" int spec_set_top_k(spec_ctx* ctx, int top_k) {
-    if (!ctx || top_k < 0) return fail(SPEC_ERR_BAD_ARG, "spec_set_top_k: top_k must be >= 0 (0: the whole vocabulary)");
+extern "C" int spec_set_truncation(spec_ctx* ctx, int top_k, float top_p) {
+    if (!ctx || top_k < 0 || !(top_p == top_p))
+        return fail(SPEC_ERR_BAD_ARG, "spec_set_truncation: top_k must be >= 0 (0: off) and top_p a number (>= 1: off)");
     ctx->top_k = top_k;
+    ctx->top_p = top_p;
     return SPEC_OK;
 }
 

@@ -810,6 +810,192 @@ topk_floor_kernel(const float* __restrict__ a, size_t a_stride, int a_rows, cons
     if (tid == 0) floors[blockIdx.x] = key_float(prefix);
 }
 
+// ---- nucleus (top-p): the lowest logit inside the smallest most-probable set of mass top_p ----
+constexpr int kFloorWarps = kFloorThreads / 32;
+constexpr int kCutSlots = 72;  // block-wide measurements per row: 1 + at most 32 + 32
+
+// One CTA per row, after topk_floor_kernel when top-k is set too (use_k: floors
+// then holds the row's k-th largest logit on entry, and the nucleus is taken
+// of the logits at or above it).  With weights w = exp((l - max) / T), the
+// answer is the largest t with mass(key >= t) >= top_p * total mass: the same
+// bit-by-bit search as topk_floor_kernel with a sum of weights for the count.
+// KPT > 0: keys in registers and weights in shared memory ([slot][thread], so
+// a pass reads them without bank conflicts); KPT = 0: both recomputed from the
+// row per pass.  Sums are taken in a fixed order (thread, shuffle tree, warps
+// in index order), so every thread sees the same totals and a row always
+// gives the same floor.
+template <bool VEC, int KPT>
+__global__ void __launch_bounds__(kFloorThreads, 1)
+nucleus_floor_kernel(const float* __restrict__ a, size_t a_stride, int a_rows, const float* __restrict__ b,
+                     size_t b_stride, int b_rows, int vocab, bool use_k, float top_p, float c2,
+                     float* __restrict__ floors) {
+    extern __shared__ float wsm[];
+    __shared__ unsigned counts[kCutSlots];
+    __shared__ float partial[kCutSlots][kFloorWarps];
+    __shared__ uint32_t warp_top[kFloorWarps];
+    __shared__ uint32_t live_key[kLiveCap];
+    __shared__ float live_w[kLiveCap];
+    pdl_trigger();
+    pdl_wait();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per_seq = a_rows + b_rows;
+    const int seq = blockIdx.x / per_seq, row = blockIdx.x % per_seq;
+    const float* src = row < a_rows ? a + (static_cast<size_t>(seq) * a_rows + row) * a_stride
+                                    : b + (static_cast<size_t>(seq) * b_rows + (row - a_rows)) * b_stride;
+    const Row<VEC> r = make_row<VEC>(src, vocab);
+    const int groups = (vocab + 3) >> 2;
+    if (tid < kCutSlots) counts[tid] = 0;
+    const uint32_t kf = use_k ? float_key(__ldcg(floors + blockIdx.x)) : 0u;
+
+    constexpr int G = KPT > 0 ? KPT / 4 : 1;
+    uint32_t keys[4 * G];
+    uint32_t top = 0;
+    if (KPT > 0) {
+#pragma unroll
+        for (int i = 0; i < G; ++i) {
+            const int g = tid + i * kFloorThreads;
+            const float4 v = g < groups ? r.raw(g, -INFINITY) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            keys[4 * i + 0] = float_key(v.x);
+            keys[4 * i + 1] = float_key(v.y);
+            keys[4 * i + 2] = float_key(v.z);
+            keys[4 * i + 3] = float_key(v.w);
+        }
+#pragma unroll
+        for (int i = 0; i < 4 * G; ++i) top = max(top, keys[i]);
+    } else {
+        for (int g = tid; g < groups; g += kFloorThreads) {
+            const float4 v = r.raw(g, -INFINITY);
+            top = max(top, max(max(float_key(v.x), float_key(v.y)), max(float_key(v.z), float_key(v.w))));
+        }
+    }
+    top = __reduce_max_sync(0xffffffffu, top);
+    if (lane == 0) warp_top[warp] = top;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kFloorWarps; ++w) top = max(top, warp_top[w]);
+    const float row_max = key_float(top);
+    auto weight = [&](float v) { return fast_exp2((v - row_max) * c2); };
+    if (KPT > 0) {
+#pragma unroll
+        for (int i = 0; i < 4 * G; ++i) wsm[i * kFloorThreads + tid] = weight(key_float(keys[i]));
+    }
+
+    // count and mass of the keys at or above t, the same values in every thread
+    int slot = 0;
+    auto measure = [&](uint32_t t, unsigned* count, float* mass) {
+        unsigned c = 0;
+        float m = 0.0f;
+        if (KPT > 0) {
+#pragma unroll
+            for (int i = 0; i < 4 * G; ++i)
+                if (keys[i] >= t) { ++c; m += wsm[i * kFloorThreads + tid]; }
+        } else {
+            for (int g = tid; g < groups; g += kFloorThreads) {
+                const float4 v = r.raw(g, -INFINITY);
+                if (float_key(v.x) >= t) { ++c; m += weight(v.x); }
+                if (float_key(v.y) >= t) { ++c; m += weight(v.y); }
+                if (float_key(v.z) >= t) { ++c; m += weight(v.z); }
+                if (float_key(v.w) >= t) { ++c; m += weight(v.w); }
+            }
+        }
+        c = __reduce_add_sync(0xffffffffu, c);
+        m = warp_sum(m);
+        if (lane == 0) {
+            if (c) atomicAdd(&counts[slot], c);
+            partial[slot][warp] = m;
+        }
+        __syncthreads();
+        float total = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kFloorWarps; ++w) total += partial[slot][w];
+        *count = counts[slot];
+        *mass = total;
+        ++slot;
+    };
+
+    unsigned at_prefix;
+    float everything;
+    measure(kf, &at_prefix, &everything);
+    const float goal = top_p * everything;
+    uint32_t prefix = 0;
+    unsigned above = 0;
+    float mass_above = 0.0f;
+    int bit = 31;
+    for (; bit >= 0 && at_prefix - above > kLiveCap; --bit) {
+        const uint32_t cand = prefix | (1u << bit);
+        unsigned c;
+        float m;
+        measure(max(cand, kf), &c, &m);
+        if (m >= goal) { prefix = cand; at_prefix = c; } else { above = c; mass_above = m; }
+    }
+    if (bit >= 0) {
+        // undecided: at or above the top-k floor and equal to `prefix` on every bit above `bit`
+        const int shift = bit + 1;
+        auto undecided = [&](uint32_t key) { return key >= kf && (shift >= 32 || ((key ^ prefix) >> shift) == 0); };
+        unsigned mine = 0;
+        if (KPT > 0) {
+#pragma unroll
+            for (int i = 0; i < 4 * G; ++i) mine += undecided(keys[i]);
+        } else {
+            for (int g = tid; g < groups; g += kFloorThreads) {
+                const float4 v = r.raw(g, -INFINITY);
+                mine += undecided(float_key(v.x)) + undecided(float_key(v.y)) + undecided(float_key(v.z)) +
+                        undecided(float_key(v.w));
+            }
+        }
+        unsigned incl = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        // warps take their places in index order, so the copy (and every sum over it) is the same in every run
+        if (lane == 31) warp_top[warp] = incl;
+        __syncthreads();
+        unsigned pos = incl - mine, n_live = 0;
+#pragma unroll
+        for (int w = 0; w < kFloorWarps; ++w) {
+            if (w < warp) pos += warp_top[w];
+            n_live += warp_top[w];
+        }
+        auto keep = [&](uint32_t key, float w) {
+            if (undecided(key)) {
+                if (pos < kLiveCap) { live_key[pos] = key; live_w[pos] = w; }
+                ++pos;
+            }
+        };
+        if (KPT > 0) {
+#pragma unroll
+            for (int i = 0; i < 4 * G; ++i) keep(keys[i], wsm[i * kFloorThreads + tid]);
+        } else {
+            for (int g = tid; g < groups; g += kFloorThreads) {
+                const float4 v = r.raw(g, -INFINITY);
+                keep(float_key(v.x), weight(v.x));
+                keep(float_key(v.y), weight(v.y));
+                keep(float_key(v.z), weight(v.z));
+                keep(float_key(v.w), weight(v.w));
+            }
+        }
+        __syncthreads();
+        const int n = static_cast<int>(min(n_live, static_cast<unsigned>(kLiveCap)));  // = at_prefix - above
+        for (; bit >= 0; --bit) {
+            const uint32_t cand = prefix | (1u << bit);
+            float m = 0.0f;
+            for (int j = tid; j < n; j += kFloorThreads)
+                if (live_key[j] >= cand) m += live_w[j];
+            m = warp_sum(m);
+            if (lane == 0) partial[slot][warp] = m;
+            __syncthreads();
+            float total = mass_above;
+#pragma unroll
+            for (int w = 0; w < kFloorWarps; ++w) total += partial[slot][w];
+            ++slot;
+            if (total >= goal) prefix = cand;
+        }
+    }
+    if (tid == 0) floors[blockIdx.x] = key_float(max(prefix, kf));
+}
+
 __global__ void uniforms_kernel(uint64_t seed, const int32_t* __restrict__ positions,
                                 const int32_t* __restrict__ sequences, uint32_t purpose, int count,
                                 float* __restrict__ out) {
@@ -854,6 +1040,10 @@ size_t verify_sample_workspace_bytes(int batch, int gamma, int vocab) {
     return stats_bytes(batch, gamma, vocab) + static_cast<size_t>(batch) * rows * sizeof(float) + 256;
 }
 
+bool cut_is_on(int vocab, float temperature, int top_k, float top_p) {
+    return temperature > 0.0f && ((top_k > 0 && top_k < vocab) || (top_p > 0.0f && top_p < 1.0f));
+}
+
 // floors[s * (a_rows + b_rows) + r] = the top_k-th largest logit of sequence s's
 // row r (its a_rows rows of `a`, then its b_rows rows of `b`).  0 < top_k < vocab.
 int launch_topk_floors(const float* a, size_t a_stride, int a_rows, const float* b, size_t b_stride, int b_rows,
@@ -877,21 +1067,65 @@ int launch_topk_floors(const float* a, size_t a_stride, int a_rows, const float*
 #undef SPEC_LAUNCH_FLOORS
 }
 
+// The same rows' nucleus floors for 0 < top_p < 1; with use_k, of the logits at or
+// above the floors already there.
+int launch_nucleus_floors(const float* a, size_t a_stride, int a_rows, const float* b, size_t b_stride, int b_rows,
+                          int seqs, int vocab, bool use_k, float top_p, float inv_t, float* floors, cudaStream_t stream) {
+    const int total = seqs * (a_rows + b_rows);
+    if (total == 0) return SPEC_OK;
+    const bool vec = vocab % 4 == 0 && a_stride % 4 == 0 && aligned16(a) && (b_rows == 0 || (b_stride % 4 == 0 && aligned16(b)));
+    const float c2 = inv_t * kLog2e;
+#define SPEC_LAUNCH_NUCLEUS(V, K)                                                                                  \
+    do {                                                                                                           \
+        /* static + dynamic shared memory exceeds the 48 KB that needs no opt-in even for the short rows */         \
+        const size_t smem = static_cast<size_t>(K) * kFloorThreads * sizeof(float);                                \
+        if (smem > 0)                                                                                              \
+            SPEC_CUDA_TRY(cudaFuncSetAttribute(nucleus_floor_kernel<V, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                               static_cast<int>(smem)));                                           \
+        return launch_pdl(nucleus_floor_kernel<V, K>, dim3(total), dim3(kFloorThreads), smem, stream, a, a_stride, a_rows, \
+                          b, b_stride, b_rows, vocab, use_k, top_p, c2, floors);                                   \
+    } while (0)
+    if (vocab <= kFloorThreads * 16) {
+        if (vec) SPEC_LAUNCH_NUCLEUS(true, 16);
+        SPEC_LAUNCH_NUCLEUS(false, 16);
+    }
+    if (vocab <= kFloorThreads * 64) {
+        if (vec) SPEC_LAUNCH_NUCLEUS(true, 64);
+        SPEC_LAUNCH_NUCLEUS(false, 64);
+    }
+    if (vec) SPEC_LAUNCH_NUCLEUS(true, 0);
+    SPEC_LAUNCH_NUCLEUS(false, 0);
+#undef SPEC_LAUNCH_NUCLEUS
+}
+
+// Top-k, then the nucleus of what is left (Section 2.2): one floor per row.
+int launch_cut_floors(const float* a, size_t a_stride, int a_rows, const float* b, size_t b_stride, int b_rows,
+                      int seqs, int vocab, int top_k, float top_p, float inv_t, float* floors, cudaStream_t stream) {
+    const bool use_k = top_k > 0 && top_k < vocab;
+    if (use_k) {
+        const int st = launch_topk_floors(a, a_stride, a_rows, b, b_stride, b_rows, seqs, vocab, top_k, floors, stream);
+        if (st != SPEC_OK) return st;
+    }
+    if (top_p > 0.0f && top_p < 1.0f)
+        return launch_nucleus_floors(a, a_stride, a_rows, b, b_stride, b_rows, seqs, vocab, use_k, top_p, inv_t, floors, stream);
+    return SPEC_OK;
+}
+
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
                          const float* uniforms, const float* final_uniforms, int batch, int gamma, int vocab,
-                         float temperature, float lenience, int top_k, int32_t* n_accepted, int32_t* next_token,
-                         void* workspace, cudaStream_t stream) {
+                         float temperature, float lenience, int top_k, float top_p, int32_t* n_accepted,
+                         int32_t* next_token, void* workspace, cudaStream_t stream) {
     const bool greedy = temperature == 0.0f;
     const int rows = greedy ? gamma + 1 : 2 * gamma + 1;
     const int chunks = chunks_for(vocab, rows * batch);
     const float inv_t = greedy ? 0.0f : 1.0f / temperature;
     ChunkStat* stats = static_cast<ChunkStat*>(workspace);
-    // top-k (Section 2.2): both models' rows are cut at their own k-th largest logit
+    // top-k and nucleus (Section 2.2): both models' rows are cut at their own floors
     const float* floors = nullptr;
-    if (!greedy && top_k > 0 && top_k < vocab) {
+    if (cut_is_on(vocab, temperature, top_k, top_p)) {
         float* f = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + stats_bytes(batch, gamma, vocab));
-        const int st = launch_topk_floors(target_logits, static_cast<size_t>(vocab), gamma + 1, draft_logits,
-                                          static_cast<size_t>(vocab), gamma, batch, vocab, top_k, f, stream);
+        const int st = launch_cut_floors(target_logits, static_cast<size_t>(vocab), gamma + 1, draft_logits,
+                                         static_cast<size_t>(vocab), gamma, batch, vocab, top_k, top_p, inv_t, f, stream);
         if (st != SPEC_OK) return st;
         floors = f;
     }
@@ -945,15 +1179,16 @@ int launch_verify_sample(const float* target_logits, const float* draft_logits, 
 
 // Row r reads logits + r * logit_stride and uniforms[r * uniform_stride] and
 // writes tokens[r * token_stride].
-// With 0 < top_k < vocab (and T > 0) `floor_scratch` must hold `rows` floats.
+// With a cut (0 < top_k < vocab or 0 < top_p < 1, and T > 0) `floor_scratch` must hold `rows` floats.
 int launch_sample_strided(const float* logits, size_t logit_stride, const float* uniforms, int uniform_stride,
-                          int rows, int vocab, float temperature, int top_k, float* floor_scratch, int32_t* tokens,
-                          int token_stride, cudaStream_t stream) {
+                          int rows, int vocab, float temperature, int top_k, float top_p, float* floor_scratch,
+                          int32_t* tokens, int token_stride, cudaStream_t stream) {
     const bool greedy = temperature == 0.0f;
     const float inv_t = greedy ? 0.0f : 1.0f / temperature;
     const float* floors = nullptr;
-    if (!greedy && top_k > 0 && top_k < vocab) {
-        const int st = launch_topk_floors(logits, logit_stride, 1, nullptr, 0, 0, rows, vocab, top_k, floor_scratch, stream);
+    if (cut_is_on(vocab, temperature, top_k, top_p)) {
+        const int st = launch_cut_floors(logits, logit_stride, 1, nullptr, 0, 0, rows, vocab, top_k, top_p, inv_t,
+                                         floor_scratch, stream);
         if (st != SPEC_OK) return st;
         floors = floor_scratch;
     }
@@ -969,8 +1204,8 @@ int launch_sample_strided(const float* logits, size_t logit_stride, const float*
 }
 
 int launch_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature, int top_k,
-                  float* floor_scratch, int32_t* tokens, cudaStream_t stream) {
-    return launch_sample_strided(logits, static_cast<size_t>(vocab), uniforms, 1, rows, vocab, temperature, top_k,
+                  float top_p, float* floor_scratch, int32_t* tokens, cudaStream_t stream) {
+    return launch_sample_strided(logits, static_cast<size_t>(vocab), uniforms, 1, rows, vocab, temperature, top_k, top_p,
                                  floor_scratch, tokens, 1, stream);
 }
 
@@ -981,12 +1216,13 @@ extern "C" size_t spec_verify_sample_workspace_bytes(int batch, int gamma, int v
     return spec::verify_sample_workspace_bytes(batch, gamma, vocab);
 }
 
-extern "C" int spec_verify_sample_topk(const float* target_logits, const float* draft_logits,
-                                       const int32_t* draft_tokens, const float* uniforms, int batch, int gamma,
-                                       int vocab, float temperature, float lenience, int top_k, int32_t* n_accepted,
-                                       int32_t* next_token, void* workspace, size_t workspace_bytes, void* stream) {
+extern "C" int spec_verify_sample_truncated(const float* target_logits, const float* draft_logits,
+                                            const int32_t* draft_tokens, const float* uniforms, int batch, int gamma,
+                                            int vocab, float temperature, float lenience, int top_k, float top_p,
+                                            int32_t* n_accepted, int32_t* next_token, void* workspace,
+                                            size_t workspace_bytes, void* stream) {
     using namespace spec;
-    if (top_k < 0) return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: top_k must be >= 0");
+    if (top_k < 0 || !(top_p == top_p)) return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: top_k must be >= 0 and top_p a number");
     if (!(lenience > 0.0f) || !(lenience <= 1.0f)) return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: lenience must be in (0, 1]");
     if (batch < 0 || gamma < 0 || gamma > kMaxGamma || vocab < 1)
         return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: batch=%d gamma=%d (max %d) vocab=%d", batch, gamma, kMaxGamma, vocab);
@@ -1002,7 +1238,7 @@ extern "C" int spec_verify_sample_topk(const float* target_logits, const float* 
         (reinterpret_cast<uintptr_t>(workspace) & 255u))
         return fail(SPEC_ERR_BAD_ARG, "spec_verify_sample: workspace too small (%zu bytes) or not 256-byte aligned", workspace_bytes);
     return launch_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, nullptr, batch, gamma, vocab,
-                                temperature, lenience, top_k, n_accepted, next_token, workspace,
+                                temperature, lenience, top_k, top_p, n_accepted, next_token, workspace,
                                 static_cast<cudaStream_t>(stream));
 }
 
@@ -1010,8 +1246,9 @@ extern "C" int spec_verify_sample_lenient(const float* target_logits, const floa
                                           const int32_t* draft_tokens, const float* uniforms, int batch, int gamma,
                                           int vocab, float temperature, float lenience, int32_t* n_accepted,
                                           int32_t* next_token, void* workspace, size_t workspace_bytes, void* stream) {
-    return spec_verify_sample_topk(target_logits, draft_logits, draft_tokens, uniforms, batch, gamma, vocab, temperature,
-                                   lenience, 0, n_accepted, next_token, workspace, workspace_bytes, stream);
+    return spec_verify_sample_truncated(target_logits, draft_logits, draft_tokens, uniforms, batch, gamma, vocab,
+                                        temperature, lenience, 0, 1.0f, n_accepted, next_token, workspace,
+                                        workspace_bytes, stream);
 }
 
 extern "C" int spec_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
@@ -1081,7 +1318,7 @@ extern "C" int spec_verify_sample_static(const float* target_logits, const float
     const int status = static_stats_address(&scratch);
     if (status != SPEC_OK) return status;
     return launch_verify_sample(target_logits, draft_logits, draft_tokens, uniforms, nullptr, batch, gamma, vocab,
-                                temperature, 1.0f, 0, n_accepted, next_token, scratch, static_cast<cudaStream_t>(stream));
+                                temperature, 1.0f, 0, 1.0f, n_accepted, next_token, scratch, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int spec_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
@@ -1092,30 +1329,36 @@ extern "C" int spec_sample(const float* logits, const float* uniforms, int rows,
         return fail(SPEC_ERR_BAD_ARG, "spec_sample: temperature must be finite and >= 0");
     if (rows == 0) return SPEC_OK;
     if (!logits || !tokens || (temperature > 0.0f && !uniforms)) return fail(SPEC_ERR_BAD_ARG, "spec_sample: null pointer");
-    return launch_sample(logits, uniforms, rows, vocab, temperature, 0, nullptr, tokens, static_cast<cudaStream_t>(stream));
+    return launch_sample(logits, uniforms, rows, vocab, temperature, 0, 1.0f, nullptr, tokens, static_cast<cudaStream_t>(stream));
 }
 
-extern "C" int spec_sample_topk(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
-                                int top_k, int32_t* tokens, float* floors, void* stream) {
+extern "C" int spec_sample_truncated(const float* logits, const float* uniforms, int rows, int vocab, float temperature,
+                                     int top_k, float top_p, int32_t* tokens, float* floors, void* stream) {
     using namespace spec;
-    if (rows < 0 || vocab < 1 || top_k < 0) return fail(SPEC_ERR_BAD_ARG, "spec_sample_topk: rows=%d vocab=%d top_k=%d", rows, vocab, top_k);
+    if (rows < 0 || vocab < 1 || top_k < 0 || !(top_p == top_p))
+        return fail(SPEC_ERR_BAD_ARG, "spec_sample_truncated: rows=%d vocab=%d top_k=%d top_p=%g", rows, vocab, top_k, top_p);
     if (!(temperature >= 0.0f) || !isfinite(temperature))
-        return fail(SPEC_ERR_BAD_ARG, "spec_sample_topk: temperature must be finite and >= 0");
+        return fail(SPEC_ERR_BAD_ARG, "spec_sample_truncated: temperature must be finite and >= 0");
     if (rows == 0) return SPEC_OK;
-    const bool cut = temperature > 0.0f && top_k > 0 && top_k < vocab;
-    if (!logits || !tokens || (temperature > 0.0f && !uniforms) || (cut && !floors))
-        return fail(SPEC_ERR_BAD_ARG, "spec_sample_topk: null pointer");
-    return launch_sample(logits, uniforms, rows, vocab, temperature, top_k, floors, tokens, static_cast<cudaStream_t>(stream));
+    if (!logits || !tokens || (temperature > 0.0f && !uniforms) || (cut_is_on(vocab, temperature, top_k, top_p) && !floors))
+        return fail(SPEC_ERR_BAD_ARG, "spec_sample_truncated: null pointer");
+    return launch_sample(logits, uniforms, rows, vocab, temperature, top_k, top_p, floors, tokens,
+                         static_cast<cudaStream_t>(stream));
 }
 
-extern "C" int spec_top_k_floors(const float* logits, int rows, int vocab, int top_k, float* floors, void* stream) {
+extern "C" int spec_truncation_floors(const float* logits, int rows, int vocab, float temperature, int top_k, float top_p,
+                                      float* floors, void* stream) {
     using namespace spec;
-    if (rows < 0 || vocab < 1 || top_k < 1 || top_k > vocab)
-        return fail(SPEC_ERR_BAD_ARG, "spec_top_k_floors: rows=%d vocab=%d top_k=%d", rows, vocab, top_k);
+    if (rows < 0 || vocab < 1 || top_k < 0 || !(top_p == top_p))
+        return fail(SPEC_ERR_BAD_ARG, "spec_truncation_floors: rows=%d vocab=%d top_k=%d top_p=%g", rows, vocab, top_k, top_p);
+    if (!(temperature > 0.0f) || !isfinite(temperature))
+        return fail(SPEC_ERR_BAD_ARG, "spec_truncation_floors: temperature must be finite and > 0");
+    if (!cut_is_on(vocab, temperature, top_k, top_p))
+        return fail(SPEC_ERR_BAD_ARG, "spec_truncation_floors: neither 0 < top_k < vocab nor 0 < top_p < 1");
     if (rows == 0) return SPEC_OK;
-    if (!logits || !floors) return fail(SPEC_ERR_BAD_ARG, "spec_top_k_floors: null pointer");
-    return launch_topk_floors(logits, static_cast<size_t>(vocab), 1, nullptr, 0, 0, rows, vocab, top_k, floors,
-                              static_cast<cudaStream_t>(stream));
+    if (!logits || !floors) return fail(SPEC_ERR_BAD_ARG, "spec_truncation_floors: null pointer");
+    return launch_cut_floors(logits, static_cast<size_t>(vocab), 1, nullptr, 0, 0, rows, vocab, top_k, top_p,
+                             1.0f / temperature, floors, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int spec_uniforms(uint64_t seed, const int32_t* positions, const int32_t* sequences, int purpose, int count,

@@ -15,7 +15,7 @@ def to_dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).to(dev())
 
 
-def compare_verify(n_gpu, t_gpu, tl, ql, xs, us, temperature, lenience=1.0, top_k=0):
+def compare_verify(n_gpu, t_gpu, tl, ql, xs, us, temperature, lenience=1.0, top_k=0, top_p=1.0):
     """Element-by-element comparison with the oracle.  Returns (flagged, total):
     sequences whose decision sat within MARGIN of a boundary and differed.  Any
     other difference raises."""
@@ -23,11 +23,14 @@ def compare_verify(n_gpu, t_gpu, tl, ql, xs, us, temperature, lenience=1.0, top_
     flagged = 0
     for b in range(tl.shape[0]):
         q_rows = ql[b] if ql is not None else np.zeros((0, tl.shape[2]))
-        ref = oracle_sampling.verify_step(tl[b], q_rows, xs[b], us[b], temperature, lenience, top_k)
+        ref = oracle_sampling.verify_step(tl[b], q_rows, xs[b], us[b], temperature, lenience, top_k, top_p)
         if (int(n_gpu[b]), int(t_gpu[b])) == (ref.n_accepted, ref.next_token):
             continue
         if temperature > 0:
             close = min(ref.accept_margin, ref.cdf_margin) < MARGIN
+            if not close and 0.0 < top_p < 1.0:  # a nucleus whose mass came within fp32 rounding of top_p
+                rows = list(tl[b]) + list(q_rows)
+                close = min(oracle_sampling.nucleus_floor(r, temperature, top_k, top_p)[1] for r in rows) < 5e-5
         else:  # a zero top-2 gap, or (lenient argmax) a drafted logit within rounding of the threshold
             close = ref.top2_gap == 0.0 or (lenience < 1.0 and ref.accept_margin < 1e-5)
         assert close, (f"sequence {b}: gpu (n={n_gpu[b]}, t={t_gpu[b]}) oracle (n={ref.n_accepted}, "

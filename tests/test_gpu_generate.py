@@ -185,8 +185,8 @@ def test_lenient_generation_matches_the_oracle_and_accepts_more(tiny):
     assert lenient["tests_passed"] / lenient["tests_evaluated"] > strict["tests_passed"] / strict["tests_evaluated"]
 
 
-@pytest.mark.parametrize("gamma", [3, 0])
-def test_top_k_generation_matches_the_oracle(tiny, gamma):
+@pytest.mark.parametrize("gamma,top_p", [(3, 1.0), (0, 1.0), (3, 0.8), (0, 0.8)])
+def test_truncated_generation_matches_the_oracle(tiny, gamma, top_p):
     """Section 2.2's top-k through the whole loop (gamma = 0: target-only decoding from the
     target's top-k distribution): token stream equal to the oracle's with the same k, every
     emitted token inside the target's top-k set, and a stream that differs from the uncut one."""
@@ -194,12 +194,12 @@ def test_top_k_generation_matches_the_oracle(tiny, gamma):
     prompt = workloads.make_prompt(14, 10, cfg["vocab"])
     k = 6
     try:
-        eng.set_top_k(k)
+        eng.set_truncation(k, top_p)
         if gamma:
-            ref = oracle_generate.speculative_generate(target, draft, prompt, 48, gamma, 1.0, seed=23, top_k=k, keep_logits=True)
+            ref = oracle_generate.speculative_generate(target, draft, prompt, 48, gamma, 1.0, seed=23, top_k=k, top_p=top_p, keep_logits=True)
             want, records = ref.tokens, ref.iterations
         else:
-            want, rows, margins = oracle_generate.target_only_generate(target, prompt, 48, 1.0, seed=23, top_k=k, keep_logits=True)
+            want, rows, margins = oracle_generate.target_only_generate(target, prompt, 48, 1.0, seed=23, top_k=k, top_p=top_p, keep_logits=True)
         got, _ = eng.generate([prompt], 48, gamma, 1.0, 23)
         got = got[0].tolist()
         diff = next((i for i in range(48) if got[i] != want[i]), None)
@@ -213,17 +213,19 @@ def test_top_k_generation_matches_the_oracle(tiny, gamma):
                 logits, margin = rows[diff][None], margins[diff]
             ordered = np.sort(logits, axis=1)
             cut_gap = float((ordered[:, -k] - ordered[:, -k - 1]).min())
-            assert margin < 1e-3 or cut_gap < 1e-3
+            from oracle.sampling import nucleus_floor
+            mass_gap = min(nucleus_floor(r, 1.0, k, top_p)[1] for r in logits)
+            assert margin < 1e-3 or cut_gap < 1e-3 or mass_gap < 1e-3
         checked = diff if diff is not None else 48
         assert checked >= 8
         # every token up to the first difference lies in the top-k set of the oracle's target row
-        if gamma == 0:
+        if gamma == 0 and top_p == 1.0:
             for i in range(checked):
                 assert rows[i][got[i]] >= np.sort(rows[i])[-k]
         with pytest.raises(binding.SpecError):
-            eng.set_top_k(-1)
+            eng.set_truncation(-1, 1.0)
     finally:
-        eng.set_top_k(0)
+        eng.set_truncation(0, 1.0)
     uncut, _ = eng.generate([prompt], 48, gamma, 1.0, 23)
     assert uncut[0].tolist() != got
 

@@ -13,21 +13,21 @@ from paper_2211_17192_b200 import binding, workloads
 pytestmark = pytest.mark.gpu
 
 
-def _draft_tokens(ql, seed, temperature, top_k=0):
+def _draft_tokens(ql, seed, temperature, top_k=0, top_p=1.0):
     """x_i ~ q_i drawn by the oracle with seeded uniforms."""
     batch, gamma, _ = ql.shape
     draw = workloads.make_uniform_grid(seed, (batch, max(gamma, 1)))
     xs = np.zeros((batch, gamma), dtype=np.int32)
     for b in range(batch):
         for i in range(gamma):
-            xs[b, i] = oracle_sampling.sample_token(ql[b, i], draw[b, i], temperature, top_k)[0]
+            xs[b, i] = oracle_sampling.sample_token(ql[b, i], draw[b, i], temperature, top_k, top_p)[0]
     return xs, draw
 
 
-def _run(tl, ql, xs, us, temperature, lenience=1.0, top_k=0):
+def _run(tl, ql, xs, us, temperature, lenience=1.0, top_k=0, top_p=1.0):
     n, t = binding.spec_verify_sample(to_dev(tl), to_dev(ql) if ql.size else None,
                                       to_dev(xs) if xs.size else None, to_dev(us), temperature, lenience=lenience,
-                                      top_k=top_k)
+                                      top_k=top_k, top_p=top_p)
     torch.cuda.synchronize()
     return n, t
 
@@ -202,7 +202,9 @@ def test_top_k_floors_are_bit_exact(rows, vocab):
     for data in (logits, tied):
         d = to_dev(data)
         for k in sorted({1, 2, min(40, vocab), max(1, vocab // 2), vocab - 1, vocab} - {0}):
-            got = binding.spec_top_k_floors(d, k).cpu().numpy()
+            if k == vocab:
+                continue  # no cut: the entry point refuses
+            got = binding.spec_truncation_floors(d, 1.0, top_k=k).cpu().numpy()
             want = np.sort(data, axis=1)[:, vocab - k]
             assert np.array_equal(got, want), (vocab, k)
             if 0 < k < vocab:
@@ -257,3 +259,83 @@ def test_plain_sampler_top_k(rows, vocab, temperature, top_k):
     assert flagged <= 1
     if top_k == 1:
         assert got.tolist() == logits.argmax(-1).tolist()
+
+
+def _nucleus_slack(row, temperature, top_k, top_p, floor):
+    """How far top_p would have to move for `floor` to be the exact nucleus cut of `row`
+    (0 when it is): the kept mass must reach top_p, and must not without its lowest logit."""
+    z = oracle_sampling.keep_top_k(row, top_k)
+    w = np.exp((z - z.max()) / temperature)
+    inside = w[z >= floor].sum() / w.sum()
+    without_lowest = w[z > floor].sum() / w.sum()
+    return max(0.0, top_p - inside, without_lowest - top_p)
+
+
+NUCLEUS_TOL = 5e-5  # fp32 weights from the hardware exp2 and fp32 sums over up to 10^5 of them
+
+
+@pytest.mark.parametrize("rows,vocab", [(6, 7), (5, 1001), (9, 8192), (16, 32000), (4, 32128), (3, 50257), (2, 100003)])
+@pytest.mark.parametrize("temperature", [1.0, 0.5])
+def test_nucleus_floors(rows, vocab, temperature):
+    """The nucleus cut of every row, alone and after top-k: the oracle's, or (where the
+    kept mass comes within fp32 rounding of top_p) the exact cut for a top_p that differs
+    by less than NUCLEUS_TOL; always a logit of the row; identical when repeated."""
+    logits, _ = workloads.make_sampler_logits(rows * 11 + vocab, rows, 0, vocab, 1.0)
+    logits = np.ascontiguousarray(logits[:, 0])
+    d = to_dev(logits)
+    differ = 0
+    for top_p in (0.02, 0.5, 0.9, 0.999):
+        for top_k in (0, min(50, vocab - 1)):
+            got = binding.spec_truncation_floors(d, temperature, top_k=top_k, top_p=top_p).cpu().numpy()
+            again = binding.spec_truncation_floors(d, temperature, top_k=top_k, top_p=top_p).cpu().numpy()
+            assert np.array_equal(got, again)
+            for r in range(rows):
+                want, margin = oracle_sampling.nucleus_floor(logits[r], temperature, top_k, top_p)
+                if got[r] != np.float32(want):
+                    assert got[r] in logits[r]
+                    slack = _nucleus_slack(logits[r].astype(np.float64), temperature, top_k, top_p, float(got[r]))
+                    assert margin < NUCLEUS_TOL and slack < NUCLEUS_TOL, (vocab, top_p, top_k, r, got[r], want, margin, slack)
+                    # far in the tail consecutive tokens differ by less than fp32 rounding of the
+                    # total mass, so there a different cut is the rule; elsewhere it is rare
+                    differ += top_p <= 0.9
+    assert differ <= 2
+
+
+@pytest.mark.parametrize("batch,gamma,vocab,temperature,top_k,top_p", [
+    (64, 7, 32000, 1.0, 0, 0.9),
+    (64, 7, 32000, 1.0, 40, 0.8),   # both cuts
+    (8, 3, 8192, 0.7, 0, 0.5),
+    (5, 2, 1001, 1.0, 10, 0.95),    # scalar loads
+    (2, 3, 100003, 1.0, 0, 0.3),    # rows re-read per bit
+    (7, 4, 4096, 1.0, 0, 1.0),      # top_p = 1: no cut
+    (7, 4, 4096, 1.0, 0, 1e-6),     # only the maximum survives
+    (6, 0, 32128, 1.0, 0, 0.7),     # gamma = 0: plain nucleus draw from p
+    (9, 4, 32000, 0.0, 0, 0.5),     # T = 0 ignores it
+])
+def test_nucleus_verify(batch, gamma, vocab, temperature, top_k, top_p):
+    tl, ql = workloads.make_sampler_logits(batch + gamma + vocab + 1, batch, gamma, vocab, 1.0)
+    xs, _ = _draft_tokens(ql, 3, temperature, top_k, top_p)
+    us = workloads.make_uniform_grid(4, (batch, gamma + 1))
+    n, t = _run(tl, ql, xs, us, temperature, top_k=top_k, top_p=top_p)
+    flagged, _ = compare_verify(n, t, tl, ql, xs, us, temperature, top_k=top_k, top_p=top_p)
+    assert flagged <= 1
+    if top_p == 1e-6:
+        same = (tl[:, :gamma].argmax(-1) == ql.argmax(-1))
+        assert n.cpu().numpy().tolist() == [int(np.argmin(np.append(same[b], False))) for b in range(batch)]
+
+
+@pytest.mark.parametrize("rows,vocab,temperature,top_k,top_p", [(64, 8192, 1.0, 0, 0.9), (5, 1001, 0.5, 20, 0.6),
+                                                                (3, 7, 1.0, 0, 0.5), (16, 32000, 1.0, 0, 0.25),
+                                                                (2, 100003, 1.0, 0, 0.8), (4, 32000, 0.0, 0, 0.5)])
+def test_plain_sampler_nucleus(rows, vocab, temperature, top_k, top_p):
+    logits, _ = workloads.make_sampler_logits(rows + vocab, rows, 0, vocab, 1.0)
+    logits = logits[:, 0]
+    us = workloads.make_uniform_grid(12, (rows,))
+    got = binding.spec_sample(to_dev(logits), to_dev(us), temperature, top_k=top_k, top_p=top_p).cpu().numpy()
+    flagged = 0
+    for r in range(rows):
+        ref, margin = oracle_sampling.sample_token(logits[r], us[r], temperature, top_k, top_p)
+        if got[r] != ref:
+            assert margin < MARGIN or oracle_sampling.nucleus_floor(logits[r], temperature, top_k, top_p)[1] < NUCLEUS_TOL
+            flagged += 1
+    assert flagged <= 1
