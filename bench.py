@@ -250,6 +250,7 @@ class GenerationWorkload:
         self.layers = layers
         self.tcfg, self.dcfg = workloads.model_config(target), workloads.model_config(draft)  # (prepare applies --layers)
         self.batch, self.prompt_len, self.n_new, self.gamma, self.temperature = batch, prompt_len, n_new, gamma, temperature
+        self.adaptive_gamma_max = 0  # set from the command line
 
     def description(self):
         return {"workload": self.name, "target": self.target_name, "draft": self.draft_name, "batch": self.batch,
@@ -271,9 +272,10 @@ class GenerationWorkload:
         self.tw = gpu_weights(self.tcfg, 100 + rank, device)
         self.dw = gpu_weights(self.dcfg, 200 + rank, device)
         grow = max(self.n_new, iterations * (self.gamma + 1) + 64)
-        self.max_len = self.prompt_len + grow + self.gamma + 2
+        top_gamma = max(self.gamma, self.adaptive_gamma_max, 1)
+        self.max_len = self.prompt_len + grow + top_gamma + 2
         self.engine = binding.Engine(self.tcfg, self.tw, self.dcfg, self.dw, max_batch=self.batch, max_len=self.max_len,
-                                     page_size=64, max_gamma=max(self.gamma, 1))
+                                     page_size=64, max_gamma=top_gamma)
         self.prompts = [workloads.make_prompt(1000 * rank + b, self.prompt_len, self.tcfg["vocab"]) for b in range(self.batch)]
         self.budget_tokens = grow
 
@@ -306,6 +308,19 @@ class GenerationWorkload:
 
     def e2e_bytes(self):
         return self.batch * self.prompt_len * 4 + self.batch * 4, self.batch * self.n_new * 4
+
+    def adaptive(self, gamma_max):
+        """Section 3.5: gamma picked by the library burst by burst; decode time only, like `timed_decode`."""
+        self.engine.generate_adaptive(self.prompts, self.n_new, gamma_max, self.temperature, 7)  # captures the graphs
+        out, st, trace = self.engine.generate_adaptive(self.prompts, self.n_new, gamma_max, self.temperature, 7)
+        used = {}
+        for g, n in trace:
+            used[g] = used.get(g, 0) + n
+        return {"gamma_max": gamma_max, "tokens_per_s": out.size / (st["decode_ms"] / 1e3),
+                "iterations_by_gamma": {str(g): used[g] for g in sorted(used)},
+                "alpha": st["tests_passed"] / max(1, st["tests_evaluated"]),
+                "note": "spec_generate_adaptive over n_new tokens: two calibration bursts (gamma 1 and gamma_max), then "
+                        "the gamma that maximises Eq. 1 over a line fitted to the measured iteration times"}
 
     def pass_times(self, repeats=20):
         """Device time of single passes (graph-replayed, events on the library's stream):
@@ -423,9 +438,10 @@ class EncDecWorkload(GenerationWorkload):
         self.tw = gpu_weights(self.tcfg, 100 + rank, device)
         self.dw = gpu_weights(self.dcfg, 200 + rank, device)
         grow = max(self.n_new, iterations * (self.gamma + 1) + 64)
-        self.max_len = 1 + grow + self.gamma + 2
+        top_gamma = max(self.gamma, self.adaptive_gamma_max, 1)
+        self.max_len = 1 + grow + top_gamma + 2
         self.engine = binding.Engine(self.tcfg, self.tw, self.dcfg, self.dw, max_batch=self.batch, max_len=self.max_len,
-                                     page_size=64, max_gamma=max(self.gamma, 1), max_src_len=self.prompt_len)
+                                     page_size=64, max_gamma=top_gamma, max_src_len=self.prompt_len)
         self.prompts = [workloads.make_prompt(1000 * rank + b, self.prompt_len, self.tcfg["vocab"]) for b in range(self.batch)]
         self.budget_tokens = grow
 
@@ -488,6 +504,12 @@ class EncDecWorkload(GenerationWorkload):
 
 
 def make_workload(args):
+    wl = _make_workload(args)
+    wl.adaptive_gamma_max = args.adaptive_gamma_max
+    return wl
+
+
+def _make_workload(args):
     if args.workload == "sampler":
         return SamplerWorkload()
     batch = args.batch or 1
@@ -693,6 +715,7 @@ def run_generation(args, wl, torch, device, local, barrier):
                                times["target_1row_ms"] * (1.0 + (times["target_rows_ms"] / times["target_1row_ms"] - 1.0) * g_ / max(wl.gamma, 1)),
                                times["draft_1row_ms"], g_)) if 0.0 < alpha < 1.0 else None},
             "imposed_acceptance_sweep": sweep,
+            **({"adaptive_gamma": wl.adaptive(wl.adaptive_gamma_max)} if wl.adaptive_gamma_max else {}),
             "verify_pass": {"bytes": pass_bytes, "ms": times["target_rows_ms"],
                             "gbs": pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9,
                             "frac": pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9 / peak,
@@ -727,6 +750,8 @@ def main():
     ap.add_argument("--draft", default="model", choices=["model", "bigram"],
                     help="llama7b workload: the 160M-shaped draft model, or a bigram table (negligible-cost draft)")
     ap.add_argument("--layers", type=int, default=None, help="override the target's depth, full width (profiling)")
+    ap.add_argument("--adaptive-gamma-max", type=int, default=0,
+                    help="also report decoding with gamma chosen by the library burst by burst, up to this value")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for cpu_baseline")
     args = ap.parse_args()

@@ -433,6 +433,43 @@ int spec_rel_bucket(int delta, int bidirectional, int n_buckets, int max_distanc
 int spec_step(spec_ctx* ctx, int iterations, int* remaining, spec_stats* stats);
 int spec_read_tokens(spec_ctx* ctx, int32_t* out_tokens);
 
+/* Choosing gamma (Section 3.5: the optimal gamma is the integer that maximises
+ * the walltime improvement for given alpha and c; the same section names
+ * varying gamma during a run as a further refinement and leaves it open).
+ *
+ * spec_choose_gamma is host arithmetic, no device involved: the gamma in
+ * [1, gamma_max] that maximises expected tokens per unit of time,
+ *   (1 + alpha + ... + alpha^gamma) / (base_cost + cost_per_guess * gamma),
+ * the numerator being Eq. 1; lowest gamma on ties.  With base_cost = 1 and
+ * cost_per_guess = c this is the maximiser of Theorem 3.8's improvement factor
+ * (1 - alpha^(gamma+1)) / ((1 - alpha)(gamma c + 1)).  Returns -1 for alpha
+ * outside [0, 1], base_cost <= 0, cost_per_guess < 0 or gamma_max < 1.
+ *
+ * spec_set_gamma changes the number of guesses per iteration of the generation
+ * in progress, between spec_step calls: 1 <= gamma <= the gamma given to
+ * spec_begin (whose capacity check covers it).  gamma = 0 is refused: such
+ * iterations would not feed the draft model.  Iteration graphs are kept per
+ * gamma, so going back to an earlier gamma costs nothing.  Because the
+ * randomness is keyed by position, the tokens depend on the sequence of gammas
+ * but on nothing else; at T = 0 they do not depend on it at all.
+ *
+ * spec_generate_adaptive is spec_generate with gamma chosen by the library:
+ * iterations run in bursts of at most `burst`; the first burst uses gamma = 1,
+ * the second gamma_max, and from then on the gamma spec_choose_gamma returns
+ * for alpha = accepted / evaluated guesses so far, with the counts of earlier
+ * bursts fading by 0.8 per burst, and a straight line fitted to the measured
+ * device time per iteration of every gamma tried.  trace (HOST int32, may be
+ * NULL with trace_capacity 0) receives (gamma, iterations) per burst, as many
+ * pairs as fit; *n_bursts (may be NULL) the number of bursts.  Replaying the
+ * trace with spec_begin / spec_set_gamma / spec_step gives the same tokens.
+ * Errors as spec_generate; gamma_max < 1 or burst < 1: SPEC_ERR_BAD_ARG. */
+int spec_choose_gamma(double alpha, double base_cost, double cost_per_guess, int gamma_max);
+int spec_set_gamma(spec_ctx* ctx, int gamma);
+int spec_generate_adaptive(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride,
+                           int batch, int n_new, int gamma_max, float temperature, uint64_t seed, int burst,
+                           int32_t* out_tokens, spec_stats* stats, int32_t* trace, int trace_capacity,
+                           int* n_bursts);
+
 /* Diagnostics for parity tests: teacher-forced forward passes on the KV caches.
  * spec_reset forgets every cached row.  spec_forward_logits feeds, for each
  * of `batch` sequences, `rows` tokens at positions cached_len[b].. of model

@@ -69,6 +69,10 @@ def speculative_generate(target, draft, prompt, n_new, gamma, temperature, seed,
                          lenience=1.0, top_k=0, top_p=1.0):
     """Algorithm 1 repeated until n_new tokens are emitted.
 
+    `gamma` is an integer, or a sequence giving the number of guesses of every
+    iteration in turn (Section 3.5 allows gamma to vary during a run; the last
+    entry is used for any further iterations).
+
     `target` and `draft` are model objects with forward_rows / forward_full /
     truncate / reset (oracle.decoder.Decoder or a table model from the tests).
     """
@@ -82,8 +86,11 @@ def speculative_generate(target, draft, prompt, n_new, gamma, temperature, seed,
             target.forward_rows(committed[:-1])
             draft.forward_rows(committed[:-1])
 
+    schedule = None if np.isscalar(gamma) else [int(g) for g in gamma]
     while len(committed) - prompt_len < n_new:
         L = len(committed)
+        if schedule is not None:
+            gamma = schedule[min(len(result.iterations), len(schedule) - 1)]
         # Draft gamma guesses autoregressively.
         xs, q_logits, draft_margins = [], [], []
         for i in range(1, gamma + 1):

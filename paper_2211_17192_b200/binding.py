@@ -207,6 +207,18 @@ def spec_sample(logits, uniforms, temperature, tokens=None, top_k=0, top_p=1.0):
     return tokens
 
 
+def spec_choose_gamma(alpha, base_cost, cost_per_guess, gamma_max):
+    """The gamma in [1, gamma_max] maximising (1 + alpha + ... + alpha^gamma) / (base_cost + cost_per_guess * gamma);
+    host arithmetic of the library (no GPU needed)."""
+    h = lib()
+    h.spec_choose_gamma.restype = ctypes.c_int
+    h.spec_choose_gamma.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_int]
+    g = h.spec_choose_gamma(float(alpha), float(base_cost), float(cost_per_guess), int(gamma_max))
+    if g < 0:
+        raise ValueError("spec_choose_gamma: alpha in [0, 1], base_cost > 0, cost_per_guess >= 0, gamma_max >= 1")
+    return g
+
+
 def spec_uniforms(seed, positions, sequences, purpose, out=None):
     """The method's uniforms for (position, sequence) pairs; int32 CUDA inputs."""
     count = positions.numel()
@@ -497,6 +509,39 @@ class Engine:
                                    float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF, out.ctypes.data,
                                    ctypes.byref(st)))
         return out, {name: getattr(st, name) for name, _ in _Stats._fields_}
+
+    def generate_adaptive(self, prompts, n_new, gamma_max, temperature, seed, burst=4):
+        """`generate` with gamma chosen by the library burst by burst (`spec_generate_adaptive`).
+        Returns (tokens [B, n_new], stats dict, trace): trace is the list of (gamma, iterations) per burst."""
+        np = self._np
+        batch = len(prompts)
+        lens = np.array([len(p) for p in prompts], dtype=np.int32)
+        stride = int(lens.max())
+        flat = np.zeros((batch, stride), dtype=np.int32)
+        for b, p in enumerate(prompts):
+            flat[b, : len(p)] = np.asarray(p, dtype=np.int32)
+        out = np.zeros((batch, n_new), dtype=np.int32)
+        capacity = 2 * (n_new + 2)  # every burst emits at least one token per unfinished sequence
+        trace = np.zeros(capacity, dtype=np.int32)
+        n_bursts = ctypes.c_int(0)
+        st = _Stats()
+        h = lib()
+        h.spec_generate_adaptive.restype = ctypes.c_int
+        h.spec_generate_adaptive.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                             ctypes.c_int, ctypes.c_int, ctypes.c_float, ctypes.c_uint64, ctypes.c_int,
+                                             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+        _check(h.spec_generate_adaptive(self._ctx, flat.ctypes.data, lens.ctypes.data, stride, batch, n_new, gamma_max,
+                                        float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF, int(burst), out.ctypes.data,
+                                        ctypes.byref(st), trace.ctypes.data, capacity, ctypes.byref(n_bursts)))
+        pairs = [(int(trace[2 * i]), int(trace[2 * i + 1])) for i in range(min(n_bursts.value, capacity // 2))]
+        return out, {name: getattr(st, name) for name, _ in _Stats._fields_}, pairs
+
+    def set_gamma(self, gamma):
+        """Number of guesses per iteration for the rest of the generation in progress (`spec_set_gamma`)."""
+        h = lib()
+        h.spec_set_gamma.restype = ctypes.c_int
+        h.spec_set_gamma.argtypes = [ctypes.c_void_p, ctypes.c_int]
+        _check(h.spec_set_gamma(self._ctx, int(gamma)))
 
     def set_lenience(self, lenience):
         """Lenience factor of Appendix A.5 for the generations that follow (1 = Algorithm 1)."""

@@ -50,8 +50,9 @@ struct spec_ctx {
     float top_p = 1.0f;           // and then over the nucleus of mass top_p; 1 = all
     float* sample_floors = nullptr;  // the draft rows' k-th largest logits, one per sequence
 
-    // cached iteration graph
-    cudaGraphExec_t graph = nullptr;
+    // cached iteration graphs, one per gamma, all for the same batch and sampling settings
+    std::vector<cudaGraphExec_t> graphs;  // indexed by gamma; nullptr = not captured yet
+    cudaGraphExec_t graph = nullptr;      // the one in use (an element of `graphs`)
     int graph_batch = -1, graph_gamma = -1;
     float graph_temperature = -1.0f, graph_lenience = 1.0f;
     int graph_top_k = 0;
@@ -59,7 +60,9 @@ struct spec_ctx {
 
     // generation in progress (spec_begin / spec_generate)
     int session_batch = 0, session_gamma = 0, session_n_new = 0;
-    long long session_replays = 0;
+    float session_temperature = 0.0f;
+    int session_gamma_cap = 0;  // the gamma the session's capacity was checked for (spec_set_gamma stays below it)
+    long long session_replays = 0, session_draft_passes = 0;
     float session_prefill_ms = 0.0f;
     std::vector<int32_t> session_prompt_len;
 
@@ -419,26 +422,38 @@ int enqueue_iteration(spec_ctx* ctx, int batch, int gamma, float temperature) {
                       ctx->tokens, ctx->length, ctx->counters);
 }
 
+void drop_graphs(spec_ctx* ctx) {
+    for (cudaGraphExec_t g : ctx->graphs)
+        if (g) cudaGraphExecDestroy(g);
+    ctx->graphs.assign(ctx->graphs.size(), nullptr);
+    ctx->graph = nullptr;
+}
+
+// Makes ctx->graph the iteration graph for (batch, gamma) under the current
+// sampling settings.  Graphs of other gammas captured under the same settings
+// are kept, so that a generation can move between gammas without re-capturing.
 int build_graph(spec_ctx* ctx, int batch, int gamma, float temperature) {
-    if (ctx->graph && ctx->graph_batch == batch && ctx->graph_gamma == gamma && ctx->graph_temperature == temperature &&
-        ctx->graph_lenience == ctx->lenience && ctx->graph_top_k == ctx->top_k && ctx->graph_top_p == ctx->top_p)
-        return SPEC_OK;
-    if (ctx->graph) {
-        cudaGraphExecDestroy(ctx->graph);
-        ctx->graph = nullptr;
+    if (ctx->graphs.size() < static_cast<size_t>(ctx->rt.max_gamma) + 1) ctx->graphs.resize(ctx->rt.max_gamma + 1, nullptr);
+    const bool same_settings = ctx->graph_batch == batch && ctx->graph_temperature == temperature &&
+                               ctx->graph_lenience == ctx->lenience && ctx->graph_top_k == ctx->top_k &&
+                               ctx->graph_top_p == ctx->top_p;
+    if (!same_settings) drop_graphs(ctx);
+    if (!ctx->graphs[gamma]) {
+        SPEC_CUDA_TRY(cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
+        const int status = enqueue_iteration(ctx, batch, gamma, temperature);
+        cudaGraph_t g = nullptr;
+        const cudaError_t err = cudaStreamEndCapture(ctx->stream, &g);
+        if (status != SPEC_OK) {
+            if (g) cudaGraphDestroy(g);
+            return status;
+        }
+        SPEC_CUDA_TRY(err);
+        const cudaError_t ierr = cudaGraphInstantiate(&ctx->graphs[gamma], g, 0);
+        cudaGraphDestroy(g);
+        if (ierr != cudaSuccess) ctx->graphs[gamma] = nullptr;
+        SPEC_CUDA_TRY(ierr);
     }
-    SPEC_CUDA_TRY(cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
-    const int status = enqueue_iteration(ctx, batch, gamma, temperature);
-    cudaGraph_t g = nullptr;
-    const cudaError_t err = cudaStreamEndCapture(ctx->stream, &g);
-    if (status != SPEC_OK) {
-        if (g) cudaGraphDestroy(g);
-        return status;
-    }
-    SPEC_CUDA_TRY(err);
-    const cudaError_t ierr = cudaGraphInstantiate(&ctx->graph, g, 0);
-    cudaGraphDestroy(g);
-    SPEC_CUDA_TRY(ierr);
+    ctx->graph = ctx->graphs[gamma];
     ctx->graph_batch = batch;
     ctx->graph_gamma = gamma;
     ctx->graph_temperature = temperature;
@@ -792,7 +807,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
 extern "C" void spec_free(spec_ctx* ctx) {
     if (!ctx) return;
     if (ctx->stream) cudaStreamSynchronize(ctx->stream);
-    if (ctx->graph) cudaGraphExecDestroy(ctx->graph);
+    drop_graphs(ctx);
     for (void* p : ctx->allocations) cudaFree(p);
     for (auto& e : ctx->ev)
         if (e) cudaEventDestroy(e);
@@ -902,6 +917,9 @@ int begin_session(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_le
     ctx->session_prefill_ms = pre;
     ctx->session_batch = batch;
     ctx->session_gamma = gamma;
+    ctx->session_gamma_cap = gamma;
+    ctx->session_temperature = temperature;
+    ctx->session_draft_passes = 0;
     ctx->session_n_new = n_new;
     ctx->session_replays = 0;
     ctx->session_prompt_len.assign(prompt_len, prompt_len + batch);
@@ -921,6 +939,7 @@ int run_iterations(spec_ctx* ctx, int iterations, float* elapsed_ms, int* remain
     for (int i = 0; i < iterations; ++i) SPEC_CUDA_TRY(cudaGraphLaunch(ctx->graph, st));
     SPEC_CUDA_TRY(cudaEventRecord(ctx->ev[2], st));
     ctx->session_replays += iterations;
+    ctx->session_draft_passes += static_cast<long long>(iterations) * ctx->session_gamma;
     SPEC_CUDA_TRY(cudaMemcpyAsync(lengths.data(), ctx->length, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     SPEC_CUDA_TRY(cudaStreamSynchronize(st));
     if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
@@ -939,7 +958,7 @@ int fill_stats(spec_ctx* ctx, double decode_ms, spec_stats* stats) {
     stats->tests_evaluated = static_cast<int64_t>(counters[2]);
     stats->tests_passed = static_cast<int64_t>(counters[3]);
     stats->target_passes = ctx->session_replays;
-    stats->draft_passes = ctx->session_replays * ctx->session_gamma;
+    stats->draft_passes = ctx->session_draft_passes;
     stats->prefill_ms = ctx->session_prefill_ms;
     stats->decode_ms = decode_ms;
     return SPEC_OK;
@@ -992,6 +1011,102 @@ extern "C" int spec_read_tokens(spec_ctx* ctx, int32_t* out_tokens) {
     SPEC_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
     for (int b = 0; b < batch; ++b)
         std::memcpy(out_tokens + static_cast<size_t>(b) * n_new, &host_tokens[static_cast<size_t>(b) * max_len + ctx->session_prompt_len[b]], n_new * sizeof(int32_t));
+    return SPEC_OK;
+}
+
+extern "C" int spec_set_gamma(spec_ctx* ctx, int gamma) {
+    if (!ctx) return fail(SPEC_ERR_BAD_ARG, "spec_set_gamma: null context");
+    if (ctx->session_batch < 1) return fail(SPEC_ERR_BAD_ARG, "spec_set_gamma: no generation in progress (call spec_begin)");
+    // gamma = 0 iterations do not feed the draft, whose cache would then lag behind the committed tokens
+    if (ctx->session_gamma_cap < 1 || gamma < 1 || gamma > ctx->session_gamma_cap)
+        return fail(SPEC_ERR_BAD_ARG, "spec_set_gamma: gamma %d outside [1, %d] (the gamma given to spec_begin)", gamma,
+                    ctx->session_gamma_cap);
+    SPEC_TRY(build_graph(ctx, ctx->session_batch, gamma, ctx->session_temperature));
+    ctx->session_gamma = gamma;
+    return SPEC_OK;
+}
+
+extern "C" int spec_choose_gamma(double alpha, double base_cost, double cost_per_guess, int gamma_max) {
+    if (!(alpha >= 0.0) || !(alpha <= 1.0) || !(base_cost > 0.0) || !(cost_per_guess >= 0.0) || gamma_max < 1) return -1;
+    int best = 1;
+    double best_rate = -1.0;
+    for (int g = 1; g <= gamma_max; ++g) {
+        // Eq. 1: expected tokens per iteration, 1 + alpha + ... + alpha^g
+        double tokens = 0.0, term = 1.0;
+        for (int i = 0; i <= g; ++i) {
+            tokens += term;
+            term *= alpha;
+        }
+        const double rate = tokens / (base_cost + cost_per_guess * g);
+        if (rate > best_rate) {
+            best_rate = rate;
+            best = g;
+        }
+    }
+    return best;
+}
+
+extern "C" int spec_generate_adaptive(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_len, int prompt_stride,
+                                      int batch, int n_new, int gamma_max, float temperature, uint64_t seed, int burst,
+                                      int32_t* out_tokens, spec_stats* stats, int32_t* trace, int trace_capacity,
+                                      int* n_bursts) {
+    if (!out_tokens || burst < 1 || gamma_max < 1 || trace_capacity < 0 || (trace_capacity > 0 && !trace))
+        return fail(SPEC_ERR_BAD_ARG, "spec_generate_adaptive: bad argument");
+    SPEC_TRY(begin_session(ctx, prompt, prompt_len, prompt_stride, batch, n_new, gamma_max, temperature, seed));
+    // Iteration time is modelled as base + per_guess * gamma (one target pass and the
+    // sampler; one draft pass and one more target row per guess) and fitted to the
+    // bursts run so far; alpha is the running estimate of Definition 3.1's E(beta).
+    std::vector<double> time_sum(gamma_max + 1, 0.0), iters(gamma_max + 1, 0.0);
+    double alpha = 0.5, decode_ms = 0.0;
+    double recent_evaluated = 0.0, recent_passed = 0.0;  // counts that fade by kFade per burst
+    constexpr double kFade = 0.8;
+    long long seen_evaluated = 0, seen_passed = 0;
+    int remaining = n_new, bursts = 0;
+    while (remaining > 0) {
+        int gamma;
+        if (bursts == 0) gamma = 1;                            // two calibration bursts span the range
+        else if (bursts == 1) gamma = gamma_max;
+        else {
+            // least squares through the mean iteration time of every gamma tried so far
+            double n = 0, sx = 0, sy = 0, sxx = 0, sxy = 0;
+            for (int g = 1; g <= gamma_max; ++g)
+                if (iters[g] > 0) {
+                    const double y = time_sum[g] / iters[g];
+                    n += 1; sx += g; sy += y; sxx += double(g) * g; sxy += g * y;
+                }
+            double per = 0.0, base = sy / n;
+            const double det = n * sxx - sx * sx;
+            if (det > 0) {
+                per = std::max(0.0, (n * sxy - sx * sy) / det);
+                base = std::max(1e-9, (sy - per * sx) / n);
+            }
+            gamma = spec_choose_gamma(alpha, base, per, gamma_max);
+        }
+        SPEC_TRY(spec_set_gamma(ctx, gamma));
+        const int count = std::min(burst, (remaining + gamma) / (gamma + 1));
+        float ms = 0.0f;
+        SPEC_TRY(run_iterations(ctx, count, &ms, &remaining));
+        decode_ms += ms;
+        time_sum[gamma] += ms;
+        iters[gamma] += count;
+        if (2 * bursts + 1 < trace_capacity) {
+            trace[2 * bursts] = gamma;
+            trace[2 * bursts + 1] = count;
+        }
+        ++bursts;
+        unsigned long long counters[4];
+        SPEC_CUDA_TRY(cudaMemcpy(counters, ctx->counters, sizeof(counters), cudaMemcpyDeviceToHost));
+        const long long evaluated = static_cast<long long>(counters[2]) - seen_evaluated;
+        const long long passed = static_cast<long long>(counters[3]) - seen_passed;
+        seen_evaluated += evaluated;
+        seen_passed += passed;
+        recent_evaluated = kFade * recent_evaluated + static_cast<double>(evaluated);
+        recent_passed = kFade * recent_passed + static_cast<double>(passed);
+        if (recent_evaluated > 0.0) alpha = recent_passed / recent_evaluated;
+    }
+    if (n_bursts) *n_bursts = bursts;
+    SPEC_TRY(spec_read_tokens(ctx, out_tokens));
+    if (stats) SPEC_TRY(fill_stats(ctx, decode_ms, stats));
     return SPEC_OK;
 }
 

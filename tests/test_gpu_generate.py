@@ -251,3 +251,40 @@ def test_bigram_table_draft_matches_the_oracle(temperature):
         assert np.array_equal(greedy, spec) and stats["draft_passes"] > 0
     finally:
         eng.close()
+
+
+def test_adaptive_gamma_generation(tiny):
+    """Section 3.5's varying gamma: the library picks gamma burst by burst.  The trace it reports,
+    replayed by the oracle (and by the phased entry points), gives the same tokens; at T = 0 the
+    output is the target's greedy decoding whatever the trace."""
+    eng, target, draft, cfg = tiny
+    prompt = workloads.make_prompt(41, 10, cfg["vocab"])
+    n_new, gamma_max = 72, 6
+    got, st, trace = eng.generate_adaptive([prompt], n_new, gamma_max, 1.0, 29, burst=3)
+    got = got[0].tolist()
+    assert trace[0][0] == 1 and trace[1][0] == gamma_max and all(1 <= g <= gamma_max for g, _ in trace)
+    assert sum(n for _, n in trace) == st["iterations"] == st["target_passes"]
+    assert sum(g * n for g, n in trace) == st["draft_passes"]
+    schedule = [g for g, n in trace for _ in range(n)]
+    ref = oracle_generate.speculative_generate(target, draft, prompt, n_new, schedule, 1.0, seed=29)
+    diff = next((k for k in range(n_new) if got[k] != ref.tokens[k]), None)
+    if diff is not None:  # a decision within tolerance of a boundary ends the comparison
+        index = len(prompt) + diff
+        it = next(i for i in ref.iterations if i.start_len <= index <= i.start_len + i.n_accepted)
+        assert min([it.accept_margin, it.cdf_margin] + list(it.draft_cdf_margins)) < 1e-3
+        assert diff >= 8
+    # the same trace through spec_begin / spec_set_gamma / spec_step
+    eng.begin([prompt], n_new, gamma_max, 1.0, 29)
+    for g, n in trace:
+        eng.set_gamma(g)
+        eng.step(n)
+    assert eng.read_tokens()[0].tolist() == got
+    with pytest.raises(binding.SpecError):
+        eng.set_gamma(0)
+    with pytest.raises(binding.SpecError):
+        eng.set_gamma(gamma_max + 1)
+    # T = 0: the target's greedy output, in a ragged batch
+    prompts = [prompt, workloads.make_prompt(42, 5, cfg["vocab"])]
+    greedy, _ = eng.generate(prompts, 40, 0, 0.0, 1)
+    adaptive, _, trace0 = eng.generate_adaptive(prompts, 40, gamma_max, 0.0, 1, burst=2)
+    assert np.array_equal(adaptive, greedy) and len({g for g, _ in trace0}) >= 2
