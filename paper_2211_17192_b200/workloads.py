@@ -48,6 +48,9 @@ def model_config(name):
         # bigram tables: negligible-cost drafts (next-token logits from the last token alone)
         "bigram_8k": dict(arch="bigram", vocab=8192, dtype="fp32", head_std=1.0),
         "bigram_32k": dict(arch="bigram", vocab=32000, dtype="bf16", head_std=0.3),
+        # copy-from-context drafts: parameter-less, guess = what followed the last `ngram` tokens before
+        "copy_8k": dict(arch="copy", vocab=8192, ngram=2, dtype="fp32"),
+        "copy_32k": dict(arch="copy", vocab=32000, ngram=2, dtype="fp32"),
         # T5-shaped encoder-decoder pair (XXL-shaped target, small-shaped draft), bf16
         "t5xxl_target": dict(arch="t5", ffn="gated_gelu", n_layers=24, n_enc_layers=24, d_model=4096, n_heads=64,
                              n_kv_heads=64, d_head=64, d_ff=10240, vocab=32128, max_positions=1024, dtype="bf16",
@@ -86,6 +89,8 @@ def tensor_shapes(cfg):
     """Ordered (name, shape, kind) of a model's tensors; kind is 'gain', 'matrix', 'bias' or 'head'."""
     if cfg["arch"] == "bigram":
         return [("table", (cfg["vocab"], cfg["vocab"]), "head")]
+    if cfg["arch"] == "copy":
+        return []
     d, H, Hkv, dh, F = cfg["d_model"], cfg["n_heads"], cfg["n_kv_heads"], cfg["d_head"], cfg["d_ff"]
     f_in = F if cfg["ffn"] == "gelu" else 2 * F
     t5 = cfg["arch"] == "t5"
@@ -163,6 +168,13 @@ def make_prompt(seed, length, vocab):
     """`length` token ids, uniform on [0, vocab)."""
     rng = np.random.default_rng([int(seed), 0x70726F6D])
     return rng.integers(0, vocab, size=length, dtype=np.int64).astype(np.int32)
+
+
+def make_repetitive_prompt(seed, length, vocab, period):
+    """`length` token ids that repeat a uniform segment of `period` tokens (contexts in which long
+    stretches recur, the case a copy-from-context draft is meant for)."""
+    segment = make_prompt(seed, period, vocab)
+    return np.tile(segment, length // period + 1)[:length].copy()
 
 
 def make_sampler_logits(seed, batch, gamma, vocab, draft_noise, logit_std=3.0):

@@ -170,3 +170,61 @@ def test_bigram_table_draft():
     want, _, _ = generate.target_only_generate(BigramTable(table), [1, 2], 25, 0.0, seed=0)
     got = generate.speculative_generate(BigramTable(table), other, [1, 2], 25, 3, 0.0, seed=0)
     assert got.tokens == want
+
+
+def test_copy_from_context_draft():
+    """Section 3.6's parameter-less draft.  The rule on hand-written sequences; a periodic target
+    accepts every guess once one period is in the context; a one-hot draft is accepted with
+    probability p(guess); T = 0 output equals the target's greedy output."""
+    from oracle.ngram import BigramTable, CopyFromContext
+    draft = CopyFromContext(10, 2)
+    #            0  1  2  3  4  5  6  7
+    assert draft.guess([1, 2, 3, 4, 1, 2]) == 3            # "1 2" was followed by 3
+    assert draft.guess([1, 2, 3, 1, 2, 5, 1, 2]) == 5      # the most recent occurrence wins
+    assert draft.guess([1, 2, 3, 4]) == 4                  # no earlier "3 4": repeat the last token
+    assert draft.guess([7]) == 7 and draft.guess([7, 7]) == 7
+    assert draft.guess([7, 7, 7]) == 7                     # overlapping occurrence: "7 7" ends at index 1
+    assert CopyFromContext(10, 1).guess([4, 9, 5, 4]) == 9
+    assert CopyFromContext(10, 3).guess([1, 2, 3, 9, 2, 3, 8, 1, 2, 3]) == 9
+    rows = draft.forward_rows([1, 2, 3, 1, 2])
+    assert rows.shape == (5, 10) and draft.cached_len == 5
+    assert np.argmax(rows[4]) == 3 and np.isneginf(np.delete(rows[4], 3)).all() and rows[4][3] == 0.0
+    assert np.array_equal(rows, draft.forward_full([1, 2, 3, 1, 2]))
+    draft.truncate(3)
+    assert np.argmax(draft.forward_rows([9])[0]) == 9
+
+    # a target that walks a fixed cycle: next = perm[last]; sharp table, so sampling follows the cycle
+    vocab, period = 12, 5
+    cycle = [3, 8, 1, 10, 6]
+    table = np.full((vocab, vocab), -40.0)
+    for a, b in zip(cycle, cycle[1:] + cycle[:1]):
+        table[a, b] = 0.0
+    for a in set(range(vocab)) - set(cycle):
+        table[a, cycle[0]] = 0.0
+    prompt = cycle + cycle[:2]  # one full period and a bit: every 2-gram has occurred
+    res = generate.speculative_generate(BigramTable(table), CopyFromContext(vocab, 2), prompt, 40, 4, 1.0, seed=2)
+    assert res.tests_passed == res.tests_evaluated and all(it.n_accepted == 4 for it in res.iterations)
+    assert res.tokens[:6] == [1, 10, 6, 3, 8, 1]
+
+    # one-hot q at x: accepted with probability p(x) (Section 2.3 with q(x) = 1), else drawn from p without x
+    target = TableModel(8, 0, seed=3)
+    p = target.prob([])
+    x = 5
+    q_row = np.full(8, -np.inf)
+    q_row[x] = 0.0
+    trials = 200_000
+    us = np.random.default_rng(1).random((trials, 2))
+    n, t = sampling.verify_trials(np.stack([target.table, target.table]), q_row[None], np.full((trials, 1), x), us, 1.0)
+    assert abs((n == 1).mean() - p[x]) < 4 * np.sqrt(p[x] * (1 - p[x]) / trials)
+    rest = p.copy()
+    rest[x] = 0.0
+    assert not np.any(t[n == 0] == x)
+    counts = np.bincount(t[n == 0], minlength=8)
+    assert stats.chisquare(np.delete(counts, x), np.delete(rest / rest.sum(), x) * counts.sum()).pvalue > 1e-3
+
+    tcfg = workloads.model_config("tiny_target")
+    model = Decoder(tcfg, workloads.make_weights(tcfg, 1))
+    rep = workloads.make_repetitive_prompt(5, 24, tcfg["vocab"], 6)
+    want, _, _ = generate.target_only_generate(model, rep, 12, 0.0, seed=0)
+    got = generate.speculative_generate(model, CopyFromContext(tcfg["vocab"], 2), rep, 12, 3, 0.0, seed=0)
+    assert got.tokens == want
