@@ -284,7 +284,7 @@ class GenerationWorkload:
         # key slices are not merged inside a cluster: long contexts); embed, final norm, head, its reduction
         long_context = self.prompt_len > 256
         fwd = lambda cfg, combine: 1 + (9 + combine) * cfg["n_layers"] + 3
-        draft = 1 if self.dcfg["arch"] == "bigram" else fwd(self.dcfg, 0)  # (few slices: merged in the cluster)
+        draft = 1 if self.dcfg["arch"] in ("bigram", "copy") else fwd(self.dcfg, 0)  # (few slices: merged in the cluster)
         target = fwd(self.tcfg, 1 if long_context else 0)
         return 1 + self.gamma * (1 + draft + 1) + 1 + target + 2 + 1
 
@@ -331,7 +331,8 @@ class GenerationWorkload:
             return eng.time_forward(which, self.batch, rows, repeats)
         eng.reset()
         chunk = max(1, 64 // self.batch)  # the teacher-forced entry point takes 64 rows per call
-        for which in (0, 1):
+        stateless = self.dcfg["arch"] in ("bigram", "copy")  # no cache to fill (a copy draft has no teacher-forced pass)
+        for which in ((0,) if stateless else (0, 1)):
             for c0 in range(0, tok.shape[1], chunk):
                 eng.forward_logits(which, tok[:, c0:c0 + chunk])
         return {"target_1row_ms": timed(0, 1), "target_rows_ms": timed(0, self.gamma + 1), "draft_1row_ms": timed(1, 1)}
@@ -387,12 +388,15 @@ class GenerationWorkload:
         from oracle.decoder import Decoder
         from paper_2211_17192_b200 import workloads
         small_t = workloads.scaled_config(self.tcfg, n_layers=min(2, self.tcfg["n_layers"]))
-        small_d = self.dcfg if self.dcfg["arch"] == "bigram" else workloads.scaled_config(self.dcfg, n_layers=min(2, self.dcfg["n_layers"]))
+        small_d = self.dcfg if self.dcfg["arch"] in ("bigram", "copy") else workloads.scaled_config(self.dcfg, n_layers=min(2, self.dcfg["n_layers"]))
         dtype = np.float32 if self.tcfg["d_model"] >= 2048 else np.float64
         if not hasattr(self, "_cpu_models"):  # built once, outside every timed sample
             if self.dcfg["arch"] == "bigram":
                 from oracle.ngram import BigramTable
                 draft_model = BigramTable(workloads.make_weights(self.dcfg, 2)["table"], dtype=np.float32)
+            elif self.dcfg["arch"] == "copy":
+                from oracle.ngram import CopyFromContext
+                draft_model = CopyFromContext(self.dcfg["vocab"], self.dcfg["ngram"])
             else:
                 draft_model = Decoder(small_d, workloads.make_weights(small_d, 2), dtype=dtype)
             self._cpu_models = (Decoder(small_t, workloads.make_weights(small_t, 1), dtype=dtype), draft_model)
@@ -523,6 +527,9 @@ def _make_workload(args):
     gamma = args.gamma or 2
     if args.draft == "bigram":  # a negligible-cost draft: one table row per step instead of a model pass
         return GenerationWorkload(f"llama7b_bigram_b{batch}_g{gamma}", "llama7b_target", "bigram_32k", batch,
+                                  args.prompt_len or 1024, 256, gamma, args.temperature, args.layers)
+    if args.draft == "copy":  # parameter-less: guesses copied from the context (Section 3.6)
+        return GenerationWorkload(f"llama7b_copy_b{batch}_g{gamma}", "llama7b_target", "copy_32k", batch,
                                   args.prompt_len or 1024, 256, gamma, args.temperature, args.layers)
     return GenerationWorkload(f"llama7b_160m_b{batch}_g{gamma}", "llama7b_target", "llama160m_draft", batch,
                               args.prompt_len or 1024, 256, gamma, args.temperature, args.layers)
@@ -747,7 +754,7 @@ def main():
     ap.add_argument("--gamma", type=int, default=None)
     ap.add_argument("--temperature", type=float, default=1.0)
     ap.add_argument("--prompt-len", type=int, default=None, help="override the workload's prompt length (profiling)")
-    ap.add_argument("--draft", default="model", choices=["model", "bigram"],
+    ap.add_argument("--draft", default="model", choices=["model", "bigram", "copy"],
                     help="llama7b workload: the 160M-shaped draft model, or a bigram table (negligible-cost draft)")
     ap.add_argument("--layers", type=int, default=None, help="override the target's depth, full width (profiling)")
     ap.add_argument("--adaptive-gamma-max", type=int, default=0,

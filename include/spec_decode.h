@@ -242,6 +242,21 @@ int spec_uniforms(uint64_t seed, const int32_t* positions, const int32_t* sequen
  *                    [vocab, vocab] (row = last token) in `dtype`; only `arch`,
  *                    `vocab` and `dtype` of the config are read, no other
  *                    weight pointer is used, and it keeps no K,V rows.
+ *   SPEC_ARCH_COPY:   a parameter-less negligible-cost approximation model
+ *                    (Section 3.6 suggests one that copies tokens from the
+ *                    context where a matching prefix is found; no procedure
+ *                    is given).  Ours: let s be the sequence so far and n =
+ *                    `ngram` >= 1.  The guess is the token that followed the
+ *                    most recent earlier occurrence of the last n tokens of s,
+ *                    i.e. s[j+1] for the largest j < len(s)-1 with
+ *                    s[j-n+1..j] == s[len-n..len-1]; if there is none (or s has
+ *                    fewer than n+1 tokens) the last token is repeated.  q is
+ *                    one-hot at the guess (logit 0 there, -inf elsewhere), so
+ *                    Algorithm 1 accepts it with probability p(guess) and
+ *                    otherwise draws from p with the guess removed.  Only
+ *                    valid as the DRAFT; only `arch`, `vocab` and `ngram` are
+ *                    read; no weights, no K,V rows; no teacher-forced pass
+ *                    (spec_forward_logits refuses it).
  *   FFN: SPEC_FFN_GELU (tanh approximation) with W_in [d_ff, d_model];
  *        SPEC_FFN_GATED_GELU / SPEC_FFN_SWIGLU with W_in [2*d_ff, d_model],
  *        rows 0..d_ff-1 the gate, rows d_ff..2*d_ff-1 the up projection.
@@ -249,7 +264,7 @@ int spec_uniforms(uint64_t seed, const int32_t* positions, const int32_t* sequen
  * bf16 as raw 16-bit patterns); gains are fp32.  The residual stream, softmax,
  * normalisation and logits are fp32 in every configuration.
  * ------------------------------------------------------------------------- */
-enum { SPEC_ARCH_GPT = 0, SPEC_ARCH_LLAMA = 1, SPEC_ARCH_T5 = 2, SPEC_ARCH_BIGRAM = 3 };
+enum { SPEC_ARCH_GPT = 0, SPEC_ARCH_LLAMA = 1, SPEC_ARCH_T5 = 2, SPEC_ARCH_BIGRAM = 3, SPEC_ARCH_COPY = 4 };
 enum { SPEC_FFN_GELU = 0, SPEC_FFN_GATED_GELU = 1, SPEC_FFN_SWIGLU = 2 };
 enum { SPEC_DTYPE_FP32 = 0, SPEC_DTYPE_BF16 = 1 };
 
@@ -271,6 +286,7 @@ typedef struct spec_model_cfg {
     int n_enc_layers;     /* T5: encoder blocks (0 otherwise) */
     int rel_buckets;      /* T5: rows of the bias tables (even, 2..256) */
     int rel_max_distance; /* T5: distance from which the last bucket is used */
+    int ngram;            /* SPEC_ARCH_COPY: length of the matched suffix (0 otherwise) */
 } spec_model_cfg;
 
 typedef struct spec_layer_weights {

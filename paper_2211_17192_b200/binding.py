@@ -304,7 +304,7 @@ class _ModelCfg(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("arch", "n_layers", "d_model", "n_heads", "n_kv_heads", "d_head", "d_ff",
                                             "ffn", "vocab", "max_positions", "tied_embeddings", "dtype")] + \
                [("rms_eps", ctypes.c_float), ("rope_base", ctypes.c_float)] + \
-               [(n, ctypes.c_int) for n in ("n_enc_layers", "rel_buckets", "rel_max_distance")]
+               [(n, ctypes.c_int) for n in ("n_enc_layers", "rel_buckets", "rel_max_distance", "ngram")]
 
 
 class _LayerWeights(ctypes.Structure):
@@ -330,7 +330,7 @@ class _Stats(ctypes.Structure):
                [("prefill_ms", ctypes.c_double), ("decode_ms", ctypes.c_double)]
 
 
-_ARCH = {"gpt": 0, "llama": 1, "t5": 2, "bigram": 3}
+_ARCH = {"gpt": 0, "llama": 1, "t5": 2, "bigram": 3, "copy": 4}
 _FFN = {"gelu": 0, "gated_gelu": 1, "swiglu": 2}
 _DTYPE = {"fp32": 0, "bf16": 1}
 _engine_declared = False
@@ -377,11 +377,13 @@ def _declare_engine(h):
 
 def _cfg_struct(cfg):
     if cfg["arch"] == "bigram":  # only arch, vocab and dtype are read
-        return _ModelCfg(_ARCH["bigram"], 0, 0, 0, 0, 0, 0, 0, cfg["vocab"], 0, 0, _DTYPE[cfg["dtype"]], 0.0, 0.0, 0, 0, 0)
+        return _ModelCfg(_ARCH["bigram"], 0, 0, 0, 0, 0, 0, 0, cfg["vocab"], 0, 0, _DTYPE[cfg["dtype"]], 0.0, 0.0, 0, 0, 0, 0)
+    if cfg["arch"] == "copy":  # only arch, vocab and ngram are read
+        return _ModelCfg(_ARCH["copy"], 0, 0, 0, 0, 0, 0, 0, cfg["vocab"], 0, 0, 0, 0.0, 0.0, 0, 0, 0, cfg["ngram"])
     return _ModelCfg(_ARCH[cfg["arch"]], cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["n_kv_heads"],
                      cfg["d_head"], cfg["d_ff"], _FFN[cfg["ffn"]], cfg["vocab"], cfg["max_positions"],
                      1 if cfg["tied"] else 0, _DTYPE[cfg["dtype"]], cfg["rms_eps"], cfg["rope_base"],
-                     cfg.get("n_enc_layers", 0), cfg.get("rel_buckets", 0), cfg.get("rel_max_distance", 0))
+                     cfg.get("n_enc_layers", 0), cfg.get("rel_buckets", 0), cfg.get("rel_max_distance", 0), 0)
 
 
 class Engine:
@@ -428,6 +430,8 @@ class Engine:
 
         if cfg["arch"] == "bigram":
             return _Weights(dev("table", True), None, None, None, None, None, None, None, None)
+        if cfg["arch"] == "copy":
+            return _Weights(None, None, None, None, None, None, None, None, None)
         t5 = cfg["arch"] == "t5"
 
         def block(p, cross):

@@ -46,6 +46,7 @@ struct spec_ctx {
     struct Params { unsigned long long seed; int n_new; float imposed_alpha; }* params = nullptr;
     float imposed_alpha = -1.0f;  // >= 0: timing instrument, see spec_set_imposed_acceptance
     float lenience = 1.0f;        // Appendix A.5; 1 = Algorithm 1 as printed
+    int iteration_gamma = 0;      // gamma of the iteration being enqueued (the copy draft indexes the guesses by it)
     int top_k = 0;                // Section 2.2: both models standardised over their k largest logits; 0 = all
     float top_p = 1.0f;           // and then over the nucleus of mass top_p; 1 = all
     float* sample_floors = nullptr;  // the draft rows' k-th largest logits, one per sequence
@@ -78,6 +79,11 @@ int check_cfg(const spec_model_cfg& c, const char* which) {
     if (c.arch == SPEC_ARCH_BIGRAM) {
         if (c.vocab < 1 || (c.dtype != SPEC_DTYPE_FP32 && c.dtype != SPEC_DTYPE_BF16))
             return fail(SPEC_ERR_BAD_CONFIG, "%s: a table model needs vocab >= 1 and a known dtype", which);
+        return SPEC_OK;
+    }
+    if (c.arch == SPEC_ARCH_COPY) {
+        if (c.vocab < 1 || c.ngram < 1 || c.ngram > 64)
+            return fail(SPEC_ERR_BAD_CONFIG, "%s: a copy model needs vocab >= 1 and 1 <= ngram <= 64", which);
         return SPEC_OK;
     }
     if (c.arch != SPEC_ARCH_GPT && c.arch != SPEC_ARCH_LLAMA && c.arch != SPEC_ARCH_T5)
@@ -211,6 +217,11 @@ int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_ro
     if (c.arch == SPEC_ARCH_BIGRAM)  // logits = table[last token]: one gather
         return n_logit_rows > 0 ? launch_table_logits(m.tok_emb, m.bf16(), c.vocab, rows.token, logit_src, logit_dst, n_logit_rows,
                                                        logits, ctx->stream)
+                                : SPEC_OK;
+    if (c.arch == SPEC_ARCH_COPY)  // one-hot at the token that followed the same suffix before: one search
+        return n_logit_rows > 0 ? launch_copy_logits(ctx->tokens, ctx->rt.max_len, ctx->length, ctx->draft_tokens,
+                                                      std::max(ctx->iteration_gamma, 1), rows, logit_src, logit_dst,
+                                                      n_logit_rows, c.ngram, c.vocab, logits, ctx->stream)
                                 : SPEC_OK;
     Pass pass{ctx, m, n_rows, m.bf16() && ctx->tensor_cores, ctx->stream};
     const int d = c.d_model;
@@ -385,6 +396,7 @@ __global__ void commit_kernel(const spec_ctx::Params* __restrict__ params, const
 // Enqueues one iteration of Algorithm 1 for the whole batch on ctx->stream.
 int enqueue_iteration(spec_ctx* ctx, int batch, int gamma, float temperature) {
     cudaStream_t st = ctx->stream;
+    ctx->iteration_gamma = gamma;
     const int vocab = ctx->model[0].cfg.vocab;
     const int threads = 128;
     const int blocks_b = (batch + threads - 1) / threads;
@@ -527,10 +539,12 @@ int pack_model(spec_ctx* ctx, Model& m) {
 int init_model(spec_ctx* ctx, int which, const spec_model_cfg& cfg, const spec_weights& w) {
     Model& m = ctx->model[which];
     m.cfg = cfg;
-    if (cfg.arch == SPEC_ARCH_BIGRAM) {  // a table: no blocks, no cache; the sizes below only keep the buffer arithmetic valid
-        if (which != 1) return fail(SPEC_ERR_BAD_CONFIG, "spec_init: a table model can only be the draft");
-        if (!w.tok_emb) return fail(SPEC_ERR_BAD_ARG, "spec_init: missing table pointer");
+    if (cfg.arch == SPEC_ARCH_BIGRAM || cfg.arch == SPEC_ARCH_COPY) {
+        // a table or a search: no blocks, no cache; the sizes below only keep the buffer arithmetic valid
+        if (which != 1) return fail(SPEC_ERR_BAD_CONFIG, "spec_init: a table or copy model can only be the draft");
+        if (cfg.arch == SPEC_ARCH_BIGRAM && !w.tok_emb) return fail(SPEC_ERR_BAD_ARG, "spec_init: missing table pointer");
         m.tok_emb = w.tok_emb;
+        m.cfg.dtype = cfg.arch == SPEC_ARCH_COPY ? SPEC_DTYPE_FP32 : cfg.dtype;
         m.cfg.n_layers = 0;
         m.cfg.d_model = m.cfg.d_ff = 8;
         m.cfg.n_heads = m.cfg.n_kv_heads = 1;
@@ -641,7 +655,8 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     if (draft_cfg) {
         SPEC_TRY(check_cfg(*draft_cfg, "draft"));
         if (draft_cfg->vocab != target_cfg->vocab) return fail(SPEC_ERR_BAD_CONFIG, "spec_init: vocabularies differ");
-        if (draft_cfg->arch != SPEC_ARCH_BIGRAM && (draft_cfg->arch == SPEC_ARCH_T5) != (target_cfg->arch == SPEC_ARCH_T5))
+        if (draft_cfg->arch != SPEC_ARCH_BIGRAM && draft_cfg->arch != SPEC_ARCH_COPY &&
+            (draft_cfg->arch == SPEC_ARCH_T5) != (target_cfg->arch == SPEC_ARCH_T5))
             return fail(SPEC_ERR_BAD_CONFIG, "spec_init: an encoder-decoder target needs an encoder-decoder draft and vice versa");
     }
     const bool t5 = target_cfg->arch == SPEC_ARCH_T5;
@@ -729,7 +744,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
         bool any_bf16 = false;
         for (int i = 0; i < (ctx->has_draft ? 2 : 1); ++i) {
             const Model& m = ctx->model[i];
-            if (!m.bf16() || m.cfg.arch == SPEC_ARCH_BIGRAM) continue;
+            if (!m.bf16() || m.cfg.arch == SPEC_ARCH_BIGRAM || m.cfg.arch == SPEC_ARCH_COPY) continue;
             any_bf16 = true;
             max_k = std::max<size_t>({max_k, static_cast<size_t>(m.cfg.d_model), static_cast<size_t>(m.q_dim()), static_cast<size_t>(m.cfg.d_ff)});
             const int shapes[7][2] = {{m.qkv_dim(), m.cfg.d_model}, {m.cfg.d_model, m.q_dim()}, {m.ffn_in_dim(), m.cfg.d_model},
@@ -1215,6 +1230,8 @@ extern "C" int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* toke
     if (!ctx || !tokens || !logits || which < 0 || which > 1 || batch < 1 || rows < 1)
         return fail(SPEC_ERR_BAD_ARG, "spec_forward_logits: bad argument");
     if (which == 1 && !ctx->has_draft) return fail(SPEC_ERR_BAD_CONFIG, "spec_forward_logits: no draft model");
+    if (ctx->model[which].cfg.arch == SPEC_ARCH_COPY)
+        return fail(SPEC_ERR_BAD_CONFIG, "spec_forward_logits: a copy model reads the generation's own tokens and has no teacher-forced pass");
     if (batch > ctx->rt.max_batch || batch * rows > ctx->max_logit_rows)
         return fail(SPEC_ERR_CAPACITY, "spec_forward_logits: %d x %d rows exceed the workspace (%d rows)", batch, rows, ctx->max_logit_rows);
     if (ctx->model[which].t5() && (!ctx->encoded || batch > ctx->encoded_batch))

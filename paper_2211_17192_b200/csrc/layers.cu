@@ -173,6 +173,43 @@ __global__ void table_logits_kernel(const void* __restrict__ table, bool bf16, i
         out[v] = load_elem(table, static_cast<size_t>(t) * vocab + v, bf16);
 }
 
+// Copy-from-context draft: logits row i is one-hot (0 at the guess, -inf elsewhere), the
+// guess being what followed the most recent earlier occurrence of the last `ngram`
+// tokens of the sequence up to the row's position, or the last token again if there is
+// none.  Positions below length[seq] read the committed tokens, later ones this
+// iteration's guesses.  grid = (chunks, rows): every CTA repeats the search (a few
+// thousand token compares) and writes its share of the row.
+__global__ void copy_logits_kernel(const int32_t* __restrict__ tokens, int max_len, const int32_t* __restrict__ length,
+                                   const int32_t* __restrict__ draft_tokens, int gamma, const int32_t* __restrict__ row_pos,
+                                   const int32_t* __restrict__ row_seq, const int32_t* __restrict__ src_rows,
+                                   const int32_t* __restrict__ dst_rows, int ngram, int vocab, float* __restrict__ logits) {
+    __shared__ int best[32];
+    pdl_trigger();
+    pdl_wait();
+    const int i = blockIdx.y;
+    const int r = src_rows ? src_rows[i] : i;
+    const int b = row_seq[r], last = row_pos[r];
+    const int committed = length[b];
+    const int32_t* seq = tokens + static_cast<size_t>(b) * max_len;
+    const int32_t* guesses = draft_tokens + static_cast<size_t>(b) * gamma;
+    auto at = [&](int p) { return p < committed ? seq[p] : guesses[min(p - committed, gamma - 1)]; };
+    // j = end of an earlier occurrence of the suffix: ngram-1 <= j <= last-1
+    int found = -1;
+    for (int j = last - 1 - static_cast<int>(threadIdx.x); j >= ngram - 1; j -= blockDim.x) {
+        bool same = true;
+        for (int k = 0; k < ngram && same; ++k) same = at(j - k) == at(last - k);
+        if (same) { found = j; break; }  // this thread's later candidates are all older
+    }
+    found = __reduce_max_sync(0xffffffffu, found);
+    if ((threadIdx.x & 31) == 0) best[threadIdx.x >> 5] = found;
+    __syncthreads();
+    for (int w = 0; w < static_cast<int>(blockDim.x) / 32; ++w) found = max(found, best[w]);
+    const int guess = min(max(at(found >= 0 ? found + 1 : last), 0), vocab - 1);
+    float* out = logits + static_cast<size_t>(dst_rows ? dst_rows[i] : i) * vocab;
+    for (int v = blockIdx.x * blockDim.x + threadIdx.x; v < vocab; v += gridDim.x * blockDim.x)
+        out[v] = v == guess ? 0.0f : -INFINITY;
+}
+
 __device__ __forceinline__ float gelu_tanh(float x) {
     const float k = 0.7978845608028654f;  // sqrt(2 / pi)
     return 0.5f * x * (1.0f + tanhf(k * (x + 0.044715f * x * x * x)));
@@ -220,6 +257,14 @@ int launch_table_logits(const void* table, bool bf16, int vocab, const int32_t* 
     const int chunks = std::max(1, std::min((vocab + 255) / 256, 32));
     return launch_pdl(table_logits_kernel, dim3(chunks, n_rows), dim3(256), 0, stream, table, bf16, vocab, token, src_rows,
                       dst_rows, logits);
+}
+
+int launch_copy_logits(const int32_t* tokens, int max_len, const int32_t* length, const int32_t* draft_tokens, int gamma,
+                       const RowMeta& rows, const int32_t* src_rows, const int32_t* dst_rows, int n_rows, int ngram,
+                       int vocab, float* logits, cudaStream_t stream) {
+    const int chunks = std::max(1, std::min((vocab + 255) / 256, 16));
+    return launch_pdl(copy_logits_kernel, dim3(chunks, n_rows), dim3(256), 0, stream, tokens, max_len, length, draft_tokens,
+                      gamma, rows.pos, rows.seq, src_rows, dst_rows, ngram, vocab, logits);
 }
 
 int launch_norm(float* h, const float* partial, int splits, int rows_total, const float* gain, const int32_t* src_rows,

@@ -67,6 +67,10 @@ int launch_table_logits(const void* table, bool bf16, int vocab, const int32_t* 
 // Row i of the output = RMSNorm(h[src(i)]) * gain, as fp32 (`out`) and/or as two
 // bf16 terms (`out_hi`, `out_lo`).  If `partial` is given (split-K results of
 // the GEMM before, [splits][rows_total][d]) it is first added into h.
+// Copy-from-context draft: one-hot logits at the token that followed the last `ngram` tokens before.
+int launch_copy_logits(const int32_t* tokens, int max_len, const int32_t* length, const int32_t* draft_tokens, int gamma,
+                       const RowMeta& rows, const int32_t* src_rows, const int32_t* dst_rows, int n_rows, int ngram,
+                       int vocab, float* logits, cudaStream_t stream);
 int launch_norm(float* h, const float* partial, int splits, int rows_total, const float* gain, const int32_t* src_rows,
                 int n_rows, int d, float eps, float* out, __nv_bfloat16* out_hi, __nv_bfloat16* out_lo,
                 cudaStream_t stream);

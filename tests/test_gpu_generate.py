@@ -253,6 +253,48 @@ def test_bigram_table_draft_matches_the_oracle(temperature):
         eng.close()
 
 
+@pytest.mark.parametrize("ngram", [2, 1, 3])
+def test_copy_from_context_draft_matches_the_oracle(ngram):
+    """The tiny fp32 target with the parameter-less copy draft.  With a random-init target a
+    guess is almost never accepted, so the guesses themselves would go unseen: argmax decoding
+    with a vanishing lenience factor accepts every guess (Appendix A.5 at T = 0), and the
+    emitted stream is then the draft's guesses interleaved with the target's tokens."""
+    from oracle.ngram import CopyFromContext
+    tcfg = workloads.model_config("tiny_target")
+    tw = workloads.make_weights(tcfg, 1)
+    dcfg = workloads.scaled_config(workloads.model_config("copy_8k"), ngram=ngram)
+    eng = binding.Engine(tcfg, tw, dcfg, {}, max_batch=2, max_len=160, page_size=32, max_gamma=4)
+    target, draft = Decoder(tcfg, tw), CopyFromContext(tcfg["vocab"], ngram)
+    try:
+        prompt = workloads.make_repetitive_prompt(15, 26, tcfg["vocab"], 7)
+        eng.set_lenience(1e-30)
+        ref = oracle_generate.speculative_generate(target, draft, prompt, 60, 3, 0.0, seed=0, lenience=1e-30)
+        assert ref.tests_passed == ref.tests_evaluated  # every guess shows in the stream
+        got, st = eng.generate([prompt], 60, 3, 0.0, 0)
+        assert st["tests_passed"] == st["tests_evaluated"]
+        got = got[0].tolist()
+        diff = next((k for k in range(60) if got[k] != ref.tokens[k]), None)
+        if diff is not None:  # only a near-tie of the target's two best logits may end the comparison
+            index = len(prompt) + diff
+            it = next(i for i in ref.iterations if i.start_len <= index <= i.start_len + i.n_accepted)
+            assert index == it.start_len + it.n_accepted and it.top2_gap <= 2e-3 and diff >= 12
+        # the first iteration copies the next three tokens of the period
+        assert got[:3] == [int(t) for t in np.tile(prompt[:7], 8)[26:29]]
+        eng.set_lenience(1.0)
+        # T = 1 decisions as the oracle's, T = 0 strict equals target-only greedy, in a ragged batch
+        flagged, _ = compare_generation(eng, target, draft, prompt, 40, 3, 1.0, seed=19, margin=1e-3, logit_tol=1e-3)
+        assert flagged <= 2
+        prompts = [prompt, workloads.make_repetitive_prompt(16, 9, tcfg["vocab"], 3)]
+        greedy, _ = eng.generate(prompts, 24, 0, 0.0, 0)
+        spec, stats = eng.generate(prompts, 24, 4, 0.0, 0)
+        assert np.array_equal(greedy, spec) and stats["draft_passes"] > 0
+        with pytest.raises(binding.SpecError):
+            eng.forward_logits(1, np.zeros((1, 1), dtype=np.int32))
+    finally:
+        eng.set_lenience(1.0)
+        eng.close()
+
+
 def test_adaptive_gamma_generation(tiny):
     """Section 3.5's varying gamma: the library picks gamma burst by burst.  The trace it reports,
     replayed by the oracle (and by the phased entry points), gives the same tokens; at T = 0 the
