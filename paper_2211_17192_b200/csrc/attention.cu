@@ -460,10 +460,11 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 #pragma unroll
         for (int i = 0; i < 4; ++i) o[n][i] = 0.0f;
 
-    // This warp's tiles: the 16-key halves of the 32-key blocks t0 + warp, t0 + warp + 4, ...
-    const int my_blocks = t0 + warp < t1 ? (t1 - t0 - warp + kMmaWarps - 1) / kMmaWarps : 0;
-    const int my_tiles = 2 * my_blocks;
-    auto first_key = [&](int i) { return 32 * (t0 + warp + (i >> 1) * kMmaWarps) + 16 * (i & 1); };  // (kMmaWarps blocks apart)
+    // This warp's tiles: the slice's 16-key tiles warp, warp + kMmaWarps, ... (a short slice
+    // then still gives every warp a tile, and the chain a warp runs through stays short)
+    const int tile0 = 2 * t0, tile1 = min(2 * t1, (seq_keys + kTileKeys - 1) / kTileKeys);
+    const int my_tiles = tile0 + warp < tile1 ? (tile1 - tile0 - warp + kMmaWarps - 1) / kMmaWarps : 0;
+    auto first_key = [&](int i) { return kTileKeys * (tile0 + warp + i * kMmaWarps); };
     auto issue = [&](int i) {  // tile i into stage i & 1 (an empty group if there is no such tile)
         if (i < my_tiles) {
             const int k0 = first_key(i);
@@ -708,11 +709,11 @@ int attention_slices(const Model& m, int batch, int m_rows, int max_len) {
     const int queries = (m.cfg.n_heads / n_kv_heads) * m_rows;
     const int tiles = (max_len + 31) / 32;
     if (attention_uses_mma(m, batch, m_rows, max_len)) {
-        // one wave of CTAs (shared memory allows one per SM at d_head 128, two at 64); a tile per warp at least
+        // one wave of CTAs (shared memory allows one per SM at d_head 128, two at 64); a 16-key tile per warp at least
         const int m_blocks = (queries + 15) / 16;
         const int resident = 148 * (m.cfg.d_head == 64 ? 2 : 1);
         const int want = std::max(1, resident / (batch * n_kv_heads * m_blocks));
-        const int most = std::max(1, (tiles + kMmaWarps - 1) / kMmaWarps);
+        const int most = std::max(1, (2 * tiles + kMmaWarps - 1) / kMmaWarps);  // (tiles: 32 keys; a warp's unit is 16)
         return std::max(1, std::min(std::min(want, most), cap));
     }
     const int ks = attention_sub_slices(queries);
