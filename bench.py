@@ -101,10 +101,12 @@ class SamplerWorkload:
     batch, gamma, vocab, temperature = 64, 7, 32000, 1.0
     noises = (0.5, 1.0, 2.0)
     dtype = "f32"
+    top_k, top_p = 0, 1.0  # Section 2.2's truncations, off in the headline workload (--top-k / --top-p)
 
     def description(self):
+        cut = {"top_k": self.top_k, "top_p": self.top_p} if (self.top_k or self.top_p != 1.0) else {}
         return {"workload": self.name, "batch": self.batch, "gamma": self.gamma, "vocab": self.vocab,
-                "temperature": self.temperature, "draft_noise": list(self.noises),
+                "temperature": self.temperature, "draft_noise": list(self.noises), **cut,
                 "l2": "inputs rotate over 3 logit sets (369 MB) > 126 MB L2",
                 "parallelism": "replicas"}
 
@@ -134,7 +136,8 @@ class SamplerWorkload:
         for tl, ql, us, draw in self.host:
             tl_d, ql_d = torch.from_numpy(tl).to(device), torch.from_numpy(ql).to(device)
             # x_i ~ q_i drawn by the library's own sampler (Algorithm 1's draft draws)
-            xs = binding.spec_sample(ql_d.view(-1, self.vocab), torch.from_numpy(draw).to(device), self.temperature)
+            xs = binding.spec_sample(ql_d.view(-1, self.vocab), torch.from_numpy(draw).to(device), self.temperature,
+                                     top_k=self.top_k, top_p=self.top_p)
             self.dev_sets.append((tl_d, ql_d, xs.view(self.batch, self.gamma).contiguous(),
                                   torch.from_numpy(us).to(device)))
         self.n = torch.empty(self.batch, dtype=torch.int32, device=device)
@@ -153,8 +156,10 @@ class SamplerWorkload:
 
     def step(self, i):
         tl, ql, xs, us = self.dev_sets[i % len(self.dev_sets)]
-        self.binding.spec_verify_sample(tl, ql, xs, us, self.temperature, self.n, self.t, self.ws)
-        return 2  # kernels of this library launched: statistics pass + finishing pass
+        self.binding.spec_verify_sample(tl, ql, xs, us, self.temperature, self.n, self.t, self.ws,
+                                        top_k=self.top_k, top_p=self.top_p)
+        # kernels of this library launched: statistics pass + finishing pass (+ one selection pass per active cut)
+        return 2 + (0 < self.top_k < self.vocab) + (0.0 < self.top_p < 1.0)
 
     def tokens_emitted(self, first_step, steps):
         """Tokens the timed steps emitted (n accepted + 1 per sequence).  Each
@@ -172,7 +177,8 @@ class SamplerWorkload:
         for d, s in zip(self.stage, src):
             d.copy_(s, non_blocking=True)
         tl, ql, xs, us = self.stage
-        self.binding.spec_verify_sample(tl, ql, xs, us, self.temperature, self.n, self.t, self.ws)
+        self.binding.spec_verify_sample(tl, ql, xs, us, self.temperature, self.n, self.t, self.ws,
+                                        top_k=self.top_k, top_p=self.top_p)
         self.n_host.copy_(self.n, non_blocking=True)
         self.t_host.copy_(self.t, non_blocking=True)
         self.torch.cuda.current_stream().synchronize()
@@ -192,8 +198,9 @@ class SamplerWorkload:
         while time.perf_counter() - t0 < budget_s or done < 2:
             b = done % self.batch
             for i in range(self.gamma):
-                xs[b, i] = oracle_sampling.sample_token(ql[b, i], draw[b * self.gamma + i], self.temperature)[0]
-            res = oracle_sampling.verify_step(tl[b], ql[b], xs[b], us[b], self.temperature)
+                xs[b, i] = oracle_sampling.sample_token(ql[b, i], draw[b * self.gamma + i], self.temperature,
+                                                        self.top_k, self.top_p)[0]
+            res = oracle_sampling.verify_step(tl[b], ql[b], xs[b], us[b], self.temperature, 1.0, self.top_k, self.top_p)
             tokens += res.n_accepted + 1
             done += 1
         dt = time.perf_counter() - t0
@@ -515,7 +522,11 @@ def make_workload(args):
 
 def _make_workload(args):
     if args.workload == "sampler":
-        return SamplerWorkload()
+        wl = SamplerWorkload()
+        wl.top_k, wl.top_p = args.top_k, args.top_p
+        if wl.top_k or wl.top_p != 1.0:
+            wl.name += f"_k{wl.top_k}_p{wl.top_p:g}"
+        return wl
     batch = args.batch or 1
     if args.workload == "t5xxl":
         gamma = args.gamma or 5
@@ -757,6 +768,8 @@ def main():
     ap.add_argument("--draft", default="model", choices=["model", "bigram", "copy"],
                     help="llama7b workload: the 160M-shaped draft model, or a bigram table (negligible-cost draft)")
     ap.add_argument("--layers", type=int, default=None, help="override the target's depth, full width (profiling)")
+    ap.add_argument("--top-k", type=int, default=0, help="sampler workload: top-k standardisation of both models")
+    ap.add_argument("--top-p", type=float, default=1.0, help="sampler workload: nucleus standardisation of both models")
     ap.add_argument("--adaptive-gamma-max", type=int, default=0,
                     help="also report decoding with gamma chosen by the library burst by burst, up to this value")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
