@@ -668,332 +668,236 @@ sample_kernel(const float* __restrict__ logits, size_t logit_stride, const float
     if (tid == 0) tokens[blockIdx.x * token_stride] = max(0, min(token, vocab - 1));
 }
 
-// ---- top-k: the k-th largest logit of every row --------------------------------
-constexpr int kFloorThreads = 512;
+// ---- top-k and nucleus: the lowest logit that each row keeps ---------------------
+// One CTA per row, several CTAs per SM.  Both cuts are a selection: the largest
+// value t such that the logits at or above t number at least k (top-k), or carry
+// at least top_p of the mass (nucleus).  The row is never sorted or held:
+//   1. one pass finds the range [lo, hi] of the logits still in play;
+//   2. one pass drops them into kSelBins equal-width bins counted from the top
+//      (a count per bin, for the nucleus also the mass), a scan finds the bin in
+//      which the target is crossed;
+//   3. if that bin holds few logits they are copied out and ranked against each
+//      other exactly; otherwise the bin's own range becomes [lo, hi] and step 2
+//      repeats (heavy ties end when lo == hi).
+// The bin of a logit is a monotone function of it, so the bins partition the row
+// by value and the result is exact (comparisons of the logits themselves decide;
+// -inf, +inf and NaN logits are never in play).  Mass is summed in 2^-40 fixed
+// point with integer atomics, so every order of summation gives the same totals:
+// a row always gives the same floor, however the threads interleave.
+constexpr int kSelThreads = 256;
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kSelBins = 2048;
+constexpr int kSelPerThread = kSelBins / kSelThreads;
+constexpr int kSelCap = 1024;   // logits ranked against each other at the end
+constexpr int kSelLevels = 40;  // every level shrinks the range; fp32 allows far fewer than this
 
-// Unsigned keys that order like the floats they come from.
-__device__ __forceinline__ uint32_t float_key(float v) {
-    const uint32_t u = __float_as_uint(v);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-__device__ __forceinline__ float key_float(uint32_t k) {
-    return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
-}
+struct SelShared {
+    unsigned cnt[kSelBins];
+    unsigned long long mass[kSelBins];
+    float cand[kSelCap];
+    unsigned long long cand_mass[kSelCap];
+    unsigned long long warp_mass[kSelWarps];
+    unsigned warp_cnt[kSelWarps];
+    float warp_lo[kSelWarps], warp_hi[kSelWarps];
+    unsigned n_cand;
+    // where the scan found the target crossed
+    int bin;
+    unsigned before_cnt;
+    unsigned long long before_mass;
+};
 
-// One CTA per row.  The k-th largest key is the largest value t with
-// count(key >= t) >= k; its 32 bits are fixed from the top, one block-wide count
-// per bit.  Keys whose upper bits differ from the bits fixed so far are settled
-// (above: counted once and for all; below: out), so as soon as at most kLiveCap
-// keys remain undecided they are copied to shared memory and the remaining
-// bits look at those alone.  KPT > 0: the row (at most kFloorThreads * KPT
-// logits) is read once and its keys stay in registers; KPT = 0: any length,
-// re-read per bit until the copy (the row stays in L2).  Rows come from two
-// arrays: sequence s owns a_rows consecutive rows of `a`, then b_rows of `b`;
-// floors has the same order.
-constexpr int kLiveCap = 2048;
-
-template <bool VEC, int KPT>
-__global__ void __launch_bounds__(kFloorThreads, 1)
-topk_floor_kernel(const float* __restrict__ a, size_t a_stride, int a_rows, const float* __restrict__ b,
-                  size_t b_stride, int b_rows, int vocab, int top_k, float* __restrict__ floors) {
-    __shared__ unsigned counts[32];
-    __shared__ unsigned n_live;
-    __shared__ uint32_t live[kLiveCap];
-    pdl_trigger();
-    pdl_wait();
-    const int tid = threadIdx.x, lane = tid & 31;
-    const int per_seq = a_rows + b_rows;
-    const int seq = blockIdx.x / per_seq, row = blockIdx.x % per_seq;
-    const float* src = row < a_rows ? a + (static_cast<size_t>(seq) * a_rows + row) * a_stride
-                                    : b + (static_cast<size_t>(seq) * b_rows + (row - a_rows)) * b_stride;
-    const Row<VEC> r = make_row<VEC>(src, vocab);
-    const int groups = (vocab + 3) >> 2;
-    if (tid < 32) counts[tid] = 0;
-    if (tid == 0) n_live = 0;
-
-    constexpr int G = KPT > 0 ? KPT / 4 : 1;
-    uint32_t keys[4 * G];
-    if (KPT > 0) {
+// f(v) for every logit of the row, four 128-bit loads in flight per thread.
+template <bool VEC, class F>
+__device__ __forceinline__ void for_each_logit(const Row<VEC>& r, int groups, F f) {
+    for (int g0 = threadIdx.x; g0 < groups; g0 += 4 * kSelThreads) {
+        float4 v[4];
 #pragma unroll
-        for (int i = 0; i < G; ++i) {
-            const int g = tid + i * kFloorThreads;
-            // past the end of the row: -inf, below every threshold that k <= vocab can give
-            const float4 v = g < groups ? r.raw(g, -INFINITY) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-            keys[4 * i + 0] = float_key(v.x);
-            keys[4 * i + 1] = float_key(v.y);
-            keys[4 * i + 2] = float_key(v.z);
-            keys[4 * i + 3] = float_key(v.w);
+        for (int i = 0; i < 4; ++i) {
+            const int g = g0 + i * kSelThreads;
+            v[i] = g < groups ? r.raw(g, -INFINITY) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f(v[i].x);
+            f(v[i].y);
+            f(v[i].z);
+            f(v[i].w);
         }
     }
-    __syncthreads();
-
-    const unsigned k = static_cast<unsigned>(top_k);
-    uint32_t prefix = 0;
-    // count(key >= prefix) and count(key >= prefix + 2^(bit+1)): the keys between the two are undecided
-    unsigned at_prefix = KPT > 0 ? 4u * G * kFloorThreads : 4u * groups;
-    unsigned above = 0;
-    int bit = 31;
-    for (; bit >= 0 && at_prefix - above > kLiveCap; --bit) {
-        const uint32_t cand = prefix | (1u << bit);
-        unsigned c = 0;
-        if (KPT > 0) {
-#pragma unroll
-            for (int i = 0; i < 4 * G; ++i) c += keys[i] >= cand;
-        } else {
-            for (int g = tid; g < groups; g += kFloorThreads) {
-                const float4 v = r.raw(g, -INFINITY);
-                c += (float_key(v.x) >= cand) + (float_key(v.y) >= cand) + (float_key(v.z) >= cand) +
-                     (float_key(v.w) >= cand);
-            }
-        }
-        c = __reduce_add_sync(0xffffffffu, c);
-        if (lane == 0 && c) atomicAdd(&counts[bit], c);
-        __syncthreads();
-        const unsigned total = counts[bit];
-        if (total >= k) { prefix = cand; at_prefix = total; } else { above = total; }
-    }
-    if (bit >= 0) {
-        // undecided: the keys that agree with `prefix` on every bit above `bit`
-        const int shift = bit + 1;
-        auto undecided = [&](uint32_t key) { return shift >= 32 || ((key ^ prefix) >> shift) == 0; };
-        // each thread counts its own, one scan per warp and one atomic per warp place them
-        unsigned mine = 0;
-        if (KPT > 0) {
-#pragma unroll
-            for (int i = 0; i < 4 * G; ++i) mine += undecided(keys[i]);
-        } else {
-            for (int g = tid; g < groups; g += kFloorThreads) {
-                const float4 v = r.raw(g, -INFINITY);
-                mine += undecided(float_key(v.x)) + undecided(float_key(v.y)) + undecided(float_key(v.z)) +
-                        undecided(float_key(v.w));
-            }
-        }
-        unsigned incl = mine;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const unsigned up = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += up;
-        }
-        unsigned base = 0;
-        if (lane == 31 && incl) base = atomicAdd(&n_live, incl);
-        unsigned pos = __shfl_sync(0xffffffffu, base, 31) + incl - mine;
-        auto keep = [&](uint32_t key) {
-            if (undecided(key)) {
-                if (pos < kLiveCap) live[pos] = key;
-                ++pos;
-            }
-        };
-        if (KPT > 0) {
-#pragma unroll
-            for (int i = 0; i < 4 * G; ++i) keep(keys[i]);
-        } else {
-            for (int g = tid; g < groups; g += kFloorThreads) {
-                const float4 v = r.raw(g, -INFINITY);
-                keep(float_key(v.x));
-                keep(float_key(v.y));
-                keep(float_key(v.z));
-                keep(float_key(v.w));
-            }
-        }
-        __syncthreads();
-        const int n = static_cast<int>(min(n_live, static_cast<unsigned>(kLiveCap)));  // = at_prefix - above
-        for (; bit >= 0; --bit) {
-            const uint32_t cand = prefix | (1u << bit);
-            unsigned c = 0;
-            for (int j = tid; j < n; j += kFloorThreads) c += live[j] >= cand;
-            c = __reduce_add_sync(0xffffffffu, c);
-            if (lane == 0 && c) atomicAdd(&counts[bit], c);
-            __syncthreads();
-            if (counts[bit] + above >= k) prefix = cand;
-        }
-    }
-    if (tid == 0) floors[blockIdx.x] = key_float(prefix);
 }
 
-// ---- nucleus (top-p): the lowest logit inside the smallest most-probable set of mass top_p ----
-constexpr int kFloorWarps = kFloorThreads / 32;
-constexpr int kCutSlots = 72;  // block-wide measurements per row: 1 + at most 32 + 32
+__device__ __forceinline__ float warp_min(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
 
-// One CTA per row, after topk_floor_kernel when top-k is set too (use_k: floors
-// then holds the row's k-th largest logit on entry, and the nucleus is taken
-// of the logits at or above it).  With weights w = exp((l - max) / T), the
-// answer is the largest t with mass(key >= t) >= top_p * total mass: the same
-// bit-by-bit search as topk_floor_kernel with a sum of weights for the count.
-// KPT > 0: keys in registers and weights in shared memory ([slot][thread], so
-// a pass reads them without bank conflicts); KPT = 0: both recomputed from the
-// row per pass.  Sums are taken in a fixed order (thread, shuffle tree, warps
-// in index order), so every thread sees the same totals and a row always
-// gives the same floor.
-template <bool VEC, int KPT>
-__global__ void __launch_bounds__(kFloorThreads, 1)
-nucleus_floor_kernel(const float* __restrict__ a, size_t a_stride, int a_rows, const float* __restrict__ b,
-                     size_t b_stride, int b_rows, int vocab, bool use_k, float top_p, float c2,
-                     float* __restrict__ floors) {
-    extern __shared__ float wsm[];
-    __shared__ unsigned counts[kCutSlots];
-    __shared__ float partial[kCutSlots][kFloorWarps];
-    __shared__ uint32_t warp_top[kFloorWarps];
-    __shared__ uint32_t live_key[kLiveCap];
-    __shared__ float live_w[kLiveCap];
-    pdl_trigger();
-    pdl_wait();
+// The floor among the finite logits >= kf: MASS = false, the k-th largest of
+// them; MASS = true, the nucleus of mass top_p with weights exp2((l - max) * c2).
+// Every thread returns the same value; -inf means "keep everything".
+template <bool VEC, bool MASS>
+__device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned k, float top_p, float c2, SelShared& sh) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // 1. range and number of the logits in play
+    float lo = INFINITY, hi = -INFINITY;
+    unsigned n = 0;
+    for_each_logit(r, groups, [&](float v) {
+        const bool in_play = fabsf(v) < INFINITY && v >= kf;
+        lo = fminf(lo, in_play ? v : INFINITY);
+        hi = fmaxf(hi, in_play ? v : -INFINITY);
+        n += in_play;
+    });
+    lo = warp_min(lo);
+    hi = warp_max(hi);
+    n = __reduce_add_sync(0xffffffffu, n);
+    __syncthreads();  // (the shared arrays may still be read by a previous call)
+    if (lane == 0) { sh.warp_lo[warp] = lo; sh.warp_hi[warp] = hi; sh.warp_cnt[warp] = n; }
+    __syncthreads();
+    lo = INFINITY; hi = -INFINITY; n = 0;
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) { lo = fminf(lo, sh.warp_lo[w]); hi = fmaxf(hi, sh.warp_hi[w]); n += sh.warp_cnt[w]; }
+    if (n == 0 || (!MASS && k > n)) return kf;  // nothing to cut
+    const float row_max = hi;
+    auto fixed_mass = [&](float v) { return __float2ull_rz(fast_exp2((v - row_max) * c2) * 1099511627776.0f); };  // 2^40
+
+    unsigned before_cnt = 0;
+    unsigned long long before_mass = 0, goal = 0;
+    for (int level = 0; level < kSelLevels; ++level) {
+        if (lo == hi) return hi;  // everything left is one value: it stays whole
+        const float top = hi, bottom = lo;
+        const float scale = fminf(static_cast<float>(kSelBins) / (top - bottom), FLT_MAX);
+        // bin of a logit in [bottom, top], counted from the top; anything else gets no bin
+        auto bin_of = [&](float v) {
+            const int b = min(kSelBins - 1, static_cast<int>((top - v) * scale));
+            return (v >= bottom && v <= top) ? b : -1;
+        };
+        // 2. counts (and masses) per bin
+        for (int i = tid; i < kSelBins; i += kSelThreads) { sh.cnt[i] = 0; if (MASS) sh.mass[i] = 0; }
+        if (tid == 0) { sh.n_cand = 0; sh.bin = kSelBins - 1; sh.before_cnt = before_cnt; sh.before_mass = before_mass; }
+        __syncthreads();
+        for_each_logit(r, groups, [&](float v) {
+            const int b = bin_of(v);
+            if (b >= 0) {
+                atomicAdd(&sh.cnt[b], 1u);
+                if (MASS) atomicAdd(&sh.mass[b], fixed_mass(v));
+            }
+        });
+        __syncthreads();
+        // scan over the bins from the top: thread t owns bins t*P .. t*P+P-1
+        unsigned my_cnt = 0;
+        unsigned long long my_mass = 0;
+#pragma unroll
+        for (int i = 0; i < kSelPerThread; ++i) {
+            my_cnt += sh.cnt[tid * kSelPerThread + i];
+            if (MASS) my_mass += sh.mass[tid * kSelPerThread + i];
+        }
+        unsigned inc_cnt = my_cnt;
+        unsigned long long inc_mass = my_mass;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned c = __shfl_up_sync(0xffffffffu, inc_cnt, d);
+            const unsigned long long m = __shfl_up_sync(0xffffffffu, inc_mass, d);
+            if (lane >= d) { inc_cnt += c; inc_mass += m; }
+        }
+        if (lane == 31) { sh.warp_cnt[warp] = inc_cnt; sh.warp_mass[warp] = inc_mass; }
+        __syncthreads();
+        unsigned ex_cnt = before_cnt + inc_cnt - my_cnt;
+        unsigned long long ex_mass = before_mass + inc_mass - my_mass, all_mass = 0;
+#pragma unroll
+        for (int w = 0; w < kSelWarps; ++w) {
+            if (w < warp) { ex_cnt += sh.warp_cnt[w]; ex_mass += sh.warp_mass[w]; }
+            all_mass += sh.warp_mass[w];
+        }
+        if (MASS && level == 0)  // the first level sees every logit in play: top_p of their mass is the target
+            goal = static_cast<unsigned long long>(ceil(static_cast<double>(top_p) * static_cast<double>(all_mass)));
+        // the one thread whose bins contain the crossing records it
+        if (MASS ? ex_mass < goal : ex_cnt < k) {
+            unsigned run_cnt = ex_cnt;
+            unsigned long long run_mass = ex_mass;
+#pragma unroll
+            for (int i = 0; i < kSelPerThread; ++i) {
+                const int b = tid * kSelPerThread + i;
+                const unsigned c = sh.cnt[b];
+                const unsigned long long m = MASS ? sh.mass[b] : 0ull;
+                const bool was_below = MASS ? run_mass < goal : run_cnt < k;
+                const bool reaches = MASS ? run_mass + m >= goal : run_cnt + c >= k;
+                if (was_below && reaches) { sh.bin = b; sh.before_cnt = run_cnt; sh.before_mass = run_mass; }
+                run_cnt += c;
+                run_mass += m;
+            }
+        }
+        __syncthreads();
+        const int bin = sh.bin;
+        before_cnt = sh.before_cnt;
+        before_mass = sh.before_mass;
+        const unsigned in_bin = sh.cnt[bin];
+        if (in_bin <= kSelCap) {
+            // 3. copy the bin's logits out and rank them against each other
+            for_each_logit(r, groups, [&](float v) {
+                if (bin_of(v) == bin) {
+                    const unsigned at = atomicAdd(&sh.n_cand, 1u);
+                    if (at < kSelCap) { sh.cand[at] = v; if (MASS) sh.cand_mass[at] = fixed_mass(v); }
+                }
+            });
+            __syncthreads();
+            const int count = static_cast<int>(min(sh.n_cand, static_cast<unsigned>(kSelCap)));
+            float best = -INFINITY;
+            for (int i = tid; i < count; i += kSelThreads) {
+                const float mine = sh.cand[i];
+                unsigned c = 0;
+                unsigned long long m = 0;
+                for (int j = 0; j < count; ++j)
+                    if (sh.cand[j] >= mine) { ++c; if (MASS) m += sh.cand_mass[j]; }
+                const bool enough = MASS ? before_mass + m >= goal : before_cnt + c >= k;
+                if (enough) best = fmaxf(best, mine);
+            }
+            best = warp_max(best);
+            if (lane == 0) sh.warp_hi[warp] = best;
+            __syncthreads();
+            best = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kSelWarps; ++w) best = fmaxf(best, sh.warp_hi[w]);
+            return best > -INFINITY ? best : bottom;
+        }
+        // the bin is crowded: its own range is searched next
+        float new_lo = INFINITY, new_hi = -INFINITY;
+        for_each_logit(r, groups, [&](float v) {
+            const bool here = bin_of(v) == bin;
+            new_lo = fminf(new_lo, here ? v : INFINITY);
+            new_hi = fmaxf(new_hi, here ? v : -INFINITY);
+        });
+        new_lo = warp_min(new_lo);
+        new_hi = warp_max(new_hi);
+        if (lane == 0) { sh.warp_lo[warp] = new_lo; sh.warp_hi[warp] = new_hi; }
+        __syncthreads();
+        lo = INFINITY; hi = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kSelWarps; ++w) { lo = fminf(lo, sh.warp_lo[w]); hi = fmaxf(hi, sh.warp_hi[w]); }
+        __syncthreads();
+    }
+    return lo;
+}
+
+// floors[s * (a_rows + b_rows) + r] for sequence s's a_rows rows of `a`, then its
+// b_rows rows of `b`: top-k first (0 < top_k < vocab), then the nucleus (0 < top_p < 1)
+// of what top-k left.
+template <bool VEC>
+__global__ void __launch_bounds__(kSelThreads)
+cut_floor_kernel(const float* __restrict__ a, size_t a_stride, int a_rows, const float* __restrict__ b,
+                 size_t b_stride, int b_rows, int vocab, int top_k, float top_p, float c2, float* __restrict__ floors) {
+    __shared__ SelShared sh;
+    pdl_trigger();
+    pdl_wait();
     const int per_seq = a_rows + b_rows;
     const int seq = blockIdx.x / per_seq, row = blockIdx.x % per_seq;
     const float* src = row < a_rows ? a + (static_cast<size_t>(seq) * a_rows + row) * a_stride
                                     : b + (static_cast<size_t>(seq) * b_rows + (row - a_rows)) * b_stride;
     const Row<VEC> r = make_row<VEC>(src, vocab);
     const int groups = (vocab + 3) >> 2;
-    if (tid < kCutSlots) counts[tid] = 0;
-    const uint32_t kf = use_k ? float_key(__ldcg(floors + blockIdx.x)) : 0u;
-
-    constexpr int G = KPT > 0 ? KPT / 4 : 1;
-    uint32_t keys[4 * G];
-    uint32_t top = 0;
-    if (KPT > 0) {
-#pragma unroll
-        for (int i = 0; i < G; ++i) {
-            const int g = tid + i * kFloorThreads;
-            const float4 v = g < groups ? r.raw(g, -INFINITY) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-            keys[4 * i + 0] = float_key(v.x);
-            keys[4 * i + 1] = float_key(v.y);
-            keys[4 * i + 2] = float_key(v.z);
-            keys[4 * i + 3] = float_key(v.w);
-        }
-#pragma unroll
-        for (int i = 0; i < 4 * G; ++i) top = max(top, keys[i]);
-    } else {
-        for (int g = tid; g < groups; g += kFloorThreads) {
-            const float4 v = r.raw(g, -INFINITY);
-            top = max(top, max(max(float_key(v.x), float_key(v.y)), max(float_key(v.z), float_key(v.w))));
-        }
-    }
-    top = __reduce_max_sync(0xffffffffu, top);
-    if (lane == 0) warp_top[warp] = top;
-    __syncthreads();
-#pragma unroll
-    for (int w = 0; w < kFloorWarps; ++w) top = max(top, warp_top[w]);
-    const float row_max = key_float(top);
-    auto weight = [&](float v) { return fast_exp2((v - row_max) * c2); };
-    if (KPT > 0) {
-#pragma unroll
-        for (int i = 0; i < 4 * G; ++i) wsm[i * kFloorThreads + tid] = weight(key_float(keys[i]));
-    }
-
-    // count and mass of the keys at or above t, the same values in every thread
-    int slot = 0;
-    auto measure = [&](uint32_t t, unsigned* count, float* mass) {
-        unsigned c = 0;
-        float m = 0.0f;
-        if (KPT > 0) {
-#pragma unroll
-            for (int i = 0; i < 4 * G; ++i)
-                if (keys[i] >= t) { ++c; m += wsm[i * kFloorThreads + tid]; }
-        } else {
-            for (int g = tid; g < groups; g += kFloorThreads) {
-                const float4 v = r.raw(g, -INFINITY);
-                if (float_key(v.x) >= t) { ++c; m += weight(v.x); }
-                if (float_key(v.y) >= t) { ++c; m += weight(v.y); }
-                if (float_key(v.z) >= t) { ++c; m += weight(v.z); }
-                if (float_key(v.w) >= t) { ++c; m += weight(v.w); }
-            }
-        }
-        c = __reduce_add_sync(0xffffffffu, c);
-        m = warp_sum(m);
-        if (lane == 0) {
-            if (c) atomicAdd(&counts[slot], c);
-            partial[slot][warp] = m;
-        }
-        __syncthreads();
-        float total = 0.0f;
-#pragma unroll
-        for (int w = 0; w < kFloorWarps; ++w) total += partial[slot][w];
-        *count = counts[slot];
-        *mass = total;
-        ++slot;
-    };
-
-    unsigned at_prefix;
-    float everything;
-    measure(kf, &at_prefix, &everything);
-    const float goal = top_p * everything;
-    uint32_t prefix = 0;
-    unsigned above = 0;
-    float mass_above = 0.0f;
-    int bit = 31;
-    for (; bit >= 0 && at_prefix - above > kLiveCap; --bit) {
-        const uint32_t cand = prefix | (1u << bit);
-        unsigned c;
-        float m;
-        measure(max(cand, kf), &c, &m);
-        if (m >= goal) { prefix = cand; at_prefix = c; } else { above = c; mass_above = m; }
-    }
-    if (bit >= 0) {
-        // undecided: at or above the top-k floor and equal to `prefix` on every bit above `bit`
-        const int shift = bit + 1;
-        auto undecided = [&](uint32_t key) { return key >= kf && (shift >= 32 || ((key ^ prefix) >> shift) == 0); };
-        unsigned mine = 0;
-        if (KPT > 0) {
-#pragma unroll
-            for (int i = 0; i < 4 * G; ++i) mine += undecided(keys[i]);
-        } else {
-            for (int g = tid; g < groups; g += kFloorThreads) {
-                const float4 v = r.raw(g, -INFINITY);
-                mine += undecided(float_key(v.x)) + undecided(float_key(v.y)) + undecided(float_key(v.z)) +
-                        undecided(float_key(v.w));
-            }
-        }
-        unsigned incl = mine;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const unsigned up = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += up;
-        }
-        // warps take their places in index order, so the copy (and every sum over it) is the same in every run
-        if (lane == 31) warp_top[warp] = incl;
-        __syncthreads();
-        unsigned pos = incl - mine, n_live = 0;
-#pragma unroll
-        for (int w = 0; w < kFloorWarps; ++w) {
-            if (w < warp) pos += warp_top[w];
-            n_live += warp_top[w];
-        }
-        auto keep = [&](uint32_t key, float w) {
-            if (undecided(key)) {
-                if (pos < kLiveCap) { live_key[pos] = key; live_w[pos] = w; }
-                ++pos;
-            }
-        };
-        if (KPT > 0) {
-#pragma unroll
-            for (int i = 0; i < 4 * G; ++i) keep(keys[i], wsm[i * kFloorThreads + tid]);
-        } else {
-            for (int g = tid; g < groups; g += kFloorThreads) {
-                const float4 v = r.raw(g, -INFINITY);
-                keep(float_key(v.x), weight(v.x));
-                keep(float_key(v.y), weight(v.y));
-                keep(float_key(v.z), weight(v.z));
-                keep(float_key(v.w), weight(v.w));
-            }
-        }
-        __syncthreads();
-        const int n = static_cast<int>(min(n_live, static_cast<unsigned>(kLiveCap)));  // = at_prefix - above
-        for (; bit >= 0; --bit) {
-            const uint32_t cand = prefix | (1u << bit);
-            float m = 0.0f;
-            for (int j = tid; j < n; j += kFloorThreads)
-                if (live_key[j] >= cand) m += live_w[j];
-            m = warp_sum(m);
-            if (lane == 0) partial[slot][warp] = m;
-            __syncthreads();
-            float total = mass_above;
-#pragma unroll
-            for (int w = 0; w < kFloorWarps; ++w) total += partial[slot][w];
-            ++slot;
-            if (total >= goal) prefix = cand;
-        }
-    }
-    if (tid == 0) floors[blockIdx.x] = key_float(max(prefix, kf));
+    float floor = -INFINITY;
+    if (top_k > 0 && top_k < vocab) floor = select_floor<VEC, false>(r, groups, floor, static_cast<unsigned>(top_k), 0.0f, 0.0f, sh);
+    if (top_p > 0.0f && top_p < 1.0f) floor = select_floor<VEC, true>(r, groups, floor, 0u, top_p, c2, sh);
+    if (threadIdx.x == 0) floors[blockIdx.x] = floor;
 }
 
 __global__ void uniforms_kernel(uint64_t seed, const int32_t* __restrict__ positions,
@@ -1044,71 +948,20 @@ bool cut_is_on(int vocab, float temperature, int top_k, float top_p) {
     return temperature > 0.0f && ((top_k > 0 && top_k < vocab) || (top_p > 0.0f && top_p < 1.0f));
 }
 
-// floors[s * (a_rows + b_rows) + r] = the top_k-th largest logit of sequence s's
-// row r (its a_rows rows of `a`, then its b_rows rows of `b`).  0 < top_k < vocab.
-int launch_topk_floors(const float* a, size_t a_stride, int a_rows, const float* b, size_t b_stride, int b_rows,
-                       int seqs, int vocab, int top_k, float* floors, cudaStream_t stream) {
-    const int total = seqs * (a_rows + b_rows);
-    if (total == 0) return SPEC_OK;
-    const bool vec = vocab % 4 == 0 && a_stride % 4 == 0 && aligned16(a) && (b_rows == 0 || (b_stride % 4 == 0 && aligned16(b)));
-#define SPEC_LAUNCH_FLOORS(V, K)                                                                              \
-    return launch_pdl(topk_floor_kernel<V, K>, dim3(total), dim3(kFloorThreads), 0, stream, a, a_stride, a_rows, b, \
-                      b_stride, b_rows, vocab, top_k, floors)
-    if (vocab <= kFloorThreads * 16) {
-        if (vec) SPEC_LAUNCH_FLOORS(true, 16);
-        SPEC_LAUNCH_FLOORS(false, 16);
-    }
-    if (vocab <= kFloorThreads * 64) {
-        if (vec) SPEC_LAUNCH_FLOORS(true, 64);
-        SPEC_LAUNCH_FLOORS(false, 64);
-    }
-    if (vec) SPEC_LAUNCH_FLOORS(true, 0);
-    SPEC_LAUNCH_FLOORS(false, 0);
-#undef SPEC_LAUNCH_FLOORS
-}
-
-// The same rows' nucleus floors for 0 < top_p < 1; with use_k, of the logits at or
-// above the floors already there.
-int launch_nucleus_floors(const float* a, size_t a_stride, int a_rows, const float* b, size_t b_stride, int b_rows,
-                          int seqs, int vocab, bool use_k, float top_p, float inv_t, float* floors, cudaStream_t stream) {
+// Top-k, then the nucleus of what is left (Section 2.2): one floor per row, one kernel.
+// floors[s * (a_rows + b_rows) + r] belongs to sequence s's row r (its a_rows rows of `a`,
+// then its b_rows rows of `b`).
+int launch_cut_floors(const float* a, size_t a_stride, int a_rows, const float* b, size_t b_stride, int b_rows,
+                      int seqs, int vocab, int top_k, float top_p, float inv_t, float* floors, cudaStream_t stream) {
     const int total = seqs * (a_rows + b_rows);
     if (total == 0) return SPEC_OK;
     const bool vec = vocab % 4 == 0 && a_stride % 4 == 0 && aligned16(a) && (b_rows == 0 || (b_stride % 4 == 0 && aligned16(b)));
     const float c2 = inv_t * kLog2e;
-#define SPEC_LAUNCH_NUCLEUS(V, K)                                                                                  \
-    do {                                                                                                           \
-        /* static + dynamic shared memory exceeds the 48 KB that needs no opt-in even for the short rows */         \
-        const size_t smem = static_cast<size_t>(K) * kFloorThreads * sizeof(float);                                \
-        if (smem > 0)                                                                                              \
-            SPEC_CUDA_TRY(cudaFuncSetAttribute(nucleus_floor_kernel<V, K>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                               static_cast<int>(smem)));                                           \
-        return launch_pdl(nucleus_floor_kernel<V, K>, dim3(total), dim3(kFloorThreads), smem, stream, a, a_stride, a_rows, \
-                          b, b_stride, b_rows, vocab, use_k, top_p, c2, floors);                                   \
-    } while (0)
-    if (vocab <= kFloorThreads * 16) {
-        if (vec) SPEC_LAUNCH_NUCLEUS(true, 16);
-        SPEC_LAUNCH_NUCLEUS(false, 16);
-    }
-    if (vocab <= kFloorThreads * 64) {
-        if (vec) SPEC_LAUNCH_NUCLEUS(true, 64);
-        SPEC_LAUNCH_NUCLEUS(false, 64);
-    }
-    if (vec) SPEC_LAUNCH_NUCLEUS(true, 0);
-    SPEC_LAUNCH_NUCLEUS(false, 0);
-#undef SPEC_LAUNCH_NUCLEUS
-}
-
-// Top-k, then the nucleus of what is left (Section 2.2): one floor per row.
-int launch_cut_floors(const float* a, size_t a_stride, int a_rows, const float* b, size_t b_stride, int b_rows,
-                      int seqs, int vocab, int top_k, float top_p, float inv_t, float* floors, cudaStream_t stream) {
-    const bool use_k = top_k > 0 && top_k < vocab;
-    if (use_k) {
-        const int st = launch_topk_floors(a, a_stride, a_rows, b, b_stride, b_rows, seqs, vocab, top_k, floors, stream);
-        if (st != SPEC_OK) return st;
-    }
-    if (top_p > 0.0f && top_p < 1.0f)
-        return launch_nucleus_floors(a, a_stride, a_rows, b, b_stride, b_rows, seqs, vocab, use_k, top_p, inv_t, floors, stream);
-    return SPEC_OK;
+    if (vec)
+        return launch_pdl(cut_floor_kernel<true>, dim3(total), dim3(kSelThreads), 0, stream, a, a_stride, a_rows, b, b_stride,
+                          b_rows, vocab, top_k, top_p, c2, floors);
+    return launch_pdl(cut_floor_kernel<false>, dim3(total), dim3(kSelThreads), 0, stream, a, a_stride, a_rows, b, b_stride,
+                      b_rows, vocab, top_k, top_p, c2, floors);
 }
 
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
