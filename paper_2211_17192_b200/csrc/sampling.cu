@@ -878,6 +878,67 @@ __device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned 
     return lo;
 }
 
+// The nucleus when top-k has already cut the row down to a few logits (those >= kf):
+// one pass copies them out, then they are ranked against each other as in step 3
+// above.  Returns false, having decided nothing, if more than kSelCap logits are
+// in play (a large tie at the top-k floor).
+template <bool VEC>
+__device__ bool nucleus_of_few(const Row<VEC>& r, int groups, float kf, float top_p, float c2, SelShared& sh, float* floor) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __syncthreads();  // (the shared arrays may still be read by a previous call)
+    if (tid == 0) sh.n_cand = 0;
+    __syncthreads();
+    for_each_logit(r, groups, [&](float v) {
+        if (fabsf(v) < INFINITY && v >= kf) {
+            const unsigned at = atomicAdd(&sh.n_cand, 1u);
+            if (at < kSelCap) sh.cand[at] = v;
+        }
+    });
+    __syncthreads();
+    const unsigned total = sh.n_cand;
+    if (total == 0 || total > kSelCap) return false;
+    const int count = static_cast<int>(total);
+    float row_max = -INFINITY;
+    for (int i = tid; i < count; i += kSelThreads) row_max = fmaxf(row_max, sh.cand[i]);
+    row_max = warp_max(row_max);
+    if (lane == 0) sh.warp_hi[warp] = row_max;
+    __syncthreads();
+    row_max = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) row_max = fmaxf(row_max, sh.warp_hi[w]);
+    unsigned long long mine_sum = 0;
+    for (int i = tid; i < count; i += kSelThreads) {
+        const unsigned long long m = __float2ull_rz(fast_exp2((sh.cand[i] - row_max) * c2) * 1099511627776.0f);  // 2^40
+        sh.cand_mass[i] = m;
+        mine_sum += m;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mine_sum += __shfl_xor_sync(0xffffffffu, mine_sum, o);
+    __syncthreads();  // (warp_hi has been read by everyone; cand_mass is complete)
+    if (lane == 0) sh.warp_mass[warp] = mine_sum;
+    __syncthreads();
+    unsigned long long all_mass = 0;
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) all_mass += sh.warp_mass[w];
+    const unsigned long long goal = static_cast<unsigned long long>(ceil(static_cast<double>(top_p) * static_cast<double>(all_mass)));
+    float best = -INFINITY;
+    for (int i = tid; i < count; i += kSelThreads) {
+        const float mine = sh.cand[i];
+        unsigned long long m = 0;
+        for (int j = 0; j < count; ++j)
+            if (sh.cand[j] >= mine) m += sh.cand_mass[j];
+        if (m >= goal) best = fmaxf(best, mine);
+    }
+    best = warp_max(best);
+    if (lane == 0) sh.warp_lo[warp] = best;
+    __syncthreads();
+    best = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) best = fmaxf(best, sh.warp_lo[w]);
+    *floor = best > -INFINITY ? best : kf;
+    return true;
+}
+
 // floors[s * (a_rows + b_rows) + r] for sequence s's a_rows rows of `a`, then its
 // b_rows rows of `b`: top-k first (0 < top_k < vocab), then the nucleus (0 < top_p < 1)
 // of what top-k left.
@@ -896,7 +957,12 @@ cut_floor_kernel(const float* __restrict__ a, size_t a_stride, int a_rows, const
     const int groups = (vocab + 3) >> 2;
     float floor = -INFINITY;
     if (top_k > 0 && top_k < vocab) floor = select_floor<VEC, false>(r, groups, floor, static_cast<unsigned>(top_k), 0.0f, 0.0f, sh);
-    if (top_p > 0.0f && top_p < 1.0f) floor = select_floor<VEC, true>(r, groups, floor, 0u, top_p, c2, sh);
+    if (top_p > 0.0f && top_p < 1.0f) {
+        // after a top-k that leaves few logits the nucleus needs no binning
+        const bool few = floor > -INFINITY && top_k <= kSelCap;
+        if (!few || !nucleus_of_few<VEC>(r, groups, floor, top_p, c2, sh, &floor))
+            floor = select_floor<VEC, true>(r, groups, floor, 0u, top_p, c2, sh);
+    }
     if (threadIdx.x == 0) floors[blockIdx.x] = floor;
 }
 
