@@ -706,18 +706,20 @@ struct SelShared {
     unsigned long long before_mass;
 };
 
-// f(v) for every logit of the row, four 128-bit loads in flight per thread.
+// f(v) for every logit of the row, kSelLoads 128-bit loads in flight per thread.
+constexpr int kSelLoads = 8;
+
 template <bool VEC, class F>
 __device__ __forceinline__ void for_each_logit(const Row<VEC>& r, int groups, F f) {
-    for (int g0 = threadIdx.x; g0 < groups; g0 += 4 * kSelThreads) {
-        float4 v[4];
+    for (int g0 = threadIdx.x; g0 < groups; g0 += kSelLoads * kSelThreads) {
+        float4 v[kSelLoads];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kSelLoads; ++i) {
             const int g = g0 + i * kSelThreads;
             v[i] = g < groups ? r.raw(g, -INFINITY) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kSelLoads; ++i) {
             f(v[i].x);
             f(v[i].y);
             f(v[i].z);
