@@ -123,12 +123,15 @@ int spec_verify_sample_lenient(const float* target_logits, const float* draft_lo
  * the first off, top_p <= 0 or >= 1 the second; with both off, or at T == 0 (the
  * maximum is always kept), this is spec_verify_sample_lenient exactly.  A
  * drafted token outside the target's kept set has p_i(x_i) = 0 and is rejected
- * unless q_i(x_i) is 0 too.  Enqueues one more kernel per active cut (the
- * per-row selections) before the other two; same workspace.  The nucleus sums
- * fp32 weights in a fixed order: a row always gives the same cut, and a cut
- * whose mass comes within rounding of top_p may differ from exact arithmetic
- * by one token.  Errors as above plus SPEC_ERR_BAD_ARG for top_k < 0 or a NaN
- * top_p. */
+ * unless q_i(x_i) is 0 too.  Enqueues one more kernel (the per-row selection,
+ * both cuts in one launch) before the other two; same workspace.  Top-k is
+ * exact.  The nucleus takes fp32 weights exp((l - max) / T) from the hardware
+ * exp2 and sums them in 2^-40 fixed point with integer additions, so a row
+ * always gives the same cut whatever the order of summation; a cut whose mass
+ * comes within the weights' rounding (about 1e-6 of the total) of top_p may
+ * differ from exact arithmetic by a neighbouring token.  Logits that are
+ * -inf, +inf or NaN are never counted.  Errors as above plus SPEC_ERR_BAD_ARG
+ * for top_k < 0 or a NaN top_p. */
 int spec_verify_sample_truncated(const float* target_logits, const float* draft_logits,
                                  const int32_t* draft_tokens, const float* uniforms,
                                  int batch, int gamma, int vocab, float temperature, float lenience,
@@ -195,7 +198,7 @@ int spec_sample(const float* logits, const float* uniforms, int rows, int vocab,
 /* The same over what top-k and the nucleus keep of each row (see
  * spec_verify_sample_truncated); floors [rows] fp32 device is scratch that
  * receives the rows' thresholds (may be NULL when both cuts are off or T == 0,
- * where the call is spec_sample).  One more kernel per active cut. */
+ * where the call is spec_sample).  One more kernel. */
 int spec_sample_truncated(const float* logits, const float* uniforms, int rows, int vocab,
                           float temperature, int top_k, float top_p, int32_t* tokens,
                           float* floors, void* stream);
