@@ -762,7 +762,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
                 if (ctx->model[i].bf16() && ctx->model[i].cfg.arch != SPEC_ARCH_BIGRAM &&
                     (status = pack_model(ctx, ctx->model[i])) != SPEC_OK)
                     return cleanup(status);
-            ctx->hi_rows = (ctx->max_rows + 127) / 128 * 128;
+            ctx->hi_rows = (ctx->max_rows + 255) / 256 * 256;  // whole token tiles of the widest GEMM variant
             SPEC_ALLOC(x_hi, static_cast<size_t>(ctx->hi_rows) * max_k);
             SPEC_ALLOC(x_lo, static_cast<size_t>(ctx->hi_rows) * max_k);
             SPEC_ALLOC(partials, partial);

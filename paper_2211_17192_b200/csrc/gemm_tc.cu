@@ -122,7 +122,8 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 
 template <int N_TOK>
 struct Smem {
-    static constexpr int kStages = N_TOK <= 16 ? 5 : N_TOK == 64 ? 3 : 4;
+    // two CTAs per SM up to 128 rows; wider tiles fill the SM alone
+    static constexpr int kStages = N_TOK <= 16 ? 5 : N_TOK <= 32 ? 4 : N_TOK <= 64 ? 3 : N_TOK <= 128 ? 2 : 3;
     static constexpr int kABytes = kTileM * kTileK * 2;   // 16 KB
     static constexpr int kBBytes = N_TOK * kTileK * 2;     // one of hi / lo
     static constexpr int kStageBytes = kABytes + 2 * kBBytes;
@@ -136,7 +137,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                const __grid_constant__ CUtensorMap map_lo, float* __restrict__ partial, int n_out, int n_rows,
                int k_blocks, int packed) {
     using S = Smem<N_TOK>;
-    constexpr int kTmemCols = N_TOK < 32 ? 32 : N_TOK;
+    constexpr int kTmemCols = N_TOK <= 32 ? 32 : N_TOK <= 64 ? 64 : N_TOK <= 128 ? 128 : 256;  // a power of two that holds N_TOK columns
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + S::kStages * S::kStageBytes);
@@ -389,7 +390,21 @@ int launch_tc(const CUtensorMap& mw, const CUtensorMap& mhi, const CUtensorMap& 
 
 }  // namespace
 
-int gemm_tc_token_tile(int n_rows) { return n_rows <= 16 ? 16 : n_rows <= 32 ? 32 : n_rows <= 64 ? 64 : 128; }
+// Rows per CTA (the MMA's N): the smallest tile that holds the rows, so that up to 192 rows
+// the weights are streamed once (the tensor-core work and the activation tiles that
+// every CTA re-reads grow with the padded row count); more rows take tiles of 128, two
+// CTAs per SM (measured: a 256-row tile leaves room for two pipeline stages only and
+// is slower than two passes of 128).
+int gemm_tc_token_tile(int n_rows) {
+    if (n_rows <= 16) return 16;
+    if (n_rows <= 32) return 32;
+    if (n_rows <= 48) return 48;
+    if (n_rows <= 64) return 64;
+    if (n_rows <= 96) return 96;
+    if (n_rows <= 128) return 128;
+    if (n_rows <= 192) return 192;
+    return 128;
+}
 
 // Split-K factor: the smallest one that fills the last wave of CTAs to 85 %, with
 // at least two k-blocks per split.
@@ -397,7 +412,7 @@ int gemm_tc_splits(int n_out, int k, int n_rows) {
     const int n_tok = gemm_tc_token_tile(n_rows);
     const int tiles = ((n_out + kTileM - 1) / kTileM) * ((n_rows + n_tok - 1) / n_tok);
     const int k_blocks = (k + kTileK - 1) / kTileK;
-    const int resident = 148 * (n_tok <= 64 ? 2 : 1);
+    const int resident = 148 * (n_tok <= 128 ? 2 : 1);
     const int max_splits = std::max(1, std::min(k_blocks / 2, 16));
     int best = 1;
     double best_eff = 0.0;
@@ -457,8 +472,11 @@ int launch_gemm_tc_partials(const __nv_bfloat16* hi, const __nv_bfloat16* lo, in
     switch (n_tok) {
         case 16: return launch_tc<16>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
         case 32: return launch_tc<32>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
+        case 48: return launch_tc<48>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
         case 64: return launch_tc<64>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
-        default: return launch_tc<128>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
+        case 96: return launch_tc<96>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
+        case 128: return launch_tc<128>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
+        default: return launch_tc<192>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
     }
 }
 
@@ -489,7 +507,7 @@ int gemm_tc_take_error() {
 // ---- C ABI: one linear layer, for tests and benchmarks of the GEMM kernels ----
 namespace {
 size_t align256(size_t v) { return (v + 255) / 256 * 256; }
-int padded_rows(int rows) { return (rows + 127) / 128 * 128; }
+int padded_rows(int rows) { return (rows + 255) / 256 * 256; }
 }  // namespace
 
 extern "C" size_t spec_linear_workspace_bytes(int rows, int n_out, int k) {

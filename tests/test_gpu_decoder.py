@@ -135,7 +135,8 @@ def test_errors_are_reported():
 
 
 @pytest.mark.parametrize("rows,n_out,k", [(1, 128, 64), (5, 300, 200), (3, 768, 768), (11, 2304, 768), (16, 704, 256),
-                                          (17, 256, 512), (70, 384, 256), (130, 256, 192), (7, 8192, 768)])
+                                          (17, 256, 512), (70, 384, 256), (130, 256, 192), (7, 8192, 768),
+                                          (40, 384, 320), (48, 256, 256), (96, 512, 192), (160, 384, 256), (250, 256, 128)])
 def test_linear_layer_paths_agree_with_the_plain_definition(rows, n_out, k):
     """y = x W^T on the FMA pipes, on the tensor cores (row-major and tile-major
     weights) against numpy in fp64; the two tensor-core layouts are bit-identical."""
