@@ -121,6 +121,29 @@ def test_temperature_zero_equals_target_only_greedy(tiny, gamma):
     assert stats["iterations"] >= 3 * 32 / (gamma + 1)
 
 
+def test_adaptive_gamma_and_truncation_on_the_encoder_decoder(tiny):
+    """The options of the generation loop on this model family too: gamma chosen by the library
+    (T = 0: still the target's greedy output), and top-k / nucleus against the oracle at T = 1."""
+    eng, (tcfg, tw), (dcfg, dw) = tiny
+    sources = _sources(tcfg["vocab"], [30, 64, 11], seed=78)
+    greedy, _ = eng.generate(sources, 32, 0, 0.0, 0)
+    adaptive, stats, trace = eng.generate_adaptive(sources, 32, 5, 0.0, 0, burst=2)
+    assert np.array_equal(greedy, adaptive) and len({g for g, _ in trace}) >= 2
+    assert sum(n for _, n in trace) == stats["target_passes"]
+    target, draft = EncoderDecoder(tcfg, tw), EncoderDecoder(dcfg, dw)
+    target.encode(sources[0])
+    draft.encode(sources[0])
+    try:
+        eng.set_truncation(8, 0.9)
+        ref = oracle_generate.speculative_generate(target, draft, [START_TOKEN], 40, 3, 1.0, seed=5, top_k=8, top_p=0.9)
+        got, _ = eng.generate([sources[0]], 40, 3, 1.0, 5)
+        got = got[0].tolist()
+        diff = next((i for i in range(40) if got[i] != ref.tokens[i]), 40)
+        assert diff >= 10, f"streams differ at token {diff}"  # (a boundary decision may end the comparison later on)
+    finally:
+        eng.set_truncation(0, 1.0)
+
+
 def test_errors(tiny):
     eng, (tcfg, tw), _ = tiny
     with pytest.raises(binding.SpecError) as e:
