@@ -389,12 +389,15 @@ __device__ __forceinline__ void stage_tile(const __nv_bfloat16* tile, int n_vali
     }
 }
 
-template <int DH>
+// IN_TURN: K and V of a tile share one buffer - V is loaded once the scores are done with K.
+// Half the shared memory per warp, so two CTAs share an SM (d_head 128), at the price of
+// a second exposed load per tile: it pays when the launch has CTAs for more than one wave.
+template <int DH, bool IN_TURN>
 struct MmaSmem {
     static constexpr int kRow = DH + 4;              // floats per staged row (bank-conflict-free fragments)
     static constexpr int kQ = 16 * kRow;             // the queries, scaled and rounded to tf32
     static constexpr int kTile = kTileKeys * kRow;   // one staged K or V tile
-    static constexpr int kStage = 2 * kTile;         // K and V of one tile
+    static constexpr int kStage = (IN_TURN ? 1 : 2) * kTile;  // K and V of one tile
     static constexpr int kPStride = 20;              // floats per row of the probabilities (bank-conflict-free)
     static constexpr int kP = 16 * kPStride;         // probabilities of one tile
     static constexpr int kPerWarp = kMmaStages * kStage + kP;
@@ -402,14 +405,14 @@ struct MmaSmem {
 };
 
 // grid = (slices, n_kv_heads * m_blocks, batch), block = 32 * kMmaWarps.
-template <typename KV, int DH, bool FUSED>
+template <typename KV, int DH, bool FUSED, bool IN_TURN>
 __global__ void __launch_bounds__(32 * kMmaWarps)
 attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __restrict__ pos,
                      const int32_t* __restrict__ seq, int m_rows, int n_heads, int n_kv_heads, int m_blocks,
                      const KV* __restrict__ kv_layer, const int32_t* __restrict__ page_table, int pages_per_seq,
                      int page_size, const int32_t* __restrict__ kv_len, const float* __restrict__ bias, int bias_span,
                      int bias_zero, float scale, float* __restrict__ part, const AttnOut out) {
-    using S = MmaSmem<DH>;
+    using S = MmaSmem<DH, IN_TURN>;
     extern __shared__ __align__(16) float smem_f[];
     __shared__ int q_pos[16], q_row[16], q_head[16];
     pdl_trigger();
@@ -474,7 +477,7 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
                                  static_cast<size_t>(k0 % page_size) * DH;
                 float* st = stage0 + (i % kMmaStages) * S::kStage;
                 stage_tile<DH>(tile, n_valid, st, lane);
-                stage_tile<DH>(tile + v_offset, n_valid, st + S::kTile, lane);
+                if (!IN_TURN) stage_tile<DH>(tile + v_offset, n_valid, st + S::kTile, lane);
             }
         }
         cp_async_commit();
@@ -494,7 +497,7 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
         __syncwarp();
         if (k0 < seq_keys) {
             const float* Kt = stage0 + (i % kMmaStages) * S::kStage;
-            const float* Vt = Kt + S::kTile;
+            const float* Vt = IN_TURN ? Kt : Kt + S::kTile;
             // S = Q K^T: two blocks of 8 keys; even and odd k-steps go to separate accumulators
             // (four independent MMA chains instead of two), added at the end
             float s[2][4], s_odd[2][4];
@@ -564,6 +567,15 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
             m_lo = new_lo;
             m_hi = new_hi;
             __syncwarp();  // every lane's probabilities are in shared memory
+            if (IN_TURN) {  // the scores are done with K: V takes its place
+                const int n_valid = min(kTileKeys, seq_keys - k0);
+                const KV* tile = kv_layer + pages[k0 / page_size] * page_stride + kv_head * head_stride +
+                                 static_cast<size_t>(k0 % page_size) * DH;
+                stage_tile<DH>(tile + v_offset, n_valid, stage0 + (i % kMmaStages) * S::kStage, lane);
+                cp_async_commit();
+                cp_async_wait<0>();
+                __syncwarp();
+            }
 
             // O = O * rescale + P V
             uint32_t pa[2][4];
@@ -774,24 +786,30 @@ int launch_attention_variant(const Model& m, const AttnSource& src, const RowMet
     const KV* pool = static_cast<const KV*>(src.pool.kv);
     int status;
     if (attention_uses_mma(m, batch, m_rows, max_keys)) {
-        static bool configured = false;
-        if (!configured) {
-            SPEC_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<KV, DH, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               static_cast<int>(MmaSmem<DH>::kBytes)));
-            SPEC_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<KV, DH, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               static_cast<int>(MmaSmem<DH>::kBytes)));
-            configured = true;
-        }
         const int m_blocks = (queries + 15) / 16;
         const dim3 grid(slices, m.cfg.n_kv_heads * m_blocks, batch);
-        status = fused ? launch_attn(attention_mma_kernel<KV, DH, true>, grid, dim3(32 * kMmaWarps), MmaSmem<DH>::kBytes, slices,
-                                     stream, src.q, src.q_stride, rows.pos, rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads,
-                                     m_blocks, pool, src.pool.page_table, src.pool.pages_per_seq, src.pool.page_size, src.kv_len,
-                                     src.bias, src.bias_span, src.bias_zero, scale, part, out)
-                       : launch_attn(attention_mma_kernel<KV, DH, false>, grid, dim3(32 * kMmaWarps), MmaSmem<DH>::kBytes, 0,
-                                     stream, src.q, src.q_stride, rows.pos, rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads,
-                                     m_blocks, pool, src.pool.page_table, src.pool.pages_per_seq, src.pool.page_size, src.kv_len,
-                                     src.bias, src.bias_span, src.bias_zero, scale, part, out);
+        // K and V of a tile in turn (two CTAs per SM) once there are (sequence, KV head, query block)
+        // groups for more than a thin wave: measured on the 7B shape, better from 32 groups on
+        const bool in_turn = batch * m.cfg.n_kv_heads * m_blocks >= 32;
+#define SPEC_LAUNCH_MMA(F, T, CLUSTER)                                                                                  \
+    do {                                                                                                                \
+        static bool configured = false;                                                                                 \
+        if (!configured) {                                                                                              \
+            SPEC_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<KV, DH, F, T>,                                      \
+                                               cudaFuncAttributeMaxDynamicSharedMemorySize,                             \
+                                               static_cast<int>(MmaSmem<DH, T>::kBytes)));                              \
+            configured = true;                                                                                          \
+        }                                                                                                               \
+        status = launch_attn(attention_mma_kernel<KV, DH, F, T>, grid, dim3(32 * kMmaWarps), MmaSmem<DH, T>::kBytes,    \
+                             CLUSTER, stream, src.q, src.q_stride, rows.pos, rows.seq, m_rows, m.cfg.n_heads,           \
+                             m.cfg.n_kv_heads, m_blocks, pool, src.pool.page_table, src.pool.pages_per_seq,            \
+                             src.pool.page_size, src.kv_len, src.bias, src.bias_span, src.bias_zero, scale, part, out); \
+    } while (0)
+        if (fused && in_turn) SPEC_LAUNCH_MMA(true, true, slices);
+        else if (fused) SPEC_LAUNCH_MMA(true, false, slices);
+        else if (in_turn) SPEC_LAUNCH_MMA(false, true, 0);
+        else SPEC_LAUNCH_MMA(false, false, 0);
+#undef SPEC_LAUNCH_MMA
     } else {
         const int ks = attention_sub_slices(queries);
         const int warps = std::min(kMaxAttnWarps, std::max(1, queries * ks));
