@@ -550,6 +550,15 @@ WORKLOAD_NAMES = ["llama7b", "t5xxl", "gpt97m", "sampler"]
 
 
 # --------------------------------------------------------------------------- #
+def load_tensor_peak():
+    """Measured dense bf16 rate of a library GEMM timed alone (burst), TFLOP/s; the earlier measurement if the file is absent."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    return 1590.0, "fallback"
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -745,6 +754,14 @@ def run_generation(args, wl, torch, device, local, barrier):
                                          "capture of the four GEMMs of a 7B-shaped block shows (363.6 MB vs 354.4 MB; "
                                          "profiles/ncu_gemm_tc_llama7b_layer.txt)",
                          "algorithmic_bytes_per_launch": nbytes / n_mats,
+                         # the same sweep against the tensor pipes: where rows approach the ridge (about 216-262 rows)
+                         # the GEMMs stop being purely bandwidth-bound; two MMAs per k-step (split activations)
+                         "tensor": (lambda tp: {"useful_tflops": rows * nbytes / (gemm_ms / 1e3) / 1e12,
+                                                "issued_tflops": 2 * rows * nbytes / (gemm_ms / 1e3) / 1e12,
+                                                "peak": tp[0], "peak_kind": f"of {tp[1]} (burst)",
+                                                "frac_issued": 2 * rows * nbytes / (gemm_ms / 1e3) / 1e12 / tp[0],
+                                                "note": "2 x rows x parameters flop per sweep; issued counts both "
+                                                        "bf16 terms of the activations"})(load_tensor_peak()),
                          "launch_us": 1e3 * gemm_ms / n_mats,
                          "note": f"all {n_mats} weight matrices of the target once at {rows} rows through spec_linear_partials "
                                  "(the GEMM kernel alone, tile-major weights, one launch per matrix back to back), "
