@@ -820,13 +820,11 @@ int launch_attention_variant(const Model& m, const AttnSource& src, const RowMet
         const bool in_turn = batch * m.cfg.n_kv_heads * m_blocks >= 32;
 #define SPEC_LAUNCH_MMA(F, T, CLUSTER)                                                                                  \
     do {                                                                                                                \
-        static bool configured = false;                                                                                 \
-        if (!configured) {                                                                                              \
+        static std::atomic<unsigned long long> configured{0};                                                           \
+        if (first_use_on_this_device(configured))                                                                       \
             SPEC_CUDA_TRY(cudaFuncSetAttribute(attention_mma_kernel<KV, DH, F, T>,                                      \
                                                cudaFuncAttributeMaxDynamicSharedMemorySize,                             \
                                                static_cast<int>(MmaSmem<DH, T>::kBytes)));                              \
-            configured = true;                                                                                          \
-        }                                                                                                               \
         status = launch_attn(attention_mma_kernel<KV, DH, F, T>, grid, dim3(32 * kMmaWarps), MmaSmem<DH, T>::kBytes,    \
                              CLUSTER, stream, qrows, rows.pos, rows.seq, m_rows, m.cfg.n_heads,                       \
                              m.cfg.n_kv_heads, m_blocks, pool, src.pool.page_table, src.pool.pages_per_seq,            \

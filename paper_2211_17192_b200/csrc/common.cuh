@@ -2,6 +2,7 @@
 // the counter-based generator.  sm_100a only.
 #pragma once
 
+#include <atomic>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -45,6 +46,16 @@ __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.lau
 
 // SPEC_NO_PDL=1 in the environment launches every kernel fully serialised (for debugging).
 bool pdl_enabled();  // api.cu
+
+// True the first time it is called on the current device for this flag word (one bit per
+// device ordinal below 64): per-device one-time setup such as a kernel's shared-memory opt-in,
+// which a process that uses several GPUs has to repeat on each of them.
+inline bool first_use_on_this_device(std::atomic<unsigned long long>& seen) {
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return true;
+    const unsigned long long bit = 1ull << device;
+    return (seen.fetch_or(bit) & bit) == 0;
+}
 
 template <typename... KArgs, typename... Args>
 inline int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {

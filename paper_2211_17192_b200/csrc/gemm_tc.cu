@@ -377,12 +377,10 @@ int cached_map(const void* base, int rows, int cols, int box_rows, CUtensorMap* 
 template <int N_TOK>
 int launch_tc(const CUtensorMap& mw, const CUtensorMap& mhi, const CUtensorMap& mlo, float* partial, int n_out,
               int n_rows, int k_blocks, int splits, int packed, cudaStream_t stream) {
-    static bool configured = false;
-    if (!configured) {
+    static std::atomic<unsigned long long> configured{0};
+    if (first_use_on_this_device(configured))
         SPEC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<N_TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            Smem<N_TOK>::kTotal));
-        configured = true;
-    }
     const dim3 grid((n_out + kTileM - 1) / kTileM, splits, (n_rows + N_TOK - 1) / N_TOK);
     return launch_pdl(gemm_tc_kernel<N_TOK>, grid, dim3(kThreads), Smem<N_TOK>::kTotal, stream, mw, mhi, mlo, partial,
                       n_out, n_rows, k_blocks, packed);
