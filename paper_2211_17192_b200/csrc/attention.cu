@@ -83,20 +83,6 @@ struct KvLoad<__nv_bfloat16> {
 // read the slices' states through distributed shared memory, merge them in
 // slice order and write the attention output.  No partial state goes through
 // global memory and no second kernel is needed.
-// The query rows: plain, or as the split-K partial sums of their projection (summed on the fly).
-struct QRows {
-    const float* base;
-    int stride;
-    int splits;
-    size_t split_stride;
-    __device__ __forceinline__ float at(size_t i) const {
-        if (splits == 0) return base[i];
-        float v = 0.0f;
-        for (int s = 0; s < splits; ++s) v += base[s * split_stride + i];  // in split order, as the reduction kernels do
-        return v;
-    }
-};
-
 struct AttnOut {
     float* att;             // fp32 [rows][n_heads * DH] or nullptr
     __nv_bfloat16 *hi, *lo;  // the same as two bf16 terms, or nullptr
@@ -164,7 +150,7 @@ __device__ __forceinline__ void cluster_merge_write(const float* fin, int n_q, i
 // grid is launched as clusters over the slice dimension and writes `out` itself.
 template <typename KV, int DH, bool FUSED>
 __global__ void __launch_bounds__(32 * kMaxAttnWarps)
-attention_kernel(const QRows qrows, const int32_t* __restrict__ pos,
+attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __restrict__ pos,
                  const int32_t* __restrict__ seq, int m_rows, int n_heads, int n_kv_heads, int ks,
                  const KV* __restrict__ kv_layer, const int32_t* __restrict__ page_table, int pages_per_seq,
                  int page_size, const int32_t* __restrict__ kv_len, const float* __restrict__ bias, int bias_span,
@@ -203,13 +189,7 @@ attention_kernel(const QRows qrows, const int32_t* __restrict__ pos,
         const int p = pos[r];
         const int32_t* pages = page_table + seq[r] * pages_per_seq;
         float qv[PER_LANE];  // this lane's share of the (scaled) query
-        const size_t q_at = static_cast<size_t>(r) * qrows.stride + head * DH + lane * PER_LANE;
-        if (qrows.splits == 0) {
-            KvLoad<float>::template load_n<PER_LANE>(qrows.base + q_at, qv);
-        } else {
-#pragma unroll
-            for (int i = 0; i < PER_LANE; ++i) qv[i] = qrows.at(q_at + i);
-        }
+        KvLoad<float>::template load_n<PER_LANE>(qkv + static_cast<size_t>(r) * q_stride + head * DH + lane * PER_LANE, qv);
 #pragma unroll
         for (int i = 0; i < PER_LANE; ++i) qv[i] *= scale;
 
@@ -427,7 +407,7 @@ struct MmaSmem {
 // grid = (slices, n_kv_heads * m_blocks, batch), block = 32 * kMmaWarps.
 template <typename KV, int DH, bool FUSED, bool IN_TURN>
 __global__ void __launch_bounds__(32 * kMmaWarps)
-attention_mma_kernel(const QRows qrows, const int32_t* __restrict__ pos,
+attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __restrict__ pos,
                      const int32_t* __restrict__ seq, int m_rows, int n_heads, int n_kv_heads, int m_blocks,
                      const KV* __restrict__ kv_layer, const int32_t* __restrict__ page_table, int pages_per_seq,
                      int page_size, const int32_t* __restrict__ kv_len, const float* __restrict__ bias, int bias_span,
@@ -507,7 +487,7 @@ attention_mma_kernel(const QRows qrows, const int32_t* __restrict__ pos,
     for (int i = 0; i < kMmaStages; ++i) issue(i);
     for (int i = tid; i < 16 * DH; i += 32 * kMmaWarps) {
         const int qi = i / DH, e = i % DH;
-        const float v = q_pos[qi] >= 0 ? qrows.at(static_cast<size_t>(q_row[qi]) * qrows.stride + q_head[qi] * DH + e) * scale : 0.0f;
+        const float v = q_pos[qi] >= 0 ? qkv[static_cast<size_t>(q_row[qi]) * q_stride + q_head[qi] * DH + e] * scale : 0.0f;
         Qs[qi * S::kRow + e] = __uint_as_float(to_tf32(v));
     }
     __syncthreads();
@@ -810,7 +790,6 @@ int launch_attention_variant(const Model& m, const AttnSource& src, const RowMet
     const int n_rows = batch * m_rows;
     const bool fused = attention_merges_in_cluster(m, batch, m_rows, max_keys) && slices <= kMaxClusterSlices;
     const KV* pool = static_cast<const KV*>(src.pool.kv);
-    const QRows qrows{src.q, src.q_stride, src.q_splits, src.q_split_stride};
     int status;
     if (attention_uses_mma(m, batch, m_rows, max_keys)) {
         const int m_blocks = (queries + 15) / 16;
@@ -826,7 +805,7 @@ int launch_attention_variant(const Model& m, const AttnSource& src, const RowMet
                                                cudaFuncAttributeMaxDynamicSharedMemorySize,                             \
                                                static_cast<int>(MmaSmem<DH, T>::kBytes)));                              \
         status = launch_attn(attention_mma_kernel<KV, DH, F, T>, grid, dim3(32 * kMmaWarps), MmaSmem<DH, T>::kBytes,    \
-                             CLUSTER, stream, qrows, rows.pos, rows.seq, m_rows, m.cfg.n_heads,                       \
+                             CLUSTER, stream, src.q, src.q_stride, rows.pos, rows.seq, m_rows, m.cfg.n_heads,           \
                              m.cfg.n_kv_heads, m_blocks, pool, src.pool.page_table, src.pool.pages_per_seq,            \
                              src.pool.page_size, src.kv_len, src.bias, src.bias_span, src.bias_zero, scale, part, out); \
     } while (0)
@@ -839,11 +818,11 @@ int launch_attention_variant(const Model& m, const AttnSource& src, const RowMet
         const int ks = attention_sub_slices(queries);
         const int warps = std::min(kMaxAttnWarps, std::max(1, queries * ks));
         const dim3 grid(slices, m.cfg.n_kv_heads, batch);
-        status = fused ? launch_attn(attention_kernel<KV, DH, true>, grid, dim3(32 * warps), 0, slices, stream, qrows,
+        status = fused ? launch_attn(attention_kernel<KV, DH, true>, grid, dim3(32 * warps), 0, slices, stream, src.q, src.q_stride,
                                      rows.pos, rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads, ks, pool, src.pool.page_table,
                                      src.pool.pages_per_seq, src.pool.page_size, src.kv_len, src.bias, src.bias_span,
                                      src.bias_zero, scale, part, out)
-                       : launch_attn(attention_kernel<KV, DH, false>, grid, dim3(32 * warps), 0, 0, stream, qrows,
+                       : launch_attn(attention_kernel<KV, DH, false>, grid, dim3(32 * warps), 0, 0, stream, src.q, src.q_stride,
                                      rows.pos, rows.seq, m_rows, m.cfg.n_heads, m.cfg.n_kv_heads, ks, pool, src.pool.page_table,
                                      src.pool.pages_per_seq, src.pool.page_size, src.kv_len, src.bias, src.bias_span,
                                      src.bias_zero, scale, part, out);

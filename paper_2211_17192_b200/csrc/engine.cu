@@ -236,14 +236,12 @@ int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_ro
         if (m.t5()) {  // cross-attention over the source's K,V (every row sees every source position)
             SPEC_TRY(pass.norm(w.lnx, nullptr, n_rows));
             SPEC_TRY(pass.proj(w.wq_x, pw.wq_x, m.q_dim(), d, ctx->a, ctx->qkv));
+            if (pass.tc)  // the partial sums become the query rows
+                SPEC_TRY(launch_qkv(c.n_heads, 0, c.d_head, nullptr, KvPool{}, rows, n_rows, ctx->qkv, ctx->partials,
+                                    pass.last_splits, ctx->stream));
             const KvPool pool = source_pool(ctx, m, static_cast<char*>(m.cross_kv) + static_cast<size_t>(l) * m.cross_stride);
             const int slices = attention_slices(m, batch, m_rows, ctx->rt.max_src_len);
-            AttnSource src{ctx->qkv, m.q_dim(), pool, ctx->src_len, nullptr, 0, 0};
-            if (pass.tc) {  // the attention kernel adds up the query projection's partial sums itself
-                src.q = ctx->partials;
-                src.q_splits = pass.last_splits;
-                src.q_split_stride = static_cast<size_t>(n_rows) * m.q_dim();
-            }
+            const AttnSource src{ctx->qkv, m.q_dim(), pool, ctx->src_len, nullptr, 0, 0};
             SPEC_TRY(launch_attention(m, src, rows, batch, m_rows, slices, ctx->rt.max_src_len, ctx->attn_part, pass.tc ? nullptr : ctx->att,
                                       pass.tc ? pass.hi() : nullptr, pass.tc ? pass.lo() : nullptr, ctx->stream));
             SPEC_TRY(pass.residual(w.wo_x, pw.wo_x, m.q_dim(), ctx->att));

@@ -130,10 +130,6 @@ struct AttnSource {
     const float* bias;
     int bias_span;
     int bias_zero;
-    // q_splits > 0: q holds the split-K partial sums of the query projection, [q_splits][rows][q_stride]
-    // (q_split_stride elements apart), and the attention kernel adds them up itself
-    int q_splits = 0;
-    size_t q_split_stride = 0;
 };
 
 // att[r, h] = softmax(scores) V for the rows of a pass; rows of sequence b are
