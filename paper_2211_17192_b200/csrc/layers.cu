@@ -24,8 +24,16 @@ __device__ __forceinline__ void store_split(__nv_bfloat16* hi, __nv_bfloat16* lo
 
 // sum of the split-K partial results of element i, in split order
 __device__ __forceinline__ float sum_partials(const float* __restrict__ partial, int splits, size_t stride, size_t i) {
-    float acc = partial[i];
-    for (int s = 1; s < splits; ++s) acc += partial[static_cast<size_t>(s) * stride + i];
+    // eight loads in flight at a time (the adds stay in split order, so the sum is the reduction kernels')
+    float acc = 0.0f;
+    for (int s0 = 0; s0 < splits; s0 += 8) {
+        float p[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) p[k] = s0 + k < splits ? partial[static_cast<size_t>(s0 + k) * stride + i] : 0.0f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (s0 + k < splits) acc = (s0 + k == 0) ? p[k] : acc + p[k];
+    }
     return acc;
 }
 
@@ -80,9 +88,15 @@ norm_kernel(float* h, const float* __restrict__ partial, int splits, int n_rows,
         if (g < groups) {
             v[j] = *reinterpret_cast<const float4*>(h + src + 4 * g);
             if (partial) {
-                for (int s = 0; s < splits; ++s) {
-                    const float4 p = *reinterpret_cast<const float4*>(partial + s * stride + src + 4 * g);
-                    v[j].x += p.x; v[j].y += p.y; v[j].z += p.z; v[j].w += p.w;
+                for (int s0 = 0; s0 < splits; s0 += 8) {  // eight loads in flight at a time, added in split order
+                    float4 p[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        p[k] = s0 + k < splits ? *reinterpret_cast<const float4*>(partial + (s0 + k) * stride + src + 4 * g)
+                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        if (s0 + k < splits) { v[j].x += p[k].x; v[j].y += p[k].y; v[j].z += p[k].z; v[j].w += p[k].w; }
                 }
                 *reinterpret_cast<float4*>(h + src + 4 * g) = v[j];
             }
