@@ -309,8 +309,15 @@ __global__ void reduce_partials_kernel(const float* __restrict__ partial, int sp
     const size_t total = static_cast<size_t>(n_rows) * n_out;
     for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < total;
          i += static_cast<size_t>(gridDim.x) * blockDim.x) {
-        float acc = partial[i];
-        for (int s = 1; s < splits; ++s) acc += partial[static_cast<size_t>(s) * total + i];
+        float acc = 0.0f;
+        for (int s0 = 0; s0 < splits; s0 += 8) {  // eight loads in flight at a time, added in split order
+            float p[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) p[k] = s0 + k < splits ? partial[static_cast<size_t>(s0 + k) * total + i] : 0.0f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (s0 + k < splits) acc = (s0 + k == 0) ? p[k] : acc + p[k];
+        }
         if (residual) acc += residual[i];
         const size_t r = i / n_out, n = i % n_out;
         y[(dst_rows ? static_cast<size_t>(dst_rows[r]) : r) * n_out + n] = acc;
