@@ -37,6 +37,29 @@ __device__ __forceinline__ float sum_partials(const float* __restrict__ partial,
     return acc;
 }
 
+// The same for two elements at once (their loads share the flight).
+__device__ __forceinline__ void sum_partials2(const float* __restrict__ partial, int splits, size_t stride, size_t i1,
+                                              size_t i2, float* out1, float* out2) {
+    float a = 0.0f, b = 0.0f;
+    for (int s0 = 0; s0 < splits; s0 += 8) {
+        float p[8], q[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const bool live = s0 + k < splits;
+            p[k] = live ? partial[static_cast<size_t>(s0 + k) * stride + i1] : 0.0f;
+            q[k] = live ? partial[static_cast<size_t>(s0 + k) * stride + i2] : 0.0f;
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (s0 + k < splits) {
+                a = (s0 + k == 0) ? p[k] : a + p[k];
+                b = (s0 + k == 0) ? q[k] : b + q[k];
+            }
+    }
+    *out1 = a;
+    *out2 = b;
+}
+
 // grid = rows, block = 128
 __global__ void embed_kernel(const void* __restrict__ tok_emb, const void* __restrict__ pos_emb, bool bf16,
                              bool add_pos, const int32_t* __restrict__ token, const int32_t* __restrict__ pos, int d,
@@ -147,8 +170,7 @@ __global__ void qkv_kernel(float* __restrict__ qkv, const float* __restrict__ pa
     float x1, x2;
     if (partial) {
         const size_t stride = static_cast<size_t>(n_rows) * width;
-        x1 = sum_partials(partial, splits, stride, at + j);
-        x2 = sum_partials(partial, splits, stride, at + j + half);
+        sum_partials2(partial, splits, stride, at + j, at + j + half, &x1, &x2);
     } else {
         x1 = qkv[at + j];
         x2 = qkv[at + j + half];
@@ -249,8 +271,13 @@ __global__ void ffn_act_kernel(const float* __restrict__ u, const float* __restr
         if (ffn == SPEC_FFN_GELU) {
             y = gelu_tanh(partial ? sum_partials(partial, splits, stride, a) : u[a]);
         } else {
-            const float gate = partial ? sum_partials(partial, splits, stride, a) : u[a];
-            const float up = partial ? sum_partials(partial, splits, stride, a + d_ff) : u[a + d_ff];
+            float gate, up;
+            if (partial) {
+                sum_partials2(partial, splits, stride, a, a + d_ff, &gate, &up);
+            } else {
+                gate = u[a];
+                up = u[a + d_ff];
+            }
             y = (ffn == SPEC_FFN_SWIGLU ? silu(gate) : gelu_tanh(gate)) * up;
         }
         if (f) f[i] = y;
