@@ -207,6 +207,22 @@ attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __r
             const KV* tile = kv_layer + pages[k0 / page_size] * page_stride + kv_head * head_stride +
                              static_cast<size_t>(k0 % page_size) * DH;
             const int in_tile = min(32, n_keys - k0);
+            // With short heads there are registers to spare: the first batch of V rows is requested
+            // together with K, so that the tile waits for memory once instead of twice.
+            constexpr bool kEarlyV = PER_LANE <= 2;
+            const KV* vt = tile + v_offset + lane * PER_LANE;
+            float v_first[kEarlyV ? kVBatch : 1][PER_LANE];
+            if (kEarlyV) {
+#pragma unroll
+                for (int jj = 0; jj < kVBatch; ++jj) {
+                    if (jj < in_tile) {
+                        KvLoad<KV>::template load_n<PER_LANE>(vt + static_cast<size_t>(jj) * DH, v_first[kEarlyV ? jj : 0]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < PER_LANE; ++i) v_first[kEarlyV ? jj : 0][i] = 0.0f;
+                    }
+                }
+            }
             // partial dot products of all 32 keys over this lane's elements ...
             float pd[32];
             const KV* kt = tile + lane * PER_LANE;
@@ -245,14 +261,16 @@ attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __r
             mx = m_new;
 #pragma unroll
             for (int i = 0; i < PER_LANE; ++i) acc[i] *= rescale;
-            const KV* vt = tile + v_offset + lane * PER_LANE;
 #pragma unroll
             for (int j0 = 0; j0 < 32; j0 += kVBatch) {
                 if (j0 < in_tile) {
                     float vv[kVBatch][PER_LANE];
 #pragma unroll
                     for (int jj = 0; jj < kVBatch; ++jj) {
-                        if (j0 + jj < in_tile) {
+                        if (kEarlyV && j0 == 0) {
+#pragma unroll
+                            for (int i = 0; i < PER_LANE; ++i) vv[jj][i] = v_first[kEarlyV ? jj : 0][i];
+                        } else if (j0 + jj < in_tile) {
                             KvLoad<KV>::template load_n<PER_LANE>(vt + static_cast<size_t>(j0 + jj) * DH, vv[jj]);
                         } else {
 #pragma unroll
