@@ -84,11 +84,12 @@ __global__ void embed_kernel(const void* __restrict__ tok_emb, const void* __res
 constexpr int kNormThreads = 1024;
 constexpr int kNormPerThread = 4;  // rows up to 16384 wide
 
-__global__ void __launch_bounds__(kNormThreads)
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS)
 norm_kernel(float* h, const float* __restrict__ partial, int splits, int n_rows, const float* __restrict__ gain,
             const int32_t* __restrict__ src_rows, int d, float eps, float* __restrict__ out,
             __nv_bfloat16* __restrict__ out_hi, __nv_bfloat16* __restrict__ out_lo) {
-    __shared__ float red[kNormThreads / 32];
+    __shared__ float red[THREADS / 32];
     pdl_trigger();
     const int r = blockIdx.x;
     const int groups = d / 4;
@@ -96,7 +97,7 @@ norm_kernel(float* h, const float* __restrict__ partial, int splits, int n_rows,
     float4 gg[kNormPerThread];
 #pragma unroll
     for (int j = 0; j < kNormPerThread; ++j) {
-        const int g = threadIdx.x + j * kNormThreads;
+        const int g = threadIdx.x + j * THREADS;
         gg[j] = g < groups ? *reinterpret_cast<const float4*>(gain + 4 * g) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     pdl_wait();
@@ -106,7 +107,7 @@ norm_kernel(float* h, const float* __restrict__ partial, int splits, int n_rows,
     float ss = 0.0f;
 #pragma unroll
     for (int j = 0; j < kNormPerThread; ++j) {
-        const int g = threadIdx.x + j * kNormThreads;
+        const int g = threadIdx.x + j * THREADS;
         v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (g < groups) {
             v[j] = *reinterpret_cast<const float4*>(h + src + 4 * g);
@@ -131,12 +132,12 @@ norm_kernel(float* h, const float* __restrict__ partial, int splits, int n_rows,
     __syncthreads();
     float total = 0.0f;
 #pragma unroll
-    for (int i = 0; i < kNormThreads / 32; ++i) total += red[i];
+    for (int i = 0; i < THREADS / 32; ++i) total += red[i];
     const float scale = rsqrtf(total / static_cast<float>(d) + eps);
     const size_t dst = static_cast<size_t>(r) * d;
 #pragma unroll
     for (int j = 0; j < kNormPerThread; ++j) {
-        const int g = threadIdx.x + j * kNormThreads;
+        const int g = threadIdx.x + j * THREADS;
         if (g < groups) {
             const float y[4] = {v[j].x * scale * gg[j].x, v[j].y * scale * gg[j].y, v[j].z * scale * gg[j].z,
                                 v[j].w * scale * gg[j].w};
@@ -313,8 +314,16 @@ int launch_norm(float* h, const float* partial, int splits, int rows_total, cons
                 cudaStream_t stream) {
     if (d % 4 || d > 4 * kNormThreads * kNormPerThread)
         return fail(SPEC_ERR_BAD_CONFIG, "norm: width %d is not a multiple of 4 or exceeds %d", d, 4 * kNormThreads * kNormPerThread);
-    return launch_pdl(norm_kernel, dim3(n_rows), dim3(kNormThreads), 0, stream, h, partial, splits, rows_total, gain,
-                      src_rows, d, eps, out, out_hi, out_lo);
+    // a thread per 128-bit group of the row where the row is narrow (fewer warps to reduce over)
+    const int groups = d / 4;
+    if (groups <= 128)
+        return launch_pdl(norm_kernel<128>, dim3(n_rows), dim3(128), 0, stream, h, partial, splits, rows_total, gain, src_rows, d,
+                          eps, out, out_hi, out_lo);
+    if (groups <= 256)
+        return launch_pdl(norm_kernel<256>, dim3(n_rows), dim3(256), 0, stream, h, partial, splits, rows_total, gain, src_rows, d,
+                          eps, out, out_hi, out_lo);
+    return launch_pdl(norm_kernel<kNormThreads>, dim3(n_rows), dim3(kNormThreads), 0, stream, h, partial, splits, rows_total,
+                      gain, src_rows, d, eps, out, out_hi, out_lo);
 }
 
 int launch_qkv(int n_heads, int n_kv_heads, int d_head, const float2* rope, const KvPool& pool, const RowMeta& rows,
