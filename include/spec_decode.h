@@ -501,6 +501,22 @@ int spec_reset(spec_ctx* ctx);
 int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* tokens, int batch, int rows, float* logits);
 int spec_truncate(spec_ctx* ctx, int which, const int32_t* lengths, int batch);
 
+/* Diagnostic for the parity tests: how the library would run the attention of a
+ * pass of model `which` over `rows` rows per sequence for `batch` sequences
+ * (Algorithm 1's parallel pass has rows = gamma + 1; a draft step has 1 or 2),
+ * `cross` != 0 for the cross-attention of an encoder-decoder block.  The choice
+ * depends on the shapes and on the context's capacities (max_len, max_src_len)
+ * only, never on the data.  plan (HOST int32 [4]) receives
+ *   plan[0]  1: the queries of a KV head are multiplied on the tensor cores
+ *               (mma.sync tf32), 0: one warp per query on the FMA pipes;
+ *   plan[1]  key slices (CTAs) per (sequence, KV head);
+ *   plan[2]  1: the slices are merged inside a thread-block cluster, 0: by a
+ *               second kernel from partial states in global memory;
+ *   plan[3]  1: K and V of a key tile share one staging buffer (tensor-core
+ *               kernel only).
+ * No device work.  Errors: SPEC_ERR_BAD_ARG, SPEC_ERR_BAD_CONFIG. */
+int spec_attention_plan(spec_ctx* ctx, int which, int batch, int rows, int cross, int* plan);
+
 /* Device time of one forward pass of model `which` over `rows` rows per
  * sequence for `batch` sequences, at the cached lengths the diagnostics above
  * have built up (the quantities c and the cost of gamma+1 parallel rows in the

@@ -101,15 +101,17 @@ class Decoder:
         positions = np.arange(start, start + len(tokens))
         return self._forward(np.asarray(tokens), positions, use_cache=True)
 
-    def forward_full(self, tokens):
-        """Cache-free: the whole sequence from position 0, nothing kept."""
+    def forward_full(self, tokens, last=None):
+        """Cache-free: the whole sequence from position 0, nothing kept.  With `last`
+        given, only the logits of the last `last` rows are formed and returned (the
+        LM head of the earlier rows is skipped; nothing else changes)."""
         saved = (self.k_cache, self.v_cache)
         self.reset()
-        out = self._forward(np.asarray(tokens), np.arange(len(tokens)), use_cache=True)
+        out = self._forward(np.asarray(tokens), np.arange(len(tokens)), use_cache=True, last=last)
         self.k_cache, self.v_cache = saved
         return out
 
-    def _forward(self, tokens, positions, use_cache):
+    def _forward(self, tokens, positions, use_cache, last=None):
         c, w = self.cfg, self.w
         H, Hkv, dh = c["n_heads"], c["n_kv_heads"], c["d_head"]
         m = len(tokens)
@@ -151,6 +153,8 @@ class Decoder:
             else:
                 raise ValueError(c["ffn"])
             h = h + f @ w[f"l{l}.w_out"].T
+        if last is not None:
+            h = h[len(tokens) - last:]
         hf = rmsnorm(h, w["ln_f"], c["rms_eps"])
         head = w["tok_emb"] if c["tied"] else w["head"]
         return hf @ head.T

@@ -575,6 +575,17 @@ class Engine:
         a = self._np.ascontiguousarray(lengths, dtype=self._np.int32)
         _check(lib().spec_truncate(self._ctx, which, a.ctypes.data, a.shape[0]))
 
+    def attention_plan(self, which, batch, rows, cross=False):
+        """How the attention of such a pass is launched (`spec_attention_plan`): dict with
+        tensor_cores, slices, cluster_merge, in_turn."""
+        h = lib()
+        h.spec_attention_plan.restype = ctypes.c_int
+        h.spec_attention_plan.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                          ctypes.POINTER(ctypes.c_int)]
+        plan = (ctypes.c_int * 4)()
+        _check(h.spec_attention_plan(self._ctx, which, batch, rows, 1 if cross else 0, plan))
+        return dict(tensor_cores=bool(plan[0]), slices=int(plan[1]), cluster_merge=bool(plan[2]), in_turn=bool(plan[3]))
+
     def time_forward(self, which, batch, rows, repeats=20):
         """Device time (ms) of one pass of model `which` over `rows` rows per sequence at
         the current cached lengths, graph-replayed `repeats` times; the caches keep their lengths."""

@@ -766,6 +766,18 @@ size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices) {
     return static_cast<size_t>(rows) * n_heads * slices * (d_head + 2);
 }
 
+// What launch_attention does for this shape: which kernel, how many key slices, whether the
+// slices merge inside a cluster (no combine kernel), whether K and V share one staging buffer.
+AttentionPlan attention_plan(const Model& m, int batch, int m_rows, int max_keys) {
+    AttentionPlan plan{};
+    plan.tensor_cores = attention_uses_mma(m, batch, m_rows, max_keys) ? 1 : 0;
+    plan.slices = attention_slices(m, batch, m_rows, max_keys);
+    plan.cluster_merge = attention_merges_in_cluster(m, batch, m_rows, max_keys) && plan.slices <= kMaxClusterSlices ? 1 : 0;
+    const int queries = (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows;
+    plan.in_turn = plan.tensor_cores && batch * m.cfg.n_kv_heads * ((queries + 15) / 16) >= 32 ? 1 : 0;
+    return plan;
+}
+
 namespace {
 
 // A launch with programmatic stream serialization and, if cluster_x > 0, clusters of

@@ -1174,6 +1174,22 @@ extern "C" int spec_truncate(spec_ctx* ctx, int which, const int32_t* lengths, i
     return SPEC_OK;
 }
 
+extern "C" int spec_attention_plan(spec_ctx* ctx, int which, int batch, int rows, int cross, int* plan) {
+    if (!ctx || !plan || which < 0 || which > 1 || batch < 1 || rows < 1)
+        return fail(SPEC_ERR_BAD_ARG, "spec_attention_plan: bad argument");
+    if (which == 1 && !ctx->has_draft) return fail(SPEC_ERR_BAD_CONFIG, "spec_attention_plan: no draft model");
+    const Model& m = ctx->model[which];
+    if (m.cfg.arch == SPEC_ARCH_BIGRAM || m.cfg.arch == SPEC_ARCH_COPY)
+        return fail(SPEC_ERR_BAD_CONFIG, "spec_attention_plan: a table or copy model has no attention");
+    if (cross && !m.t5()) return fail(SPEC_ERR_BAD_CONFIG, "spec_attention_plan: only encoder-decoder models have cross-attention");
+    const AttentionPlan p = attention_plan(m, batch, rows, cross ? ctx->rt.max_src_len : ctx->rt.max_len);
+    plan[0] = p.tensor_cores;
+    plan[1] = p.slices;
+    plan[2] = p.cluster_merge;
+    plan[3] = p.in_turn;
+    return SPEC_OK;
+}
+
 extern "C" int spec_time_forward(spec_ctx* ctx, int which, int batch, int rows, int repeats, float* ms_per_pass) {
     if (!ctx || !ms_per_pass || which < 0 || which > 1 || batch < 1 || rows < 1 || repeats < 1)
         return fail(SPEC_ERR_BAD_ARG, "spec_time_forward: bad argument");

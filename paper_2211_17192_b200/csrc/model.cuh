@@ -135,6 +135,10 @@ struct AttnSource {
 // att[r, h] = softmax(scores) V for the rows of a pass; rows of sequence b are
 // rows b*m_rows .. of the pass.  Output as fp32 and/or two bf16 terms.
 int attention_slices(const Model& m, int batch, int m_rows, int max_len);
+struct AttentionPlan {
+    int tensor_cores, slices, cluster_merge, in_turn;
+};
+AttentionPlan attention_plan(const Model& m, int batch, int m_rows, int max_keys);
 size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices);
 // (slices from attention_slices with the same batch, m_rows and max_keys, the capacity of the key set)
 int launch_attention(const Model& m, const AttnSource& src, const RowMeta& rows, int batch, int m_rows, int slices,
