@@ -517,6 +517,19 @@ int spec_truncate(spec_ctx* ctx, int which, const int32_t* lengths, int batch);
  * No device work.  Errors: SPEC_ERR_BAD_ARG, SPEC_ERR_BAD_CONFIG. */
 int spec_attention_plan(spec_ctx* ctx, int which, int batch, int rows, int cross, int* plan);
 
+/* Diagnostic: where the time of one pass goes.  Passes of at most 16 rows of a bf16
+ * decoder-only model run as one persistent kernel (one CTA per SM) whose steps (GEMMs,
+ * rotary + append, attention, merge) are separated by grid-wide barriers.  This call runs
+ * such a pass twice at the cached lengths (as spec_time_forward does; the second run is
+ * the traced one) and returns the CTAs' clocks: stamps_ns[0] is the number of CTAs P,
+ * stamps_ns[1] the start of the pass, and stamps_ns[2 + (k - 1) * P + c] the time CTA c
+ * arrived at the k-th barrier (k = 1, 2, ...), in nanoseconds of the GPU's global timer;
+ * a barrier opens when its last CTA has arrived.  *count entries are valid.  HOST buffer
+ * of `capacity` entries.  Synchronises and, unlike every other entry point, allocates and
+ * frees device memory for the stamps.
+ * Errors: SPEC_ERR_BAD_CONFIG if such a pass does not take the persistent kernel. */
+int spec_pass_trace(spec_ctx* ctx, int which, int batch, int rows, unsigned long long* stamps_ns, int capacity, int* count);
+
 /* Device time of one forward pass of model `which` over `rows` rows per
  * sequence for `batch` sequences, at the cached lengths the diagnostics above
  * have built up (the quantities c and the cost of gamma+1 parallel rows in the
@@ -539,8 +552,10 @@ int spec_time_forward(spec_ctx* ctx, int which, int batch, int rows, int repeats
  *           tile-major layout that spec_pack_weight produces, which is what
  *           the engine streams: every [128 x 64] tile of W is contiguous
  *           (tiles ordered by 128-row band, then by 64-column block; rows and
- *           columns past the matrix are zero), so that a CTA's weight stream
- *           is one sequential run of HBM.
+ *           columns past the matrix are zero; inside a tile row the eight
+ *           16-byte chunks are stored in shared-memory swizzle order, chunk c
+ *           of row r at position c ^ (r & 7)), so that a CTA's weight stream
+ *           is one sequential run of HBM and a tile is copied as it is.
  * The tensor-core path splits x into two bf16 terms and sums split-K partial
  * results in a fixed order; it needs `workspace` (device, 256-byte aligned, at
  * least spec_linear_workspace_bytes(rows, n_out, k) bytes, contents arbitrary,

@@ -586,6 +586,20 @@ class Engine:
         _check(h.spec_attention_plan(self._ctx, which, batch, rows, 1 if cross else 0, plan))
         return dict(tensor_cores=bool(plan[0]), slices=int(plan[1]), cluster_merge=bool(plan[2]), in_turn=bool(plan[3]))
 
+    def pass_trace(self, which, batch, rows, capacity=65536):
+        """The CTAs' clocks at the grid barriers of one persistent-kernel pass (`spec_pass_trace`):
+        returns (start_ns, arrivals) with arrivals a numpy int64 array [barriers, CTAs]."""
+        h = lib()
+        h.spec_pass_trace.restype = ctypes.c_int
+        h.spec_pass_trace.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_int,
+                                      ctypes.POINTER(ctypes.c_int)]
+        out = self._np.zeros(capacity, dtype=self._np.uint64)
+        count = ctypes.c_int()
+        _check(h.spec_pass_trace(self._ctx, which, batch, rows, out.ctypes.data, capacity, ctypes.byref(count)))
+        ctas = int(out[0])
+        barriers = (count.value - 2) // ctas
+        return int(out[1]), out[2:2 + barriers * ctas].astype(self._np.int64).reshape(barriers, ctas)
+
     def time_forward(self, which, batch, rows, repeats=20):
         """Device time (ms) of one pass of model `which` over `rows` rows per sequence at
         the current cached lengths, graph-replayed `repeats` times; the caches keep their lengths."""

@@ -22,59 +22,10 @@
 #include <cfloat>
 #include <cstdlib>
 
-#include "model.cuh"
+#include "attn_unit.cuh"
 
 namespace spec {
 namespace {
-
-constexpr int kMaxAttnWarps = 16;
-constexpr int kVBatch = 16;
-
-template <typename KV>
-struct KvLoad;
-
-template <>
-struct KvLoad<float> {
-    static constexpr int kVec = 4;  // elements per 16-byte load
-    __device__ static __forceinline__ void load(const float* p, float* out) {
-        const float4 t = *reinterpret_cast<const float4*>(p);
-        out[0] = t.x; out[1] = t.y; out[2] = t.z; out[3] = t.w;
-    }
-    template <int N>
-    __device__ static __forceinline__ void load_n(const float* p, float* out) {
-        if (N == 4) {
-            load(p, out);
-        } else {
-            const float2 t = *reinterpret_cast<const float2*>(p);
-            out[0] = t.x; out[1] = t.y;
-        }
-    }
-};
-
-template <>
-struct KvLoad<__nv_bfloat16> {
-    static constexpr int kVec = 8;
-    __device__ static __forceinline__ void load(const __nv_bfloat16* p, float* out) {
-        const uint4 t = *reinterpret_cast<const uint4*>(p);
-        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            out[2 * i] = __uint_as_float(w[i] << 16);
-            out[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-        }
-    }
-    template <int N>
-    __device__ static __forceinline__ void load_n(const __nv_bfloat16* p, float* out) {
-        if (N == 4) {
-            const uint2 t = *reinterpret_cast<const uint2*>(p);
-            out[0] = __uint_as_float(t.x << 16); out[1] = __uint_as_float(t.x & 0xffff0000u);
-            out[2] = __uint_as_float(t.y << 16); out[3] = __uint_as_float(t.y & 0xffff0000u);
-        } else {
-            const uint32_t t = *reinterpret_cast<const uint32_t*>(p);
-            out[0] = __uint_as_float(t << 16); out[1] = __uint_as_float(t & 0xffff0000u);
-        }
-    }
-};
 
 // ---- merging the key slices inside a thread-block cluster ---------------------
 // The CTAs of one (sequence, KV head) - one per key slice - are launched as a
@@ -159,180 +110,12 @@ attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __r
     __shared__ float share[kMaxAttnWarps][DH + 2];  // states of the warps that share a query (ks > 1)
     pdl_trigger();
     pdl_wait();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
-    const int slice = blockIdx.x, slices = gridDim.x, kv_head = blockIdx.y, b = blockIdx.z;
+    attend_slice<KV, DH, CtaSync>(qkv, q_stride, pos, seq, m_rows, n_heads, n_kv_heads, ks, kv_layer, page_table, pages_per_seq,
+                                  page_size, kv_len, bias, bias_span, bias_zero, scale, part, blockIdx.x, gridDim.x, blockIdx.y,
+                                  blockIdx.z, threadIdx.x >> 5, blockDim.x >> 5, threadIdx.x & 31, share, FUSED);
+    const int slices = gridDim.x, kv_head = blockIdx.y, b = blockIdx.z;
     const int group = n_heads / n_kv_heads;
     const int queries = group * m_rows;
-
-    // the key range of this slice: whole tiles, same for every query of the sequence
-    int seq_keys = 0;
-    if (kv_len) {
-        seq_keys = kv_len[seq[b * m_rows]];
-    } else {
-        for (int j = 0; j < m_rows; ++j) seq_keys = max(seq_keys, pos[b * m_rows + j] + 1);
-    }
-    const int tiles = (seq_keys + 31) / 32;
-    const int t0 = static_cast<int>(static_cast<long long>(tiles) * slice / slices);
-    const int t1 = static_cast<int>(static_cast<long long>(tiles) * (slice + 1) / slices);
-
-    const size_t head_stride = static_cast<size_t>(page_size) * DH;               // one head inside a page
-    const size_t page_stride = 2 * static_cast<size_t>(n_kv_heads) * head_stride;  // K block + V block
-    const size_t v_offset = static_cast<size_t>(n_kv_heads) * head_stride;
-
-    // Work unit u = (query q, sub-slice sub): with ks > 1 the ks warps q, q + queries,
-    // ... share query q and take every ks-th tile of the slice (then the block has
-    // exactly queries * ks warps and this loop runs once).
-    for (int u = warp; u < queries * ks; u += warps) {
-        const int q = u % queries, sub = u / queries;
-        const int j = q / group, head = kv_head * group + q % group;
-        const int r = b * m_rows + j;
-        const int p = pos[r];
-        const int32_t* pages = page_table + seq[r] * pages_per_seq;
-        float qv[PER_LANE];  // this lane's share of the (scaled) query
-        KvLoad<float>::template load_n<PER_LANE>(qkv + static_cast<size_t>(r) * q_stride + head * DH + lane * PER_LANE, qv);
-#pragma unroll
-        for (int i = 0; i < PER_LANE; ++i) qv[i] *= scale;
-
-        float mx = -FLT_MAX, l = 0.0f;
-        float acc[PER_LANE];
-#pragma unroll
-        for (int i = 0; i < PER_LANE; ++i) acc[i] = 0.0f;
-        // causal: positions 0..p; otherwise the sequence's key set (p < 0: inactive row, no keys)
-        const int n_keys = kv_len ? (p >= 0 ? seq_keys : 0) : p + 1;
-        const float* bias_row = bias ? bias + static_cast<size_t>(head) * bias_span + (bias_zero - p) : nullptr;
-        for (int t = t0 + sub; t < t1; t += ks) {
-            const int k0 = 32 * t;
-            if (k0 >= n_keys) break;
-            // the whole tile lives in one page
-            const KV* tile = kv_layer + pages[k0 / page_size] * page_stride + kv_head * head_stride +
-                             static_cast<size_t>(k0 % page_size) * DH;
-            const int in_tile = min(32, n_keys - k0);
-            // With short heads there are registers to spare: the first batch of V rows is requested
-            // together with K, so that the tile waits for memory once instead of twice.
-            constexpr bool kEarlyV = PER_LANE <= 2;
-            const KV* vt = tile + v_offset + lane * PER_LANE;
-            float v_first[kEarlyV ? kVBatch : 1][PER_LANE];
-            if (kEarlyV) {
-#pragma unroll
-                for (int jj = 0; jj < kVBatch; ++jj) {
-                    if (jj < in_tile) {
-                        KvLoad<KV>::template load_n<PER_LANE>(vt + static_cast<size_t>(jj) * DH, v_first[kEarlyV ? jj : 0]);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < PER_LANE; ++i) v_first[kEarlyV ? jj : 0][i] = 0.0f;
-                    }
-                }
-            }
-            // partial dot products of all 32 keys over this lane's elements ...
-            float pd[32];
-            const KV* kt = tile + lane * PER_LANE;
-#pragma unroll
-            for (int k = 0; k < 32; ++k) {
-                float kv[PER_LANE];
-                if (k < in_tile) {
-                    KvLoad<KV>::template load_n<PER_LANE>(kt + static_cast<size_t>(k) * DH, kv);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < PER_LANE; ++i) kv[i] = 0.0f;
-                }
-                float d = 0.0f;
-#pragma unroll
-                for (int i = 0; i < PER_LANE; ++i) d = fmaf(qv[i], kv[i], d);
-                pd[k] = d;
-            }
-            // ... summed over the lanes by a butterfly that halves the live values
-            // at every step: lane l ends with the full score of key l
-#pragma unroll
-            for (int step = 16; step > 0; step >>= 1) {
-                const bool upper = (lane & step) != 0;
-#pragma unroll
-                for (int i = 0; i < step; ++i) {
-                    const float keep = upper ? pd[i + step] : pd[i];
-                    const float send = upper ? pd[i] : pd[i + step];
-                    pd[i] = keep + __shfl_xor_sync(kFullMask, send, step);
-                }
-            }
-            float s = -FLT_MAX;
-            if (lane < in_tile) s = bias_row ? pd[0] + bias_row[k0 + lane] : pd[0];
-            const float m_new = fmaxf(mx, warp_max(s));
-            const float pr = lane < in_tile ? expf(s - m_new) : 0.0f;
-            const float rescale = expf(mx - m_new);
-            l = l * rescale + warp_sum(pr);
-            mx = m_new;
-#pragma unroll
-            for (int i = 0; i < PER_LANE; ++i) acc[i] *= rescale;
-#pragma unroll
-            for (int j0 = 0; j0 < 32; j0 += kVBatch) {
-                if (j0 < in_tile) {
-                    float vv[kVBatch][PER_LANE];
-#pragma unroll
-                    for (int jj = 0; jj < kVBatch; ++jj) {
-                        if (kEarlyV && j0 == 0) {
-#pragma unroll
-                            for (int i = 0; i < PER_LANE; ++i) vv[jj][i] = v_first[kEarlyV ? jj : 0][i];
-                        } else if (j0 + jj < in_tile) {
-                            KvLoad<KV>::template load_n<PER_LANE>(vt + static_cast<size_t>(j0 + jj) * DH, vv[jj]);
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < PER_LANE; ++i) vv[jj][i] = 0.0f;
-                        }
-                    }
-#pragma unroll
-                    for (int jj = 0; jj < kVBatch; ++jj) {
-                        const float pj = __shfl_sync(kFullMask, pr, j0 + jj);
-#pragma unroll
-                        for (int i = 0; i < PER_LANE; ++i) acc[i] = fmaf(pj, vv[jj][i], acc[i]);
-                    }
-                }
-            }
-        }
-        if (ks > 1 || FUSED) {  // park the state (ks > 1: warp `q` merges the ks of them below)
-            if (lane == 0) {
-                share[warp][0] = mx;
-                share[warp][1] = l;
-            }
-#pragma unroll
-            for (int i = 0; i < PER_LANE; ++i) share[warp][2 + lane * PER_LANE + i] = acc[i];
-        } else {
-            // partial state of (row r, head, slice): [max, sum, acc[DH]]
-            float* dst = part + ((static_cast<size_t>(r) * n_heads + head) * slices + slice) * (DH + 2);
-            if (lane == 0) {
-                dst[0] = mx;
-                dst[1] = l;
-            }
-#pragma unroll
-            for (int i = 0; i < PER_LANE; ++i) dst[2 + lane * PER_LANE + i] = acc[i];
-        }
-    }
-    if (ks > 1) {
-        __syncthreads();
-        if (warp < queries) {
-            const int q = warp;
-            const int j = q / group, head = kv_head * group + q % group;
-            const int r = b * m_rows + j;
-            float mm = -FLT_MAX;
-            for (int s = 0; s < ks; ++s) mm = fmaxf(mm, share[q + s * queries][0]);
-            float l = 0.0f, acc[PER_LANE];
-#pragma unroll
-            for (int i = 0; i < PER_LANE; ++i) acc[i] = 0.0f;
-            for (int s = 0; s < ks; ++s) {  // sub-slices in index order
-                const float* st = share[q + s * queries];
-                const float w = expf(st[0] - mm);
-                l += st[1] * w;
-#pragma unroll
-                for (int i = 0; i < PER_LANE; ++i) acc[i] += st[2 + lane * PER_LANE + i] * w;
-            }
-            // (warp q is the only reader of the rows it merged, so it may reuse row q)
-            float* dst = FUSED ? share[q] : part + ((static_cast<size_t>(r) * n_heads + head) * slices + slice) * (DH + 2);
-            __syncwarp();
-            if (lane == 0) {
-                dst[0] = mm;
-                dst[1] = l;
-            }
-#pragma unroll
-            for (int i = 0; i < PER_LANE; ++i) dst[2 + lane * PER_LANE + i] = acc[i];
-        }
-    }
     if (FUSED) {
         __syncthreads();
         cluster_merge_write<DH>(&share[0][0], queries, 0, queries, b, m_rows, group, kv_head, n_heads, slices, out);

@@ -31,9 +31,12 @@ struct spec_ctx {
     // tensor-core GEMM path: bf16 hi/lo copies of the GEMM input, split-K partial sums
     __nv_bfloat16 *x_hi = nullptr, *x_lo = nullptr;
     float* partials = nullptr;
+    unsigned long long* pass_trace = nullptr;  // set while spec_pass_trace runs
+    int pass_trace_capacity = 0;
     float* attn_part = nullptr;  // per key slice: (max, sum, accumulator) of every (row, head)
     int hi_rows = 0;
     bool tensor_cores = true;
+    spec::PassScratch pass;  // the persistent pass kernel's scratch (passes of at most 16 rows of a bf16 model)
     int32_t *row_token = nullptr, *row_pos = nullptr, *row_seq = nullptr, *logit_src = nullptr, *logit_dst = nullptr;
     int32_t* page_table = nullptr;
 
@@ -196,6 +199,12 @@ struct Pass {
     }
 };
 
+// Non-zero (and cleared) if a tensor-core GEMM or the persistent pass kernel gave up on a bounded wait.
+int device_gave_up(spec_ctx* ctx) {
+    const int gemm = gemm_tc_take_error(), pass = pass_take_error();
+    return gemm ? gemm : pass;
+}
+
 KvPool layer_pool(const spec_ctx* ctx, const Model& m, int layer) {
     return KvPool{static_cast<char*>(m.kv) + static_cast<size_t>(layer) * m.layer_stride, m.kv_elem_bytes, ctx->page_table,
                   ctx->pages_per_seq, ctx->rt.page_size};
@@ -223,6 +232,14 @@ int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_ro
                                                       std::max(ctx->iteration_gamma, 1), rows, logit_src, logit_dst,
                                                       n_logit_rows, c.ngram, c.vocab, logits, ctx->stream)
                                 : SPEC_OK;
+    const int which = &m == &ctx->model[1] ? 1 : 0;
+    if (ctx->tensor_cores && pass_kernel_serves(ctx->pass, m, which, n_rows, n_logit_rows)) {
+        // a few rows: the whole pass is one persistent kernel
+        const PassTables tables{ctx->page_table, ctx->pages_per_seq, ctx->rt.page_size, ctx->src_page_table,
+                                ctx->src_pages_per_seq, ctx->src_len, ctx->rt.max_len, ctx->rt.max_len - 1};
+        return launch_pass(ctx->pass, m, which, rows, tables, batch, m_rows, n_logit_rows, logit_src, logit_dst, logits, ctx->stream,
+                           ctx->pass_trace, ctx->pass_trace_capacity);
+    }
     Pass pass{ctx, m, n_rows, m.bf16() && ctx->tensor_cores, ctx->stream};
     const int d = c.d_model;
     const float* bias = m.t5() ? m.dec_bias : nullptr;
@@ -768,6 +785,8 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
             SPEC_ALLOC(partials, partial);
             cudaMemset(ctx->x_hi, 0, static_cast<size_t>(ctx->hi_rows) * max_k * 2);
             cudaMemset(ctx->x_lo, 0, static_cast<size_t>(ctx->hi_rows) * max_k * 2);
+            if ((status = pass_scratch_init(ctx->pass, ctx->model, ctx->has_draft ? 2 : 1, ctx->allocations)) != SPEC_OK)
+                return cleanup(status);
         }
     }
     SPEC_ALLOC(row_token, R);
@@ -823,6 +842,7 @@ extern "C" void spec_free(spec_ctx* ctx) {
     if (!ctx) return;
     if (ctx->stream) cudaStreamSynchronize(ctx->stream);
     drop_graphs(ctx);
+    pass_scratch_release(ctx->pass);
     for (void* p : ctx->allocations) cudaFree(p);
     for (auto& e : ctx->ev)
         if (e) cudaEventDestroy(e);
@@ -865,7 +885,7 @@ int encode_sources(spec_ctx* ctx, const int32_t* source, const int32_t* source_l
     for (int which = 0; which < n_models; ++which)
         if (ctx->model[which].t5()) SPEC_TRY(encode(ctx, ctx->model[which], batch, longest));  // (a table draft has no encoder)
     SPEC_CUDA_TRY(cudaStreamSynchronize(st));  // the host vectors go out of scope
-    if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
+    if (const int gave_up = device_gave_up(ctx)) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (code %d)", gave_up);
     ctx->encoded = true;
     ctx->encoded_batch = batch;
     return SPEC_OK;
@@ -957,7 +977,7 @@ int run_iterations(spec_ctx* ctx, int iterations, float* elapsed_ms, int* remain
     ctx->session_draft_passes += static_cast<long long>(iterations) * ctx->session_gamma;
     SPEC_CUDA_TRY(cudaMemcpyAsync(lengths.data(), ctx->length, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     SPEC_CUDA_TRY(cudaStreamSynchronize(st));
-    if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
+    if (const int gave_up = device_gave_up(ctx)) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (code %d)", gave_up);
     SPEC_CUDA_TRY(cudaEventElapsedTime(elapsed_ms, ctx->ev[1], ctx->ev[2]));
     *remaining = 0;
     for (int b = 0; b < batch; ++b)
@@ -1190,6 +1210,54 @@ extern "C" int spec_attention_plan(spec_ctx* ctx, int which, int batch, int rows
     return SPEC_OK;
 }
 
+extern "C" int spec_pass_trace(spec_ctx* ctx, int which, int batch, int rows, unsigned long long* stamps_ns, int capacity,
+                               int* count) {
+    if (!ctx || !stamps_ns || !count || capacity < 2 || which < 0 || which > 1 || batch < 1 || rows < 1)
+        return fail(SPEC_ERR_BAD_ARG, "spec_pass_trace: bad argument");
+    if (which == 1 && !ctx->has_draft) return fail(SPEC_ERR_BAD_CONFIG, "spec_pass_trace: no draft model");
+    const Model& m = ctx->model[which];
+    const int n = batch * rows;
+    if (batch > ctx->rt.max_batch || !ctx->tensor_cores || !pass_kernel_serves(ctx->pass, m, which, n, n))
+        return fail(SPEC_ERR_BAD_CONFIG, "spec_pass_trace: a pass of %d x %d rows of this model does not run as the persistent kernel", batch, rows);
+    ctx->session_batch = 0;
+    std::vector<int32_t> tok(n, 0), pos(n), seq(n);
+    for (int b = 0; b < batch; ++b) {
+        if (ctx->cached[which][b] + rows > std::min(ctx->rt.max_len, m.cfg.max_positions))
+            return fail(SPEC_ERR_CAPACITY, "spec_pass_trace: sequence %d would exceed the cache", b);
+        for (int j = 0; j < rows; ++j) {
+            pos[b * rows + j] = ctx->cached[which][b] + j;
+            seq[b * rows + j] = b;
+        }
+    }
+    cudaStream_t st = ctx->stream;
+    unsigned long long* dev = nullptr;
+    SPEC_CUDA_TRY(cudaMalloc(&dev, static_cast<size_t>(capacity) * sizeof(unsigned long long)));
+    cudaError_t err = cudaMemsetAsync(dev, 0, static_cast<size_t>(capacity) * sizeof(unsigned long long), st);
+    if (err == cudaSuccess) err = cudaMemcpyAsync(ctx->row_token, tok.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st);
+    if (err == cudaSuccess) err = cudaMemcpyAsync(ctx->row_pos, pos.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st);
+    if (err == cudaSuccess) err = cudaMemcpyAsync(ctx->row_seq, seq.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st);
+    int status = SPEC_OK;
+    if (err == cudaSuccess) {
+        status = forward(ctx, m, batch, rows, n, nullptr, nullptr, ctx->target_logits);  // untimed: warms the caches
+        ctx->pass_trace = dev;
+        ctx->pass_trace_capacity = capacity;
+        if (status == SPEC_OK) status = forward(ctx, m, batch, rows, n, nullptr, nullptr, ctx->target_logits);
+        ctx->pass_trace = nullptr;
+        ctx->pass_trace_capacity = 0;
+    }
+    if (err == cudaSuccess) err = cudaMemcpyAsync(stamps_ns, dev, static_cast<size_t>(capacity) * sizeof(unsigned long long), cudaMemcpyDeviceToHost, st);
+    if (err == cudaSuccess) err = cudaStreamSynchronize(st);
+    cudaFree(dev);
+    SPEC_CUDA_TRY(err);
+    if (status != SPEC_OK) return status;
+    if (const int gave_up = device_gave_up(ctx)) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (code %d)", gave_up);
+    int used = 0;
+    for (int i = 0; i < capacity; ++i)
+        if (stamps_ns[i]) used = i + 1;
+    *count = used;
+    return SPEC_OK;
+}
+
 extern "C" int spec_time_forward(spec_ctx* ctx, int which, int batch, int rows, int repeats, float* ms_per_pass) {
     if (!ctx || !ms_per_pass || which < 0 || which > 1 || batch < 1 || rows < 1 || repeats < 1)
         return fail(SPEC_ERR_BAD_ARG, "spec_time_forward: bad argument");
@@ -1235,7 +1303,7 @@ extern "C" int spec_time_forward(spec_ctx* ctx, int which, int batch, int rows, 
     if (err == cudaSuccess) err = cudaStreamSynchronize(st);
     cudaGraphExecDestroy(exec);
     SPEC_CUDA_TRY(err);
-    if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
+    if (const int gave_up = device_gave_up(ctx)) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (code %d)", gave_up);
     float ms = 0.0f;
     SPEC_CUDA_TRY(cudaEventElapsedTime(&ms, ctx->ev[1], ctx->ev[2]));
     *ms_per_pass = ms / static_cast<float>(repeats);
@@ -1273,7 +1341,7 @@ extern "C" int spec_forward_logits(spec_ctx* ctx, int which, const int32_t* toke
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->row_seq, seq.data(), n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SPEC_TRY(forward(ctx, m, batch, rows, n, nullptr, nullptr, logits));
     SPEC_CUDA_TRY(cudaStreamSynchronize(st));
-    if (gemm_tc_take_error()) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a tensor-core GEMM gave up on a bounded wait");
+    if (const int gave_up = device_gave_up(ctx)) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (code %d)", gave_up);
     for (int b = 0; b < batch; ++b) ctx->cached[which][b] += rows;
     return SPEC_OK;
 }

@@ -264,8 +264,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
 // Tile-major copy of a row-major bf16 matrix W [n_out, k]: tile (t, kb) holds rows
 // t*128 .. t*128+127, columns kb*64 .. kb*64+63 as 128 consecutive 128-byte rows,
-// tiles ordered (t, kb); rows and columns past the matrix are zero.  One 16-byte
-// vector (8 elements) per thread.
+// tiles ordered (t, kb); rows and columns past the matrix are zero.  Inside a row
+// the eight 16-byte chunks are stored in the order of the 128-byte shared-memory
+// swizzle (chunk c of row r sits at position c ^ (r & 7)), so that a plain copy of
+// the 16 KB tile to a 1024-byte aligned address is the layout the MMA's operand
+// descriptor expects.  One 16-byte vector (8 elements) per thread.
 __global__ void pack_weight_kernel(const __nv_bfloat16* __restrict__ w, int n_out, int k, int k_blocks, size_t vectors,
                                    __nv_bfloat16* __restrict__ out) {
     for (size_t v = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; v < vectors;
@@ -274,7 +277,7 @@ __global__ void pack_weight_kernel(const __nv_bfloat16* __restrict__ w, int n_ou
         const int within = static_cast<int>(v % (kTileM * kTileK / 8));
         const int r = within / (kTileK / 8), c8 = within % (kTileK / 8);
         const int row = static_cast<int>(tile_index / k_blocks) * kTileM + r;
-        const int col = static_cast<int>(tile_index % k_blocks) * kTileK + c8 * 8;
+        const int col = static_cast<int>(tile_index % k_blocks) * kTileK + (c8 ^ (r & 7)) * 8;
         uint4 val = make_uint4(0u, 0u, 0u, 0u);
         if (row < n_out && col < k) val = *reinterpret_cast<const uint4*>(w + static_cast<size_t>(row) * k + col);
         *reinterpret_cast<uint4*>(out + v * 8) = val;
@@ -341,8 +344,9 @@ EncodeFn encode_fn() {
     return fn;
 }
 
-// A bf16 matrix [rows, cols] row-major, fetched in boxes of [box_rows, 64] with 128-byte swizzle.
-int make_map(const void* base, int rows, int cols, int box_rows, CUtensorMap* out) {
+// A bf16 matrix [rows, cols] row-major, fetched in boxes of [box_rows, 64], with the 128-byte
+// swizzle applied on the way in unless the data is stored swizzled already.
+int make_map(const void* base, int rows, int cols, int box_rows, bool swizzle, CUtensorMap* out) {
     EncodeFn fn = encode_fn();
     if (!fn) return fail(SPEC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
@@ -350,7 +354,8 @@ int make_map(const void* base, int rows, int cols, int box_rows, CUtensorMap* ou
     const cuuint32_t box[2] = {kTileK, static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t elem[2] = {1, 1};
     const CUresult res = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (res != CUDA_SUCCESS) return fail(SPEC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", static_cast<int>(res));
     return SPEC_OK;
@@ -358,22 +363,22 @@ int make_map(const void* base, int rows, int cols, int box_rows, CUtensorMap* ou
 
 struct MapKey {
     const void* base;
-    int rows, cols, box_rows;
+    int rows, cols, box_rows, swizzle;
     bool operator<(const MapKey& o) const {
-        return std::tie(base, rows, cols, box_rows) < std::tie(o.base, o.rows, o.cols, o.box_rows);
+        return std::tie(base, rows, cols, box_rows, swizzle) < std::tie(o.base, o.rows, o.cols, o.box_rows, o.swizzle);
     }
 };
 
 // Tensor maps are pure functions of (address, shape, box): cached process-wide.
-int cached_map(const void* base, int rows, int cols, int box_rows, CUtensorMap* out) {
+int cached_map(const void* base, int rows, int cols, int box_rows, bool swizzle, CUtensorMap* out) {
     static std::mutex mu;
     static std::map<MapKey, CUtensorMap> cache;
     std::lock_guard<std::mutex> lock(mu);
-    const MapKey key{base, rows, cols, box_rows};
+    const MapKey key{base, rows, cols, box_rows, swizzle ? 1 : 0};
     auto it = cache.find(key);
     if (it == cache.end()) {
         CUtensorMap m;
-        const int status = make_map(base, rows, cols, box_rows, &m);
+        const int status = make_map(base, rows, cols, box_rows, swizzle, &m);
         if (status != SPEC_OK) return status;
         it = cache.emplace(key, m).first;
     }
@@ -469,9 +474,11 @@ int launch_gemm_tc_partials(const __nv_bfloat16* hi, const __nv_bfloat16* lo, in
     CUtensorMap mw, mhi, mlo;
     const int tiles = (n_out + kTileM - 1) / kTileM;
     // tile-major weights are one long [tiles * k_blocks * 128, 64] matrix of 128-byte rows
-    int status = packed ? cached_map(w, tiles * k_blocks * kTileM, kTileK, kTileM, &mw) : cached_map(w, n_out, k, kTileM, &mw);
-    if (status == SPEC_OK) status = cached_map(hi, hi_rows, k, n_tok, &mhi);
-    if (status == SPEC_OK) status = cached_map(lo, hi_rows, k, n_tok, &mlo);
+    // (stored swizzled already: copied as they are)
+    int status = packed ? cached_map(w, tiles * k_blocks * kTileM, kTileK, kTileM, false, &mw)
+                        : cached_map(w, n_out, k, kTileM, true, &mw);
+    if (status == SPEC_OK) status = cached_map(hi, hi_rows, k, n_tok, true, &mhi);
+    if (status == SPEC_OK) status = cached_map(lo, hi_rows, k, n_tok, true, &mlo);
     if (status != SPEC_OK) return status;
     const int pk = packed ? 1 : 0;
     switch (n_tok) {
@@ -580,4 +587,7 @@ extern "C" int spec_pack_weight(const void* w, int n_out, int k, void* packed, v
     return launch_pack_weight(w, n_out, k, packed, static_cast<cudaStream_t>(stream));
 }
 
-extern "C" int spec_device_error(void) { return spec::gemm_tc_take_error(); }
+extern "C" int spec_device_error(void) {
+    const int gemm = spec::gemm_tc_take_error(), pass = spec::pass_take_error();
+    return gemm ? gemm : pass;
+}

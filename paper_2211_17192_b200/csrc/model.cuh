@@ -148,6 +148,34 @@ int launch_attention(const Model& m, const AttnSource& src, const RowMeta& rows,
 int launch_ffn_act(const float* u, const float* partial, int splits, int n_rows, int d_ff, int ffn, float* f,
                    __nv_bfloat16* f_hi, __nv_bfloat16* f_lo, cudaStream_t stream);
 
+// mega.cu: one forward pass over at most 16 rows as one persistent cooperative kernel
+// (bf16 decoder-only models).
+struct PassScratch {
+    float *h[2] = {nullptr, nullptr}, *ssq[2] = {nullptr, nullptr}, *part[2] = {nullptr, nullptr};
+    float *q = nullptr, *att = nullptr, *attn_part = nullptr;
+    unsigned* sync = nullptr;
+    void* layers[2] = {nullptr, nullptr};  // per model: device array of its blocks' pointers (nullptr: not served)
+    void* tile_counts[2] = {nullptr, nullptr};  // per model: parts per tile of every GEMM kind (bytes)
+    int count_offset[2][7] = {};
+    int count_total[2] = {0, 0};
+    int ctas = 0;                          // 0: the kernel is not available
+};
+struct PassTables {
+    const int32_t* page_table;
+    int pages_per_seq, page_size;
+    const int32_t* src_page_table;
+    int src_pages_per_seq;
+    const int32_t* src_len;
+    int bias_span, bias_zero;
+};
+int pass_scratch_init(PassScratch& s, const Model* models, int n_models, std::vector<void*>& allocations);
+bool pass_kernel_serves(const PassScratch& s, const Model& m, int which, int n_rows, int n_logit_rows);
+int launch_pass(const PassScratch& s, const Model& m, int which, const RowMeta& rows, const PassTables& t, int batch, int m_rows,
+                int n_logit_rows, const int32_t* logit_src, const int32_t* logit_dst, float* logits, cudaStream_t stream,
+                unsigned long long* trace = nullptr, int trace_capacity = 0);
+void pass_scratch_release(PassScratch& s);
+int pass_take_error();
+
 // sampling.cu
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
                          const float* uniforms, const float* final_uniforms, int batch, int gamma, int vocab,
