@@ -331,6 +331,11 @@ typedef struct spec_runtime_cfg {
                              bf16 halves the KV traffic but rounds every cached row to 8 mantissa
                              bits, which on deep models moves logits by more than 2e-2. */
     int max_src_len;      /* T5: longest source the encoders are given (0 for decoder-only models) */
+    int pass_kernel;      /* 0 (default): every pass is a chain of kernels.  1: passes of at most 16 rows of
+                             a bf16 GPT- or Llama-shaped model run as one persistent cooperative kernel
+                             (one CTA per SM, grid-wide barriers between the steps, weights streamed
+                             ahead of the steps that wait); same results within the parity tolerances,
+                             measured slower than the chain on a B200 (see spec_pass_trace). */
 } spec_runtime_cfg;
 
 typedef struct spec_ctx spec_ctx;

@@ -321,7 +321,7 @@ class _Weights(ctypes.Structure):
 
 class _RuntimeCfg(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("max_batch", "max_len", "page_size", "max_gamma", "kv_dtype",
-                                            "max_src_len")]
+                                            "max_src_len", "pass_kernel")]
 
 
 class _Stats(ctypes.Structure):
@@ -396,7 +396,7 @@ class Engine:
     """
 
     def __init__(self, target_cfg, target_weights, draft_cfg=None, draft_weights=None, max_batch=1, max_len=256,
-                 page_size=64, max_gamma=8, kv_dtype="fp32", device=None, max_src_len=0):
+                 page_size=64, max_gamma=8, kv_dtype="fp32", device=None, max_src_len=0, pass_kernel=False):
         import numpy as np
         self._np = np
         h = lib()
@@ -407,7 +407,7 @@ class Engine:
         structs = []
         for cfg, weights in ((target_cfg, target_weights), (draft_cfg, draft_weights)):
             structs.append(None if cfg is None else self._upload(cfg, weights))
-        rt = _RuntimeCfg(max_batch, max_len, page_size, max_gamma, _DTYPE[kv_dtype], max_src_len)
+        rt = _RuntimeCfg(max_batch, max_len, page_size, max_gamma, _DTYPE[kv_dtype], max_src_len, 1 if pass_kernel else 0)
         self.max_batch, self.max_len, self.max_gamma = max_batch, max_len, max_gamma
         ctx = ctypes.c_void_p()
         tc = _cfg_struct(target_cfg)

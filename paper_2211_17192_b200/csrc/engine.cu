@@ -233,7 +233,7 @@ int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_ro
                                                       n_logit_rows, c.ngram, c.vocab, logits, ctx->stream)
                                 : SPEC_OK;
     const int which = &m == &ctx->model[1] ? 1 : 0;
-    if (ctx->tensor_cores && pass_kernel_serves(ctx->pass, m, which, n_rows, n_logit_rows)) {
+    if (ctx->rt.pass_kernel && ctx->tensor_cores && pass_kernel_serves(ctx->pass, m, which, n_rows, n_logit_rows)) {
         // a few rows: the whole pass is one persistent kernel
         const PassTables tables{ctx->page_table, ctx->pages_per_seq, ctx->rt.page_size, ctx->src_page_table,
                                 ctx->src_pages_per_seq, ctx->src_len, ctx->rt.max_len, ctx->rt.max_len - 1};
@@ -683,7 +683,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     const spec_runtime_cfg& rt = *runtime;
     if (rt.max_batch < 1 || rt.max_batch > 4096 || rt.max_len < 2 || rt.max_gamma < 0 || rt.max_gamma > 64 ||
         rt.page_size < 32 || rt.page_size > 256 || (rt.page_size & (rt.page_size - 1)) ||
-        (rt.kv_dtype != SPEC_DTYPE_FP32 && rt.kv_dtype != SPEC_DTYPE_BF16))
+        (rt.kv_dtype != SPEC_DTYPE_FP32 && rt.kv_dtype != SPEC_DTYPE_BF16) || (rt.pass_kernel != 0 && rt.pass_kernel != 1))
         return fail(SPEC_ERR_BAD_CONFIG, "spec_init: runtime config out of range");
     int device_count = 0;
     if (cudaGetDeviceCount(&device_count) != cudaSuccess || device_count == 0) {
@@ -785,7 +785,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
             SPEC_ALLOC(partials, partial);
             cudaMemset(ctx->x_hi, 0, static_cast<size_t>(ctx->hi_rows) * max_k * 2);
             cudaMemset(ctx->x_lo, 0, static_cast<size_t>(ctx->hi_rows) * max_k * 2);
-            if ((status = pass_scratch_init(ctx->pass, ctx->model, ctx->has_draft ? 2 : 1, ctx->allocations)) != SPEC_OK)
+            if (rt.pass_kernel && (status = pass_scratch_init(ctx->pass, ctx->model, ctx->has_draft ? 2 : 1, ctx->allocations)) != SPEC_OK)
                 return cleanup(status);
         }
     }
@@ -1217,7 +1217,9 @@ extern "C" int spec_pass_trace(spec_ctx* ctx, int which, int batch, int rows, un
     if (which == 1 && !ctx->has_draft) return fail(SPEC_ERR_BAD_CONFIG, "spec_pass_trace: no draft model");
     const Model& m = ctx->model[which];
     const int n = batch * rows;
-    if (batch > ctx->rt.max_batch || !ctx->tensor_cores || !pass_kernel_serves(ctx->pass, m, which, n, n))
+    if (batch > ctx->rt.max_batch || n > ctx->max_logit_rows)
+        return fail(SPEC_ERR_CAPACITY, "spec_pass_trace: %d x %d rows exceed the workspace (%d rows)", batch, rows, ctx->max_logit_rows);
+    if (!ctx->rt.pass_kernel || !ctx->tensor_cores || !pass_kernel_serves(ctx->pass, m, which, n, n))
         return fail(SPEC_ERR_BAD_CONFIG, "spec_pass_trace: a pass of %d x %d rows of this model does not run as the persistent kernel", batch, rows);
     ctx->session_batch = 0;
     std::vector<int32_t> tok(n, 0), pos(n), seq(n);

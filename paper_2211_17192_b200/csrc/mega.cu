@@ -1,10 +1,10 @@
-// One forward pass over a few rows as ONE persistent kernel.
+// One forward pass over a few rows as ONE persistent kernel (an option of the context:
+// spec_runtime_cfg::pass_kernel; the chain of kernels in engine.cu is the default, see below).
 //
 // A decoding pass over gamma + 1 rows is a stream of weights (Section 3.4: the rows share
 // one read of every matrix) interrupted by short dependent steps: normalisation, rotary
-// positions, attention, the activation.  Launched as a chain of kernels, every one of those
-// steps leaves HBM idle while it runs and while the next GEMM fills its pipeline.  Here the
-// whole pass is one cooperative kernel with one CTA per SM:
+// positions, attention, the activation.  Here the whole pass is one cooperative kernel with
+// one CTA per SM:
 //
 //   * warp 0 streams weight tiles with bulk copies into a ring of shared-memory stages.  It
 //     depends on nothing but free stages, so it runs ahead through every dependent step
@@ -14,23 +14,31 @@
 //     of a matrix, in the tile-major order in which they are stored, are dealt out in
 //     equal contiguous runs, one per CTA, so that every SM streams the same number of
 //     bytes of every matrix whatever its shape.  A run covers parts of one to three
-//     tiles; each part is accumulated in tensor memory (tcgen05.mma, M 128 x N 16) and
-//     written as a partial sum; the consumer adds the parts of a tile in CTA order.
-//   * the activation operand of a GEMM is built by its consumer: a few warps of every CTA
-//     form the 16 x 64 block that goes with a weight tile straight from the producer's
-//     results (residual stream + partial sums, times the norm gain; attention output;
-//     gated activation of the FFN-in partial sums), split it into two bf16 terms and
-//     store it in the MMA's swizzled layout.  RMSNorm's row scale is applied by whoever
-//     consumes the GEMM (W (s x) = s (W x)), so no step waits for a row reduction.
-//   * between dependent steps there is one grid-wide barrier (a counter in global
-//     memory); steps: qkv GEMM | rotary + K,V append | attention | slice merge | out
-//     projection | FFN-in | FFN-out, and at the end LM head | logits.
+//     tiles; each part is accumulated in tensor memory (tcgen05.mma, M 128 x N 16).  A
+//     tile with one part is finished by its CTA; otherwise the parts go to global memory
+//     and the CTA that writes the last one (a counter per tile) adds them up in CTA order.
+//   * the activation operand of a GEMM is built by its consumer: eight warps of every CTA
+//     form the 16 x 64 block that goes with a weight tile from the step before (residual
+//     stream times the norm gain; attention output; gated activation of the FFN-in
+//     rows), split it into two bf16 terms and store it in the MMA's swizzled layout.
+//     RMSNorm's row scale is applied by whoever consumes the GEMM (W (s x) = s (W x)); the
+//     sums of squares come from the CTAs that finish the tiles of the residual stream.
+//   * between dependent steps there is one grid-wide barrier (a counter in global memory
+//     that is never reset); steps per block: qkv GEMM | rotary + K,V append | attention |
+//     slice merge | out-projection | FFN-in | FFN-out; at the end the LM head, whose
+//     finished tiles are the logits.
 //
 // Every wait (mbarrier, grid barrier) is bounded; on expiry the kernel records an error,
 // tells the other CTAs, waits for its own copies in flight, frees its tensor memory and
 // returns.
+//
+// Measured on a B200 (7B-shaped blocks, 3 rows, 1024 cached tokens): the weight stream alone
+// runs at the HBM copy rate, but every step pays about two microseconds of barrier and two
+// to four of start-up and finish (operand load, part count, part re-read: each a round
+// trip to L2), seven times per block: 109 us per block against 88 us for the kernel chain,
+// and more on small models whose steps move almost no bytes.  Hence an option, not the
+// default.
 #include <algorithm>
-#include <cstdlib>
 #include <mutex>
 #include <vector>
 
@@ -66,10 +74,10 @@ struct Smem {
     static constexpr int kRing = kStages * kStageBytes;
     static constexpr int kBars = kRing;                                // wfull, bfull, empty [kStages]; acc_full, acc_empty [2]
     static constexpr int kTmemSlot = kBars + (3 * kStages + 4) * 8;
-    static constexpr int kAbort = kTmemSlot + 4;                      // abort flag, then the barrier's verdict
-    static constexpr int kScale = kAbort + 8;                         // row scales [16]
-    static constexpr int kRowPos = kScale + 16 * 4;                   // the rows' positions, sequence slots; key count per sequence
-    static constexpr int kShare = (kRowPos + 3 * 16 * 4 + 15) / 16 * 16;  // attention states, one per worker warp
+    static constexpr int kAbort = kTmemSlot + 4;                      // abort flag, the barrier's verdict, the epilogue's "last part" flag
+    static constexpr int kScale = kAbort + 12;                        // row scales [16]
+    static constexpr int kRowPos = kScale + 16 * 4;                   // per row: position, sequence slot, (per sequence) key count, token, logits row
+    static constexpr int kShare = (kRowPos + 5 * 16 * 4 + 15) / 16 * 16;  // attention states, one per worker warp
     static constexpr int kCounts = kShare + kWorkers * (128 + 2) * 4;     // parts per tile of every GEMM shape
     static constexpr int kTotal = kCounts + kMaxTileCounts + 1024 /* alignment slack */;
 };
@@ -194,6 +202,13 @@ __device__ __forceinline__ float ld_f1(const float* p) {
     return v;
 }
 
+// (past L1: for values that another SM wrote during this phase)
+__device__ __forceinline__ float ld_cg_f1(const float* p) {
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+
 // ---- what the kernel is given --------------------------------------------------
 struct MegaLayer {
     const float *ln1, *ln2, *lnx;
@@ -223,15 +238,16 @@ struct MegaArgs {
     int n_rows, m_rows, batch;
     const int32_t *row_token, *row_pos, *row_seq;
     int n_logit_rows;
-    const int32_t *logit_src, *logit_dst;
+    const int32_t *logit_src, *logit_dst;  // (distinct source rows)
     float* logits;
     // scratch
-    float* h[2];      // residual stream [16][d], two copies used in turn
-    float* ssq[2];    // per 64-column block of a row: sum of squares [k_blocks][16]
-    float* part[2];   // partial sums of the GEMMs, used in turn
-    float* q;         // q rows (and nothing else) [16][n_heads * dh]
+    float* h;         // residual stream [16][d]
+    float* ssq[2];    // sums of squares of the stream's rows per 32-column group [d / 32][16], used in turn
+    float* part[2];   // partial sums of the GEMMs' tiles, used in turn
+    float* out;       // output of the GEMM before (projection rows, FFN-in rows) [16][n_out]
     float* att;       // attention output [16][n_heads * dh]
     float* attn_part; // per key slice: (max, sum, accumulator) of every (row, head)
+    unsigned* ticket[2];  // per tile: parts written so far (back to zero once the tile is finished)
     unsigned* sync;   // [0..1] the grid barrier's 64-bit arrival count, [2] the give-up flag
     // parts per tile of every GEMM shape of the model (bytes, made on the host): offsets by kind
     // 0 qkv, 1 out-projection, 2 cross q, 3 cross out-projection, 4 FFN-in, 5 FFN-out, 6 LM head
@@ -275,9 +291,7 @@ __device__ __forceinline__ GemmDesc gemm_desc(const MegaArgs& a, int g) {
     const int q_dim = a.n_heads * a.dh, kv_dim = a.n_kv_heads * a.dh;
     if (g >= per * a.n_layers) return make_desc(a.head, a.vocab, a.d);
     const MegaLayer& L = a.layers[g / per];
-    int which = g % per;
-    if (a.arch != SPEC_ARCH_T5 && which >= 2) which += 2;
-    switch (which) {
+    switch (gemm_kind(a, g)) {
         case 0: return make_desc(L.wqkv, q_dim + 2 * kv_dim, a.d);
         case 1: return make_desc(L.wo, a.d, q_dim);
         case 2: return make_desc(L.wq_x, q_dim, a.d);
@@ -297,22 +311,6 @@ __host__ __device__ __forceinline__ int cta_of_unit(unsigned units, unsigned u, 
     return c;
 }
 
-// Partial sums of a GEMM: for tile t the part of CTA c is slot j = c - first(t), first(t) the CTA
-// that owns the tile's first unit; [(t * jmax + j) * 16 + row][128 features].  (A matrix with
-// fewer units than CTAs gives a CTA one unit or none: then slot j is the tile's j-th unit.)
-struct TileParts {
-    const float* base;  // part 0, row 0, feature 0 of the tile; parts are 16 * 128 floats apart
-    int count;
-};
-struct PartialView {
-    const float* base;
-    const uint8_t* counts;  // parts per tile (shared memory)
-    int jmax;
-    __device__ __forceinline__ TileParts tile(int t) const {
-        return TileParts{base + static_cast<size_t>(t) * jmax * (kMaxRows * 128), counts[t]};
-    }
-};
-
 // The most CTAs that contribute to one tile: a tile's kbn units meet runs of per = units / P
 // (or one more) units.
 __host__ __device__ inline int max_contributors(unsigned units, int kbn, int P) {
@@ -321,50 +319,28 @@ __host__ __device__ inline int max_contributors(unsigned units, int kbn, int P) 
     return static_cast<int>((kbn + per - 2) / per + 1);
 }
 
-__device__ __forceinline__ PartialView partial_view(const MegaArgs& a, int g, int P, const uint8_t* counts_sh) {
-    const GemmDesc gd = gemm_desc(a, g);
-    PartialView v;
-    v.base = a.part[g & 1];
-    v.counts = counts_sh + a.count_offset[gemm_kind(a, g)];
-    v.jmax = max_contributors(gd.units, gd.kbn, P);
-    return v;
-}
-
-// sum of a column pair (features off, off + 1 of the tile) over the tile's parts, in CTA order
-__device__ __forceinline__ float2 sum_parts2(const TileParts& tp, int off, int row) {
-    const float* p0 = tp.base + row * 128 + off;
-    float2 acc = *reinterpret_cast<const float2*>(p0);
-    for (int j = 1; j < tp.count; ++j) {
-        const float2 p = *reinterpret_cast<const float2*>(p0 + static_cast<size_t>(j) * (kMaxRows * 128));
-        acc.x += p.x;
-        acc.y += p.y;
-    }
-    return acc;
-}
-
 __device__ __forceinline__ float gelu_tanh(float x) {
     const float k = 0.7978845608028654f;
     return 0.5f * x * (1.0f + tanhf(k * (x + 0.044715f * x * x * x)));
 }
 __device__ __forceinline__ float silu(float x) { return x / (1.0f + expf(-x)); }
 
-// RMSNorm's scale of a row from the per-block sums of squares (every warp that needs it
-// evaluates the same expression on the same values).
-// This lane's share of a row's sum of squares: blocks lane, lane + 32, ..., four loads in flight.
-__device__ __forceinline__ float row_ssq_share(const float* ssq, int kbn, int row, int lane) {
+// RMSNorm's scale of a row from the sums of squares of its 32-column groups (every warp that needs
+// it evaluates the same expression on the same values): this lane's share, four loads in flight.
+__device__ __forceinline__ float row_ssq_share(const float* ssq, int groups, int row, int lane) {
     float s = 0.0f;
-    for (int kb0 = lane; kb0 < kbn; kb0 += 128) {
+    for (int g0 = lane; g0 < groups; g0 += 128) {
         float v[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) v[i] = ld_f1(ssq + min(kb0 + 32 * i, kbn - 1) * kMaxRows + row);
+        for (int i = 0; i < 4; ++i) v[i] = ld_f1(ssq + min(g0 + 32 * i, groups - 1) * kMaxRows + row);
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            if (kb0 + 32 * i < kbn) s += v[i];
+            if (g0 + 32 * i < groups) s += v[i];
     }
     return s;
 }
-__device__ __forceinline__ float row_scale(const float* ssq, int kbn, int row, int d, float eps, int lane) {
-    return rsqrtf(warp_sum(row_ssq_share(ssq, kbn, row, lane)) / static_cast<float>(d) + eps);
+__device__ __forceinline__ float row_scale(const float* ssq, int groups, int row, int d, float eps, int lane) {
+    return rsqrtf(warp_sum(row_ssq_share(ssq, groups, row, lane)) / static_cast<float>(d) + eps);
 }
 
 // Per-thread view of the kernel's shared state.
@@ -373,9 +349,10 @@ struct Cta {
     uint64_t *wfull, *bfull, *empty, *acc_full, *acc_empty;
     volatile int* abort_flag;
     volatile int* verdict;  // written by one thread inside the grid barrier: 1 = carry on, 0 = unwind
+    volatile int* last;     // written by one epilogue thread: 1 = this CTA wrote a tile's last part
     float* scale;
-    const int *row_pos, *row_seq, *seq_keys;  // shared-memory copies: per row, per row, per sequence of the pass
-    const uint8_t* counts;                    // shared-memory copy of MegaArgs::tile_counts
+    const int *row_pos, *row_seq, *seq_keys, *row_tok, *row_logit;  // shared-memory copies: per row / per sequence of the pass
+    const uint8_t* counts;  // shared-memory copy of MegaArgs::tile_counts
     uint32_t tmem;
     int c, P;         // this CTA, CTAs
     unsigned n;       // units this CTA has been through (all GEMMs so far)
@@ -383,7 +360,8 @@ struct Cta {
     int barriers;     // grid barriers this CTA has been through
 };
 
-enum Source { kSrcEmbed, kSrcResid, kSrcPlain, kSrcAct };
+enum Source { kSrcNorm, kSrcPlain, kSrcAct };
+enum Sink { kSinkRows, kSinkStream, kSinkLogits };
 
 // Grid-wide barrier of everybody but the weight producers.
 __device__ __forceinline__ unsigned long long global_ns() {
@@ -474,14 +452,11 @@ __device__ void produce_weights(const MegaArgs& a, Cta& cta) {
 // swizzled K-major layout of the MMA's N side.
 struct BuildCtx {
     Source src;
-    int k_total;                 // inner dimension of this GEMM
-    const float* gain;           // norm gain (embed / resid)
-    const float* h_in;           // resid: residual stream before the update
-    float* h_out;                // embed / resid: updated residual stream (written by the tile-0 units)
-    float* ssq_out;
-    const float* ssq_in;         // act: the sums of squares that go with the FFN-in GEMM's operand
-    PartialView prev;            // resid / act: the producer GEMM's partial sums
-    const float* plain;          // plain: fp32 rows [16][k_total]
+    int k_total;        // inner dimension of this GEMM
+    const float* gain;  // norm: the gain; the row scale is left to whoever consumes the GEMM
+    const float* rows;  // norm: the residual stream [16][k_total]; plain: fp32 rows [16][k_total];
+                        // act: the FFN-in rows [16][d_ff or 2 d_ff]
+    const float* ssq;   // act: the sums of squares that go with the FFN-in GEMM's operand
 };
 
 __device__ __forceinline__ void store_pair(uint8_t* stage, int row, int lane, float x0, float x1) {
@@ -498,136 +473,54 @@ __device__ __forceinline__ void store_pair(uint8_t* stage, int row, int lane, fl
 
 constexpr int kRowBatch = 4;  // rows of a block whose loads are requested together
 
-// Parts j0 .. j0 + N - 1 of a column pair of one row, requested together.  Every load is
-// unconditional (an index past the last part re-reads the last part; the sum skips it): a load
-// whose result feeds a select would make the thread wait for it before it requests the next one.
-template <int N>
-__device__ __forceinline__ void load_parts(const TileParts& tp, int off, int row, int j0, float2 (&p)[N]) {
-    const float* p0 = tp.base + row * 128 + off;
-#pragma unroll
-    for (int j = 0; j < N; ++j)
-        p[j] = ld_f2(p0 + static_cast<size_t>(min(j0 + j, tp.count - 1)) * (kMaxRows * 128));
-}
-// their sum in part order, continued over the parts beyond the first N (rare: many CTAs on one tile)
-template <int N>
-__device__ __forceinline__ float2 sum_loaded(const TileParts& tp, int off, int row, const float2 (&p)[N]) {
-    float2 acc = p[0];
-#pragma unroll
-    for (int j = 1; j < N; ++j)
-        if (j < tp.count) {
-            acc.x += p[j].x;
-            acc.y += p[j].y;
-        }
-    for (int j0 = N; j0 < tp.count; j0 += N) {
-        float2 more[N];
-        load_parts<N>(tp, off, row, j0, more);
-#pragma unroll
-        for (int j = 0; j < N; ++j)
-            if (j0 + j < tp.count) {
-                acc.x += more[j].x;
-                acc.y += more[j].y;
-            }
-    }
-    return acc;
-}
-
 template <int SRC>
-__device__ __forceinline__ void build_block(const MegaArgs& a, const Cta& cta, const BuildCtx& b, uint8_t* stage, int tile, int kb,
-                                            int lane) {
-    constexpr int PB = SRC == kSrcAct ? 4 : 8;      // parts in flight per row and tile
-    constexpr int UP = SRC == kSrcAct ? PB : 1;
+__device__ __forceinline__ void build_block(const MegaArgs& a, const Cta& cta, const BuildCtx& b, uint8_t* stage, int kb, int lane) {
     const int col = kb * 64 + 2 * lane;
-    const bool live = col < b.k_total;
-    const bool writer = tile == 0 && (SRC == kSrcEmbed || SRC == kSrcResid);
+    const bool live = col < b.k_total;  // (columns past the matrix meet zero weights: they must be finite, so zero)
     const bool gated = SRC == kSrcAct && a.ffn != SPEC_FFN_GELU;
-    float2 gain = make_float2(0.f, 0.f);
-    if (live && b.gain) gain = *reinterpret_cast<const float2*>(b.gain + col);
-    // the parts of the producer's tile(s) this lane's columns come from
-    TileParts tp{nullptr, 0}, tp_up{nullptr, 0};
-    if (live && (SRC == kSrcResid || SRC == kSrcAct)) tp = b.prev.tile(col >> 7);
-    if (live && gated) tp_up = b.prev.tile((a.d_ff + col) >> 7);
-    const int off = col & 127, off_up = (a.d_ff + col) & 127;
+    const int width = SRC == kSrcAct ? (gated ? 2 * a.d_ff : a.d_ff) : b.k_total;
+    float2 gain = make_float2(1.f, 1.f);
+    if (SRC == kSrcNorm && live) gain = ld_f2(b.gain + col);
     for (int r0 = 0; r0 < a.n_rows; r0 += kRowBatch) {
-        float2 v[kRowBatch], pa[kRowBatch][PB], pb[kRowBatch][UP];
+        float2 v[kRowBatch], up[kRowBatch];
         // ---- every load of these rows is requested before anything is used ----
 #pragma unroll
         for (int i = 0; i < kRowBatch; ++i) {
-            const int r = r0 + i;
-            v[i] = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int j = 0; j < PB; ++j) pa[i][j] = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int j = 0; j < UP; ++j) pb[i][j] = make_float2(0.f, 0.f);
-            if (!live || r >= a.n_rows) continue;
-            if (SRC == kSrcEmbed) {
-                const int t = min(max(a.row_token[r], 0), a.vocab - 1);
-                const size_t at = static_cast<size_t>(t) * a.d + col;
-                if (a.emb_bf16) {
-                    const __nv_bfloat162 e = *reinterpret_cast<const __nv_bfloat162*>(static_cast<const __nv_bfloat16*>(a.tok_emb) + at);
-                    v[i] = make_float2(__bfloat162float(e.x), __bfloat162float(e.y));
-                } else {
-                    v[i] = *reinterpret_cast<const float2*>(static_cast<const float*>(a.tok_emb) + at);
-                }
-                if (a.arch == SPEC_ARCH_GPT) {
-                    const int p = min(max(a.row_pos[r], 0), a.max_positions - 1);
-                    const size_t pat = static_cast<size_t>(p) * a.d + col;
-                    if (a.emb_bf16) {
-                        const __nv_bfloat162 e = *reinterpret_cast<const __nv_bfloat162*>(static_cast<const __nv_bfloat16*>(a.pos_emb) + pat);
-                        v[i].x += __bfloat162float(e.x);
-                        v[i].y += __bfloat162float(e.y);
-                    } else {
-                        const float2 e = *reinterpret_cast<const float2*>(static_cast<const float*>(a.pos_emb) + pat);
-                        v[i].x += e.x;
-                        v[i].y += e.y;
-                    }
-                }
-            } else if (SRC == kSrcResid) {
-                v[i] = ld_f2(b.h_in + static_cast<size_t>(r) * a.d + col);
-                load_parts<PB>(tp, off, r, 0, pa[i]);
-            } else if (SRC == kSrcPlain) {
-                v[i] = ld_f2(b.plain + static_cast<size_t>(r) * b.k_total + col);
-            } else {
-                load_parts<PB>(tp, off, r, 0, pa[i]);
-                if (gated) load_parts<UP>(tp_up, off_up, r, 0, pb[i]);
+            const int r = min(r0 + i, a.n_rows - 1);
+            v[i] = up[i] = make_float2(0.f, 0.f);
+            if (live) {
+                v[i] = ld_f2(b.rows + static_cast<size_t>(r) * width + col);
+                if (gated) up[i] = ld_f2(b.rows + static_cast<size_t>(r) * width + a.d_ff + col);
             }
         }
-        // ---- combine, keep the updated stream (tile-0 units), split, store ----
 #pragma unroll
         for (int i = 0; i < kRowBatch; ++i) {
             const int r = r0 + i;
             if (r >= a.n_rows) break;
             float2 x = v[i];
-            if (live && SRC == kSrcResid) {
-                const float2 p = sum_loaded<PB>(tp, off, r, pa[i]);
-                x.x += p.x;
-                x.y += p.y;
-            } else if (live && SRC == kSrcAct) {  // the FFN's activation of the FFN-in sums, RMSNorm's scale applied here
-                const float s = cta.scale[r];
-                const float2 gate = sum_loaded<PB>(tp, off, r, pa[i]);
-                if (!gated) {
-                    x = make_float2(gelu_tanh(s * gate.x), gelu_tanh(s * gate.y));
-                } else {
-                    const float2 up = sum_loaded<UP>(tp_up, off_up, r, pb[i]);
-                    if (a.ffn == SPEC_FFN_SWIGLU) x = make_float2(silu(s * gate.x) * (s * up.x), silu(s * gate.y) * (s * up.y));
-                    else x = make_float2(gelu_tanh(s * gate.x) * (s * up.x), gelu_tanh(s * gate.y) * (s * up.y));
-                }
-            }
-            if (writer) {  // one unit per column block keeps the new residual stream and its sum of squares
-                if (live) *reinterpret_cast<float2*>(b.h_out + static_cast<size_t>(r) * a.d + col) = x;
-                const float ss = warp_sum(x.x * x.x + x.y * x.y);
-                if (lane == 0) b.ssq_out[kb * kMaxRows + r] = ss;
-            }
-            if (b.gain) {
+            if (SRC == kSrcNorm) {
                 x.x *= gain.x;
                 x.y *= gain.y;
+            } else if (SRC == kSrcAct && live) {  // the FFN's activation, RMSNorm's scale of the FFN-in operand applied here
+                const float s = cta.scale[r];
+                if (!gated) x = make_float2(gelu_tanh(s * x.x), gelu_tanh(s * x.y));
+                else if (a.ffn == SPEC_FFN_SWIGLU) x = make_float2(silu(s * x.x) * (s * up[i].x), silu(s * x.y) * (s * up[i].y));
+                else x = make_float2(gelu_tanh(s * x.x) * (s * up[i].x), gelu_tanh(s * x.y) * (s * up[i].y));
             }
             store_pair(stage, r, lane, x.x, x.y);
         }
     }
 }
 
+// ---- what becomes of a GEMM's output tiles ------------------------------------------------
+struct SinkCtx {
+    Sink sink;
+    float* rows;          // rows: [16][n_out]
+    float* ssq_out;       // stream: sums of squares of the updated stream, per 32-column group
+    const float* ssq_in;  // logits: the sums of squares that go with the LM head's operand
+};
+
 // ---- one GEMM: every role of the CTA but the weight producer ---------------------------
-// Leaves the partial sums of this CTA's parts in a.part[g & 1].
 // Roles.  The ring is two interleaved half-rings: the units this CTA goes through are numbered
 // n = 0, 1, 2, ... over the whole pass; unit n uses stage n % kStages (kStages is even), so even
 // units use even stages and odd units odd stages.  Issuer X (warp 1 + X) takes the units of
@@ -635,8 +528,13 @@ __device__ __forceinline__ void build_block(const MegaArgs& a, const Cta& cta, c
 // n % 8 == b, in order.  Every mbarrier of a stage is therefore waited on by threads that go
 // through that stage's phases in order (a wait by parity cannot tell a phase from the one two
 // before it, so nobody may get two phases ahead of a barrier).
+//
+// A tile's parts (one per CTA whose run meets the tile) go to global memory; the CTA that
+// writes the last one (a counter per tile tells) adds them up in CTA order, so the sum does
+// not depend on who does it, and passes the tile on: rows for the next step, the residual
+// stream with its sums of squares, or logits.
 template <typename Prefetch>
-__device__ void gemm_step(const MegaArgs& a, Cta& cta, int g, const BuildCtx& b, Prefetch prefetch) {
+__device__ void gemm_step(const MegaArgs& a, Cta& cta, int g, const BuildCtx& b, const SinkCtx& o, Prefetch prefetch) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const GemmDesc gd = gemm_desc(a, g);
     const unsigned u0 = unit_begin(gd.units, cta.c, cta.P), u1 = unit_begin(gd.units, cta.c + 1, cta.P);
@@ -682,9 +580,20 @@ __device__ void gemm_step(const MegaArgs& a, Cta& cta, int g, const BuildCtx& b,
             if (!ok) atomicCAS(&g_mega_error, 0, 2);
         }
     } else if (warp >= 4 && warp < 8) {
-        // ---- epilogue: warp w reads accumulator lanes 32 (w & 3) .. + 31 ----
-        float* out = a.part[g & 1];
+        // ---- epilogue: warp w holds features 32 (w & 3) .. + 31 of the tile, one per lane ----
+        const int quarter = warp & 3;
+        float* parts = a.part[g & 1];
+        unsigned* ticket = a.ticket[g & 1];
+        const uint8_t* counts = cta.counts + a.count_offset[gemm_kind(a, g)];
         const int jmax = max_contributors(gd.units, gd.kbn, cta.P);
+        const int groups_d = (a.d + 31) / 32;
+        if (o.sink == kSinkLogits) {  // RMSNorm's scale of every row, from the LM head's operand
+            for (int r = quarter; r < a.n_rows; r += 4) {
+                const float s = row_scale(o.ssq_in, groups_d, r, a.d, a.eps, lane);
+                if (lane == 0) cta.scale[r] = s;
+            }
+            named_sync<4, 128>();
+        }
         for (int part = 0; part < n_parts; ++part) {
             const int t = t_first + part;
             const unsigned a0 = max(u0, static_cast<unsigned>(t) * gd.kbn), a1 = min(u1, static_cast<unsigned>(t + 1) * gd.kbn);
@@ -697,7 +606,7 @@ __device__ void gemm_step(const MegaArgs& a, Cta& cta, int g, const BuildCtx& b,
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             // accumulator X holds the part's units of parity X: at least one of the two was used
             const bool both = n1 - n0 > 1;
-            const uint32_t lanes = static_cast<uint32_t>((warp & 3) * 32) << 16;
+            const uint32_t lanes = static_cast<uint32_t>(quarter * 32) << 16;
             float v[16];
             tmem_ld16(cta.tmem + lanes + static_cast<uint32_t>((2 * buf + (both ? 0 : (n0 & 1u))) * kMaxRows), v);
             if (both) {
@@ -709,13 +618,83 @@ __device__ void gemm_step(const MegaArgs& a, Cta& cta, int g, const BuildCtx& b,
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(&cta.acc_empty[buf]);
-            const int j = gd.units < static_cast<unsigned>(cta.P)
-                              ? static_cast<int>(u0 % gd.kbn)
-                              : cta.c - cta_of_unit(gd.units, static_cast<unsigned>(t) * gd.kbn, cta.P);
-            float* dst = out + ((static_cast<size_t>(t) * jmax + j) * kMaxRows) * 128 + (warp & 3) * 32 + lane;
+            const int feature = quarter * 32 + lane, col = t * 128 + feature;
+            const int n_parts_of_tile = counts[t];
+            if (n_parts_of_tile > 1) {
+                // this CTA's part to memory; whoever writes a tile's last part adds them all up
+                const int j = gd.units < static_cast<unsigned>(cta.P)
+                                  ? static_cast<int>(u0 % gd.kbn)
+                                  : cta.c - cta_of_unit(gd.units, static_cast<unsigned>(t) * gd.kbn, cta.P);
+                float* tile_parts = parts + static_cast<size_t>(t) * jmax * (kMaxRows * 128);
+                float* dst = tile_parts + static_cast<size_t>(j) * (kMaxRows * 128) + feature;
 #pragma unroll
-            for (int r = 0; r < kMaxRows; ++r)
-                if (r < a.n_rows) dst[r * 128] = v[r];
+                for (int r = 0; r < kMaxRows; ++r)
+                    if (r < a.n_rows) dst[r * 128] = v[r];
+                named_sync<4, 128>();  // (the four warps' stores come before the count below: it releases them)
+                if (warp == 4 && lane == 0) {
+                    unsigned before;
+                    asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], %2;" : "=r"(before) : "l"(ticket + t), "r"(1u) : "memory");
+                    const int last = before == static_cast<unsigned>(n_parts_of_tile - 1) ? 1 : 0;
+                    if (last) ticket[t] = 0u;  // (nobody touches it again before the next GEMM that uses this array)
+                    *cta.last = last;
+                }
+                named_sync<4, 128>();
+                if (!*cta.last) continue;
+                // the parts in CTA order, four rows' loads in flight at a time (read past L1: other SMs wrote them)
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    if (q4 * 4 >= a.n_rows) break;
+                    for (int j0 = 0; j0 < n_parts_of_tile; j0 += 8) {
+                        float p[4][8];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int jj = 0; jj < 8; ++jj)
+                                p[i][jj] = ld_cg_f1(tile_parts + static_cast<size_t>(min(j0 + jj, n_parts_of_tile - 1)) * (kMaxRows * 128) +
+                                                    min(q4 * 4 + i, a.n_rows - 1) * 128 + feature);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            float acc = j0 == 0 ? p[i][0] : v[q4 * 4 + i] + p[i][0];
+#pragma unroll
+                            for (int jj = 1; jj < 8; ++jj)
+                                if (j0 + jj < n_parts_of_tile) acc += p[i][jj];
+                            v[q4 * 4 + i] = acc;
+                        }
+                    }
+                }
+            }
+            // ---- the finished tile ----
+            if (o.sink == kSinkRows) {
+                if (col < gd.n_out) {
+#pragma unroll
+                    for (int r = 0; r < kMaxRows; ++r)
+                        if (r < a.n_rows) o.rows[static_cast<size_t>(r) * gd.n_out + col] = v[r];
+                }
+            } else if (o.sink == kSinkStream) {  // h += tile; the new rows' sums of squares per 32-column group
+                float hv[16];
+#pragma unroll
+                for (int r = 0; r < kMaxRows; ++r)
+                    hv[r] = (r < a.n_rows && col < a.d) ? ld_cg_f1(a.h + static_cast<size_t>(r) * a.d + col) : 0.0f;
+#pragma unroll
+                for (int r = 0; r < kMaxRows; ++r) {
+                    if (r < a.n_rows) {
+                        const float x = col < a.d ? hv[r] + v[r] : 0.0f;
+                        if (col < a.d) a.h[static_cast<size_t>(r) * a.d + col] = x;
+                        const float ss = warp_sum(x * x);
+                        if (lane == 0 && t * 4 + quarter < groups_d) o.ssq_out[(t * 4 + quarter) * kMaxRows + r] = ss;
+                    }
+                }
+            } else {  // logits of the rows that have a destination
+                if (col < gd.n_out) {
+#pragma unroll
+                    for (int r = 0; r < kMaxRows; ++r) {
+                        if (r < a.n_rows) {
+                            const int dst = cta.row_logit[r];
+                            if (dst >= 0) a.logits[static_cast<size_t>(dst) * a.vocab + col] = v[r] * cta.scale[r];
+                        }
+                    }
+                }
+            }
         }
     } else if (warp == 3) {
         prefetch(lane);  // (the one warp without a role in a GEMM)
@@ -725,7 +704,7 @@ __device__ void gemm_step(const MegaArgs& a, Cta& cta, int g, const BuildCtx& b,
         const unsigned bi = warp - 8;
         if (b.src == kSrcAct) {  // RMSNorm's scale of every row, from the FFN-in GEMM's operand
             for (int r = bi; r < a.n_rows; r += kBuilders) {
-                const float s = row_scale(b.ssq_in, (a.d + 63) / 64, r, a.d, a.eps, lane);
+                const float s = row_scale(b.ssq, (a.d + 31) / 32, r, a.d, a.eps, lane);
                 if (lane == 0) cta.scale[r] = s;
             }
             named_sync<2, kBuilders * 32>();
@@ -738,12 +717,11 @@ __device__ void gemm_step(const MegaArgs& a, Cta& cta, int g, const BuildCtx& b,
                 break;
             }
             uint8_t* stage = cta.ring + s * kStageBytes;
-            const int tile = static_cast<int>(u / gd.kbn), kb = static_cast<int>(u % gd.kbn);
+            const int kb = static_cast<int>(u % gd.kbn);
             switch (b.src) {
-                case kSrcEmbed: build_block<kSrcEmbed>(a, cta, b, stage, tile, kb, lane); break;
-                case kSrcResid: build_block<kSrcResid>(a, cta, b, stage, tile, kb, lane); break;
-                case kSrcPlain: build_block<kSrcPlain>(a, cta, b, stage, tile, kb, lane); break;
-                default: build_block<kSrcAct>(a, cta, b, stage, tile, kb, lane); break;
+                case kSrcNorm: build_block<kSrcNorm>(a, cta, b, stage, kb, lane); break;
+                case kSrcPlain: build_block<kSrcPlain>(a, cta, b, stage, kb, lane); break;
+                default: build_block<kSrcAct>(a, cta, b, stage, kb, lane); break;
             }
             fence_async_smem();
             if (!warp_wait(&cta.wfull[s], (n / kStages) & 1u, cta.abort_flag, lane)) {
@@ -759,16 +737,41 @@ __device__ void gemm_step(const MegaArgs& a, Cta& cta, int g, const BuildCtx& b,
     __syncwarp();  // (the issuers' warps re-converge before the barrier that follows)
 }
 
-// ---- rotary positions, K,V append, q rows: finishes the projection GEMM g ----------------
-// n_kv_heads = 0: queries only (cross-attention).
-template <typename KV>
-__device__ void qkv_step(const MegaArgs& a, const Cta& cta, int g, const float* ssq, int n_heads, int n_kv_heads, bool rope,
-                         KV* kv_layer) {
+// ---- the residual stream's first value: token (+ position) embeddings, and its sums of squares ----
+__device__ void embed_step(const MegaArgs& a, const Cta& cta, float* ssq_out) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp < 2) return;
-    const PartialView pv = partial_view(a, g, cta.P, cta.counts);
+    const int groups = (a.d + 31) / 32;  // a warp per 32 columns
+    for (int i = cta.c + cta.P * (warp - 2); i < groups; i += cta.P * kWorkers) {
+        const int col = i * 32 + lane;
+        for (int r = 0; r < a.n_rows; ++r) {
+            float x = 0.0f;
+            if (col < a.d) {
+                const int t = min(max(cta.row_tok[r], 0), a.vocab - 1);
+                const size_t at = static_cast<size_t>(t) * a.d + col;
+                x = a.emb_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.tok_emb)[at]) : static_cast<const float*>(a.tok_emb)[at];
+                if (a.arch == SPEC_ARCH_GPT) {
+                    const int p = min(max(cta.row_pos[r], 0), a.max_positions - 1);
+                    const size_t pat = static_cast<size_t>(p) * a.d + col;
+                    x += a.emb_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.pos_emb)[pat]) : static_cast<const float*>(a.pos_emb)[pat];
+                }
+                a.h[static_cast<size_t>(r) * a.d + col] = x;
+            }
+            const float ss = warp_sum(x * x);
+            if (lane == 0) ssq_out[i * kMaxRows + r] = ss;
+        }
+    }
+}
+
+// ---- rotary positions, K,V append, q rows: finishes the projection whose rows are in a.out -----
+// n_kv_heads = 0: queries only (cross-attention).
+template <typename KV>
+__device__ void qkv_step(const MegaArgs& a, const Cta& cta, const float* ssq, int n_heads, int n_kv_heads, bool rope, KV* kv_layer) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp < 2) return;
     const int heads = n_heads + 2 * n_kv_heads, half = a.dh / 2;
-    const int kbn_d = (a.d + 63) / 64;
+    const int width = heads * a.dh;
+    const int groups_d = (a.d + 31) / 32;
     const int units = a.n_rows * heads;
     // unit i -> CTA i % P, worker (i / P) % kWorkers
     for (int i = cta.c + cta.P * (warp - 2); i < units; i += cta.P * kWorkers) {
@@ -776,33 +779,27 @@ __device__ void qkv_step(const MegaArgs& a, const Cta& cta, int g, const float* 
         const int p = cta.row_pos[r];
         const bool is_q = head < n_heads, is_k = !is_q && head < n_heads + n_kv_heads;
         // lane owns the pairs (j, j + 1) of the first half and the same of the second half; every
-        // load of the unit (sums of squares, parts, rotation, page) is requested before any is used
+        // load of the unit (sums of squares, values, rotation, page) is requested before any is used
         const int j = 2 * lane;
         const bool live = j < half;
         const int col = head * a.dh + j;
-        const float sq = row_ssq_share(ssq, kbn_d, r, lane);
-        TileParts t1{nullptr, 0}, t2{nullptr, 0};
-        float2 p1[8], p2[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) p1[k] = p2[k] = make_float2(0.f, 0.f);
+        const float sq = row_ssq_share(ssq, groups_d, r, lane);
+        float2 x1 = make_float2(0.f, 0.f), x2 = x1;
         float4 cs = make_float4(1.f, 0.f, 1.f, 0.f);
         int page = 0;
         if (live) {
-            t1 = pv.tile(col >> 7);
-            t2 = pv.tile((col + half) >> 7);
-            load_parts<8>(t1, col & 127, r, 0, p1);
-            load_parts<8>(t2, (col + half) & 127, r, 0, p2);
+            x1 = ld_f2(a.out + static_cast<size_t>(r) * width + col);
+            x2 = ld_f2(a.out + static_cast<size_t>(r) * width + col + half);
             if (rope && p >= 0 && (is_q || is_k)) cs = *reinterpret_cast<const float4*>(a.rope + static_cast<size_t>(p) * half + j);  // (cos, sin) x 2
             if (!is_q && p >= 0) page = a.page_table[cta.row_seq[r] * a.pages_per_seq + p / a.page_size];
         }
         const float s = rsqrtf(warp_sum(sq) / static_cast<float>(a.d) + a.eps);
         if (!live) continue;
-        float2 x1 = sum_loaded<8>(t1, col & 127, r, p1), x2 = sum_loaded<8>(t2, (col + half) & 127, r, p2);
         x1.x *= s; x1.y *= s; x2.x *= s; x2.y *= s;
         const float2 y1 = make_float2(x1.x * cs.x - x2.x * cs.y, x1.y * cs.z - x2.y * cs.w);
         const float2 y2 = make_float2(x2.x * cs.x + x1.x * cs.y, x2.y * cs.z + x1.y * cs.w);
-        if (is_q) {
-            float* dst = a.q + static_cast<size_t>(r) * (n_heads * a.dh) + col;
+        if (is_q) {  // q stays in place (rotated, scaled) for the attention
+            float* dst = a.out + static_cast<size_t>(r) * width + col;
             *reinterpret_cast<float2*>(dst) = y1;
             *reinterpret_cast<float2*>(dst + half) = y2;
         } else if (p >= 0) {
@@ -819,8 +816,9 @@ __device__ void qkv_step(const MegaArgs& a, const Cta& cta, int g, const float* 
 
 // ---- attention: (sequence, KV head, key slice) pieces dealt out to the CTAs ----------------
 template <typename KV, int DH>
-__device__ void attention_step(const MegaArgs& a, const Cta& cta, const KV* kv_layer, const int32_t* page_table,
-                               int pages_per_seq, const int32_t* kv_len, const float* bias, int slices, float (*share)[DH + 2]) {
+__device__ void attention_step(const MegaArgs& a, const Cta& cta, const float* q, int q_stride, const KV* kv_layer,
+                               const int32_t* page_table, int pages_per_seq, const int32_t* kv_len, const float* bias, int slices,
+                               float (*share)[DH + 2]) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp < 2) return;
     const int queries = (a.n_heads / a.n_kv_heads) * a.m_rows;
@@ -829,7 +827,7 @@ __device__ void attention_step(const MegaArgs& a, const Cta& cta, const KV* kv_l
     const int pieces = a.batch * a.n_kv_heads * slices;
     for (int u = cta.c; u < pieces; u += cta.P) {
         const int slice = u % slices, kv_head = (u / slices) % a.n_kv_heads, b = u / (slices * a.n_kv_heads);
-        attend_slice<KV, DH, NamedSync<3, kWorkers * 32>>(a.q, a.n_heads * DH, a.row_pos, a.row_seq, a.m_rows, a.n_heads, a.n_kv_heads,
+        attend_slice<KV, DH, NamedSync<3, kWorkers * 32>>(q, q_stride, a.row_pos, a.row_seq, a.m_rows, a.n_heads, a.n_kv_heads,
                                                          ks, kv_layer, page_table, pages_per_seq, a.page_size, kv_len, bias,
                                                          a.bias_span, a.bias_zero, scale, a.attn_part, slice, slices, kv_head, b,
                                                          warp - 2, kWorkers, lane, share, false, kv_len ? -1 : cta.seq_keys[b]);
@@ -934,6 +932,7 @@ __global__ void __launch_bounds__(kThreads, 1) pass_kernel(const __grid_constant
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + Smem::kTmemSlot);
     cta.abort_flag = reinterpret_cast<volatile int*>(smem + Smem::kAbort);
     cta.verdict = cta.abort_flag + 1;
+    cta.last = cta.abort_flag + 2;
     cta.scale = reinterpret_cast<float*>(smem + Smem::kScale);
     float(*share)[DH + 2] = reinterpret_cast<float(*)[DH + 2]>(smem + Smem::kShare);
     cta.c = blockIdx.x;
@@ -965,15 +964,13 @@ __global__ void __launch_bounds__(kThreads, 1) pass_kernel(const __grid_constant
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(64));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    cta.tmem = *tmem_slot;
-    {
+    {   // what every step needs of the rows, in shared memory
         int* rows_sh = reinterpret_cast<int*>(smem + Smem::kRowPos);
         cta.row_pos = rows_sh;
         cta.row_seq = rows_sh + 16;
         cta.seq_keys = rows_sh + 32;
+        cta.row_tok = rows_sh + 48;
+        cta.row_logit = rows_sh + 64;
         if (threadIdx.x < 16) {
             const int r = threadIdx.x;
             rows_sh[r] = r < a.n_rows ? a.row_pos[r] : -1;
@@ -982,12 +979,23 @@ __global__ void __launch_bounds__(kThreads, 1) pass_kernel(const __grid_constant
             if (r < a.batch)
                 for (int j = 0; j < a.m_rows; ++j) keys = max(keys, a.row_pos[r * a.m_rows + j] + 1);
             rows_sh[32 + r] = keys;
+            rows_sh[48 + r] = r < a.n_rows ? a.row_token[r] : 0;
+            // the logits row that pass row r feeds (none: -1)
+            rows_sh[64 + r] = !a.logit_src && r < a.n_logit_rows ? (a.logit_dst ? a.logit_dst[r] : r) : -1;
         }
         uint8_t* counts_sh = smem + Smem::kCounts;
         for (int i = threadIdx.x; i < a.count_total; i += kThreads) counts_sh[i] = a.tile_counts[i];
         cta.counts = counts_sh;
-        __syncthreads();
     }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    cta.tmem = *tmem_slot;
+    if (a.logit_src && threadIdx.x < a.n_logit_rows) {
+        const int src = a.logit_src[threadIdx.x];
+        if (src >= 0 && src < 16) reinterpret_cast<int*>(smem + Smem::kRowPos)[64 + src] = a.logit_dst ? a.logit_dst[threadIdx.x] : threadIdx.x;
+    }
+    __syncthreads();
     if (a.trace && cta.c == 0 && threadIdx.x == 32 && a.trace_capacity > 1) {  // (CTAs; start of the pass)
         a.trace[0] = gridDim.x;
         a.trace[1] = global_ns();
@@ -998,102 +1006,48 @@ __global__ void __launch_bounds__(kThreads, 1) pass_kernel(const __grid_constant
         __syncwarp();
     } else {
         const int per = gemms_per_layer(a);
-        const int q_dim = a.n_heads * DH;
-        int hb = 0;  // which copy of the residual stream (and of the sums of squares) is current
-        bool ok = true;
+        const int q_dim = a.n_heads * DH, qkv_dim = (a.n_heads + 2 * a.n_kv_heads) * DH;
+        int hb = 0;  // which copy of the stream's sums of squares is current
         // the longest key set of any sequence of the pass
         int longest = 0;
         for (int b = 0; b < a.batch; ++b) longest = max(longest, cta.seq_keys[b]);
         const int slices = choose_slices(a, cta.P, longest);
+        embed_step(a, cta, a.ssq[0]);
+        bool ok = grid_sync(a, cta);
         for (int l = 0; l < a.n_layers && ok; ++l) {
             const MegaLayer& L = a.layers[l];
             int g = l * per;
-            BuildCtx b{};
-            // ---- projection of the normalised stream; the stream itself is brought up to date on the way ----
-            b.src = l == 0 ? kSrcEmbed : kSrcResid;
-            b.k_total = a.d;
-            b.gain = L.ln1;
-            b.h_in = a.h[hb];
-            b.h_out = a.h[hb ^ 1];
-            b.ssq_out = a.ssq[hb ^ 1];
-            if (l > 0) b.prev = partial_view(a, g - 1, cta.P, cta.counts);
-            gemm_step(a, cta, g, b, [&](int ln) { prefetch_keys<KV, DH>(a, cta, static_cast<const KV*>(L.kv), slices, ln); });
-            hb ^= 1;
+            // ---- projection of the normalised stream ----
+            gemm_step(a, cta, g, BuildCtx{kSrcNorm, a.d, L.ln1, a.h, nullptr}, SinkCtx{kSinkRows, a.out, nullptr, nullptr},
+                      [&](int ln) { prefetch_keys<KV, DH>(a, cta, static_cast<const KV*>(L.kv), slices, ln); });
             if (!(ok = grid_sync(a, cta))) break;
-            qkv_step<KV>(a, cta, g, a.ssq[hb], a.n_heads, a.n_kv_heads, a.arch == SPEC_ARCH_LLAMA, static_cast<KV*>(L.kv));
+            qkv_step<KV>(a, cta, a.ssq[hb], a.n_heads, a.n_kv_heads, a.arch == SPEC_ARCH_LLAMA, static_cast<KV*>(L.kv));
             if (!(ok = grid_sync(a, cta))) break;
-            attention_step<KV, DH>(a, cta, static_cast<const KV*>(L.kv), a.page_table, a.pages_per_seq, nullptr,
+            attention_step<KV, DH>(a, cta, a.out, qkv_dim, static_cast<const KV*>(L.kv), a.page_table, a.pages_per_seq, nullptr,
                                    a.arch == SPEC_ARCH_T5 ? a.dec_bias : nullptr, slices, share);
             if (!(ok = grid_sync(a, cta))) break;
             combine_step<DH>(a, cta, slices);
             if (!(ok = grid_sync(a, cta))) break;
-            // ---- out-projection ----
+            // ---- out-projection into the stream ----
             ++g;
-            b = BuildCtx{};
-            b.src = kSrcPlain;
-            b.k_total = q_dim;
-            b.plain = a.att;
-            gemm_step(a, cta, g, b, [](int) {});
-            if (!(ok = grid_sync(a, cta))) break;
-            // ---- FFN-in on the normalised, updated stream ----
-            ++g;
-            b = BuildCtx{};
-            b.src = kSrcResid;
-            b.k_total = a.d;
-            b.gain = L.ln2;
-            b.h_in = a.h[hb];
-            b.h_out = a.h[hb ^ 1];
-            b.ssq_out = a.ssq[hb ^ 1];
-            b.prev = partial_view(a, g - 1, cta.P, cta.counts);
-            gemm_step(a, cta, g, b, [](int) {});
+            gemm_step(a, cta, g, BuildCtx{kSrcPlain, q_dim, nullptr, a.att, nullptr}, SinkCtx{kSinkStream, nullptr, a.ssq[hb ^ 1], nullptr},
+                      [](int) {});
             hb ^= 1;
             if (!(ok = grid_sync(a, cta))) break;
-            // ---- FFN-out on the activation of the FFN-in sums ----
+            // ---- FFN-in on the normalised stream ----
             ++g;
-            b = BuildCtx{};
-            b.src = kSrcAct;
-            b.k_total = a.d_ff;
-            b.ssq_in = a.ssq[hb];
-            b.prev = partial_view(a, g - 1, cta.P, cta.counts);
-            gemm_step(a, cta, g, b, [](int) {});
+            gemm_step(a, cta, g, BuildCtx{kSrcNorm, a.d, L.ln2, a.h, nullptr}, SinkCtx{kSinkRows, a.out, nullptr, nullptr}, [](int) {});
+            if (!(ok = grid_sync(a, cta))) break;
+            // ---- FFN-out on the activation of the FFN-in rows, into the stream ----
+            ++g;
+            gemm_step(a, cta, g, BuildCtx{kSrcAct, a.d_ff, nullptr, a.out, a.ssq[hb]}, SinkCtx{kSinkStream, nullptr, a.ssq[hb ^ 1], nullptr},
+                      [](int) {});
+            hb ^= 1;
             if (!(ok = grid_sync(a, cta))) break;
         }
-        if (ok && a.n_logit_rows > 0) {
-            // ---- final norm and LM head ----
-            const int g = per * a.n_layers;
-            BuildCtx b{};
-            b.src = kSrcResid;
-            b.k_total = a.d;
-            b.gain = a.ln_f;
-            b.h_in = a.h[hb];
-            b.h_out = a.h[hb ^ 1];
-            b.ssq_out = a.ssq[hb ^ 1];
-            b.prev = partial_view(a, g - 1, cta.P, cta.counts);
-            gemm_step(a, cta, g, b, [](int) {});
-            hb ^= 1;
-            ok = grid_sync(a, cta);
-            if (ok) {
-                // logits[dst(i)][n] = scale(src(i)) * sum of the parts
-                const int kbn_d = (a.d + 63) / 64;
-                if (warp >= 2)
-                    for (int r = warp - 2; r < a.n_rows; r += kWorkers) {
-                        const float s = row_scale(a.ssq[hb], kbn_d, r, a.d, a.eps, lane);
-                        if (lane == 0) cta.scale[r] = s;
-                    }
-                named_sync<1, kBarThreads>();
-                const PartialView pv = partial_view(a, g, cta.P, cta.counts);
-                const int pairs = a.vocab / 2;  // (the vocabulary is even whenever this kernel is used)
-                const long long total = static_cast<long long>(a.n_logit_rows) * pairs;
-                for (long long i = static_cast<long long>(cta.c) * kBarThreads + (threadIdx.x - 32); i < total;
-                     i += static_cast<long long>(cta.P) * kBarThreads) {
-                    const int li = static_cast<int>(i / pairs), col = 2 * static_cast<int>(i % pairs);
-                    const int src = a.logit_src ? a.logit_src[li] : li, dst = a.logit_dst ? a.logit_dst[li] : li;
-                    const float2 v = sum_parts2(pv.tile(col >> 7), col & 127, src);
-                    const float s = cta.scale[src];
-                    *reinterpret_cast<float2*>(a.logits + static_cast<size_t>(dst) * a.vocab + col) = make_float2(v.x * s, v.y * s);
-                }
-            }
-        }
+        if (ok && a.n_logit_rows > 0)  // ---- final norm and LM head: the finished tiles are the logits ----
+            gemm_step(a, cta, per * a.n_layers, BuildCtx{kSrcNorm, a.d, a.ln_f, a.h, nullptr},
+                      SinkCtx{kSinkLogits, nullptr, nullptr, a.ssq[hb]}, [](int) {});
         if (!ok) atomicCAS(&g_mega_error, 0, 5);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -1141,8 +1095,12 @@ struct Shape {
     int n_out, k;
 };
 
+struct LiveScratch {
+    unsigned *sync, *ticket[2];
+    int ticket_count;
+};
 std::mutex g_sync_mutex;
-std::vector<unsigned*> g_sync_words;  // the barrier words of every live context
+std::vector<LiveScratch> g_live;  // the barrier words and part counters of every live context
 
 std::vector<Shape> gemm_shapes(const Model& m) {
     const spec_model_cfg& c = m.cfg;
@@ -1196,7 +1154,7 @@ int pass_scratch_init(PassScratch& s, const Model* models, int n_models, std::ve
     SPEC_TRY_STATUS(resident_ctas<__nv_bfloat16, 128>(&other));
     ctas = std::min(ctas, other);
     if (ctas < 1) return SPEC_OK;
-    size_t d = 0, q = 0, part = 0, attn = 0;
+    size_t d = 0, q = 0, part = 0, attn = 0, out = 0, tiles_most = 0;
     bool any = false;
     for (int i = 0; i < n_models; ++i) {
         const Model& m = models[i];
@@ -1204,14 +1162,16 @@ int pass_scratch_init(PassScratch& s, const Model* models, int n_models, std::ve
         any = true;
         d = std::max<size_t>(d, m.cfg.d_model);
         q = std::max<size_t>(q, m.q_dim());
+        out = std::max<size_t>({out, static_cast<size_t>(m.qkv_dim()), static_cast<size_t>(m.ffn_in_dim()), static_cast<size_t>(m.q_dim())});
         attn = std::max<size_t>(attn, static_cast<size_t>(kMaxRows) * m.cfg.n_heads * kMaxSlices * (m.cfg.d_head + 2));
         for (const Shape& sh : gemm_shapes(m)) {
             const int tiles = (sh.n_out + 127) / 128, kbn = (sh.k + 63) / 64;
+            tiles_most = std::max<size_t>(tiles_most, tiles);
             part = std::max(part, static_cast<size_t>(tiles) * max_contributors(static_cast<unsigned>(tiles) * kbn, kbn, ctas) * kMaxRows * 128);
         }
     }
     if (!any) return SPEC_OK;
-    auto alloc = [&](void** out, size_t bytes) -> int {
+    auto alloc = [&](void** out_ptr, size_t bytes) -> int {
         void* p = nullptr;
         const cudaError_t err = cudaMalloc(&p, std::max<size_t>(bytes, 256));
         if (err != cudaSuccess) {
@@ -1219,15 +1179,18 @@ int pass_scratch_init(PassScratch& s, const Model* models, int n_models, std::ve
             return fail(SPEC_ERR_OOM, "cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(err));
         }
         allocations.push_back(p);
-        *out = p;
+        *out_ptr = p;
         return SPEC_OK;
     };
+    SPEC_TRY_STATUS(alloc(reinterpret_cast<void**>(&s.h), kMaxRows * d * sizeof(float)));
     for (int i = 0; i < 2; ++i) {
-        SPEC_TRY_STATUS(alloc(reinterpret_cast<void**>(&s.h[i]), kMaxRows * d * sizeof(float)));
-        SPEC_TRY_STATUS(alloc(reinterpret_cast<void**>(&s.ssq[i]), ((d + 63) / 64) * kMaxRows * sizeof(float)));
+        SPEC_TRY_STATUS(alloc(reinterpret_cast<void**>(&s.ssq[i]), ((d + 31) / 32) * kMaxRows * sizeof(float)));
         SPEC_TRY_STATUS(alloc(reinterpret_cast<void**>(&s.part[i]), part * sizeof(float)));
+        SPEC_TRY_STATUS(alloc(reinterpret_cast<void**>(&s.ticket[i]), tiles_most * sizeof(unsigned)));
+        SPEC_CUDA_TRY(cudaMemset(s.ticket[i], 0, tiles_most * sizeof(unsigned)));
     }
-    SPEC_TRY_STATUS(alloc(reinterpret_cast<void**>(&s.q), kMaxRows * q * sizeof(float)));
+    s.ticket_count = static_cast<int>(tiles_most);
+    SPEC_TRY_STATUS(alloc(reinterpret_cast<void**>(&s.out), kMaxRows * out * sizeof(float)));
     SPEC_TRY_STATUS(alloc(reinterpret_cast<void**>(&s.att), kMaxRows * q * sizeof(float)));
     SPEC_TRY_STATUS(alloc(reinterpret_cast<void**>(&s.attn_part), attn * sizeof(float)));
     SPEC_TRY_STATUS(alloc(reinterpret_cast<void**>(&s.sync), 256));
@@ -1278,7 +1241,7 @@ int pass_scratch_init(PassScratch& s, const Model* models, int n_models, std::ve
     }
     s.ctas = ctas;
     std::lock_guard<std::mutex> lock(g_sync_mutex);
-    g_sync_words.push_back(s.sync);
+    g_live.push_back(LiveScratch{s.sync, {s.ticket[0], s.ticket[1]}, s.ticket_count});
     return SPEC_OK;
 }
 
@@ -1328,12 +1291,13 @@ int launch_pass(const PassScratch& s, const Model& m, int which, const RowMeta& 
     a.logit_src = logit_src;
     a.logit_dst = logit_dst;
     a.logits = logits;
+    a.h = s.h;
     for (int i = 0; i < 2; ++i) {
-        a.h[i] = s.h[i];
         a.ssq[i] = s.ssq[i];
         a.part[i] = s.part[i];
+        a.ticket[i] = s.ticket[i];
     }
-    a.q = s.q;
+    a.out = s.out;
     a.att = s.att;
     a.attn_part = s.attn_part;
     a.sync = s.sync;
@@ -1349,19 +1313,23 @@ int launch_pass(const PassScratch& s, const Model& m, int which, const RowMeta& 
 
 void pass_scratch_release(PassScratch& s) {
     std::lock_guard<std::mutex> lock(g_sync_mutex);
-    g_sync_words.erase(std::remove(g_sync_words.begin(), g_sync_words.end(), s.sync), g_sync_words.end());
+    g_live.erase(std::remove_if(g_live.begin(), g_live.end(), [&](const LiveScratch& l) { return l.sync == s.sync; }), g_live.end());
     s.ctas = 0;
 }
 
 // Non-zero if the pass kernel gave up on a bounded wait since the last call (then the barrier
-// words of every context are reset, so that the next launch starts clean).  Synchronises.
+// words and part counters of every context are reset, so that the next launch starts clean).
+// Synchronises.
 int pass_take_error() {
     int v = 0, zero = 0;
     if (cudaMemcpyFromSymbol(&v, g_mega_error, sizeof(int)) != cudaSuccess) return -1;
     if (v) {
         cudaMemcpyToSymbol(g_mega_error, &zero, sizeof(int));
         std::lock_guard<std::mutex> lock(g_sync_mutex);
-        for (unsigned* w : g_sync_words) cudaMemset(w, 0, 256);
+        for (const LiveScratch& l : g_live) {
+            cudaMemset(l.sync, 0, 256);
+            for (int i = 0; i < 2; ++i) cudaMemset(l.ticket[i], 0, l.ticket_count * sizeof(unsigned));
+        }
     }
     return v;
 }

@@ -151,9 +151,10 @@ int launch_ffn_act(const float* u, const float* partial, int splits, int n_rows,
 // mega.cu: one forward pass over at most 16 rows as one persistent cooperative kernel
 // (bf16 decoder-only models).
 struct PassScratch {
-    float *h[2] = {nullptr, nullptr}, *ssq[2] = {nullptr, nullptr}, *part[2] = {nullptr, nullptr};
-    float *q = nullptr, *att = nullptr, *attn_part = nullptr;
-    unsigned* sync = nullptr;
+    float *h = nullptr, *ssq[2] = {nullptr, nullptr}, *part[2] = {nullptr, nullptr};
+    float *out = nullptr, *att = nullptr, *attn_part = nullptr;
+    unsigned *sync = nullptr, *ticket[2] = {nullptr, nullptr};
+    int ticket_count = 0;
     void* layers[2] = {nullptr, nullptr};  // per model: device array of its blocks' pointers (nullptr: not served)
     void* tile_counts[2] = {nullptr, nullptr};  // per model: parts per tile of every GEMM kind (bytes)
     int count_offset[2][7] = {};
