@@ -269,7 +269,7 @@ int spec_uniforms(uint64_t seed, const int32_t* positions, const int32_t* sequen
  * ------------------------------------------------------------------------- */
 enum { SPEC_ARCH_GPT = 0, SPEC_ARCH_LLAMA = 1, SPEC_ARCH_T5 = 2, SPEC_ARCH_BIGRAM = 3, SPEC_ARCH_COPY = 4 };
 enum { SPEC_FFN_GELU = 0, SPEC_FFN_GATED_GELU = 1, SPEC_FFN_SWIGLU = 2 };
-enum { SPEC_DTYPE_FP32 = 0, SPEC_DTYPE_BF16 = 1 };
+enum { SPEC_DTYPE_FP32 = 0, SPEC_DTYPE_BF16 = 1, SPEC_DTYPE_FP16 = 2 /* cached K,V rows only */ };
 
 typedef struct spec_model_cfg {
     int arch;             /* SPEC_ARCH_* */
@@ -327,9 +327,11 @@ typedef struct spec_runtime_cfg {
     int max_len;          /* tokens per sequence the KV caches can hold (prompt + new + gamma) */
     int page_size;        /* tokens per KV page (power of two, 32..256) */
     int max_gamma;        /* largest gamma spec_generate will be asked for */
-    int kv_dtype;         /* SPEC_DTYPE_FP32 or SPEC_DTYPE_BF16: element type of the cached K,V rows.
-                             bf16 halves the KV traffic but rounds every cached row to 8 mantissa
-                             bits, which on deep models moves logits by more than 2e-2. */
+    int kv_dtype;         /* element type of the cached K,V rows: SPEC_DTYPE_FP32, SPEC_DTYPE_FP16 or
+                             SPEC_DTYPE_BF16.  The 16-bit types halve the K,V traffic.  fp16 keeps 11
+                             significant bits (values beyond +-65504 are stored as +-65504) and stays
+                             inside the 2e-2 logit tolerance of bf16 models; bf16 keeps 8, which on
+                             wide or deep models moves logits by more than that. */
     int max_src_len;      /* T5: longest source the encoders are given (0 for decoder-only models) */
     int pass_kernel;      /* 0 (default): every pass is a chain of kernels.  1: passes of at most 16 rows of
                              a bf16 GPT- or Llama-shaped model run as one persistent cooperative kernel

@@ -332,7 +332,7 @@ class _Stats(ctypes.Structure):
 
 _ARCH = {"gpt": 0, "llama": 1, "t5": 2, "bigram": 3, "copy": 4}
 _FFN = {"gelu": 0, "gated_gelu": 1, "swiglu": 2}
-_DTYPE = {"fp32": 0, "bf16": 1}
+_DTYPE = {"fp32": 0, "bf16": 1, "fp16": 2}
 _engine_declared = False
 
 
@@ -396,11 +396,14 @@ class Engine:
     """
 
     def __init__(self, target_cfg, target_weights, draft_cfg=None, draft_weights=None, max_batch=1, max_len=256,
-                 page_size=64, max_gamma=8, kv_dtype="fp32", device=None, max_src_len=0, pass_kernel=False):
+                 page_size=64, max_gamma=8, kv_dtype=None, device=None, max_src_len=0, pass_kernel=False):
         import numpy as np
         self._np = np
         h = lib()
         _declare_engine(h)
+        if kv_dtype is None:  # cached K,V rows: fp16 for bf16 models (inside their logit tolerance), fp32 for fp32 models
+            kv_dtype = "fp16" if target_cfg["dtype"] == "bf16" else "fp32"
+        self.kv_dtype = kv_dtype
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
         self.cfgs = [target_cfg, draft_cfg]
         self._keep = []

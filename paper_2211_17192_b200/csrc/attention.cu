@@ -172,14 +172,15 @@ __device__ __forceinline__ void stage_tile(const float* tile, int n_valid, float
         cp_async16(dst + row * (DH + 4) + 4 * c, tile + static_cast<size_t>(valid ? row : 0) * DH + 4 * c, valid);
     }
 }
-template <int DH>
-__device__ __forceinline__ void stage_tile(const __nv_bfloat16* tile, int n_valid, float* dst, int lane) {
+// (16-bit rows: converted on the way into shared memory)
+template <int DH, typename KV16>
+__device__ __forceinline__ void stage_tile(const KV16* tile, int n_valid, float* dst, int lane) {
     constexpr int kChunks = DH / 8;
     for (int i = lane; i < kTileKeys * kChunks; i += 32) {
         const int row = i / kChunks, c = i % kChunks;
         float v[8];
         if (row < n_valid) {
-            KvLoad<__nv_bfloat16>::load(tile + static_cast<size_t>(row) * DH + 8 * c, v);
+            KvLoad<KV16>::load(tile + static_cast<size_t>(row) * DH + 8 * c, v);
         } else {
 #pragma unroll
             for (int e = 0; e < 8; ++e) v[e] = 0.0f;
@@ -650,9 +651,13 @@ int launch_attention_variant(const Model& m, const AttnSource& src, const RowMet
 int launch_attention(const Model& m, const AttnSource& src, const RowMeta& rows, int batch, int m_rows, int slices,
                      int max_keys, float* part, float* att, __nv_bfloat16* att_hi, __nv_bfloat16* att_lo, cudaStream_t stream) {
     const AttnOut out{att, att_hi, att_lo};
-    if (src.pool.elem_bytes == 2) {
+    if (src.pool.dtype == SPEC_DTYPE_BF16) {
         if (m.cfg.d_head == 64) return launch_attention_variant<__nv_bfloat16, 64>(m, src, rows, batch, m_rows, slices, max_keys, part, out, stream);
         return launch_attention_variant<__nv_bfloat16, 128>(m, src, rows, batch, m_rows, slices, max_keys, part, out, stream);
+    }
+    if (src.pool.dtype == SPEC_DTYPE_FP16) {
+        if (m.cfg.d_head == 64) return launch_attention_variant<__half, 64>(m, src, rows, batch, m_rows, slices, max_keys, part, out, stream);
+        return launch_attention_variant<__half, 128>(m, src, rows, batch, m_rows, slices, max_keys, part, out, stream);
     }
     if (m.cfg.d_head == 64) return launch_attention_variant<float, 64>(m, src, rows, batch, m_rows, slices, max_keys, part, out, stream);
     return launch_attention_variant<float, 128>(m, src, rows, batch, m_rows, slices, max_keys, part, out, stream);

@@ -14,6 +14,7 @@
 #pragma once
 
 #include <cfloat>
+#include <cuda_fp16.h>
 
 #include "model.cuh"
 
@@ -67,6 +68,39 @@ struct KvLoad<__nv_bfloat16> {
         }
     }
 };
+
+template <>
+struct KvLoad<__half> {
+    static constexpr int kVec = 8;
+    __device__ static __forceinline__ void load(const __half* p, float* out) {
+        const uint4 t = *reinterpret_cast<const uint4*>(p);
+        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+            out[2 * i] = f.x;
+            out[2 * i + 1] = f.y;
+        }
+    }
+    template <int N>
+    __device__ static __forceinline__ void load_n(const __half* p, float* out) {
+        if (N == 4) {
+            const uint2 t = *reinterpret_cast<const uint2*>(p);
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&t.x)), b = __half22float2(*reinterpret_cast<const __half2*>(&t.y));
+            out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
+        } else {
+            const uint32_t t = *reinterpret_cast<const uint32_t*>(p);
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&t));
+            out[0] = a.x; out[1] = a.y;
+        }
+    }
+};
+
+// A value as it is stored in a cached K,V row (fp16: clamped to the finite range first).
+template <typename KV>
+__device__ __forceinline__ KV to_cached(float x) { return static_cast<KV>(x); }
+template <>
+__device__ __forceinline__ __half to_cached<__half>(float x) { return __float2half_rn(fminf(fmaxf(x, -65504.0f), 65504.0f)); }
 
 // Synchronisation of the warps that take part: the whole CTA, or a named barrier.
 struct CtaSync {

@@ -206,12 +206,12 @@ int device_gave_up(spec_ctx* ctx) {
 }
 
 KvPool layer_pool(const spec_ctx* ctx, const Model& m, int layer) {
-    return KvPool{static_cast<char*>(m.kv) + static_cast<size_t>(layer) * m.layer_stride, m.kv_elem_bytes, ctx->page_table,
+    return KvPool{static_cast<char*>(m.kv) + static_cast<size_t>(layer) * m.layer_stride, m.kv_elem_bytes, m.kv_dtype, ctx->page_table,
                   ctx->pages_per_seq, ctx->rt.page_size};
 }
 
 KvPool source_pool(const spec_ctx* ctx, const Model& m, void* base) {
-    return KvPool{base, m.kv_elem_bytes, ctx->src_page_table, ctx->src_pages_per_seq, ctx->rt.page_size};
+    return KvPool{base, m.kv_elem_bytes, m.kv_dtype, ctx->src_page_table, ctx->src_pages_per_seq, ctx->rt.page_size};
 }
 
 // One forward pass of `m` over batch * m_rows rows (rows of sequence b are rows
@@ -593,7 +593,8 @@ int init_model(spec_ctx* ctx, int which, const spec_model_cfg& cfg, const spec_w
             if (!l.lnx || !l.wq_x || !l.wkv_x || !l.wo_x)
                 return fail(SPEC_ERR_BAD_ARG, "spec_init: missing cross-attention weight pointer");
     }
-    m.kv_elem_bytes = ctx->rt.kv_dtype == SPEC_DTYPE_BF16 ? 2 : 4;
+    m.kv_dtype = ctx->rt.kv_dtype;
+    m.kv_elem_bytes = ctx->rt.kv_dtype == SPEC_DTYPE_FP32 ? 4 : 2;
     const size_t n_pages = static_cast<size_t>(ctx->rt.max_batch) * ctx->pages_per_seq;
     m.layer_stride = n_pages * 2 * cfg.n_kv_heads * ctx->rt.page_size * cfg.d_head * m.kv_elem_bytes;
     char* kv = nullptr;
@@ -683,7 +684,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     const spec_runtime_cfg& rt = *runtime;
     if (rt.max_batch < 1 || rt.max_batch > 4096 || rt.max_len < 2 || rt.max_gamma < 0 || rt.max_gamma > 64 ||
         rt.page_size < 32 || rt.page_size > 256 || (rt.page_size & (rt.page_size - 1)) ||
-        (rt.kv_dtype != SPEC_DTYPE_FP32 && rt.kv_dtype != SPEC_DTYPE_BF16) || (rt.pass_kernel != 0 && rt.pass_kernel != 1))
+        (rt.kv_dtype != SPEC_DTYPE_FP32 && rt.kv_dtype != SPEC_DTYPE_BF16 && rt.kv_dtype != SPEC_DTYPE_FP16) || (rt.pass_kernel != 0 && rt.pass_kernel != 1))
         return fail(SPEC_ERR_BAD_CONFIG, "spec_init: runtime config out of range");
     int device_count = 0;
     if (cudaGetDeviceCount(&device_count) != cudaSuccess || device_count == 0) {

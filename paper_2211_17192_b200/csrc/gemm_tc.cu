@@ -72,6 +72,15 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
         : "memory");
 }
 
+// The same with an L2 eviction-priority hint.  The weights are read once per pass: marked
+// evict-first they do not push the activations, partial sums and prefetched K,V rows out of L2.
+__device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes
 // long and 128-byte swizzled: 8-row groups are 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
@@ -176,9 +185,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // ring of weight tiles is already streaming while that kernel finishes.
         // Weight tile of k-block kb: in the row-major matrix the box at (kb*64, tile*128);
         // in the tile-major copy the 128 consecutive 128-byte rows of tile (tile, kb).
+        uint64_t stream_once;
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream_once));
         auto load_w = [&](void* dst, int kb, uint64_t* bar) {
-            if (packed) tma_load_2d(dst, &map_w, 0, (tile * k_blocks + kb) * kTileM, bar);
-            else tma_load_2d(dst, &map_w, kb * kTileK, tile * kTileM, bar);
+            if (packed) tma_load_2d_hint(dst, &map_w, 0, (tile * k_blocks + kb) * kTileM, bar, stream_once);
+            else tma_load_2d_hint(dst, &map_w, kb * kTileK, tile * kTileM, bar, stream_once);
         };
         const int total = kb1 - kb0;
         const int ahead = min(total, S::kStages);

@@ -6,7 +6,7 @@
 // out-projection GEMM, norm, FFN-in GEMM, activation, FFN-out GEMM.
 #include <cmath>
 
-#include "model.cuh"
+#include "attn_unit.cuh"
 
 namespace spec {
 namespace {
@@ -193,8 +193,8 @@ __global__ void qkv_kernel(float* __restrict__ qkv, const float* __restrict__ pa
     const int page = page_table[seq[r] * pages_per_seq + p / page_size];
     const size_t block = (static_cast<size_t>(page) * 2 + (is_k ? 0 : 1)) * n_kv_heads + kv_head;
     KV* dst = kv_layer + (block * page_size + p % page_size) * d_head;
-    dst[j] = static_cast<KV>(x1);
-    dst[j + half] = static_cast<KV>(x2);
+    dst[j] = to_cached<KV>(x1);
+    dst[j + half] = to_cached<KV>(x2);
 }
 
 // logits[dst(i)] = table[token[src(i)]] for a table model: grid = (chunks, rows), block = 256.
@@ -330,7 +330,11 @@ int launch_qkv(int n_heads, int n_kv_heads, int d_head, const float2* rope, cons
                int n_rows, float* qkv, const float* partial, int splits, cudaStream_t stream) {
     const dim3 grid(n_heads + 2 * n_kv_heads, n_rows);
     const dim3 block(d_head / 2);
-    if (pool.elem_bytes == 2)
+    if (pool.dtype == SPEC_DTYPE_FP16)
+        return launch_pdl(qkv_kernel<__half>, grid, block, 0, stream, qkv, partial, splits, n_rows, rows.pos, rows.seq, n_heads,
+                          n_kv_heads, d_head, rope, static_cast<__half*>(pool.kv), pool.page_table, pool.pages_per_seq,
+                          pool.page_size);
+    if (pool.dtype == SPEC_DTYPE_BF16)
         return launch_pdl(qkv_kernel<__nv_bfloat16>, grid, block, 0, stream, qkv, partial, splits, n_rows, rows.pos,
                           rows.seq, n_heads, n_kv_heads, d_head, rope, static_cast<__nv_bfloat16*>(pool.kv),
                           pool.page_table, pool.pages_per_seq, pool.page_size);

@@ -54,7 +54,6 @@ namespace spec {
 namespace {
 
 constexpr int kThreads = 512;
-constexpr int kWarps = kThreads / 32;
 constexpr int kStages = 10;                       // even: see the roles of gemm_step
 constexpr int kABytes = 128 * 64 * 2;             // one weight tile
 constexpr int kBBytes = 16 * 64 * 2;              // one term of the activation block (16 rows)
@@ -806,10 +805,10 @@ __device__ void qkv_step(const MegaArgs& a, const Cta& cta, const float* ssq, in
             const int kv_head = is_k ? head - n_heads : head - n_heads - n_kv_heads;
             const size_t block = (static_cast<size_t>(page) * 2 + (is_k ? 0 : 1)) * n_kv_heads + kv_head;
             KV* dst = kv_layer + (block * a.page_size + p % a.page_size) * a.dh + j;
-            dst[0] = static_cast<KV>(y1.x);
-            dst[1] = static_cast<KV>(y1.y);
-            dst[half] = static_cast<KV>(y2.x);
-            dst[half + 1] = static_cast<KV>(y2.y);
+            dst[0] = to_cached<KV>(y1.x);
+            dst[1] = to_cached<KV>(y1.y);
+            dst[half] = to_cached<KV>(y2.x);
+            dst[half + 1] = to_cached<KV>(y2.y);
         }
     }
 }
@@ -1153,6 +1152,10 @@ int pass_scratch_init(PassScratch& s, const Model* models, int n_models, std::ve
     ctas = std::min(ctas, other);
     SPEC_TRY_STATUS(resident_ctas<__nv_bfloat16, 128>(&other));
     ctas = std::min(ctas, other);
+    SPEC_TRY_STATUS(resident_ctas<__half, 64>(&other));
+    ctas = std::min(ctas, other);
+    SPEC_TRY_STATUS(resident_ctas<__half, 128>(&other));
+    ctas = std::min(ctas, other);
     if (ctas < 1) return SPEC_OK;
     size_t d = 0, q = 0, part = 0, attn = 0, out = 0, tiles_most = 0;
     bool any = false;
@@ -1306,9 +1309,11 @@ int launch_pass(const PassScratch& s, const Model& m, int which, const RowMeta& 
     a.count_total = s.count_total[which];
     a.trace = trace;
     a.trace_capacity = trace_capacity;
-    const bool kv16 = m.kv_elem_bytes == 2;
-    if (c.d_head == 64) return kv16 ? launch_variant<__nv_bfloat16, 64>(a, s.ctas, stream) : launch_variant<float, 64>(a, s.ctas, stream);
-    return kv16 ? launch_variant<__nv_bfloat16, 128>(a, s.ctas, stream) : launch_variant<float, 128>(a, s.ctas, stream);
+    if (m.kv_dtype == SPEC_DTYPE_FP16)
+        return c.d_head == 64 ? launch_variant<__half, 64>(a, s.ctas, stream) : launch_variant<__half, 128>(a, s.ctas, stream);
+    if (m.kv_dtype == SPEC_DTYPE_BF16)
+        return c.d_head == 64 ? launch_variant<__nv_bfloat16, 64>(a, s.ctas, stream) : launch_variant<__nv_bfloat16, 128>(a, s.ctas, stream);
+    return c.d_head == 64 ? launch_variant<float, 64>(a, s.ctas, stream) : launch_variant<float, 128>(a, s.ctas, stream);
 }
 
 void pass_scratch_release(PassScratch& s) {

@@ -27,6 +27,7 @@ struct Model {
     void* kv = nullptr;
     size_t layer_stride = 0;
     int kv_elem_bytes = 4;
+    int kv_dtype = SPEC_DTYPE_FP32;  // SPEC_DTYPE_FP32 / FP16 / BF16
     const float2* rope_table = nullptr;  // Llama: (cos, sin) [positions][d_head / 2], owned
 
     // Encoder-decoder (T5) only.  The bias tables are the bucket tables expanded by
@@ -102,7 +103,8 @@ int gemm_tc_take_error();
 // (sequence slot, position / page_size) to a pool page.
 struct KvPool {
     void* kv;
-    int elem_bytes;  // 4 (fp32) or 2 (bf16)
+    int elem_bytes;  // 4 (fp32) or 2 (fp16, bf16)
+    int dtype;       // SPEC_DTYPE_*
     const int32_t* page_table;
     int pages_per_seq;
     int page_size;

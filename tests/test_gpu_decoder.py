@@ -76,6 +76,24 @@ def test_bf16_kv_cache_option_stays_close():
     eng.close()
 
 
+def test_sixteen_bit_kv_rows_on_a_wide_block():
+    """One block of the 7B width (32 query / 8 KV heads of 128): fp16 K,V rows, the default for bf16
+    models, stay inside the parity bar like fp32 rows; bf16 rows keep 8 bits and are looser."""
+    cfg, w = _pair("llama7b_target", n_layers=1, vocab=4096, d_ff=1024)
+    tokens = workloads.make_prompt(3, 96, cfg["vocab"])
+    ref = Decoder(cfg, w).forward_full(tokens)
+    errs = {}
+    for kv in ("fp32", "fp16", "bf16"):
+        eng = binding.Engine(cfg, w, max_batch=1, max_len=128, page_size=32, max_gamma=3, kv_dtype=kv)
+        eng.reset()
+        got = np.concatenate([eng.forward_logits(0, tokens[None, :64]).cpu().numpy()[0],
+                              eng.forward_logits(0, tokens[None, 64:96]).cpu().numpy()[0]])
+        errs[kv] = np.abs(got - ref).max()
+        eng.close()
+    assert errs["fp32"] <= BF16_ABS and errs["fp16"] <= BF16_ABS, errs
+    assert errs["fp16"] < errs["bf16"] < 1e-1, errs
+
+
 def test_batched_sequences_are_independent_and_page_size_is_invisible():
     cfg, w = _pair("llama_test_target")
     seqs = [workloads.make_prompt(10 + b, 30, cfg["vocab"]) for b in range(3)]
