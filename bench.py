@@ -262,12 +262,13 @@ class GenerationWorkload:
     def description(self):
         return {"workload": self.name, "target": self.target_name, "draft": self.draft_name, "batch": self.batch,
                 "prompt_len": self.prompt_len, "n_new": self.n_new, "gamma": self.gamma,
-                "temperature": self.temperature, "kv_dtype": "fp32",
+                "temperature": self.temperature, "kv_dtype": "fp16" if self.tcfg["dtype"] == "bf16" else "fp32",
                 **({"target_layers_override": self.layers} if self.layers else {}),
                 "l2": "one pass streams the target's weights (>> 126 MB L2) from HBM",
                 "parallelism": "replicas"}
 
-    def prepare(self, rank, device, iterations):
+    def prepare(self, rank, device, iterations, weights=None):
+        """`weights`: (target, draft) tensors of another workload on the same pair of shapes (not drawn again)."""
         import torch
         from paper_2211_17192_b200 import binding, workloads
         self.torch, self.binding, self.device = torch, binding, device
@@ -276,8 +277,7 @@ class GenerationWorkload:
             self.tcfg = workloads.scaled_config(self.tcfg, n_layers=self.layers)
         self.dcfg = workloads.model_config(self.draft_name)
         self.dtype = "bf16" if self.tcfg["dtype"] == "bf16" else "f32"
-        self.tw = gpu_weights(self.tcfg, 100 + rank, device)
-        self.dw = gpu_weights(self.dcfg, 200 + rank, device)
+        self.tw, self.dw = weights if weights else (gpu_weights(self.tcfg, 100 + rank, device), gpu_weights(self.dcfg, 200 + rank, device))
         grow = max(self.n_new, iterations * (self.gamma + 1) + 64)
         top_gamma = max(self.gamma, self.adaptive_gamma_max, 1)
         self.max_len = self.prompt_len + grow + top_gamma + 2
@@ -285,6 +285,16 @@ class GenerationWorkload:
                                      page_size=64, max_gamma=top_gamma)
         self.prompts = [workloads.make_prompt(1000 * rank + b, self.prompt_len, self.tcfg["vocab"]) for b in range(self.batch)]
         self.budget_tokens = grow
+        self.kv_elem_bytes = 2 if self.engine.kv_dtype in ("fp16", "bf16") else 4
+
+    def close(self):
+        self.engine.close()
+        self.engine = None
+
+    def kv_bytes(self, context):
+        """K,V bytes one target pass reads: the cached rows of every sequence, in the cache's element type."""
+        c = self.tcfg
+        return self.batch * context * 2 * c["n_layers"] * c["n_kv_heads"] * c["d_head"] * self.kv_elem_bytes
 
     def launches_per_iteration(self):
         # per block: 4 GEMMs, 2 norms, RoPE/append, attention, activation (+ the combine kernel when the
@@ -342,6 +352,7 @@ class GenerationWorkload:
         for which in ((0,) if stateless else (0, 1)):
             for c0 in range(0, tok.shape[1], chunk):
                 eng.forward_logits(which, tok[:, c0:c0 + chunk])
+        self.pass_context = self.prompt_len - 1
         return {"target_1row_ms": timed(0, 1), "target_rows_ms": timed(0, self.gamma + 1), "draft_1row_ms": timed(1, 1)}
 
     def gemm_roofline(self, rows):
@@ -376,13 +387,16 @@ class GenerationWorkload:
                 sweep()
             graph.replay()
             stream.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            graph.replay()
-            b.record(stream)
-            stream.synchronize()
+            samples = []
+            for _ in range(7):  # the median of several replays, each timed on its own
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                graph.replay()
+                b.record(stream)
+                stream.synchronize()
+                samples.append(a.elapsed_time(b))
         nbytes = sum(t.numel() * t.element_size() for _, t in mats)
-        ms = a.elapsed_time(b)
+        ms = statistics.median(samples)
         del packed
         torch.cuda.empty_cache()
         return nbytes, ms, len(mats)
@@ -437,7 +451,7 @@ class EncDecWorkload(GenerationWorkload):
         d["l2"] = "one pass streams the target decoder's weights (>> 126 MB L2) from HBM"
         return d
 
-    def prepare(self, rank, device, iterations):
+    def prepare(self, rank, device, iterations, weights=None):
         import torch
         from paper_2211_17192_b200 import binding, workloads
         self.torch, self.binding, self.device = torch, binding, device
@@ -455,6 +469,7 @@ class EncDecWorkload(GenerationWorkload):
                                      page_size=64, max_gamma=top_gamma, max_src_len=self.prompt_len)
         self.prompts = [workloads.make_prompt(1000 * rank + b, self.prompt_len, self.tcfg["vocab"]) for b in range(self.batch)]
         self.budget_tokens = grow
+        self.kv_elem_bytes = 2 if self.engine.kv_dtype in ("fp16", "bf16") else 4
 
     def launches_per_iteration(self):
         # per decoder block: 7 GEMMs, 3 norms, K/V append, cross-attention queries, 2 attentions, activation
@@ -463,7 +478,7 @@ class EncDecWorkload(GenerationWorkload):
 
     def kv_bytes(self, context):
         c = self.tcfg
-        per_position = 2 * c["n_layers"] * c["n_kv_heads"] * c["d_head"] * 4
+        per_position = 2 * c["n_layers"] * c["n_kv_heads"] * c["d_head"] * self.kv_elem_bytes
         return self.batch * (context + self.prompt_len) * per_position  # self-attention rows + cross-attention rows
 
     def pass_times(self, repeats=20):
@@ -607,7 +622,9 @@ def run_reference(args, wl):
     out = {
         "impl": "reference", "metric": "generated tokens/s", "value": value, "unit": "tokens/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1000.0 * dt / args.steps,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if getattr(wl, "tcfg", {}).get("d_model", 0) >= 2048 else "f64",  # what the oracle computes in here
+        "data": "synthetic",
         "config": wl.description(),
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cpu_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -671,13 +688,61 @@ def run_sampler(args, wl, torch, device, local, barrier):
                 clocks=clock_info, extras=extras)
 
 
+def measure_pair(wl, analysis, peak, warmup, steps):
+    """Tokens/s, target-only tokens/s, acceptance, cost ratios and the target pass against the HBM
+    roofline for one prepared generation workload."""
+    tokens, ms, stats = wl.timed_decode(warmup, steps, wl.gamma)
+    base_tokens, base_ms, _ = wl.timed_decode(warmup, steps, 0)  # target-only, same kernels
+    times = wl.pass_times(10)
+    alpha = stats["tests_passed"] / max(1, stats["tests_evaluated"])
+    tpi = stats["tokens"] / max(1, stats["iterations"])
+    pass_bytes = weight_stream_bytes(wl.tcfg) + wl.kv_bytes(wl.pass_context)
+    gbs = pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9
+    return {"workload": wl.name, "batch": wl.batch, "gamma": wl.gamma, "iterations": steps,
+            "tokens_per_s": tokens / (ms / 1e3), "target_only_tokens_per_s": base_tokens / (base_ms / 1e3),
+            "speedup_vs_target_only": (tokens / ms) / (base_tokens / base_ms), "alpha": alpha,
+            "c": times["draft_1row_ms"] / times["target_1row_ms"], "kappa": times["target_rows_ms"] / times["target_1row_ms"],
+            "generalised_closed_form": analysis.generalised_speedup(tpi, times["target_1row_ms"], times["target_rows_ms"],
+                                                                    times["draft_1row_ms"], wl.gamma),
+            "pass_ms": times, "verify_pass": {"bytes": pass_bytes, "gbs": gbs, "frac": gbs / peak}}
+
+
+def sampler_point(torch, device):
+    """The standalone sampler workload (batch 64 x 8 positions x vocabulary 32000) in the same run:
+    microseconds per call (CUDA graph of 60 calls over three rotating input sets, events) and the
+    fraction of the measured HBM rate."""
+    wl = SamplerWorkload()
+    wl.prepare(0, device)
+    stream = torch.cuda.Stream(device)
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            wl.step(i)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(60):
+                wl.step(i)
+        graph.replay()
+        stream.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        graph.replay()
+        b.record(stream)
+        stream.synchronize()
+    us = 1e3 * a.elapsed_time(b) / 60
+    peak, kind = load_peaks()
+    gbs = wl.algorithmic_bytes() / (us / 1e6) / 1e9
+    return {"workload": wl.name, "us_per_call": us, "gbs": gbs, "frac": gbs / peak, "peak_kind": f"of {kind}"}
+
+
 def run_generation(args, wl, torch, device, local, barrier):
     """Timed region: K iterations of Algorithm 1 (gamma draft passes, one target pass
     over gamma+1 rows, speculative sampling, commit and roll-back), replayed as a
     CUDA graph per iteration by the library and timed with events on its stream."""
     from oracle import analysis  # closed forms only, for the report (rank 0)
     rank = int(os.environ.get("RANK", "0"))
-    wl.prepare(rank, device, args.warmup + args.steps)
+    long_steps = max(200, args.steps)  # (also measured: a stretch long enough for the acceptance rate to settle)
+    wl.prepare(rank, device, args.warmup + long_steps)
     clocks = ClockSampler(local)
     clocks.start()
     time.sleep(0.15)
@@ -718,12 +783,34 @@ def run_generation(args, wl, torch, device, local, barrier):
                           "generalised": analysis.generalised_speedup(s_tpi, times["target_1row_ms"], times["target_rows_ms"],
                                                                       times["draft_1row_ms"], wl.gamma)})
         wl.engine.set_imposed_acceptance(None)
-        if hasattr(wl, "kv_bytes"):
-            kv_bytes = wl.kv_bytes(wl.pass_context)
-        else:
-            kv_bytes = wl.batch * wl.prompt_len * 2 * wl.tcfg["n_layers"] * wl.tcfg["n_kv_heads"] * wl.tcfg["d_head"] * 4
+        kv_bytes = wl.kv_bytes(wl.pass_context)
         pass_bytes = weight_stream_bytes(wl.tcfg) + kv_bytes
+        pass_gbs = pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9
+        long_tokens, long_ms, long_stats = wl.timed_decode(args.warmup, long_steps, wl.gamma)
+        # the other configurations of the scope, measured in this same run (short: 30 iterations each)
+        others = []
+        if args.workload == "llama7b" and args.configs and not args.layers:
+            for batch, gamma in ((16, 4), (32, 6)):
+                other = GenerationWorkload(f"llama7b_160m_b{batch}_g{gamma}", wl.target_name, wl.draft_name, batch, wl.prompt_len,
+                                           wl.n_new, gamma, wl.temperature)
+                other.prepare(rank, device, 3 + 30, weights=(wl.tw, wl.dw))
+                others.append(measure_pair(other, analysis, peak, 3, 30))
+                other.close()
+            wl.close()
+            del wl.tw, wl.dw
+            torch.cuda.empty_cache()
+            for other in (GenerationWorkload("gpt97m_6m_b1", "gpt97m_target", "gpt6m_draft", 1, 128, 512, 5, wl.temperature),
+                          EncDecWorkload("t5xxl_small_b1_g5", "t5xxl_target", "t5small_draft", 1, 512, 128, 5, wl.temperature)):
+                other.prepare(rank, device, 3 + 30)
+                others.append(measure_pair(other, analysis, peak, 3, 30))
+                other.close()
+                del other.tw, other.dw
+                torch.cuda.empty_cache()
+            others.append(sampler_point(torch, device))
         extras = {
+            "value_long": {"tokens_per_s": long_tokens / (long_ms / 1e3), "iterations": long_steps,
+                           "alpha": long_stats["tests_passed"] / max(1, long_stats["tests_evaluated"])},
+            "configs": others,
             "speedup_vs_target_only": (tokens / elapsed_ms) / (base_tokens / base_ms),
             "target_only_tokens_per_s": base_tokens / (base_ms / 1e3),
             "alpha": alpha, "tokens_per_iteration": tok_per_iter, "c": c,
@@ -743,16 +830,23 @@ def run_generation(args, wl, torch, device, local, barrier):
                                times["draft_1row_ms"], g_)) if 0.0 < alpha < 1.0 else None},
             "imposed_acceptance_sweep": sweep,
             **({"adaptive_gamma": wl.adaptive(wl.adaptive_gamma_max)} if wl.adaptive_gamma_max else {}),
-            "verify_pass": {"bytes": pass_bytes, "ms": times["target_rows_ms"],
-                            "gbs": pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9,
-                            "frac": pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9 / peak,
-                            "note": "weights + fp32 K,V rows read (context; for encoder-decoders also the source), one pass over gamma+1 rows, graph replays timed with events"},
-            "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbs": achieved / 8000.0,
-                         "traffic": 1.026 * nbytes / n_mats,
-                         "traffic_note": "dram read+write bytes per launch: algorithmic bytes x 1.026, the ratio the ncu "
-                                         "capture of the four GEMMs of a 7B-shaped block shows (363.6 MB vs 354.4 MB; "
+            # the quantity the metric names: one target pass over gamma+1 rows, weights + the cached K,V rows it
+            # reads, against the HBM copy rate (the whole pass: GEMM chain, attention and the small kernels between)
+            "roofline": {"bound": "hbm", "kernel": "target pass over gamma+1 rows (gemm_tc_kernel chain, attention, small kernels)",
+                         "achieved": pass_gbs, "peak": peak, "unit": "GB/s", "frac": pass_gbs / peak,
+                         "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbs": pass_gbs / 8000.0,
+                         "algorithmic_bytes_per_pass": pass_bytes, "weight_bytes": weight_stream_bytes(wl.tcfg),
+                         "kv_bytes": kv_bytes, "ms_per_pass": times["target_rows_ms"],
+                         "traffic": None,
+                         "traffic_note": "not captured for the whole pass; from profile: the four GEMMs of a 7B-shaped block "
+                                         "move 363.6 MB of DRAM traffic for 354.4 MB of weights (x 1.026, "
                                          "profiles/ncu_gemm_tc_llama7b_layer.txt)",
+                         "note": "weights + K,V rows of the context in the cache's element type (for encoder-decoders also "
+                                 "the source rows), one pass over gamma+1 rows, graph replays timed with events on the "
+                                 "library's stream",
+                         "gemm_kernel": {
+                         "kernel": "gemm_tc_kernel", "achieved": achieved, "frac": achieved / peak,
+                         "frac_of_nominal_8tbs": achieved / 8000.0,
                          "algorithmic_bytes_per_launch": nbytes / n_mats,
                          # the same sweep against the tensor pipes: where rows approach the ridge (about 216-262 rows)
                          # the GEMMs stop being purely bandwidth-bound; two MMAs per k-step (split activations)
@@ -765,7 +859,7 @@ def run_generation(args, wl, torch, device, local, barrier):
                          "launch_us": 1e3 * gemm_ms / n_mats,
                          "note": f"all {n_mats} weight matrices of the target once at {rows} rows through spec_linear_partials "
                                  "(the GEMM kernel alone, tile-major weights, one launch per matrix back to back), "
-                                 "CUDA graph, events on its stream"},
+                                 "CUDA graph, median of 7 replays, events on its stream"}},
         }
     launches = wl.launches_per_iteration() * args.steps
     return dict(tokens=tokens, elapsed_ms=elapsed_ms, e2e_tokens=e2e_tokens, e2e_s=e2e_s, launches=launches,
@@ -789,6 +883,8 @@ def main():
     ap.add_argument("--top-p", type=float, default=1.0, help="sampler workload: nucleus standardisation of both models")
     ap.add_argument("--adaptive-gamma-max", type=int, default=0,
                     help="also report decoding with gamma chosen by the library burst by burst, up to this value")
+    ap.add_argument("--no-configs", dest="configs", action="store_false",
+                    help="llama7b workload: skip the other configurations (batch 16 and 32, GPT 97M/6M, T5-XXL/small, sampler)")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for cpu_baseline")
     args = ap.parse_args()

@@ -172,16 +172,25 @@ __device__ __forceinline__ void stage_tile(const float* tile, int n_valid, float
         cp_async16(dst + row * (DH + 4) + 4 * c, tile + static_cast<size_t>(valid ? row : 0) * DH + 4 * c, valid);
     }
 }
-// (16-bit rows: converted on the way into shared memory)
+// (16-bit rows: converted on the way into shared memory; a lane requests all its 16-byte chunks of
+// the tile before it converts the first, so that they are in flight together)
 template <int DH, typename KV16>
 __device__ __forceinline__ void stage_tile(const KV16* tile, int n_valid, float* dst, int lane) {
     constexpr int kChunks = DH / 8;
-    for (int i = lane; i < kTileKeys * kChunks; i += 32) {
-        const int row = i / kChunks, c = i % kChunks;
+    constexpr int kPerLane = kTileKeys * kChunks / 32;
+    uint4 raw[kPerLane];
+#pragma unroll
+    for (int j = 0; j < kPerLane; ++j) {
+        const int i = lane + 32 * j, row = i / kChunks, c = i % kChunks;
+        raw[j] = *reinterpret_cast<const uint4*>(tile + static_cast<size_t>(row < n_valid ? row : 0) * DH + 8 * c);
+    }
+#pragma unroll
+    for (int j = 0; j < kPerLane; ++j) {
+        const int i = lane + 32 * j, row = i / kChunks, c = i % kChunks;
         float v[8];
-        if (row < n_valid) {
-            KvLoad<KV16>::load(tile + static_cast<size_t>(row) * DH + 8 * c, v);
-        } else {
+        const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+        KvLoad<KV16>::template convert_n<8>(w, v);
+        if (row >= n_valid) {
 #pragma unroll
             for (int e = 0; e < 8; ++e) v[e] = 0.0f;
         }

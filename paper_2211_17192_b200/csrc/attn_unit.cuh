@@ -57,6 +57,14 @@ struct KvLoad<__nv_bfloat16> {
         }
     }
     template <int N>
+    __device__ static __forceinline__ void convert_n(const uint32_t* w, float* out) {  // N / 2 packed words
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i) {
+            out[2 * i] = __uint_as_float(w[i] << 16);
+            out[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+    template <int N>
     __device__ static __forceinline__ void load_n(const __nv_bfloat16* p, float* out) {
         if (N == 4) {
             const uint2 t = *reinterpret_cast<const uint2*>(p);
@@ -69,6 +77,16 @@ struct KvLoad<__nv_bfloat16> {
     }
 };
 
+// fp16 -> fp32 with integer operations and one multiplication by a power of two (exact for zeros,
+// subnormals and normals; cached rows are finite, see to_cached): plain arithmetic that the compiler
+// schedules freely around the loads, unlike an opaque conversion instruction.
+__device__ __forceinline__ float2 half2_bits_to_float2(uint32_t w) {
+    const float lo = __uint_as_float((w & 0x7fffu) << 13) * 0x1p112f;
+    const float hi = __uint_as_float((w >> 3) & 0x0fffe000u) * 0x1p112f;
+    return make_float2(__uint_as_float(__float_as_uint(lo) | ((w & 0x8000u) << 16)),
+                       __uint_as_float(__float_as_uint(hi) | (w & 0x80000000u)));
+}
+
 template <>
 struct KvLoad<__half> {
     static constexpr int kVec = 8;
@@ -77,7 +95,16 @@ struct KvLoad<__half> {
         const uint32_t w[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+            const float2 f = half2_bits_to_float2(w[i]);
+            out[2 * i] = f.x;
+            out[2 * i + 1] = f.y;
+        }
+    }
+    template <int N>
+    __device__ static __forceinline__ void convert_n(const uint32_t* w, float* out) {  // N / 2 packed words
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i) {
+            const float2 f = half2_bits_to_float2(w[i]);
             out[2 * i] = f.x;
             out[2 * i + 1] = f.y;
         }
@@ -86,11 +113,10 @@ struct KvLoad<__half> {
     __device__ static __forceinline__ void load_n(const __half* p, float* out) {
         if (N == 4) {
             const uint2 t = *reinterpret_cast<const uint2*>(p);
-            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&t.x)), b = __half22float2(*reinterpret_cast<const __half2*>(&t.y));
+            const float2 a = half2_bits_to_float2(t.x), b = half2_bits_to_float2(t.y);
             out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
         } else {
-            const uint32_t t = *reinterpret_cast<const uint32_t*>(p);
-            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&t));
+            const float2 a = half2_bits_to_float2(*reinterpret_cast<const uint32_t*>(p));
             out[0] = a.x; out[1] = a.y;
         }
     }
@@ -194,19 +220,45 @@ __device__ __forceinline__ void attend_slice(const float* __restrict__ qkv, int 
             // partial dot products of all 32 keys over this lane's elements ...
             float pd[32];
             const KV* kt = tile + lane * PER_LANE;
+            if constexpr (sizeof(KV) == 2) {
+                // 16-bit rows: every key's raw words are requested before the first one is converted (the
+                // conversion arithmetic between a load and the next would otherwise keep few loads in flight)
+                uint32_t raw[32][PER_LANE / 2];
 #pragma unroll
-            for (int k = 0; k < 32; ++k) {
-                float kv[PER_LANE];
-                if (k < in_tile) {
-                    KvLoad<KV>::template load_n<PER_LANE>(kt + static_cast<size_t>(k) * DH, kv);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < PER_LANE; ++i) kv[i] = 0.0f;
+                for (int k = 0; k < 32; ++k) {
+                    const uint32_t* src = reinterpret_cast<const uint32_t*>(kt + static_cast<size_t>(k < in_tile ? k : 0) * DH);
+                    if (PER_LANE == 4) {
+                        const uint2 t = *reinterpret_cast<const uint2*>(src);
+                        raw[k][0] = t.x;
+                        raw[k][PER_LANE / 2 - 1] = t.y;
+                    } else {
+                        raw[k][0] = *src;
+                    }
                 }
-                float d = 0.0f;
 #pragma unroll
-                for (int i = 0; i < PER_LANE; ++i) d = fmaf(qv[i], kv[i], d);
-                pd[k] = d;
+                for (int k = 0; k < 32; ++k) {
+                    float kv[PER_LANE];
+                    KvLoad<KV>::template convert_n<PER_LANE>(raw[k], kv);
+                    float d = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < PER_LANE; ++i) d = fmaf(qv[i], kv[i], d);
+                    pd[k] = k < in_tile ? d : 0.0f;
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 32; ++k) {
+                    float kv[PER_LANE];
+                    if (k < in_tile) {
+                        KvLoad<KV>::template load_n<PER_LANE>(kt + static_cast<size_t>(k) * DH, kv);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < PER_LANE; ++i) kv[i] = 0.0f;
+                    }
+                    float d = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < PER_LANE; ++i) d = fmaf(qv[i], kv[i], d);
+                    pd[k] = d;
+                }
             }
             // ... summed over the lanes by a butterfly that halves the live values
             // at every step: lane l ends with the full score of key l
@@ -238,11 +290,37 @@ __device__ __forceinline__ void attend_slice(const float* __restrict__ qkv, int 
                         if (kEarlyV && j0 == 0) {
 #pragma unroll
                             for (int i = 0; i < PER_LANE; ++i) vv[jj][i] = v_first[kEarlyV ? jj : 0][i];
-                        } else if (j0 + jj < in_tile) {
-                            KvLoad<KV>::template load_n<PER_LANE>(vt + static_cast<size_t>(j0 + jj) * DH, vv[jj]);
-                        } else {
+                        } else if constexpr (sizeof(KV) != 2) {
+                            if (j0 + jj < in_tile) {
+                                KvLoad<KV>::template load_n<PER_LANE>(vt + static_cast<size_t>(j0 + jj) * DH, vv[jj]);
+                            } else {
 #pragma unroll
-                            for (int i = 0; i < PER_LANE; ++i) vv[jj][i] = 0.0f;
+                                for (int i = 0; i < PER_LANE; ++i) vv[jj][i] = 0.0f;
+                            }
+                        }
+                    }
+                    if constexpr (sizeof(KV) == 2) {  // raw words of the whole batch first, then the conversions
+                        if (!(kEarlyV && j0 == 0)) {
+                            uint32_t raw[kVBatch][PER_LANE / 2];
+#pragma unroll
+                            for (int jj = 0; jj < kVBatch; ++jj) {
+                                const uint32_t* src = reinterpret_cast<const uint32_t*>(vt + static_cast<size_t>(j0 + jj < in_tile ? j0 + jj : 0) * DH);
+                                if (PER_LANE == 4) {
+                                    const uint2 t = *reinterpret_cast<const uint2*>(src);
+                                    raw[jj][0] = t.x;
+                                    raw[jj][PER_LANE / 2 - 1] = t.y;
+                                } else {
+                                    raw[jj][0] = *src;
+                                }
+                            }
+#pragma unroll
+                            for (int jj = 0; jj < kVBatch; ++jj) {
+                                KvLoad<KV>::template convert_n<PER_LANE>(raw[jj], vv[jj]);
+                                if (j0 + jj >= in_tile) {
+#pragma unroll
+                                    for (int i = 0; i < PER_LANE; ++i) vv[jj][i] = 0.0f;
+                                }
+                            }
                         }
                     }
 #pragma unroll
