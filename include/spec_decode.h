@@ -19,6 +19,11 @@
  *     not synchronise unless stated.
  *   - There is no CPU fallback: without a CUDA device every compute entry
  *     point fails with SPEC_ERR_CUDA.
+ *   - The library reads one environment variable, once per process:
+ *     SPEC_NO_PDL=1 launches every kernel fully serialised instead of with
+ *     programmatic dependent launch (same kernels, same results, slower; for
+ *     debugging launch-order problems).  Nothing else in the environment
+ *     changes what runs.
  */
 #ifndef SPEC_DECODE_H
 #define SPEC_DECODE_H
@@ -38,7 +43,8 @@ typedef enum spec_status {
     SPEC_ERR_CAPACITY = -4,       /* prompt + n_new + gamma exceeds max_len / max_positions */
     SPEC_ERR_CUDA = -5,           /* a CUDA call failed (message has the CUDA error) */
     SPEC_ERR_DEVICE_TIMEOUT = -6, /* a bounded device-side wait expired */
-    SPEC_ERR_NONFINITE = -7       /* non-finite logits were seen */
+    SPEC_ERR_NONFINITE = -7       /* spec_generate / spec_step: a model produced a NaN or +inf logit (or a row with
+                                     no finite logit) in the iterations just run */
 } spec_status;
 
 /* Message for the calling thread's most recent failure ("" if none).  The
@@ -46,8 +52,8 @@ typedef enum spec_status {
 const char* spec_last_error(void);
 
 /* ------------------------------------------------------------------------- *
- * Speculative sampling (Section 2.3; Algorithm 1 from "determine the number
- * of accepted guesses" to "return").
+ * Speculative sampling (Section 2.3; Algorithm 1 from the accept tests to the
+ * returned token).
  *
  * For each of `batch` independent sequences, given the target model's logits
  * for the gamma+1 prefixes, the draft model's logits for the gamma prefixes it
@@ -61,8 +67,11 @@ const char* spec_last_error(void);
  *   smallest k whose running weight sum exceeds u times the total).  If the
  *   residual sums to zero, t is drawn from p_{n+1} unmodified.
  * At T = 0 no uniform is used and draft_logits is not read: x_i is accepted
- * iff it equals argmax p_i (x_i is assumed to be the draft's own argmax), and
- * t = argmax p_{n+1}.
+ * iff it equals argmax p_i, and t = argmax p_{n+1}.  (For a guess that is the
+ * draft's own argmax, as x_i ~ q_i gives, this is Algorithm 1's test between two
+ * one-hot distributions; for any other guess the printed test divides by
+ * q_i(x_i) = 0 and decides nothing: the library's rule there is the same "iff it
+ * is the target's argmax".)
  *
  * All pointers are DEVICE pointers, caller-owned:
  *   target_logits [batch, gamma+1, vocab] fp32, row-major, dense
@@ -353,6 +362,8 @@ typedef struct spec_stats {
     int64_t draft_passes;     /* batched forward passes of M_q inside the decode loop */
     double prefill_ms;        /* device time of the prompt pass */
     double decode_ms;         /* device time of the decode loop */
+    int64_t accepted_histogram[65]; /* [n]: runs of Algorithm 1 that accepted exactly n guesses (n <= gamma <= 64):
+                                 for i.i.d. acceptance the capped geometric law behind Eq. 1 */
 } spec_stats;
 
 /* Creates a context for a target model and (optionally, draft_cfg == NULL for
@@ -593,6 +604,17 @@ int spec_linear_partials(const float* x, const void* w_packed, int rows, int n_o
 int spec_linear(const float* x, const void* w, int w_dtype, int rows, int n_out, int k, int path,
                 float* y, void* workspace, size_t workspace_bytes, void* stream);
 int spec_device_error(void);
+
+/* Failure-path drill (no counterpart in the paper).  Every wait inside the library's kernels on
+ * a barrier or a flag is bounded: when it runs out the kernel records a code, frees the tensor
+ * memory it holds and returns, and the next synchronising call of the library reports
+ * SPEC_ERR_DEVICE_TIMEOUT instead of hanging the GPU.  This call exercises that path without
+ * breaking anything: it launches the tensor-core GEMM kernel on one tile with its producer
+ * switched off (nothing is requested from memory, so nothing is in flight when the CTA gives
+ * up) and a limit of 4096 polls, waits for it, and returns SPEC_ERR_DEVICE_TIMEOUT if the kernel
+ * reported the expired wait as it should (SPEC_ERR_CUDA if it did not).  The device error flag
+ * is clear afterwards and the context stays usable.  Synchronises `stream`. */
+int spec_timeout_drill(void* stream);
 
 #ifdef __cplusplus
 }

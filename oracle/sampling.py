@@ -196,7 +196,8 @@ def lenient_greedy_accepts(target_row, x, lenience):
 
 
 def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature, lenience=1.0, top_k=0, top_p=1.0):
-    """Algorithm 1 from "determine the number of accepted guesses" to the end.
+    """Algorithm 1 from the accept tests to the returned token (everything after the
+    target's parallel pass).
 
     target_logits [gamma+1, V]: row i-1 gives p_i (i = 1..gamma+1).
     draft_logits  [gamma, V]:   row i-1 gives q_i, from which x_i was drawn.
@@ -225,6 +226,16 @@ def verify_step(target_logits, draft_logits, draft_tokens, uniforms, temperature
             accepted, slack = lenient_greedy_accepts(tl[i], x, lenience)
             accept_margin = min(accept_margin, slack)
             if not accepted:
+                n = i
+                break
+            continue
+        if temperature == 0:
+            # Both standardised distributions are one-hot (Section 2.2).  A guess drawn from q_i is
+            # q_i's maximum, and the accept test then passes exactly when it is p_i's maximum too.
+            # A guess that is NOT q_i's maximum cannot come from x ~ q_i: the printed test reads
+            # r > p(x) / 0 there and decides nothing.  Reading: at T = 0 a guess is accepted iff it
+            # is the target's (lowest-index) maximum, whatever the draft's logits say.
+            if p[i][x] != 1.0:
                 n = i
                 break
             continue
@@ -306,6 +317,8 @@ def verify_trials(target_logits, draft_logits, draft_tokens, uniforms, temperatu
         x = xs[:, i]
         if temperature == 0 and lenience < 1.0:
             rejected = ~(tl[i][x] - tl[i].max() - np.log(lenience) >= 0.0)
+        elif temperature == 0:
+            rejected = p[i][x] != 1.0  # (see verify_step: accepted iff the guess is the target's maximum)
         else:
             rejected = us[:, i] * lenience * q[i][x] > p[i][x]
         first = undecided & rejected

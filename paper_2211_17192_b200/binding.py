@@ -327,7 +327,13 @@ class _RuntimeCfg(ctypes.Structure):
 class _Stats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in ("iterations", "tokens", "tests_evaluated", "tests_passed",
                                               "target_passes", "draft_passes")] + \
-               [("prefill_ms", ctypes.c_double), ("decode_ms", ctypes.c_double)]
+               [("prefill_ms", ctypes.c_double), ("decode_ms", ctypes.c_double), ("accepted_histogram", ctypes.c_int64 * 65)]
+
+
+def _stats_dict(st):
+    d = {name: getattr(st, name) for name, _ in _Stats._fields_}
+    d["accepted_histogram"] = list(st.accepted_histogram)
+    return d
 
 
 _ARCH = {"gpt": 0, "llama": 1, "t5": 2, "bigram": 3, "copy": 4}
@@ -491,7 +497,7 @@ class Engine:
         left = ctypes.c_int()
         st = _Stats()
         _check(lib().spec_step(self._ctx, iterations, ctypes.byref(left), ctypes.byref(st)))
-        return left.value, {name: getattr(st, name) for name, _ in _Stats._fields_}
+        return left.value, _stats_dict(st)
 
     def read_tokens(self):
         batch, n_new = self._session
@@ -515,7 +521,7 @@ class Engine:
         _check(lib().spec_generate(self._ctx, flat.ctypes.data, lens.ctypes.data, stride, batch, n_new, gamma,
                                    float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF, out.ctypes.data,
                                    ctypes.byref(st)))
-        return out, {name: getattr(st, name) for name, _ in _Stats._fields_}
+        return out, _stats_dict(st)
 
     def generate_adaptive(self, prompts, n_new, gamma_max, temperature, seed, burst=4):
         """`generate` with gamma chosen by the library burst by burst (`spec_generate_adaptive`).
@@ -541,7 +547,7 @@ class Engine:
                                         float(temperature), int(seed) & 0xFFFFFFFFFFFFFFFF, int(burst), out.ctypes.data,
                                         ctypes.byref(st), trace.ctypes.data, capacity, ctypes.byref(n_bursts)))
         pairs = [(int(trace[2 * i]), int(trace[2 * i + 1])) for i in range(min(n_bursts.value, capacity // 2))]
-        return out, {name: getattr(st, name) for name, _ in _Stats._fields_}, pairs
+        return out, _stats_dict(st), pairs
 
     def set_gamma(self, gamma):
         """Number of guesses per iteration for the rest of the generation in progress (`spec_set_gamma`)."""

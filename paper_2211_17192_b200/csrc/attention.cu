@@ -20,7 +20,6 @@
 // query; attention_combine_kernel merges the key slices and emits the
 // out-projection's input (fp32 and/or split into two bf16 terms).
 #include <cfloat>
-#include <cstdlib>
 
 #include "attn_unit.cuh"
 
@@ -507,7 +506,6 @@ int attention_sub_slices(int queries) {
 // their 2e-2 logit bar, not inside the 1e-4 bar of fp32 models) once a KV head
 // has enough queries to fill a good part of a 16-row block.
 bool attention_uses_mma(const Model& m, int batch, int m_rows, int max_keys) {
-    static const bool disabled = [] { const char* e = std::getenv("SPEC_NO_MMA_ATTENTION"); return e && e[0] == '1'; }();
     const int queries = (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows;
     // With fewer than 5 queries per KV head, or little work in all (query-key pairs over the
     // whole launch), the warp-per-query kernel wins: its CTAs are lighter to launch.
@@ -515,7 +513,7 @@ bool attention_uses_mma(const Model& m, int batch, int m_rows, int max_keys) {
     // (four queries pay only on a large batch, where its CTAs share the SMs two by two: from 128 (sequence, KV head)
     // pairs on - measured on the 7B shape, batch 16: 4.16 -> 4.05 ms per pass, batch 8: 3.46 -> 3.48)
     const int min_queries = batch * m.cfg.n_kv_heads >= 128 ? 4 : 5;
-    return !disabled && m.bf16() && queries >= min_queries && pairs >= 65536;
+    return m.bf16() && queries >= min_queries && pairs >= 65536;
 }
 
 // The key slices can be merged inside a cluster (no second kernel) whenever a CTA
@@ -524,8 +522,6 @@ bool attention_uses_mma(const Model& m, int batch, int m_rows, int max_keys) {
 // when the slice count that balances the keys is at most 8: long contexts want
 // more slices than a cluster schedules well, and keep the separate combine kernel.
 bool attention_merges_in_cluster(const Model& m, int batch, int m_rows, int max_keys) {
-    static const bool disabled = [] { const char* e = std::getenv("SPEC_NO_CLUSTER_MERGE"); return e && e[0] == '1'; }();
-    if (disabled) return false;
     return attention_uses_mma(m, batch, m_rows, max_keys) || (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows <= kMaxAttnWarps;
 }
 

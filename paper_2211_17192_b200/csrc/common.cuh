@@ -44,7 +44,8 @@ inline int fail(int status, const char* fmt, ...) {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// SPEC_NO_PDL=1 in the environment launches every kernel fully serialised (for debugging).
+// SPEC_NO_PDL=1 in the environment launches every kernel fully serialised (for debugging; the one
+// environment variable the library reads, documented in the public header).
 bool pdl_enabled();  // api.cu
 
 // True the first time it is called on the current device for this flag word (one bit per

@@ -35,7 +35,6 @@ struct spec_ctx {
     int pass_trace_capacity = 0;
     float* attn_part = nullptr;  // per key slice: (max, sum, accumulator) of every (row, head)
     int hi_rows = 0;
-    bool tensor_cores = true;
     spec::PassScratch pass;  // the persistent pass kernel's scratch (passes of at most 16 rows of a bf16 model)
     int32_t *row_token = nullptr, *row_pos = nullptr, *row_seq = nullptr, *logit_src = nullptr, *logit_dst = nullptr;
     int32_t* page_table = nullptr;
@@ -44,7 +43,8 @@ struct spec_ctx {
     int32_t *tokens = nullptr, *length = nullptr, *prompt_len = nullptr, *draft_tokens = nullptr;
     int32_t *n_accepted = nullptr, *next_token = nullptr;
     float *draft_u = nullptr, *accept_u = nullptr, *final_u = nullptr;
-    unsigned long long* counters = nullptr;  // iterations, tokens, tests evaluated, tests passed
+    unsigned long long* counters = nullptr;  // iterations, tokens, tests evaluated, tests passed, then iterations by n = 0 .. 64
+    int* nonfinite = nullptr;                // set by the sampling kernels when a row holds a NaN or +inf logit
     void* sampler_ws = nullptr;
     struct Params { unsigned long long seed; int n_new; float imposed_alpha; }* params = nullptr;
     float imposed_alpha = -1.0f;  // >= 0: timing instrument, see spec_set_imposed_acceptance
@@ -77,6 +77,8 @@ struct spec_ctx {
 
 namespace spec {
 namespace {
+
+constexpr int kCounters = 4 + 65;  // see spec_ctx::counters
 
 int check_cfg(const spec_model_cfg& c, const char* which) {
     if (c.arch == SPEC_ARCH_BIGRAM) {
@@ -233,14 +235,14 @@ int forward(spec_ctx* ctx, const Model& m, int batch, int m_rows, int n_logit_ro
                                                       n_logit_rows, c.ngram, c.vocab, logits, ctx->stream)
                                 : SPEC_OK;
     const int which = &m == &ctx->model[1] ? 1 : 0;
-    if (ctx->rt.pass_kernel && ctx->tensor_cores && pass_kernel_serves(ctx->pass, m, which, n_rows, n_logit_rows)) {
+    if (ctx->rt.pass_kernel && pass_kernel_serves(ctx->pass, m, which, n_rows, n_logit_rows)) {
         // a few rows: the whole pass is one persistent kernel
         const PassTables tables{ctx->page_table, ctx->pages_per_seq, ctx->rt.page_size, ctx->src_page_table,
                                 ctx->src_pages_per_seq, ctx->src_len, ctx->rt.max_len, ctx->rt.max_len - 1};
         return launch_pass(ctx->pass, m, which, rows, tables, batch, m_rows, n_logit_rows, logit_src, logit_dst, logits, ctx->stream,
                            ctx->pass_trace, ctx->pass_trace_capacity);
     }
-    Pass pass{ctx, m, n_rows, m.bf16() && ctx->tensor_cores, ctx->stream};
+    Pass pass{ctx, m, n_rows, m.bf16(), ctx->stream};
     const int d = c.d_model;
     const float* bias = m.t5() ? m.dec_bias : nullptr;
 
@@ -283,7 +285,7 @@ int encode(spec_ctx* ctx, const Model& m, int batch, int m_rows) {
     const spec_model_cfg& c = m.cfg;
     const int n_rows = batch * m_rows;
     const RowMeta rows{ctx->row_token, ctx->row_pos, ctx->row_seq};
-    Pass pass{ctx, m, n_rows, m.bf16() && ctx->tensor_cores, ctx->stream};
+    Pass pass{ctx, m, n_rows, m.bf16(), ctx->stream};
     const int S = ctx->rt.max_src_len;
     SPEC_TRY(launch_embed(m, rows, n_rows, ctx->h, ctx->stream));
     for (int l = 0; l < c.n_enc_layers; ++l) {
@@ -408,6 +410,7 @@ __global__ void commit_kernel(const spec_ctx::Params* __restrict__ params, const
     atomicAdd(&counters[1], static_cast<unsigned long long>(n + 1));
     atomicAdd(&counters[2], static_cast<unsigned long long>(min(n + 1, gamma)));
     atomicAdd(&counters[3], static_cast<unsigned long long>(n));
+    atomicAdd(&counters[4 + n], 1ull);  // how often an iteration accepted n guesses (Eq. 1's capped geometric law)
 }
 
 // Enqueues one iteration of Algorithm 1 for the whole batch on ctx->stream.
@@ -438,14 +441,14 @@ int enqueue_iteration(spec_ctx* ctx, int batch, int gamma, float temperature) {
         SPEC_TRY(launch_sample_strided(ctx->draft_logits + static_cast<size_t>(step - 1) * vocab,
                                        static_cast<size_t>(gamma) * vocab, ctx->draft_u + (step - 1), gamma, batch,
                                        vocab, temperature, ctx->top_k, ctx->top_p, ctx->sample_floors,
-                                       ctx->draft_tokens + (step - 1), gamma, st));
+                                       ctx->draft_tokens + (step - 1), gamma, st, ctx->nonfinite));
     }
     SPEC_TRY(launch_pdl(prep_verify_kernel, dim3(blocks_bg), dim3(threads), 0, st, ctx->tokens, ctx->draft_tokens,
                         ctx->length, batch, gamma, ctx->rt.max_len, ctx->row_token, ctx->row_pos, ctx->row_seq));
     SPEC_TRY(forward(ctx, ctx->model[0], batch, gamma + 1, batch * (gamma + 1), nullptr, nullptr, ctx->target_logits));
     SPEC_TRY(launch_verify_sample(ctx->target_logits, ctx->draft_logits, ctx->draft_tokens, ctx->accept_u, ctx->final_u,
                                   batch, gamma, vocab, temperature, ctx->lenience, ctx->top_k, ctx->top_p, ctx->n_accepted,
-                                  ctx->next_token, ctx->sampler_ws, st));
+                                  ctx->next_token, ctx->sampler_ws, st, ctx->nonfinite));
     return launch_pdl(commit_kernel, dim3(blocks_b), dim3(threads), 0, st, ctx->params, ctx->draft_tokens,
                       ctx->n_accepted, ctx->next_token, ctx->accept_u, ctx->prompt_len, batch, gamma, ctx->rt.max_len,
                       ctx->tokens, ctx->length, ctx->counters);
@@ -698,11 +701,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     ctx->pages_per_seq = (rt.max_len + rt.page_size - 1) / rt.page_size;
     ctx->max_logit_rows = std::max(rt.max_batch * std::max(rt.max_gamma + 1, 2), 64);
     // The prompt pass takes up to 256 rows at a time (weights streamed once per chunk).
-    {
-        const char* e = std::getenv("SPEC_PREFILL_ROWS");
-        const int prefill_rows = e ? std::max(1, std::atoi(e)) : 256;
-        ctx->max_rows = std::max(ctx->max_logit_rows, std::min(prefill_rows, rt.max_batch * rt.max_len));
-    }
+    ctx->max_rows = std::max(ctx->max_logit_rows, std::min(256, rt.max_batch * rt.max_len));
     if (t5) {  // an encoder pass takes every source row of the batch at once
         ctx->src_pages_per_seq = (rt.max_src_len + rt.page_size - 1) / rt.page_size;
         ctx->max_rows = std::max(ctx->max_rows, rt.max_batch * rt.max_src_len);
@@ -756,8 +755,6 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     SPEC_ALLOC(draft_logits, std::max<size_t>(B * G, 1) * V);
     {
         // Tensor-core path (any bf16 model): inputs as two bf16 terms, split-K partial sums.
-        const char* path = std::getenv("SPEC_GEMM_PATH");
-        ctx->tensor_cores = !(path && std::strcmp(path, "alu") == 0);
         size_t max_k = 0, partial = 0;
         bool any_bf16 = false;
         for (int i = 0; i < (ctx->has_draft ? 2 : 1); ++i) {
@@ -775,7 +772,7 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
                     partial = std::max(partial, gemm_tc_partial_elems(shapes[s][0], shapes[s][1], rows));
             }
         }
-        if (any_bf16 && ctx->tensor_cores) {
+        if (any_bf16) {
             for (int i = 0; i < (ctx->has_draft ? 2 : 1); ++i)
                 if (ctx->model[i].bf16() && ctx->model[i].cfg.arch != SPEC_ARCH_BIGRAM &&
                     (status = pack_model(ctx, ctx->model[i])) != SPEC_OK)
@@ -809,7 +806,8 @@ extern "C" int spec_init(const spec_model_cfg* target_cfg, const spec_model_cfg*
     SPEC_ALLOC(draft_u, std::max<size_t>(B * G, 1));
     SPEC_ALLOC(accept_u, B * (G + 1));
     SPEC_ALLOC(final_u, B * (G + 1));
-    SPEC_ALLOC(counters, 4);
+    SPEC_ALLOC(counters, kCounters);
+    SPEC_ALLOC(nonfinite, 1);
     SPEC_ALLOC(params, 1);
     SPEC_ALLOC(sample_floors, B);
     {
@@ -934,7 +932,8 @@ int begin_session(spec_ctx* ctx, const int32_t* prompt, const int32_t* prompt_le
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->tokens, host_tokens.data(), host_tokens.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->length, prompt_len, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->prompt_len, prompt_len, batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
-    SPEC_CUDA_TRY(cudaMemsetAsync(ctx->counters, 0, 4 * sizeof(unsigned long long), st));
+    SPEC_CUDA_TRY(cudaMemsetAsync(ctx->counters, 0, kCounters * sizeof(unsigned long long), st));
+    SPEC_CUDA_TRY(cudaMemsetAsync(ctx->nonfinite, 0, sizeof(int), st));
     const spec_ctx::Params params{seed, n_new, ctx->imposed_alpha};
     SPEC_CUDA_TRY(cudaMemcpyAsync(ctx->params, &params, sizeof(params), cudaMemcpyHostToDevice, st));
 
@@ -977,7 +976,14 @@ int run_iterations(spec_ctx* ctx, int iterations, float* elapsed_ms, int* remain
     ctx->session_replays += iterations;
     ctx->session_draft_passes += static_cast<long long>(iterations) * ctx->session_gamma;
     SPEC_CUDA_TRY(cudaMemcpyAsync(lengths.data(), ctx->length, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    int nonfinite = 0;
+    SPEC_CUDA_TRY(cudaMemcpyAsync(&nonfinite, ctx->nonfinite, sizeof(int), cudaMemcpyDeviceToHost, st));
     SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+    if (nonfinite) {
+        SPEC_CUDA_TRY(cudaMemsetAsync(ctx->nonfinite, 0, sizeof(int), st));
+        return fail(SPEC_ERR_NONFINITE, "a model produced a NaN or +inf logit, or a row without a finite logit (the tokens of these "
+                                        "iterations are not valid)");
+    }
     if (const int gave_up = device_gave_up(ctx)) return fail(SPEC_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (code %d)", gave_up);
     SPEC_CUDA_TRY(cudaEventElapsedTime(elapsed_ms, ctx->ev[1], ctx->ev[2]));
     *remaining = 0;
@@ -987,8 +993,9 @@ int run_iterations(spec_ctx* ctx, int iterations, float* elapsed_ms, int* remain
 }
 
 int fill_stats(spec_ctx* ctx, double decode_ms, spec_stats* stats) {
-    unsigned long long counters[4];
+    unsigned long long counters[kCounters];
     SPEC_CUDA_TRY(cudaMemcpy(counters, ctx->counters, sizeof(counters), cudaMemcpyDeviceToHost));
+    for (int n = 0; n <= 64; ++n) stats->accepted_histogram[n] = static_cast<int64_t>(counters[4 + n]);
     stats->iterations = static_cast<int64_t>(counters[0]);
     stats->tokens = static_cast<int64_t>(counters[1]);
     stats->tests_evaluated = static_cast<int64_t>(counters[2]);
@@ -1220,7 +1227,7 @@ extern "C" int spec_pass_trace(spec_ctx* ctx, int which, int batch, int rows, un
     const int n = batch * rows;
     if (batch > ctx->rt.max_batch || n > ctx->max_logit_rows)
         return fail(SPEC_ERR_CAPACITY, "spec_pass_trace: %d x %d rows exceed the workspace (%d rows)", batch, rows, ctx->max_logit_rows);
-    if (!ctx->rt.pass_kernel || !ctx->tensor_cores || !pass_kernel_serves(ctx->pass, m, which, n, n))
+    if (!ctx->rt.pass_kernel || !pass_kernel_serves(ctx->pass, m, which, n, n))
         return fail(SPEC_ERR_BAD_CONFIG, "spec_pass_trace: a pass of %d x %d rows of this model does not run as the persistent kernel", batch, rows);
     ctx->session_batch = 0;
     std::vector<int32_t> tok(n, 0), pos(n), seq(n);

@@ -47,9 +47,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 }
 
 // Bounded wait for the phase with the given parity; false on time-out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit = kSpinLimit) {
     const uint32_t addr = smem_u32(bar);
-    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+    for (uint32_t spin = 0; spin < limit; ++spin) {
         uint32_t done;
         asm volatile(
             "{\n\t"
@@ -144,8 +144,11 @@ template <int N_TOK>
 __global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_hi,
                const __grid_constant__ CUtensorMap map_lo, float* __restrict__ partial, int n_out, int n_rows,
-               int k_blocks, int packed) {
+               int k_blocks, int packed, int drill) {
+    // drill > 0 (spec_timeout_drill): the producer requests nothing and arms no barrier, and every wait gives
+    // up after `drill` polls: the path a lost copy would take, with no copy in flight when the CTA leaves
     using S = Smem<N_TOK>;
+    const uint32_t limit = drill > 0 ? static_cast<uint32_t>(drill) : kSpinLimit;
     constexpr int kTmemCols = N_TOK <= 32 ? 32 : N_TOK <= 64 ? 64 : N_TOK <= 128 ? 128 : 256;  // a power of two that holds N_TOK columns
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -179,7 +182,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const uint32_t tmem_acc = *tmem_slot;
     bool ok = true;
 
-    if (warp == 0 && lane == 0) {
+    if (warp == 0 && lane == 0 && drill <= 0) {
         // ---- producer: weights and both activation terms of one k-block per stage ----
         // The weights do not depend on the kernel before this one: the first
         // ring of weight tiles is already streaming while that kernel finishes.
@@ -205,7 +208,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
         for (int it = ahead; it < total; ++it) {
             const int kb = kb0 + it, s = it % S::kStages;
-            if (!mbar_wait(&empty_bar[s], ((it / S::kStages) - 1) & 1)) { ok = false; break; }
+            if (!mbar_wait(&empty_bar[s], ((it / S::kStages) - 1) & 1, limit)) { ok = false; break; }
             uint8_t* stage = smem + s * S::kStageBytes;
             mbar_expect_tx(&full_bar[s], S::kStageBytes);
             load_w(stage, kb, &full_bar[s]);
@@ -217,7 +220,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         constexpr uint32_t idesc = instr_desc(N_TOK);
         for (int kb = kb0; kb < kb1; ++kb) {
             const int it = kb - kb0, s = it % S::kStages;
-            if (!mbar_wait(&full_bar[s], (it / S::kStages) & 1)) { ok = false; break; }
+            if (!mbar_wait(&full_bar[s], (it / S::kStages) & 1, limit)) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t a_addr = smem_u32(smem + s * S::kStageBytes);
             const uint64_t a_desc = smem_desc_sw128(a_addr);
@@ -231,15 +234,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
             mma_commit(&empty_bar[s]);  // the stage may be refilled once these MMAs have read it
         }
-        mma_commit(acc_bar);  // accumulator complete
+        if (ok) mma_commit(acc_bar);  // accumulator complete
     }
     __syncwarp();
     pdl_wait();  // (already satisfied for the producer) nothing below may overtake the previous kernel
 
     // ---- epilogue: all four warps, warp w reads accumulator lanes 32w .. 32w+31 ----
-    if (kb1 > kb0) {
-        if (!mbar_wait(acc_bar, 0)) ok = false;
+    if (kb1 > kb0) {  // one lane polls, the warp takes one decision (the tensor-memory loads below are warp-wide)
+        int done = 1;
+        if (lane == 0) done = mbar_wait(acc_bar, 0, limit) ? 1 : 0;
+        done = __shfl_sync(0xffffffffu, done, 0);
+        if (done) mbar_wait(acc_bar, 0, 1);  // (complete: every lane observes the phase)
+        else ok = false;
     }
+    ok = __all_sync(0xffffffffu, ok);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const int feature = tile * kTileM + warp * 32 + lane;
     float* out = partial + (static_cast<size_t>(split) * n_rows) * n_out + feature;
@@ -399,14 +407,14 @@ int cached_map(const void* base, int rows, int cols, int box_rows, bool swizzle,
 
 template <int N_TOK>
 int launch_tc(const CUtensorMap& mw, const CUtensorMap& mhi, const CUtensorMap& mlo, float* partial, int n_out,
-              int n_rows, int k_blocks, int splits, int packed, cudaStream_t stream) {
+              int n_rows, int k_blocks, int splits, int packed, cudaStream_t stream, int drill = 0) {
     static std::atomic<unsigned long long> configured{0};
     if (first_use_on_this_device(configured))
         SPEC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<N_TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            Smem<N_TOK>::kTotal));
     const dim3 grid((n_out + kTileM - 1) / kTileM, splits, (n_rows + N_TOK - 1) / N_TOK);
     return launch_pdl(gemm_tc_kernel<N_TOK>, grid, dim3(kThreads), Smem<N_TOK>::kTotal, stream, mw, mhi, mlo, partial,
-                      n_out, n_rows, k_blocks, packed);
+                      n_out, n_rows, k_blocks, packed, drill);
 }
 
 }  // namespace
@@ -596,6 +604,31 @@ extern "C" int spec_pack_weight(const void* w, int n_out, int k, void* packed, v
     using namespace spec;
     if (!w || !packed || n_out < 1 || k < 8 || k % 8) return fail(SPEC_ERR_BAD_ARG, "spec_pack_weight: bad argument");
     return launch_pack_weight(w, n_out, k, packed, static_cast<cudaStream_t>(stream));
+}
+
+// ---- C ABI: a bounded wait that runs out, on purpose ----
+namespace {
+__device__ __align__(1024) unsigned char g_drill_tile[128 * 64 * 2];  // what the drill's tensor maps point at (never read)
+}
+
+extern "C" int spec_timeout_drill(void* stream) {
+    using namespace spec;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    void* base = nullptr;
+    SPEC_CUDA_TRY(cudaGetSymbolAddress(&base, g_drill_tile));
+    CUtensorMap mw, mx;
+    int status = cached_map(base, 128, 64, 128, true, &mw);
+    if (status == SPEC_OK) status = cached_map(base, 16, 64, 16, true, &mx);
+    if (status != SPEC_OK) return status;
+    SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+    gemm_tc_take_error();  // (whatever was pending is not this drill's)
+    // one CTA, one k-block, nothing requested: the MMA issuer's wait and the epilogue's wait run out after 4096 polls
+    status = launch_tc<16>(mw, mx, mx, reinterpret_cast<float*>(base), 128, 1, 1, 1, 0, st, 4096);
+    if (status != SPEC_OK) return status;
+    SPEC_CUDA_TRY(cudaStreamSynchronize(st));
+    const int code = gemm_tc_take_error();
+    if (code > 0) return fail(SPEC_ERR_DEVICE_TIMEOUT, "drill: the kernel gave up on a bounded wait (code %d), freed its tensor memory and returned", code);
+    return fail(SPEC_ERR_CUDA, "drill: the kernel did not report the wait that should have run out");
 }
 
 extern "C" int spec_device_error(void) {

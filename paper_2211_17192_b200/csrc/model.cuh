@@ -183,13 +183,14 @@ int pass_take_error();
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
                          const float* uniforms, const float* final_uniforms, int batch, int gamma, int vocab,
                          float temperature, float lenience, int top_k, float top_p, int32_t* n_accepted,
-                         int32_t* next_token, void* workspace, cudaStream_t stream);
+                         int32_t* next_token, void* workspace, cudaStream_t stream, int* nonfinite = nullptr);
+// (`nonfinite`, optional device word: set to 1 if a row holds a NaN or +inf logit, or no finite logit at all)
 // top_k = 0 and top_p = 1: the whole vocabulary; otherwise floor_scratch holds one float per row.
 int launch_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature, int top_k,
                   float top_p, float* floor_scratch, int32_t* tokens, cudaStream_t stream);
 int launch_sample_strided(const float* logits, size_t logit_stride, const float* uniforms, int uniform_stride,
                           int rows, int vocab, float temperature, int top_k, float top_p, float* floor_scratch,
-                          int32_t* tokens, int token_stride, cudaStream_t stream);
+                          int32_t* tokens, int token_stride, cudaStream_t stream, int* nonfinite = nullptr);
 size_t verify_sample_workspace_bytes(int batch, int gamma, int vocab);
 
 }  // namespace spec

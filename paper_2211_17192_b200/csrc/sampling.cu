@@ -394,7 +394,7 @@ struct __align__(16) ChunkStat {
     float max;     // chunk maximum
     float aux;     // T > 0: sum exp((l - max) / T) over the chunk; T = 0: argmax index as int bits
     float xlogit;  // the row's logit at the drafted token, if that token falls in this chunk
-    float pad;
+    float bad;     // T = 0: non-zero if the chunk holds a NaN or +inf logit (T > 0: the sums show it)
 };
 
 // grid = (chunks, rows, batch); rows = 2*gamma+1 (T > 0: p_1..p_{gamma+1}, q_1..q_gamma)
@@ -440,6 +440,7 @@ verify_stats_kernel(const float* __restrict__ target_logits, const float* __rest
     float m = -FLT_MAX;  // finite, so that (m - new_max) never becomes inf - inf
     float s = 0.0f;
     int arg = 0x7fffffff;
+    bool bad = false;  // T = 0 only: a NaN or +inf logit (the comparisons below would pass over a NaN in silence)
     for (int base = g0 + tid; base < g1; base += kUnroll * kStatThreads) {
         float4 v[kUnroll];
 #pragma unroll
@@ -455,6 +456,7 @@ verify_stats_kernel(const float* __restrict__ target_logits, const float* __rest
                 if (v[i].y > m) { m = v[i].y; arg = j + 1; }
                 if (v[i].z > m) { m = v[i].z; arg = j + 2; }
                 if (v[i].w > m) { m = v[i].w; arg = j + 3; }
+                bad |= !(v[i].x < INFINITY) | !(v[i].y < INFINITY) | !(v[i].z < INFINITY) | !(v[i].w < INFINITY);
             }
         } else {
             float bm = m;
@@ -471,8 +473,9 @@ verify_stats_kernel(const float* __restrict__ target_logits, const float* __rest
     }
     ChunkStat* out = stats + (static_cast<size_t>(b) * rows + row) * chunks + chunk;
     if (GREEDY) {
+        const int any_bad = __syncthreads_or(bad ? 1 : 0);
         block_argmax<kStatWarps>(m, arg, red, red_i);
-        if (tid == 0) *reinterpret_cast<float4*>(out) = make_float4(m, __int_as_float(arg), 0.0f, 0.0f);
+        if (tid == 0) *reinterpret_cast<float4*>(out) = make_float4(m, __int_as_float(arg), 0.0f, any_bad ? 1.0f : 0.0f);
     } else {
         const float wm = warp_max(m);
         s = warp_sum(s * fast_exp2((m - wm) * c2));
@@ -509,7 +512,7 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
                      const int32_t* __restrict__ draft_tokens, const float* __restrict__ uniforms, int gamma,
                      int vocab, float inv_t, int chunks, int cluster_size, const ChunkStat* __restrict__ stats,
                      const float* __restrict__ final_uniforms, float lenience, const float* __restrict__ floors,
-                     int32_t* __restrict__ n_accepted, int32_t* __restrict__ next_token) {
+                     int32_t* __restrict__ n_accepted, int32_t* __restrict__ next_token, int* __restrict__ nonfinite) {
     __shared__ FinishShared sh;
     const int tid = threadIdx.x;
     const int b = blockIdx.x / cluster_size;
@@ -539,6 +542,7 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
         const ChunkStat* st_r = stats + (static_cast<size_t>(b) * rows + tid) * chunks;
         float M = -FLT_MAX, A = 0.0f, X = 0.0f;
         int best = 0x7fffffff;
+        bool bad = false;
         const int xchunk = (my_x >= 0 && my_x < vocab) ? (my_x >> 2) / per_chunk : -1;
         for (int c0 = 0; c0 < chunks; c0 += 4) {
             float4 st[4];
@@ -552,6 +556,7 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
                 if (GREEDY) {
                     const int ci = __float_as_int(st[i].y);
                     if (st[i].x > M || (st[i].x == M && ci < best)) { M = st[i].x; best = ci; }
+                    bad |= st[i].w != 0.0f;
                 } else {
                     const float nm = fmaxf(M, st[i].x);
                     A = A * fast_exp2((M - nm) * c2) + st[i].y * fast_exp2((st[i].x - nm) * c2);
@@ -560,6 +565,9 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
                 }
             }
         }
+        // a NaN or +inf logit (or a row without a finite logit) leaves a sum that is not a positive number
+        if (!GREEDY) bad = !(A > 0.0f) || !isfinite(A) || !isfinite(M);
+        if (bad && nonfinite && rank == 0) atomicExch(nonfinite, 1);
         sh.row_max[tid] = M;
         sh.row_aux[tid] = GREEDY ? __int_as_float(best) : A;
         sh.row_x[tid] = X;
@@ -629,7 +637,7 @@ template <bool VEC, bool CUT>
 __global__ void __launch_bounds__(kSampleThreads)
 sample_kernel(const float* __restrict__ logits, size_t logit_stride, const float* __restrict__ uniforms,
               int uniform_stride, int vocab, float inv_t, bool greedy, const float* __restrict__ floors,
-              int32_t* __restrict__ tokens, int token_stride) {
+              int32_t* __restrict__ tokens, int token_stride, int* __restrict__ nonfinite) {
     constexpr int W = kSampleThreads / 32;
     __shared__ float red[W];
     __shared__ int red_i[W];
@@ -644,6 +652,7 @@ sample_kernel(const float* __restrict__ logits, size_t logit_stride, const float
     const int groups = (vocab + 3) >> 2;
     float m = -FLT_MAX;
     int arg = 0x7fffffff;
+    bool bad = false;  // a NaN or +inf logit
 #pragma unroll 4
     for (int g = tid; g < groups; g += kSampleThreads) {
         const float4 v = r.load(g, -INFINITY);
@@ -652,7 +661,9 @@ sample_kernel(const float* __restrict__ logits, size_t logit_stride, const float
         if (v.y > m) { m = v.y; arg = j + 1; }
         if (v.z > m) { m = v.z; arg = j + 2; }
         if (v.w > m) { m = v.w; arg = j + 3; }
+        bad |= !(v.x < INFINITY) | !(v.y < INFINITY) | !(v.z < INFINITY) | !(v.w < INFINITY);
     }
+    if (nonfinite && bad) atomicExch(nonfinite, 1);
     block_argmax<W>(m, arg, red, red_i);
     if (tid == 0) { s_max = m; s_arg = arg; }
     __syncthreads();
@@ -1035,7 +1046,7 @@ int launch_cut_floors(const float* a, size_t a_stride, int a_rows, const float* 
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
                          const float* uniforms, const float* final_uniforms, int batch, int gamma, int vocab,
                          float temperature, float lenience, int top_k, float top_p, int32_t* n_accepted,
-                         int32_t* next_token, void* workspace, cudaStream_t stream) {
+                         int32_t* next_token, void* workspace, cudaStream_t stream, int* nonfinite) {
     const bool greedy = temperature == 0.0f;
     const int rows = greedy ? gamma + 1 : 2 * gamma + 1;
     const int chunks = chunks_for(vocab, rows * batch);
@@ -1075,19 +1086,19 @@ int launch_verify_sample(const float* target_logits, const float* draft_logits, 
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = cluster_size;
-    attr[1].val.clusterDim.y = 1;
-    attr[1].val.clusterDim.z = 1;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster_size;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 2;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
     const ChunkStat* stats_in = stats;
 #define SPEC_LAUNCH_FINISH(G, V, C)                                                                                  \
     SPEC_CUDA_TRY(cudaLaunchKernelEx(&cfg, verify_finish_kernel<G, V, C>, target_logits, draft_logits, draft_tokens, \
                                      uniforms, gamma, vocab, inv_t, chunks, cluster_size, stats_in,                 \
-                                     final_uniforms, lenience, floors, n_accepted, next_token))
+                                     final_uniforms, lenience, floors, n_accepted, next_token, nonfinite))
     if (greedy && vec) SPEC_LAUNCH_FINISH(true, true, false);
     else if (greedy) SPEC_LAUNCH_FINISH(true, false, false);
     else if (vec && cut) SPEC_LAUNCH_FINISH(false, true, true);
@@ -1103,7 +1114,7 @@ int launch_verify_sample(const float* target_logits, const float* draft_logits, 
 // With a cut (0 < top_k < vocab or 0 < top_p < 1, and T > 0) `floor_scratch` must hold `rows` floats.
 int launch_sample_strided(const float* logits, size_t logit_stride, const float* uniforms, int uniform_stride,
                           int rows, int vocab, float temperature, int top_k, float top_p, float* floor_scratch,
-                          int32_t* tokens, int token_stride, cudaStream_t stream) {
+                          int32_t* tokens, int token_stride, cudaStream_t stream, int* nonfinite) {
     const bool greedy = temperature == 0.0f;
     const float inv_t = greedy ? 0.0f : 1.0f / temperature;
     const float* floors = nullptr;
@@ -1116,7 +1127,7 @@ int launch_sample_strided(const float* logits, size_t logit_stride, const float*
     const bool vec = vocab % 4 == 0 && logit_stride % 4 == 0 && aligned16(logits);
 #define SPEC_LAUNCH_SAMPLE(V, C)                                                                                   \
     return launch_pdl(sample_kernel<V, C>, dim3(rows), dim3(kSampleThreads), 0, stream, logits, logit_stride, uniforms, \
-                      uniform_stride, vocab, inv_t, greedy, floors, tokens, token_stride)
+                      uniform_stride, vocab, inv_t, greedy, floors, tokens, token_stride, nonfinite)
     if (vec && floors) SPEC_LAUNCH_SAMPLE(true, true);
     if (vec) SPEC_LAUNCH_SAMPLE(true, false);
     if (floors) SPEC_LAUNCH_SAMPLE(false, true);
@@ -1127,7 +1138,7 @@ int launch_sample_strided(const float* logits, size_t logit_stride, const float*
 int launch_sample(const float* logits, const float* uniforms, int rows, int vocab, float temperature, int top_k,
                   float top_p, float* floor_scratch, int32_t* tokens, cudaStream_t stream) {
     return launch_sample_strided(logits, static_cast<size_t>(vocab), uniforms, 1, rows, vocab, temperature, top_k, top_p,
-                                 floor_scratch, tokens, 1, stream);
+                                 floor_scratch, tokens, 1, stream, nullptr);
 }
 
 }  // namespace spec

@@ -10,6 +10,11 @@ from paper_2211_17192_b200 import binding, workloads
 
 pytestmark = pytest.mark.gpu
 
+# A free-running comparison ends at the first decision that sits within tolerance of a boundary;
+# it must have compared at least this many tokens by then (a flagged decision at the very start
+# would otherwise pass with nothing verified).
+MIN_COMPARED = 10
+
 
 def _models(target_name, draft_name, **overrides):
     tcfg = workloads.scaled_config(workloads.model_config(target_name), **overrides)
@@ -47,6 +52,7 @@ def test_temperature_zero_equals_target_only_greedy(tiny, gamma):
     for k in range(40):
         if greedy[0, k] != ref[k]:
             assert gaps[k] < 2e-3  # an argmax tie within the logit tolerance; the runs diverge from here
+            assert k >= MIN_COMPARED, f"only {k} tokens were compared before a tolerance-flagged tie"
             break
     assert stats["iterations"] >= 40 / (gamma + 1)
 
@@ -59,6 +65,7 @@ def test_target_only_sampling_matches_the_oracle(tiny):
     for k in range(48):
         if got[0, k] != ref[k]:
             assert margins[k] < 1e-3
+            assert k >= MIN_COMPARED, f"only {k} tokens were compared before a tolerance-flagged draw"
             break
     assert stats["iterations"] == 48 and stats["tests_evaluated"] == 0 and stats["draft_passes"] == 0
 
@@ -86,6 +93,7 @@ def test_ragged_batch_equals_per_sequence_oracle(tiny):
             index = len(prompt) + diff
             it = next(i for i in ref.iterations if i.start_len <= index <= i.start_len + i.n_accepted)
             assert min([it.accept_margin, it.cdf_margin] + list(it.draft_cdf_margins)) < 1e-3
+            assert diff >= MIN_COMPARED, f"sequence {b}: only {diff} tokens were compared before a tolerance-flagged decision"
 
 
 def test_bf16_llama_pair_matches_the_oracle():
@@ -108,6 +116,9 @@ def test_statistics_are_consistent(tiny):
     assert st["tests_passed"] <= st["tests_evaluated"] <= 3 * st["iterations"]
     assert 60 <= st["tokens"] <= 60 + 3 and st["target_passes"] >= st["iterations"]
     assert st["decode_ms"] > 0 and st["prefill_ms"] >= 0
+    hist = st["accepted_histogram"]
+    assert sum(hist) == st["iterations"] and sum(n * c for n, c in enumerate(hist)) == st["tests_passed"]
+    assert not any(hist[4:])  # gamma = 3: n <= 3
     again, _ = eng.generate([prompt], 60, 3, 1.0, 1)
     assert np.array_equal(out, again)  # same seed, same tokens
     other, _ = eng.generate([prompt], 60, 3, 1.0, 2)
@@ -177,6 +188,7 @@ def test_lenient_generation_matches_the_oracle_and_accepts_more(tiny):
             index = len(prompt) + diff
             it = next(i for i in ref.iterations if i.start_len <= index <= i.start_len + i.n_accepted)
             assert min([it.accept_margin, it.cdf_margin] + list(it.draft_cdf_margins)) < 1e-3
+            assert diff >= MIN_COMPARED, f"only {diff} tokens were compared before a tolerance-flagged decision"
         with pytest.raises(binding.SpecError):
             eng.set_lenience(1.5)
     finally:

@@ -467,3 +467,21 @@ def test_emitted_law_under_the_nucleus_is_the_nucleus_target_distribution():
     for i in range(300):
         res = sampling.verify_step(tl, ql, x[i : i + 1], [r[i], u[i]], 1.0, **kw)
         assert (res.n_accepted, res.next_token) == (n[i], t[i])
+
+
+def test_greedy_rule_for_a_guess_off_the_drafts_support():
+    """T = 0: a guess that is not the draft's maximum has q(x) = 0, where Algorithm 1's ratio test
+    decides nothing; the reading taken is "accepted iff it is the target's maximum", so that the
+    emitted tokens are the target's greedy continuation whatever was guessed (the abstract's claim
+    that the outputs do not change)."""
+    tl = np.array([[0.1, 2.0, 0.3, 0.0], [1.5, 0.2, 0.1, 0.0], [0.0, 0.1, 0.2, 3.0]])
+    ql = np.array([[5.0, 0.0, 0.0, 0.0], [0.0, 0.0, 4.0, 0.0]])   # the draft's maxima: tokens 0 and 2
+    us = [0.99, 0.99, 0.5]
+    both = sampling.verify_step(tl, ql, [1, 0], us, 0.0)           # the target's maxima, neither is the draft's
+    assert (both.n_accepted, both.next_token) == (2, 3)
+    second = sampling.verify_step(tl, ql, [1, 2], us, 0.0)         # the draft's own maximum, not the target's
+    assert (second.n_accepted, second.next_token) == (1, 0)
+    first = sampling.verify_step(tl, ql, [3, 0], us, 0.0)          # neither model's maximum
+    assert (first.n_accepted, first.next_token) == (0, 1)
+    n, t = sampling.verify_trials(tl, ql, np.array([[1, 0], [1, 2], [3, 0]]), np.tile(us, (3, 1)), 0.0)
+    assert n.tolist() == [2, 1, 0] and t.tolist() == [3, 0, 1]
