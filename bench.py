@@ -1,6 +1,7 @@
 """Benchmark of the speculative-decoding hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--batch B] [--gamma G] [--impl reference]
+    python bench.py --profile-pass --model NAME [--layers L] [--batch B] [--rows R] [--context C]   (profiler driver)
 
 Prints ONE JSON line (rank 0).  For N > 1 it is launched with torchrun, one
 process per GPU; ranks are independent replicas (the path has no exchange
@@ -866,6 +867,42 @@ def run_generation(args, wl, torch, device, local, barrier):
                 clocks=clock_info, extras=extras)
 
 
+def profile_pass(args):
+    """One forward-pass shape, repeated, for profilers (`--profile-pass`): builds the named model of
+    `workloads.model_config` (optionally at reduced depth, full width; weights drawn on the GPU), feeds
+    `--context` tokens per sequence through the teacher-forced entry point, and then replays one pass
+    over `--rows` new rows per sequence `--repeats` times with `spec_time_forward`.  Every kernel of the
+    decode path therefore appears in the launch list with exactly the shape it has in a verification pass
+    (rows = gamma + 1) or a draft step (rows = 1), which is what `ncu -k regex:<kernel>` wants.  Prints
+    the device time per pass."""
+    import torch
+
+    import __graft_entry__ as entry
+    from paper_2211_17192_b200 import binding, workloads
+    entry.build()
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    cfg = workloads.model_config(args.model)
+    if args.layers:
+        cfg = workloads.scaled_config(cfg, n_layers=args.layers, n_enc_layers=min(cfg["n_enc_layers"], args.layers))
+    t5 = cfg["arch"] == "t5"
+    batch = args.batch or 1
+    eng = binding.Engine(cfg, gpu_weights(cfg, 1, device), max_batch=batch, max_len=args.context + args.rows + 8,
+                         page_size=64, max_gamma=max(args.rows - 1, 1), kv_dtype=args.kv_dtype,
+                         max_src_len=args.source if t5 else 0, pass_kernel=args.pass_kernel)
+    if t5:
+        eng.encode([workloads.make_prompt(b, args.source, cfg["vocab"]) for b in range(batch)])
+    tokens = np.stack([workloads.make_prompt(100 + b, args.context, cfg["vocab"]) for b in range(batch)])
+    chunk = max(1, 64 // batch)
+    for c0 in range(0, args.context, chunk):
+        eng.forward_logits(0, tokens[:, c0:c0 + chunk])
+    ms = eng.time_forward(0, batch, args.rows, args.repeats)
+    print(json.dumps({"profile_pass": args.model, "layers": cfg["n_layers"], "batch": batch, "rows": args.rows,
+                      "context": args.context, "kv_dtype": eng.kv_dtype, "pass_kernel": bool(args.pass_kernel),
+                      "ms_per_pass": ms}))
+    eng.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -885,9 +922,21 @@ def main():
                     help="also report decoding with gamma chosen by the library burst by burst, up to this value")
     ap.add_argument("--no-configs", dest="configs", action="store_false",
                     help="llama7b workload: skip the other configurations (batch 16 and 32, GPT 97M/6M, T5-XXL/small, sampler)")
+    ap.add_argument("--profile-pass", action="store_true",
+                    help="profiler driver: replay one pass shape (--model --layers --batch --rows --context --repeats) and exit")
+    ap.add_argument("--model", default="llama7b_target", help="--profile-pass: model name of workloads.model_config")
+    ap.add_argument("--rows", type=int, default=3, help="--profile-pass: new rows per sequence in the timed pass")
+    ap.add_argument("--context", type=int, default=1024, help="--profile-pass: cached tokens per sequence before the timed pass")
+    ap.add_argument("--source", type=int, default=512, help="--profile-pass: source length (encoder-decoder models)")
+    ap.add_argument("--repeats", type=int, default=3, help="--profile-pass: replays of the pass")
+    ap.add_argument("--kv-dtype", default=None, choices=["fp32", "fp16", "bf16"], help="--profile-pass: cached K,V row type")
+    ap.add_argument("--pass-kernel", action="store_true", help="--profile-pass: the persistent pass kernel instead of the kernel chain")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for cpu_baseline")
     args = ap.parse_args()
+    if args.profile_pass:
+        profile_pass(args)
+        return
     if args.steps is None:
         args.steps = 300 if args.workload == "sampler" else 100
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
