@@ -743,6 +743,11 @@ def run_generation(args, wl, torch, device, local, barrier):
     from oracle import analysis  # closed forms only, for the report (rank 0)
     rank = int(os.environ.get("RANK", "0"))
     long_steps = max(200, args.steps)  # (also measured: a stretch long enough for the acceptance rate to settle)
+    # ... as far as the model's positions reach: every iteration may add gamma + 1 tokens to the context
+    context0 = 1 if isinstance(wl, EncDecWorkload) else wl.prompt_len
+    from paper_2211_17192_b200 import workloads
+    room = workloads.model_config(wl.target_name)["max_positions"] - context0 - 64 - wl.gamma - 3
+    long_steps = max(args.steps, min(long_steps, room // (wl.gamma + 1) - args.warmup))
     wl.prepare(rank, device, args.warmup + long_steps)
     clocks = ClockSampler(local)
     clocks.start()

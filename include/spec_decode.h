@@ -525,8 +525,10 @@ int spec_truncate(spec_ctx* ctx, int which, const int32_t* lengths, int batch);
  * `cross` != 0 for the cross-attention of an encoder-decoder block.  The choice
  * depends on the shapes and on the context's capacities (max_len, max_src_len)
  * only, never on the data.  plan (HOST int32 [4]) receives
- *   plan[0]  1: the queries of a KV head are multiplied on the tensor cores
- *               (mma.sync tf32), 0: one warp per query on the FMA pipes;
+ *   plan[0]  0: one warp per query on the FMA pipes; 1: the queries of a KV head
+ *               are multiplied on the tensor cores in tf32 from rows converted to
+ *               fp32; 2: in f16 straight from fp16 rows, all the queries of a KV
+ *               head in one CTA;
  *   plan[1]  key slices (CTAs) per (sequence, KV head);
  *   plan[2]  1: the slices are merged inside a thread-block cluster, 0: by a
  *               second kernel from partial states in global memory;

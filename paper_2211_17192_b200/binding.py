@@ -593,7 +593,8 @@ class Engine:
                                           ctypes.POINTER(ctypes.c_int)]
         plan = (ctypes.c_int * 4)()
         _check(h.spec_attention_plan(self._ctx, which, batch, rows, 1 if cross else 0, plan))
-        return dict(tensor_cores=bool(plan[0]), slices=int(plan[1]), cluster_merge=bool(plan[2]), in_turn=bool(plan[3]))
+        return dict(tensor_cores=bool(plan[0]), f16=plan[0] == 2, slices=int(plan[1]), cluster_merge=bool(plan[2]),
+                    in_turn=bool(plan[3]))
 
     def pass_trace(self, which, batch, rows, capacity=65536):
         """The CTAs' clocks at the grid barriers of one persistent-kernel pass (`spec_pass_trace`):

@@ -20,6 +20,8 @@
 // query; attention_combine_kernel merges the key slices and emits the
 // out-projection's input (fp32 and/or split into two bf16 terms).
 #include <cfloat>
+#include <climits>
+#include <type_traits>
 
 #include "attn_unit.cuh"
 
@@ -77,9 +79,11 @@ __device__ __forceinline__ void cluster_merge_write(const float* fin, int n_q, i
             float l = 0.0f, o = 0.0f;
 #pragma unroll
             for (int s = 0; s < kMaxClusterSlices; ++s) {  // slices in index order
-                const float w = s < slices ? expf(ms[s] - mm) : 0.0f;
-                l += ls[s] * w;
-                o += os[s] * w;
+                if (s < slices) {                              // (uniform: absent slices cost no exponential)
+                    const float w = expf(ms[s] - mm);
+                    l += ls[s] * w;
+                    o += os[s] * w;
+                }
             }
             const float y = l > 0.0f ? o / l : 0.0f;  // an inactive row has no keys
             if (out.att) out.att[at + e] = y;
@@ -456,6 +460,358 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     }
 }
 
+// ---- fp16 K,V rows on the f16 tensor-core path --------------------------------
+//
+// With 16-bit rows the cache needs no conversion: 64-key tiles of K and of V go
+// from the pool to shared memory as they are (cp.async, two stages: tile i + 1
+// loads while tile i is multiplied) and feed mma.sync.m16n8k16 (f16 operands,
+// fp32 accumulate) through ldmatrix.  A CTA owns (key slice, KV head, sequence)
+// and ALL the queries of that KV head - up to 64, as MB blocks of 16 - so K and
+// V of the slice are fetched once, whatever the number of rows.  Its four warps
+// are (query block, part of the tile's keys): warp w takes query block w % MB
+// and keys [16 MB (w / MB), 16 MB (w / MB + 1)) of every tile; the key parts of a
+// query block merge at the end.  Scores, the online softmax and the output
+// accumulate in fp32; q (scaled) and the probabilities are rounded to fp16 (11
+// significant bits, one more than the tf32 path above keeps).
+constexpr int kF16Warps = 4;
+constexpr int kF16TileKeys = 64;
+constexpr int kF16Stages = 2;
+constexpr int kF16MaxQueries = 64;  // per CTA (MB = 4)
+
+template <int DH, int MB>
+struct F16Smem {
+    static constexpr int kRow = DH + 8;                  // halves per staged row: consecutive rows are 16 bytes apart
+                                                         // modulo 128, so ldmatrix sees no bank conflict
+    static constexpr int kQ = 16 * MB * kRow;            // the queries (halves)
+    static constexpr int kTile = kF16TileKeys * kRow;    // one K or V tile (halves)
+    static constexpr int kStage = 2 * kTile;             // K, then V
+    static constexpr size_t kBytes = static_cast<size_t>(kQ + kF16Stages * kStage) * sizeof(__half);
+    // the epilogue reuses the stages: four warps' states in stage 0, the merged states in stage 1
+    static_assert(kF16Warps * 16 * (DH + 2) * sizeof(float) <= kStage * sizeof(__half), "states must fit a stage");
+    static_assert(16 * MB * (DH + 2) * sizeof(float) <= kStage * sizeof(__half), "merged states must fit a stage");
+};
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const __half* p) {
+    const uint32_t a = static_cast<uint32_t>(__cvta_generic_to_shared(p));
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], const __half* p) {
+    const uint32_t a = static_cast<uint32_t>(__cvta_generic_to_shared(p));
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_half2(float a, float b) {
+    const __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+__device__ __forceinline__ float exp2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// grid = (slices, n_kv_heads * q_blocks, batch), block = 128; q_blocks = ceil(queries / 64).
+// Scores are kept in base-2 units (q is scaled by log2(e) / sqrt(d_head), the bias by log2(e)), so every
+// exponential is one ex2.approx; the running maximum goes back to natural units when the state is stored.
+template <int DH, int MB, bool FUSED>
+__global__ void __launch_bounds__(32 * kF16Warps)
+attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __restrict__ pos,
+                     const int32_t* __restrict__ seq, int m_rows, int n_heads, int n_kv_heads, int q_blocks,
+                     const __half* __restrict__ kv_layer, const int32_t* __restrict__ page_table, int pages_per_seq,
+                     int page_size, const int32_t* __restrict__ kv_len, const float* __restrict__ bias, int bias_span,
+                     int bias_zero, float scale, float* __restrict__ part, const AttnOut out) {
+    using S = F16Smem<DH, MB>;
+    constexpr int KP = kF16Warps / MB;        // key parts of a tile
+    constexpr int KW = kF16TileKeys / KP;     // keys of a tile that one warp multiplies (16 MB)
+    constexpr int NB = KW / 8;                // 8-key blocks of those
+    constexpr int CH = DH / 8;                // 16-byte chunks of a row
+    constexpr int QN = 16 * MB;               // queries of this CTA
+    constexpr int kRowsPerSweep = 32 * kF16Warps / CH;        // rows that the CTA's threads copy at once (one chunk each)
+    constexpr int kSweeps = kF16TileKeys / kRowsPerSweep;     // sweeps per K (or V) tile
+    constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ int q_pos[QN], q_row[QN], q_head[QN];
+    __half* Qs = reinterpret_cast<__half*>(smem_raw);
+    __half* stages = Qs + S::kQ;
+    pdl_trigger();
+    pdl_wait();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int mb = warp % MB, kw0 = (warp / MB) * KW;
+    const int slice = blockIdx.x, slices = gridDim.x, b = blockIdx.z;
+    const int kv_head = blockIdx.y / q_blocks, qb = blockIdx.y % q_blocks;
+    const int group = n_heads / n_kv_heads;
+    const int queries = group * m_rows;
+
+    if (tid < QN) {
+        const int q = qb * kF16MaxQueries + tid;
+        const bool live = q < queries;
+        const int j = live ? q / group : 0;
+        q_row[tid] = b * m_rows + j;
+        q_head[tid] = kv_head * group + (live ? q % group : 0);
+        q_pos[tid] = live ? pos[b * m_rows + j] : -1;
+    }
+    int seq_keys = 0;
+    if (kv_len) {
+        seq_keys = kv_len[seq[b * m_rows]];
+    } else {
+        for (int j = 0; j < m_rows; ++j) seq_keys = max(seq_keys, pos[b * m_rows + j] + 1);
+    }
+    const int tiles = (seq_keys + kF16TileKeys - 1) / kF16TileKeys;
+    const int t0 = static_cast<int>(static_cast<long long>(tiles) * slice / slices);
+    const int t1 = static_cast<int>(static_cast<long long>(tiles) * (slice + 1) / slices);
+    const int my_tiles = t1 - t0;
+    const size_t head_stride = static_cast<size_t>(page_size) * DH;
+    const size_t page_stride = 2 * static_cast<size_t>(n_kv_heads) * head_stride;
+    const size_t v_offset = static_cast<size_t>(n_kv_heads) * head_stride;
+    const int32_t* pages = page_table + seq[b * m_rows] * pages_per_seq;
+    const int page_shift = __ffs(page_size) - 1;  // (pages hold a power of two of tokens)
+    const __half* head_base = kv_layer + kv_head * head_stride;
+
+    // Tile i of the slice into stage i % 2.  A thread copies one 16-byte chunk per sweep: chunk tid % CH of
+    // row tid / CH + kRowsPerSweep * sweep, of K and of V.  A 32-key half of the tile lies inside one page;
+    // keys at or beyond seq_keys become zeros.
+    const int copy_row = tid / CH, copy_off = copy_row * DH + 8 * (tid % CH);
+    const uint32_t copy_dst = static_cast<uint32_t>(__cvta_generic_to_shared(stages)) +
+                              static_cast<uint32_t>((copy_row * S::kRow + 8 * (tid % CH)) * sizeof(__half));
+    // (the page entries of a tile are fetched one tile ahead of the copies that need them, so that no
+    // copy waits for a page-table load)
+    auto fetch_pages = [&](int i, int (&pg)[2]) {
+        if (i < my_tiles) {
+            const int k0 = kF16TileKeys * (t0 + i);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) pg[h] = pages[min(k0 + 32 * h, seq_keys - 1) >> page_shift];
+        }
+    };
+    auto issue = [&](int i, const int (&pg)[2]) {
+        if (i < my_tiles) {
+            const int k0 = kF16TileKeys * (t0 + i);
+            const uint32_t dst = copy_dst + static_cast<uint32_t>((i % kF16Stages) * S::kStage * sizeof(__half));
+            const __half* half_base[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+                half_base[h] = head_base + pg[h] * page_stride + static_cast<size_t>((k0 + 32 * h) & (page_size - 1)) * DH + copy_off;
+            const int n_valid = seq_keys - k0 - copy_row;  // row r of this thread is valid iff r_in_tile - copy_row < n_valid
+#pragma unroll
+            for (int sw = 0; sw < kSweeps; ++sw) {
+                constexpr int kSweepsPerHalf = 32 / kRowsPerSweep;
+                const bool valid = sw * kRowsPerSweep < n_valid;
+                const __half* src = half_base[sw / kSweepsPerHalf] + (valid ? (sw % kSweepsPerHalf) * kRowsPerSweep * DH : -copy_row * DH);
+                const uint32_t d = dst + static_cast<uint32_t>(sw * kRowsPerSweep * S::kRow * sizeof(__half));
+                const int bytes = valid ? 16 : 0;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d + static_cast<uint32_t>(S::kTile * sizeof(__half))),
+                             "l"(src + v_offset), "r"(bytes) : "memory");
+            }
+        }
+        cp_async_commit();
+    };
+    int pg_now[2] = {0, 0}, pg_next[2] = {0, 0};
+    fetch_pages(0, pg_now);
+    fetch_pages(1, pg_next);
+    issue(0, pg_now);  // (requested before the queries are staged)
+    __syncthreads();  // (the queries' positions)
+    const float q_scale = scale * kLog2e;
+    for (int i = tid; i < QN * DH; i += 32 * kF16Warps) {
+        const int qi = i / DH, e = i % DH;
+        const float v = q_pos[qi] >= 0 ? qkv[static_cast<size_t>(q_row[qi]) * q_stride + q_head[qi] * DH + e] * q_scale : 0.0f;
+        Qs[qi * S::kRow + e] = __float2half_rn(v);
+    }
+
+    // the two query rows of this lane: g and g + 8 of query block mb.  A row beyond the live queries sees
+    // every key (its output is never written): it then never forces the masked path on its warp.
+    const int p_lo = q_pos[mb * 16 + g], p_hi = q_pos[mb * 16 + g + 8];
+    const int keys_lo = p_lo < 0 ? INT_MAX : kv_len ? seq_keys : p_lo + 1;
+    const int keys_hi = p_hi < 0 ? INT_MAX : kv_len ? seq_keys : p_hi + 1;
+    const float* bias_lo = bias && p_lo >= 0 ? bias + static_cast<size_t>(q_head[mb * 16 + g]) * bias_span + (bias_zero - p_lo) : nullptr;
+    const float* bias_hi = bias && p_hi >= 0 ? bias + static_cast<size_t>(q_head[mb * 16 + g + 8]) * bias_span + (bias_zero - p_hi) : nullptr;
+    float m_lo = -FLT_MAX, m_hi = -FLT_MAX, l_lo = 0.0f, l_hi = 0.0f;
+    float o[DH / 8][4];
+#pragma unroll
+    for (int n = 0; n < DH / 8; ++n)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[n][i] = 0.0f;
+    uint32_t qf[DH / 16][4];
+    // keys that every row of this warp sees (no mask needed below it), and that any live row sees
+    const int all_see = min(__reduce_min_sync(kFullMask, min(keys_lo, keys_hi)), seq_keys);
+    const int any_sees = min(__reduce_max_sync(kFullMask, max(p_lo < 0 ? 0 : keys_lo, p_hi < 0 ? 0 : keys_hi)), seq_keys);
+
+    for (int i = 0; i < my_tiles; ++i) {
+        cp_async_wait<0>();
+        __syncthreads();  // tile i has landed for every thread; everybody is done with tile i - 1
+        issue(i + 1, pg_next);
+        fetch_pages(i + 2, pg_next);
+        if (i == 0) {  // (the first barrier also covered the staged queries)
+#pragma unroll
+            for (int ks = 0; ks < DH / 16; ++ks)
+                ldsm_x4(qf[ks], Qs + (mb * 16 + (lane & 7) + 8 * ((lane >> 3) & 1)) * S::kRow + ks * 16 + 8 * (lane >> 4));
+        }
+        const int k0 = kF16TileKeys * (t0 + i) + kw0;  // this warp's first key of the tile
+        if (k0 >= any_sees) continue;  // nothing here that a live row of this warp may see
+        const __half* Kt = stages + (i % kF16Stages) * S::kStage + kw0 * S::kRow;
+        const __half* Vt = Kt + S::kTile;
+        // S = Q K^T
+        float s[NB][4];
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) s[nb][j] = 0.0f;
+#pragma unroll
+        for (int kp = 0; kp < DH / 32; ++kp) {
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb) {
+                uint32_t kf[4];
+                ldsm_x4(kf, Kt + (nb * 8 + (lane & 7)) * S::kRow + kp * 32 + 8 * (lane >> 3));
+                mma_f16(s[nb], qf[2 * kp], kf[0], kf[1]);
+                mma_f16(s[nb], qf[2 * kp + 1], kf[2], kf[3]);
+            }
+        }
+        // bias and mask (rows g and g + 8; a row's KW scores sit in its quad of lanes)
+        if (bias) {
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int key = k0 + nb * 8 + 2 * t + (j & 1);
+                    const float* bp = j >= 2 ? bias_hi : bias_lo;
+                    if (bp && key < (j >= 2 ? keys_hi : keys_lo)) s[nb][j] = fmaf(bp[key], kLog2e, s[nb][j]);
+                }
+        }
+        if (k0 + KW > all_see) {  // (warp-uniform) some row of this warp does not see some key of the block
+#pragma unroll
+            for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int key = k0 + nb * 8 + 2 * t + (j & 1);
+                    if (key >= (j >= 2 ? keys_hi : keys_lo) || key >= seq_keys) s[nb][j] = -FLT_MAX;
+                }
+        }
+        float tmax_lo = -FLT_MAX, tmax_hi = -FLT_MAX;
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+            tmax_lo = fmaxf(tmax_lo, fmaxf(s[nb][0], s[nb][1]));
+            tmax_hi = fmaxf(tmax_hi, fmaxf(s[nb][2], s[nb][3]));
+        }
+        tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(kFullMask, tmax_lo, 1));
+        tmax_lo = fmaxf(tmax_lo, __shfl_xor_sync(kFullMask, tmax_lo, 2));
+        tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(kFullMask, tmax_hi, 1));
+        tmax_hi = fmaxf(tmax_hi, __shfl_xor_sync(kFullMask, tmax_hi, 2));
+        const float new_lo = fmaxf(m_lo, tmax_lo), new_hi = fmaxf(m_hi, tmax_hi);
+        // (a masked score is -FLT_MAX: minus the maximum it stays far below ex2's underflow, unless the whole
+        // row is masked so far - then the maximum is -FLT_MAX too and the terms are dropped explicitly)
+        const bool none_lo = new_lo == -FLT_MAX, none_hi = new_hi == -FLT_MAX;
+        float sum_lo = 0.0f, sum_hi = 0.0f;
+        uint32_t pa[NB / 2][4];  // the probabilities as A fragments: 16 keys per k-step
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+            const float p0 = none_lo ? 0.0f : exp2_approx(s[nb][0] - new_lo), p1 = none_lo ? 0.0f : exp2_approx(s[nb][1] - new_lo);
+            const float p2 = none_hi ? 0.0f : exp2_approx(s[nb][2] - new_hi), p3 = none_hi ? 0.0f : exp2_approx(s[nb][3] - new_hi);
+            sum_lo += p0 + p1;
+            sum_hi += p2 + p3;
+            pa[nb / 2][(nb & 1) * 2] = pack_half2(p0, p1);
+            pa[nb / 2][(nb & 1) * 2 + 1] = pack_half2(p2, p3);
+        }
+        sum_lo += __shfl_xor_sync(kFullMask, sum_lo, 1);
+        sum_lo += __shfl_xor_sync(kFullMask, sum_lo, 2);
+        sum_hi += __shfl_xor_sync(kFullMask, sum_hi, 1);
+        sum_hi += __shfl_xor_sync(kFullMask, sum_hi, 2);
+        // O = O * rescale + P V (the rescale is skipped while no row of the warp has a new maximum)
+        if (__any_sync(kFullMask, new_lo != m_lo || new_hi != m_hi)) {
+            const float r_lo = exp2_approx(m_lo - new_lo), r_hi = exp2_approx(m_hi - new_hi);
+            l_lo *= r_lo;
+            l_hi *= r_hi;
+#pragma unroll
+            for (int n = 0; n < DH / 8; ++n) {
+                o[n][0] *= r_lo; o[n][1] *= r_lo; o[n][2] *= r_hi; o[n][3] *= r_hi;
+            }
+            m_lo = new_lo;
+            m_hi = new_hi;
+        }
+        l_lo += sum_lo;
+        l_hi += sum_hi;
+#pragma unroll
+        for (int n2 = 0; n2 < DH / 16; ++n2) {
+#pragma unroll
+            for (int kk = 0; kk < NB / 2; ++kk) {
+                uint32_t vf[4];
+                ldsm_x4_trans(vf, Vt + (kk * 16 + (lane & 7) + 8 * ((lane >> 3) & 1)) * S::kRow + n2 * 16 + 8 * (lane >> 4));
+                mma_f16(o[2 * n2], pa[kk], vf[0], vf[1]);
+                mma_f16(o[2 * n2 + 1], pa[kk], vf[2], vf[3]);
+            }
+        }
+    }
+    cp_async_wait<0>();
+
+    // park this warp's state in stage 0: [warp][query of the block][max (base-2 units), sum, O[DH]]
+    __syncthreads();
+    float* states = reinterpret_cast<float*>(stages);
+    float* merged_buf = reinterpret_cast<float*>(stages + S::kStage);
+    {
+        float* st = states + warp * 16 * (DH + 2);
+#pragma unroll
+        for (int n = 0; n < DH / 8; ++n) {
+            *reinterpret_cast<float2*>(st + g * (DH + 2) + 2 + n * 8 + 2 * t) = make_float2(o[n][0], o[n][1]);
+            *reinterpret_cast<float2*>(st + (g + 8) * (DH + 2) + 2 + n * 8 + 2 * t) = make_float2(o[n][2], o[n][3]);
+        }
+        if (t == 0) {
+            st[g * (DH + 2)] = m_lo;
+            st[g * (DH + 2) + 1] = l_lo;
+            st[(g + 8) * (DH + 2)] = m_hi;
+            st[(g + 8) * (DH + 2) + 1] = l_hi;
+        }
+    }
+    __syncthreads();
+    // Merge the key parts of every query block (in part order).  One slice in all: the merged state is the
+    // whole answer and is normalised and written here.  Otherwise the slice's state of every live query goes
+    // to the cluster merge (FUSED) or to global memory for the combine kernel, its maximum in natural units.
+    const bool whole = FUSED && slices == 1;
+    for (int i = tid; i < QN * (DH + 2); i += 32 * kF16Warps) {
+        const int qi = i / (DH + 2), e = i % (DH + 2);
+        const int q = qb * kF16MaxQueries + qi;
+        if (q >= queries && !(FUSED && !whole)) continue;
+        const float* sw0 = states + ((qi / 16) * 16 * (DH + 2)) + (qi % 16) * (DH + 2);  // warp (qi / 16) + MB * part
+        float mm = -FLT_MAX;
+#pragma unroll
+        for (int kp = 0; kp < KP; ++kp) mm = fmaxf(mm, sw0[kp * MB * 16 * (DH + 2)]);
+        float merged = 0.0f, l = 0.0f;
+#pragma unroll
+        for (int kp = 0; kp < KP; ++kp) {
+            const float* sw = sw0 + kp * MB * 16 * (DH + 2);
+            const float w = exp2_approx(sw[0] - mm);  // (both -FLT_MAX: weight 1 on an empty state)
+            merged += sw[e] * w;
+            l += sw[1] * w;
+        }
+        if (e == 0) merged = mm == -FLT_MAX ? -FLT_MAX : mm * kLn2;
+        if (whole) {
+            if (e < 2) continue;
+            const float y = l > 0.0f ? merged / l : 0.0f;  // an inactive row has no keys
+            const size_t at = (static_cast<size_t>(q_row[qi]) * n_heads + q_head[qi]) * DH + (e - 2);
+            if (out.att) out.att[at] = y;
+            if (out.hi) {
+                const __nv_bfloat16 h = __float2bfloat16_rn(y);
+                out.hi[at] = h;
+                out.lo[at] = __float2bfloat16_rn(y - __bfloat162float(h));
+            }
+        } else if (FUSED) {
+            merged_buf[i] = merged;
+        } else {
+            part[((static_cast<size_t>(q_row[qi]) * n_heads + q_head[qi]) * slices + slice) * (DH + 2) + e] = merged;
+        }
+    }
+    if (FUSED && !whole) {
+        __syncthreads();
+        cluster_merge_write<DH>(merged_buf, QN, qb * kF16MaxQueries, queries, b, m_rows, group, kv_head, n_heads, slices, out);
+    }
+}
+
 // grid = rows * n_heads, block = DH: merge the key slices of one (row, head).
 template <int DH>
 __global__ void attention_combine_kernel(const float* __restrict__ part, int slices, float* __restrict__ att,
@@ -516,6 +872,14 @@ bool attention_uses_mma(const Model& m, int batch, int m_rows, int max_keys) {
     return m.bf16() && queries >= min_queries && pairs >= 65536;
 }
 
+// fp16 K,V rows take the f16 tensor-core kernel where the tf32 one would run, from 32 (sequence, KV head)
+// pairs on: measured on the 7B shape with 1024 cached tokens, per block, against the tf32 kernel converting
+// the same rows: batch 4 x 3 rows 104 vs 110 us, 8 x 3 113 vs 135, 16 x 5 165 vs 227, 32 x 7 317 vs 452,
+// 32 x 1 141 vs 185; at batch 1 (8 pairs) its 64-key tiles leave too few CTAs and it loses 1 - 4 us per block.
+bool attention_uses_f16(const Model& m, int batch, int m_rows, int max_keys) {
+    return m.kv_dtype == SPEC_DTYPE_FP16 && batch * m.cfg.n_kv_heads >= 32 && attention_uses_mma(m, batch, m_rows, max_keys);
+}
+
 // The key slices can be merged inside a cluster (no second kernel) whenever a CTA
 // holds all its queries' states at once: always on the tensor-core path, and on
 // the warp-per-query path when the queries fit one round of warps.  It is done
@@ -530,6 +894,14 @@ int attention_slices(const Model& m, int batch, int m_rows, int max_len) {
     const int n_kv_heads = m.cfg.n_kv_heads;
     const int queries = (m.cfg.n_heads / n_kv_heads) * m_rows;
     const int tiles = (max_len + 31) / 32;
+    if (attention_uses_f16(m, batch, m_rows, max_len)) {
+        // one wave of CTAs (two per SM at d_head 128, four at 64), a 64-key tile per slice at least
+        const int groups = batch * n_kv_heads * ((queries + kF16MaxQueries - 1) / kF16MaxQueries);
+        const int resident = 148 * (m.cfg.d_head == 64 ? 4 : 2);
+        const int want = std::max(1, resident / groups);
+        const int most = std::max(1, (max_len + kF16TileKeys - 1) / kF16TileKeys);
+        return std::max(1, std::min(std::min(want, most), cap));
+    }
     if (attention_uses_mma(m, batch, m_rows, max_len)) {
         // one wave of CTAs (shared memory allows one per SM at d_head 128, two at 64; twice that from 64
         // (sequence, KV head, query block) groups on, where K and V share a buffer - measured: 16 sequences
@@ -559,11 +931,11 @@ size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices) {
 // slices merge inside a cluster (no combine kernel), whether K and V share one staging buffer.
 AttentionPlan attention_plan(const Model& m, int batch, int m_rows, int max_keys) {
     AttentionPlan plan{};
-    plan.tensor_cores = attention_uses_mma(m, batch, m_rows, max_keys) ? 1 : 0;
+    plan.tensor_cores = attention_uses_f16(m, batch, m_rows, max_keys) ? 2 : attention_uses_mma(m, batch, m_rows, max_keys) ? 1 : 0;
     plan.slices = attention_slices(m, batch, m_rows, max_keys);
     plan.cluster_merge = attention_merges_in_cluster(m, batch, m_rows, max_keys) && plan.slices <= kMaxClusterSlices ? 1 : 0;
     const int queries = (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows;
-    plan.in_turn = plan.tensor_cores && batch * m.cfg.n_kv_heads * ((queries + 15) / 16) >= 32 ? 1 : 0;
+    plan.in_turn = plan.tensor_cores == 1 && batch * m.cfg.n_kv_heads * ((queries + 15) / 16) >= 32 ? 1 : 0;
     return plan;
 }
 
@@ -610,6 +982,32 @@ int launch_attention_variant(const Model& m, const AttnSource& src, const RowMet
     const bool fused = attention_merges_in_cluster(m, batch, m_rows, max_keys) && slices <= kMaxClusterSlices;
     const KV* pool = static_cast<const KV*>(src.pool.kv);
     int status;
+    if constexpr (std::is_same<KV, __half>::value) {
+        if (attention_uses_f16(m, batch, m_rows, max_keys)) {
+            const int q_blocks = (queries + kF16MaxQueries - 1) / kF16MaxQueries;
+            const int per_cta = std::min(queries, kF16MaxQueries);
+            const dim3 grid(slices, m.cfg.n_kv_heads * q_blocks, batch);
+#define SPEC_LAUNCH_F16(MB, F, CLUSTER)                                                                                 \
+    do {                                                                                                                \
+        static std::atomic<unsigned long long> configured{0};                                                           \
+        if (first_use_on_this_device(configured))                                                                       \
+            SPEC_CUDA_TRY(cudaFuncSetAttribute(attention_f16_kernel<DH, MB, F>,                                         \
+                                               cudaFuncAttributeMaxDynamicSharedMemorySize,                             \
+                                               static_cast<int>(F16Smem<DH, MB>::kBytes)));                             \
+        status = launch_attn(attention_f16_kernel<DH, MB, F>, grid, dim3(32 * kF16Warps), F16Smem<DH, MB>::kBytes,      \
+                             CLUSTER, stream, src.q, src.q_stride, rows.pos, rows.seq, m_rows, m.cfg.n_heads,           \
+                             m.cfg.n_kv_heads, q_blocks, pool, src.pool.page_table, src.pool.pages_per_seq,             \
+                             src.pool.page_size, src.kv_len, src.bias, src.bias_span, src.bias_zero, scale, part, out); \
+    } while (0)
+            if (per_cta <= 16) { if (fused) SPEC_LAUNCH_F16(1, true, slices); else SPEC_LAUNCH_F16(1, false, 0); }
+            else if (per_cta <= 32) { if (fused) SPEC_LAUNCH_F16(2, true, slices); else SPEC_LAUNCH_F16(2, false, 0); }
+            else { if (fused) SPEC_LAUNCH_F16(4, true, slices); else SPEC_LAUNCH_F16(4, false, 0); }
+#undef SPEC_LAUNCH_F16
+            if (status != SPEC_OK || fused) return status;
+            return launch_pdl(attention_combine_kernel<DH>, dim3(n_rows * m.cfg.n_heads), dim3(DH), 0, stream,
+                              static_cast<const float*>(part), slices, out.att, out.hi, out.lo);
+        }
+    }
     if (attention_uses_mma(m, batch, m_rows, max_keys)) {
         const int m_blocks = (queries + 15) / 16;
         const dim3 grid(slices, m.cfg.n_kv_heads * m_blocks, batch);

@@ -60,16 +60,24 @@ def test_long_context_verify_rows_at_batch_one(wide_block):
         eng.close()
 
 
-def test_ragged_batch_of_sixteen_with_rollback(wide_block):
+_RAGGED_ORACLE = {}
+
+
+@pytest.mark.parametrize("kv_dtype", ["fp16", "fp32"])
+def test_ragged_batch_of_sixteen_with_rollback(wide_block, kv_dtype):
     """16 sequences x 5 rows over ragged cached lengths (453 .. 1008 tokens), then a ragged roll-back
-    (0 .. 4 of the 5 rows kept) and 5 more rows: the tensor-core attention with K and V staged in
-    turn (two CTAs per SM), two 16-query blocks per KV head, 80-row GEMM tiles."""
+    (0 .. 4 of the 5 rows kept) and 5 more rows, 80-row GEMM tiles.  fp16 rows (the default): the f16
+    tensor-core attention, the 20 queries of a KV head in one CTA, two key slices merged in a cluster.
+    fp32 rows: the tf32 tensor-core attention with K and V staged in turn, two 16-query blocks per KV head."""
     cfg, w, oracle = wide_block
     B, rows = 16, 5
-    eng = binding.Engine(cfg, w, max_batch=B, max_len=MAX_LEN, page_size=64, max_gamma=15)
+    eng = binding.Engine(cfg, w, max_batch=B, max_len=MAX_LEN, page_size=64, max_gamma=15, kv_dtype=kv_dtype)
     try:
         plan = eng.attention_plan(0, B, rows)
-        assert plan["tensor_cores"] and plan["in_turn"], plan
+        if kv_dtype == "fp16":
+            assert plan["f16"] and plan["cluster_merge"] and plan["slices"] == 2, plan
+        else:
+            assert plan["tensor_cores"] and not plan["f16"] and plan["in_turn"], plan
         seqs = np.stack([workloads.make_prompt(100 + b, 1008 + 2 * rows, cfg["vocab"]) for b in range(B)])
         eng.reset()
         _feed(eng, 0, seqs[:, :1008], 16)
@@ -84,8 +92,11 @@ def test_ragged_batch_of_sixteen_with_rollback(wide_block):
         assert binding.spec_device_error() == 0
         worst = 0.0
         for b in (0, 3, 6, 9, 12, 15):                         # the oracle is slow at this width: six of the sixteen
-            a = oracle.forward_full(np.concatenate([seqs[b, :lengths[b]], first[b]]), last=rows)
-            c = oracle.forward_full(np.concatenate([seqs[b, :lengths[b]], first[b, :keep[b]], second[b]]), last=rows)
+            if b not in _RAGGED_ORACLE:                        # (the same for both cache types)
+                _RAGGED_ORACLE[b] = (
+                    oracle.forward_full(np.concatenate([seqs[b, :lengths[b]], first[b]]), last=rows),
+                    oracle.forward_full(np.concatenate([seqs[b, :lengths[b]], first[b, :keep[b]], second[b]]), last=rows))
+            a, c = _RAGGED_ORACLE[b]
             worst = max(worst, np.abs(got1[b] - a).max(), np.abs(got2[b] - c).max())
         assert worst <= BF16_ABS, f"max absolute logit error {worst:.3g}"
     finally:
@@ -111,14 +122,14 @@ def test_benchmark_gemm_shapes_against_the_plain_definition(rows, n_out, k):
 
 def test_cross_attention_over_a_long_source_on_the_tensor_cores():
     """Six decoder rows of eight sequences over sources of up to 512 tokens: the cross-attention
-    (and here the self-attention too) takes the tensor-core kernel."""
+    (and here the self-attention too, with its relative-position bias) takes the f16 tensor-core kernel."""
     cfg = workloads.model_config("t5_test_target")
     w = workloads.make_weights(cfg, 1)
     B, rows = 8, 6
     eng = binding.Engine(cfg, w, max_batch=B, max_len=512, page_size=64, max_gamma=rows - 1, max_src_len=512)
     try:
-        assert eng.attention_plan(0, B, rows, cross=True)["tensor_cores"]
-        assert eng.attention_plan(0, B, rows)["tensor_cores"]
+        assert eng.attention_plan(0, B, rows, cross=True)["f16"]
+        assert eng.attention_plan(0, B, rows)["f16"]
         sources = [workloads.make_prompt(300 + b, n, cfg["vocab"]) for b, n in enumerate([512, 509, 480, 333, 257, 129, 64, 7])]
         eng.encode(sources)
         tokens = np.stack([np.concatenate([[START_TOKEN], workloads.make_prompt(400 + b, 2 * rows - 1, cfg["vocab"])])
