@@ -792,6 +792,14 @@ def run_generation(args, wl, torch, device, local, barrier):
         kv_bytes = wl.kv_bytes(wl.pass_context)
         pass_bytes = weight_stream_bytes(wl.tcfg) + kv_bytes
         pass_gbs = pass_bytes / (times["target_rows_ms"] / 1e3) / 1e9
+        # DRAM bytes of one pass from the ncu capture of a 2-block cut of the 7B-shaped target (batch 1, 3 rows, 1024 cached
+        # tokens): 363.7 MB per block (354.4 MB of weights), 266.8 MB for the head, embedding and final norm; traffic grows in
+        # proportion to the blocks.  Only for the workload that capture is of.
+        pass_traffic, pass_traffic_note = None, "no capture for this workload"
+        if args.workload == "llama7b" and wl.batch == 1 and wl.gamma == 2 and not args.layers:
+            pass_traffic = wl.tcfg["n_layers"] * 363.7e6 + 266.8e6
+            pass_traffic_note = ("dram__bytes_read.sum + dram__bytes_write.sum of every kernel of a pass, captured on a 2-block "
+                                 "cut and scaled by the block count (profiles/ncu_pass_traffic_llama7b_rows3_ctx1024.txt)")
         long_tokens, long_ms, long_stats = wl.timed_decode(args.warmup, long_steps, wl.gamma)
         # the other configurations of the scope, measured in this same run (short: 30 iterations each)
         others = []
@@ -843,10 +851,8 @@ def run_generation(args, wl, torch, device, local, barrier):
                          "peak_kind": f"of {peak_kind}", "frac_of_nominal_8tbs": pass_gbs / 8000.0,
                          "algorithmic_bytes_per_pass": pass_bytes, "weight_bytes": weight_stream_bytes(wl.tcfg),
                          "kv_bytes": kv_bytes, "ms_per_pass": times["target_rows_ms"],
-                         "traffic": None,
-                         "traffic_note": "not captured for the whole pass; from profile: the four GEMMs of a 7B-shaped block "
-                                         "move 363.6 MB of DRAM traffic for 354.4 MB of weights (x 1.026, "
-                                         "profiles/ncu_gemm_tc_llama7b_layer.txt)",
+                         "traffic": pass_traffic,
+                         "traffic_note": pass_traffic_note,
                          "note": "weights + K,V rows of the context in the cache's element type (for encoder-decoders also "
                                  "the source rows), one pass over gamma+1 rows, graph replays timed with events on the "
                                  "library's stream",

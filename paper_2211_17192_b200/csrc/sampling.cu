@@ -7,11 +7,14 @@
 //      to (max, sum exp) with an online rescale, and also picks up the row's
 //      logit at the drafted token.  No CTA talks to another: the kernel is a
 //      pure map-reduce and runs at streaming bandwidth.
-//   2. verify_finish_kernel, one CTA per sequence, merges the chunk statistics,
-//      runs the gamma accept tests, and re-reads only row n+1 of p and q (still
-//      in L2) to normalise the residual max(0, p - q) and draw from it by
-//      inverse CDF.  It is chained with programmatic dependent launch, so its
-//      launch latency and prologue overlap the tail of the first kernel.
+//   2. verify_finish_kernel, one cluster of CTAs per sequence, merges the chunk
+//      statistics, runs the gamma accept tests, and re-reads only row n+1 of p
+//      and q (still in L2) to normalise the residual max(0, p - q) and draw from
+//      it by inverse CDF: every warp keeps the weights of its segment in
+//      registers, the segment totals are scanned once across the cluster, and
+//      the warp whose segment holds the target walks it without another trip to
+//      memory.  It is chained with programmatic dependent launch, so its launch
+//      latency and prologue overlap the tail of the first kernel.
 #include <algorithm>
 #include <cfloat>
 #include <mutex>
@@ -25,11 +28,12 @@ namespace cg = cooperative_groups;
 namespace spec {
 namespace {
 
-constexpr int kStatThreads = 512;
+constexpr int kStatThreads = 256;
 constexpr int kStatWarps = kStatThreads / 32;
 constexpr int kUnroll = 4;              // 128-bit loads in flight per thread while streaming
-constexpr int kMinChunkGroups = 1024;   // a CTA streams at least 4096 logits (unless the row is shorter)
-constexpr int kTargetCtas = 148 * 24;   // about six waves of resident CTAs, so that the last wave costs little
+constexpr int kMinChunkGroups = 1000;   // a CTA streams at least 4000 logits (unless the row is shorter)
+constexpr int kTargetCtas = 148 * 48;   // about six waves of resident CTAs (eight of 256 threads per SM), so that the last wave
+                                        // costs little; smaller CTAs stagger their reduce-and-restart pauses (512 threads: +0.8 us)
 constexpr int kFinishThreads = 512;
 constexpr int kCdfBatch = 8;            // groups fetched per thread before any is consumed (inverse CDF, one CTA)
 constexpr int kClusterCdfBatch = 4;     // the same when a cluster shares the row
@@ -186,6 +190,37 @@ __device__ __forceinline__ int pick_part(PartAt part_at, int count, float target
     return hit;
 }
 
+// One step of the walk: the 128 elements of groups gs .. gs + 31 (lane l holds the four weights of group
+// gs + l), in index order after the weight `run` already passed.  Sets `found` to the first index whose running
+// sum exceeds `rem` (if want_hit), keeps `last_pos` = the last index with positive weight so far.
+__device__ __forceinline__ void walk_step(const float4& v, int gs, int lane, bool want_hit, float rem, float& run, int& found,
+                                          int& last_pos) {
+    const float mine = (v.x + v.y) + (v.z + v.w);
+    const float incl = warp_inclusive_scan(mine, lane);
+    const unsigned over = want_hit ? __ballot_sync(kFullMask, run + incl > rem) : 0u;
+    const unsigned pos = __ballot_sync(kFullMask, mine > 0.0f);
+    if (pos) {
+        const int pl = 31 - __clz(pos);  // last lane with positive weight in this step
+        const float py = __shfl_sync(kFullMask, v.y, pl), pz = __shfl_sync(kFullMask, v.z, pl),
+                    pw = __shfl_sync(kFullMask, v.w, pl);
+        const int pg = 4 * (gs + pl);
+        last_pos = pw > 0.f ? pg + 3 : pz > 0.f ? pg + 2 : py > 0.f ? pg + 1 : pg;
+    }
+    if (over) {
+        const int hl = __ffs(over) - 1;
+        const float excl = __shfl_sync(kFullMask, incl - mine, hl) + run;
+        const float hx = __shfl_sync(kFullMask, v.x, hl), hy = __shfl_sync(kFullMask, v.y, hl),
+                    hz = __shfl_sync(kFullMask, v.z, hl);
+        const int hg = 4 * (gs + hl);
+        float c = excl + hx;
+        if (c > rem) found = hg;
+        else if ((c += hy) > rem) found = hg + 1;
+        else if ((c += hz) > rem) found = hg + 2;
+        else found = hg + 3;
+    }
+    run += __shfl_sync(kFullMask, incl, 31);
+}
+
 // The draw inside one contiguous range of groups [r0, r1) by a whole CTA: `rem`
 // is the target minus the weight in front of the range.  Long ranges are first
 // cut into one sub-range per warp; warp 0 then walks the chosen (sub-)range 128
@@ -232,31 +267,7 @@ __device__ int locate_in_range(const Weights& w, int r0, int r1, float rem, bool
             for (int i = 0; i < kWalkBatch; ++i) {
                 const int gs = gb + 32 * i;
                 if (gs >= r1 || found >= 0) break;
-                const float4 v = w.weigh(raw[i]);
-                const float mine = (v.x + v.y) + (v.z + v.w);
-                const float incl = warp_inclusive_scan(mine, lane);
-                const unsigned over = want_hit ? __ballot_sync(kFullMask, run + incl > rem) : 0u;
-                const unsigned pos = __ballot_sync(kFullMask, mine > 0.0f);
-                if (pos) {
-                    const int pl = 31 - __clz(pos);  // last lane with positive weight in this step
-                    const float py = __shfl_sync(kFullMask, v.y, pl), pz = __shfl_sync(kFullMask, v.z, pl),
-                                pw = __shfl_sync(kFullMask, v.w, pl);
-                    const int pg = 4 * (gs + pl);
-                    last_pos = pw > 0.f ? pg + 3 : pz > 0.f ? pg + 2 : py > 0.f ? pg + 1 : pg;
-                }
-                if (over) {
-                    const int hl = __ffs(over) - 1;
-                    const float excl = __shfl_sync(kFullMask, incl - mine, hl) + run;
-                    const float hx = __shfl_sync(kFullMask, v.x, hl), hy = __shfl_sync(kFullMask, v.y, hl),
-                                hz = __shfl_sync(kFullMask, v.z, hl);
-                    const int hg = 4 * (gs + hl);
-                    float c = excl + hx;
-                    if (c > rem) found = hg;
-                    else if ((c += hy) > rem) found = hg + 1;
-                    else if ((c += hz) > rem) found = hg + 2;
-                    else found = hg + 3;
-                }
-                run += __shfl_sync(kFullMask, incl, 31);
+                walk_step(w.weigh(raw[i]), gs, lane, want_hit, rem, run, found, last_pos);
             }
         }
         if (lane == 0) {
@@ -323,7 +334,29 @@ __device__ int cluster_inverse_cdf(const Weights& w, int vocab, float u, CdfScra
         return min(c1, seg_begin(part) + seg);
     };
     const int mine = rank * WARPS + warp;
-    const float acc = warp_range_sum<kClusterCdfBatch>(w, seg_begin(mine), seg_end(mine), lane);
+    const int b0 = seg_begin(mine), b1 = seg_end(mine);
+    // When a warp's segment fits one batch of fetches, the weights stay in registers: the warp whose segment
+    // holds the target then walks it without going back to memory.
+    const bool keep = seg <= 32 * kClusterCdfBatch;  // (uniform across the cluster)
+    float4 kept[kClusterCdfBatch];
+    float acc;
+    if (keep) {
+        typename Weights::Raw raw[kClusterCdfBatch];
+#pragma unroll
+        for (int i = 0; i < kClusterCdfBatch; ++i) {
+            const int g = b0 + lane + 32 * i;
+            raw[i] = g < b1 ? w.fetch(g) : w.nothing();
+        }
+        acc = 0.0f;
+#pragma unroll
+        for (int i = 0; i < kClusterCdfBatch; ++i) {
+            kept[i] = w.weigh(raw[i]);
+            acc += (kept[i].x + kept[i].y) + (kept[i].z + kept[i].w);
+        }
+        acc = warp_sum(acc);
+    } else {
+        acc = warp_range_sum<kClusterCdfBatch>(w, b0, b1, lane);
+    }
     if (lane == 0) s.part[warp] = acc;
     cluster.sync();
     // warp 0 copies every CTA's totals into this CTA's shared memory ...
@@ -331,6 +364,9 @@ __device__ int cluster_inverse_cdf(const Weights& w, int vocab, float u, CdfScra
     if (warp == 0)
         for (int i = lane; i < parts; i += 32) s.all[i] = cluster.map_shared_rank(s.part, i / WARPS)[i % WARPS];
     __syncthreads();
+    // (this CTA has read its peers' totals: it arrives at the cluster barrier now and waits for the others only
+    // when it is about to leave, so the CTA that resolves the draw does not stand still meanwhile)
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     // ... and scans them: lane l takes the consecutive parts [l*per, (l+1)*per)
     if (warp == 0) {
         const int per = (parts + 31) / 32;
@@ -360,14 +396,35 @@ __device__ int cluster_inverse_cdf(const Weights& w, int vocab, float u, CdfScra
     const float total = s.pick_total;
     const float target = u * total;
     const float before = s.pick_before;
-    int hit = s.pick_part_index;
-    const bool want_hit_flag = s.pick_hit != 0;
-    cluster.sync();  // nobody reads another CTA's totals after this point
-    const bool want_hit = want_hit_flag;
+    const int hit = s.pick_part_index;
+    const bool want_hit = s.pick_hit != 0;
     *total_out = total;
-    if (hit / WARPS != rank) return -1;
-    const int k = locate_in_range<WARPS>(w, seg_begin(hit), seg_end(hit), target - before, want_hit, s);
-    return max(0, min(k, vocab - 1));
+    int k = -1;
+    if (hit / WARPS == rank) {  // (uniform across the CTA)
+        if (keep) {
+            if (warp == hit % WARPS) {
+                float run = 0.0f;
+                int found = -1, last_pos = -1;
+#pragma unroll
+                for (int i = 0; i < kClusterCdfBatch; ++i) {
+                    const int gs = b0 + 32 * i;
+                    if (gs >= b1 || found >= 0) break;
+                    walk_step(kept[i], gs, lane, want_hit, target - before, run, found, last_pos);
+                }
+                if (lane == 0) {
+                    s.result = found;
+                    s.last_positive = last_pos;
+                }
+            }
+            __syncthreads();
+            k = s.result >= 0 ? s.result : s.last_positive;
+        } else {
+            k = locate_in_range<WARPS>(w, seg_begin(hit), seg_end(hit), target - before, want_hit, s);
+        }
+        k = max(0, min(k, vocab - 1));
+    }
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");  // nobody reads this CTA's totals any more
+    return k;
 }
 
 // (max, lowest index attaining it) across a CTA of 32 * WARPS threads; the
@@ -498,6 +555,7 @@ struct FinishShared {
     float row_aux[kMaxRows];
     float row_x[kMaxRows];
     CdfScratch<kFinishThreads / 32> cdf;
+    float u_cand[kMaxGamma + 1];
     float u_final;
     int n;
 };
@@ -534,24 +592,28 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
     // lenient argmax decoding compares the target's logit at the drafted token with the row maximum
     float my_xlogit = 0.0f;
     if (GREEDY && lenience < 1.0f && tid < gamma && my_x >= 0 && my_x < vocab) my_xlogit = __ldg(tl + static_cast<size_t>(tid) * vocab + my_x);
+    // The generation loop keys the final draw by the position it decides, which depends on n: it passes one
+    // candidate uniform per possible n; all of them are fetched now.
+    if (!GREEDY && final_uniforms && tid <= gamma) sh.u_cand[tid] = __ldg(final_uniforms + static_cast<size_t>(b) * (gamma + 1) + tid);
     pdl_trigger();
     pdl_wait();
 
-    // merge the chunk statistics of row `tid` (four loads in flight at a time)
+    // merge the chunk statistics of row `tid` (eight loads in flight at a time)
     if (tid < rows) {
         const ChunkStat* st_r = stats + (static_cast<size_t>(b) * rows + tid) * chunks;
         float M = -FLT_MAX, A = 0.0f, X = 0.0f;
         int best = 0x7fffffff;
         bool bad = false;
         const int xchunk = (my_x >= 0 && my_x < vocab) ? (my_x >> 2) / per_chunk : -1;
-        for (int c0 = 0; c0 < chunks; c0 += 4) {
-            float4 st[4];
+        constexpr int kMergeBatch = 8;  // chunk statistics fetched together
+        for (int c0 = 0; c0 < chunks; c0 += kMergeBatch) {
+            float4 st[kMergeBatch];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < kMergeBatch; ++i)
                 st[i] = c0 + i < chunks ? __ldcg(reinterpret_cast<const float4*>(st_r + c0 + i))
                                         : make_float4(-FLT_MAX, __int_as_float(0x7fffffff), 0.0f, 0.0f);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < kMergeBatch; ++i) {
                 if (c0 + i >= chunks) break;
                 if (GREEDY) {
                     const int ci = __float_as_int(st[i].y);
@@ -602,9 +664,7 @@ verify_finish_kernel(const float* __restrict__ target_logits, const float* __res
         if (rank == 0) token = __float_as_int(sh.row_aux[n]);
     } else {
         constexpr int W = kFinishThreads / 32;
-        // The generation loop keys the final draw by the position it decides, which
-        // depends on n: it passes one candidate uniform per possible n.
-        const float u = final_uniforms ? __ldg(final_uniforms + static_cast<size_t>(b) * (gamma + 1) + n) : sh.u_final;
+        const float u = final_uniforms ? sh.u_cand[n] : sh.u_final;
         PlainWeights<VEC, CUT> pw;
         const float* fl = CUT ? floors + static_cast<size_t>(b) * rows : nullptr;
         pw.p = make_row<VEC, CUT>(tl + static_cast<size_t>(n) * vocab, vocab, CUT ? __ldcg(fl + n) : -INFINITY);
