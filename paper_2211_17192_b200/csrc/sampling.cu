@@ -522,10 +522,13 @@ verify_stats_kernel(const float* __restrict__ target_logits, const float* __rest
                 bm = fmaxf(bm, fmaxf(fmaxf(v[i].x, v[i].y), fmaxf(v[i].z, v[i].w)));
             s *= fast_exp2((m - bm) * c2);
             m = bm;
+            // exp2(v * c2 - m * c2): one multiply-add per logit (the kernel is close to issue-bound).  A thread that has
+            // seen only padding keeps m = -FLT_MAX: the product is clamped so that -inf * c2 + it stays -inf.
+            const float mc = fminf(-m * c2, FLT_MAX);
 #pragma unroll
             for (int i = 0; i < kUnroll; ++i)
-                s += (fast_exp2((v[i].x - m) * c2) + fast_exp2((v[i].y - m) * c2)) +
-                     (fast_exp2((v[i].z - m) * c2) + fast_exp2((v[i].w - m) * c2));
+                s += (fast_exp2(fmaf(v[i].x, c2, mc)) + fast_exp2(fmaf(v[i].y, c2, mc))) +
+                     (fast_exp2(fmaf(v[i].z, c2, mc)) + fast_exp2(fmaf(v[i].w, c2, mc)));
         }
     }
     ChunkStat* out = stats + (static_cast<size_t>(b) * rows + row) * chunks + chunk;
