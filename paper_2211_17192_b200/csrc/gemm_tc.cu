@@ -157,7 +157,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     uint64_t* acc_bar = empty_bar + S::kStages;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_bar + 1);
 
-    pdl_trigger();  // the next kernel may start its own prologue
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x, split = blockIdx.y, splits = gridDim.y, tok0 = blockIdx.z * N_TOK;
     const int kb0 = static_cast<int>(static_cast<long long>(k_blocks) * split / splits);
@@ -238,6 +237,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     }
     __syncwarp();
     pdl_wait();  // (already satisfied for the producer) nothing below may overtake the previous kernel
+    // The next kernel is released here, when this CTA's copies and MMAs have been issued, not at the top: the small
+    // kernel that follows a GEMM has no prologue worth starting early, and its CTAs arriving while the stream is at
+    // full rate cost more than they gain (measured per block: 97M shape 28.8 -> 27.0 us, 7B 94.8 -> 94.5).
+    pdl_trigger();
 
     // ---- epilogue: all four warps, warp w reads accumulator lanes 32w .. 32w+31 ----
     if (kb1 > kb0) {  // one lane polls, the warp takes one decision (the tensor-memory loads below are warp-wide)
