@@ -90,7 +90,6 @@ norm_kernel(float* h, const float* __restrict__ partial, int splits, int n_rows,
             const int32_t* __restrict__ src_rows, int d, float eps, float* __restrict__ out,
             __nv_bfloat16* __restrict__ out_hi, __nv_bfloat16* __restrict__ out_lo) {
     __shared__ float red[THREADS / 32];
-    pdl_trigger();
     const int r = blockIdx.x;
     const int groups = d / 4;
     // the gains are constants: fetched while the kernel before this one is still finishing
@@ -101,6 +100,10 @@ norm_kernel(float* h, const float* __restrict__ partial, int splits, int n_rows,
         gg[j] = g < groups ? *reinterpret_cast<const float4*>(gain + 4 * g) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     pdl_wait();
+    // The GEMM that follows is released only now, when the GEMM before this kernel is complete: released earlier, its CTAs
+    // take the places of that GEMM's leaving CTAs and their first weight tiles compete with the tail of its stream
+    // (measured per 7B block: 94.5 -> 93.1 us; releasing at the end of this kernel instead: 95.1).
+    pdl_trigger();
     const size_t src = static_cast<size_t>(src_rows ? src_rows[r] : r) * d;
     const size_t stride = static_cast<size_t>(n_rows) * d;
     float4 v[kNormPerThread];
