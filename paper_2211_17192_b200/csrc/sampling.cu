@@ -125,8 +125,10 @@ struct ResidualWeights {
         return Raw{z, z};
     }
     __device__ __forceinline__ float one(float lp, float lq) const {
-        const float pv = fast_exp2((lp - max_p) * c2) * inv_sum_p;
-        const float qv = fast_exp2((lq - max_q) * c2) * inv_sum_q;
+        // (both products are rounded before the subtraction: contracted into a multiply-add, one of them would not
+        // be, and p = q would leave rounding residue instead of the exact zero that the fallback to p tests for)
+        const float pv = __fmul_rn(fast_exp2((lp - max_p) * c2), inv_sum_p);
+        const float qv = __fmul_rn(fast_exp2((lq - max_q) * c2), inv_sum_q);
         return fmaxf(0.0f, pv - qv);
     }
     __device__ __forceinline__ float4 weigh(const Raw& r) const {

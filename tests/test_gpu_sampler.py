@@ -110,6 +110,24 @@ def test_identical_and_disjoint_distributions():
     compare_verify(n, t, tl2, ql2, xs2, us, 1.0)
 
 
+@pytest.mark.parametrize("vocab", [32000, 4096])
+def test_vanished_residual_falls_back_to_the_target_row(vocab):
+    """p = q and a rejection all the same (a guess outside the vocabulary is rejected by rule): max(0, p - q)
+    sums to zero, so t is a plain draw from p_{n+1} (the reading taken for a vanishing normaliser).  At vocabulary
+    32000 the draw runs in a 4-CTA cluster and the inverse CDF is entered twice (residual, then plain)."""
+    batch, gamma = 3, 2
+    tl, _ = workloads.make_sampler_logits(12, batch, gamma, vocab, 1.0)
+    ql = np.ascontiguousarray(tl[:, :gamma])
+    first = oracle_sampling.sample_token(ql[2, 0], 0.37, 1.0)[0]  # a guess q_1 can give: accepted, since p_1 = q_1
+    xs = np.array([[-1, 5], [vocab, 1], [first, -1]], dtype=np.int32)
+    us = workloads.make_uniform_grid(13, (batch, gamma + 1))
+    n, t = _run(tl, ql, xs, us, 1.0)
+    assert n.cpu().tolist() == [0, 0, 1]
+    for b, rows_kept in enumerate([0, 0, 1]):
+        ref, margin = oracle_sampling.sample_token(tl[b, rows_kept], us[b, gamma], 1.0)
+        assert int(t[b]) == ref or margin < MARGIN
+
+
 def test_out_of_range_draft_token_is_rejected():
     tl, ql = workloads.make_sampler_logits(6, 2, 3, 500, 0.1)
     xs = np.array([[1, 500, 2], [-1, 3, 4]], dtype=np.int32)
