@@ -57,6 +57,23 @@ def test_temperature_zero_equals_target_only_greedy(tiny, gamma):
     assert stats["iterations"] >= 40 / (gamma + 1)
 
 
+def test_shortest_prompts_fewest_tokens_and_surplus_guesses(tiny):
+    """Prompts of 1, 2 and 3 tokens (the first draft step feeds positions L-2 and L-1: with one token there is
+    no L-2), 1, 2 and 5 new tokens with gamma = 1 and gamma = 8 (more guesses than tokens wanted: the surplus of
+    the last iteration is dropped), sampled and greedy: token for token the oracle's stream."""
+    eng, target, draft, cfg = tiny
+    for plen in (1, 2, 3):
+        prompt = workloads.make_prompt(40 + plen, plen, cfg["vocab"])
+        for n_new in (1, 2, 5):
+            for gamma in (1, 8):
+                for temperature in (1.0, 0.0):
+                    got, _ = eng.generate([prompt], n_new, gamma, temperature, 3)
+                    ref = oracle_generate.speculative_generate(target, draft, prompt, n_new, gamma, temperature, 3)
+                    if list(got[0]) != list(ref.tokens[:n_new]):  # (a handful of decisions: none may sit on a boundary)
+                        raise AssertionError(f"prompt {plen}, {n_new} new, gamma {gamma}, T {temperature}: "
+                                             f"{list(got[0])} against {ref.tokens[:n_new]}")
+
+
 def test_target_only_sampling_matches_the_oracle(tiny):
     eng, target, _, cfg = tiny
     prompt = workloads.make_prompt(9, 5, cfg["vocab"])

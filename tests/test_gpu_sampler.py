@@ -61,6 +61,9 @@ def test_standalone_sampler_workload(noise):
     (9, 4, 32000, 0.0),      # greedy
     (6, 6, 1001, 0.0),
     (3, 64, 257, 1.0),       # maximum gamma
+    (6, 3, 32000, 0.05),     # cold: nearly one-hot rows, exponents scaled by 29
+    (6, 3, 32000, 8.0),      # hot: nearly flat rows
+    (5, 2, 50257, 0.1),      # cold, scalar loads
 ])
 def test_shapes_and_edges(batch, gamma, vocab, temperature):
     tl, ql = workloads.make_sampler_logits(batch * 1000 + gamma, batch, gamma, vocab, 1.0)
