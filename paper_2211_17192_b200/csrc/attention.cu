@@ -109,7 +109,6 @@ attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __r
                  const KV* __restrict__ kv_layer, const int32_t* __restrict__ page_table, int pages_per_seq,
                  int page_size, const int32_t* __restrict__ kv_len, const float* __restrict__ bias, int bias_span,
                  int bias_zero, float scale, float* __restrict__ part, const AttnOut out) {
-    constexpr int PER_LANE = DH / 32;
     __shared__ float share[kMaxAttnWarps][DH + 2];  // states of the warps that share a query (ks > 1)
     pdl_trigger();
     pdl_wait();
@@ -130,12 +129,14 @@ attention_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __r
 // With grouped query heads, several new rows per sequence and a batch of
 // sequences, the kernel above re-reads every K,V tile from L1 once per query.
 // Here the (up to 16) queries that share a KV head form the M side of
-// mma.sync.m16n8k8 (tf32, fp32 accumulate): a warp stages 16-key tiles of K and
-// of V in shared memory once (cp.async, two tiles in flight: the next one loads
-// while this one is multiplied), computes S = Q K^T for all queries, keeps the
-// online softmax in the accumulator layout (a row's maximum and sum live in a
-// quad of lanes), and accumulates O += P V.  The warps of a CTA take the 32-key
-// blocks of its key slice in turn and merge their states at the end; the partial state per (row, head, slice) has the same
+// mma.sync.m16n8k8 (tf32, fp32 accumulate): a warp stages a 16-key tile of K and
+// of V in shared memory once (cp.async for fp32 rows; 16-bit rows are converted
+// on the way in), computes S = Q K^T for all queries, keeps the online softmax in
+// the accumulator layout (a row's maximum and sum live in a quad of lanes), and
+// accumulates O += P V.  The warps of a CTA take the 16-key tiles of its key slice
+// in turn (a slice is short enough that a warp seldom sees a second tile, so one
+// staged tile per warp is kept: a second stage halves the CTAs per SM) and merge
+// their states at the end; the partial state per (row, head, slice) has the same
 // format as above, so attention_combine_kernel serves both.
 constexpr int kMmaWarps = 8;
 constexpr int kMmaStages = 1;  // staged tiles per warp (2: the next tile loads while this one is multiplied)
