@@ -115,3 +115,37 @@ def test_greedy_equivalence_on_the_other_benchmark_pairs(target, draft, prompt_l
         assert sum(hist) == stats["iterations"] and stats["tokens"] == sum((n + 1) * c for n, c in enumerate(hist))
     finally:
         eng.close()
+
+
+def test_greedy_equivalence_in_a_ragged_batch_of_sixteen():
+    """Config 5's batched corner at full size: 16 sequences with prompts of 1000 .. 1015 tokens, gamma = 4 (80-row
+    verification passes, the f16 attention kernel, ragged roll-back every iteration): every sequence's greedy
+    speculative stream is its greedy target-only stream."""
+    device = torch.device("cuda", 0)
+    tcfg, dcfg = workloads.model_config("llama7b_target"), workloads.model_config("llama160m_draft")
+    batch, gamma, new = 16, 4, 12
+    eng = binding.Engine(tcfg, bench.gpu_weights(tcfg, 1, device), dcfg, bench.gpu_weights(dcfg, 2, device), max_batch=batch,
+                         max_len=1016 + new + gamma + 2, page_size=64, max_gamma=gamma)
+    try:
+        assert eng.attention_plan(0, batch, gamma + 1)["f16"]
+        prompts = [workloads.make_prompt(60 + b, 1000 + b, tcfg["vocab"]) for b in range(batch)]
+        greedy, _ = eng.generate(prompts, new, 0, 0.0, 0)
+        spec, stats = eng.generate(prompts, new, gamma, 0.0, 0)
+        assert binding.spec_device_error() == 0
+        for b in range(batch):
+            differ = np.nonzero(greedy[b] != spec[b])[0]
+            if not differ.size:
+                continue
+            k = int(differ[0])  # only a tie within the tolerance may fall either way
+            seq = np.concatenate([prompts[b], greedy[b, :k]]).astype(np.int32)
+            eng.reset()
+            last = None
+            for at in range(0, len(seq), 64):
+                last = eng.forward_logits(0, seq[None, at:at + 64])
+            row = np.sort(last[0, -1].cpu().numpy())
+            assert row[-1] - row[-2] <= 2 * BF16_ABS, f"sequence {b} differs at token {k} with a top-2 gap of {row[-1] - row[-2]:.3g}"
+        hist = stats["accepted_histogram"][:gamma + 1]
+        assert stats["tokens"] == sum((n + 1) * c for n, c in enumerate(hist))  # over all sequences and iterations
+        assert stats["tests_passed"] == sum(n * c for n, c in enumerate(hist))
+    finally:
+        eng.close()
