@@ -139,7 +139,7 @@ struct Smem {
     static constexpr int kTotal = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
 };
 
-// grid = (tiles of 128 features, splits, token tiles), block = 128.
+// grid = (tiles of 128 features x token tiles, splits), block = 128.
 template <int N_TOK>
 __global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_hi,
@@ -158,7 +158,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_bar + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile = blockIdx.x, split = blockIdx.y, splits = gridDim.y, tok0 = blockIdx.z * N_TOK;
+    // (the token tiles of one weight tile are neighbours in launch order: they run side by side and the second
+    // finds the weights in L2 - with the token tile as the slowest grid dimension a 224-row launch read every
+    // weight from HBM twice)
+    const int token_tiles = (n_rows + N_TOK - 1) / N_TOK;
+    const int tile = blockIdx.x / token_tiles, split = blockIdx.y, splits = gridDim.y, tok0 = (blockIdx.x % token_tiles) * N_TOK;
     const int kb0 = static_cast<int>(static_cast<long long>(k_blocks) * split / splits);
     const int kb1 = static_cast<int>(static_cast<long long>(k_blocks) * (split + 1) / splits);
 
@@ -415,7 +419,7 @@ int launch_tc(const CUtensorMap& mw, const CUtensorMap& mhi, const CUtensorMap& 
     if (first_use_on_this_device(configured))
         SPEC_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<N_TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            Smem<N_TOK>::kTotal));
-    const dim3 grid((n_out + kTileM - 1) / kTileM, splits, (n_rows + N_TOK - 1) / N_TOK);
+    const dim3 grid(((n_out + kTileM - 1) / kTileM) * ((n_rows + N_TOK - 1) / N_TOK), splits, 1);
     return launch_pdl(gemm_tc_kernel<N_TOK>, grid, dim3(kThreads), Smem<N_TOK>::kTotal, stream, mw, mhi, mlo, partial,
                       n_out, n_rows, k_blocks, packed, drill);
 }
