@@ -230,6 +230,7 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     using S = MmaSmem<DH, IN_TURN>;
     extern __shared__ __align__(16) float smem_f[];
     __shared__ int q_pos[16], q_row[16], q_head[16];
+    __shared__ float merge_w[16][kMmaWarps], merge_m[16];
     pdl_trigger();
     pdl_wait();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -433,24 +434,32 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
         st[(g + 8) * (DH + 2) + 1] = l_hi;
     }
     __syncthreads();
+    // The weight exp(m_w - max) of every (query, warp) is formed once - thread 8 q + w takes warp w's state of
+    // query q, the maximum goes round its group of eight lanes - instead of once per element of the state.
+    if (tid < 16 * kMmaWarps) {
+        static_assert(kMmaWarps == 8, "the groups of eight lanes below are the warps of one query");
+        const int qi = tid / kMmaWarps, w = tid % kMmaWarps;
+        const float m_w = smem_f[S::kQ + w * S::kPerWarp + qi * (DH + 2)];
+        float mm = m_w;
+        mm = fmaxf(mm, __shfl_xor_sync(kFullMask, mm, 1));
+        mm = fmaxf(mm, __shfl_xor_sync(kFullMask, mm, 2));
+        mm = fmaxf(mm, __shfl_xor_sync(kFullMask, mm, 4));
+        merge_w[qi][w] = expf(m_w - mm);
+        if (w == 0) merge_m[qi] = mm;
+    }
+    __syncthreads();
     // merge the warps (in warp order) and write the slice's partial state of every live query
     // (fused: into the queries' buffer, which nobody needs any more, for the cluster merge)
     for (int i = tid; i < 16 * (DH + 2); i += 32 * kMmaWarps) {
         const int qi = i / (DH + 2), e = i % (DH + 2);
         if (mb * 16 + qi >= queries) continue;
-        float mm = -FLT_MAX;
-#pragma unroll
-        for (int w = 0; w < kMmaWarps; ++w) mm = fmaxf(mm, smem_f[S::kQ + w * S::kPerWarp + qi * (DH + 2)]);
         float merged;
         if (e == 0) {
-            merged = mm;
+            merged = merge_m[qi];
         } else {
             merged = 0.0f;
 #pragma unroll
-            for (int w = 0; w < kMmaWarps; ++w) {
-                const float* sw = smem_f + S::kQ + w * S::kPerWarp + qi * (DH + 2);
-                merged += sw[e] * expf(sw[0] - mm);
-            }
+            for (int w = 0; w < kMmaWarps; ++w) merged += smem_f[S::kQ + w * S::kPerWarp + qi * (DH + 2) + e] * merge_w[qi][w];
         }
         if (FUSED) Qs[i] = merged;
         else part[((static_cast<size_t>(q_row[qi]) * n_heads + q_head[qi]) * slices + slice) * (DH + 2) + e] = merged;
