@@ -132,7 +132,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 template <int N_TOK>
 struct Smem {
     // two CTAs per SM up to 128 rows; wider tiles fill the SM alone
-    static constexpr int kStages = N_TOK <= 16 ? 5 : N_TOK <= 32 ? 4 : N_TOK <= 64 ? 3 : N_TOK <= 128 ? 2 : 3;
+    static constexpr int kStages = N_TOK <= 16 ? 5 : N_TOK <= 32 ? 4 : N_TOK <= 80 ? 3 : N_TOK <= 128 ? 2 : 3;
     static constexpr int kABytes = kTileM * kTileK * 2;   // 16 KB
     static constexpr int kBBytes = N_TOK * kTileK * 2;     // one of hi / lo
     static constexpr int kStageBytes = kABytes + 2 * kBBytes;
@@ -426,19 +426,25 @@ int launch_tc(const CUtensorMap& mw, const CUtensorMap& mhi, const CUtensorMap& 
 
 }  // namespace
 
-// Rows per CTA (the MMA's N): the smallest tile that holds the rows, so that up to 192 rows
-// the weights are streamed once (the tensor-core work and the activation tiles that
-// every CTA re-reads grow with the padded row count); more rows take tiles of 128, two
-// CTAs per SM (measured: a 256-row tile leaves room for two pipeline stages only and
-// is slower than two passes of 128).
+// Rows per CTA (the MMA's N): the smallest multiple of 16 that holds the rows, so that up to 192 rows
+// the weights are streamed once and no MMA column is padding (the tensor-core work and the activation
+// tiles that every CTA re-reads grow with the padded row count: an 80-row tile for 80 rows instead of
+// a 96-row one took 8 % off the pass at batch 16 x 5 rows); more rows take several tiles, neighbours in
+// launch order (measured: a 256-row tile leaves room for two pipeline stages only and is slower than
+// two passes of 128).
 int gemm_tc_token_tile(int n_rows) {
     if (n_rows <= 16) return 16;
     if (n_rows <= 32) return 32;
     if (n_rows <= 48) return 48;
     if (n_rows <= 64) return 64;
+    if (n_rows <= 80) return 80;
     if (n_rows <= 96) return 96;
+    if (n_rows <= 112) return 112;
     if (n_rows <= 128) return 128;
+    if (n_rows <= 160) return 160;
     if (n_rows <= 192) return 192;
+    if (n_rows <= 240) return 80;  // three tiles of 80 (three stages each) beat two of 112 or 128: 274 / 302 / 313 us
+                                   // per 7B block at 224 rows
     return 128;
 }
 
@@ -512,8 +518,11 @@ int launch_gemm_tc_partials(const __nv_bfloat16* hi, const __nv_bfloat16* lo, in
         case 32: return launch_tc<32>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
         case 48: return launch_tc<48>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
         case 64: return launch_tc<64>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
+        case 80: return launch_tc<80>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
         case 96: return launch_tc<96>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
+        case 112: return launch_tc<112>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
         case 128: return launch_tc<128>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
+        case 160: return launch_tc<160>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
         default: return launch_tc<192>(mw, mhi, mlo, partial, n_out, n_rows, k_blocks, splits, pk, stream);
     }
 }
