@@ -473,8 +473,8 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 // ---- fp16 K,V rows on the f16 tensor-core path --------------------------------
 //
 // With 16-bit rows the cache needs no conversion: 64-key tiles of K and of V go
-// from the pool to shared memory as they are (cp.async, two stages: tile i + 1
-// loads while tile i is multiplied) and feed mma.sync.m16n8k16 (f16 operands,
+// from the pool to shared memory as they are (cp.async, a ring of two or three stages:
+// the next tiles load while tile i is multiplied) and feed mma.sync.m16n8k16 (f16 operands,
 // fp32 accumulate) through ldmatrix.  A CTA owns (key slice, KV head, sequence)
 // and ALL the queries of that KV head - up to 64, as MB blocks of 16 - so K and
 // V of the slice are fetched once, whatever the number of rows.  Its four warps
@@ -485,21 +485,28 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 // significant bits, one more than the tf32 path above keeps).
 constexpr int kF16Warps = 4;
 constexpr int kF16TileKeys = 64;
-constexpr int kF16Stages = 2;
 constexpr int kF16MaxQueries = 64;  // per CTA (MB = 4)
 
+// Rows are stored without padding; inside a row the 16-byte chunks are permuted, chunk c of row r at position
+// c ^ (r & 7), so that the eight rows an ldmatrix reads hit eight different bank groups.  Three stages (tiles
+// i + 1 and i + 2 on their way while tile i is multiplied) for up to 32 queries, two for 64: two CTAs per SM
+// either way, and 128 KB of K,V in flight per SM instead of 64 - the kernel is bound by the latency of the tiles.
 template <int DH, int MB>
 struct F16Smem {
-    static constexpr int kRow = DH + 8;                  // halves per staged row: consecutive rows are 16 bytes apart
-                                                         // modulo 128, so ldmatrix sees no bank conflict
+    static constexpr int kStages = MB <= 2 ? 3 : 2;
+    static constexpr int kRow = DH;                      // halves per staged row
     static constexpr int kQ = 16 * MB * kRow;            // the queries (halves)
     static constexpr int kTile = kF16TileKeys * kRow;    // one K or V tile (halves)
     static constexpr int kStage = 2 * kTile;             // K, then V
-    static constexpr size_t kBytes = static_cast<size_t>(kQ + kF16Stages * kStage) * sizeof(__half);
-    // the epilogue reuses the stages: four warps' states in stage 0, the merged states in stage 1
-    static_assert(kF16Warps * 16 * (DH + 2) * sizeof(float) <= kStage * sizeof(__half), "states must fit a stage");
-    static_assert(16 * MB * (DH + 2) * sizeof(float) <= kStage * sizeof(__half), "merged states must fit a stage");
+    static constexpr size_t kBytes = static_cast<size_t>(kQ + kStages * kStage) * sizeof(__half);
+    // the epilogue reuses the stages: four warps' states first, the merged states behind them (in place when a
+    // query block has a single key part, MB = 4: there is nothing to merge then)
+    static_assert((kF16Warps * 16 + (MB == kF16Warps ? 0 : 16 * MB)) * (DH + 2) * sizeof(float) <= kStages * kStage * sizeof(__half),
+                  "states and merged states must fit the stages");
 };
+// Offset (in halves) of element `col` (a multiple of 8) of row `row` in a staged tile or in the staged queries.
+template <int DH>
+__device__ __forceinline__ int f16_at(int row, int col) { return row * DH + ((((col >> 3) ^ row) & 7) << 3) + (col & ~63); }
 
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const __half* p) {
     const uint32_t a = static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -591,7 +598,7 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     // keys at or beyond seq_keys become zeros.
     const int copy_row = tid / CH, copy_off = copy_row * DH + 8 * (tid % CH);
     const uint32_t copy_dst = static_cast<uint32_t>(__cvta_generic_to_shared(stages)) +
-                              static_cast<uint32_t>((copy_row * S::kRow + 8 * (tid % CH)) * sizeof(__half));
+                              static_cast<uint32_t>(f16_at<DH>(copy_row, 8 * (tid % CH)) * sizeof(__half));
     // (the page entries of a tile are fetched one tile ahead of the copies that need them, so that no
     // copy waits for a page-table load)
     auto fetch_pages = [&](int i, int (&pg)[2]) {
@@ -604,7 +611,7 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     auto issue = [&](int i, const int (&pg)[2]) {
         if (i < my_tiles) {
             const int k0 = kF16TileKeys * (t0 + i);
-            const uint32_t dst = copy_dst + static_cast<uint32_t>((i % kF16Stages) * S::kStage * sizeof(__half));
+            const uint32_t dst = copy_dst + static_cast<uint32_t>((i % S::kStages) * S::kStage * sizeof(__half));
             const __half* half_base[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h)
@@ -624,16 +631,19 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
         }
         cp_async_commit();
     };
-    int pg_now[2] = {0, 0}, pg_next[2] = {0, 0};
-    fetch_pages(0, pg_now);
-    fetch_pages(1, pg_next);
-    issue(0, pg_now);  // (requested before the queries are staged)
+    int pg_next[2] = {0, 0};
+#pragma unroll
+    for (int t = 0; t < S::kStages - 1; ++t) {  // the first tiles are requested before the queries are staged
+        fetch_pages(t, pg_next);
+        issue(t, pg_next);
+    }
+    fetch_pages(S::kStages - 1, pg_next);
     __syncthreads();  // (the queries' positions)
     const float q_scale = scale * kLog2e;
     for (int i = tid; i < QN * DH; i += 32 * kF16Warps) {
         const int qi = i / DH, e = i % DH;
         const float v = q_pos[qi] >= 0 ? qkv[static_cast<size_t>(q_row[qi]) * q_stride + q_head[qi] * DH + e] * q_scale : 0.0f;
-        Qs[qi * S::kRow + e] = __float2half_rn(v);
+        Qs[f16_at<DH>(qi, e & ~7) + (e & 7)] = __float2half_rn(v);
     }
 
     // the two query rows of this lane: g and g + 8 of query block mb.  A row beyond the live queries sees
@@ -655,18 +665,18 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     const int any_sees = min(__reduce_max_sync(kFullMask, max(p_lo < 0 ? 0 : keys_lo, p_hi < 0 ? 0 : keys_hi)), seq_keys);
 
     for (int i = 0; i < my_tiles; ++i) {
-        cp_async_wait<0>();
-        __syncthreads();  // tile i has landed for every thread; everybody is done with tile i - 1
-        issue(i + 1, pg_next);
-        fetch_pages(i + 2, pg_next);
+        cp_async_wait<S::kStages - 2>();  // tile i has landed (the later ones may still be on their way)
+        __syncthreads();                  // ... for every thread; everybody is done with tile i - 1, whose stage
+        issue(i + S::kStages - 1, pg_next);  // takes the tile that is kStages - 1 ahead
+        fetch_pages(i + S::kStages, pg_next);
         if (i == 0) {  // (the first barrier also covered the staged queries)
 #pragma unroll
             for (int ks = 0; ks < DH / 16; ++ks)
-                ldsm_x4(qf[ks], Qs + (mb * 16 + (lane & 7) + 8 * ((lane >> 3) & 1)) * S::kRow + ks * 16 + 8 * (lane >> 4));
+                ldsm_x4(qf[ks], Qs + f16_at<DH>(mb * 16 + (lane & 7) + 8 * ((lane >> 3) & 1), ks * 16 + 8 * (lane >> 4)));
         }
         const int k0 = kF16TileKeys * (t0 + i) + kw0;  // this warp's first key of the tile
         if (k0 >= any_sees) continue;  // nothing here that a live row of this warp may see
-        const __half* Kt = stages + (i % kF16Stages) * S::kStage + kw0 * S::kRow;
+        const __half* Kt = stages + (i % S::kStages) * S::kStage + kw0 * S::kRow;  // (kw0 is a multiple of 16: the permutation is unchanged)
         const __half* Vt = Kt + S::kTile;
         // S = Q K^T
         float s[NB][4];
@@ -679,7 +689,7 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb) {
                 uint32_t kf[4];
-                ldsm_x4(kf, Kt + (nb * 8 + (lane & 7)) * S::kRow + kp * 32 + 8 * (lane >> 3));
+                ldsm_x4(kf, Kt + f16_at<DH>(nb * 8 + (lane & 7), kp * 32 + 8 * (lane >> 3)));
                 mma_f16(s[nb], qf[2 * kp], kf[0], kf[1]);
                 mma_f16(s[nb], qf[2 * kp + 1], kf[2], kf[3]);
             }
@@ -752,7 +762,7 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 #pragma unroll
             for (int kk = 0; kk < NB / 2; ++kk) {
                 uint32_t vf[4];
-                ldsm_x4_trans(vf, Vt + (kk * 16 + (lane & 7) + 8 * ((lane >> 3) & 1)) * S::kRow + n2 * 16 + 8 * (lane >> 4));
+                ldsm_x4_trans(vf, Vt + f16_at<DH>(kk * 16 + (lane & 7) + 8 * ((lane >> 3) & 1), n2 * 16 + 8 * (lane >> 4)));
                 mma_f16(o[2 * n2], pa[kk], vf[0], vf[1]);
                 mma_f16(o[2 * n2 + 1], pa[kk], vf[2], vf[3]);
             }
@@ -763,7 +773,8 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     // park this warp's state in stage 0: [warp][query of the block][max (base-2 units), sum, O[DH]]
     __syncthreads();
     float* states = reinterpret_cast<float*>(stages);
-    float* merged_buf = reinterpret_cast<float*>(stages + S::kStage);
+    // (one key part per query block: every weight below is 1 and the merged state is the state, in place)
+    float* merged_buf = KP == 1 ? states : states + kF16Warps * 16 * (DH + 2);
     {
         float* st = states + warp * 16 * (DH + 2);
 #pragma unroll
