@@ -660,6 +660,14 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 #pragma unroll
         for (int i = 0; i < 4; ++i) o[n][i] = 0.0f;
     uint32_t qf[DH / 16][4];
+    // lane-dependent parts of the ldmatrix addresses, formed once (the chunk permutation XORs with lane & 7):
+    // K: row (nb*8 + l7), chunk kp*4 + (lane >> 3); V: row (kk*16 + l7 + 8*((lane >> 3) & 1)), chunk n2*2 + (lane >> 4)
+    const int l7 = lane & 7;
+    const int k_lane = l7 * DH + ((((lane >> 3) ^ l7) & 7) << 3);            // even kp; odd kp flips chunk bit 2
+    const int v_row = (l7 + 8 * ((lane >> 3) & 1)) * DH;
+    int v_chunk[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v_chunk[j] = ((((j << 1) | (lane >> 4)) ^ l7) & 7) << 3;
     // keys that every row of this warp sees (no mask needed below it), and that any live row sees
     const int all_see = min(__reduce_min_sync(kFullMask, min(keys_lo, keys_hi)), seq_keys);
     const int any_sees = min(__reduce_max_sync(kFullMask, max(p_lo < 0 ? 0 : keys_lo, p_hi < 0 ? 0 : keys_hi)), seq_keys);
@@ -689,7 +697,7 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb) {
                 uint32_t kf[4];
-                ldsm_x4(kf, Kt + f16_at<DH>(nb * 8 + (lane & 7), kp * 32 + 8 * (lane >> 3)));
+                ldsm_x4(kf, Kt + nb * 8 * DH + (kp >> 1) * 64 + ((kp & 1) ? (k_lane ^ 32) : k_lane));
                 mma_f16(s[nb], qf[2 * kp], kf[0], kf[1]);
                 mma_f16(s[nb], qf[2 * kp + 1], kf[2], kf[3]);
             }
@@ -762,7 +770,7 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 #pragma unroll
             for (int kk = 0; kk < NB / 2; ++kk) {
                 uint32_t vf[4];
-                ldsm_x4_trans(vf, Vt + f16_at<DH>(kk * 16 + (lane & 7) + 8 * ((lane >> 3) & 1), n2 * 16 + 8 * (lane >> 4)));
+                ldsm_x4_trans(vf, Vt + kk * 16 * DH + v_row + (n2 >> 2) * 64 + v_chunk[n2 & 3]);
                 mma_f16(o[2 * n2], pa[kk], vf[0], vf[1]);
                 mma_f16(o[2 * n2 + 1], pa[kk], vf[2], vf[3]);
             }
