@@ -124,6 +124,45 @@ def test_bf16_llama_pair_matches_the_oracle():
     eng.close()
 
 
+@pytest.mark.parametrize("prompt_len", [200, 257, 300, 470])
+def test_long_prompts_through_the_prompt_pass(prompt_len):
+    """Prompts longer than one chunk of the prompt pass (256 rows per chunk: 200 rows in one chunk of three
+    80-row token tiles, 256 + 1, 256 + 44, 256 + 214), several pages and key tiles, then free-running
+    generation against the oracle, sampled and greedy: a wrong row anywhere in the cached prompt changes the
+    stream."""
+    tcfg, tw, dcfg, dw = _models("llama_test_target", "llama_test_draft")
+    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=1, max_len=512, page_size=32, max_gamma=3)
+    prompt = workloads.make_prompt(50 + prompt_len, prompt_len, tcfg["vocab"])
+    try:
+        for temperature in (1.0, 0.0):
+            flagged, iters = compare_generation(eng, Decoder(tcfg, tw), Decoder(dcfg, dw), prompt, 24, 3, temperature,
+                                                seed=6, margin=5e-3, logit_tol=5e-3)
+            assert flagged <= 3, f"{flagged} flagged of {iters}"
+    finally:
+        eng.close()
+
+
+def test_ragged_long_prompts_in_one_batch():
+    """Three sequences with prompts of 300, 130 and 77 tokens decoded together: the prompt pass cuts each into its
+    own chunks; every sequence's greedy stream equals the one it gives alone, and the first equals the oracle's."""
+    tcfg, tw, dcfg, dw = _models("llama_test_target", "llama_test_draft")
+    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=3, max_len=512, page_size=32, max_gamma=3)
+    try:
+        prompts = [workloads.make_prompt(70 + b, n, tcfg["vocab"]) for b, n in enumerate([300, 130, 77])]
+        together, _ = eng.generate(prompts, 20, 3, 0.0, 0)
+        for b in range(3):
+            alone, _ = eng.generate([prompts[b]], 20, 3, 0.0, 0)
+            assert np.array_equal(alone[0], together[b]), f"sequence {b}"
+        ref, rows, _ = oracle_generate.target_only_generate(Decoder(tcfg, tw), prompts[0], 20, 0.0, 0, keep_logits=True)
+        for k in range(20):
+            if together[0, k] != ref[k]:
+                gap = np.sort(rows[k])[-1] - np.sort(rows[k])[-2]
+                assert gap < 2e-2 and k >= MIN_COMPARED, f"token {k}: top-2 gap {gap:.3g}"
+                break
+    finally:
+        eng.close()
+
+
 def test_statistics_are_consistent(tiny):
     eng, _, _, cfg = tiny
     prompt = workloads.make_prompt(4, 12, cfg["vocab"])
