@@ -163,6 +163,46 @@ def test_ragged_long_prompts_in_one_batch():
         eng.close()
 
 
+def test_batch_of_sixteen_on_the_f16_attention_path_matches_the_oracle():
+    """16 ragged sequences of the bf16 Llama-shaped test pair decoded together (32 (sequence, KV head) pairs: the
+    verification passes take the f16 tensor-core attention, with a ragged roll-back every iteration): at T = 0 every
+    sequence's stream is the oracle's greedy stream of the target, up to a tie within the logit tolerance."""
+    tcfg, tw, dcfg, dw = _models("llama_test_target", "llama_test_draft")
+    batch, gamma, new = 16, 3, 16
+    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=batch, max_len=512, page_size=32, max_gamma=gamma)
+    try:
+        assert eng.attention_plan(0, batch, gamma + 1)["f16"]
+        prompts = [workloads.make_prompt(90 + b, 20 + 2 * b, tcfg["vocab"]) for b in range(batch)]
+        got, stats = eng.generate(prompts, new, gamma, 0.0, 0)
+        target = Decoder(tcfg, tw)
+        compared = 0
+        for b in range(batch):
+            ref, rows, _ = oracle_generate.target_only_generate(target, prompts[b], new, 0.0, 0, keep_logits=True)
+            for k in range(new):
+                if got[b, k] != ref[k]:
+                    gap = np.sort(rows[k])[-1] - np.sort(rows[k])[-2]
+                    assert gap < 2e-2, f"sequence {b}, token {k}: top-2 gap {gap:.3g}"
+                    break
+                compared += 1
+        assert compared >= batch * new * 3 // 4, f"only {compared} of {batch * new} tokens were compared before ties"
+        # sampled: accepted guesses and rejections mix, so the roll-back is ragged; each sequence against its own oracle run
+        out, stats = eng.generate(prompts, new, gamma, 1.0, 23)
+        draft = Decoder(dcfg, dw)
+        compared = 0
+        for b in range(batch):
+            ref = oracle_generate.speculative_generate(target, draft, prompts[b], new, gamma, 1.0, 23, sequence=b)
+            diff = next((k for k in range(new) if out[b, k] != ref.tokens[k]), None)
+            if diff is not None:
+                index = len(prompts[b]) + diff
+                it = next(i for i in ref.iterations if i.start_len <= index <= i.start_len + i.n_accepted)
+                assert min([it.accept_margin, it.cdf_margin] + list(it.draft_cdf_margins)) < 5e-3, f"sequence {b}, token {diff}"
+            compared += new if diff is None else diff
+        assert compared >= batch * new // 2, f"only {compared} of {batch * new} tokens were compared before flagged decisions"
+        assert 0 < stats["tests_passed"] < stats["tests_evaluated"]
+    finally:
+        eng.close()
+
+
 def test_statistics_are_consistent(tiny):
     eng, _, _, cfg = tiny
     prompt = workloads.make_prompt(4, 12, cfg["vocab"])
