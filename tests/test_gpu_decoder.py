@@ -37,6 +37,7 @@ def _pair(name, seed=1, **overrides):
     ("gpt97m_target", {}),
     ("gpt6m_draft", {}),                                   # tied embeddings
     ("llama160m_draft", {"n_layers": 2, "vocab": 4096}),   # d_head 64 rotary, wide FFN
+    ("llama160m_draft", {}),                               # the benchmark's draft at full size (12 blocks, vocabulary 32000)
     ("llama7b_target", {"n_layers": 1, "vocab": 4096, "d_ff": 1024}),  # d_head 128, 32 query / 8 KV heads
 ])
 def test_teacher_forced_logits_with_rollback(name, overrides):

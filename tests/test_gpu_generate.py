@@ -203,6 +203,22 @@ def test_batch_of_sixteen_on_the_f16_attention_path_matches_the_oracle():
         eng.close()
 
 
+def test_gpt_97m_and_6m_pair_at_full_size_matches_the_oracle():
+    """The GPT-like pair of the paper's Section 4.2 shapes at full size (97M-parameter target, 6M-parameter draft with
+    tied embeddings, bf16), as the benchmark runs it: 128-token prompt, gamma = 5.  The oracle is fast enough here to
+    follow the free-running stream."""
+    tcfg, tw, dcfg, dw = _models("gpt97m_target", "gpt6m_draft")
+    eng = binding.Engine(tcfg, tw, dcfg, dw, max_batch=1, max_len=128 + 64, page_size=64, max_gamma=5)
+    prompt = workloads.make_prompt(77, 128, tcfg["vocab"])
+    try:
+        for temperature in (1.0, 0.0):
+            flagged, iters = compare_generation(eng, Decoder(tcfg, tw), Decoder(dcfg, dw), prompt, 32, 5, temperature,
+                                                seed=8, margin=5e-3, logit_tol=5e-3)
+            assert flagged <= 3, f"{flagged} flagged of {iters}"
+    finally:
+        eng.close()
+
+
 def test_statistics_are_consistent(tiny):
     eng, _, _, cfg = tiny
     prompt = workloads.make_prompt(4, 12, cfg["vocab"])
