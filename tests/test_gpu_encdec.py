@@ -74,6 +74,18 @@ def test_teacher_forced_logits_bf16():
         eng.close()
 
 
+def test_teacher_forced_logits_of_the_t5_small_shape_at_full_size():
+    """The benchmark's draft for the encoder-decoder pair at full size (6 + 6 blocks, d 512, 8 heads, vocabulary
+    32128), here as the only model of a context: sources of 96 and 40 tokens."""
+    cfg = workloads.model_config("t5small_draft")
+    w = workloads.make_weights(cfg, 6)
+    eng = binding.Engine(cfg, w, max_batch=2, max_len=64, page_size=32, max_gamma=3, max_src_len=96)
+    try:
+        _teacher_forced(eng, ((cfg, w),), [96, 40], 2e-2, False)
+    finally:
+        eng.close()
+
+
 def _first_difference(got, want):
     return next((k for k in range(len(want)) if got[k] != want[k]), None)
 
