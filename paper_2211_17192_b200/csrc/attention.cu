@@ -890,23 +890,28 @@ int attention_sub_slices(int queries) {
 // The tensor-core kernel serves bf16 models (its tf32 products stay far inside
 // their 2e-2 logit bar, not inside the 1e-4 bar of fp32 models) once a KV head
 // has enough queries to fill a good part of a 16-row block.
+constexpr int kF16MinPairs = 16;  // (sequence, KV head) pairs from which fp16 K,V rows take the f16 kernel
+
 bool attention_uses_mma(const Model& m, int batch, int m_rows, int max_keys) {
     const int queries = (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows;
     // With fewer than 5 queries per KV head, or little work in all (query-key pairs over the
     // whole launch), the warp-per-query kernel wins: its CTAs are lighter to launch.
     const long long pairs = static_cast<long long>(batch) * m.cfg.n_kv_heads * queries * max_keys;
-    // (four queries pay only on a large batch, where its CTAs share the SMs two by two: from 128 (sequence, KV head)
-    // pairs on - measured on the 7B shape, batch 16: 4.16 -> 4.05 ms per pass, batch 8: 3.46 -> 3.48)
-    const int min_queries = batch * m.cfg.n_kv_heads >= 128 ? 4 : 5;
+    // (four queries - a one-row pass of a model with four query heads per KV head - pay where the CTAs share the SMs:
+    // with fp16 K,V rows, i.e. the f16 kernel, from 16 (sequence, KV head) pairs on - measured on the 7B shape, one row,
+    // per block, against the warp-per-query kernel: 4 sequences 95 vs 104 us, 8 sequences 101 vs 120, at 1788 cached
+    // tokens 105 vs 138; with fp32 rows from 128 pairs on: batch 16 4.16 -> 4.05 ms per pass, batch 8 3.46 -> 3.48)
+    const int min_queries = batch * m.cfg.n_kv_heads >= (m.kv_dtype == SPEC_DTYPE_FP16 ? kF16MinPairs : 128) ? 4 : 5;
     return m.bf16() && queries >= min_queries && pairs >= 65536;
 }
 
-// fp16 K,V rows take the f16 tensor-core kernel where the tf32 one would run, from 32 (sequence, KV head)
+// fp16 K,V rows take the f16 tensor-core kernel where the tf32 one would run, from 16 (sequence, KV head)
 // pairs on: measured on the 7B shape with 1024 cached tokens, per block, against the tf32 kernel converting
-// the same rows: batch 4 x 3 rows 104 vs 110 us, 8 x 3 113 vs 135, 16 x 5 165 vs 227, 32 x 7 317 vs 452,
-// 32 x 1 141 vs 185; at batch 1 (8 pairs) its 64-key tiles leave too few CTAs and it loses 1 - 4 us per block.
+// the same rows: batch 2 x 3 rows 97.0 vs 97.8 us, 2 x 7 105 vs 108, 3 x 3 99 vs 117, 3 x 7 113 vs 136,
+// 4 x 3 104 vs 110, 8 x 3 113 vs 135, 16 x 5 165 vs 227, 32 x 7 317 vs 452, 32 x 1 141 vs 185; at batch 1
+// (8 pairs) its 64-key tiles leave too few CTAs and it loses up to 3 us per block (7 rows: 100 vs 97).
 bool attention_uses_f16(const Model& m, int batch, int m_rows, int max_keys) {
-    return m.kv_dtype == SPEC_DTYPE_FP16 && batch * m.cfg.n_kv_heads >= 32 && attention_uses_mma(m, batch, m_rows, max_keys);
+    return m.kv_dtype == SPEC_DTYPE_FP16 && batch * m.cfg.n_kv_heads >= kF16MinPairs && attention_uses_mma(m, batch, m_rows, max_keys);
 }
 
 // The key slices can be merged inside a cluster (no second kernel) whenever a CTA
@@ -929,7 +934,12 @@ int attention_slices(const Model& m, int batch, int m_rows, int max_len) {
         const int resident = 148 * (m.cfg.d_head == 64 ? 4 : 2);
         const int want = std::max(1, resident / groups);
         const int most = std::max(1, (max_len + kF16TileKeys - 1) / kF16TileKeys);
-        return std::max(1, std::min(std::min(want, most), cap));
+        int slices = std::max(1, std::min(std::min(want, most), cap));
+        // clusters are placed a cluster at a time: past 128 SMs' worth of CTAs a launch waits for room (7B shape, one
+        // row, per block: 12 sequences 3 slices x 96 heads 119 us, 2 x 96 106; 6 sequences 6 x 48 109, 5 x 48 99)
+        const int room = 128 * (m.cfg.d_head == 64 ? 4 : 2);
+        if (slices <= kMaxClusterSlices && groups * slices > room) slices = std::max(1, room / groups);
+        return slices;
     }
     if (attention_uses_mma(m, batch, m_rows, max_len)) {
         // one wave of CTAs (shared memory allows one per SM at d_head 128, two at 64; twice that from 64
@@ -947,9 +957,22 @@ int attention_slices(const Model& m, int batch, int m_rows, int max_len) {
     // SM takes 16 warps of it; one wave of CTAs beats more, thinner slices
     const int warps = std::min(kMaxAttnWarps, std::max(1, queries * ks));
     const int resident = 148 * std::max(1, 16 / warps);
-    const int want = std::max(1, resident / (batch * n_kv_heads));
-    const int most = std::max(1, (tiles + ks - 1) / ks);
-    return std::max(1, std::min(std::min(want, most), cap));
+    const int groups = batch * n_kv_heads;
+    const int want = std::max(1, resident / groups);
+    int most = std::max(1, (tiles + ks - 1) / ks);
+    // A lone query per KV head (a draft model's serial step): a tile per warp would leave the K,V rows of a
+    // head to a few SMs, whose ingest then bounds the kernel; a full cluster of thinner slices spreads them
+    // (measured per block of the 160M-shaped draft, 1024 cached tokens: 3 slices 30.3 us, 8 slices 29.4;
+    // 1788 tokens: 31.5 -> 31.0; more than a cluster merges, with the combine kernel: 29.6 - 29.8).
+    if (queries == 1) most = std::max(1, std::min(kMaxClusterSlices, (tiles + 3) / 4));
+    int slices = std::max(1, std::min(std::min(want, most), cap));
+    // Clusters of these SM-filling CTAs are placed a cluster at a time, beside the neighbouring kernels that overlap
+    // them: beyond 128 CTAs a launch waits for room (draft, 4 sequences: 3 slices x 48 heads 42.4 us per block,
+    // 2 x 48 35.6; 2 sequences: 6 x 24 39.7, 5 x 24 32.3).  Launches without clusters do not mind.
+    if (warps == kMaxAttnWarps && slices <= kMaxClusterSlices && attention_merges_in_cluster(m, batch, m_rows, max_len) &&
+        groups * slices > 128)
+        slices = std::max(1, 128 / groups);
+    return slices;
 }
 
 size_t attention_partial_elems(int rows, int n_heads, int d_head, int slices) {
