@@ -757,9 +757,14 @@ sample_kernel(const float* __restrict__ logits, size_t logit_stride, const float
 //      repeats (heavy ties end when lo == hi).
 // The bin of a logit is a monotone function of it, so the bins partition the row
 // by value and the result is exact (comparisons of the logits themselves decide;
-// -inf, +inf and NaN logits are never in play).  Mass is summed in 2^-40 fixed
-// point with integer atomics, so every order of summation gives the same totals:
-// a row always gives the same floor, however the threads interleave.
+// -inf, +inf and NaN logits are never in play).  Mass is summed in fixed point
+// (units of 2^-32 of the largest weight) with integer atomics, so every order of
+// summation gives the same totals: a row always gives the same floor, however the
+// threads interleave.  The kernel is bound by instruction issue, not by memory
+// (the passes after the first hit L2), so the per-logit work is kept short: no
+// float-to-int conversion for the bin, one 32-bit atomic plus a rare carry for
+// the mass (a 64-bit shared-memory atomic cost 48 us of 180 on 960 rows of 32000),
+// a two-instruction test before a logit is asked whether it is in the chosen bin.
 constexpr int kSelThreads = 256;
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kSelBins = 2048;
@@ -821,8 +826,9 @@ __device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned 
     unsigned n = 0;
     for_each_logit(r, groups, [&](float v) {
         const bool in_play = fabsf(v) < INFINITY && v >= kf;
-        lo = fminf(lo, in_play ? v : INFINITY);
-        hi = fmaxf(hi, in_play ? v : -INFINITY);
+        const float u = in_play ? v : __int_as_float(0x7fc00000);  // (fminf and fmaxf pass over a NaN operand)
+        lo = fminf(lo, u);
+        hi = fmaxf(hi, u);
         n += in_play;
     });
     lo = warp_min(lo);
@@ -835,18 +841,22 @@ __device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned 
 #pragma unroll
     for (int w = 0; w < kSelWarps; ++w) { lo = fminf(lo, sh.warp_lo[w]); hi = fmaxf(hi, sh.warp_hi[w]); n += sh.warp_cnt[w]; }
     if (n == 0 || (!MASS && k > n)) return kf;  // nothing to cut
-    const float row_max = hi;
-    auto fixed_mass = [&](float v) { return __float2ull_rz(fast_exp2((v - row_max) * c2) * 1099511627776.0f); };  // 2^40
+    // weight exp2((l - max) * c2) of a logit in units of 2^-32 (the largest float below 2^32, so that the row's
+    // maximum still fits 32 bits): a bin's mass is then one 32-bit shared-memory atomic and, rarely, a carry
+    const float mc = fminf(-hi * c2, FLT_MAX);
+    auto fixed_mass = [&](float v) { return __float2uint_rz(fast_exp2(fmaf(v, c2, mc)) * 4294967040.0f); };
 
     unsigned before_cnt = 0;
     unsigned long long before_mass = 0, goal = 0;
     for (int level = 0; level < kSelLevels; ++level) {
         if (lo == hi) return hi;  // everything left is one value: it stays whole
         const float top = hi, bottom = lo;
-        const float scale = fminf(static_cast<float>(kSelBins) / (top - bottom), FLT_MAX);
-        // bin of a logit in [bottom, top], counted from the top; anything else gets no bin
+        // (top - v) * scale stays below kSelBins for every v >= bottom: the quarter bin absorbs the roundings
+        const float scale = fminf((static_cast<float>(kSelBins) - 0.25f) / (top - bottom), FLT_MAX);
+        // bin of a logit in [bottom, top], counted from the top; anything else gets no bin.  The floor is taken by
+        // adding 2^23 with rounding toward zero (the sum's last bit is then worth one) instead of a conversion.
         auto bin_of = [&](float v) {
-            const int b = min(kSelBins - 1, static_cast<int>((top - v) * scale));
+            const int b = __float_as_int(__fmaf_rz(top - v, scale, 8388608.0f)) & 0x7fffff;
             return (v >= bottom && v <= top) ? b : -1;
         };
         // 2. counts (and masses) per bin
@@ -857,7 +867,12 @@ __device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned 
             const int b = bin_of(v);
             if (b >= 0) {
                 atomicAdd(&sh.cnt[b], 1u);
-                if (MASS) atomicAdd(&sh.mass[b], fixed_mass(v));
+                if (MASS) {
+                    unsigned* word = reinterpret_cast<unsigned*>(&sh.mass[b]);  // (low word first)
+                    const unsigned m = fixed_mass(v);
+                    const unsigned was = atomicAdd(word, m);
+                    if (was + m < was) atomicAdd(word + 1, 1u);
+                }
             }
         });
         __syncthreads();
@@ -909,10 +924,15 @@ __device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned 
         before_cnt = sh.before_cnt;
         before_mass = sh.before_mass;
         const unsigned in_bin = sh.cnt[bin];
+        // a cheap test that no logit of the bin fails (its centre, half its width and the roundings of bin_of, with
+        // room to spare); the few that pass are then asked for their bin
+        const float centre = top - (static_cast<float>(bin) + 0.5f) / scale;
+        const float reach = 0.51f / scale + 2e-6f * fmaxf(fabsf(top), fabsf(bottom));
+        auto in_the_bin = [&](float v) { return fabsf(v - centre) <= reach && bin_of(v) == bin; };
         if (in_bin <= kSelCap) {
             // 3. copy the bin's logits out and rank them against each other
             for_each_logit(r, groups, [&](float v) {
-                if (bin_of(v) == bin) {
+                if (in_the_bin(v)) {
                     const unsigned at = atomicAdd(&sh.n_cand, 1u);
                     if (at < kSelCap) { sh.cand[at] = v; if (MASS) sh.cand_mass[at] = fixed_mass(v); }
                 }
@@ -940,7 +960,7 @@ __device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned 
         // the bin is crowded: its own range is searched next
         float new_lo = INFINITY, new_hi = -INFINITY;
         for_each_logit(r, groups, [&](float v) {
-            const bool here = bin_of(v) == bin;
+            const bool here = in_the_bin(v);
             new_lo = fminf(new_lo, here ? v : INFINITY);
             new_hi = fmaxf(new_hi, here ? v : -INFINITY);
         });
