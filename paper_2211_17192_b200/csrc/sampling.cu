@@ -774,7 +774,7 @@ constexpr int kSelLevels = 40;  // every level shrinks the range; fp32 allows fa
 
 struct SelShared {
     unsigned cnt[kSelBins];
-    unsigned long long mass[kSelBins];
+    unsigned mass_lo[kSelBins], mass_hi[kSelBins];  // a bin's mass, low and high word (apart: the low words then spread over all banks)
     float cand[kSelCap];
     unsigned long long cand_mass[kSelCap];
     unsigned long long warp_mass[kSelWarps];
@@ -860,18 +860,20 @@ __device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned 
             return (v >= bottom && v <= top) ? b : -1;
         };
         // 2. counts (and masses) per bin
-        for (int i = tid; i < kSelBins; i += kSelThreads) { sh.cnt[i] = 0; if (MASS) sh.mass[i] = 0; }
+        for (int i = tid; i < kSelBins; i += kSelThreads) {
+            if (MASS) { sh.mass_lo[i] = 0; sh.mass_hi[i] = 0; } else { sh.cnt[i] = 0; }
+        }
         if (tid == 0) { sh.n_cand = 0; sh.bin = kSelBins - 1; sh.before_cnt = before_cnt; sh.before_mass = before_mass; }
         __syncthreads();
         for_each_logit(r, groups, [&](float v) {
             const int b = bin_of(v);
             if (b >= 0) {
-                atomicAdd(&sh.cnt[b], 1u);
                 if (MASS) {
-                    unsigned* word = reinterpret_cast<unsigned*>(&sh.mass[b]);  // (low word first)
                     const unsigned m = fixed_mass(v);
-                    const unsigned was = atomicAdd(word, m);
-                    if (was + m < was) atomicAdd(word + 1, 1u);
+                    const unsigned was = atomicAdd(&sh.mass_lo[b], m);
+                    if (was + m < was) atomicAdd(&sh.mass_hi[b], 1u);
+                } else {
+                    atomicAdd(&sh.cnt[b], 1u);
                 }
             }
         });
@@ -881,8 +883,9 @@ __device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned 
         unsigned long long my_mass = 0;
 #pragma unroll
         for (int i = 0; i < kSelPerThread; ++i) {
-            my_cnt += sh.cnt[tid * kSelPerThread + i];
-            if (MASS) my_mass += sh.mass[tid * kSelPerThread + i];
+            const int b = tid * kSelPerThread + i;
+            if (MASS) my_mass += (static_cast<unsigned long long>(sh.mass_hi[b]) << 32) | sh.mass_lo[b];
+            else my_cnt += sh.cnt[b];
         }
         unsigned inc_cnt = my_cnt;
         unsigned long long inc_mass = my_mass;
@@ -910,8 +913,8 @@ __device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned 
 #pragma unroll
             for (int i = 0; i < kSelPerThread; ++i) {
                 const int b = tid * kSelPerThread + i;
-                const unsigned c = sh.cnt[b];
-                const unsigned long long m = MASS ? sh.mass[b] : 0ull;
+                const unsigned c = MASS ? 0u : sh.cnt[b];
+                const unsigned long long m = MASS ? (static_cast<unsigned long long>(sh.mass_hi[b]) << 32) | sh.mass_lo[b] : 0ull;
                 const bool was_below = MASS ? run_mass < goal : run_cnt < k;
                 const bool reaches = MASS ? run_mass + m >= goal : run_cnt + c >= k;
                 if (was_below && reaches) { sh.bin = b; sh.before_cnt = run_cnt; sh.before_mass = run_mass; }
@@ -923,13 +926,14 @@ __device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned 
         const int bin = sh.bin;
         before_cnt = sh.before_cnt;
         before_mass = sh.before_mass;
-        const unsigned in_bin = sh.cnt[bin];
+        // top-k knows how many logits the bin holds; the nucleus keeps no counts and finds out by copying them
+        const bool few = MASS || sh.cnt[bin] <= kSelCap;
         // a cheap test that no logit of the bin fails (its centre, half its width and the roundings of bin_of, with
         // room to spare); the few that pass are then asked for their bin
         const float centre = top - (static_cast<float>(bin) + 0.5f) / scale;
         const float reach = 0.51f / scale + 2e-6f * fmaxf(fabsf(top), fabsf(bottom));
         auto in_the_bin = [&](float v) { return fabsf(v - centre) <= reach && bin_of(v) == bin; };
-        if (in_bin <= kSelCap) {
+        if (few) {
             // 3. copy the bin's logits out and rank them against each other
             for_each_logit(r, groups, [&](float v) {
                 if (in_the_bin(v)) {
@@ -938,24 +942,26 @@ __device__ float select_floor(const Row<VEC>& r, int groups, float kf, unsigned 
                 }
             });
             __syncthreads();
-            const int count = static_cast<int>(min(sh.n_cand, static_cast<unsigned>(kSelCap)));
-            float best = -INFINITY;
-            for (int i = tid; i < count; i += kSelThreads) {
-                const float mine = sh.cand[i];
-                unsigned c = 0;
-                unsigned long long m = 0;
-                for (int j = 0; j < count; ++j)
-                    if (sh.cand[j] >= mine) { ++c; if (MASS) m += sh.cand_mass[j]; }
-                const bool enough = MASS ? before_mass + m >= goal : before_cnt + c >= k;
-                if (enough) best = fmaxf(best, mine);
-            }
-            best = warp_max(best);
-            if (lane == 0) sh.warp_hi[warp] = best;
-            __syncthreads();
-            best = -INFINITY;
+            if (sh.n_cand <= kSelCap) {  // (always so for top-k)
+                const int count = static_cast<int>(min(sh.n_cand, static_cast<unsigned>(kSelCap)));
+                float best = -INFINITY;
+                for (int i = tid; i < count; i += kSelThreads) {
+                    const float mine = sh.cand[i];
+                    unsigned c = 0;
+                    unsigned long long m = 0;
+                    for (int j = 0; j < count; ++j)
+                        if (sh.cand[j] >= mine) { ++c; if (MASS) m += sh.cand_mass[j]; }
+                    const bool enough = MASS ? before_mass + m >= goal : before_cnt + c >= k;
+                    if (enough) best = fmaxf(best, mine);
+                }
+                best = warp_max(best);
+                if (lane == 0) sh.warp_hi[warp] = best;
+                __syncthreads();
+                best = -INFINITY;
 #pragma unroll
-            for (int w = 0; w < kSelWarps; ++w) best = fmaxf(best, sh.warp_hi[w]);
-            return best > -INFINITY ? best : bottom;
+                for (int w = 0; w < kSelWarps; ++w) best = fmaxf(best, sh.warp_hi[w]);
+                return best > -INFINITY ? best : bottom;
+            }
         }
         // the bin is crowded: its own range is searched next
         float new_lo = INFINITY, new_hi = -INFINITY;

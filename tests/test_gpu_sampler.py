@@ -322,6 +322,37 @@ def test_nucleus_floors(rows, vocab, temperature):
     assert differ <= 2
 
 
+@pytest.mark.parametrize("vocab", [32000, 32003])
+@pytest.mark.parametrize("temperature", [1.0, 0.3])
+def test_nucleus_floors_with_ties_and_masked_logits(vocab, temperature):
+    """Rows the binned selection has to work for: logits rounded to halves (thousands of equal values: the bin
+    where the mass is crossed holds more logits than are ranked at once, and its range collapses to one value),
+    a third of the row masked with -inf (not every element is in play), all logits equal, one finite logit."""
+    base, _ = workloads.make_sampler_logits(77 + vocab, 6, 0, vocab, 1.0)
+    base = np.ascontiguousarray(base[:, 0])
+    rng = np.random.default_rng(5)
+    logits = base.copy()
+    logits[0] = np.round(base[0] * 2) / 2
+    logits[1] = np.round(base[1] * 8) / 8
+    logits[2, rng.random(vocab) < 1 / 3] = -np.inf
+    logits[3] = 1.25
+    logits[4] = -np.inf
+    logits[4, vocab // 2] = 0.5
+    logits[5] = np.round(base[5] * 2) / 2
+    logits[5, rng.random(vocab) < 0.5] = -np.inf
+    d = to_dev(logits)
+    for top_p in (0.1, 0.5, 0.9, 0.99):
+        got = binding.spec_truncation_floors(d, temperature, top_k=0, top_p=top_p).cpu().numpy()
+        again = binding.spec_truncation_floors(d, temperature, top_k=0, top_p=top_p).cpu().numpy()
+        assert np.array_equal(got, again)
+        for r in range(logits.shape[0]):
+            want, margin = oracle_sampling.nucleus_floor(logits[r], temperature, 0, top_p)
+            if got[r] != np.float32(want):
+                assert got[r] in logits[r]
+                slack = _nucleus_slack(logits[r].astype(np.float64), temperature, 0, top_p, float(got[r]))
+                assert margin < NUCLEUS_TOL and slack < NUCLEUS_TOL, (vocab, top_p, r, got[r], want, margin, slack)
+
+
 @pytest.mark.parametrize("batch,gamma,vocab,temperature,top_k,top_p", [
     (64, 7, 32000, 1.0, 0, 0.9),
     (64, 7, 32000, 1.0, 40, 0.8),   # both cuts
