@@ -891,6 +891,7 @@ int attention_sub_slices(int queries) {
 // their 2e-2 logit bar, not inside the 1e-4 bar of fp32 models) once a KV head
 // has enough queries to fill a good part of a 16-row block.
 constexpr int kF16MinPairs = 16;  // (sequence, KV head) pairs from which fp16 K,V rows take the f16 kernel
+constexpr int kF16LoneQueryPairs = 64;  // ... and from which it takes passes of fewer than four queries per KV head
 
 bool attention_uses_mma(const Model& m, int batch, int m_rows, int max_keys) {
     const int queries = (m.cfg.n_heads / m.cfg.n_kv_heads) * m_rows;
@@ -901,7 +902,13 @@ bool attention_uses_mma(const Model& m, int batch, int m_rows, int max_keys) {
     // with fp16 K,V rows, i.e. the f16 kernel, from 16 (sequence, KV head) pairs on - measured on the 7B shape, one row,
     // per block, against the warp-per-query kernel: 4 sequences 95 vs 104 us, 8 sequences 101 vs 120, at 1788 cached
     // tokens 105 vs 138; with fp32 rows from 128 pairs on: batch 16 4.16 -> 4.05 ms per pass, batch 8 3.46 -> 3.48)
-    const int min_queries = batch * m.cfg.n_kv_heads >= (m.kv_dtype == SPEC_DTYPE_FP16 ? kF16MinPairs : 128) ? 4 : 5;
+    const int groups = batch * m.cfg.n_kv_heads;
+    int min_queries = groups >= (m.kv_dtype == SPEC_DTYPE_FP16 ? kF16MinPairs : 128) ? 4 : 5;
+    // from 64 pairs on the f16 kernel also takes a lone query (a draft model's step in a batch): its tiles come through
+    // a cp.async ring, where the warp-per-query kernel's CTAs, by then several tiles per warp, wait on each in turn
+    // (160M-shaped draft, one row, per block: 6 sequences 36.7 vs 41.5 us, 16 sequences 42.8 vs 58.5, 32 sequences 54.3 vs
+    // 80.2; 4 sequences 34.7 vs 35.3: no difference below)
+    if (m.kv_dtype == SPEC_DTYPE_FP16 && groups >= kF16LoneQueryPairs) min_queries = 1;
     return m.bf16() && queries >= min_queries && pairs >= 65536;
 }
 

@@ -15,10 +15,10 @@ pytestmark = pytest.mark.gpu
 BF16_ABS = 2e-2
 
 
-def _model(d_head):
+def _model(d_head, n_kv_heads=2):
     base = workloads.model_config("llama_test_target")
     return workloads.scaled_config(base, n_layers=1, d_head=d_head, d_model=4 * d_head,  # 4 query heads, 2 KV heads
-                                   max_positions=1024)
+                                   n_kv_heads=n_kv_heads, max_positions=1024)
 
 
 def _run(cfg, w, batch, rows, max_len, context, expect, check=(0, 1, -1)):
@@ -79,3 +79,13 @@ def test_a_single_key_slice_is_written_directly():
     cfg = _model(128)
     w = workloads.make_weights(cfg, 24)
     _run(cfg, w, 160, 4, 128, 100, dict(slices=1), check=(0, 77, 159))
+
+
+@pytest.mark.parametrize("n_kv_heads,d_head", [(4, 64), (2, 64), (4, 128)])
+def test_one_row_passes_of_a_batch(n_kv_heads, d_head):
+    """A draft model's step in a batch: one row per sequence, so one query per KV head (4 KV heads for 4 query
+    heads) or two (2 KV heads); 40 sequences give 160 or 80 (sequence, KV head) pairs, enough for the f16 kernel
+    to take them; 700 .. 1000 cached tokens so that the pass has work for it."""
+    cfg = _model(d_head, n_kv_heads)
+    w = workloads.make_weights(cfg, 25)
+    _run(cfg, w, 40, 1, 1024, 1000, {}, check=(0, 19, 39))
