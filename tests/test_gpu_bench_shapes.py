@@ -145,3 +145,31 @@ def test_cross_attention_over_a_long_source_on_the_tensor_cores():
         assert worst <= BF16_ABS, f"max absolute logit error {worst:.3g}"
     finally:
         eng.close()
+
+
+def test_one_row_steps_of_a_batch_over_a_long_source_on_the_tensor_cores():
+    """A draft step of an encoder-decoder in a batch: one decoder row for each of 32 sequences (one query per head,
+    128 (sequence, head) pairs), sources of up to 512 tokens; both the cross-attention and the biased self-attention
+    take the f16 tensor-core kernel.  Five steps, four of the sequences against the oracle."""
+    cfg = workloads.model_config("t5_test_target")
+    w = workloads.make_weights(cfg, 1)
+    B, steps = 32, 5
+    eng = binding.Engine(cfg, w, max_batch=B, max_len=512, page_size=64, max_gamma=1, max_src_len=512)
+    try:
+        assert eng.attention_plan(0, B, 1, cross=True)["f16"]
+        assert eng.attention_plan(0, B, 1)["f16"]
+        lengths = [512 - 16 * b for b in range(B)]
+        sources = [workloads.make_prompt(500 + b, n, cfg["vocab"]) for b, n in enumerate(lengths)]
+        eng.encode(sources)
+        tokens = np.stack([np.concatenate([[START_TOKEN], workloads.make_prompt(600 + b, steps - 1, cfg["vocab"])])
+                           for b in range(B)])
+        got = np.stack([eng.forward_logits(0, tokens[:, t:t + 1]).cpu().numpy()[:, 0] for t in range(steps)], axis=1)
+        assert binding.spec_device_error() == 0
+        worst = 0.0
+        for b in (0, 11, 22, 31):
+            o = EncoderDecoder(cfg, w)
+            o.encode(sources[b])
+            worst = max(worst, np.abs(got[b] - o.forward_rows(tokens[b])).max())
+        assert worst <= BF16_ABS, f"max absolute logit error {worst:.3g}"
+    finally:
+        eng.close()
