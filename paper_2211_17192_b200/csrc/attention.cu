@@ -473,8 +473,9 @@ attention_mma_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 // ---- fp16 K,V rows on the f16 tensor-core path --------------------------------
 //
 // With 16-bit rows the cache needs no conversion: 64-key tiles of K and of V go
-// from the pool to shared memory as they are (cp.async, a ring of two or three stages:
-// the next tiles load while tile i is multiplied) and feed mma.sync.m16n8k16 (f16 operands,
+// from the pool to shared memory as they are (tiled TMA copies that one thread asks
+// for, completion counted on an mbarrier per stage; a ring of two or three stages: the
+// next tiles load while tile i is multiplied) and feed mma.sync.m16n8k16 (f16 operands,
 // fp32 accumulate) through ldmatrix.  A CTA owns (key slice, KV head, sequence)
 // and ALL the queries of that KV head - up to 64, as MB blocks of 16 - so K and
 // V of the slice are fetched once, whatever the number of rows.  Its four warps
@@ -487,14 +488,15 @@ constexpr int kF16Warps = 4;
 constexpr int kF16TileKeys = 64;
 constexpr int kF16MaxQueries = 64;  // per CTA (MB = 4)
 
-// Rows are stored without padding; inside a row the 16-byte chunks are permuted, chunk c of row r at position
+// A staged K or V tile is DH / 64 column blocks of [64 keys][64 halves], as the copies' 128-byte swizzle leaves them:
+// rows of 128 bytes without padding, the 16-byte chunks of a row permuted, chunk c of row r at position
 // c ^ (r & 7), so that the eight rows an ldmatrix reads hit eight different bank groups.  Three stages (tiles
 // i + 1 and i + 2 on their way while tile i is multiplied) for up to 32 queries, two for 64: two CTAs per SM
 // either way, and 128 KB of K,V in flight per SM instead of 64 - the kernel is bound by the latency of the tiles.
 template <int DH, int MB>
 struct F16Smem {
     static constexpr int kStages = MB <= 2 ? 3 : 2;
-    static constexpr int kRow = DH;                      // halves per staged row
+    static constexpr int kRow = DH;                      // halves per staged query row (K and V rows: 64 per column block)
     static constexpr int kQ = 16 * MB * kRow;            // the queries (halves)
     static constexpr int kTile = kF16TileKeys * kRow;    // one K or V tile (halves)
     static constexpr int kStage = 2 * kTile;             // K, then V
@@ -535,14 +537,36 @@ __device__ __forceinline__ float exp2_approx(float x) {
     return y;
 }
 
-// grid = (slices, n_kv_heads * q_blocks, batch), block = 128; q_blocks = ceil(queries / 64).
+__device__ int g_attn_error;  // set when the bounded wait for a tile of the f16 kernel ran out (0 = none)
+
+// Waits, with a limit, for the phase of the given parity; false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = static_cast<uint32_t>(__cvta_generic_to_shared(bar));
+    for (uint32_t spin = 0; spin < (1u << 22); ++spin) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t"
+            "}"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// grid = (slices, n_kv_heads * q_blocks, batch), block = 128; q_blocks = ceil(queries / 64).  kv_map: the layer's pool
+// as a matrix of rows of DH halves (cached_f16_rows_map).
 // Scores are kept in base-2 units (q is scaled by log2(e) / sqrt(d_head), the bias by log2(e)), so every
 // exponential is one ex2.approx; the running maximum goes back to natural units when the state is stored.
 template <int DH, int MB, bool FUSED>
 __global__ void __launch_bounds__(32 * kF16Warps)
 attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t* __restrict__ pos,
                      const int32_t* __restrict__ seq, int m_rows, int n_heads, int n_kv_heads, int q_blocks,
-                     const __half* __restrict__ kv_layer, const int32_t* __restrict__ page_table, int pages_per_seq,
+                     const __grid_constant__ CUtensorMap kv_map, const int32_t* __restrict__ page_table, int pages_per_seq,
                      int page_size, const int32_t* __restrict__ kv_len, const float* __restrict__ bias, int bias_span,
                      int bias_zero, float scale, float* __restrict__ part, const AttnOut out) {
     using S = F16Smem<DH, MB>;
@@ -551,16 +575,22 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     constexpr int NB = KW / 8;                // 8-key blocks of those
     constexpr int CH = DH / 8;                // 16-byte chunks of a row
     constexpr int QN = 16 * MB;               // queries of this CTA
-    constexpr int kRowsPerSweep = 32 * kF16Warps / CH;        // rows that the CTA's threads copy at once (one chunk each)
-    constexpr int kSweeps = kF16TileKeys / kRowsPerSweep;     // sweeps per K (or V) tile
     constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    extern __shared__ __align__(1024) unsigned char smem_raw[];  // (the swizzled boxes want 1024-byte alignment)
     __shared__ int q_pos[QN], q_row[QN], q_head[QN];
+    __shared__ __align__(8) uint64_t landed[S::kStages];  // a stage's tile has arrived (counted in bytes)
     __half* Qs = reinterpret_cast<__half*>(smem_raw);
     __half* stages = Qs + S::kQ;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+#pragma unroll
+        for (int st = 0; st < S::kStages; ++st)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(&landed[st]))));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
     pdl_trigger();
     pdl_wait();
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int mb = warp % MB, kw0 = (warp / MB) * KW;
     const int slice = blockIdx.x, slices = gridDim.x, b = blockIdx.z;
@@ -586,50 +616,46 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     const int t0 = static_cast<int>(static_cast<long long>(tiles) * slice / slices);
     const int t1 = static_cast<int>(static_cast<long long>(tiles) * (slice + 1) / slices);
     const int my_tiles = t1 - t0;
-    const size_t head_stride = static_cast<size_t>(page_size) * DH;
-    const size_t page_stride = 2 * static_cast<size_t>(n_kv_heads) * head_stride;
-    const size_t v_offset = static_cast<size_t>(n_kv_heads) * head_stride;
     const int32_t* pages = page_table + seq[b * m_rows] * pages_per_seq;
     const int page_shift = __ffs(page_size) - 1;  // (pages hold a power of two of tokens)
-    const __half* head_base = kv_layer + kv_head * head_stride;
 
-    // Tile i of the slice into stage i % 2.  A thread copies one 16-byte chunk per sweep: chunk tid % CH of
-    // row tid / CH + kRowsPerSweep * sweep, of K and of V.  A 32-key half of the tile lies inside one page;
-    // keys at or beyond seq_keys become zeros.
-    const int copy_row = tid / CH, copy_off = copy_row * DH + 8 * (tid % CH);
-    const uint32_t copy_dst = static_cast<uint32_t>(__cvta_generic_to_shared(stages)) +
-                              static_cast<uint32_t>(f16_at<DH>(copy_row, 8 * (tid % CH)) * sizeof(__half));
-    // (the page entries of a tile are fetched one tile ahead of the copies that need them, so that no
-    // copy waits for a page-table load)
+    // Tile i of the slice into stage i % kStages: thread 0 asks for it as tiled copies of 32 rows x 64 halves (a
+    // 32-key half of the tile lies inside one page; the pool is one matrix of rows of DH halves, the rows of page p
+    // being ((2 p + [V]) n_kv_heads + head) page_size + token), which arrive with the 16-byte chunks of every
+    // 128-byte row permuted - chunk c of row r at c ^ (r & 7) - so that ldmatrix sees no bank conflict.  A stage
+    // holds K then V, each as DH / 64 column blocks of [64 keys][64 halves].  Keys at or beyond seq_keys are
+    // whatever the pool holds there (zeros or an earlier sequence's rows): they are masked, and finite.
+    // (the page entries of a tile are fetched one tile ahead of the copies that need them)
     auto fetch_pages = [&](int i, int (&pg)[2]) {
-        if (i < my_tiles) {
+        if (tid == 0 && i < my_tiles) {
             const int k0 = kF16TileKeys * (t0 + i);
 #pragma unroll
             for (int h = 0; h < 2; ++h) pg[h] = pages[min(k0 + 32 * h, seq_keys - 1) >> page_shift];
         }
     };
     auto issue = [&](int i, const int (&pg)[2]) {
-        if (i < my_tiles) {
+        if (tid == 0 && i < my_tiles) {
             const int k0 = kF16TileKeys * (t0 + i);
-            const uint32_t dst = copy_dst + static_cast<uint32_t>((i % S::kStages) * S::kStage * sizeof(__half));
-            const __half* half_base[2];
+            const int st = i % S::kStages;
+            const uint32_t bar = static_cast<uint32_t>(__cvta_generic_to_shared(&landed[st]));
+            const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(stages + st * S::kStage));
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the stage was read with ldmatrix before
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(static_cast<uint32_t>(S::kStage * sizeof(__half)))
+                         : "memory");
 #pragma unroll
-            for (int h = 0; h < 2; ++h)
-                half_base[h] = head_base + pg[h] * page_stride + static_cast<size_t>((k0 + 32 * h) & (page_size - 1)) * DH + copy_off;
-            const int n_valid = seq_keys - k0 - copy_row;  // row r of this thread is valid iff r_in_tile - copy_row < n_valid
+            for (int v = 0; v < 2; ++v)
 #pragma unroll
-            for (int sw = 0; sw < kSweeps; ++sw) {
-                constexpr int kSweepsPerHalf = 32 / kRowsPerSweep;
-                const bool valid = sw * kRowsPerSweep < n_valid;
-                const __half* src = half_base[sw / kSweepsPerHalf] + (valid ? (sw % kSweepsPerHalf) * kRowsPerSweep * DH : -copy_row * DH);
-                const uint32_t d = dst + static_cast<uint32_t>(sw * kRowsPerSweep * S::kRow * sizeof(__half));
-                const int bytes = valid ? 16 : 0;
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d + static_cast<uint32_t>(S::kTile * sizeof(__half))),
-                             "l"(src + v_offset), "r"(bytes) : "memory");
-            }
+                for (int h = 0; h < 2; ++h) {
+                    const int row = ((2 * pg[h] + v) * n_kv_heads + kv_head) * page_size + ((k0 + 32 * h) & (page_size - 1));
+#pragma unroll
+                    for (int c = 0; c < DH / 64; ++c) {
+                        const uint32_t d = dst + static_cast<uint32_t>((v * S::kTile + c * kF16TileKeys * 64 + h * 32 * 64) * sizeof(__half));
+                        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                                     ::"r"(d), "l"(&kv_map), "r"(c * 64), "r"(row), "r"(bar)
+                                     : "memory");
+                    }
+                }
         }
-        cp_async_commit();
     };
     int pg_next[2] = {0, 0};
 #pragma unroll
@@ -663,8 +689,8 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     // lane-dependent parts of the ldmatrix addresses, formed once (the chunk permutation XORs with lane & 7):
     // K: row (nb*8 + l7), chunk kp*4 + (lane >> 3); V: row (kk*16 + l7 + 8*((lane >> 3) & 1)), chunk n2*2 + (lane >> 4)
     const int l7 = lane & 7;
-    const int k_lane = l7 * DH + ((((lane >> 3) ^ l7) & 7) << 3);            // even kp; odd kp flips chunk bit 2
-    const int v_row = (l7 + 8 * ((lane >> 3) & 1)) * DH;
+    const int k_lane = l7 * 64 + ((((lane >> 3) ^ l7) & 7) << 3);            // even kp; odd kp flips chunk bit 2
+    const int v_row = (l7 + 8 * ((lane >> 3) & 1)) * 64;
     int v_chunk[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) v_chunk[j] = ((((j << 1) | (lane >> 4)) ^ l7) & 7) << 3;
@@ -673,8 +699,10 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
     const int any_sees = min(__reduce_max_sync(kFullMask, max(p_lo < 0 ? 0 : keys_lo, p_hi < 0 ? 0 : keys_hi)), seq_keys);
 
     for (int i = 0; i < my_tiles; ++i) {
-        cp_async_wait<S::kStages - 2>();  // tile i has landed (the later ones may still be on their way)
-        __syncthreads();                  // ... for every thread; everybody is done with tile i - 1, whose stage
+        // tile i has landed (a wait that runs out is recorded and the pass goes on with what the stage holds: no
+        // thread leaves the loop alone, and the host sees the error)
+        if (!mbar_wait_bounded(&landed[i % S::kStages], (i / S::kStages) & 1)) atomicCAS(&g_attn_error, 0, 1);
+        __syncthreads();                     // everybody is done with tile i - 1, whose stage
         issue(i + S::kStages - 1, pg_next);  // takes the tile that is kStages - 1 ahead
         fetch_pages(i + S::kStages, pg_next);
         if (i == 0) {  // (the first barrier also covered the staged queries)
@@ -684,7 +712,7 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
         }
         const int k0 = kF16TileKeys * (t0 + i) + kw0;  // this warp's first key of the tile
         if (k0 >= any_sees) continue;  // nothing here that a live row of this warp may see
-        const __half* Kt = stages + (i % S::kStages) * S::kStage + kw0 * S::kRow;  // (kw0 is a multiple of 16: the permutation is unchanged)
+        const __half* Kt = stages + (i % S::kStages) * S::kStage + kw0 * 64;  // (kw0 is a multiple of 16: the permutation is unchanged)
         const __half* Vt = Kt + S::kTile;
         // S = Q K^T
         float s[NB][4];
@@ -697,7 +725,7 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 #pragma unroll
             for (int nb = 0; nb < NB; ++nb) {
                 uint32_t kf[4];
-                ldsm_x4(kf, Kt + nb * 8 * DH + (kp >> 1) * 64 + ((kp & 1) ? (k_lane ^ 32) : k_lane));
+                ldsm_x4(kf, Kt + nb * 8 * 64 + (kp >> 1) * (kF16TileKeys * 64) + ((kp & 1) ? (k_lane ^ 32) : k_lane));
                 mma_f16(s[nb], qf[2 * kp], kf[0], kf[1]);
                 mma_f16(s[nb], qf[2 * kp + 1], kf[2], kf[3]);
             }
@@ -770,13 +798,13 @@ attention_f16_kernel(const float* __restrict__ qkv, int q_stride, const int32_t*
 #pragma unroll
             for (int kk = 0; kk < NB / 2; ++kk) {
                 uint32_t vf[4];
-                ldsm_x4_trans(vf, Vt + kk * 16 * DH + v_row + (n2 >> 2) * 64 + v_chunk[n2 & 3]);
+                ldsm_x4_trans(vf, Vt + kk * 16 * 64 + v_row + (n2 >> 2) * (kF16TileKeys * 64) + v_chunk[n2 & 3]);
                 mma_f16(o[2 * n2], pa[kk], vf[0], vf[1]);
                 mma_f16(o[2 * n2 + 1], pa[kk], vf[2], vf[3]);
             }
         }
     }
-    cp_async_wait<0>();
+    // (every tile that was asked for has been waited for: nothing is in flight)
 
     // park this warp's state in stage 0: [warp][query of the block][max (base-2 units), sum, O[DH]]
     __syncthreads();
@@ -905,7 +933,7 @@ bool attention_uses_mma(const Model& m, int batch, int m_rows, int max_keys) {
     const int groups = batch * m.cfg.n_kv_heads;
     int min_queries = groups >= (m.kv_dtype == SPEC_DTYPE_FP16 ? kF16MinPairs : 128) ? 4 : 5;
     // from 64 pairs on the f16 kernel also takes a lone query (a draft model's step in a batch): its tiles come through
-    // a cp.async ring, where the warp-per-query kernel's CTAs, by then several tiles per warp, wait on each in turn
+    // a ring of asynchronous copies, where the warp-per-query kernel's CTAs, by then several tiles per warp, wait on each in turn
     // (160M-shaped draft, one row, per block: 6 sequences 36.7 vs 41.5 us, 16 sequences 42.8 vs 58.5, 32 sequences 54.3 vs
     // 80.2; 4 sequences 34.7 vs 35.3: no difference below)
     if (m.kv_dtype == SPEC_DTYPE_FP16 && groups >= kF16LoneQueryPairs) min_queries = 1;
@@ -998,6 +1026,13 @@ AttentionPlan attention_plan(const Model& m, int batch, int m_rows, int max_keys
     return plan;
 }
 
+int attention_take_error() {
+    int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_attn_error, sizeof(int)) != cudaSuccess) return -1;
+    if (v) cudaMemcpyToSymbol(g_attn_error, &zero, sizeof(int));
+    return v;
+}
+
 namespace {
 
 // A launch with programmatic stream serialization and, if cluster_x > 0, clusters of
@@ -1046,6 +1081,10 @@ int launch_attention_variant(const Model& m, const AttnSource& src, const RowMet
             const int q_blocks = (queries + kF16MaxQueries - 1) / kF16MaxQueries;
             const int per_cta = std::min(queries, kF16MaxQueries);
             const dim3 grid(slices, m.cfg.n_kv_heads * q_blocks, batch);
+            CUtensorMap kv_map;  // the layer's pool as rows of d_head halves
+            status = cached_f16_rows_map(src.pool.kv, static_cast<unsigned long long>(src.pool.n_pages) * 2 * m.cfg.n_kv_heads *
+                                                          src.pool.page_size, DH, &kv_map);
+            if (status != SPEC_OK) return status;
 #define SPEC_LAUNCH_F16(MB, F, CLUSTER)                                                                                 \
     do {                                                                                                                \
         static std::atomic<unsigned long long> configured{0};                                                           \
@@ -1055,7 +1094,7 @@ int launch_attention_variant(const Model& m, const AttnSource& src, const RowMet
                                                static_cast<int>(F16Smem<DH, MB>::kBytes)));                             \
         status = launch_attn(attention_f16_kernel<DH, MB, F>, grid, dim3(32 * kF16Warps), F16Smem<DH, MB>::kBytes,      \
                              CLUSTER, stream, src.q, src.q_stride, rows.pos, rows.seq, m_rows, m.cfg.n_heads,           \
-                             m.cfg.n_kv_heads, q_blocks, pool, src.pool.page_table, src.pool.pages_per_seq,             \
+                             m.cfg.n_kv_heads, q_blocks, kv_map, src.pool.page_table, src.pool.pages_per_seq,           \
                              src.pool.page_size, src.kv_len, src.bias, src.bias_span, src.bias_zero, scale, part, out); \
     } while (0)
             if (per_cta <= 16) { if (fused) SPEC_LAUNCH_F16(1, true, slices); else SPEC_LAUNCH_F16(1, false, 0); }

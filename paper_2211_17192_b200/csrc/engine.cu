@@ -203,17 +203,18 @@ struct Pass {
 
 // Non-zero (and cleared) if a tensor-core GEMM or the persistent pass kernel gave up on a bounded wait.
 int device_gave_up(spec_ctx* ctx) {
-    const int gemm = gemm_tc_take_error(), pass = pass_take_error();
-    return gemm ? gemm : pass;
+    const int gemm = gemm_tc_take_error(), pass = pass_take_error(), attn = attention_take_error();
+    return gemm ? gemm : pass ? pass : attn;
 }
 
 KvPool layer_pool(const spec_ctx* ctx, const Model& m, int layer) {
     return KvPool{static_cast<char*>(m.kv) + static_cast<size_t>(layer) * m.layer_stride, m.kv_elem_bytes, m.kv_dtype, ctx->page_table,
-                  ctx->pages_per_seq, ctx->rt.page_size};
+                  ctx->pages_per_seq, ctx->rt.page_size, ctx->rt.max_batch * ctx->pages_per_seq};
 }
 
 KvPool source_pool(const spec_ctx* ctx, const Model& m, void* base) {
-    return KvPool{base, m.kv_elem_bytes, m.kv_dtype, ctx->src_page_table, ctx->src_pages_per_seq, ctx->rt.page_size};
+    return KvPool{base, m.kv_elem_bytes, m.kv_dtype, ctx->src_page_table, ctx->src_pages_per_seq, ctx->rt.page_size,
+                  ctx->rt.max_batch * ctx->src_pages_per_seq};
 }
 
 // One forward pass of `m` over batch * m_rows rows (rows of sequence b are rows
@@ -602,6 +603,9 @@ int init_model(spec_ctx* ctx, int which, const spec_model_cfg& cfg, const spec_w
     m.layer_stride = n_pages * 2 * cfg.n_kv_heads * ctx->rt.page_size * cfg.d_head * m.kv_elem_bytes;
     char* kv = nullptr;
     SPEC_TRY(dev_alloc(ctx, &kv, m.layer_stride * cfg.n_layers));
+    // (rows that no sequence has written yet are read, and masked, by the attention kernels that fetch whole tiles:
+    // they must hold numbers, not whatever the allocation held)
+    SPEC_CUDA_TRY(cudaMemset(kv, 0, m.layer_stride * cfg.n_layers));
     m.kv = kv;
     if (cfg.arch == SPEC_ARCH_LLAMA) {
         std::vector<float2> table;
@@ -618,6 +622,8 @@ int init_model(spec_ctx* ctx, int which, const spec_model_cfg& cfg, const spec_w
         char *enc_kv = nullptr, *cross = nullptr;
         SPEC_TRY(dev_alloc(ctx, &enc_kv, m.cross_stride));
         SPEC_TRY(dev_alloc(ctx, &cross, m.cross_stride * cfg.n_layers));
+        SPEC_CUDA_TRY(cudaMemset(enc_kv, 0, m.cross_stride));
+        SPEC_CUDA_TRY(cudaMemset(cross, 0, m.cross_stride * cfg.n_layers));
         m.enc_kv = enc_kv;
         m.cross_kv = cross;
         // bias tables by relative position, from the bucket tables

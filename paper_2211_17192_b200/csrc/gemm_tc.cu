@@ -448,6 +448,30 @@ int gemm_tc_token_tile(int n_rows) {
     return 128;
 }
 
+int cached_f16_rows_map(const void* base, unsigned long long rows, int cols, CUtensorMap* out) {
+    static std::mutex mu;
+    static std::map<std::tuple<const void*, unsigned long long, int>, CUtensorMap> cache;
+    std::lock_guard<std::mutex> lock(mu);
+    const auto key = std::make_tuple(base, rows, cols);
+    auto it = cache.find(key);
+    if (it == cache.end()) {
+        EncodeFn fn = encode_fn();
+        if (!fn) return fail(SPEC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+        const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+        const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * 2};
+        const cuuint32_t box[2] = {64, 32};
+        const cuuint32_t elem[2] = {1, 1};
+        CUtensorMap m;
+        const CUresult res = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (res != CUDA_SUCCESS) return fail(SPEC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", static_cast<int>(res));
+        it = cache.emplace(key, m).first;
+    }
+    *out = it->second;
+    return SPEC_OK;
+}
+
 // Split-K factor: the smallest one that fills the last wave of CTAs to 85 %, with
 // at least two k-blocks per split.
 int gemm_tc_splits(int n_out, int k, int n_rows) {
@@ -648,6 +672,6 @@ extern "C" int spec_timeout_drill(void* stream) {
 }
 
 extern "C" int spec_device_error(void) {
-    const int gemm = spec::gemm_tc_take_error(), pass = spec::pass_take_error();
-    return gemm ? gemm : pass;
+    const int gemm = spec::gemm_tc_take_error(), pass = spec::pass_take_error(), attn = spec::attention_take_error();
+    return gemm ? gemm : pass ? pass : attn;
 }

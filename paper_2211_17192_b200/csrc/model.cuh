@@ -1,6 +1,7 @@
 // Internal structures of the decoder engine and the launchers of its kernels.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include <vector>
@@ -108,6 +109,7 @@ struct KvPool {
     const int32_t* page_table;
     int pages_per_seq;
     int page_size;
+    int n_pages;  // pages in the pool (of one layer)
 };
 
 // Finishes a projection GEMM whose output row is [n_heads q heads | n_kv_heads k
@@ -178,6 +180,12 @@ int launch_pass(const PassScratch& s, const Model& m, int which, const RowMeta& 
                 unsigned long long* trace = nullptr, int trace_capacity = 0);
 void pass_scratch_release(PassScratch& s);
 int pass_take_error();
+
+// A tensor map over `rows` rows of `cols` (64 or 128) fp16 elements starting at `base`, fetched in boxes of 64 elements
+// by 32 rows with the 128-byte swizzle; maps are cached by (base, rows, cols).  gemm_tc.cu
+int cached_f16_rows_map(const void* base, unsigned long long rows, int cols, CUtensorMap* out);
+// Non-zero (and cleared) if the f16 attention kernel gave up on a bounded wait for a tile.  attention.cu
+int attention_take_error();
 
 // sampling.cu
 int launch_verify_sample(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
