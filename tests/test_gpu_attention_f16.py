@@ -21,10 +21,10 @@ def _model(d_head, n_kv_heads=2):
                                    n_kv_heads=n_kv_heads, max_positions=1024)
 
 
-def _run(cfg, w, batch, rows, max_len, context, expect, check=(0, 1, -1)):
+def _run(cfg, w, batch, rows, max_len, context, expect, check=(0, 1, -1), page_size=32):
     """`batch` sequences with ragged cached lengths (context - 5 b, wrapped into [context // 2, context]),
     then one pass of `rows` new rows each."""
-    eng = binding.Engine(cfg, w, max_batch=batch, max_len=max_len, page_size=32, max_gamma=max(rows - 1, 1))
+    eng = binding.Engine(cfg, w, max_batch=batch, max_len=max_len, page_size=page_size, max_gamma=max(rows - 1, 1))
     try:
         plan = eng.attention_plan(0, batch, rows)
         assert plan["f16"], plan
@@ -89,3 +89,13 @@ def test_one_row_passes_of_a_batch(n_kv_heads, d_head):
     cfg = _model(d_head, n_kv_heads)
     w = workloads.make_weights(cfg, 25)
     _run(cfg, w, 40, 1, 1024, 1000, {}, check=(0, 19, 39))
+
+
+@pytest.mark.parametrize("page_size", [64, 128, 256])
+def test_larger_pages(page_size):
+    """The tiles are fetched as 32-key boxes inside a page: pages of 64, 128 and 256 tokens (a tile then lies in one
+    page, or two tiles, or four), 16 sequences x 5 rows on 128-wide heads, ragged lengths."""
+    cfg = _model(128)
+    w = workloads.make_weights(cfg, 26)
+    _run(cfg, w, 16, 5, 512, 420, {}, page_size=page_size)
+
