@@ -342,15 +342,22 @@ def test_nucleus_floors_with_ties_and_masked_logits(vocab, temperature):
     logits[5, rng.random(vocab) < 0.5] = -np.inf
     d = to_dev(logits)
     for top_p in (0.1, 0.5, 0.9, 0.99):
-        got = binding.spec_truncation_floors(d, temperature, top_k=0, top_p=top_p).cpu().numpy()
-        again = binding.spec_truncation_floors(d, temperature, top_k=0, top_p=top_p).cpu().numpy()
-        assert np.array_equal(got, again)
+        for top_k in (0, 50, 300):  # alone; after a top-k found through the threads' maxima; after a binned top-k
+            got = binding.spec_truncation_floors(d, temperature, top_k=top_k, top_p=top_p).cpu().numpy()
+            again = binding.spec_truncation_floors(d, temperature, top_k=top_k, top_p=top_p).cpu().numpy()
+            assert np.array_equal(got, again)
+            for r in range(logits.shape[0]):
+                want, margin = oracle_sampling.nucleus_floor(logits[r], temperature, top_k, top_p)
+                if got[r] != np.float32(want):
+                    assert got[r] in logits[r]
+                    slack = _nucleus_slack(logits[r].astype(np.float64), temperature, top_k, top_p, float(got[r]))
+                    assert margin < NUCLEUS_TOL and slack < NUCLEUS_TOL, (vocab, top_p, top_k, r, got[r], want, margin, slack)
+    for top_k in (1, 50, 128, 129, 300):  # top-k alone on the same rows: the k-th largest by a sort, or -inf when
+        got = binding.spec_truncation_floors(d, temperature, top_k=top_k, top_p=1.0).cpu().numpy()  # fewer logits are finite
         for r in range(logits.shape[0]):
-            want, margin = oracle_sampling.nucleus_floor(logits[r], temperature, 0, top_p)
-            if got[r] != np.float32(want):
-                assert got[r] in logits[r]
-                slack = _nucleus_slack(logits[r].astype(np.float64), temperature, 0, top_p, float(got[r]))
-                assert margin < NUCLEUS_TOL and slack < NUCLEUS_TOL, (vocab, top_p, r, got[r], want, margin, slack)
+            finite = np.sort(logits[r][np.isfinite(logits[r])])[::-1]
+            want = finite[top_k - 1] if top_k <= finite.size else -np.inf
+            assert got[r] == np.float32(want), (vocab, top_k, r, got[r], want)
 
 
 @pytest.mark.parametrize("batch,gamma,vocab,temperature,top_k,top_p", [
